@@ -1,0 +1,218 @@
+/*
+ * distsim.h -- C ABI of the batched strategy-timeline engine (CUDA, sm_100a).
+ *
+ * The engine evaluates DistSim's event-based activity timeline (paper Sec. 3.2
+ * and 4.3) for very many candidate hybrid-parallel training strategies at once.
+ * A candidate is x = (mp, pp, dp = N/(mp*pp), stage bounds 0=c_0<..<c_pp=L,
+ * micro-batch count m, pipeline schedule); the model enters as an event table:
+ * per event class (mp, micro-batch size b) the elapsed time of every layer's
+ * forward and backward computation event, and alpha-beta constants for the
+ * communication events.
+ *
+ * Conventions
+ *   - Every function returns DISTSIM_OK (0) or a negative DISTSIM_E_* code; it
+ *     never throws, aborts or prints.  distsim_last_error() gives the text of
+ *     the most recent failure on that context.
+ *   - "h_" pointers are HOST memory, "d_" pointers are DEVICE memory on the
+ *     context's device.  Host inputs are copied before the call returns.
+ *     Device buffers are allocated and owned by the caller; the library owns
+ *     only its copies of the tables and its scratch.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls enqueue work on it and return without synchronising,
+ *     except where a result is returned to host memory (stated per function).
+ *   - All times are int64 nanoseconds.  A context is not thread-safe: use one
+ *     per host thread.
+ *   - There is no CPU fallback: without a CUDA device distsim_create fails.
+ */
+#ifndef DISTSIM_H
+#define DISTSIM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DISTSIM_MAX_PP      64     /* pipeline stages                              */
+#define DISTSIM_MAX_LAYERS  256
+#define DISTSIM_MAX_M       4096   /* micro-batches per candidate                  */
+
+enum {
+    DISTSIM_OK = 0,
+    DISTSIM_E_ARG = -1,        /* null pointer, malformed table or space            */
+    DISTSIM_E_STATE = -2,      /* table or space not loaded yet                     */
+    DISTSIM_E_RANGE = -3,      /* candidate index outside [0, n_candidates)         */
+    DISTSIM_E_CAPACITY = -4,   /* caller's output buffer too small                  */
+    DISTSIM_E_OVERFLOW = -5,   /* a time or count bound does not fit 62 bits        */
+    DISTSIM_E_CUDA = -6,       /* a CUDA runtime call failed                        */
+    DISTSIM_E_TIMEOUT = -7,    /* a bounded device-side wait gave up                */
+    DISTSIM_E_UNSUPPORTED = -8 /* e.g. degrees that are not powers of two           */
+};
+
+/* Event kinds in distsim_record.kind. */
+enum {
+    DISTSIM_COMPUTE_F = 0, DISTSIM_COMPUTE_B = 1,   /* layer computation event       */
+    DISTSIM_MP_AR_F = 2,   DISTSIM_MP_AR_B = 3,     /* model-parallel all-reduce     */
+    DISTSIM_A2A_F = 4,     DISTSIM_A2A_B = 5,       /* expert-layer all-to-all       */
+    DISTSIM_SEND_F = 6,    DISTSIM_SEND_B = 7,      /* transfer to the neighbour     */
+    DISTSIM_DP_AR = 8                               /* gradient all-reduce bucket    */
+};
+
+typedef struct distsim_ctx distsim_ctx;
+
+/* Creates a context on the given CUDA device.  Fails with DISTSIM_E_CUDA when
+ * there is no such device or it is not compute capability 10.x. */
+int distsim_create(distsim_ctx **out, int cuda_device);
+void distsim_destroy(distsim_ctx *ctx);
+/* Text of the last error on this context ("" if none); valid until the next call. */
+const char *distsim_last_error(const distsim_ctx *ctx);
+
+/*
+ * The event table (paper Sec. 3.2 "event", Sec. 4.1-4.2; the layer-to-events
+ * mapping MAP(L->E) that Algorithm 1 takes as input).  All pointers are host
+ * memory, read during the call only.
+ *   fwd_ns/bwd_ns [n_classes][n_layers]  elapsed time of the layer's computation
+ *                                        event for class k = (class_mp[k], class_b[k])
+ *   layer_is_expert [n_layers]           1: the layer also has an all-to-all event
+ *   grad_bytes [n_layers]                gradient bytes of the layer at mp = 1
+ *   alpha_*_ns, beta_* (bytes per ns)    link latency / bandwidth inside a node
+ *                                        and between nodes (the intra/inter-node
+ *                                        attribute of communication events, Sec. 4.1)
+ *   dp_bucket_bytes                      gradient all-reduce bucket size; 0 = one
+ *                                        all-reduce event per stage (paper Sec. 4.3,
+ *                                        DP modeling)
+ *   dp_overlap                           0: buckets start after the device's last
+ *                                        event; 1: a bucket starts once the layer
+ *                                        holding its last byte has finished the
+ *                                        last micro-batch's backward
+ * Communication costs: ring all-reduce over n devices of S bytes
+ * 2(n-1)alpha + ceil(2(n-1)S / (n beta)) (per-device volume 2(n-1)S/n, Sec. 4.2);
+ * transfer alpha + ceil(S/beta); all-to-all (n-1)alpha + ceil((n-1)S/(n beta)).
+ * Requirements: n_devices, gpus_per_node powers of two; 1 <= n_layers <=
+ * DISTSIM_MAX_LAYERS; all times, bytes and constants >= 0, betas >= 1.
+ * Returns DISTSIM_E_OVERFLOW if an upper bound on any batch time reaches 2^62.
+ * Loading a table invalidates the current search space.
+ */
+typedef struct {
+    int32_t n_layers, n_classes, n_devices, gpus_per_node;
+    int64_t global_batch, seq, hidden;
+    int64_t alpha_intra_ns, beta_intra, alpha_inter_ns, beta_inter;
+    int64_t dp_bucket_bytes;
+    int32_t dp_overlap;
+    int32_t act_bytes_per_elem;
+    const int32_t *class_mp, *class_b;
+    const int64_t *fwd_ns, *bwd_ns;
+    const uint8_t *layer_is_expert;
+    const int64_t *grad_bytes;
+} distsim_event_table;
+
+int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *h_table);
+
+/*
+ * The search space (paper Sec. 5: grid over parallel degrees with dp =
+ * GPUs/mp/pp, invalid combinations dropped).  Candidates are numbered in this
+ * canonical order, outermost first: mp ascending over powers of two <= mp_max;
+ * pp ascending over powers of two <= min(pp_max, n_layers) with mp*pp | N and
+ * dp | global_batch; m ascending over the valid entries of m_list (m_rule 0: m
+ * divides Bp = global_batch/dp; 1: any m <= Bp, micro-batch size ceil(Bp/m));
+ * stage partition (partition_mode 0: the balanced one, c_j = floor(j L / pp);
+ * 1: every composition, lexicographic in (c_1..c_{pp-1})); schedule GPipe then
+ * 1F1B as enabled in sched_mask (bit 0 GPipe, bit 1 1F1B/Dapple).
+ * Candidates are never materialised: the device decodes them from the index.
+ * Fails with DISTSIM_E_ARG if a needed class (mp, b) is not in the table, with
+ * DISTSIM_E_OVERFLOW if the count does not fit 62 bits.  *n_candidates receives
+ * the size of the space.
+ */
+typedef struct {
+    int32_t mp_max, pp_max, n_m;
+    const int32_t *m_list;          /* host, ascending, 1 <= m <= DISTSIM_MAX_M */
+    int32_t m_rule;
+    int32_t partition_mode;
+    int32_t sched_mask;
+} distsim_space;
+
+int distsim_set_space(distsim_ctx *ctx, const distsim_space *h_space, int64_t *n_candidates);
+
+typedef struct {
+    int32_t mp, pp, dp, m, sched;   /* sched 0: GPipe, 1: 1F1B                     */
+    int32_t micro_batch_size;       /* b = ceil(Bp / m)                            */
+    int32_t class_index;            /* row of the event table                      */
+    int32_t bounds[DISTSIM_MAX_PP + 1];
+} distsim_candidate;
+
+/* Host-side decode of one index, for reporting (the device decodes on its own). */
+int distsim_decode(distsim_ctx *ctx, int64_t index, distsim_candidate *h_out);
+
+/*
+ * Batch time of candidates [first, first + count): for each, MP modeling, the
+ * pipeline recurrence of Algorithm 1 (an item starts at the later of its input's
+ * arrival and its device becoming free), DP modeling, and the critical path.
+ *   d_batch_ns      [count]            out
+ *   d_stage_busy_ns [count][pp_max]    out, nullable: activity time of one device
+ *                                      of each stage (all replicas are identical);
+ *                                      entries d >= pp are 0
+ * Asynchronous on `stream`.
+ */
+int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64_t count,
+                            int64_t *d_batch_ns, int64_t *d_stage_busy_ns);
+
+/*
+ * Best strategy of a range (paper Sec. 5: the grid search keeps the fastest):
+ * smallest d_batch_ns[i], ties to the smallest index.  d_batch_ns[i] belongs to
+ * candidate first + i.  Results go to host memory; the call synchronises `stream`.
+ */
+int distsim_argmin(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int64_t first,
+                   int64_t count, int64_t *h_best_index, int64_t *h_best_batch_ns);
+
+/*
+ * The k fastest candidates of a range, ascending by (batch time, index).
+ *   d_indices [k] out (candidate indices, first + i);  d_times [k] out, nullable.
+ * Requires 1 <= k <= min(count, 4096).  Asynchronous on `stream`.
+ */
+int distsim_topk(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int64_t first,
+                 int64_t count, int32_t k, int64_t *d_indices, int64_t *d_times);
+
+/* One timeline record: event `kind` of `layer` for micro-batch `microbatch`
+ * occupying [start_ns, end_ns) on its device.  For transfers, `layer` is the
+ * stage's boundary layer; for gradient buckets it is the bucket number and
+ * microbatch is -1. */
+typedef struct { int64_t kind, layer, microbatch, start_ns, end_ns; } distsim_record;
+
+/*
+ * Full per-device timelines of n selected candidates (the simulator's output,
+ * paper Sec. 3.2; the per-device event lists F of Algorithm 1 after DP
+ * modeling).  Device rank (r*pp + d)*mp + q holds stage d of replica r.
+ * A device's records are its main lane in time order, then its gradient buckets.
+ *   d_indices  [n]                 candidate indices (device memory)
+ *   d_records  [capacity_records]  out, nullable: NULL = sizing pass only
+ *   d_offsets  [n*N + 1]           out: record offset of device k of selection i at
+ *                                  [i*N + k]; last entry = total
+ *   d_busy_ns  [n*N], d_util [n*N] out: activity time (union of the device's event
+ *                                  intervals) and busy / batch time
+ *   h_total_records                out (host): records needed
+ * If capacity_records is too small nothing is written to d_records and the call
+ * returns DISTSIM_E_CAPACITY with *h_total_records set.  Synchronises `stream`.
+ */
+int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indices, int32_t n,
+                           distsim_record *d_records, int64_t capacity_records,
+                           int64_t *d_offsets, int64_t *d_busy_ns, double *d_util,
+                           int64_t *h_total_records);
+
+/*
+ * Whole search from host memory: loads the table and space, evaluates every
+ * candidate, and returns the best one and the k fastest to host buffers.
+ *   h_topk_indices/h_topk_times [k]  out, nullable when k == 0
+ * Synchronises.  Uses internal device scratch for the batch times.
+ */
+int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table,
+                        const distsim_space *h_space, int32_t k, int64_t *h_n_candidates,
+                        int64_t *h_best_index, int64_t *h_best_batch_ns,
+                        int64_t *h_topk_indices, int64_t *h_topk_times);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+int64_t distsim_launch_count(const distsim_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DISTSIM_H */

@@ -1,0 +1,585 @@
+/*
+ * distsim_oracle.c -- TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-threaded CPU restatement of DistSim's hierarchical
+ * modeling (paper Sec. 4.3): MP modeling, PP modeling (Algorithm 1, run as a
+ * literal worklist over explicit event objects), DP modeling, and the timeline
+ * analyses (batch time, per-device busy time, utilisation; paper Sec. 3.2).
+ * It exists so that the CUDA engine can be compared against something that can
+ * be checked against the paper by eye.  It shares no code, header, table or
+ * helper with the CUDA path and must never be called from the product path:
+ * only the test-suite, the smoke check and the benchmark's CPU-baseline leg
+ * may build, load or run it.
+ *
+ * Nothing here is blocked, fused, vectorised or reordered.  All times are
+ * int64 nanoseconds; the only arithmetic is +, max and round-up division in
+ * the communication cost formulas; utilisation is one fp64 division.
+ *
+ * Notation (paper Sec. 4.3 / Algorithm 1 plus the alpha-beta cost model):
+ *   N devices, G per node, L layers, B global batch, s sequence, h hidden,
+ *   e bytes per activation element.  A candidate strategy is
+ *   x = (mp, pp, dp = N/(mp*pp), stage bounds 0=c_0<..<c_pp=L, m, sched);
+ *   Bp = B/dp, b = ceil(Bp/m); the event class is (mp, b).
+ *   Device index: rank(r,d,q) = (r*pp + d)*mp + q  (Algorithm 1 indexes the
+ *   pipeline lists as d*MP + m_p; DP modeling duplicates them DP times, so the
+ *   replica index r is outermost).  node(rank) = rank / G.
+ *
+ * Pins for every function here live in tests/test_oracle_pins.py (closed
+ * forms, invariants, brute-force longest path, hand-worked examples, printed
+ * counts from the paper).  The paper's measured accuracy against real clusters
+ * cannot be reproduced here: parity with measured reality is unpinned.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_MAX_PP 64
+
+enum {
+    ORC_OK = 0,
+    ORC_E_ARG = -1,       /* malformed argument                                 */
+    ORC_E_CLASS = -2,     /* event class (mp, b) missing from the table         */
+    ORC_E_LOCALITY = -3,  /* replicas of one stage would see different links    */
+    ORC_E_DEADLOCK = -4,  /* the worklist found no available schedule item      */
+    ORC_E_NOMEM = -5
+};
+
+/* Event kinds written to the `kind` field of a record. */
+enum {
+    ORC_COMPUTE_F = 0, ORC_COMPUTE_B = 1,
+    ORC_MP_AR_F = 2,   ORC_MP_AR_B = 3,
+    ORC_A2A_F = 4,     ORC_A2A_B = 5,
+    ORC_SEND_F = 6,    ORC_SEND_B = 7,
+    ORC_DP_AR = 8
+};
+
+/* The event table: profiled (here: synthetic) event times per class, plus the
+ * cluster constants of the alpha-beta communication model. */
+typedef struct {
+    int32_t n_layers, n_classes, n_devices, gpus_per_node;
+    int64_t global_batch, seq, hidden;
+    int64_t alpha_intra_ns, beta_intra;   /* beta in bytes per ns */
+    int64_t alpha_inter_ns, beta_inter;
+    int64_t dp_bucket_bytes;              /* 0: one all-reduce per stage          */
+    int32_t dp_overlap;                   /* 0: after the last event; 1: overlap  */
+    int32_t act_bytes_per_elem;
+    const int32_t *class_mp, *class_b;    /* [n_classes]                          */
+    const int64_t *fwd_ns, *bwd_ns;       /* [n_classes][n_layers]                */
+    const uint8_t *layer_is_expert;       /* [n_layers]                           */
+    const int64_t *grad_bytes;            /* [n_layers], at mp = 1                */
+} orc_table;
+
+/* The search space (paper Sec. 5: grid search over parallel degrees). */
+typedef struct {
+    int32_t mp_max, pp_max, n_m;
+    const int32_t *m_list;                /* ascending                            */
+    int32_t m_rule;                       /* 0: m divides Bp; 1: any m <= Bp      */
+    int32_t partition_mode;               /* 0: balanced; 1: all compositions     */
+    int32_t sched_mask;                   /* bit 0: GPipe, bit 1: 1F1B (Dapple)   */
+} orc_space;
+
+typedef struct {
+    int32_t mp, pp, dp, m, sched;         /* sched 0: GPipe, 1: 1F1B              */
+    int32_t bounds[ORC_MAX_PP + 1];       /* c_0 .. c_pp                          */
+} orc_candidate;
+
+typedef struct { int64_t kind, layer, mb, start, end; } orc_event;
+typedef struct { orc_event *ev; int64_t n, cap; } orc_list;
+
+typedef struct {
+    int32_t n_lists;          /* N (replicate) or pp (one device per stage)       */
+    int64_t batch_ns;
+    orc_list *lists;          /* final per-device event lists                     */
+    int64_t *busy_ns;         /* [n_lists] union measure of the event intervals   */
+    double *util;             /* [n_lists] busy / batch                           */
+} orc_result;
+
+/* ------------------------------------------------------------------------- */
+/* small helpers                                                              */
+
+static int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static int64_t max64(int64_t a, int64_t b) { return a > b ? a : b; }
+
+static int list_push(orc_list *l, orc_event e)
+{
+    if (l->n == l->cap) {
+        int64_t nc = l->cap ? 2 * l->cap : 64;
+        orc_event *p = (orc_event *)realloc(l->ev, (size_t)nc * sizeof(orc_event));
+        if (!p) return ORC_E_NOMEM;
+        l->ev = p; l->cap = nc;
+    }
+    l->ev[l->n++] = e;
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Communication events: alpha-beta costs.                                    */
+/* The per-device volume of a ring all-reduce over n devices of a P-byte      */
+/* tensor is 2(n-1)P/n (paper Sec. 4.2, all-reduce profiling); each of its    */
+/* 2(n-1) steps also pays the link latency alpha.                             */
+
+int64_t orc_ring_allreduce_ns(int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
+{
+    return 2 * (n - 1) * alpha + cdiv(2 * (n - 1) * bytes, n * beta);
+}
+/* Pairwise-exchange all-to-all: n-1 steps, each moving 1/n of the buffer. */
+int64_t orc_all_to_all_ns(int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
+{
+    return (n - 1) * alpha + cdiv((n - 1) * bytes, n * beta);
+}
+/* Point-to-point activation transfer between adjacent stages. */
+int64_t orc_p2p_ns(int64_t bytes, int64_t alpha, int64_t beta)
+{
+    return alpha + cdiv(bytes, beta);
+}
+
+/* Intra/inter-node attribute of communication events (paper Sec. 4.1): a
+ * transfer is intra-node iff source and destination rank share a node; a
+ * collective is intra-node iff all its members do.  Found by brute force over
+ * every group the strategy creates; all replicas must agree, because the
+ * method models them with one event.  Returns 0 intra, 1 inter, -1 mixed. */
+static int64_t rank_of(const orc_candidate *x, int64_t r, int64_t d, int64_t q)
+{
+    return (r * x->pp + d) * x->mp + q;
+}
+static int merge_loc(int cur, int v) { return cur == -2 ? v : (cur == v ? cur : -1); }
+
+static int loc_mp_groups(const orc_table *T, const orc_candidate *x)
+{
+    int cur = -2;
+    for (int64_t r = 0; r < x->dp; ++r)
+        for (int64_t d = 0; d < x->pp; ++d) {
+            int inter = 0;
+            int64_t n0 = rank_of(x, r, d, 0) / T->gpus_per_node;
+            for (int64_t q = 1; q < x->mp; ++q)
+                if (rank_of(x, r, d, q) / T->gpus_per_node != n0) inter = 1;
+            cur = merge_loc(cur, inter);
+        }
+    return cur;
+}
+static int loc_dp_groups(const orc_table *T, const orc_candidate *x)
+{
+    int cur = -2;
+    for (int64_t d = 0; d < x->pp; ++d)
+        for (int64_t q = 0; q < x->mp; ++q) {
+            int inter = 0;
+            int64_t n0 = rank_of(x, 0, d, q) / T->gpus_per_node;
+            for (int64_t r = 1; r < x->dp; ++r)
+                if (rank_of(x, r, d, q) / T->gpus_per_node != n0) inter = 1;
+            cur = merge_loc(cur, inter);
+        }
+    return cur;
+}
+static int loc_boundary(const orc_table *T, const orc_candidate *x, int64_t d)
+{
+    int cur = -2;
+    for (int64_t r = 0; r < x->dp; ++r)
+        for (int64_t q = 0; q < x->mp; ++q) {
+            int inter = rank_of(x, r, d, q) / T->gpus_per_node !=
+                        rank_of(x, r, d + 1, q) / T->gpus_per_node;
+            cur = merge_loc(cur, inter);
+        }
+    return cur;
+}
+static int64_t alpha_of(const orc_table *T, int loc) { return loc ? T->alpha_inter_ns : T->alpha_intra_ns; }
+static int64_t beta_of(const orc_table *T, int loc) { return loc ? T->beta_inter : T->beta_intra; }
+
+/* ------------------------------------------------------------------------- */
+/* Search-space enumeration by nested loops, outermost first:                  */
+/*   mp ascending over powers of two <= mp_max;                                */
+/*   pp ascending over powers of two <= min(pp_max, L) with mp*pp | N, dp | B; */
+/*   m ascending over the valid entries of m_list;                             */
+/*   stage partition in lexicographic order of (c_1..c_{pp-1});                */
+/*   schedule: GPipe, then 1F1B.                                               */
+/* The paper's own grid (Sec. 5) walks mp and pp over powers of two and takes  */
+/* dp = GPUs/mp/pp, dropping the invalid combinations.                         */
+
+static int valid_m(const orc_space *S, int64_t Bp, int64_t m)
+{
+    if (m < 1 || m > Bp) return 0;
+    return S->m_rule == 0 ? (Bp % m == 0) : 1;
+}
+
+/* Advances bounds c_1..c_{pp-1} to the next (pp-1)-subset of {1..L-1} in
+ * lexicographic order; returns 0 when the last one has been passed. */
+static int next_partition(int32_t *c, int pp, int L)
+{
+    int i = pp - 1;
+    while (i >= 1 && c[i] == L - (pp - i)) --i;
+    if (i < 1) return 0;
+    ++c[i];
+    for (int j = i + 1; j <= pp - 1; ++j) c[j] = c[j - 1] + 1;
+    return 1;
+}
+
+typedef int (*orc_visit_fn)(void *ctx, int64_t index, const orc_candidate *x);
+
+/* Walks the whole space in canonical order; stops early when visit returns
+ * non-zero.  Returns the number of candidates visited (or the full count). */
+static int64_t walk_space(const orc_table *T, const orc_space *S, orc_visit_fn visit, void *ctx)
+{
+    int64_t index = 0;
+    const int L = T->n_layers;
+    for (int64_t mp = 1; mp <= S->mp_max; mp *= 2)
+        for (int64_t pp = 1; pp <= S->pp_max && pp <= L; pp *= 2) {
+            if (T->n_devices % (mp * pp) != 0) continue;
+            int64_t dp = T->n_devices / (mp * pp);
+            if (T->global_batch % dp != 0) continue;
+            int64_t Bp = T->global_batch / dp;
+            for (int mi = 0; mi < S->n_m; ++mi) {
+                int64_t m = S->m_list[mi];
+                if (!valid_m(S, Bp, m)) continue;
+                orc_candidate x;
+                memset(&x, 0, sizeof x);
+                x.mp = (int32_t)mp; x.pp = (int32_t)pp; x.dp = (int32_t)dp; x.m = (int32_t)m;
+                x.bounds[0] = 0; x.bounds[pp] = L;
+                if (S->partition_mode == 0)
+                    for (int j = 1; j < pp; ++j) x.bounds[j] = (int32_t)((int64_t)j * L / pp);
+                else
+                    for (int j = 1; j < pp; ++j) x.bounds[j] = j;
+                do {
+                    for (int sc = 0; sc < 2; ++sc) {
+                        if (!(S->sched_mask & (1 << sc))) continue;
+                        x.sched = sc;
+                        if (visit && visit(ctx, index, &x)) return index + 1;
+                        ++index;
+                    }
+                } while (S->partition_mode == 1 && next_partition(x.bounds, (int)pp, L));
+            }
+        }
+    return index;
+}
+
+int64_t orc_count(const orc_table *T, const orc_space *S)
+{
+    return walk_space(T, S, NULL, NULL);
+}
+
+typedef struct { const int64_t *idx; int64_t n, next; orc_candidate *out; } pick_ctx;
+static int pick_visit(void *vc, int64_t index, const orc_candidate *x)
+{
+    pick_ctx *c = (pick_ctx *)vc;
+    while (c->next < c->n && c->idx[c->next] == index) c->out[c->next++] = *x;
+    return c->next >= c->n;
+}
+/* Decodes the candidates at the given ascending indices by walking the loops. */
+int orc_enumerate_at(const orc_table *T, const orc_space *S, const int64_t *sorted_idx,
+                     int64_t n, orc_candidate *out)
+{
+    for (int64_t i = 1; i < n; ++i) if (sorted_idx[i] < sorted_idx[i - 1]) return ORC_E_ARG;
+    if (n > 0 && sorted_idx[0] < 0) return ORC_E_ARG;
+    pick_ctx c = { sorted_idx, n, 0, out };
+    walk_space(T, S, pick_visit, &c);
+    return c.next == n ? ORC_OK : ORC_E_ARG;
+}
+
+/* ------------------------------------------------------------------------- */
+/* The simulation of one candidate.                                           */
+
+typedef struct { int32_t is_bwd, mb; } orc_op;
+
+static int find_class(const orc_table *T, int64_t mp, int64_t b)
+{
+    for (int k = 0; k < T->n_classes; ++k)
+        if (T->class_mp[k] == mp && T->class_b[k] == b) return k;
+    return -1;
+}
+
+void orc_result_free(orc_result *R)
+{
+    if (!R) return;
+    if (R->lists) { for (int i = 0; i < R->n_lists; ++i) free(R->lists[i].ev); free(R->lists); }
+    free(R->busy_ns); free(R->util); free(R);
+}
+
+static int cmp_event_start(const void *a, const void *b)
+{
+    const orc_event *x = (const orc_event *)a, *y = (const orc_event *)b;
+    if (x->start != y->start) return x->start < y->start ? -1 : 1;
+    if (x->end != y->end) return x->end < y->end ? -1 : 1;
+    return 0;
+}
+/* Measure of the union of a device's event intervals (its activity time). */
+static int64_t union_measure(const orc_list *l)
+{
+    if (l->n == 0) return 0;
+    orc_event *tmp = (orc_event *)malloc((size_t)l->n * sizeof(orc_event));
+    memcpy(tmp, l->ev, (size_t)l->n * sizeof(orc_event));
+    qsort(tmp, (size_t)l->n, sizeof(orc_event), cmp_event_start);
+    int64_t total = 0, lo = tmp[0].start, hi = tmp[0].end;
+    for (int64_t i = 1; i < l->n; ++i) {
+        if (tmp[i].start > hi) { total += hi - lo; lo = tmp[i].start; hi = tmp[i].end; }
+        else hi = max64(hi, tmp[i].end);
+    }
+    total += hi - lo;
+    free(tmp);
+    return total;
+}
+
+/*
+ * orc_simulate
+ *   replicate    1: keep a list for every one of the N devices;
+ *                0: keep only the device (r=0, q=0) of every stage (pp lists).
+ *   reverse_scan 0: first_available scans stages 0..pp-1; 1: pp-1..0.  The
+ *                result must not depend on it (each item's start depends only
+ *                on its two predecessors).
+ */
+orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replicate,
+                         int reverse_scan, int *err)
+{
+    int e = ORC_OK;
+    orc_result *R = NULL;
+    orc_list *F = NULL;          /* Algorithm 1's event lists, pipeline only      */
+    orc_op *ops = NULL;          /* schedule S: per stage, 2m items in order      */
+    int64_t *endF = NULL, *endB = NULL;
+    orc_event *tmp = NULL;
+    const int pp = x->pp, mp = x->mp, dp = x->dp, m = x->m, L = T->n_layers;
+
+    if (pp < 1 || pp > ORC_MAX_PP || mp < 1 || dp < 1 || m < 1 ||
+        (int64_t)mp * pp * dp != T->n_devices || T->global_batch % dp != 0 ||
+        x->bounds[0] != 0 || x->bounds[pp] != L || (x->sched != 0 && x->sched != 1)) {
+        e = ORC_E_ARG; goto fail;
+    }
+    for (int d = 0; d < pp; ++d) if (x->bounds[d + 1] <= x->bounds[d]) { e = ORC_E_ARG; goto fail; }
+
+    /* ---- Step 1: events and their elapsed times (MP modeling) ------------- */
+    const int64_t Bp = T->global_batch / dp;
+    const int64_t b = cdiv(Bp, m);
+    const int kappa = find_class(T, mp, b);
+    if (kappa < 0) { e = ORC_E_CLASS; goto fail; }
+    const int64_t *f = T->fwd_ns + (int64_t)kappa * L;
+    const int64_t *g = T->bwd_ns + (int64_t)kappa * L;
+    const int64_t act = b * T->seq * T->hidden * T->act_bytes_per_elem;
+
+    int64_t AR = 0, A2A = 0, P2P[ORC_MAX_PP];
+    int loc_dp = 0;
+    if (mp > 1) {
+        int loc = loc_mp_groups(T, x);
+        if (loc < 0) { e = ORC_E_LOCALITY; goto fail; }
+        AR = orc_ring_allreduce_ns(mp, 2 * act, alpha_of(T, loc), beta_of(T, loc));
+    }
+    if (dp > 1) {
+        loc_dp = loc_dp_groups(T, x);
+        if (loc_dp < 0) { e = ORC_E_LOCALITY; goto fail; }
+        A2A = orc_all_to_all_ns(dp, act, alpha_of(T, loc_dp), beta_of(T, loc_dp));
+    }
+    for (int d = 0; d + 1 < pp; ++d) {
+        int loc = loc_boundary(T, x, d);
+        if (loc < 0) { e = ORC_E_LOCALITY; goto fail; }
+        P2P[d] = orc_p2p_ns(act, alpha_of(T, loc), beta_of(T, loc));
+    }
+
+    /* ---- Step 2: the pipeline schedule S(D, L, M) -------------------------- */
+    ops = (orc_op *)malloc((size_t)pp * 2 * m * sizeof(orc_op));
+    endF = (int64_t *)malloc((size_t)pp * m * sizeof(int64_t));
+    endB = (int64_t *)malloc((size_t)pp * m * sizeof(int64_t));
+    tmp = (orc_event *)malloc((size_t)(3 * L + 1) * sizeof(orc_event));
+    const int mp_lists = replicate ? mp : 1;
+    F = (orc_list *)calloc((size_t)pp * mp_lists, sizeof(orc_list));
+    if (!ops || !endF || !endB || !tmp || !F) { e = ORC_E_NOMEM; goto fail; }
+    for (int64_t i = 0; i < (int64_t)pp * m; ++i) endF[i] = endB[i] = -1;
+    for (int d = 0; d < pp; ++d) {
+        orc_op *o = ops + (int64_t)d * 2 * m;
+        int k = 0;
+        if (x->sched == 0) {                      /* GPipe: all forwards, then all backwards */
+            for (int j = 0; j < m; ++j) { o[k].is_bwd = 0; o[k++].mb = j; }
+            for (int j = 0; j < m; ++j) { o[k].is_bwd = 1; o[k++].mb = j; }
+        } else {                                  /* 1F1B (Dapple): warm-up, then one-B-one-F */
+            int w = pp - d < m ? pp - d : m;
+            int nf = 0, nb = 0;
+            for (; nf < w; ++nf) { o[k].is_bwd = 0; o[k++].mb = nf; }
+            while (nb < m) {
+                o[k].is_bwd = 1; o[k++].mb = nb++;
+                if (nf < m) { o[k].is_bwd = 0; o[k++].mb = nf++; }
+            }
+        }
+    }
+
+    /* ---- Step 3: Algorithm 1 as a worklist ---------------------------------- */
+    {
+        int32_t head[ORC_MAX_PP];
+        int64_t device_free[ORC_MAX_PP];
+        int64_t remaining = (int64_t)pp * 2 * m;
+        for (int d = 0; d < pp; ++d) { head[d] = 0; device_free[d] = 0; }
+        while (remaining > 0) {
+            /* first_available: the first stage whose next item has its data ready */
+            int pick = -1; int64_t t = 0;
+            for (int s = 0; s < pp && pick < 0; ++s) {
+                int d = reverse_scan ? pp - 1 - s : s;
+                if (head[d] == 2 * m) continue;
+                orc_op o = ops[(int64_t)d * 2 * m + head[d]];
+                int64_t dep;
+                if (!o.is_bwd) dep = d == 0 ? 0 : endF[(int64_t)(d - 1) * m + o.mb];
+                else dep = d == pp - 1 ? endF[(int64_t)d * m + o.mb] : endB[(int64_t)(d + 1) * m + o.mb];
+                if (dep < 0) continue;
+                pick = d; t = max64(device_free[d], dep);
+            }
+            if (pick < 0) { e = ORC_E_DEADLOCK; goto fail; }
+            const int d = pick;
+            const orc_op o = ops[(int64_t)d * 2 * m + head[d]];
+            /* e <- MAP[l]: the stage's layers, each a computation event followed by
+             * its all-reduce event (mp > 1) and its all-to-all event (expert layer,
+             * dp > 1); then e_comm, the transfer to the neighbouring stage. */
+            int n = 0;
+            if (!o.is_bwd) {
+                for (int l = x->bounds[d]; l < x->bounds[d + 1]; ++l) {
+                    tmp[n++] = (orc_event){ ORC_COMPUTE_F, l, o.mb, t, t + f[l] }; t += f[l];
+                    if (mp > 1) { tmp[n++] = (orc_event){ ORC_MP_AR_F, l, o.mb, t, t + AR }; t += AR; }
+                    if (T->layer_is_expert[l] && dp > 1) { tmp[n++] = (orc_event){ ORC_A2A_F, l, o.mb, t, t + A2A }; t += A2A; }
+                }
+                if (d < pp - 1) { tmp[n++] = (orc_event){ ORC_SEND_F, x->bounds[d + 1] - 1, o.mb, t, t + P2P[d] }; t += P2P[d]; }
+                endF[(int64_t)d * m + o.mb] = t;
+            } else {
+                for (int l = x->bounds[d + 1] - 1; l >= x->bounds[d]; --l) {
+                    tmp[n++] = (orc_event){ ORC_COMPUTE_B, l, o.mb, t, t + g[l] }; t += g[l];
+                    if (mp > 1) { tmp[n++] = (orc_event){ ORC_MP_AR_B, l, o.mb, t, t + AR }; t += AR; }
+                    if (T->layer_is_expert[l] && dp > 1) { tmp[n++] = (orc_event){ ORC_A2A_B, l, o.mb, t, t + A2A }; t += A2A; }
+                }
+                if (d > 0) { tmp[n++] = (orc_event){ ORC_SEND_B, x->bounds[d], o.mb, t, t + P2P[d - 1] }; t += P2P[d - 1]; }
+                endB[(int64_t)d * m + o.mb] = t;
+            }
+            device_free[d] = t;
+            for (int q = 0; q < mp_lists; ++q)          /* every device of the MP group */
+                for (int i = 0; i < n; ++i)
+                    if ((e = list_push(&F[d * mp_lists + q], tmp[i])) != ORC_OK) goto fail;
+            ++head[d]; --remaining;                      /* S <- S - st */
+        }
+    }
+
+    /* ---- Step 4: DP modeling -------------------------------------------------- */
+    R = (orc_result *)calloc(1, sizeof(orc_result));
+    if (!R) { e = ORC_E_NOMEM; goto fail; }
+    R->n_lists = replicate ? T->n_devices : pp;
+    R->lists = (orc_list *)calloc((size_t)R->n_lists, sizeof(orc_list));
+    R->busy_ns = (int64_t *)calloc((size_t)R->n_lists, sizeof(int64_t));
+    R->util = (double *)calloc((size_t)R->n_lists, sizeof(double));
+    if (!R->lists || !R->busy_ns || !R->util) { e = ORC_E_NOMEM; goto fail; }
+    {
+        const int dp_lists = replicate ? dp : 1;
+        for (int r = 0; r < dp_lists; ++r)
+            for (int d = 0; d < pp; ++d)
+                for (int q = 0; q < mp_lists; ++q) {
+                    /* duplicate the pipeline list of (d, q) for replica r */
+                    orc_list *src = &F[d * mp_lists + q];
+                    orc_list *dst = &R->lists[(r * pp + d) * mp_lists + q];
+                    for (int64_t i = 0; i < src->n; ++i)
+                        if ((e = list_push(dst, src->ev[i])) != ORC_OK) goto fail;
+                    if (dp == 1) continue;
+                    /* gradient all-reduce events: the stage's gradients, in the
+                     * order the backward pass produces them (last layer first),
+                     * cut into buckets; each bucket is a ring all-reduce over
+                     * the dp replicas on a separate communication lane. */
+                    const int64_t main_end = src->n ? src->ev[src->n - 1].end : 0;
+                    int64_t W = 0;
+                    for (int l = x->bounds[d]; l < x->bounds[d + 1]; ++l) W += cdiv(T->grad_bytes[l], mp);
+                    if (W == 0) continue;
+                    const int64_t bucket = T->dp_bucket_bytes > 0 ? T->dp_bucket_bytes : W;
+                    const int64_t nb = cdiv(W, bucket);
+                    int64_t prev_end = 0;
+                    for (int64_t k = 0; k < nb; ++k) {
+                        const int64_t lo = k * bucket;
+                        const int64_t hi = lo + bucket < W ? lo + bucket : W;
+                        int64_t ready = main_end;
+                        if (T->dp_overlap) {
+                            /* the layer holding the bucket's last byte (position hi-1) */
+                            int64_t pos = 0; int last = -1;
+                            for (int l = x->bounds[d + 1] - 1; l >= x->bounds[d]; --l) {
+                                int64_t gl = cdiv(T->grad_bytes[l], mp);
+                                if (hi - 1 >= pos && hi - 1 < pos + gl) { last = l; break; }
+                                pos += gl;
+                            }
+                            /* ready when that layer's backward events of the LAST
+                             * microbatch's backward pass have all finished */
+                            ready = -1;
+                            for (int64_t i = 0; i < src->n; ++i) {
+                                const orc_event *v = &src->ev[i];
+                                if (v->layer == last && v->mb == m - 1 &&
+                                    (v->kind == ORC_COMPUTE_B || v->kind == ORC_MP_AR_B || v->kind == ORC_A2A_B))
+                                    ready = max64(ready, v->end);
+                            }
+                            if (ready < 0) { e = ORC_E_ARG; goto fail; }
+                        }
+                        const int64_t start = max64(ready, prev_end);
+                        const int64_t end = start + orc_ring_allreduce_ns(dp, hi - lo, alpha_of(T, loc_dp), beta_of(T, loc_dp));
+                        if ((e = list_push(dst, (orc_event){ ORC_DP_AR, k, -1, start, end })) != ORC_OK) goto fail;
+                        prev_end = end;
+                    }
+                }
+    }
+
+    /* ---- Step 5: timeline analyses --------------------------------------------- */
+    R->batch_ns = 0;
+    for (int i = 0; i < R->n_lists; ++i)
+        for (int64_t k = 0; k < R->lists[i].n; ++k)
+            R->batch_ns = max64(R->batch_ns, R->lists[i].ev[k].end);
+    for (int i = 0; i < R->n_lists; ++i) {
+        R->busy_ns[i] = union_measure(&R->lists[i]);
+        R->util[i] = R->batch_ns > 0 ? (double)R->busy_ns[i] / (double)R->batch_ns : 0.0;
+    }
+
+    for (int i = 0; i < pp * mp_lists; ++i) free(F[i].ev);
+    free(F); free(ops); free(endF); free(endB); free(tmp);
+    if (err) *err = ORC_OK;
+    return R;
+
+fail:
+    if (F) { for (int i = 0; i < pp * (replicate ? mp : 1); ++i) free(F[i].ev); free(F); }
+    free(ops); free(endF); free(endB); free(tmp);
+    orc_result_free(R);
+    if (err) *err = e;
+    return NULL;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Accessors for callers that cannot see the struct layout.                    */
+
+int64_t orc_result_batch(const orc_result *R) { return R->batch_ns; }
+int32_t orc_result_n_lists(const orc_result *R) { return R->n_lists; }
+int64_t orc_result_total_records(const orc_result *R)
+{
+    int64_t t = 0;
+    for (int i = 0; i < R->n_lists; ++i) t += R->lists[i].n;
+    return t;
+}
+/* offsets[n_lists+1] (in records), records[total][5], busy[n_lists], util[n_lists] */
+void orc_result_copy(const orc_result *R, int64_t *offsets, int64_t *records, int64_t *busy, double *util)
+{
+    int64_t t = 0;
+    for (int i = 0; i < R->n_lists; ++i) {
+        if (offsets) offsets[i] = t;
+        if (records) memcpy(records + 5 * t, R->lists[i].ev, (size_t)R->lists[i].n * sizeof(orc_event));
+        if (busy) busy[i] = R->busy_ns[i];
+        if (util) util[i] = R->util[i];
+        t += R->lists[i].n;
+    }
+    if (offsets) offsets[R->n_lists] = t;
+}
+
+/* Batch time and per-stage busy time (device r=0, q=0 of each stage) of the
+ * candidates at the given ascending indices.  stage_busy is [n][pp_stride],
+ * unused entries set to 0; nullable.  Single-threaded. */
+int orc_eval_indices(const orc_table *T, const orc_space *S, const int64_t *sorted_idx, int64_t n,
+                     int replicate, int64_t *batch_ns, int64_t *stage_busy, int32_t pp_stride)
+{
+    orc_candidate *c = (orc_candidate *)malloc((size_t)(n > 0 ? n : 1) * sizeof(orc_candidate));
+    if (!c) return ORC_E_NOMEM;
+    int e = orc_enumerate_at(T, S, sorted_idx, n, c);
+    for (int64_t i = 0; i < n && e == ORC_OK; ++i) {
+        orc_result *R = orc_simulate(T, &c[i], replicate, 0, &e);
+        if (!R) break;
+        batch_ns[i] = R->batch_ns;
+        if (stage_busy) {
+            for (int d = 0; d < pp_stride; ++d) stage_busy[i * pp_stride + d] = 0;
+            for (int d = 0; d < c[i].pp && d < pp_stride; ++d) {
+                /* with replicate, stage d's first device is rank (0*pp + d)*mp + 0 */
+                int li = replicate ? d * c[i].mp : d;
+                stage_busy[i * pp_stride + d] = R->busy_ns[li];
+            }
+        }
+        orc_result_free(R);
+    }
+    free(c);
+    return e;
+}
+
+int orc_sizeof_candidate(void) { return (int)sizeof(orc_candidate); }

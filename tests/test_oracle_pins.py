@@ -1,0 +1,405 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+Nothing here touches the CUDA engine.  Each test names the fact it pins; together
+they are chosen so that a dropped term, a wrong sign or index, or a transposed
+operand in the oracle fails at least one.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import Candidate, KINDS
+from paper_2306_08423_b200 import workloads as W
+from tests.dag_bruteforce import longest_path_timeline
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def make_table(f, g, *, n_devices, gpus_per_node, global_batch, classes, seq=0, hidden=1,
+               expert=None, grad=None, scale_by_b=False, **kw):
+    """Table whose every class has the same per-layer times f, g (or b*f, b*g)."""
+    L = len(f)
+    fwd = np.array([[(b if scale_by_b else 1) * v for v in f] for (_, b) in classes], np.int64)
+    bwd = np.array([[(b if scale_by_b else 1) * v for v in g] for (_, b) in classes], np.int64)
+    return W.EventTable(
+        n_layers=L, n_devices=n_devices, gpus_per_node=gpus_per_node, global_batch=global_batch,
+        seq=seq, hidden=hidden, class_mp=[c[0] for c in classes], class_b=[c[1] for c in classes],
+        fwd_ns=fwd, bwd_ns=bwd,
+        layer_is_expert=np.zeros(L, np.uint8) if expert is None else expert,
+        grad_bytes=np.zeros(L, np.int64) if grad is None else grad, **kw)
+
+
+def balanced(L, pp):
+    return tuple(j * L // pp for j in range(pp + 1))
+
+
+# --------------------------------------------------------------------------- #
+# communication cost formulas
+
+def test_ring_allreduce_volume_matches_paper_formula():
+    # Sec. 4.2: per-device volume of an N-device ring all-reduce of P bytes is 2(N-1)P/N.
+    for n in (2, 3, 8, 64, 1024):
+        for p in (1, 7, 1000, 26214400):
+            assert oracle.ring_allreduce_ns(n, p, 0, 1) == math.ceil(2 * (n - 1) * p / n) == -(-2 * (n - 1) * p // n)
+    # ... which tends to 2P for large N
+    assert oracle.ring_allreduce_ns(10**6, 10**6, 0, 1) == 2 * 10**6 - 2
+    # latency term: 2(N-1) steps; bandwidth divides
+    assert oracle.ring_allreduce_ns(8, 0, 5, 3) == 70
+    assert oracle.ring_allreduce_ns(2, 300, 0, 300) == 1
+    assert oracle.ring_allreduce_ns(2, 301, 0, 300) == 2  # rounds up
+
+
+def test_p2p_and_all_to_all_formulas():
+    assert oracle.p2p_ns(1000, 7, 10) == 107
+    assert oracle.p2p_ns(1001, 7, 10) == 108
+    assert oracle.all_to_all_ns(4, 1000, 3, 5) == 3 * 3 + 150
+    assert oracle.all_to_all_ns(1, 1000, 3, 5) == 0
+
+
+# --------------------------------------------------------------------------- #
+# P-1: uniform stages, zero comm, dp = 1: batch = (m + pp - 1)(t_f + t_b)
+
+@pytest.mark.parametrize("sched", [0, 1])
+@pytest.mark.parametrize("pp,m", [(1, 1), (2, 2), (4, 8), (8, 3), (4, 1), (16, 5), (2, 9)])
+def test_uniform_pipeline_closed_form(pp, m, sched):
+    tf, tb, per_stage = 7, 13, 3
+    L = pp * per_stage
+    T = make_table([tf] * L, [tb] * L, n_devices=pp, gpus_per_node=1, global_batch=m,
+                   classes=[(1, 1)], alpha_intra_ns=0, alpha_inter_ns=0)
+    r = oracle.simulate(T, Candidate(1, pp, 1, m, sched, balanced(L, pp)))
+    assert r.batch_ns == (m + pp - 1) * per_stage * (tf + tb)
+    assert (r.busy_ns == m * per_stage * (tf + tb)).all()
+
+
+# P-2: pure data parallelism, one all-reduce after the last event
+@pytest.mark.parametrize("n", [2, 4, 16])
+def test_pure_data_parallel_closed_form(n):
+    f, g = [5, 11, 3], [9, 20, 8]
+    grad = np.array([1000, 555, 77], np.int64)
+    T = make_table(f, g, n_devices=n, gpus_per_node=4, global_batch=n, classes=[(1, 1)],
+                   grad=grad, dp_bucket_bytes=0, dp_overlap=0,
+                   alpha_intra_ns=3, beta_intra=16, alpha_inter_ns=40, beta_inter=2)
+    r = oracle.simulate(T, Candidate(1, 1, n, 1, 0, (0, 3)))
+    a, be = (3, 16) if n <= 4 else (40, 2)
+    S = int(grad.sum())
+    expect = sum(f) + sum(g) + 2 * (n - 1) * a + -(-2 * (n - 1) * S // (n * be))
+    assert r.batch_ns == expect
+    assert (r.busy_ns == expect).all() and np.allclose(r.util, 1.0, rtol=0, atol=0)
+
+
+# P-3: GPipe with per-stage-constant item times: identical-job flow-shop identity
+@pytest.mark.parametrize("seed", range(6))
+def test_gpipe_flow_shop_identity(seed):
+    rng = np.random.default_rng(seed)
+    pp, m, L = int(rng.integers(2, 6)), int(rng.integers(1, 7)), 11
+    cuts = sorted(rng.choice(np.arange(1, L), pp - 1, replace=False).tolist())
+    bounds = (0, *cuts, L)
+    f = rng.integers(1, 50, L).tolist()
+    g = rng.integers(1, 90, L).tolist()
+    T = make_table(f, g, n_devices=pp, gpus_per_node=2, global_batch=m, classes=[(1, 1)],
+                   seq=10, hidden=10, alpha_intra_ns=4, beta_intra=7, alpha_inter_ns=30, beta_inter=3)
+    r = oracle.simulate(T, Candidate(1, pp, 1, m, 0, bounds))
+    act = 1 * 10 * 10 * 2
+    p2p = [(4 + -(-act // 7)) if (d // 2 == (d + 1) // 2) else (30 + -(-act // 3)) for d in range(pp - 1)]
+    a = [sum(f[bounds[d]:bounds[d + 1]]) + (p2p[d] if d < pp - 1 else 0) for d in range(pp)]
+    gg = [sum(g[bounds[d]:bounds[d + 1]]) + (p2p[d - 1] if d > 0 else 0) for d in range(pp)]
+    for d in range(pp):
+        rec = r.records[r.offsets[d]:r.offsets[d + 1]]
+        for j in range(m):
+            endF = rec[(rec[:, 2] == j) & np.isin(rec[:, 0], [0, 2, 4, 6])][:, 4].max()
+            endB = rec[(rec[:, 2] == j) & np.isin(rec[:, 0], [1, 3, 5, 7])][:, 4].max()
+            assert endF == sum(a[:d + 1]) + j * max(a[:d + 1])
+            last_f = sum(a) + (m - 1) * max(a)
+            assert endB == last_f + sum(gg[d:]) + j * max(gg[d:])
+
+
+# P-4: no pipeline: m sequential forward+backward passes with their all-reduces
+def test_single_stage_sum():
+    f, g = [3, 4, 5], [6, 8, 10]
+    T = make_table(f, g, n_devices=4, gpus_per_node=4, global_batch=8, classes=[(4, 2)], seq=3,
+                   hidden=5, alpha_intra_ns=2, beta_intra=4)
+    r = oracle.simulate(T, Candidate(4, 1, 1, 4, 1, (0, 3)))
+    act = 2 * 3 * 5 * 2
+    ar = 2 * 3 * 2 + -(-2 * 3 * 2 * act // (4 * 4))
+    assert r.batch_ns == 4 * (sum(f) + sum(g) + 6 * ar)
+    assert r.offsets[-1] == 4 * (4 * 2 * 3 * 2)    # 4 devices x 4 mb x (F,B) x 3 layers x (compute, AR)
+
+
+# P-10: hand-worked examples (tests/golden/worked_pipeline_examples.txt)
+def test_hand_worked_examples():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "worked_pipeline_examples.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) == 4
+    for name, p2p, sched, batch, busy0, busy1 in rows:
+        T = make_table([1, 1], [2, 2], n_devices=2, gpus_per_node=1, global_batch=2, classes=[(1, 1)],
+                       alpha_intra_ns=int(p2p), alpha_inter_ns=int(p2p))
+        r = oracle.simulate(T, Candidate(1, 2, 1, 2, int(sched), (0, 1, 2)))
+        assert r.batch_ns == int(batch), name
+        assert r.busy_ns.tolist() == [int(busy0), int(busy1)]
+        assert r.util.tolist() == [int(busy0) / int(batch), int(busy1) / int(batch)]
+
+
+# --------------------------------------------------------------------------- #
+# P-6: brute-force longest path over the explicit event DAG, every record
+
+def _tiny_cases():
+    for seed in range(10):
+        w = W.random_small(seed, n_devices=8, gpus_per_node=4, n_layers=4, global_batch=8,
+                           mp_max=2, pp_max=4, m_list=(1, 2, 3), dp_overlap=seed % 2,
+                           dp_bucket_bytes=0 if seed % 5 == 4 else 700)
+        yield w
+
+
+@pytest.mark.parametrize("w", list(_tiny_cases()), ids=lambda w: w.name)
+def test_brute_force_longest_path(w):
+    n = oracle.count(w.table, w.space)
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(n))
+    assert any(c.pp == 4 and c.sched == 1 for c in cands)
+    for c in cands:
+        r = oracle.simulate(w.table, c, replicate=False)
+        batch, lanes = longest_path_timeline(w.table, c)
+        assert r.batch_ns == batch
+        for d in range(c.pp):
+            got = [tuple(x) for x in r.records[r.offsets[d]:r.offsets[d + 1]].tolist()]
+            assert got == lanes[d], (c, d)
+
+
+# --------------------------------------------------------------------------- #
+# P-5: invariants
+
+def _cases(seeds, **kw):
+    for seed in seeds:
+        w = W.random_small(seed, **kw)
+        n = oracle.count(w.table, w.space)
+        idx = np.unique(np.linspace(0, n - 1, 12).astype(np.int64))
+        for c in oracle.enumerate_at(w.table, w.space, idx):
+            yield w, c
+
+
+def test_replicas_identical_busy_is_sum_and_batch_dominates():
+    for w, c in _cases(range(20, 26)):
+        r = oracle.simulate(w.table, c, replicate=True)
+        red = oracle.simulate(w.table, c, replicate=False)
+        rev = oracle.simulate(w.table, c, replicate=True, reverse_scan=True)
+        assert r.batch_ns == red.batch_ns == rev.batch_ns
+        assert (r.records == rev.records).all() and (r.offsets == rev.offsets).all()
+        assert len(r.offsets) == w.table.n_devices + 1          # MP x PP x DP event lists (Sec. 4.3)
+        for rr in range(c.dp):
+            for d in range(c.pp):
+                for q in range(c.mp):
+                    k = (rr * c.pp + d) * c.mp + q                # Algorithm 1: F[d*MP + m_p]
+                    a = r.records[r.offsets[k]:r.offsets[k + 1]]
+                    bq = red.records[red.offsets[d]:red.offsets[d + 1]]
+                    assert (a == bq).all()
+                    assert r.busy_ns[k] == red.busy_ns[d]
+        assert r.batch_ns >= r.busy_ns.max()
+        assert (r.records[:, 4] >= r.records[:, 3]).all() and (r.records[:, 3] >= 0).all()
+        assert r.records[:, 3].min() == 0                         # time origin: first item starts at 0
+
+
+def test_busy_equals_sum_of_durations_without_overlap():
+    for w, c in _cases(range(30, 34), dp_overlap=0):
+        r = oracle.simulate(w.table, c, replicate=False)
+        for d in range(c.pp):
+            rec = r.records[r.offsets[d]:r.offsets[d + 1]]
+            assert r.busy_ns[d] == int((rec[:, 4] - rec[:, 3]).sum())
+
+
+def test_main_lane_is_serial_and_bucket_lane_is_serial():
+    for w, c in _cases(range(40, 44)):
+        r = oracle.simulate(w.table, c, replicate=False)
+        for d in range(c.pp):
+            rec = r.records[r.offsets[d]:r.offsets[d + 1]]
+            main, bk = rec[rec[:, 0] != 8], rec[rec[:, 0] == 8]
+            assert (main[1:, 3] >= main[:-1, 4]).all()
+            assert (bk[1:, 3] >= bk[:-1, 4]).all()
+            assert (bk[:, 1] == np.arange(len(bk))).all() and (bk[:, 2] == -1).all()
+            if c.dp == 1:
+                assert len(bk) == 0
+
+
+def _batch(table, c):
+    return oracle.simulate(table, c, replicate=False, want_records=False).batch_ns
+
+
+def test_monotone_in_durations_and_link_constants():
+    import copy
+    for w, c in _cases(range(50, 54)):
+        base = _batch(w.table, c)
+        rng = np.random.default_rng(w.seed)
+        for _ in range(4):
+            t = copy.deepcopy(w.table)
+            k, l = int(rng.integers(t.n_classes)), int(rng.integers(t.n_layers))
+            (t.fwd_ns if rng.integers(2) else t.bwd_ns)[:, l] += int(rng.integers(1, 5000))
+            assert _batch(t, c) >= base
+        for name, sign in (("alpha_intra_ns", 1), ("alpha_inter_ns", 1), ("beta_intra", -1), ("beta_inter", -1)):
+            t = copy.deepcopy(w.table)
+            setattr(t, name, getattr(t, name) + 3)
+            assert sign * (_batch(t, c) - base) >= 0
+        t = copy.deepcopy(w.table); t.dp_overlap = 0
+        appended = _batch(t, c)
+        assert appended >= base                                    # overlapping never hurts
+        # gradient volume: monotone when every bucket waits for the end of the lane (with
+        # overlap, more bytes can move a fixed-size bucket's last byte into an earlier layer)
+        t.grad_bytes = t.grad_bytes + 999
+        assert _batch(t, c) >= appended
+
+
+# P-11: bucket properties
+def test_bucket_chain_properties():
+    f, g = [10, 10, 10, 10], [20, 20, 20, 20]
+    grad = np.array([400, 400, 400, 400], np.int64)
+    kw = dict(n_devices=4, gpus_per_node=4, global_batch=4, classes=[(1, 1), (1, 2)], grad=grad,
+              alpha_intra_ns=1, beta_intra=1)
+    # one layer per stage and bucket >= W_d: overlapped equals appended only for the first
+    # stage (no trailing transfer there); with a transfer, overlap starts the bucket earlier.
+    for bucket in (0, 400, 1000):
+        Ta = make_table(f, g, dp_bucket_bytes=bucket, dp_overlap=1, **kw)
+        Tb = make_table(f, g, dp_bucket_bytes=bucket, dp_overlap=0, **kw)
+        c = Candidate(1, 2, 2, 1, 0, (0, 2, 4))
+        ra, rb = oracle.simulate(Ta, c, replicate=False), oracle.simulate(Tb, c, replicate=False)
+        a0 = ra.records[ra.offsets[0]:ra.offsets[1]]; b0 = rb.records[rb.offsets[0]:rb.offsets[1]]
+        if bucket in (0, 1000):
+            assert (a0 == b0).all()                                # stage 0: last layer ends the lane
+    # identical ready times: K full buckets back to back = K * T_full
+    T0 = make_table(f, g, dp_bucket_bytes=100, dp_overlap=0, **kw)
+    r = oracle.simulate(T0, Candidate(1, 1, 4, 1, 0, (0, 4)), replicate=False)
+    bk = r.records[r.records[:, 0] == 8]
+    t_full = oracle.ring_allreduce_ns(4, 100, 1, 1)
+    assert len(bk) == 16 and (bk[:, 4] - bk[:, 3] == t_full).all()
+    assert bk[-1, 4] - bk[0, 3] == 16 * t_full
+    # partial last bucket carries the remainder
+    T1 = make_table(f, g, dp_bucket_bytes=300, dp_overlap=1, **kw)
+    r = oracle.simulate(T1, Candidate(1, 1, 4, 1, 0, (0, 4)), replicate=False)
+    bk = r.records[r.records[:, 0] == 8]
+    assert len(bk) == 6 and bk[-1, 4] - bk[-1, 3] == oracle.ring_allreduce_ns(4, 100, 1, 1)
+    # bucket k (bytes [300k, 300k+300)) ends inside layer 3 - (300k+299)//400; ready when that
+    # layer's backward of the last microbatch ends; layers run 3,2,1,0 taking 20 ns each after
+    # the forward pass (40 ns)
+    fwd_end = 40
+    prev = 0
+    for k in range(6):
+        last = min(300 * k + 299, 1599)
+        ready = fwd_end + 20 * (last // 400 + 1)
+        start = max(ready, prev)
+        assert bk[k, 3] == start
+        prev = bk[k, 4]
+
+
+# --------------------------------------------------------------------------- #
+# enumeration pins
+
+def test_paper_grid_has_15_valid_settings():
+    # Sec. 5: degrees {1,2,4,8,16} on 16 GPUs -> 15 valid (mp, pp) settings, dp = GPUs/mp/pp
+    sp = W.SearchSpace(mp_max=16, pp_max=16, m_list=[1], sched_mask=1)
+    T = make_table([1] * 48, [1] * 48, n_devices=16, gpus_per_node=4, global_batch=16, classes=[(1, 1)])
+    n = oracle.count(T, sp)
+    assert n == 15
+    cands = oracle.enumerate_at(T, sp, np.arange(n))
+    assert len({(c.mp, c.pp) for c in cands}) == 15
+    assert all(c.mp * c.pp * c.dp == 16 for c in cands)
+
+
+def test_paper_per_stage_example_item_counts():
+    # Sec. 6.4: "2m4p1d", 4 micro-batches -> 32 forward and backward items, 4 (each) per GPU
+    T = make_table([5] * 8, [9] * 8, n_devices=8, gpus_per_node=4, global_batch=4, classes=[(2, 1)],
+                   seq=4, hidden=4)
+    for sched in (0, 1):
+        r = oracle.simulate(T, Candidate(2, 4, 1, 4, sched, (0, 2, 4, 6, 8)))
+        assert len(r.offsets) == 9
+        tot_f = tot_b = 0
+        for k in range(8):
+            rec = r.records[r.offsets[k]:r.offsets[k + 1]]
+            first_layer = (k // 2) * 2
+            nf = int(((rec[:, 0] == 0) & (rec[:, 1] == first_layer)).sum())
+            nb = int(((rec[:, 0] == 1) & (rec[:, 1] == first_layer)).sum())
+            assert nf == 4 and nb == 4
+            tot_f += nf; tot_b += nb
+        assert tot_f == 32 and tot_b == 32
+        # the two GPUs of an MP group behave identically (Sec. 6.4)
+        for k in range(0, 8, 2):
+            assert (r.records[r.offsets[k]:r.offsets[k + 1]] == r.records[r.offsets[k + 1]:r.offsets[k + 2]]).all()
+
+
+def test_composition_count_and_lexicographic_order():
+    L = 9
+    T = make_table([1] * L, [1] * L, n_devices=4, gpus_per_node=4, global_batch=4, classes=[(1, 1), (1, 2), (1, 4)])
+    sp = W.SearchSpace(mp_max=1, pp_max=4, m_list=[1], partition_mode=W.PARTITION_ALL, sched_mask=2)
+    n = oracle.count(T, sp)
+    assert n == sum(math.comb(L - 1, pp - 1) for pp in (1, 2, 4))
+    cands = oracle.enumerate_at(T, sp, np.arange(n))
+    expect = []
+    for pp in (1, 2, 4):
+        for cut in itertools.combinations(range(1, L), pp - 1):     # lexicographic
+            expect.append((pp, (0, *cut, L)))
+    assert [(c.pp, c.bounds) for c in cands] == expect
+
+
+def test_canonical_order_against_python_loops():
+    for cfg in (0, 2):
+        w = W.CONFIGS[cfg]()
+        T, sp = w.table, w.space
+        expect = []
+        mp = 1
+        while mp <= sp.mp_max:
+            pp = 1
+            while pp <= min(sp.pp_max, T.n_layers):
+                if T.n_devices % (mp * pp) == 0 and T.global_batch % (T.n_devices // (mp * pp)) == 0:
+                    dp = T.n_devices // (mp * pp)
+                    bp = T.global_batch // dp
+                    for m in sp.m_list.tolist():
+                        ok = m <= bp and (bp % m == 0 if sp.m_rule == 0 else True)
+                        if ok:
+                            for sc in (0, 1):
+                                expect.append((mp, pp, dp, m, sc, balanced(T.n_layers, pp)))
+                pp *= 2
+            mp *= 2
+        n = oracle.count(T, sp)
+        assert n == len(expect) == {0: 88, 2: 4176}[cfg]
+        got = oracle.enumerate_at(T, sp, np.arange(n))
+        assert [(c.mp, c.pp, c.dp, c.m, c.sched, c.bounds) for c in got] == expect
+
+
+def test_candidate_counts_of_the_benchmark_spaces():
+    assert oracle.count(W.config1().table, W.config1().space) == 38_838_764
+    assert oracle.count(W.config3().table, W.config3().space) == 650_420
+
+
+def test_locality_of_collectives():
+    w = W.config0()
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(88))
+    T = w.table
+    for c in cands:
+        if c.m != 1 or c.sched != 0:
+            continue
+        r = oracle.simulate(T, c, replicate=False)
+        rec = r.records
+        b = T.global_batch // c.dp
+        act = b * T.seq * T.hidden * 2
+        ar = rec[rec[:, 0] == KINDS["MP_AR_F"]]
+        if c.mp > 1:
+            inter = c.mp > T.gpus_per_node                  # 8-way MP spans both 4-GPU nodes
+            a, be = (T.alpha_inter_ns, T.beta_inter) if inter else (T.alpha_intra_ns, T.beta_intra)
+            assert (ar[:, 4] - ar[:, 3] == oracle.ring_allreduce_ns(c.mp, 2 * act, a, be)).all()
+        else:
+            assert len(ar) == 0
+        snd = rec[rec[:, 0] == KINDS["SEND_F"]]
+        for row in snd:
+            d = list(c.bounds).index(row[1] + 1) - 1
+            inter = (d * c.mp) // 4 != ((d + 1) * c.mp) // 4
+            a, be = (T.alpha_inter_ns, T.beta_inter) if inter else (T.alpha_intra_ns, T.beta_intra)
+            assert row[4] - row[3] == oracle.p2p_ns(act, a, be)
+
+
+def test_errors():
+    T = make_table([1, 1], [1, 1], n_devices=2, gpus_per_node=1, global_batch=2, classes=[(1, 1)])
+    with pytest.raises(oracle.OracleError):
+        oracle.simulate(T, Candidate(1, 2, 1, 1, 0, (0, 1, 2)))      # class (1, 2) missing
+    with pytest.raises(oracle.OracleError):
+        oracle.simulate(T, Candidate(1, 2, 1, 2, 0, (0, 2, 2)))      # empty stage
+    with pytest.raises(oracle.OracleError):
+        oracle.simulate(T, Candidate(1, 1, 1, 2, 0, (0, 2)))         # degrees do not multiply to N
