@@ -1,0 +1,531 @@
+// Host side of the C ABI: context, validation, search-space bookkeeping, kernel launches.
+// No timeline arithmetic happens here; the host only counts the space, looks up event classes
+// and decides launch shapes.
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+#include <utility>
+#include <vector>
+
+#include "engine.h"
+
+using namespace distsim;
+
+namespace {
+
+struct DevBuf {
+    void *p = nullptr;
+    size_t cap = 0;
+    ~DevBuf() { if (p) cudaFree(p); }
+    cudaError_t reserve(size_t bytes)
+    {
+        if (bytes <= cap) return cudaSuccess;
+        if (p) { cudaFree(p); p = nullptr; cap = 0; }
+        cudaError_t e = cudaMalloc(&p, bytes);
+        if (e == cudaSuccess) cap = bytes;
+        return e;
+    }
+    template <class T> T *as() const { return static_cast<T *>(p); }
+};
+
+bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+
+int64_t sat_mul(int64_t a, int64_t b)
+{
+    const __int128 r = (__int128)a * b;
+    return r >= (__int128)kSat ? kSat : (int64_t)r;
+}
+int64_t sat_add(int64_t a, int64_t b)
+{
+    const __int128 r = (__int128)a + b;
+    return r >= (__int128)kSat ? kSat : (int64_t)r;
+}
+
+}  // namespace
+
+struct distsim_ctx {
+    int device = 0;
+    std::string err;
+    bool table_loaded = false, space_set = false;
+    int64_t launches = 0;
+
+    // table
+    TableConst tc{};
+    std::vector<int32_t> class_mp, class_b;
+    std::vector<int64_t> fwd, bwd, grad;
+    std::vector<uint8_t> expert;
+    DevBuf d_class_mp, d_class_b, d_fwd, d_bwd, d_expert, d_grad, d_next_grad, d_pe;
+    RawTable raw{};
+
+    // space
+    SpaceConst sc{};
+    std::vector<Row> rows;
+    std::vector<Entry> entries;
+    std::vector<int64_t> binom;
+    int64_t time_bound = 0;
+    int64_t op_words_per_cand = 0;
+    DevBuf d_rows, d_entries, d_etf, d_etb, d_nb, d_tp, d_binom;
+
+    // scratch
+    DevBuf d_status, d_sel, d_result, d_plans, d_op_start, d_totals, d_batch, d_topk;
+    int64_t *h_pinned = nullptr;          // 8 words of pinned host memory for small results
+
+    DeviceView view() const
+    {
+        DeviceView v{};
+        v.tc = tc; v.sc = sc; v.raw = raw;
+        v.rows = d_rows.as<Row>(); v.entries = d_entries.as<Entry>();
+        v.etf = d_etf.as<int64_t>(); v.etb = d_etb.as<int64_t>();
+        v.nb = d_nb.as<int64_t>(); v.tp = d_tp.as<int64_t>();
+        v.binom = d_binom.as<int64_t>();
+        v.next_grad = d_next_grad.as<int32_t>(); v.pe = d_pe.as<int32_t>();
+        v.status = d_status.as<int32_t>();
+        return v;
+    }
+    SelectScratch select_scratch() const
+    {
+        SelectScratch s{};
+        unsigned long long *base = d_sel.as<unsigned long long>();
+        s.key = base; s.hist = base + 8; s.sel_state = base + 8 + 256;
+        s.cand_time = reinterpret_cast<int64_t *>(base + 8 + 256 + 8);
+        s.cand_idx = s.cand_time + 4096;
+        return s;
+    }
+};
+
+namespace {
+
+int fail(distsim_ctx *c, int code, const char *msg)
+{
+    if (c) c->err = msg;
+    return code;
+}
+int cuda_fail(distsim_ctx *c, cudaError_t e, const char *what)
+{
+    if (c) c->err = std::string(what) + ": " + cudaGetErrorString(e);
+    return DISTSIM_E_CUDA;
+}
+
+#define CU(call, what)                                               \
+    do {                                                             \
+        cudaError_t e__ = (call);                                    \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, what);    \
+    } while (0)
+
+int set_device(distsim_ctx *ctx)
+{
+    CU(cudaSetDevice(ctx->device), "cudaSetDevice");
+    return DISTSIM_OK;
+}
+
+template <class T>
+int upload(distsim_ctx *ctx, DevBuf &b, const T *src, size_t n, const char *what)
+{
+    CU(b.reserve(n ? n * sizeof(T) : sizeof(T)), what);
+    if (n) CU(cudaMemcpy(b.p, src, n * sizeof(T), cudaMemcpyHostToDevice), what);
+    return DISTSIM_OK;
+}
+
+// Reads and clears the device status word; synchronises the stream.
+int read_status(distsim_ctx *ctx, cudaStream_t s)
+{
+    int32_t *st = reinterpret_cast<int32_t *>(ctx->h_pinned + 4);
+    CU(cudaMemcpyAsync(st, ctx->d_status.p, sizeof(int32_t), cudaMemcpyDeviceToHost, s), "status read");
+    CU(cudaStreamSynchronize(s), "status sync");
+    const int32_t code = *st;
+    if (code != 0) {
+        cudaMemsetAsync(ctx->d_status.p, 0, sizeof(int32_t), s);
+        if (code == DISTSIM_E_TIMEOUT)
+            return fail(ctx, code, "a bounded device-side wait gave up (the affected blocks read their tables from global memory instead)");
+        if (code == DISTSIM_E_RANGE) return fail(ctx, code, "candidate index out of range");
+        return fail(ctx, code, "device reported an error");
+    }
+    return DISTSIM_OK;
+}
+
+int floor_log2(int64_t v) { int b = -1; while (v > 0) { ++b; v >>= 1; } return b; }
+
+}  // namespace
+
+extern "C" {
+
+int distsim_create(distsim_ctx **out, int cuda_device)
+{
+    if (!out) return DISTSIM_E_ARG;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || cuda_device < 0 || cuda_device >= n) return DISTSIM_E_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cuda_device) != cudaSuccess) return DISTSIM_E_CUDA;
+    if (prop.major != 10) return DISTSIM_E_CUDA;           // built for sm_100a only
+    distsim_ctx *ctx = new (std::nothrow) distsim_ctx;
+    if (!ctx) return DISTSIM_E_ARG;
+    ctx->device = cuda_device;
+    if (cudaSetDevice(cuda_device) != cudaSuccess ||
+        ctx->d_status.reserve(64) != cudaSuccess ||
+        ctx->d_sel.reserve((8 + 256 + 8 + 2 * 4096) * sizeof(int64_t)) != cudaSuccess ||
+        ctx->d_result.reserve(64) != cudaSuccess || ctx->d_totals.reserve(64) != cudaSuccess ||
+        cudaMemset(ctx->d_status.p, 0, 64) != cudaSuccess ||
+        cudaMallocHost(&ctx->h_pinned, 8 * sizeof(int64_t)) != cudaSuccess) {
+        delete ctx;
+        return DISTSIM_E_CUDA;
+    }
+    *out = ctx;
+    return DISTSIM_OK;
+}
+
+void distsim_destroy(distsim_ctx *ctx)
+{
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
+    delete ctx;
+}
+
+const char *distsim_last_error(const distsim_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int64_t distsim_launch_count(const distsim_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *t)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!t) return fail(ctx, DISTSIM_E_ARG, "null table");
+    if (!t->class_mp || !t->class_b || !t->fwd_ns || !t->bwd_ns || !t->layer_is_expert || !t->grad_bytes)
+        return fail(ctx, DISTSIM_E_ARG, "null array in table");
+    if (t->n_layers < 1 || t->n_layers > DISTSIM_MAX_LAYERS) return fail(ctx, DISTSIM_E_ARG, "n_layers out of range");
+    if (t->n_classes < 1) return fail(ctx, DISTSIM_E_ARG, "no event classes");
+    if (!is_pow2(t->n_devices) || !is_pow2(t->gpus_per_node))
+        return fail(ctx, DISTSIM_E_UNSUPPORTED, "n_devices and gpus_per_node must be powers of two");
+    if (t->global_batch < 1 || t->seq < 0 || t->hidden < 0 || t->act_bytes_per_elem < 0)
+        return fail(ctx, DISTSIM_E_ARG, "negative size");
+    if (t->alpha_intra_ns < 0 || t->alpha_inter_ns < 0 || t->beta_intra < 1 || t->beta_inter < 1 || t->dp_bucket_bytes < 0)
+        return fail(ctx, DISTSIM_E_ARG, "bad link constants");
+    const int64_t L = t->n_layers, K = t->n_classes;
+    for (int64_t i = 0; i < K * L; ++i)
+        if (t->fwd_ns[i] < 0 || t->bwd_ns[i] < 0) return fail(ctx, DISTSIM_E_ARG, "negative event time");
+    for (int64_t k = 0; k < K; ++k)
+        if (t->class_mp[k] < 1 || t->class_b[k] < 1) return fail(ctx, DISTSIM_E_ARG, "bad event class");
+    int64_t gsum = 0;
+    for (int64_t l = 0; l < L; ++l) {
+        if (t->grad_bytes[l] < 0) return fail(ctx, DISTSIM_E_ARG, "negative gradient size");
+        gsum = sat_add(gsum, t->grad_bytes[l]);
+    }
+    if (gsum >= kSat / (4 * (int64_t)t->n_devices)) return fail(ctx, DISTSIM_E_OVERFLOW, "gradient volume too large");
+    if (int rc = set_device(ctx)) return rc;
+
+    ctx->table_loaded = false; ctx->space_set = false;
+    TableConst &tc = ctx->tc;
+    tc.n_layers = t->n_layers; tc.n_classes = t->n_classes; tc.n_devices = t->n_devices;
+    tc.gpus_per_node = t->gpus_per_node; tc.global_batch = t->global_batch; tc.seq = t->seq;
+    tc.hidden = t->hidden; tc.alpha_intra = t->alpha_intra_ns; tc.beta_intra = t->beta_intra;
+    tc.alpha_inter = t->alpha_inter_ns; tc.beta_inter = t->beta_inter; tc.bucket = t->dp_bucket_bytes;
+    tc.overlap = t->dp_overlap ? 1 : 0; tc.elem_bytes = t->act_bytes_per_elem;
+    tc.lp = (int32_t)((L + 1 + 1) & ~1); tc.pad = 0;
+    ctx->class_mp.assign(t->class_mp, t->class_mp + K);
+    ctx->class_b.assign(t->class_b, t->class_b + K);
+    ctx->fwd.assign(t->fwd_ns, t->fwd_ns + K * L);
+    ctx->bwd.assign(t->bwd_ns, t->bwd_ns + K * L);
+    ctx->grad.assign(t->grad_bytes, t->grad_bytes + L);
+    ctx->expert.assign(t->layer_is_expert, t->layer_is_expert + L);
+
+    if (int rc = upload(ctx, ctx->d_class_mp, ctx->class_mp.data(), K, "upload class_mp")) return rc;
+    if (int rc = upload(ctx, ctx->d_class_b, ctx->class_b.data(), K, "upload class_b")) return rc;
+    if (int rc = upload(ctx, ctx->d_fwd, ctx->fwd.data(), K * L, "upload fwd")) return rc;
+    if (int rc = upload(ctx, ctx->d_bwd, ctx->bwd.data(), K * L, "upload bwd")) return rc;
+    if (int rc = upload(ctx, ctx->d_expert, ctx->expert.data(), L, "upload expert")) return rc;
+    if (int rc = upload(ctx, ctx->d_grad, ctx->grad.data(), L, "upload grad")) return rc;
+    CU(ctx->d_next_grad.reserve((L + 1) * sizeof(int32_t)), "alloc next_grad");
+    CU(ctx->d_pe.reserve((L + 1) * sizeof(int32_t)), "alloc pe");
+    ctx->raw.class_mp = ctx->d_class_mp.as<int32_t>(); ctx->raw.class_b = ctx->d_class_b.as<int32_t>();
+    ctx->raw.fwd = ctx->d_fwd.as<int64_t>(); ctx->raw.bwd = ctx->d_bwd.as<int64_t>();
+    ctx->raw.expert = ctx->d_expert.as<uint8_t>(); ctx->raw.grad = ctx->d_grad.as<int64_t>();
+    launch_build_layer_tables(0, tc, ctx->raw, ctx->d_next_grad.as<int32_t>(), ctx->d_pe.as<int32_t>(), &ctx->launches);
+    CU(cudaGetLastError(), "layer tables launch");
+    ctx->table_loaded = true;
+    return DISTSIM_OK;
+}
+
+int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_candidates)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!sp || !n_candidates) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (!ctx->table_loaded) return fail(ctx, DISTSIM_E_STATE, "no event table loaded");
+    if (sp->mp_max < 1 || sp->pp_max < 1 || sp->n_m < 1 || !sp->m_list) return fail(ctx, DISTSIM_E_ARG, "empty space");
+    if (sp->pp_max > DISTSIM_MAX_PP) return fail(ctx, DISTSIM_E_ARG, "pp_max too large");
+    if ((sp->sched_mask & 3) == 0 || (sp->sched_mask & ~3)) return fail(ctx, DISTSIM_E_ARG, "bad sched_mask");
+    if (sp->m_rule < 0 || sp->m_rule > 1 || sp->partition_mode < 0 || sp->partition_mode > 1)
+        return fail(ctx, DISTSIM_E_ARG, "bad m_rule or partition_mode");
+    for (int i = 0; i < sp->n_m; ++i) {
+        if (sp->m_list[i] < 1 || sp->m_list[i] > DISTSIM_MAX_M) return fail(ctx, DISTSIM_E_ARG, "m out of range");
+        if (i && sp->m_list[i] <= sp->m_list[i - 1]) return fail(ctx, DISTSIM_E_ARG, "m_list must ascend");
+    }
+    if (int rc = set_device(ctx)) return rc;
+    ctx->space_set = false;
+    const TableConst &tc = ctx->tc;
+    const int L = tc.n_layers;
+    const int64_t N = tc.n_devices, B = tc.global_batch;
+
+    std::map<std::pair<int, int>, int> class_of;
+    for (int k = 0; k < tc.n_classes; ++k) class_of.emplace(std::make_pair(ctx->class_mp[k], ctx->class_b[k]), k);
+
+    // binomials C(n, k), n < L, k < binom_k, saturated
+    int pp_cap = 1;
+    while (pp_cap * 2 <= sp->pp_max && pp_cap * 2 <= L) pp_cap *= 2;
+    const int bk = pp_cap;
+    std::vector<int64_t> binom((size_t)L * bk, 0);
+    for (int n = 0; n < L; ++n)
+        for (int k = 0; k < bk; ++k) {
+            int64_t v;
+            if (k == 0) v = 1;
+            else if (n == 0) v = 0;
+            else v = sat_add(binom[(size_t)(n - 1) * bk + k - 1], binom[(size_t)(n - 1) * bk + k]);
+            binom[(size_t)n * bk + k] = v;
+        }
+
+    std::vector<Row> rows;
+    std::vector<Entry> entries;
+    int64_t total = 0, op_words = 0;
+    long double tb = 0;
+    const int n_sched = (sp->sched_mask == 3) ? 2 : 1;
+    const int sched0 = (sp->sched_mask & 1) ? 0 : 1;
+    long double fg_max = 0;                       // largest per-class sum of layer times
+    for (int k = 0; k < tc.n_classes; ++k) {
+        long double s = 0;
+        for (int l = 0; l < L; ++l) s += (long double)ctx->fwd[(size_t)k * L + l] + ctx->bwd[(size_t)k * L + l];
+        if (s > fg_max) fg_max = s;
+    }
+    long double gsum = 0;
+    for (int l = 0; l < L; ++l) gsum += ctx->grad[l];
+    const long double a_max = (long double)(tc.alpha_inter > tc.alpha_intra ? tc.alpha_inter : tc.alpha_intra);
+    const long double b_min = (long double)(tc.beta_inter < tc.beta_intra ? tc.beta_inter : tc.beta_intra);
+
+    for (int64_t mp = 1; mp <= sp->mp_max; mp *= 2)
+        for (int64_t pp = 1; pp <= sp->pp_max && pp <= L; pp *= 2) {
+            if (N % (mp * pp)) continue;
+            const int64_t dp = N / (mp * pp);
+            if (B % dp) continue;
+            const int64_t Bp = B / dp;
+            Row r{};
+            r.mp = (int32_t)mp; r.pp = (int32_t)pp; r.dp = (int32_t)dp; r.log2_mp = floor_log2(mp);
+            r.entry0 = (int32_t)entries.size(); r.n_entries = 0;
+            r.n_sched = n_sched; r.sched0 = sched0;
+            r.p2p_period = mp >= tc.gpus_per_node ? 1 : (int32_t)(tc.gpus_per_node / mp);
+            r.n_part = sp->partition_mode == 0 ? 1 : binom[(size_t)(L - 1) * bk + (pp - 1)];
+            for (int i = 0; i < sp->n_m; ++i) {
+                const int64_t m = sp->m_list[i];
+                if (m > Bp) continue;
+                if (sp->m_rule == 0 && Bp % m) continue;
+                const int64_t b = (Bp + m - 1) / m;
+                auto it = class_of.find(std::make_pair((int)mp, (int)b));
+                if (it == class_of.end()) {
+                    char msg[128];
+                    snprintf(msg, sizeof msg, "event class (mp=%lld, b=%lld) is not in the table", (long long)mp, (long long)b);
+                    return fail(ctx, DISTSIM_E_ARG, msg);
+                }
+                Entry en{};
+                en.m = (int32_t)m; en.b = (int32_t)b; en.cls = it->second; en.row = (int32_t)rows.size();
+                entries.push_back(en);
+                ++r.n_entries;
+                if (2 * m * pp > op_words) op_words = 2 * m * pp;
+                // generous upper bound on any batch time of this entry: every item in sequence
+                const long double act = (long double)b * tc.seq * tc.hidden * tc.elem_bytes;
+                const long double comm = 2.0L * mp * a_max + 4.0L * act / b_min + 2 + dp * a_max + act / b_min + 2;
+                const long double p2p = a_max + act / b_min + 2;
+                const long double nbk = tc.bucket > 0 ? gsum / tc.bucket + L + 1 : L + 1;
+                const long double bsz = tc.bucket > 0 ? (long double)tc.bucket : gsum;
+                const long double e_bound = (long double)m * (fg_max + 2.0L * L * comm + 2.0L * pp * p2p) +
+                                            nbk * (2.0L * dp * a_max + 2.0L * bsz / b_min + 2);
+                if (e_bound > tb) tb = e_bound;
+            }
+            if (r.n_entries == 0) continue;
+            r.size = sat_mul(sat_mul(r.n_part, r.n_entries), r.n_sched);
+            r.offset = total;
+            r.row_tab_off = (int64_t)rows.size() * (L + 1) * (L + 1);
+            total = sat_add(total, r.size);
+            if (r.n_part >= kSat || total >= kSat) return fail(ctx, DISTSIM_E_OVERFLOW, "candidate count does not fit 62 bits");
+            rows.push_back(r);
+        }
+    if (rows.empty()) return fail(ctx, DISTSIM_E_ARG, "the space has no valid candidate");
+    if (tb >= (long double)kSat) return fail(ctx, DISTSIM_E_OVERFLOW, "batch-time bound does not fit 62 bits");
+
+    ctx->rows = rows; ctx->entries = entries; ctx->binom = binom;
+    ctx->time_bound = (int64_t)tb + 1;
+    ctx->op_words_per_cand = op_words;
+    SpaceConst &sc = ctx->sc;
+    sc.n_rows = (int32_t)rows.size(); sc.n_entries = (int32_t)entries.size();
+    sc.pp_max = sp->pp_max; sc.partition_mode = sp->partition_mode; sc.binom_k = bk; sc.pad = 0;
+    sc.n_candidates = total;
+
+    if (int rc = upload(ctx, ctx->d_rows, rows.data(), rows.size(), "upload rows")) return rc;
+    if (int rc = upload(ctx, ctx->d_entries, entries.data(), entries.size(), "upload entries")) return rc;
+    if (int rc = upload(ctx, ctx->d_binom, binom.data(), binom.size(), "upload binomials")) return rc;
+    CU(ctx->d_etf.reserve(entries.size() * tc.lp * sizeof(int64_t)), "alloc prefix");
+    CU(ctx->d_etb.reserve(entries.size() * tc.lp * sizeof(int64_t)), "alloc prefix");
+    const size_t tab = rows.size() * (size_t)(L + 1) * (L + 1) * sizeof(int64_t);
+    CU(ctx->d_nb.reserve(tab), "alloc bucket tables");
+    CU(ctx->d_tp.reserve(tab), "alloc bucket tables");
+    launch_fill_entries(0, tc, ctx->d_rows.as<Row>(), sc.n_rows, ctx->d_entries.as<Entry>(), sc.n_entries, &ctx->launches);
+    launch_build_prefix(0, tc, ctx->raw, ctx->d_entries.as<Entry>(), sc.n_entries, ctx->d_etf.as<int64_t>(),
+                        ctx->d_etb.as<int64_t>(), &ctx->launches);
+    launch_build_bucket_tables(0, tc, ctx->raw, ctx->d_rows.as<Row>(), sc.n_rows, ctx->d_nb.as<int64_t>(),
+                               ctx->d_tp.as<int64_t>(), &ctx->launches);
+    CU(cudaGetLastError(), "set-up launch");
+    // the host copy of the rows takes the device-filled fields; this copy also waits for set-up
+    CU(cudaMemcpy(ctx->rows.data(), ctx->d_rows.p, rows.size() * sizeof(Row), cudaMemcpyDeviceToHost), "rows readback");
+    ctx->space_set = true;
+    *n_candidates = total;
+    return DISTSIM_OK;
+}
+
+int distsim_decode(distsim_ctx *ctx, int64_t index, distsim_candidate *out)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!out) return fail(ctx, DISTSIM_E_ARG, "null output");
+    if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
+    if (index < 0 || index >= ctx->sc.n_candidates) return fail(ctx, DISTSIM_E_RANGE, "candidate index out of range");
+    size_t r = 0;
+    while (r + 1 < ctx->rows.size() && ctx->rows[r + 1].offset <= index) ++r;
+    const Row &row = ctx->rows[r];
+    const int64_t local = index - row.offset;
+    const int64_t per_entry = row.n_part * row.n_sched;
+    const int64_t e = local / per_entry, rem = local % per_entry;
+    int64_t rank = rem / row.n_sched;
+    const Entry &en = ctx->entries[row.entry0 + e];
+    memset(out, 0, sizeof *out);
+    out->mp = row.mp; out->pp = row.pp; out->dp = row.dp; out->m = en.m;
+    out->sched = row.sched0 + (int32_t)(rem % row.n_sched);
+    out->micro_batch_size = en.b; out->class_index = en.cls;
+    const int L = ctx->tc.n_layers, pp = row.pp, bk = ctx->sc.binom_k;
+    out->bounds[0] = 0; out->bounds[pp] = L;
+    if (ctx->sc.partition_mode == 0) {
+        for (int j = 1; j < pp; ++j) out->bounds[j] = (int32_t)((int64_t)j * L / pp);
+    } else {
+        int c = 0;
+        for (int i = 1; i < pp; ++i) {
+            ++c;
+            while (true) {
+                const int64_t cnt = ctx->binom[(size_t)(L - 1 - c) * bk + (pp - 1 - i)];
+                if (rank < cnt) break;
+                rank -= cnt; ++c;
+            }
+            out->bounds[i] = c;
+        }
+    }
+    return DISTSIM_OK;
+}
+
+int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64_t count,
+                            int64_t *d_batch_ns, int64_t *d_stage_busy_ns)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
+    if (!d_batch_ns) return fail(ctx, DISTSIM_E_ARG, "null output");
+    if (first < 0 || count < 0 || first > ctx->sc.n_candidates || count > ctx->sc.n_candidates - first)
+        return fail(ctx, DISTSIM_E_RANGE, "candidate range outside the space");
+    if (count == 0) return DISTSIM_OK;
+    if (int rc = set_device(ctx)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const DeviceView v = ctx->view();
+    const int64_t last = first + count;
+    for (size_t r = 0; r < ctx->rows.size(); ++r) {
+        const Row &row = ctx->rows[r];
+        const int64_t lo = first > row.offset ? first - row.offset : 0;
+        const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
+        if (hi <= lo) continue;
+        launch_eval_row(s, v, (int)r, row, lo, hi, first, d_batch_ns, d_stage_busy_ns, &ctx->launches);
+    }
+    CU(cudaGetLastError(), "evaluation launch");
+    return DISTSIM_OK;
+}
+
+int distsim_argmin(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int64_t first,
+                   int64_t count, int64_t *h_best_index, int64_t *h_best_batch_ns)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
+    if (!d_batch_ns || !h_best_index || !h_best_batch_ns) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (count < 1 || first < 0) return fail(ctx, DISTSIM_E_RANGE, "empty range");
+    if (int rc = set_device(ctx)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    launch_argmin(s, d_batch_ns, count, ctx->time_bound, ctx->select_scratch(), ctx->d_result.as<int64_t>(), &ctx->launches);
+    CU(cudaGetLastError(), "argmin launch");
+    CU(cudaMemcpyAsync(ctx->h_pinned, ctx->d_result.p, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, s), "argmin readback");
+    if (int rc = read_status(ctx, s)) return rc;          // synchronises
+    *h_best_batch_ns = ctx->h_pinned[0];
+    *h_best_index = first + ctx->h_pinned[1];
+    return DISTSIM_OK;
+}
+
+int distsim_topk(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int64_t first,
+                 int64_t count, int32_t k, int64_t *d_indices, int64_t *d_times)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
+    if (!d_batch_ns || !d_indices) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (count < 1 || first < 0) return fail(ctx, DISTSIM_E_RANGE, "empty range");
+    if (k < 1 || k > 4096 || k > count) return fail(ctx, DISTSIM_E_ARG, "k must be in [1, min(count, 4096)]");
+    if (int rc = set_device(ctx)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    launch_topk(s, d_batch_ns, first, count, k, ctx->select_scratch(), d_indices, d_times, &ctx->launches);
+    CU(cudaGetLastError(), "top-k launch");
+    return DISTSIM_OK;
+}
+
+int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indices, int32_t n,
+                           distsim_record *d_records, int64_t capacity_records, int64_t *d_offsets,
+                           int64_t *d_busy_ns, double *d_util, int64_t *h_total_records)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
+    if (!d_indices || !h_total_records) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (n < 1 || n > 65535) return fail(ctx, DISTSIM_E_ARG, "n must be in [1, 65535]");
+    if (d_records && capacity_records < 0) return fail(ctx, DISTSIM_E_ARG, "negative capacity");
+    if (int rc = set_device(ctx)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CU(ctx->d_plans.reserve((size_t)n * sizeof(EmitPlan)), "alloc emission plans");
+    CU(ctx->d_op_start.reserve((size_t)n * ctx->op_words_per_cand * sizeof(int64_t)), "alloc item start times");
+    const DeviceView v = ctx->view();
+    launch_emit_plan(s, v, d_indices, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
+                     ctx->op_words_per_cand, d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), &ctx->launches);
+    CU(cudaGetLastError(), "emission planning launch");
+    CU(cudaMemcpyAsync(ctx->h_pinned, ctx->d_totals.p, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, s), "totals readback");
+    if (int rc = read_status(ctx, s)) return rc;       // synchronises
+    *h_total_records = ctx->h_pinned[0];
+    if (!d_records) return DISTSIM_OK;
+    if (ctx->h_pinned[0] > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");
+    launch_emit_records(s, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
+                        ctx->op_words_per_cand, ctx->h_pinned[1], d_records, &ctx->launches);
+    CU(cudaGetLastError(), "emission launch");
+    CU(cudaStreamSynchronize(s), "emission sync");
+    return DISTSIM_OK;
+}
+
+int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table, const distsim_space *h_space,
+                        int32_t k, int64_t *h_n_candidates, int64_t *h_best_index,
+                        int64_t *h_best_batch_ns, int64_t *h_topk_indices, int64_t *h_topk_times)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!h_n_candidates || !h_best_index || !h_best_batch_ns) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (k < 0 || (k > 0 && (!h_topk_indices || !h_topk_times))) return fail(ctx, DISTSIM_E_ARG, "bad top-k arguments");
+    if (int rc = distsim_load_event_table(ctx, h_table)) return rc;
+    int64_t n = 0;
+    if (int rc = distsim_set_space(ctx, h_space, &n)) return rc;
+    *h_n_candidates = n;
+    CU(ctx->d_batch.reserve((size_t)n * sizeof(int64_t)), "alloc batch times");
+    int64_t *d_batch = ctx->d_batch.as<int64_t>();
+    if (int rc = distsim_eval_strategies(ctx, nullptr, 0, n, d_batch, nullptr)) return rc;
+    if (k > 0) {
+        if (k > n) k = (int32_t)n;
+        if (k > 4096) k = 4096;
+        CU(ctx->d_topk.reserve((size_t)2 * k * sizeof(int64_t)), "alloc top-k");
+        int64_t *d_idx = ctx->d_topk.as<int64_t>();
+        if (int rc = distsim_topk(ctx, nullptr, d_batch, 0, n, k, d_idx, d_idx + k)) return rc;
+        CU(cudaMemcpyAsync(h_topk_indices, d_idx, (size_t)k * sizeof(int64_t), cudaMemcpyDeviceToHost, 0), "top-k readback");
+        CU(cudaMemcpyAsync(h_topk_times, d_idx + k, (size_t)k * sizeof(int64_t), cudaMemcpyDeviceToHost, 0), "top-k readback");
+    }
+    return distsim_argmin(ctx, nullptr, d_batch, 0, n, h_best_index, h_best_batch_ns);
+}
+
+}  // extern "C"

@@ -1,0 +1,393 @@
+// Timeline emission: per-device event records (kind, layer, microbatch, start_ns, end_ns) of
+// selected candidates, plus per-device activity time and utilisation.
+//
+//   emit_plan_kernel     one warp per selected candidate: decode it, run the lock-step recurrence
+//                        while recording every item's start time into scratch, count records.
+//   emit_scan_kernel     one block: exclusive scan of the per-candidate record totals.
+//   emit_devices_kernel  per (candidate, device): record offset, activity time, utilisation.
+//   emit_items_kernel    the bandwidth-bound part.  A block owns (candidate, stage, chunk of
+//                        items, chunk of replicas).  It builds the stage's forward and backward
+//                        item templates (records relative to the item's start) in shared memory
+//                        once, then each warp streams whole items: the flat int64 words of an
+//                        item are template word + {0, 0, microbatch, start, start}, written with
+//                        fully coalesced 8-byte stores to each of the stage's mp*dp replicas
+//                        (all replicas of a stage have identical lists).
+//   emit_buckets_kernel  gradient-bucket records of every stage.
+#include "recurrence.cuh"
+
+namespace distsim {
+
+namespace {
+
+constexpr int kItemThreads = 256;
+constexpr int kTileItems = 32;      // schedule items per block
+constexpr int kTileReplicas = 16;   // replicas per block
+
+__device__ __forceinline__ int find_row(const DeviceView &v, int64_t index)
+{
+    int lo = 0, hi = v.sc.n_rows - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (v.rows[mid].offset <= index) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+template <int S>
+__device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &row, int row_index,
+                                               int64_t index, EmitPlan *plan, int64_t *rec)
+{
+    const int lane = threadIdx.x & 31;
+    const int wl = row.pp / S;
+    const int seg_lane = lane % wl;
+    const bool owner = lane < wl;          // the other segments of the warp shadow the same candidate
+    const CandidateCoords cc = split_local(row, index - row.offset);
+    const Entry en = v.entries[cc.entry];
+    const int64_t *pf = v.etf + (int64_t)cc.entry * v.tc.lp;
+    const int64_t *pb = v.etb + (int64_t)cc.entry * v.tc.lp;
+    const int n_slots = 2 * (en.m + row.pp - 1);
+    const StageResult<S> R = lockstep_candidate<S, true>(v, row, en, pf, pb, cc.sched, cc.part_rank,
+                                                         seg_lane, wl, n_slots, owner ? rec : nullptr);
+    if (owner) {
+        const int L1 = v.tc.n_layers + 1;
+#pragma unroll
+        for (int k = 0; k < S; ++k) {
+            const int d = seg_lane * S + k;
+            const int a = R.a[k], e = R.e[k];
+            const int n_layers = e - a;
+            const int n_exp = v.pe[e] - v.pe[a];
+            const int64_t per_dir = (int64_t)n_layers * (row.mp > 1 ? 2 : 1) + (row.dp > 1 ? n_exp : 0);
+            const int64_t rf = per_dir + (d < row.pp - 1 ? 1 : 0);
+            const int64_t rb = per_dir + (d > 0 ? 1 : 0);
+            int64_t kb = 0;
+            if (row.dp > 1) {
+                const int64_t *nbt = v.nb + row.row_tab_off, *tpt = v.tp + row.row_tab_off;
+                kb = nbt[(int64_t)e * L1 + a] + (tpt[(int64_t)e * L1 + a] > 0 ? 1 : 0);
+            }
+            plan->bounds[d] = a;
+            if (d == row.pp - 1) plan->bounds[row.pp] = e;
+            plan->rf[d] = (int32_t)rf; plan->rb[d] = (int32_t)rb;
+            plan->n_buckets[d] = kb;
+            plan->stage_recs[d] = (int64_t)en.m * (rf + rb) + kb;
+            plan->busy[d] = R.busy[k];
+            plan->main_end[d] = R.main_end[k];
+            plan->last_b_start[d] = R.last_b_start[k];
+        }
+        if (lane == 0) {
+            plan->index = index; plan->batch_ns = R.batch;
+            plan->row = row_index; plan->entry = cc.entry; plan->m = en.m; plan->sched = cc.sched;
+            plan->pp = row.pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1;
+        }
+    }
+    __syncwarp();
+    if (lane == 0) {
+        int64_t acc = 0;
+        for (int d = 0; d < row.pp; ++d) { plan->stage_rec_prefix[d] = acc; acc += plan->stage_recs[d]; }
+        plan->stage_rec_prefix[row.pp] = acc;
+        plan->rec_total = acc * row.mp * row.dp;
+    }
+}
+
+__global__ void __launch_bounds__(128)
+emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitPlan *plans,
+                 int64_t *op_start, int64_t op_words_per_cand)
+{
+    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (i >= n) return;
+    EmitPlan *plan = plans + i;
+    const int64_t index = indices[i];
+    if (index < 0 || index >= v.sc.n_candidates) {
+        if ((threadIdx.x & 31) == 0) {
+            plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
+            plan->mp = 1; plan->dp = 1;
+            atomicCAS(v.status, 0, DISTSIM_E_RANGE);
+        }
+        return;
+    }
+    const int r = find_row(v, index);
+    const Row row = v.rows[r];
+    int64_t *rec = op_start + (int64_t)i * op_words_per_cand;
+    if (row.pp > 32) plan_candidate<2>(v, row, r, index, plan, rec);
+    else plan_candidate<1>(v, row, r, index, plan, rec);
+}
+
+// Exclusive scan of rec_total over the selections (n is small: one block, serial per chunk).
+__global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /*[2]: records, max tiles*/)
+{
+    __shared__ int64_t chunk_sum[1024];
+    const int t = threadIdx.x, nt = blockDim.x;
+    const int per = (n + nt - 1) / nt;
+    const int b = min(n, t * per), e = min(n, b + per);
+    int64_t s = 0, mt = 0;
+    for (int i = b; i < e; ++i) s += plans[i].rec_total;
+    chunk_sum[t] = s;
+    __syncthreads();
+    if (t == 0) {
+        int64_t acc = 0;
+        for (int k = 0; k < nt; ++k) { const int64_t x = chunk_sum[k]; chunk_sum[k] = acc; acc += x; }
+        totals[0] = acc;
+    }
+    __syncthreads();
+    int64_t acc = chunk_sum[t];
+    for (int i = b; i < e; ++i) {
+        plans[i].rec_base = acc; acc += plans[i].rec_total;
+        if (plans[i].ok) {
+            const int64_t reps = (int64_t)plans[i].mp * plans[i].dp;
+            const int64_t tiles = (int64_t)plans[i].pp * ((2 * plans[i].m + kTileItems - 1) / kTileItems) *
+                                  ((reps + kTileReplicas - 1) / kTileReplicas);
+            mt = max64(mt, tiles);
+        }
+    }
+    if (mt > 0) atomicMax((unsigned long long *)&totals[1], (unsigned long long)mt);
+}
+
+__global__ void __launch_bounds__(256)
+emit_devices_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int n, int64_t *offsets,
+                    int64_t *busy, double *util, const int64_t *totals)
+{
+    const int64_t N = v.tc.n_devices;
+    const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g == 0 && offsets) offsets[(int64_t)n * N] = totals[0];
+    if (g >= (int64_t)n * N) return;
+    const int i = (int)(g / N);
+    const int k = (int)(g - (int64_t)i * N);
+    const EmitPlan &p = plans[i];
+    if (!p.ok) {
+        if (offsets) offsets[g] = p.rec_base;
+        if (busy) busy[g] = 0;
+        if (util) util[g] = 0.0;
+        return;
+    }
+    const int q = k % p.mp, d = (k / p.mp) % p.pp, r = k / (p.mp * p.pp);
+    if (offsets)
+        offsets[g] = p.rec_base + (int64_t)r * p.mp * p.stage_rec_prefix[p.pp] +
+                     (int64_t)p.mp * p.stage_rec_prefix[d] + (int64_t)q * p.stage_recs[d];
+    if (busy) busy[g] = p.busy[d];
+    if (util) util[g] = p.batch_ns > 0 ? (double)p.busy[d] / (double)p.batch_ns : 0.0;
+}
+
+// Position `s` in stage d's schedule order -> (is backward, micro-batch, items of each kind before it).
+__device__ __forceinline__ void item_at(int sched, int pp, int m, int d, int s, bool &bwd, int &j, int &nf, int &nb)
+{
+    if (sched == 0) {
+        if (s < m) { bwd = false; j = s; nf = s; nb = 0; }
+        else { bwd = true; j = s - m; nf = m; nb = s - m; }
+        return;
+    }
+    const int w = min(pp - d, m);
+    if (s < w) { bwd = false; j = s; nf = s; nb = 0; }
+    else if (s < 2 * m - w) {
+        const int t = s - w;
+        if (!(t & 1)) { bwd = true; j = t >> 1; nf = w + (t >> 1); nb = t >> 1; }
+        else { bwd = false; j = w + (t >> 1); nf = w + (t >> 1); nb = (t >> 1) + 1; }
+    } else { bwd = true; j = s - m; nf = m; nb = s - m; }
+}
+
+__global__ void __launch_bounds__(kItemThreads)
+emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_t *__restrict__ op_start,
+                  int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */)
+{
+    extern __shared__ __align__(16) int64_t tmpl[];     // [rf*5] forward, then [rb*5] backward
+    const int i = blockIdx.y;
+    const EmitPlan &p = plans[i];
+    if (!p.ok) return;
+    const int m = p.m, pp = p.pp;
+    const int reps = p.mp * p.dp;
+    const int item_chunks = (2 * m + kTileItems - 1) / kTileItems;
+    const int rep_chunks = (reps + kTileReplicas - 1) / kTileReplicas;
+    int tile = blockIdx.x;
+    if (tile >= pp * item_chunks * rep_chunks) return;
+    const int rc = tile % rep_chunks; tile /= rep_chunks;
+    const int ic = tile % item_chunks;
+    const int d = tile / item_chunks;
+
+    const Row row = v.rows[p.row];
+    const Entry en = v.entries[p.entry];
+    const int a = p.bounds[d], e = p.bounds[d + 1];
+    const int rf = p.rf[d], rb = p.rb[d];
+    const int64_t *pf = v.etf + (int64_t)p.entry * v.tc.lp;
+    const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
+    const int64_t *f = v.raw.fwd + (int64_t)en.cls * v.tc.n_layers;
+    const int64_t *g = v.raw.bwd + (int64_t)en.cls * v.tc.n_layers;
+    const int per_layer = row.mp > 1 ? 2 : 1;
+    int64_t *tf = tmpl, *tb = tmpl + (int64_t)rf * 5;
+
+    // ---- item templates: records relative to the item's start --------------------------
+    for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
+        const bool ex = row.dp > 1 && v.raw.expert[l];
+        {   // forward: layers ascending
+            const int r = (l - a) * per_layer + (row.dp > 1 ? v.pe[l] - v.pe[a] : 0);
+            int64_t t = pf[l] - pf[a];
+            int64_t *w = tf + (int64_t)r * 5;
+            w[0] = DISTSIM_COMPUTE_F; w[1] = l; w[2] = 0; w[3] = t; t += f[l]; w[4] = t; w += 5;
+            if (row.mp > 1) { w[0] = DISTSIM_MP_AR_F; w[1] = l; w[2] = 0; w[3] = t; t += en.ar; w[4] = t; w += 5; }
+            if (ex) { w[0] = DISTSIM_A2A_F; w[1] = l; w[2] = 0; w[3] = t; t += en.a2a; w[4] = t; }
+        }
+        {   // backward: layers descending
+            const int r = (e - 1 - l) * per_layer + (row.dp > 1 ? v.pe[e] - v.pe[l + 1] : 0);
+            int64_t t = pb[e] - pb[l + 1];
+            int64_t *w = tb + (int64_t)r * 5;
+            w[0] = DISTSIM_COMPUTE_B; w[1] = l; w[2] = 0; w[3] = t; t += g[l]; w[4] = t; w += 5;
+            if (row.mp > 1) { w[0] = DISTSIM_MP_AR_B; w[1] = l; w[2] = 0; w[3] = t; t += en.ar; w[4] = t; w += 5; }
+            if (ex) { w[0] = DISTSIM_A2A_B; w[1] = l; w[2] = 0; w[3] = t; t += en.a2a; w[4] = t; }
+        }
+    }
+    if (threadIdx.x == 0) {
+        if (d < pp - 1) {
+            int64_t *w = tf + (int64_t)(rf - 1) * 5;
+            const int64_t t = pf[e] - pf[a];
+            w[0] = DISTSIM_SEND_F; w[1] = e - 1; w[2] = 0; w[3] = t; w[4] = t + p2p_cost(row, en, d);
+        }
+        if (d > 0) {
+            int64_t *w = tb + (int64_t)(rb - 1) * 5;
+            const int64_t t = pb[e] - pb[a];
+            w[0] = DISTSIM_SEND_B; w[1] = a; w[2] = 0; w[3] = t; w[4] = t + p2p_cost(row, en, d - 1);
+        }
+    }
+    __syncthreads();
+
+    // ---- stream the items of this tile -------------------------------------------------
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int s_end = min(2 * m, (ic + 1) * kTileItems);
+    const int rep0 = rc * kTileReplicas, rep1 = min(reps, rep0 + kTileReplicas);
+    const int64_t stage_words = p.stage_recs[d] * 5;                    // one device of this stage
+    const int64_t replica_words = (int64_t)p.mp * p.stage_rec_prefix[pp] * 5;   // one whole replica r
+    const int64_t stage_base = (p.rec_base + (int64_t)p.mp * p.stage_rec_prefix[d]) * 5;
+    const int64_t *starts = op_start + (int64_t)i * op_words_per_cand + (int64_t)d * 2 * m;
+    for (int s = ic * kTileItems + warp; s < s_end; s += n_warps) {
+        bool bwd; int j, nf, nb;
+        item_at(p.sched, pp, m, d, s, bwd, j, nf, nb);
+        const int64_t t0 = starts[s];
+        const int64_t *src = bwd ? tb : tf;
+        const int n_words = (bwd ? rb : rf) * 5;
+        const int64_t item_off = ((int64_t)nf * rf + (int64_t)nb * rb) * 5;
+        int field = lane % 5;
+        for (int w = lane; w < n_words; w += 32) {
+            int64_t val = src[w];
+            val += field == 2 ? (int64_t)j : (field >= 3 ? t0 : 0);
+            field += 2; if (field >= 5) field -= 5;                      // (w + 32) mod 5
+            for (int rep = rep0; rep < rep1; ++rep) {
+                const int r = rep / p.mp, q = rep - r * p.mp;
+                out[stage_base + (int64_t)r * replica_words + (int64_t)q * stage_words + item_off + w] = val;
+            }
+        }
+    }
+}
+
+// Gradient-bucket records of stage blockIdx.x of selection blockIdx.y.  Buckets whose last byte
+// lies in the same layer share a ready time, so once the first of them has started the rest
+// follow back to back: per layer one serial step, inside a layer a closed form.
+__global__ void __launch_bounds__(256)
+emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *__restrict__ out)
+{
+    __shared__ int64_t g_start[DISTSIM_MAX_LAYERS + 1];   // start of the first bucket ending in layer a+i
+    __shared__ int64_t g_first[DISTSIM_MAX_LAYERS + 1];   // number of that bucket
+    __shared__ int64_t part_start;
+    const int i = blockIdx.y, d = blockIdx.x;
+    const EmitPlan &p = plans[i];
+    if (!p.ok || d >= p.pp || p.dp == 1) return;
+    const int64_t kb = p.n_buckets[d];
+    if (kb == 0) return;
+    const Row row = v.rows[p.row];
+    const int a = p.bounds[d], e = p.bounds[d + 1];
+    const int L1 = v.tc.n_layers + 1;
+    const int64_t *nbe = v.nb + row.row_tab_off + (int64_t)e * L1;
+    const int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
+    const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
+    const int64_t n_full = nbe[a];
+    if (threadIdx.x == 0) {
+        int64_t end = 0, nb_prev = 0;
+        const int64_t tbs = p.last_b_start[d], main_end = p.main_end[d];
+        for (int l = e - 1; l >= a; --l) {
+            const int64_t nb_l = nbe[l], n_l = nb_l - nb_prev;
+            const int64_t ready = v.tc.overlap ? tbs + (pb[e] - pb[l]) : main_end;
+            g_first[l - a] = nb_prev;
+            g_start[l - a] = max64(end, ready);
+            if (n_l > 0) end = g_start[l - a] + n_l * row.t_full;
+            nb_prev = nb_l;
+        }
+        if (part > 0) {
+            const int ls = v.next_grad[a];
+            const int64_t ready = v.tc.overlap ? tbs + (pb[e] - pb[ls]) : main_end;
+            part_start = max64(end, ready);
+        }
+    }
+    __syncthreads();
+    const int reps = p.mp * p.dp;
+    const int rep_chunks = gridDim.z;
+    const int per = (reps + rep_chunks - 1) / rep_chunks;
+    const int rep0 = blockIdx.z * per, rep1 = min(reps, rep0 + per);
+    const int64_t stage_words = p.stage_recs[d] * 5;
+    const int64_t replica_words = (int64_t)p.mp * p.stage_rec_prefix[p.pp] * 5;
+    const int64_t base = (p.rec_base + (int64_t)p.mp * p.stage_rec_prefix[d]) * 5 +
+                         (int64_t)p.m * (p.rf[d] + p.rb[d]) * 5;
+    for (int64_t w = threadIdx.x; w < kb * 5; w += blockDim.x) {
+        const int64_t k = w / 5;
+        const int field = (int)(w - k * 5);
+        int64_t val;
+        if (field == 0) val = DISTSIM_DP_AR;
+        else if (field == 1) val = k;
+        else if (field == 2) val = -1;
+        else {
+            int64_t start, dur;
+            if (k >= n_full) { start = part_start; dur = part; }
+            else {
+                // the layer whose group holds bucket k: the largest l with nb[e][l] > k
+                // (nb[e][l] grows as l decreases, and nb[e][a] = n_full > k)
+                int lo = a, hi = e - 1;
+                while (lo < hi) {
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (nbe[mid] > k) lo = mid; else hi = mid - 1;
+                }
+                start = g_start[lo - a] + (k - g_first[lo - a]) * row.t_full;
+                dur = row.t_full;
+            }
+            val = field == 3 ? start : start + dur;
+        }
+        for (int rep = rep0; rep < rep1; ++rep) {
+            const int r = rep / p.mp, q = rep - r * p.mp;
+            out[base + (int64_t)r * replica_words + (int64_t)q * stage_words + w] = val;
+        }
+    }
+}
+
+}  // namespace
+
+void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
+                      EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand,
+                      int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
+                      int64_t *launches)
+{
+    cudaMemsetAsync(d_totals, 0, 2 * sizeof(int64_t), s);
+    emit_plan_kernel<<<(n + 3) / 4, 128, 0, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand);
+    emit_scan_kernel<<<1, 1024, 0, s>>>(plans, n, d_totals);
+    *launches += 2;
+    if (offsets || busy || util) {
+        const int64_t total = (int64_t)n * v.tc.n_devices + 1;
+        emit_devices_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(v, plans, n, offsets, busy, util, d_totals);
+        ++*launches;
+    }
+}
+
+void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
+                         const int64_t *op_start, int64_t op_words_per_cand, int64_t max_tiles,
+                         distsim_record *records, int64_t *launches)
+{
+    if (n == 0 || max_tiles == 0) return;
+    const size_t smem = (size_t)(2 * (3 * v.tc.n_layers + 1)) * 5 * sizeof(int64_t);
+    static size_t smem_set = 0;
+    if (smem > 48 * 1024 && smem > smem_set) {
+        cudaFuncSetAttribute(emit_items_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        smem_set = smem;
+    }
+    int64_t *out = reinterpret_cast<int64_t *>(records);
+    emit_items_kernel<<<dim3((unsigned)max_tiles, (unsigned)n), kItemThreads, smem, s>>>(
+        v, plans, op_start, op_words_per_cand, out);
+    ++*launches;
+    if (v.tc.n_devices > 1) {
+        emit_buckets_kernel<<<dim3((unsigned)v.sc.pp_max, (unsigned)n, 4), 256, 0, s>>>(v, plans, out);
+        ++*launches;
+    }
+}
+
+}  // namespace distsim

@@ -1,0 +1,150 @@
+// Internal declarations shared by the engine's translation units (not part of the C ABI).
+//
+// Device-resident data (all built by kernels in setup_kernels.cu from the raw event table):
+//
+//   Row      one per valid (mp, pp) pair, in canonical order.  A row owns a contiguous block of
+//            candidate indices: (entry, partition, schedule) with the schedule fastest.
+//   Entry    one per valid micro-batch count m of a row: m, micro-batch size b, event class and
+//            the communication-event costs that depend on (dp, b).
+//   ETF/ETB  per entry, exclusive prefix sums over layers of the layer composites
+//              phi(l)   = fwd(l) + AR + [expert l] * A2A      (MP modeling, paper Sec. 4.3)
+//              gamma(l) = bwd(l) + AR + [expert l] * A2A
+//            so that any contiguous stage's item cost is one subtraction.  Row stride `lp` is
+//            n_layers + 1 rounded up to an even count, which keeps every row 16-byte aligned for
+//            bulk copies into shared memory.
+//   NB/TP    per row, [e][l] tables for the gradient buckets of a stage that ends at layer e:
+//            NB = number of full buckets completed once layers e-1..l have produced their
+//            gradients; TP = cost of the trailing partial bucket of the stage [l, e).
+//   binom    C(n, k), saturated at 2^62, for unranking stage partitions.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/distsim.h"
+
+namespace distsim {
+
+constexpr int64_t kSat = (int64_t)1 << 62;
+
+struct TableConst {
+    int32_t n_layers, n_classes, n_devices, gpus_per_node;
+    int64_t global_batch, seq, hidden;
+    int64_t alpha_intra, beta_intra, alpha_inter, beta_inter;
+    int64_t bucket;       // dp_bucket_bytes
+    int32_t overlap;
+    int32_t elem_bytes;
+    int32_t lp;           // padded prefix-row length (int64 words)
+    int32_t pad;
+};
+
+struct Row {
+    int64_t offset;       // first candidate index of the row
+    int64_t n_part;       // stage partitions per entry
+    int64_t size;         // n_entries * n_part * n_sched
+    int64_t t_full;       // cost of one full gradient bucket (0 if dp == 1)   [device-filled]
+    int64_t row_tab_off;  // offset (words) of this row's NB / TP tables
+    int32_t mp, pp, dp, log2_mp;
+    int32_t n_entries, entry0;
+    int32_t n_sched, sched0;
+    int32_t p2p_period;   // boundary d|d+1 is inter-node iff ((d+1) & (p2p_period-1)) == 0
+    int32_t pad;
+};
+
+struct Entry {
+    int32_t m, b, cls, row;
+    int64_t p2p_intra, p2p_inter, a2a, ar;   // [device-filled]
+};
+
+struct SpaceConst {
+    int32_t n_rows, n_entries, pp_max, partition_mode;   // partition_mode 0 balanced, 1 all
+    int32_t binom_k;      // second dimension of binom
+    int32_t pad;
+    int64_t n_candidates;
+};
+
+// Raw table on the device (inputs of the set-up kernels; the emission kernels read the
+// per-class layer times from it as well).
+struct RawTable {
+    const int32_t *class_mp, *class_b;
+    const int64_t *fwd, *bwd;        // [n_classes][n_layers]
+    const uint8_t *expert;           // [n_layers]
+    const int64_t *grad;             // [n_layers]
+};
+
+// Everything a kernel needs, passed by value.
+struct DeviceView {
+    TableConst tc;
+    SpaceConst sc;
+    RawTable raw;
+    const Row *rows;
+    const Entry *entries;
+    const int64_t *etf, *etb;        // [n_entries][lp]
+    const int64_t *nb, *tp;          // per row [L+1][L+1]
+    const int64_t *binom;            // [n_layers][binom_k]
+    const int32_t *next_grad;        // [L+1] smallest l' >= l with grad_bytes[l'] > 0 (L if none)
+    const int32_t *pe;               // [L+1] number of expert layers before layer l
+    int32_t *status;                 // device status word: 0 ok, else first error code
+};
+
+// ---- set-up kernels (setup_kernels.cu) -------------------------------------------------
+void launch_fill_entries(cudaStream_t s, const TableConst &tc, Row *rows, int n_rows,
+                         Entry *entries, int n_entries, int64_t *launches);
+void launch_build_prefix(cudaStream_t s, const TableConst &tc, const RawTable &raw,
+                         const Entry *entries, int n_entries, int64_t *etf, int64_t *etb,
+                         int64_t *launches);
+void launch_build_bucket_tables(cudaStream_t s, const TableConst &tc, const RawTable &raw,
+                                const Row *rows, int n_rows, int64_t *nb, int64_t *tp,
+                                int64_t *launches);
+void launch_build_layer_tables(cudaStream_t s, const TableConst &tc, const RawTable &raw,
+                               int32_t *next_grad, int32_t *pe, int64_t *launches);
+
+// ---- evaluation (eval_kernels.cu) ------------------------------------------------------
+// Evaluates candidates [lo, hi) of row `row_index` (indices local to the row); results go to
+// batch_out[row.offset + local - first] and, if non-null, busy_out[(same) * pp_max + d].
+void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const Row &row_host,
+                     int64_t lo, int64_t hi, int64_t first, int64_t *batch_out, int64_t *busy_out,
+                     int64_t *launches);
+
+// ---- selection (select_kernels.cu) -----------------------------------------------------
+struct SelectScratch {
+    unsigned long long *key;        // [2] packed / two-pass argmin keys
+    unsigned long long *hist;       // [256] radix histogram
+    unsigned long long *sel_state;  // [8] radix-select state
+    int64_t *cand_time, *cand_idx;  // [4096] selected pairs before sorting
+};
+// d_result[0] = smallest time, d_result[1] = its smallest position in `batch`.
+void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t time_bound,
+                   const SelectScratch &sc, int64_t *d_result, int64_t *launches);
+void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
+                 const SelectScratch &sc, int64_t *d_indices, int64_t *d_times, int64_t *launches);
+
+// ---- emission (emit_kernels.cu) --------------------------------------------------------
+struct EmitPlan {                    // per selected candidate, written by the planning kernel
+    int64_t index;
+    int64_t batch_ns;
+    int64_t rec_base;                // first record of the selection (after the scan)
+    int64_t rec_total;               // records of all its devices
+    int32_t row, entry, m, sched, pp, mp, dp, ok;
+    int32_t bounds[DISTSIM_MAX_PP + 1];
+    int32_t pad;
+    int32_t rf[DISTSIM_MAX_PP], rb[DISTSIM_MAX_PP];   // records of one forward / backward item
+    int64_t n_buckets[DISTSIM_MAX_PP];
+    int64_t stage_recs[DISTSIM_MAX_PP];               // records of one device of stage d
+    int64_t stage_rec_prefix[DISTSIM_MAX_PP + 1];
+    int64_t busy[DISTSIM_MAX_PP];
+    int64_t main_end[DISTSIM_MAX_PP];
+    int64_t last_b_start[DISTSIM_MAX_PP];
+};
+// Plans the n selections: item start times into op_start (op_words_per_cand words each), record
+// counts, offsets / busy / util (each nullable); d_totals[0] = records, d_totals[1] = largest
+// number of item tiles of any selection.
+void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
+                      EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand,
+                      int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
+                      int64_t *launches);
+void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
+                         const int64_t *op_start, int64_t op_words_per_cand, int64_t max_tiles,
+                         distsim_record *records, int64_t *launches);
+
+}  // namespace distsim

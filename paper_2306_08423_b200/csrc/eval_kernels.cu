@@ -1,0 +1,107 @@
+// Evaluation kernels: batch time (and optionally per-stage activity time) of a range of
+// candidates of one row.
+//
+// eval_lockstep_kernel: a segment of pp/S consecutive lanes evaluates one candidate, lane =
+// stage (S = 2 stages per lane when pp = 64), 32/(pp/S) candidates per warp, all segments of a
+// warp advancing through the slots of the lock-step recurrence together.  The prefix rows of
+// the entries a block touches are staged into shared memory with one bulk copy per table
+// (cp.async.bulk, completion on the block's own mbarrier, no multicast).
+#include "recurrence.cuh"
+#include "smem_stage.cuh"
+
+namespace distsim {
+
+namespace {
+
+constexpr int kEvalThreads = 256;
+
+template <int S>
+__global__ void __launch_bounds__(kEvalThreads)
+eval_lockstep_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t first,
+                     int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out,
+                     int max_stage_entries)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bar;
+    const Row row = v.rows[row_index];
+    const int pp = row.pp;
+    const int wl = pp / S;                         // lanes per candidate
+    const int cpw = 32 / wl;                       // candidates per warp
+    const int warps = blockDim.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t cta_first = lo + (int64_t)blockIdx.x * warps * cpw;
+    if (cta_first >= hi) return;
+    const int64_t cta_last = min(hi, cta_first + (int64_t)warps * cpw) - 1;
+
+    // ---- stage the prefix rows of the entries this block touches -----------------------
+    const int e_lo = split_local(row, cta_first).entry;
+    const int e_hi = split_local(row, cta_last).entry;
+    const int n_stage = e_hi - e_lo + 1;
+    const int lp = v.tc.lp;
+    int64_t *sm_f = reinterpret_cast<int64_t *>(smem_raw);
+    int64_t *sm_b = sm_f + (int64_t)max_stage_entries * lp;
+    bool staged = false;
+    if (max_stage_entries > 0 && n_stage <= max_stage_entries) {
+        const uint32_t bytes = (uint32_t)(n_stage * lp * sizeof(int64_t));
+        staged = stage_two_tables(&bar, sm_f, v.etf + (int64_t)e_lo * lp, sm_b,
+                                  v.etb + (int64_t)e_lo * lp, bytes, v.status);
+    }
+
+    const int seg = lane / wl, seg_lane = lane - seg * wl;
+    int64_t local = cta_first + (int64_t)warp * cpw + seg;
+    const bool valid = local < hi;
+    if (!valid) local = hi - 1;                    // idle segments shadow a real candidate
+    const CandidateCoords cc = split_local(row, local);
+    const Entry en = v.entries[cc.entry];
+    const int64_t *pf = staged ? sm_f + (int64_t)(cc.entry - e_lo) * lp : v.etf + (int64_t)cc.entry * lp;
+    const int64_t *pb = staged ? sm_b + (int64_t)(cc.entry - e_lo) * lp : v.etb + (int64_t)cc.entry * lp;
+
+    int n_slots = 2 * (en.m + pp - 1);
+    n_slots = __reduce_max_sync(0xffffffffu, n_slots);
+
+    const StageResult<S> R = lockstep_candidate<S, false>(v, row, en, pf, pb, cc.sched, cc.part_rank,
+                                                          seg_lane, wl, n_slots, nullptr);
+    if (!valid) return;
+    const int64_t out = row.offset + local - first;
+    if (seg_lane == 0) batch_out[out] = R.batch;
+    if (busy_out) {
+        int64_t *bo = busy_out + out * v.sc.pp_max;
+#pragma unroll
+        for (int k = 0; k < S; ++k) bo[seg_lane * S + k] = R.busy[k];
+        for (int d = pp + seg_lane; d < v.sc.pp_max; d += wl) bo[d] = 0;
+    }
+}
+
+}  // namespace
+
+void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const Row &row,
+                     int64_t lo, int64_t hi, int64_t first, int64_t *batch_out, int64_t *busy_out,
+                     int64_t *launches)
+{
+    if (hi <= lo) return;
+    const int S = row.pp > 32 ? 2 : 1;
+    const int wl = row.pp / S;
+    const int cpb = (kEvalThreads / 32) * (32 / wl);      // candidates per block
+    const int64_t blocks = (hi - lo + cpb - 1) / cpb;
+    // entries a block can touch: its candidates span at most this many entries
+    const int64_t per_entry = row.n_part * row.n_sched;
+    int64_t span = (cpb + per_entry - 1) / per_entry + 1;
+    if (span > row.n_entries) span = row.n_entries;
+    int max_stage = (int)span;
+    size_t smem = (size_t)max_stage * v.tc.lp * sizeof(int64_t) * 2;
+    if (smem > 96 * 1024) { max_stage = 0; smem = 0; }   // too wide: read the rows from global
+    if (S == 1) {
+        if (smem > 48 * 1024)
+            cudaFuncSetAttribute(eval_lockstep_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_lockstep_kernel<1><<<(unsigned)blocks, kEvalThreads, smem, s>>>(v, row_index, lo, hi, first,
+                                                                           batch_out, busy_out, max_stage);
+    } else {
+        if (smem > 48 * 1024)
+            cudaFuncSetAttribute(eval_lockstep_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_lockstep_kernel<2><<<(unsigned)blocks, kEvalThreads, smem, s>>>(v, row_index, lo, hi, first,
+                                                                           batch_out, busy_out, max_stage);
+    }
+    ++*launches;
+}
+
+}  // namespace distsim

@@ -1,0 +1,236 @@
+// Device code shared by the evaluation and the emission-planning kernels: candidate decoding
+// and the lock-step form of the pipeline recurrence.
+//
+// Pipeline recurrence (Algorithm 1 of the paper): a schedule item (forward or backward pass of
+// one micro-batch on one stage) starts at the later of (a) the end of the item it takes its
+// input from on the neighbouring stage, including that item's trailing transfer event, and
+// (b) the end of the previous item on its own device.  Because every micro-batch of a stage
+// costs the same, an item is described by its stage's forward cost `fop` or backward cost `bop`.
+//
+// Lock-step form.  Give every item a unit-time "slot" s; then in both schedules
+//   GPipe : F(d,j) runs in slot d + j,              B(d,j) in slot (m + 2pp - 2 - d) + j
+//   1F1B  : F(d,j) runs in slot d + j  (j <  w_d),  B(d,j) in slot (2pp - 1 - d) + 2j
+//           F(d,j) runs in slot d + 2j (j >= w_d),  with w_d = min(pp - d, m)
+// all items finish within 2(m + pp - 1) slots, a stage runs at most one item per slot in its
+// schedule's order, and when an item runs, the *most recent* forward (backward) item finished
+// by the previous (next) stage before this slot is exactly the one it depends on.  So a lane
+// that owns a stage keeps only `last_f` and `last_b` (end of its latest forward / backward
+// item) and `free_at`; per slot it fetches the neighbour's value with one shuffle each way.
+#pragma once
+
+#include "engine.h"
+
+namespace distsim {
+
+__device__ __forceinline__ int64_t max64(int64_t a, int64_t b) { return a > b ? a : b; }
+
+// Bounds c_{d0} .. c_{d0+S} of partition number `part_rank` of the row's partitions.
+// Balanced mode: c_j = floor(j L / pp).  All-compositions mode: the (pp-1)-subsets of
+// {1..L-1} in lexicographic order, decoded with the combinatorial number system: position i
+// takes the smallest value c whose block of C(L-1-c, pp-1-i) completions contains the rank.
+template <int S>
+__device__ __forceinline__ void partition_bounds(const DeviceView &v, int pp, int64_t part_rank,
+                                                 int d0, int (&out)[S + 1])
+{
+    const int L = v.tc.n_layers;
+    if (v.sc.partition_mode == 0) {
+#pragma unroll
+        for (int k = 0; k <= S; ++k) out[k] = (int)((int64_t)(d0 + k) * L / pp);
+        return;
+    }
+#pragma unroll
+    for (int k = 0; k <= S; ++k) out[k] = (d0 + k == 0) ? 0 : L;
+    int64_t r = part_rank;
+    int c = 0;
+    const int last = min(pp - 1, d0 + S);
+    for (int i = 1; i <= last; ++i) {
+        ++c;
+        const int kk = pp - 1 - i;
+        while (true) {
+            const int64_t cnt = __ldg(&v.binom[(int64_t)(L - 1 - c) * v.sc.binom_k + kk]);
+            if (r < cnt) break;
+            r -= cnt;
+            ++c;
+        }
+#pragma unroll
+        for (int k = 0; k <= S; ++k) if (i == d0 + k) out[k] = c;
+    }
+}
+
+struct CandidateCoords {
+    int entry;           // global entry index
+    int sched;           // 0 GPipe, 1 1F1B
+    int64_t part_rank;
+};
+
+// Row-local index -> (entry, partition, schedule); the schedule varies fastest.
+__device__ __forceinline__ CandidateCoords split_local(const Row &row, int64_t local)
+{
+    CandidateCoords cc;
+    if (row.size < ((int64_t)1 << 32)) {
+        const uint32_t l32 = (uint32_t)local;
+        const uint32_t per_entry = (uint32_t)(row.n_part * row.n_sched);
+        const uint32_t e = l32 / per_entry;
+        const uint32_t rem = l32 - e * per_entry;
+        cc.entry = row.entry0 + (int)e;
+        cc.part_rank = rem / (uint32_t)row.n_sched;
+        cc.sched = row.sched0 + (int)(rem - (uint32_t)cc.part_rank * (uint32_t)row.n_sched);
+    } else {
+        const int64_t per_entry = row.n_part * row.n_sched;
+        const int64_t e = local / per_entry;
+        const int64_t rem = local - e * per_entry;
+        cc.entry = row.entry0 + (int)e;
+        cc.part_rank = rem / row.n_sched;
+        cc.sched = row.sched0 + (int)(rem - cc.part_rank * row.n_sched);
+    }
+    return cc;
+}
+
+// Does stage d run a forward / backward item in slot s?
+__device__ __forceinline__ void slot_activity(int sched, int pp, int m, int d, int s, bool &do_f, bool &do_b)
+{
+    const int x = s - d;
+    if (sched == 0) {
+        do_f = x >= 0 && x < m;
+        const int y = s - (m + 2 * pp - 2 - d);
+        do_b = y >= 0 && y < m;
+    } else {
+        const int w = min(pp - d, m);
+        do_f = (x >= 0 && x < w) || (x >= 2 * w && !(x & 1) && (x >> 1) < m);
+        const int y = s - (2 * pp - 1 - d);
+        do_b = y >= 0 && !(y & 1) && (y >> 1) < m;
+    }
+}
+
+// Gradient all-reduce buckets of one stage [a, e) on the communication lane (DP modeling).
+// `tb` is the start of the stage's last backward item, `main_end` the end of the main lane.
+// pb: the entry's backward prefix row; nbt/tpt: the row's bucket tables.  Returns the end of the
+// last bucket (main_end when the stage sends no gradients).
+__device__ __forceinline__ int64_t bucket_lane_end(const DeviceView &v, const Row &row,
+                                                   const int64_t *pb, const int64_t *nbt,
+                                                   const int64_t *tpt, int a, int e, int64_t tb,
+                                                   int64_t main_end)
+{
+    if (row.dp == 1) return main_end;
+    const int L1 = v.tc.n_layers + 1;
+    const int64_t *nbe = nbt + (int64_t)e * L1;
+    const int64_t part = __ldg(&tpt[(int64_t)e * L1 + a]);
+    if (!v.tc.overlap) {
+        const int64_t full = __ldg(&nbe[a]);
+        if (full == 0 && part == 0) return main_end;
+        return main_end + full * row.t_full + part;
+    }
+    // a bucket is ready when the layer holding its last byte has finished its backward
+    // composite in the last backward item; buckets then run back to back
+    int64_t end = 0;
+    bool any = false;
+    const int64_t pbe = pb[e];
+    if (v.tc.bucket > 0) {
+        int64_t nb_prev = 0;                   // nb[e][l+1]
+        for (int l = e - 1; l >= a; --l) {
+            const int64_t nb_l = __ldg(&nbe[l]);
+            const int64_t n_l = nb_l - nb_prev; // full buckets whose last byte lies in layer l
+            if (n_l > 0) { end = max64(end, tb + (pbe - pb[l])) + n_l * row.t_full; any = true; }
+            nb_prev = nb_l;
+        }
+    }
+    if (part > 0) {
+        // the trailing bucket ends in the stage's first layer that has any gradient bytes
+        const int lstar = __ldg(&v.next_grad[a]);
+        end = max64(end, tb + (pbe - pb[lstar])) + part;
+        any = true;
+    }
+    return any ? end : main_end;
+}
+
+// Result of one candidate on the lanes that own its stages (S stages per lane).
+template <int S>
+struct StageResult {
+    int a[S], e[S];              // layer range [a, e) of each owned stage
+    int64_t fop[S], bop[S];      // cost of a forward / backward item incl. trailing transfer
+    int64_t main_end[S];         // end of the stage's last item
+    int64_t last_b_start[S];     // start of the stage's last backward item
+    int64_t dp_end[S];           // end of the gradient-bucket lane
+    int64_t busy[S];             // activity time of a device of the stage
+    int64_t batch;               // max over all stages (same on every lane of the segment)
+};
+
+// Cost of the transfer across boundary d | d+1 for this entry.
+__device__ __forceinline__ int64_t p2p_cost(const Row &row, const Entry &en, int d)
+{
+    return (((d + 1) & (row.p2p_period - 1)) == 0) ? en.p2p_inter : en.p2p_intra;
+}
+
+// Lock-step evaluation of one candidate by `wl` consecutive lanes (wl * S == pp), every lane of
+// the warp calling this together (lanes of other segments work on their own candidates).
+//   seg_lane   lane index inside the segment;  n_slots_warp: loop bound, uniform over the warp
+//   pf, pb     the entry's forward / backward prefix rows (shared or global memory)
+//   rec        if kRecord and non-null: item start times go to rec[d * 2m + position in stage order]
+template <int S, bool kRecord>
+__device__ __forceinline__ StageResult<S> lockstep_candidate(
+    const DeviceView &v, const Row &row, const Entry &en, const int64_t *pf, const int64_t *pb,
+    int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec)
+{
+    StageResult<S> R;
+    const int pp = row.pp, m = en.m;
+    const int d0 = seg_lane * S;
+    int bounds[S + 1];
+    partition_bounds<S>(v, pp, part_rank, d0, bounds);
+#pragma unroll
+    for (int k = 0; k < S; ++k) {
+        const int d = d0 + k;
+        R.a[k] = bounds[k]; R.e[k] = bounds[k + 1];
+        R.fop[k] = pf[R.e[k]] - pf[R.a[k]] + (d < pp - 1 ? p2p_cost(row, en, d) : 0);
+        R.bop[k] = pb[R.e[k]] - pb[R.a[k]] + (d > 0 ? p2p_cost(row, en, d - 1) : 0);
+        R.last_b_start[k] = 0;
+    }
+    int64_t last_f[S], last_b[S], free_at[S];
+    int n_done[S];
+#pragma unroll
+    for (int k = 0; k < S; ++k) { last_f[k] = 0; last_b[k] = 0; free_at[k] = 0; n_done[k] = 0; }
+
+    for (int s = 0; s < n_slots_warp; ++s) {
+        const int64_t up_f = __shfl_up_sync(0xffffffffu, last_f[S - 1], 1, wl);
+        const int64_t dn_b = __shfl_down_sync(0xffffffffu, last_b[0], 1, wl);
+        int64_t old_f[S], old_b[S];
+#pragma unroll
+        for (int k = 0; k < S; ++k) { old_f[k] = last_f[k]; old_b[k] = last_b[k]; }
+#pragma unroll
+        for (int k = 0; k < S; ++k) {
+            const int d = d0 + k;
+            bool do_f, do_b;
+            slot_activity(sched, pp, m, d, s, do_f, do_b);
+            if (do_f) {
+                const int64_t dep = (k == 0) ? (seg_lane == 0 ? 0 : up_f) : old_f[k > 0 ? k - 1 : 0];
+                const int64_t st = max64(dep, free_at[k]);
+                if (kRecord && rec) rec[(int64_t)d * 2 * m + n_done[k]] = st;
+                last_f[k] = free_at[k] = st + R.fop[k];
+                ++n_done[k];
+            } else if (do_b) {
+                const int64_t dep = (k == S - 1) ? (seg_lane == wl - 1 ? 0 : dn_b) : old_b[k < S - 1 ? k + 1 : 0];
+                const int64_t st = max64(dep, free_at[k]);
+                if (kRecord && rec) rec[(int64_t)d * 2 * m + n_done[k]] = st;
+                R.last_b_start[k] = st;
+                last_b[k] = free_at[k] = st + R.bop[k];
+                ++n_done[k];
+            }
+        }
+    }
+
+    const int64_t *nbt = v.nb + row.row_tab_off;
+    const int64_t *tpt = v.tp + row.row_tab_off;
+    int64_t mx = 0;
+#pragma unroll
+    for (int k = 0; k < S; ++k) {
+        R.main_end[k] = free_at[k];
+        R.dp_end[k] = bucket_lane_end(v, row, pb, nbt, tpt, R.a[k], R.e[k], R.last_b_start[k], R.main_end[k]);
+        const int64_t extra = R.dp_end[k] - R.main_end[k];
+        R.busy[k] = (int64_t)m * (R.fop[k] + R.bop[k]) + (extra > 0 ? extra : 0);
+        mx = max64(mx, max64(R.main_end[k], R.dp_end[k]));
+    }
+    for (int off = 1; off < wl; off <<= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, off, wl));
+    R.batch = mx;
+    return R;
+}
+
+}  // namespace distsim

@@ -1,0 +1,260 @@
+// Selection kernels: best candidate (argmin) and the k fastest candidates (top-k) of an array
+// of batch times.  Ordering is always by (batch time, index): ties go to the smaller index.
+#include "engine.h"
+
+namespace distsim {
+
+namespace {
+
+using u64 = unsigned long long;
+constexpr int kSelThreads = 256;
+
+__device__ __forceinline__ u64 warp_min_u64(u64 x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const u64 y = __shfl_xor_sync(0xffffffffu, x, o);
+        x = y < x ? y : x;
+    }
+    return x;
+}
+
+__device__ __forceinline__ u64 block_min_u64(u64 x)
+{
+    __shared__ u64 part[kSelThreads / 32];
+    x = warp_min_u64(x);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        x = threadIdx.x < kSelThreads / 32 ? part[threadIdx.x] : ~0ull;
+        x = warp_min_u64(x);
+    }
+    __syncthreads();
+    return x;   // valid on thread 0
+}
+
+// Packed argmin: key = (time << idx_bits) | index fits 64 bits, one atomicMin per block.
+__global__ void __launch_bounds__(kSelThreads)
+argmin_packed_kernel(const int64_t *__restrict__ t, int64_t n, int idx_bits, u64 *key)
+{
+    u64 best = ~0ull;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const u64 k = ((u64)t[i] << idx_bits) | (u64)i;
+        best = k < best ? k : best;
+    }
+    best = block_min_u64(best);
+    if (threadIdx.x == 0 && best != ~0ull) atomicMin(key, best);
+}
+
+// Two-pass argmin for times too wide to pack: first the smallest time, then the smallest index
+// among the elements that have it.
+__global__ void __launch_bounds__(kSelThreads)
+argmin_time_kernel(const int64_t *__restrict__ t, int64_t n, u64 *key)
+{
+    u64 best = ~0ull;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const u64 k = (u64)t[i];
+        best = k < best ? k : best;
+    }
+    best = block_min_u64(best);
+    if (threadIdx.x == 0 && best != ~0ull) atomicMin(key, best);
+}
+__global__ void __launch_bounds__(kSelThreads)
+argmin_index_kernel(const int64_t *__restrict__ t, int64_t n, u64 *key)
+{
+    const u64 tmin = key[0];
+    u64 best = ~0ull;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        if ((u64)t[i] == tmin) { best = (u64)i < best ? (u64)i : best; }
+    best = block_min_u64(best);
+    if (threadIdx.x == 0 && best != ~0ull) atomicMin(key + 1, best);
+}
+__global__ void argmin_unpack_kernel(const u64 *key, int idx_bits, int packed, int64_t *result)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (packed) {
+        result[0] = (int64_t)(key[0] >> idx_bits);
+        result[1] = (int64_t)(key[0] & ((1ull << idx_bits) - 1ull));
+    } else {
+        result[0] = (int64_t)key[0];
+        result[1] = (int64_t)key[1];
+    }
+}
+
+// ---- top-k ---------------------------------------------------------------------------------
+// Radix select, most significant byte first: first on the time, then on the index among the
+// elements whose time equals the threshold.  `rank` is the rank still to resolve inside the
+// current group; blocks_done counts finished blocks of a pass; cursor is the output cursor.
+struct SelState { u64 tprefix, tmask, rank, iprefix, imask, blocks_done, cursor, pad; };
+
+template <bool kIndexPhase>
+__global__ void __launch_bounds__(kSelThreads)
+radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, u64 *hist, SelState *st)
+{
+    __shared__ unsigned int sh[256];
+    __shared__ bool last;
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) sh[i] = 0;
+    __syncthreads();
+    const u64 tprefix = st->tprefix, tmask = st->tmask, iprefix = st->iprefix, imask = st->imask;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const u64 x = (u64)t[i];
+        if ((x & tmask) != tprefix) continue;
+        if (kIndexPhase) {
+            if (((u64)i & imask) != iprefix) continue;
+            atomicAdd(&sh[((u64)i >> shift) & 255u], 1u);
+        } else {
+            atomicAdd(&sh[(x >> shift) & 255u], 1u);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) if (sh[i]) atomicAdd(&hist[i], (u64)sh[i]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&st->blocks_done, 1ull) == (u64)gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    // the last block to finish picks the bin that holds the wanted rank
+    __threadfence();
+    if (threadIdx.x == 0) {
+        u64 rank = st->rank, cum = 0;
+        int bin = 255;
+        for (int b = 0; b < 256; ++b) {
+            const u64 h = *((volatile u64 *)&hist[b]);
+            if (rank < cum + h) { bin = b; break; }
+            cum += h;
+        }
+        st->rank = rank - cum;
+        if (kIndexPhase) { st->iprefix = iprefix | ((u64)bin << shift); st->imask = imask | (255ull << shift); }
+        else { st->tprefix = tprefix | ((u64)bin << shift); st->tmask = tmask | (255ull << shift); }
+        st->blocks_done = 0;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+}
+
+__global__ void sel_init_kernel(SelState *st, u64 *hist, int k)
+{
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+    if (threadIdx.x == 0) { SelState z = {0, 0, (u64)(k - 1), 0, 0, 0, 0, 0}; *st = z; }
+}
+
+// Collects the k elements that are not above the threshold pair (time, index), in any order.
+__global__ void __launch_bounds__(kSelThreads)
+collect_kernel(const int64_t *__restrict__ t, int64_t n, SelState *st, int k, int64_t *ct, int64_t *ci)
+{
+    const u64 T = st->tprefix, I = st->iprefix;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const u64 x = (u64)t[i];
+        if (x < T || (x == T && (u64)i <= I)) {
+            const u64 pos = atomicAdd(&st->cursor, 1ull);
+            if (pos < (u64)k) { ct[pos] = (int64_t)x; ci[pos] = i; }
+        }
+    }
+}
+
+// One block sorts up to 4096 (time, index) pairs ascending (bitonic network in shared memory)
+// and writes the first k.  Also the whole top-k for arrays of at most 4096 elements.
+constexpr int kSortMax = 4096;
+__global__ void __launch_bounds__(1024)
+sort_pairs_kernel(const int64_t *__restrict__ ct, const int64_t *__restrict__ ci, int n_in, int k,
+                  int64_t first, int64_t *out_idx, int64_t *out_time)
+{
+    extern __shared__ __align__(16) unsigned char sm[];
+    int64_t *st = reinterpret_cast<int64_t *>(sm);
+    int64_t *si = st + kSortMax;
+    int np2 = 1;
+    while (np2 < n_in) np2 <<= 1;
+    for (int i = threadIdx.x; i < np2; i += blockDim.x) {
+        st[i] = i < n_in ? ct[i] : INT64_MAX;
+        si[i] = i < n_in ? (ci ? ci[i] : (int64_t)i) : INT64_MAX;
+    }
+    __syncthreads();
+    for (int size = 2; size <= np2; size <<= 1)
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int i = threadIdx.x; i < np2 / 2; i += blockDim.x) {
+                const int a = 2 * i - (i & (stride - 1));
+                const int b = a + stride;
+                const bool up = (a & size) == 0;
+                const bool gt = st[a] > st[b] || (st[a] == st[b] && si[a] > si[b]);
+                if (gt == up) {
+                    const int64_t x = st[a]; st[a] = st[b]; st[b] = x;
+                    const int64_t y = si[a]; si[a] = si[b]; si[b] = y;
+                }
+            }
+            __syncthreads();
+        }
+    for (int i = threadIdx.x; i < k; i += blockDim.x) {
+        out_idx[i] = first + si[i];
+        if (out_time) out_time[i] = st[i];
+    }
+}
+
+int bits_for(int64_t v)       // number of bits needed to represent v >= 0
+{
+    int b = 0;
+    while (v > 0) { ++b; v >>= 1; }
+    return b;
+}
+
+int grid_for(int64_t n)
+{
+    int64_t g = (n + kSelThreads * 8 - 1) / (kSelThreads * 8);
+    if (g < 1) g = 1;
+    if (g > 148 * 8) g = 148 * 8;
+    return (int)g;
+}
+
+}  // namespace
+
+void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t time_bound,
+                   const SelectScratch &sc, int64_t *d_result, int64_t *launches)
+{
+    const int idx_bits = bits_for(count - 1) > 0 ? bits_for(count - 1) : 1;
+    const bool packed = bits_for(time_bound) + idx_bits <= 63;
+    cudaMemsetAsync(sc.key, 0xFF, 2 * sizeof(u64), s);
+    const int g = grid_for(count);
+    if (packed) {
+        argmin_packed_kernel<<<g, kSelThreads, 0, s>>>(batch, count, idx_bits, sc.key);
+        ++*launches;
+    } else {
+        argmin_time_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc.key);
+        argmin_index_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc.key);
+        *launches += 2;
+    }
+    argmin_unpack_kernel<<<1, 32, 0, s>>>(sc.key, idx_bits, packed ? 1 : 0, d_result);
+    ++*launches;
+}
+
+void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
+                 const SelectScratch &sc, int64_t *d_indices, int64_t *d_times, int64_t *launches)
+{
+    static bool attr_set = false;
+    const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
+    if (!attr_set) {
+        cudaFuncSetAttribute(sort_pairs_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem);
+        attr_set = true;
+    }
+    if (count <= kSortMax) {
+        sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(batch, nullptr, (int)count, k, first, d_indices, d_times);
+        ++*launches;
+        return;
+    }
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    sel_init_kernel<<<1, 256, 0, s>>>(st, sc.hist, k);
+    ++*launches;
+    const int g = grid_for(count);
+    for (int shift = 56; shift >= 0; shift -= 8) {
+        radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, shift, sc.hist, st);
+        ++*launches;
+    }
+    const int ib = bits_for(count - 1);
+    for (int shift = ((ib + 7) / 8 - 1) * 8; shift >= 0; shift -= 8) {
+        radix_pass_kernel<true><<<g, kSelThreads, 0, s>>>(batch, count, shift, sc.hist, st);
+        ++*launches;
+    }
+    collect_kernel<<<g, kSelThreads, 0, s>>>(batch, count, st, k, sc.cand_time, sc.cand_idx);
+    sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, k, k, first, d_indices, d_times);
+    *launches += 2;
+}
+
+}  // namespace distsim

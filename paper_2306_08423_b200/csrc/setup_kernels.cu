@@ -1,0 +1,157 @@
+// Set-up kernels: turn the raw event table into the device tables the hot kernels read.
+// They run once per (table, search space), so they favour clarity over speed; every
+// division of the communication cost model happens here and none in the hot kernels.
+#include "engine.h"
+
+namespace distsim {
+
+namespace {
+
+__device__ __forceinline__ int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Ring all-reduce over n devices of `bytes`: 2(n-1) steps, each paying the latency and moving
+// 1/n of the tensor, i.e. a per-device volume of 2(n-1)*bytes/n (paper Sec. 4.2).
+__device__ __forceinline__ int64_t ring_cost(int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
+{
+    return 2 * (n - 1) * alpha + ceil_div(2 * (n - 1) * bytes, n * beta);
+}
+
+// One thread per entry: the communication-event costs that depend on (mp, dp, b).
+// The first thread of each row also fills the row's full-bucket cost.
+__global__ void fill_entries_kernel(TableConst tc, Row *rows, int n_rows, Entry *entries, int n_entries)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_entries) return;
+    Entry en = entries[i];
+    const Row row = rows[en.row];
+    const int64_t act = (int64_t)en.b * tc.seq * tc.hidden * tc.elem_bytes;
+    // a collective is intra-node iff all members share a node: for power-of-two degrees an MP
+    // group of aligned consecutive ranks fits a node iff mp <= G; a DP group has stride mp*pp
+    // and spans nodes whenever the cluster has more than one node
+    const bool mp_inter = row.mp > tc.gpus_per_node;
+    const bool dp_inter = tc.n_devices > tc.gpus_per_node;
+    en.ar = 0;
+    if (row.mp > 1)
+        en.ar = ring_cost(row.mp, 2 * act, mp_inter ? tc.alpha_inter : tc.alpha_intra,
+                          mp_inter ? tc.beta_inter : tc.beta_intra);
+    en.a2a = 0;
+    if (row.dp > 1) {
+        const int64_t a = dp_inter ? tc.alpha_inter : tc.alpha_intra;
+        const int64_t be = dp_inter ? tc.beta_inter : tc.beta_intra;
+        en.a2a = (row.dp - 1) * a + ceil_div((int64_t)(row.dp - 1) * act, (int64_t)row.dp * be);
+    }
+    en.p2p_intra = tc.alpha_intra + ceil_div(act, tc.beta_intra);
+    en.p2p_inter = tc.alpha_inter + ceil_div(act, tc.beta_inter);
+    entries[i] = en;
+    if (i == row.entry0) {
+        int64_t t_full = 0;
+        if (row.dp > 1 && tc.bucket > 0)
+            t_full = ring_cost(row.dp, tc.bucket, dp_inter ? tc.alpha_inter : tc.alpha_intra,
+                               dp_inter ? tc.beta_inter : tc.beta_intra);
+        rows[en.row].t_full = t_full;
+    }
+}
+
+// One thread per entry: exclusive prefix sums of the layer composites.
+__global__ void build_prefix_kernel(TableConst tc, RawTable raw, const Entry *entries, int n_entries,
+                                    int64_t *etf, int64_t *etb)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_entries) return;
+    const Entry en = entries[i];
+    const int64_t *f = raw.fwd + (int64_t)en.cls * tc.n_layers;
+    const int64_t *g = raw.bwd + (int64_t)en.cls * tc.n_layers;
+    int64_t *pf = etf + (int64_t)i * tc.lp;
+    int64_t *pb = etb + (int64_t)i * tc.lp;
+    int64_t sf = 0, sb = 0;
+    for (int l = 0; l < tc.n_layers; ++l) {
+        pf[l] = sf; pb[l] = sb;
+        const int64_t comm = en.ar + (raw.expert[l] ? en.a2a : 0);
+        sf += f[l] + comm;
+        sb += g[l] + comm;
+    }
+    for (int l = tc.n_layers; l < tc.lp; ++l) { pf[l] = sf; pb[l] = sb; }
+}
+
+// One thread per (row, e): for a stage that ends at layer e (exclusive) and starts at layer l,
+// the gradient stream is layers e-1, e-2, .., l with ceil(grad/mp) bytes each.
+//   nb[e][l] = full buckets completed by the time layer l has produced its gradients
+//   tp[e][l] = cost of the partial bucket left over for the stage [l, e)  (0 if none)
+// With bucket size 0 the whole stage is one bucket: nb = 0 and tp = its cost.
+__global__ void build_bucket_tables_kernel(TableConst tc, RawTable raw, const Row *rows, int n_rows,
+                                           int64_t *nb, int64_t *tp)
+{
+    const int L1 = tc.n_layers + 1;
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_rows * L1) return;
+    const int r = i / L1, e = i % L1;
+    const Row row = rows[r];
+    int64_t *nbr = nb + row.row_tab_off + (int64_t)e * L1;
+    int64_t *tpr = tp + row.row_tab_off + (int64_t)e * L1;
+    const bool dp_inter = tc.n_devices > tc.gpus_per_node;
+    const int64_t a = dp_inter ? tc.alpha_inter : tc.alpha_intra;
+    const int64_t be = dp_inter ? tc.beta_inter : tc.beta_intra;
+    int64_t w = 0;
+    for (int l = e; l >= 0; --l) {
+        if (l < e) w += ceil_div(raw.grad[l], row.mp);
+        int64_t full = 0, rem = w;
+        if (tc.bucket > 0) { full = w / tc.bucket; rem = w - full * tc.bucket; }
+        nbr[l] = full;
+        tpr[l] = (rem > 0 && row.dp > 1) ? ring_cost(row.dp, rem, a, be) : 0;
+    }
+    for (int l = e + 1; l < L1; ++l) { nbr[l] = 0; tpr[l] = 0; }
+}
+
+// next_grad[l] = smallest l' >= l whose gradient is non-empty (n_layers if none);
+// pe[l] = number of expert layers before layer l.
+__global__ void build_layer_tables_kernel(TableConst tc, RawTable raw, int32_t *next_grad, int32_t *pe)
+{
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    int nxt = tc.n_layers;
+    next_grad[tc.n_layers] = nxt;
+    for (int l = tc.n_layers - 1; l >= 0; --l) {
+        if (raw.grad[l] > 0) nxt = l;
+        next_grad[l] = nxt;
+    }
+    int acc = 0;
+    for (int l = 0; l < tc.n_layers; ++l) { pe[l] = acc; acc += raw.expert[l] ? 1 : 0; }
+    pe[tc.n_layers] = acc;
+}
+
+}  // namespace
+
+void launch_fill_entries(cudaStream_t s, const TableConst &tc, Row *rows, int n_rows,
+                         Entry *entries, int n_entries, int64_t *launches)
+{
+    if (n_entries == 0) return;
+    fill_entries_kernel<<<(n_entries + 127) / 128, 128, 0, s>>>(tc, rows, n_rows, entries, n_entries);
+    ++*launches;
+}
+
+void launch_build_prefix(cudaStream_t s, const TableConst &tc, const RawTable &raw,
+                         const Entry *entries, int n_entries, int64_t *etf, int64_t *etb,
+                         int64_t *launches)
+{
+    if (n_entries == 0) return;
+    build_prefix_kernel<<<(n_entries + 127) / 128, 128, 0, s>>>(tc, raw, entries, n_entries, etf, etb);
+    ++*launches;
+}
+
+void launch_build_bucket_tables(cudaStream_t s, const TableConst &tc, const RawTable &raw,
+                                const Row *rows, int n_rows, int64_t *nb, int64_t *tp,
+                                int64_t *launches)
+{
+    const int n = n_rows * (tc.n_layers + 1);
+    if (n == 0) return;
+    build_bucket_tables_kernel<<<(n + 127) / 128, 128, 0, s>>>(tc, raw, rows, n_rows, nb, tp);
+    ++*launches;
+}
+
+void launch_build_layer_tables(cudaStream_t s, const TableConst &tc, const RawTable &raw,
+                               int32_t *next_grad, int32_t *pe, int64_t *launches)
+{
+    build_layer_tables_kernel<<<1, 32, 0, s>>>(tc, raw, next_grad, pe);
+    ++*launches;
+}
+
+}  // namespace distsim

@@ -1,0 +1,241 @@
+"""Thin ctypes binding of the engine's C ABI (``include/distsim.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  Device buffers are PyTorch tensors (PyTorch is used for device memory
+and streams, nothing else); their ``data_ptr()`` is what crosses the boundary.
+There is no fallback: if ``libdistsim.so`` has not been built, importing this
+module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdistsim.so")
+MAX_PP = 64
+
+OK, E_ARG, E_STATE, E_RANGE, E_CAPACITY, E_OVERFLOW, E_CUDA, E_TIMEOUT, E_UNSUPPORTED = (
+    0, -1, -2, -3, -4, -5, -6, -7, -8)
+
+EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error", "distsim_launch_count",
+           "distsim_load_event_table", "distsim_set_space", "distsim_decode",
+           "distsim_eval_strategies", "distsim_argmin", "distsim_topk",
+           "distsim_emit_timelines", "distsim_search_host")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2306_08423_b200.build` "
+                      "(there is no CPU fallback)")
+_lib = C.CDLL(LIB_PATH)
+
+
+class DistsimError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"distsim error {code}: {msg}")
+        self.code = code
+
+
+class _Table(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_classes", C.c_int32), ("n_devices", C.c_int32),
+                ("gpus_per_node", C.c_int32), ("global_batch", C.c_int64), ("seq", C.c_int64),
+                ("hidden", C.c_int64), ("alpha_intra_ns", C.c_int64), ("beta_intra", C.c_int64),
+                ("alpha_inter_ns", C.c_int64), ("beta_inter", C.c_int64),
+                ("dp_bucket_bytes", C.c_int64), ("dp_overlap", C.c_int32),
+                ("act_bytes_per_elem", C.c_int32), ("class_mp", C.c_void_p),
+                ("class_b", C.c_void_p), ("fwd_ns", C.c_void_p), ("bwd_ns", C.c_void_p),
+                ("layer_is_expert", C.c_void_p), ("grad_bytes", C.c_void_p)]
+
+
+class _Space(C.Structure):
+    _fields_ = [("mp_max", C.c_int32), ("pp_max", C.c_int32), ("n_m", C.c_int32),
+                ("m_list", C.c_void_p), ("m_rule", C.c_int32), ("partition_mode", C.c_int32),
+                ("sched_mask", C.c_int32)]
+
+
+class _Candidate(C.Structure):
+    _fields_ = [("mp", C.c_int32), ("pp", C.c_int32), ("dp", C.c_int32), ("m", C.c_int32),
+                ("sched", C.c_int32), ("micro_batch_size", C.c_int32), ("class_index", C.c_int32),
+                ("bounds", C.c_int32 * (MAX_PP + 1))]
+
+
+_lib.distsim_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
+_lib.distsim_destroy.argtypes = [C.c_void_p]
+_lib.distsim_destroy.restype = None
+_lib.distsim_last_error.argtypes = [C.c_void_p]
+_lib.distsim_last_error.restype = C.c_char_p
+_lib.distsim_launch_count.argtypes = [C.c_void_p]
+_lib.distsim_launch_count.restype = C.c_int64
+_lib.distsim_load_event_table.argtypes = [C.c_void_p, C.POINTER(_Table)]
+_lib.distsim_set_space.argtypes = [C.c_void_p, C.POINTER(_Space), C.POINTER(C.c_int64)]
+_lib.distsim_decode.argtypes = [C.c_void_p, C.c_int64, C.POINTER(_Candidate)]
+_lib.distsim_eval_strategies.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
+_lib.distsim_argmin.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
+                                C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+_lib.distsim_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
+                              C.c_void_p, C.c_void_p]
+_lib.distsim_emit_timelines.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                        C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.POINTER(C.c_int64)]
+_lib.distsim_search_host.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_Space), C.c_int32,
+                                     C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                                     C.c_void_p, C.c_void_p]
+
+
+def _np_ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _table_struct(t):
+    arrs = [np.ascontiguousarray(t.class_mp, np.int32), np.ascontiguousarray(t.class_b, np.int32),
+            np.ascontiguousarray(t.fwd_ns, np.int64), np.ascontiguousarray(t.bwd_ns, np.int64),
+            np.ascontiguousarray(t.layer_is_expert, np.uint8),
+            np.ascontiguousarray(t.grad_bytes, np.int64)]
+    s = _Table(t.n_layers, arrs[0].shape[0], t.n_devices, t.gpus_per_node, t.global_batch, t.seq,
+               t.hidden, t.alpha_intra_ns, t.beta_intra, t.alpha_inter_ns, t.beta_inter,
+               t.dp_bucket_bytes, t.dp_overlap, t.act_bytes_per_elem, *[_np_ptr(a) for a in arrs])
+    return s, arrs
+
+
+def _space_struct(sp):
+    ml = np.ascontiguousarray(sp.m_list, np.int32)
+    return _Space(sp.mp_max, sp.pp_max, ml.shape[0], _np_ptr(ml), sp.m_rule, sp.partition_mode,
+                  sp.sched_mask), ml
+
+
+def _dev_ptr(t, dtype_name: str, min_elems: int, what: str):
+    """Device pointer of a contiguous CUDA tensor after checking dtype and size."""
+    import torch
+    if t is None:
+        return None
+    want = getattr(torch, dtype_name)
+    if not t.is_cuda or t.dtype != want or not t.is_contiguous():
+        raise ValueError(f"{what}: need a contiguous CUDA tensor of {dtype_name}")
+    if t.numel() < min_elems:
+        raise ValueError(f"{what}: need at least {min_elems} elements, got {t.numel()}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+class Context:
+    """Owns one ``distsim_ctx`` on a CUDA device."""
+
+    def __init__(self, device: int = 0):
+        self._h = C.c_void_p()
+        rc = _lib.distsim_create(C.byref(self._h), device)
+        if rc != OK:
+            raise DistsimError(rc, "distsim_create failed (no CUDA device of compute capability 10.x?)")
+        self.device = device
+        self.n_candidates = 0
+        self.n_devices = 0
+        self.pp_max = 0
+
+    def close(self):
+        if self._h:
+            _lib.distsim_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int):
+        if rc != OK:
+            raise DistsimError(rc, _lib.distsim_last_error(self._h).decode())
+
+    @property
+    def launch_count(self) -> int:
+        return int(_lib.distsim_launch_count(self._h))
+
+
+def distsim_load_event_table(ctx: Context, table) -> None:
+    s, _keep = _table_struct(table)
+    ctx._check(_lib.distsim_load_event_table(ctx._h, C.byref(s)))
+    ctx.n_devices = int(table.n_devices)
+    ctx.n_candidates = 0
+
+
+def distsim_set_space(ctx: Context, space) -> int:
+    s, _keep = _space_struct(space)
+    n = C.c_int64(0)
+    ctx._check(_lib.distsim_set_space(ctx._h, C.byref(s), C.byref(n)))
+    ctx.n_candidates = int(n.value)
+    ctx.pp_max = int(space.pp_max)
+    return ctx.n_candidates
+
+
+def distsim_decode(ctx: Context, index: int) -> dict:
+    c = _Candidate()
+    ctx._check(_lib.distsim_decode(ctx._h, index, C.byref(c)))
+    return dict(mp=c.mp, pp=c.pp, dp=c.dp, m=c.m, sched=c.sched, micro_batch_size=c.micro_batch_size,
+                class_index=c.class_index, bounds=tuple(c.bounds[: c.pp + 1]))
+
+
+def distsim_eval_strategies(ctx: Context, first: int, count: int, d_batch_ns,
+                            d_stage_busy_ns=None, stream=None) -> None:
+    pb = _dev_ptr(d_batch_ns, "int64", count, "d_batch_ns")
+    ps = _dev_ptr(d_stage_busy_ns, "int64", count * ctx.pp_max, "d_stage_busy_ns")
+    ctx._check(_lib.distsim_eval_strategies(ctx._h, _stream(stream), first, count, pb, ps))
+
+
+def distsim_argmin(ctx: Context, d_batch_ns, first: int, count: int, stream=None):
+    pb = _dev_ptr(d_batch_ns, "int64", count, "d_batch_ns")
+    bi, bt = C.c_int64(0), C.c_int64(0)
+    ctx._check(_lib.distsim_argmin(ctx._h, _stream(stream), pb, first, count, C.byref(bi), C.byref(bt)))
+    return int(bi.value), int(bt.value)
+
+
+def distsim_topk(ctx: Context, d_batch_ns, first: int, count: int, k: int, d_indices,
+                 d_times=None, stream=None) -> None:
+    pb = _dev_ptr(d_batch_ns, "int64", count, "d_batch_ns")
+    pi = _dev_ptr(d_indices, "int64", k, "d_indices")
+    pt = _dev_ptr(d_times, "int64", k, "d_times")
+    ctx._check(_lib.distsim_topk(ctx._h, _stream(stream), pb, first, count, k, pi, pt))
+
+
+def distsim_emit_timelines(ctx: Context, d_indices, n: int, d_records, capacity_records: int,
+                           d_offsets=None, d_busy_ns=None, d_util=None, stream=None) -> int:
+    """Returns the number of records needed; raises DistsimError(E_CAPACITY) if
+    ``d_records`` is given but too small.  ``d_records`` is an int64 tensor of
+    at least ``5 * capacity_records`` elements (or None for a sizing pass)."""
+    pi = _dev_ptr(d_indices, "int64", n, "d_indices")
+    pr = _dev_ptr(d_records, "int64", 5 * capacity_records, "d_records")
+    nn = n * ctx.n_devices
+    po = _dev_ptr(d_offsets, "int64", nn + 1, "d_offsets")
+    pbz = _dev_ptr(d_busy_ns, "int64", nn, "d_busy_ns")
+    pu = _dev_ptr(d_util, "float64", nn, "d_util")
+    total = C.c_int64(0)
+    rc = _lib.distsim_emit_timelines(ctx._h, _stream(stream), pi, n, pr, capacity_records, po, pbz, pu,
+                                     C.byref(total))
+    if rc == E_CAPACITY:
+        e = DistsimError(rc, _lib.distsim_last_error(ctx._h).decode())
+        e.total_records = int(total.value)
+        raise e
+    ctx._check(rc)
+    return int(total.value)
+
+
+def distsim_search_host(ctx: Context, table, space, k: int = 0):
+    """Whole search from host memory.  Returns (n_candidates, best_index,
+    best_batch_ns, topk_indices, topk_times) with numpy arrays for the last two."""
+    ts, _k1 = _table_struct(table)
+    ss, _k2 = _space_struct(space)
+    n, bi, bt = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+    idx = np.zeros(max(k, 1), np.int64)
+    tim = np.zeros(max(k, 1), np.int64)
+    ctx._check(_lib.distsim_search_host(ctx._h, C.byref(ts), C.byref(ss), k, C.byref(n), C.byref(bi),
+                                        C.byref(bt), _np_ptr(idx) if k else None,
+                                        _np_ptr(tim) if k else None))
+    ctx.n_devices = int(table.n_devices)
+    ctx.n_candidates = int(n.value)
+    ctx.pp_max = int(space.pp_max)
+    kk = min(k, ctx.n_candidates, 4096)
+    return ctx.n_candidates, int(bi.value), int(bt.value), idx[:kk], tim[:kk]

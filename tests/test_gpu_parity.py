@@ -1,0 +1,298 @@
+"""Parity of the CUDA engine against the CPU oracle, through the C ABI.
+
+Integer outputs (batch time, activity time, argmin, top-k, every emitted record and
+offset) must be bit-exact; utilisation is fp64 within 1e-12 relative.
+"""
+import copy
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2306_08423_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+THREADS = max(1, min(32, (os.cpu_count() or 2)))
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_2306_08423_b200 import engine
+    return engine
+
+
+@pytest.fixture()
+def ctx(E):
+    c = E.Context(0)
+    yield c
+    c.close()
+
+
+def dev(n, dtype=torch.int64):
+    return torch.empty(n, dtype=dtype, device="cuda")
+
+
+def load(E, ctx, w):
+    E.distsim_load_event_table(ctx, w.table)
+    n = E.distsim_set_space(ctx, w.space)
+    assert n == oracle.count(w.table, w.space)
+    return n
+
+
+def eval_all(E, ctx, n, busy=True):
+    batch = dev(n)
+    sb = dev(n * ctx.pp_max) if busy else None
+    E.distsim_eval_strategies(ctx, 0, n, batch, sb)
+    torch.cuda.synchronize()
+    return batch, (sb.view(n, ctx.pp_max) if busy else None)
+
+
+def check_emission(E, ctx, w, indices):
+    """Emits the given candidates and compares every record with the oracle."""
+    N = w.table.n_devices
+    idx = torch.tensor(list(indices), dtype=torch.int64, device="cuda")
+    n = len(indices)
+    offsets, busy, util = dev(n * N + 1), dev(n * N), dev(n * N, torch.float64)
+    total = E.distsim_emit_timelines(ctx, idx, n, None, 0, offsets, busy, util)
+    records = dev(max(1, total) * 5)
+    records.fill_(-7)
+    total2 = E.distsim_emit_timelines(ctx, idx, n, records, total, offsets, busy, util)
+    assert total2 == total
+    torch.cuda.synchronize()
+    rec = records.cpu().numpy()[: total * 5].reshape(total, 5)
+    off = offsets.cpu().numpy(); bz = busy.cpu().numpy(); ut = util.cpu().numpy()
+    assert off[0] == 0 and off[-1] == total
+    order = np.argsort(np.asarray(indices), kind="stable")
+    cands = oracle.enumerate_at(w.table, w.space, np.asarray(indices)[order])
+    for pos, c in zip(order, cands):
+        r = oracle.simulate(w.table, c, replicate=True)
+        base = off[pos * N]
+        assert (off[pos * N: pos * N + N + 1] - base == r.offsets).all(), c
+        got = rec[base: base + r.offsets[-1]]
+        if not (got == r.records).all():
+            bad = np.argwhere((got != r.records).any(axis=1))[0, 0]
+            raise AssertionError(f"{c}: record {bad}: got {got[bad]}, want {r.records[bad]}")
+        assert (bz[pos * N: pos * N + N] == r.busy_ns).all(), c
+        np.testing.assert_allclose(ut[pos * N: pos * N + N], r.util, rtol=1e-12, atol=0)
+    return total
+
+
+def test_config0_everything(E, ctx):
+    w = W.config0()
+    n = load(E, ctx, w)
+    assert n == 88
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices(w.table, w.space, np.arange(n), replicate=True, pp_stride=w.space.pp_max)
+    assert (batch.cpu().numpy() == ob).all()
+    assert (sb.cpu().numpy() == obusy).all()
+    # host decode == oracle's loop enumeration
+    for i, c in enumerate(oracle.enumerate_at(w.table, w.space, np.arange(n))):
+        d = E.distsim_decode(ctx, i)
+        assert (d["mp"], d["pp"], d["dp"], d["m"], d["sched"], d["bounds"]) == (c.mp, c.pp, c.dp, c.m, c.sched, c.bounds)
+    bi, bt = E.distsim_argmin(ctx, batch, 0, n)
+    order = np.lexsort((np.arange(n), ob))
+    assert (bi, bt) == (order[0], ob[order[0]])
+    ki, kt = dev(10), dev(10)
+    E.distsim_topk(ctx, batch, 0, n, 10, ki, kt)
+    assert (ki.cpu().numpy() == order[:10]).all() and (kt.cpu().numpy() == ob[order[:10]]).all()
+    check_emission(E, ctx, w, list(range(n)))
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_small_full_parity(E, ctx, seed):
+    kw = dict(dp_overlap=seed % 2, dp_bucket_bytes=0 if seed % 4 == 3 else 3000)
+    if seed >= 4:
+        kw.update(n_devices=16, gpus_per_node=2, n_layers=9, global_batch=24, mp_max=4, pp_max=8,
+                  m_list=(1, 2, 3, 5, 6, 12), partition_mode=W.PARTITION_ALL)
+    w = W.random_small(100 + seed, **kw)
+    n = load(E, ctx, w)
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    gb = batch.cpu().numpy()
+    assert (gb == ob).all(), np.argwhere(gb != ob)[:5]
+    assert (sb.cpu().numpy() == obusy).all()
+    bi, bt = E.distsim_argmin(ctx, batch, 0, n)
+    order = np.lexsort((np.arange(n), ob))
+    assert (bi, bt) == (order[0], ob[order[0]])
+    k = min(n, 37)
+    ki = dev(k)
+    E.distsim_topk(ctx, batch, 0, n, k, ki)
+    assert (ki.cpu().numpy() == order[:k]).all()
+    rng = np.random.default_rng(seed)
+    pick = rng.choice(n, size=min(n, 24), replace=False).tolist()
+    check_emission(E, ctx, w, pick)
+
+
+def test_ranges_straddle_rows_and_empty(E, ctx):
+    w = W.random_small(7, partition_mode=W.PARTITION_ALL)
+    n = load(E, ctx, w)
+    full, _ = eval_all(E, ctx, n, busy=False)
+    full = full.cpu().numpy()
+    rng = np.random.default_rng(0)
+    for _ in range(12):
+        first = int(rng.integers(0, n))
+        count = int(rng.integers(0, n - first + 1))
+        out = dev(max(1, count)); out.fill_(-1)
+        E.distsim_eval_strategies(ctx, first, count, out)
+        torch.cuda.synchronize()
+        assert (out.cpu().numpy()[:count] == full[first:first + count]).all()
+        if count:
+            bi, bt = E.distsim_argmin(ctx, out, first, count)
+            seg = full[first:first + count]
+            assert bt == seg.min() and bi == first + int(np.argmin(seg))
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_eval_strategies(ctx, n - 1, 2, dev(2))
+    assert ei.value.code == E.E_RANGE
+
+
+def test_config2_long_pipelines(E, ctx):
+    w = W.config2()
+    n = load(E, ctx, w)
+    assert n == 4176
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    gb = batch.cpu().numpy()
+    assert (gb == ob).all(), np.argwhere(gb != ob)[:5]
+    assert (sb.cpu().numpy() == obusy).all()
+    order = np.lexsort((np.arange(n), ob))
+    bi, bt = E.distsim_argmin(ctx, batch, 0, n)
+    assert (bi, bt) == (order[0], ob[order[0]])
+    ki, kt = dev(1024), dev(1024)
+    E.distsim_topk(ctx, batch, 0, n, 1024, ki, kt)
+    assert (ki.cpu().numpy() == order[:1024]).all() and (kt.cpu().numpy() == ob[order[:1024]]).all()
+    # full timelines of three of the fastest (1024 devices each) and two pp = 64 candidates
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(n))
+    pp64 = [i for i, c in enumerate(cands) if c.pp == 64 and c.m == 7]
+    check_emission(E, ctx, w, [int(order[0]), int(order[517]), int(order[1023]), pp64[0], pp64[1]])
+
+
+def _sampled_parity(E, ctx, w, n_sample, seed):
+    n = load(E, ctx, w)
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    rng = np.random.default_rng(seed)
+    idx = np.unique(np.concatenate([np.linspace(0, n - 1, n_sample // 2).astype(np.int64),
+                                    rng.integers(0, n, n_sample // 2), [0, n - 1]]))
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, idx, THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    gb = batch[torch.from_numpy(idx).cuda()].cpu().numpy()
+    assert (gb == ob).all(), idx[np.argwhere(gb != ob)[:5, 0]]
+    # per-stage activity time on sampled candidates (evaluated one by one)
+    for i in idx[:: max(1, len(idx) // 64)]:
+        b1, s1 = dev(1), dev(ctx.pp_max)
+        E.distsim_eval_strategies(ctx, int(i), 1, b1, s1)
+        k = int(np.searchsorted(idx, i))
+        assert b1.item() == ob[k] and (s1.cpu().numpy() == obusy[k]).all()
+    # argmin over the whole space: agrees with a reduction of the device array, and the
+    # winner's time agrees with the oracle
+    bi, bt = E.distsim_argmin(ctx, batch, 0, n)
+    tmin = int(batch.min().item())
+    assert bt == tmin and bi == int((batch == tmin).nonzero()[0].item())
+    assert oracle.eval_indices(w.table, w.space, np.array([bi]))[0][0] == bt
+    # top-k: sorted by (time, index), equal to a stable sort of the device array
+    k = 1024
+    ki, kt = dev(k), dev(k)
+    E.distsim_topk(ctx, batch, 0, n, k, ki, kt)
+    st, si = torch.sort(batch, stable=True)
+    assert (kt == st[:k]).all() and (ki == si[:k]).all()
+    return n, batch, ki
+
+
+def test_config3_moe_sampled(E, ctx):
+    w = W.config3()
+    n, batch, ki = _sampled_parity(E, ctx, w, 3000, 3)
+    assert n == 650_420
+    pick = ki.cpu().numpy()[[0, 1, 500]].tolist() + [12345, n - 1]
+    check_emission(E, ctx, w, pick)
+
+
+def test_config1_full_size_sampled(E, ctx):
+    w = W.config1()
+    n, batch, ki = _sampled_parity(E, ctx, w, 6000, 1)
+    assert n == 38_838_764
+    pick = ki.cpu().numpy()[[0, 7, 1023]].tolist() + [0, 20_000_001, n - 1]
+    check_emission(E, ctx, w, pick)
+
+
+def test_two_pass_argmin_for_wide_times(E, ctx):
+    # times near 2^55 with a large count cannot be packed with the index into 64 bits
+    w = W.random_small(3, lo=2**44, hi=2**45, partition_mode=W.PARTITION_ALL, n_layers=12, pp_max=4,
+                       m_list=(1, 2, 4, 8))
+    n = load(E, ctx, w)
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    ob, _ = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS)
+    assert (batch.cpu().numpy() == ob).all()
+    reps = (1 << 21) // n + 1
+    big = batch.repeat(reps)                       # duplicates: ties must go to the first copy
+    bi, bt = E.distsim_argmin(ctx, big, 5, big.numel())
+    assert bt == ob.min() and bi == 5 + int(np.argmin(ob))
+    # top-k with massive ties: the k smallest indices among equal times
+    k = 300
+    ki, kt = dev(k), dev(k)
+    E.distsim_topk(ctx, big, 0, big.numel(), k, ki, kt)
+    st, si = torch.sort(big, stable=True)
+    assert (kt == st[:k]).all() and (ki == si[:k]).all()
+
+
+def test_api_errors(E, ctx):
+    w = W.config0()
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_set_space(ctx, w.space)
+    assert ei.value.code == E.E_STATE
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_eval_strategies(ctx, 0, 1, dev(1))
+    assert ei.value.code == E.E_STATE
+    t = copy.deepcopy(w.table); t.n_devices = 12
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_load_event_table(ctx, t)
+    assert ei.value.code == E.E_UNSUPPORTED
+    t = copy.deepcopy(w.table); t.fwd_ns[0, 0] = -1
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_load_event_table(ctx, t)
+    assert ei.value.code == E.E_ARG
+    t = copy.deepcopy(w.table); t.fwd_ns[:] = 2**60
+    E.distsim_load_event_table(ctx, t)
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_set_space(ctx, w.space)
+    assert ei.value.code == E.E_OVERFLOW
+    # a class the space needs is missing from the table
+    t = copy.deepcopy(w.table)
+    t.class_mp, t.class_b, t.fwd_ns, t.bwd_ns = t.class_mp[1:], t.class_b[1:], t.fwd_ns[1:], t.bwd_ns[1:]
+    E.distsim_load_event_table(ctx, t)
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_set_space(ctx, w.space)
+    assert ei.value.code == E.E_ARG and "not in the table" in str(ei.value)
+    # capacity and range errors of emission
+    n = load(E, ctx, w)
+    idx = torch.tensor([0, 5], dtype=torch.int64, device="cuda")
+    total = E.distsim_emit_timelines(ctx, idx, 2, None, 0)
+    small = dev(5 * (total - 1)); small.fill_(-1)
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_emit_timelines(ctx, idx, 2, small, total - 1)
+    assert ei.value.code == E.E_CAPACITY and ei.value.total_records == total
+    assert (small == -1).all()                     # nothing was written
+    bad = torch.tensor([0, n], dtype=torch.int64, device="cuda")
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_emit_timelines(ctx, bad, 2, None, 0)
+    assert ei.value.code == E.E_RANGE
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_topk(ctx, dev(n), 0, n, n + 1, dev(n + 1))
+    assert ei.value.code == E.E_ARG
+    with pytest.raises(E.DistsimError):
+        E.distsim_decode(ctx, n)
+    # the context is still usable afterwards
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    assert (batch.cpu().numpy() == oracle.eval_indices(w.table, w.space, np.arange(n))[0]).all()
+
+
+def test_search_host_matches_device_path(E, ctx):
+    w = W.config0()
+    n, bi, bt, ki, kt = E.distsim_search_host(ctx, w.table, w.space, 16)
+    ob, _ = oracle.eval_indices(w.table, w.space, np.arange(n))
+    order = np.lexsort((np.arange(n), ob))
+    assert (bi, bt) == (order[0], ob[order[0]])
+    assert (ki == order[:16]).all() and (kt == ob[order[:16]]).all()
