@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the batched strategy-timeline engine.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole hot path over one synthetic search: evaluate every candidate
+of the 64-device workload (every stage composition, 38.8 M candidates), find the best one,
+select the 1024 fastest and emit their full per-device timelines.  The headline value is
+candidates per second with the event table already resident in HBM; ``e2e`` times the same
+through host buffers (table upload, result download).  One JSON line is printed by rank 0.
+
+With N > 1 (launched under torchrun) every rank runs its own search (seed 1 + rank): the path
+shards by independent problems, no collective is on the data path, scaling is weak.
+``--impl reference`` times the CPU oracle, as it stands, on a bounded sample of the same
+workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2306_08423_b200 import workloads as W  # noqa: E402
+
+TOP_K = 1024
+INT_OPS_PER_CELL = 6      # int64 max (compare pair + two selects) + int64 add (add, add-with-carry)
+RECORD_BYTES = 40
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle on a bounded sample
+
+def oracle_sample_rate(w, n_total, sample, threads):
+    import oracle
+    idx = np.unique(np.linspace(0, n_total - 1, sample).astype(np.int64))
+    t0 = time.perf_counter()
+    oracle.eval_indices_parallel(w.table, w.space, idx, threads, replicate=False)
+    dt = time.perf_counter() - t0
+    return len(idx) / dt, dt, len(idx)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    w = W.config1()
+    n_total, cells = W.count_candidates_and_cells(w.table, w.space)
+    threads = os.cpu_count() or 1
+    rate, dt, ns = oracle_sample_rate(w, n_total, 2000, threads)          # calibration, untimed
+    sample = int(max(2000, min(400_000, rate * 8.0)))                      # about 8 s per step
+    for _ in range(args.warmup):
+        oracle_sample_rate(w, n_total, max(500, sample // 20), threads)
+    times, counts = [], []
+    for _ in range(args.steps):
+        r, dt, ns = oracle_sample_rate(w, n_total, sample, threads)
+        times.append(dt); counts.append(ns)
+    value = sum(counts) / sum(times)
+    desc = f"{counts[0]} evenly strided candidates of {n_total} per step"
+    line = {
+        "impl": "reference", "metric": "strategy_candidates_per_sec", "value": value, "unit": "candidates/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": w.name, "candidates": n_total, "sample_per_step": counts[0]},
+        "events_per_sec": value * cells / n_total,
+        "cpu_baseline": {"value": value, "unit": "candidates/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "candidates/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        with open(self.tmp.name) as f:
+            rows = [r.strip().split(", ") for r in f if r.strip()]
+        os.unlink(self.tmp.name)
+        sm, names = [], ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = set()
+        for r in rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); out["sm_max_mhz"] = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.strip() == "Active":
+                    reasons.add(name)
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        return out
+
+
+# ----------------------------------------------------------------------------------------------
+# our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2306_08423_b200 import engine as E
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    peaks, peak_kind = measured_peaks()
+
+    w = W.config1(seed=1 + rank)
+    table, space = w.table, w.space
+    n_total, cells = W.count_candidates_and_cells(table, space)
+    N = table.n_devices
+    ctx = E.Context(local)
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    E.distsim_load_event_table(ctx, table)
+    assert E.distsim_set_space(ctx, space) == n_total
+    batch = torch.empty(n_total, dtype=torch.int64, device=dev)
+    top_i = torch.empty(TOP_K, dtype=torch.int64, device=dev)
+    top_t = torch.empty(TOP_K, dtype=torch.int64, device=dev)
+    offsets = torch.empty(TOP_K * N + 1, dtype=torch.int64, device=dev)
+    busy = torch.empty(TOP_K * N, dtype=torch.int64, device=dev)
+    util = torch.empty(TOP_K * N, dtype=torch.float64, device=dev)
+    flush = torch.empty(256 * 2**20, dtype=torch.uint8, device=dev)          # > L2 (126 MB)
+
+    # sizing pass (untimed): how many records the 1024 fastest need
+    E.distsim_eval_strategies(ctx, 0, n_total, batch)
+    E.distsim_topk(ctx, batch, 0, n_total, TOP_K, top_i, top_t)
+    total_records = E.distsim_emit_timelines(ctx, top_i, TOP_K, None, 0)
+    capacity = total_records + total_records // 8 + 1024
+    records = torch.empty(capacity * 5, dtype=torch.int64, device=dev)
+
+    def step(timers=None):
+        e0, e1, e2, e3 = (ev(), ev(), ev(), ev()) if timers is not None else (None,) * 4
+        if timers is not None:
+            e0.record(stream)
+        E.distsim_eval_strategies(ctx, 0, n_total, batch)
+        if timers is not None:
+            e1.record(stream)
+        best = E.distsim_argmin(ctx, batch, 0, n_total)
+        E.distsim_topk(ctx, batch, 0, n_total, TOP_K, top_i, top_t)
+        if timers is not None:
+            e2.record(stream)
+        tot = E.distsim_emit_timelines(ctx, top_i, TOP_K, records, capacity, offsets, busy, util)
+        if timers is not None:
+            e3.record(stream)
+            timers.append((e0, e1, e2, e3))
+        return best, tot
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+        flush.fill_(1)
+    gpu_id = str(local)
+    try:
+        gpu_id = str(torch.cuda.get_device_properties(local).uuid)
+        if not gpu_id.startswith("GPU-"):
+            gpu_id = "GPU-" + gpu_id
+    except Exception:
+        gpu_id = str(local)
+    barrier()
+    sampler = ClockSampler(gpu_id) if rank == 0 else None
+    launches0 = ctx.launch_count
+    timers = []
+    for _ in range(args.steps):
+        best, tot = step(timers)
+        flush.fill_(1)                         # evict L2 between timed iterations
+    barrier()
+    launches = ctx.launch_count - launches0
+    # keep the clock sampler running through the end-to-end loop as well
+    step_ms = [t[0].elapsed_time(t[3]) for t in timers]
+    eval_ms = [t[0].elapsed_time(t[1]) for t in timers]
+    sel_ms = [t[1].elapsed_time(t[2]) for t in timers]
+    emit_ms = [t[2].elapsed_time(t[3]) for t in timers]
+    total_ms = sum(step_ms)
+
+    # ---- end to end through host buffers ----------------------------------------------------
+    h_top_i = torch.empty(TOP_K, dtype=torch.int64).pin_memory()
+    h_top_t = torch.empty(TOP_K, dtype=torch.int64).pin_memory()
+    h_off = torch.empty(TOP_K * N + 1, dtype=torch.int64).pin_memory()
+    h_busy = torch.empty(TOP_K * N, dtype=torch.int64).pin_memory()
+    h_util = torch.empty(TOP_K * N, dtype=torch.float64).pin_memory()
+    h_rec = torch.empty(capacity * 5, dtype=torch.int64).pin_memory()
+    h2d = sum(a.nbytes for a in (table.class_mp, table.class_b, table.fwd_ns, table.bwd_ns,
+                                 table.layer_is_expert, table.grad_bytes, space.m_list)) + 128
+
+    def e2e_step():
+        E.distsim_load_event_table(ctx, table)                    # host -> device
+        E.distsim_set_space(ctx, space)
+        E.distsim_eval_strategies(ctx, 0, n_total, batch)
+        best = E.distsim_argmin(ctx, batch, 0, n_total)           # -> host
+        E.distsim_topk(ctx, batch, 0, n_total, TOP_K, top_i, top_t)
+        tot = E.distsim_emit_timelines(ctx, top_i, TOP_K, records, capacity, offsets, busy, util)
+        h_top_i.copy_(top_i, non_blocking=True); h_top_t.copy_(top_t, non_blocking=True)
+        h_off.copy_(offsets, non_blocking=True); h_busy.copy_(busy, non_blocking=True)
+        h_util.copy_(util, non_blocking=True)
+        h_rec[: tot * 5].copy_(records[: tot * 5], non_blocking=True)
+        torch.cuda.synchronize()
+        return 16 + 2 * TOP_K * 8 + h_off.numel() * 8 + h_busy.numel() * 16 + tot * RECORD_BYTES
+
+    e2e_step()
+    barrier()
+    e2e_times = []
+    d2h = 0
+    for _ in range(max(1, min(args.steps, 3))):
+        flush.fill_(1)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        d2h = e2e_step()
+        e2e_times.append(time.perf_counter() - t0)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+
+    # ---- max over ranks -----------------------------------------------------------------------
+    red = torch.tensor([total_ms, sum(e2e_times) / len(e2e_times)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(red, op=dist.ReduceOp.MAX)
+    total_ms_max, e2e_s_max = red.tolist()
+    ms_per_step = total_ms_max / args.steps
+    value = world * n_total / (ms_per_step * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- rooflines -----------------------------------------------------------------------------
+    # integer-issue peak, measured now with a dependency-free add/xor stream
+    pe0, pe1 = ev(), ev()
+    E.distsim_int_issue_probe(ctx, 148 * 16, 2000)
+    pe0.record(stream)
+    ops = E.distsim_int_issue_probe(ctx, 148 * 16, 20000)
+    pe1.record(stream)
+    torch.cuda.synchronize()
+    int_peak_gops = ops / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
+    eval_s = statistics.mean(eval_ms) * 1e-3
+    achieved_gops = cells * INT_OPS_PER_CELL / eval_s / 1e9
+    roofline = {"bound": "alu", "kernel": "eval_lockstep_kernel", "achieved": achieved_gops, "peak": int_peak_gops,
+                "unit": "Gop/s (32-bit integer instructions; 6 per recurrence cell)",
+                "frac": achieved_gops / int_peak_gops, "traffic": None,
+                "peak_kind": "measured in this run (add/xor issue probe)",
+                "ms_per_launch_set": statistics.mean(eval_ms)}
+    emit_bytes = tot * RECORD_BYTES + TOP_K * N * 24 + 8
+    emit_gbs = emit_bytes / (statistics.mean(emit_ms) * 1e-3) / 1e9
+    roofline_emit = {"bound": "hbm", "kernel": "emit_items_kernel (+plan, scan, devices, buckets)",
+                     "achieved": emit_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": emit_gbs / peaks["hbm_gbs"], "traffic": None, "peak_kind": peak_kind,
+                     "bytes_per_step": emit_bytes, "ms": statistics.mean(emit_ms)}
+
+    line = {
+        "metric": "strategy_candidates_per_sec", "value": value, "unit": "candidates/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "candidates": n_total, "recurrence_cells": cells, "devices": N,
+                   "layers": table.n_layers, "top_k_emitted": TOP_K, "records_emitted": tot,
+                   "l2": "256 MB flush between timed iterations", "seed": "1 + rank"},
+        "events_per_sec": world * cells / (ms_per_step * 1e-3),
+        "phase_ms": {"eval": statistics.mean(eval_ms), "argmin_topk": statistics.mean(sel_ms),
+                     "emit": statistics.mean(emit_ms)},
+        "eval_only": {"candidates_per_sec": n_total / eval_s, "events_per_sec": cells / eval_s},
+        "best": {"index": best[0], "batch_ns": best[1]},
+        "roofline": roofline, "roofline_emit": roofline_emit,
+        "e2e": {"value": world * n_total / e2e_s_max, "unit": "candidates/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s_max * 1e3},
+        "gpu_launches": launches, "clocks": clocks,
+    }
+
+    if world == 1:
+        if not args.no_workloads:
+            line["workloads"] = other_workloads(E, ctx, torch, dev, peaks)
+        if not args.no_cpu:
+            import oracle
+            oracle.build()
+            threads = os.cpu_count() or 1
+            rate, dt, ns = oracle_sample_rate(w, n_total, 2000, threads)
+            sample = int(max(2000, min(400_000, rate * 12.0)))
+            rate, dt, ns = oracle_sample_rate(w, n_total, sample, threads)
+            line["cpu_baseline"] = {"value": rate, "unit": "candidates/s", "cores": threads, "kind": "oracle",
+                                    "sample": f"{ns} evenly strided candidates of {n_total}, {dt:.1f} s"}
+    ctx.close()
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def other_workloads(E, ctx, torch, dev, peaks):
+    """Evaluation rate on the other search workloads and emission rate on the 1024 fastest
+    candidates of the 1024-device workload (device-resident, CUDA events)."""
+    out = {}
+    stream = torch.cuda.current_stream()
+    for cfg in (0, 2, 3):
+        w = W.CONFIGS[cfg]()
+        n, cells = W.count_candidates_and_cells(w.table, w.space)
+        E.distsim_load_event_table(ctx, w.table)
+        E.distsim_set_space(ctx, w.space)
+        batch = torch.empty(n, dtype=torch.int64, device=dev)
+        times = []
+        for it in range(8):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            E.distsim_eval_strategies(ctx, 0, n, batch)
+            e1.record(stream)
+            best = E.distsim_argmin(ctx, batch, 0, n)
+            if it >= 3:
+                times.append(e0.elapsed_time(e1) * 1e-3)
+        t = statistics.median(times)
+        out[w.name] = {"candidates": n, "cells": cells, "eval_ms": t * 1e3, "candidates_per_sec": n / t,
+                       "events_per_sec": cells / t, "best_index": best[0], "best_batch_ns": best[1]}
+    # emission: still loaded with the 1024-device workload?  reload it to be explicit
+    w = W.config4()
+    n, _ = W.count_candidates_and_cells(w.table, w.space)
+    N = w.table.n_devices
+    E.distsim_load_event_table(ctx, w.table)
+    E.distsim_set_space(ctx, w.space)
+    batch = torch.empty(n, dtype=torch.int64, device=dev)
+    E.distsim_eval_strategies(ctx, 0, n, batch)
+    top = torch.empty(w.top_k, dtype=torch.int64, device=dev)
+    E.distsim_topk(ctx, batch, 0, n, w.top_k, top)
+    chunk = 32
+    sizes = [E.distsim_emit_timelines(ctx, top[i:i + chunk], min(chunk, w.top_k - i), None, 0)
+             for i in range(0, w.top_k, chunk)]
+    cap = max(sizes) + 1024
+    records = torch.empty(cap * 5, dtype=torch.int64, device=dev)
+    offsets = torch.empty(chunk * N + 1, dtype=torch.int64, device=dev)
+    busy = torch.empty(chunk * N, dtype=torch.int64, device=dev)
+    util = torch.empty(chunk * N, dtype=torch.float64, device=dev)
+    for i in range(0, 3 * chunk, chunk):                                     # warm-up
+        E.distsim_emit_timelines(ctx, top[i:i + chunk], chunk, records, cap, offsets, busy, util)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    total = 0
+    e0.record(stream)
+    for i in range(0, w.top_k, chunk):
+        c = min(chunk, w.top_k - i)
+        total += E.distsim_emit_timelines(ctx, top[i:i + c], c, records, cap, offsets, busy, util)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t = e0.elapsed_time(e1) * 1e-3
+    nbytes = total * RECORD_BYTES + w.top_k * N * 24
+    out[w.name] = {"candidates": w.top_k, "records": total, "bytes": nbytes, "seconds": t,
+                   "records_per_sec": total / t, "GB_per_sec": nbytes / t / 1e9,
+                   "frac_of_measured_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
+                   "frac_of_nominal_8TBs": nbytes / t / 1e9 / 8000.0,
+                   "chunk_candidates": chunk, "buffer_GB": cap * RECORD_BYTES / 1e9}
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the per-workload summary")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -209,6 +209,16 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table,
                         int64_t *h_best_index, int64_t *h_best_batch_ns,
                         int64_t *h_topk_indices, int64_t *h_topk_times);
 
+/*
+ * Measurement helper (no counterpart in the paper): enqueues a kernel of `blocks` x 256 threads
+ * that issues a dependency-free stream of 32-bit integer add / logic instructions, `iters`
+ * rounds of 16 per thread, and stores the total instruction count (threads x instructions) in
+ * *h_ops.  Timed by the caller with events on `stream`, it gives the device's plain-integer
+ * issue rate under the clocks of the moment.  Asynchronous.
+ */
+int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t blocks, int32_t iters,
+                            int64_t *h_ops);
+
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t distsim_launch_count(const distsim_ctx *ctx);
 

@@ -13,7 +13,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_PKG, "csrc")
 _OBJ = os.path.join(_PKG, "_build")
 LIB = os.path.join(_PKG, "libdistsim.so")
-SOURCES = ["distsim_api.cu", "setup_kernels.cu", "eval_kernels.cu", "select_kernels.cu", "emit_kernels.cu"]
+SOURCES = ["distsim_api.cu", "setup_kernels.cu", "eval_kernels.cu", "select_kernels.cu", "emit_kernels.cu",
+           "probe_kernels.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -528,4 +528,15 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table, co
     return distsim_argmin(ctx, nullptr, d_batch, 0, n, h_best_index, h_best_batch_ns);
 }
 
+int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t blocks, int32_t iters, int64_t *h_ops)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!h_ops || blocks < 1 || iters < 1) return fail(ctx, DISTSIM_E_ARG, "bad probe arguments");
+    if (int rc = set_device(ctx)) return rc;
+    *h_ops = launch_int_issue_probe(static_cast<cudaStream_t>(stream), blocks, iters,
+                                    ctx->d_result.as<int64_t>() + 4, &ctx->launches);
+    CU(cudaGetLastError(), "probe launch");
+    return DISTSIM_OK;
+}
+
 }  // extern "C"

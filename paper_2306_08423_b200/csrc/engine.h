@@ -147,4 +147,9 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
                          const int64_t *op_start, int64_t op_words_per_cand, int64_t max_tiles,
                          distsim_record *records, int64_t *launches);
 
+// ---- probe (probe_kernels.cu) ----------------------------------------------------------
+// Launches the integer-issue probe; returns the number of integer instructions (per thread,
+// summed over threads) it executes.
+int64_t launch_int_issue_probe(cudaStream_t s, int blocks, int iters, int64_t *sink, int64_t *launches);
+
 }  // namespace distsim

@@ -23,7 +23,7 @@ OK, E_ARG, E_STATE, E_RANGE, E_CAPACITY, E_OVERFLOW, E_CUDA, E_TIMEOUT, E_UNSUPP
 EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error", "distsim_launch_count",
            "distsim_load_event_table", "distsim_set_space", "distsim_decode",
            "distsim_eval_strategies", "distsim_argmin", "distsim_topk",
-           "distsim_emit_timelines", "distsim_search_host")
+           "distsim_emit_timelines", "distsim_search_host", "distsim_int_issue_probe")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2306_08423_b200.build` "
@@ -81,6 +81,9 @@ _lib.distsim_emit_timelines.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_
 _lib.distsim_search_host.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_Space), C.c_int32,
                                      C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                                      C.c_void_p, C.c_void_p]
+
+
+_lib.distsim_int_issue_probe.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]
 
 
 def _np_ptr(a: np.ndarray):
@@ -239,3 +242,10 @@ def distsim_search_host(ctx: Context, table, space, k: int = 0):
     ctx.pp_max = int(space.pp_max)
     kk = min(k, ctx.n_candidates, 4096)
     return ctx.n_candidates, int(bi.value), int(bt.value), idx[:kk], tim[:kk]
+
+
+def distsim_int_issue_probe(ctx: Context, blocks: int, iters: int, stream=None) -> int:
+    """Enqueues the integer-issue probe; returns the number of integer instructions it runs."""
+    ops = C.c_int64(0)
+    ctx._check(_lib.distsim_int_issue_probe(ctx._h, _stream(stream), blocks, iters, C.byref(ops)))
+    return int(ops.value)

@@ -142,6 +142,38 @@ def event_classes(n_devices: int, global_batch: int, n_layers: int, space: Searc
     return sorted(classes)
 
 
+def space_shape(table, space):
+    """Rows of the search space for reporting: a list of (mp, pp, dp, [valid m], partitions,
+    schedules).  Pure counting; candidates = sum(len(ms) * partitions * schedules)."""
+    rows = []
+    n_sched = bin(space.sched_mask & 3).count("1")
+    for mp in _pow2_upto(space.mp_max):
+        for pp in _pow2_upto(min(space.pp_max, table.n_layers)):
+            if table.n_devices % (mp * pp):
+                continue
+            dp = table.n_devices // (mp * pp)
+            if table.global_batch % dp:
+                continue
+            bp = table.global_batch // dp
+            ms = [m for m in space.m_list.tolist()
+                  if 1 <= m <= bp and (space.m_rule == M_RULE_CEIL or bp % m == 0)]
+            if not ms:
+                continue
+            parts = 1 if space.partition_mode == PARTITION_BALANCED else math.comb(table.n_layers - 1, pp - 1)
+            rows.append((mp, pp, dp, ms, parts, n_sched))
+    return rows
+
+
+def count_candidates_and_cells(table, space):
+    """(candidates, recurrence cells) of a space; a candidate has 2 * m * pp cells (one per
+    schedule item: forward and backward of every micro-batch on every stage)."""
+    cands = cells = 0
+    for mp, pp, dp, ms, parts, n_sched in space_shape(table, space):
+        cands += len(ms) * parts * n_sched
+        cells += sum(2 * m * pp for m in ms) * parts * n_sched
+    return cands, cells
+
+
 def build_table(*, per_sample_fwd_ns, per_sample_bwd_extra_ns, n_devices, gpus_per_node,
                 global_batch, seq, hidden, space, layer_is_expert=None, grad_bytes=None,
                 **cluster) -> EventTable:
