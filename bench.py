@@ -67,8 +67,9 @@ def run_reference(args):
     w = W.config1()
     n_total, cells = W.count_candidates_and_cells(w.table, w.space)
     threads = os.cpu_count() or 1
-    rate, dt, ns = oracle_sample_rate(w, n_total, 2000, threads)          # calibration, untimed
-    sample = int(max(2000, min(400_000, rate * 8.0)))                      # about 8 s per step
+    oracle_sample_rate(w, n_total, 4000, threads)                          # warms the thread pool
+    rate, dt, ns = oracle_sample_rate(w, n_total, 40_000, threads)         # calibration, untimed
+    sample = int(max(40_000, min(4_000_000, rate * 8.0)))                  # about 8 s per step
     for _ in range(args.warmup):
         oracle_sample_rate(w, n_total, max(500, sample // 20), threads)
     times, counts = [], []
@@ -332,8 +333,9 @@ def run_ours(args):
             import oracle
             oracle.build()
             threads = os.cpu_count() or 1
-            rate, dt, ns = oracle_sample_rate(w, n_total, 2000, threads)
-            sample = int(max(2000, min(400_000, rate * 12.0)))
+            oracle_sample_rate(w, n_total, 4000, threads)                   # warms the thread pool
+            rate, dt, ns = oracle_sample_rate(w, n_total, 40_000, threads)  # calibration
+            sample = int(max(40_000, min(4_000_000, rate * 15.0)))          # about 15 s of work
             rate, dt, ns = oracle_sample_rate(w, n_total, sample, threads)
             line["cpu_baseline"] = {"value": rate, "unit": "candidates/s", "cores": threads, "kind": "oracle",
                                     "sample": f"{ns} evenly strided candidates of {n_total}, {dt:.1f} s"}
