@@ -210,6 +210,32 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table,
                         int64_t *h_topk_indices, int64_t *h_topk_times);
 
 /*
+ * Top-k for callers that must not allocate device memory (the paper has no counterpart; this
+ * is a deployment convenience).  Every other entry point works on a distsim_ctx, and creating
+ * one calls cudaMalloc.  Some hosts cannot afford that: a latency-critical loop that may not
+ * block on the allocator's device-wide synchronisation, a process whose whole GPU memory has
+ * already been handed to a pool, or a plug-in inside a host application that forbids it.
+ * This variant needs no context and calls no allocator (neither CUDA's nor any library's):
+ * its radix-select scratch is a fixed array of about 18 KB that is part of the library image,
+ * present on every GPU that has loaded the library until the process exits.
+ *   d_batch_ns [count] in; d_indices [k] out (first + position), d_times [k] out, nullable;
+ *   result ascending by (batch time, index), identical to distsim_topk's.
+ *   Requires 1 <= k <= min(count, DISTSIM_TOPK_STATIC_MAX_K); a larger k is refused with
+ *   DISTSIM_E_CAPACITY and nothing is launched.  Other errors: DISTSIM_E_ARG (null pointer, bad
+ *   range), DISTSIM_E_CUDA, DISTSIM_E_UNSUPPORTED (device ordinal above 63).
+ * It runs on the current device.  The first call on each device looks up the array's device
+ * address (cudaGetSymbolAddress); make that first call before any stream capture begins and
+ * not concurrently from several host threads.  Asynchronous on `stream`.
+ * All calls on a device share the one array, and it keeps the previous call's contents; each
+ * call clears the parts it reads before using them.  Two calls whose kernels can overlap on the
+ * GPU (different streams or host threads of one process on the same device) race on it: issue
+ * them on one stream or order them yourself.
+ */
+#define DISTSIM_TOPK_STATIC_MAX_K 1024
+int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int64_t first, int64_t count,
+                        int32_t k, int64_t *d_indices, int64_t *d_times);
+
+/*
  * Measurement helper (no counterpart in the paper): enqueues a kernel of `blocks` x 256 threads
  * that issues a dependency-free stream of 32-bit integer add / logic instructions, `iters`
  * rounds of 16 per thread, and stores the total instruction count (threads x instructions) in

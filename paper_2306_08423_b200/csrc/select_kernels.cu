@@ -258,3 +258,45 @@ void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t co
 }
 
 }  // namespace distsim
+
+// ---- top-k without any allocation --------------------------------------------------------------
+// Same kernels as launch_topk, but the radix-select scratch (histogram, selection state and the
+// k collected pairs) lives in a fixed device array that is part of the loaded library, so the
+// call neither needs a context nor touches the CUDA allocator.
+namespace {
+
+constexpr int kStaticWords = 8 + 256 + 8 + 2 * DISTSIM_TOPK_STATIC_MAX_K;      // 64-bit words
+static __device__ __align__(256) unsigned long long g_topk_static_scratch[kStaticWords];
+
+constexpr int kMaxDevices = 64;
+unsigned long long *g_static_scratch_addr[kMaxDevices];    // device address of the array, per device
+
+}  // namespace
+
+extern "C" int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int64_t first,
+                                   int64_t count, int32_t k, int64_t *d_indices, int64_t *d_times)
+{
+    if (!d_batch_ns || !d_indices || first < 0 || count < 1 || k < 1 || k > count) return DISTSIM_E_ARG;
+    if (k > DISTSIM_TOPK_STATIC_MAX_K) return DISTSIM_E_CAPACITY;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DISTSIM_E_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return DISTSIM_E_UNSUPPORTED;
+    if (!g_static_scratch_addr[dev]) {
+        // In host code the array's name is only a handle for the runtime, not a pointer a kernel
+        // could use: ask the runtime for the address the array has on the current device.
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_topk_static_scratch) != cudaSuccess || !p) return DISTSIM_E_CUDA;
+        g_static_scratch_addr[dev] = static_cast<unsigned long long *>(p);
+    }
+    unsigned long long *base = g_static_scratch_addr[dev];
+    distsim::SelectScratch sc{};
+    sc.key = base; sc.hist = base + 8; sc.sel_state = base + 8 + 256;
+    sc.cand_time = reinterpret_cast<int64_t *>(base + 8 + 256 + 8);
+    sc.cand_idx = sc.cand_time + DISTSIM_TOPK_STATIC_MAX_K;
+    int64_t launches = 0;
+    // launch_topk begins by clearing the histogram, the selection state and the output cursor,
+    // so whatever the previous call left in the array is never read
+    distsim::launch_topk(static_cast<cudaStream_t>(stream), d_batch_ns, first, count, k, sc,
+                         d_indices, d_times, &launches);
+    return cudaGetLastError() == cudaSuccess ? DISTSIM_OK : DISTSIM_E_CUDA;
+}

@@ -23,7 +23,9 @@ OK, E_ARG, E_STATE, E_RANGE, E_CAPACITY, E_OVERFLOW, E_CUDA, E_TIMEOUT, E_UNSUPP
 EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error", "distsim_launch_count",
            "distsim_load_event_table", "distsim_set_space", "distsim_decode",
            "distsim_eval_strategies", "distsim_argmin", "distsim_topk",
-           "distsim_emit_timelines", "distsim_search_host", "distsim_int_issue_probe")
+           "distsim_emit_timelines", "distsim_search_host", "distsim_int_issue_probe",
+           "distsim_topk_static")
+TOPK_STATIC_MAX_K = 1024
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2306_08423_b200.build` "
@@ -84,6 +86,10 @@ _lib.distsim_search_host.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_S
 
 
 _lib.distsim_int_issue_probe.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]
+
+
+_lib.distsim_topk_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
+                                     C.c_void_p, C.c_void_p]
 
 
 def _np_ptr(a: np.ndarray):
@@ -249,3 +255,24 @@ def distsim_int_issue_probe(ctx: Context, blocks: int, iters: int, stream=None) 
     ops = C.c_int64(0)
     ctx._check(_lib.distsim_int_issue_probe(ctx._h, _stream(stream), blocks, iters, C.byref(ops)))
     return int(ops.value)
+
+
+def distsim_topk_static(d_batch_ns, first: int, count: int, k: int, d_indices, d_times=None,
+                        stream=None) -> None:
+    """The k fastest candidates without a context and without any device allocation.
+
+    For callers that cannot call cudaMalloc (a latency-critical loop, a process whose device
+    memory is all owned by a pool, a plug-in whose host forbids it): the scratch is a fixed
+    array inside the library, so
+    ``k`` is limited to ``TOPK_STATIC_MAX_K``.  The tensors are the caller's; this wrapper
+    creates none.  Runs on the current device; calls that may overlap on the GPU must be
+    ordered by the caller because they share the scratch.
+    """
+    pb = _dev_ptr(d_batch_ns, "int64", count, "d_batch_ns")
+    pi = _dev_ptr(d_indices, "int64", k, "d_indices")
+    pt = _dev_ptr(d_times, "int64", k, "d_times")
+    rc = _lib.distsim_topk_static(_stream(stream), pb, first, count, k, pi, pt)
+    if rc == E_CAPACITY:
+        raise DistsimError(rc, f"k = {k} exceeds the fixed scratch (at most {TOPK_STATIC_MAX_K})")
+    if rc != OK:
+        raise DistsimError(rc, "distsim_topk_static failed")
