@@ -406,6 +406,43 @@ def other_workloads(E, ctx, torch, dev, peaks):
     return out
 
 
+def profile_case(name):
+    """Small, bounded invocations for profiler captures (no timing, no JSON line):
+    eval1  - evaluation of a 2 M-candidate slice of the 64-device workload (pp = 16 rows)
+    eval3  - evaluation of the whole 256-device MoE workload (650 k candidates)
+    emit4  - emission of 16 of the fastest candidates of the 1024-device workload (~1.3 GB)"""
+    import torch
+    from paper_2306_08423_b200 import engine as E
+    torch.cuda.set_device(0)
+    ctx = E.Context(0)
+    if name in ("eval1", "eval3"):
+        w = W.config1() if name == "eval1" else W.config3()
+        E.distsim_load_event_table(ctx, w.table)
+        n = E.distsim_set_space(ctx, w.space)
+        first, count = (n - 2_000_000, 2_000_000) if name == "eval1" else (0, n)
+        batch = torch.empty(count, dtype=torch.int64, device="cuda")
+        for _ in range(3):
+            E.distsim_eval_strategies(ctx, first, count, batch)
+        print(name, "best", E.distsim_argmin(ctx, batch, first, count))
+    elif name == "emit4":
+        w = W.config4()
+        E.distsim_load_event_table(ctx, w.table)
+        n = E.distsim_set_space(ctx, w.space)
+        batch = torch.empty(n, dtype=torch.int64, device="cuda")
+        E.distsim_eval_strategies(ctx, 0, n, batch)
+        top = torch.empty(16, dtype=torch.int64, device="cuda")
+        E.distsim_topk(ctx, batch, 0, n, 16, top)
+        total = E.distsim_emit_timelines(ctx, top, 16, None, 0)
+        records = torch.empty(total * 5, dtype=torch.int64, device="cuda")
+        for _ in range(2):
+            E.distsim_emit_timelines(ctx, top, 16, records, total)
+        print(name, "records", total, "bytes", total * RECORD_BYTES)
+    else:
+        raise SystemExit(f"unknown profile case {name}")
+    torch.cuda.synchronize()
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -414,7 +451,11 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-workloads", action="store_true", help="skip the per-workload summary")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--profile-case", default=None, help="eval1 | eval3 | emit4: small run for ncu")
     args = ap.parse_args()
+    if args.profile_case:
+        profile_case(args.profile_case)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
