@@ -342,7 +342,7 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
             if (r.n_entries == 0) continue;
             r.size = sat_mul(sat_mul(r.n_part, r.n_entries), r.n_sched);
             r.offset = total;
-            r.row_tab_off = (int64_t)rows.size() * (L + 1) * (L + 1);
+            r.row_tab_off = (int64_t)rows.size() * (((L + 1) * (L + 1) + 1) & ~1);   // even: 16-byte aligned tables
             total = sat_add(total, r.size);
             if (r.n_part >= kSat || total >= kSat) return fail(ctx, DISTSIM_E_OVERFLOW, "candidate count does not fit 62 bits");
             rows.push_back(r);
@@ -363,7 +363,7 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     if (int rc = upload(ctx, ctx->d_binom, binom.data(), binom.size(), "upload binomials")) return rc;
     CU(ctx->d_etf.reserve(entries.size() * tc.lp * sizeof(int64_t)), "alloc prefix");
     CU(ctx->d_etb.reserve(entries.size() * tc.lp * sizeof(int64_t)), "alloc prefix");
-    const size_t tab = rows.size() * (size_t)(L + 1) * (L + 1) * sizeof(int64_t);
+    const size_t tab = rows.size() * (size_t)(((L + 1) * (L + 1) + 1) & ~1) * sizeof(int64_t);
     CU(ctx->d_nb.reserve(tab), "alloc bucket tables");
     CU(ctx->d_tp.reserve(tab), "alloc bucket tables");
     launch_fill_entries(0, tc, ctx->d_rows.as<Row>(), sc.n_rows, ctx->d_entries.as<Entry>(), sc.n_entries, &ctx->launches);

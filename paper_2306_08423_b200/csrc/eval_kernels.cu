@@ -8,6 +8,7 @@
 // (cp.async.bulk, completion on the block's own mbarrier, no multicast).
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
+#include "eval_thread.cuh"
 
 namespace distsim {
 
@@ -72,6 +73,45 @@ eval_lockstep_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_
     }
 }
 
+template <int PP>
+void launch_thread_kernel(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo,
+                          int64_t hi, int64_t first, int e_begin, int e_end, int ept, int64_t p_lo,
+                          int64_t p_hi, int64_t *batch_out, int64_t *busy_out)
+{
+    const int lp = v.tc.lp;
+    const int L1 = v.tc.n_layers + 1;
+    const int tab_words = (L1 * L1 + 1) & ~1;
+    ThreadKernelSmem plan{};
+    size_t words = 0;
+    const size_t budget_words = (200 * 1024 - sizeof(int64_t) * PP * kThreadBlock) / sizeof(int64_t);
+    // prefix rows of every entry of the row, then the row's two bucket tables, as far as they fit
+    if ((size_t)row.n_entries * lp * 2 <= 8192) {
+        plan.n_entries_staged = row.n_entries;
+        plan.off_etb = row.n_entries * lp;
+        words = (size_t)row.n_entries * lp * 2;
+    }
+    if (words + 2 * (size_t)tab_words <= (budget_words < 12288 ? budget_words : 12288)) {
+        plan.tables_staged = 1;
+        plan.off_nb = (int32_t)words;
+        plan.off_tp = (int32_t)words + tab_words;
+        words += 2 * (size_t)tab_words;
+    }
+    const size_t smem = words * sizeof(int64_t);
+    const int64_t n_threads = p_hi - p_lo;
+    dim3 grid((unsigned)((n_threads + kThreadBlock - 1) / kThreadBlock), (unsigned)((e_end - e_begin + ept - 1) / ept));
+    if (busy_out) {
+        if (smem > 32 * 1024)
+            cudaFuncSetAttribute(eval_thread_kernel<PP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_thread_kernel<PP, true><<<grid, kThreadBlock, smem, s>>>(v, row_index, lo, hi, first, e_begin, e_end, ept,
+                                                                      p_lo, p_hi, batch_out, busy_out, plan, tab_words);
+    } else {
+        if (smem > 32 * 1024)
+            cudaFuncSetAttribute(eval_thread_kernel<PP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_thread_kernel<PP, false><<<grid, kThreadBlock, smem, s>>>(v, row_index, lo, hi, first, e_begin, e_end, ept,
+                                                                       p_lo, p_hi, batch_out, busy_out, plan, tab_words);
+    }
+}
+
 }  // namespace
 
 void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const Row &row,
@@ -79,6 +119,30 @@ void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const R
                      int64_t *launches)
 {
     if (hi <= lo) return;
+    // Rows with many partitions and short pipelines: one partition per thread.
+    if (row.pp <= 16) {
+        const int64_t per_entry = row.n_part * row.n_sched;
+        const int e_begin = (int)(lo / per_entry), e_end = (int)((hi - 1) / per_entry) + 1;
+        int64_t p_lo = 0, p_hi = row.n_part;
+        if (e_end - e_begin == 1) {
+            p_lo = (lo - (int64_t)e_begin * per_entry) / row.n_sched;
+            p_hi = (hi - 1 - (int64_t)e_begin * per_entry) / row.n_sched + 1;
+        }
+        const int64_t n_parts = p_hi - p_lo;
+        const int n_e = e_end - e_begin;
+        const int ept = n_parts >= 148 * 4 * kThreadBlock ? n_e : 1;       // entries per thread
+        if (n_parts * ((n_e + ept - 1) / ept) >= 2048) {
+            switch (row.pp) {
+            case 1: launch_thread_kernel<1>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+            case 2: launch_thread_kernel<2>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+            case 4: launch_thread_kernel<4>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+            case 8: launch_thread_kernel<8>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+            default: launch_thread_kernel<16>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+            }
+            ++*launches;
+            return;
+        }
+    }
     const int S = row.pp > 32 ? 2 : 1;
     const int wl = row.pp / S;
     const int cpb = (kEvalThreads / 32) * (32 / wl);      // candidates per block

@@ -6,7 +6,7 @@
 // DISTSIM_E_TIMEOUT in the status word and reads the tables from global memory instead; it
 // polls once more (again bounded) before leaving so that no copy is still in flight when the
 // block's shared memory is released.
-// Requirements: source and destination 16-byte aligned, size a multiple of 16 bytes.
+// Requirements: sources and destinations 16-byte aligned, sizes multiples of 16 bytes.
 #pragma once
 
 #include "engine.h"
@@ -32,11 +32,13 @@ __device__ __forceinline__ bool mbar_poll(uint32_t bar, uint32_t phase, int max_
     return false;
 }
 
-// Copies `bytes` from src_a to dst_a and from src_b to dst_b (both shared destinations).
-// Must be called by every thread of the block.  Returns true when the shared copies are usable.
-__device__ __forceinline__ bool stage_two_tables(uint64_t *bar_ptr, void *dst_a, const void *src_a,
-                                                 void *dst_b, const void *src_b, uint32_t bytes,
-                                                 int32_t *status)
+struct StageCopy { void *dst; const void *src; uint32_t bytes; };
+
+// Issues up to kMaxCopies bulk copies (entries with bytes == 0 are skipped) and waits for all of
+// them.  Must be called once per block, by every thread.  Returns true when the shared copies
+// are usable by the whole block.
+constexpr int kMaxCopies = 4;
+__device__ __forceinline__ bool stage_tables(uint64_t *bar_ptr, const StageCopy (&c)[kMaxCopies], int32_t *status)
 {
     const uint32_t bar = smem_addr(bar_ptr);
     if (threadIdx.x == 0) {
@@ -45,14 +47,17 @@ __device__ __forceinline__ bool stage_two_tables(uint64_t *bar_ptr, void *dst_a,
     }
     __syncthreads();
     if (threadIdx.x == 0) {
+        uint32_t total = 0;
+#pragma unroll
+        for (int i = 0; i < kMaxCopies; ++i) total += c[i].bytes;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                     :: "r"(bar), "r"(2 * bytes) : "memory");
-        asm volatile(
-            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-            :: "r"(smem_addr(dst_a)), "l"(src_a), "r"(bytes), "r"(bar) : "memory");
-        asm volatile(
-            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-            :: "r"(smem_addr(dst_b)), "l"(src_b), "r"(bytes), "r"(bar) : "memory");
+                     :: "r"(bar), "r"(total) : "memory");
+#pragma unroll
+        for (int i = 0; i < kMaxCopies; ++i)
+            if (c[i].bytes)
+                asm volatile(
+                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                    :: "r"(smem_addr(c[i].dst)), "l"(c[i].src), "r"(c[i].bytes), "r"(bar) : "memory");
     }
     // each try_wait already blocks for a bounded, implementation-defined time
     bool ok = mbar_poll(bar, 0, 1 << 16);
@@ -63,6 +68,14 @@ __device__ __forceinline__ bool stage_two_tables(uint64_t *bar_ptr, void *dst_a,
     // the block must agree: a table that one thread could not see is read from global by all
     ok = __syncthreads_and(ok);
     return ok;
+}
+
+__device__ __forceinline__ bool stage_two_tables(uint64_t *bar_ptr, void *dst_a, const void *src_a,
+                                                 void *dst_b, const void *src_b, uint32_t bytes,
+                                                 int32_t *status)
+{
+    const StageCopy c[kMaxCopies] = {{dst_a, src_a, bytes}, {dst_b, src_b, bytes}, {nullptr, nullptr, 0}, {nullptr, nullptr, 0}};
+    return stage_tables(bar_ptr, c, status);
 }
 
 }  // namespace distsim
