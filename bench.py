@@ -408,7 +408,7 @@ def other_workloads(E, ctx, torch, dev, peaks):
 
 def profile_case(name):
     """Small, bounded invocations for profiler captures (no timing, no JSON line):
-    eval1  - evaluation of a 2 M-candidate slice of the 64-device workload (pp = 16 rows)
+    eval1  - evaluation of a 2 M-candidate slice of the 64-device workload (a pp = 16 row)
     eval3  - evaluation of the whole 256-device MoE workload (650 k candidates)
     emit4  - emission of 16 of the fastest candidates of the 1024-device workload (~1.3 GB)"""
     import torch
@@ -419,7 +419,14 @@ def profile_case(name):
         w = W.config1() if name == "eval1" else W.config3()
         E.distsim_load_event_table(ctx, w.table)
         n = E.distsim_set_space(ctx, w.space)
-        first, count = (n - 2_000_000, 2_000_000) if name == "eval1" else (0, n)
+        first, count = 0, n
+        if name == "eval1":
+            # two whole entries (m = 16 and 32) of the (mp = 1, pp = 16) row: 1.96 M candidates
+            off = 0
+            for mp, pp, dp, ms, parts, n_sched in W.space_shape(w.table, w.space):
+                if (mp, pp) == (1, 16):
+                    first, count = off + 4 * parts * n_sched, 2 * parts * n_sched
+                off += len(ms) * parts * n_sched
         batch = torch.empty(count, dtype=torch.int64, device="cuda")
         for _ in range(3):
             E.distsim_eval_strategies(ctx, first, count, batch)

@@ -168,6 +168,9 @@ int distsim_argmin(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, in
  * The k fastest candidates of a range, ascending by (batch time, index).
  *   d_indices [k] out (candidate indices, first + i);  d_times [k] out, nullable.
  * Requires 1 <= k <= min(count, 4096).  Asynchronous on `stream`.
+ * distsim_argmin and distsim_topk assume that d_batch_ns holds batch times produced by
+ * distsim_eval_strategies for the current table and space (they use the load-time upper bound
+ * on any batch time to skip empty high-order bits).
  */
 int distsim_topk(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int64_t first,
                  int64_t count, int32_t k, int64_t *d_indices, int64_t *d_times);

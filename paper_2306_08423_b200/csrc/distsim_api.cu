@@ -468,7 +468,7 @@ int distsim_topk(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int6
     if (k < 1 || k > 4096 || k > count) return fail(ctx, DISTSIM_E_ARG, "k must be in [1, min(count, 4096)]");
     if (int rc = set_device(ctx)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    launch_topk(s, d_batch_ns, first, count, k, ctx->select_scratch(), d_indices, d_times, &ctx->launches);
+    launch_topk(s, d_batch_ns, first, count, k, ctx->time_bound, ctx->select_scratch(), d_indices, d_times, &ctx->launches);
     CU(cudaGetLastError(), "top-k launch");
     return DISTSIM_OK;
 }

@@ -188,6 +188,7 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
                   int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */)
 {
     extern __shared__ __align__(16) int64_t tmpl[];     // [rf*5] forward, then [rb*5] backward
+    __shared__ int64_t rep_off_s[kTileReplicas];
     const int i = blockIdx.y;
     const EmitPlan &p = plans[i];
     if (!p.ok) return;
@@ -232,6 +233,19 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
             if (ex) { w[0] = DISTSIM_A2A_B; w[1] = l; w[2] = 0; w[3] = t; t += en.a2a; w[4] = t; }
         }
     }
+    // word offset of every replica (r, q) of this tile relative to replica 0 of the stage
+    const int rep0 = rc * kTileReplicas;
+    const int n_rep = min(reps, rep0 + kTileReplicas) - rep0;
+    if (threadIdx.x >= 32 && threadIdx.x < 32 + kTileReplicas) {
+        const int k = threadIdx.x - 32;
+        int64_t off = 0;
+        if (k < n_rep) {
+            const int rep = rep0 + k;
+            const int r = rep / p.mp, q = rep - r * p.mp;
+            off = (int64_t)r * p.mp * p.stage_rec_prefix[pp] * 5 + (int64_t)q * p.stage_recs[d] * 5;
+        }
+        rep_off_s[k] = off;
+    }
     if (threadIdx.x == 0) {
         if (d < pp - 1) {
             int64_t *w = tf + (int64_t)(rf - 1) * 5;
@@ -249,10 +263,10 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     // ---- stream the items of this tile -------------------------------------------------
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     const int s_end = min(2 * m, (ic + 1) * kTileItems);
-    const int rep0 = rc * kTileReplicas, rep1 = min(reps, rep0 + kTileReplicas);
-    const int64_t stage_words = p.stage_recs[d] * 5;                    // one device of this stage
-    const int64_t replica_words = (int64_t)p.mp * p.stage_rec_prefix[pp] * 5;   // one whole replica r
-    const int64_t stage_base = (p.rec_base + (int64_t)p.mp * p.stage_rec_prefix[d]) * 5;
+    int64_t roff[kTileReplicas];                     // word offset of each replica of this tile
+#pragma unroll
+    for (int k = 0; k < kTileReplicas; ++k) roff[k] = rep_off_s[k];
+    int64_t *stage_out = out + (p.rec_base + (int64_t)p.mp * p.stage_rec_prefix[d]) * 5;
     const int64_t *starts = op_start + (int64_t)i * op_words_per_cand + (int64_t)d * 2 * m;
     for (int s = ic * kTileItems + warp; s < s_end; s += n_warps) {
         bool bwd; int j, nf, nb;
@@ -260,16 +274,16 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         const int64_t t0 = starts[s];
         const int64_t *src = bwd ? tb : tf;
         const int n_words = (bwd ? rb : rf) * 5;
-        const int64_t item_off = ((int64_t)nf * rf + (int64_t)nb * rb) * 5;
+        int64_t *item_out = stage_out + ((int64_t)nf * rf + (int64_t)nb * rb) * 5;
         int field = lane % 5;
         for (int w = lane; w < n_words; w += 32) {
             int64_t val = src[w];
             val += field == 2 ? (int64_t)j : (field >= 3 ? t0 : 0);
             field += 2; if (field >= 5) field -= 5;                      // (w + 32) mod 5
-            for (int rep = rep0; rep < rep1; ++rep) {
-                const int r = rep / p.mp, q = rep - r * p.mp;
-                out[stage_base + (int64_t)r * replica_words + (int64_t)q * stage_words + item_off + w] = val;
-            }
+            int64_t *dst = item_out + w;
+#pragma unroll
+            for (int k = 0; k < kTileReplicas; ++k)
+                if (k < n_rep) __stcs(dst + roff[k], val);
         }
     }
 }
@@ -321,6 +335,7 @@ emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *_
     const int64_t replica_words = (int64_t)p.mp * p.stage_rec_prefix[p.pp] * 5;
     const int64_t base = (p.rec_base + (int64_t)p.mp * p.stage_rec_prefix[d]) * 5 +
                          (int64_t)p.m * (p.rf[d] + p.rb[d]) * 5;
+    const int r0 = rep0 / p.mp, q0 = rep0 - r0 * p.mp;
     for (int64_t w = threadIdx.x; w < kb * 5; w += blockDim.x) {
         const int64_t k = w / 5;
         const int field = (int)(w - k * 5);
@@ -344,9 +359,12 @@ emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *_
             }
             val = field == 3 ? start : start + dur;
         }
+        int r = r0, q = q0;
+        int64_t *dst = out + base + (int64_t)r * replica_words + (int64_t)q * stage_words + w;
         for (int rep = rep0; rep < rep1; ++rep) {
-            const int r = rep / p.mp, q = rep - r * p.mp;
-            out[base + (int64_t)r * replica_words + (int64_t)q * stage_words + w] = val;
+            __stcs(dst, val);
+            dst += stage_words;
+            if (++q == p.mp) { q = 0; ++r; dst = out + base + (int64_t)r * replica_words + w; }
         }
     }
 }

@@ -116,8 +116,10 @@ struct SelectScratch {
 // d_result[0] = smallest time, d_result[1] = its smallest position in `batch`.
 void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t time_bound,
                    const SelectScratch &sc, int64_t *d_result, int64_t *launches);
+// time_bound: an upper bound on every element of `batch` (INT64_MAX if unknown).
 void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
-                 const SelectScratch &sc, int64_t *d_indices, int64_t *d_times, int64_t *launches);
+                 int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
+                 int64_t *launches);
 
 // ---- emission (emit_kernels.cu) --------------------------------------------------------
 struct EmitPlan {                    // per selected candidate, written by the planning kernel

@@ -85,7 +85,7 @@ __global__ void argmin_unpack_kernel(const u64 *key, int idx_bits, int packed, i
 // Radix select, most significant byte first: first on the time, then on the index among the
 // elements whose time equals the threshold.  `rank` is the rank still to resolve inside the
 // current group; blocks_done counts finished blocks of a pass; cursor is the output cursor.
-struct SelState { u64 tprefix, tmask, rank, iprefix, imask, blocks_done, cursor, pad; };
+struct SelState { u64 tprefix, tmask, rank, iprefix, imask, blocks_done, cursor, skip_index; };
 
 template <bool kIndexPhase>
 __global__ void __launch_bounds__(kSelThreads)
@@ -93,6 +93,8 @@ radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, u64 *hist
 {
     __shared__ unsigned int sh[256];
     __shared__ bool last;
+    // no ties at the threshold time: every element equal to it is wanted, no index pass needed
+    if (kIndexPhase && st->skip_index) return;
     for (int i = threadIdx.x; i < 256; i += blockDim.x) sh[i] = 0;
     __syncthreads();
     const u64 tprefix = st->tprefix, tmask = st->tmask, iprefix = st->iprefix, imask = st->imask;
@@ -116,14 +118,18 @@ radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, u64 *hist
     // the last block to finish picks the bin that holds the wanted rank
     __threadfence();
     if (threadIdx.x == 0) {
-        u64 rank = st->rank, cum = 0;
+        u64 rank = st->rank, cum = 0, in_bin = 0;
         int bin = 255;
         for (int b = 0; b < 256; ++b) {
             const u64 h = *((volatile u64 *)&hist[b]);
-            if (rank < cum + h) { bin = b; break; }
+            if (rank < cum + h) { bin = b; in_bin = h; break; }
             cum += h;
         }
         st->rank = rank - cum;
+        if (!kIndexPhase && shift == 0 && in_bin == rank - cum + 1) {
+            // the elements equal to the threshold time are exactly the ones still needed
+            st->skip_index = 1; st->iprefix = ~0ull;
+        }
         if (kIndexPhase) { st->iprefix = iprefix | ((u64)bin << shift); st->imask = imask | (255ull << shift); }
         else { st->tprefix = tprefix | ((u64)bin << shift); st->tmask = tmask | (255ull << shift); }
         st->blocks_done = 0;
@@ -226,7 +232,8 @@ void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t 
 }
 
 void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
-                 const SelectScratch &sc, int64_t *d_indices, int64_t *d_times, int64_t *launches)
+                 int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
+                 int64_t *launches)
 {
     static bool attr_set = false;
     const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
@@ -243,7 +250,9 @@ void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t co
     sel_init_kernel<<<1, 256, 0, s>>>(st, sc.hist, k);
     ++*launches;
     const int g = grid_for(count);
-    for (int shift = 56; shift >= 0; shift -= 8) {
+    // bytes above the bound on any time are zero everywhere: start below them
+    const int tb = bits_for(time_bound);
+    for (int shift = ((tb + 7) / 8 - 1) * 8; shift >= 0; shift -= 8) {
         radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, shift, sc.hist, st);
         ++*launches;
     }
@@ -296,7 +305,7 @@ extern "C" int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int6
     int64_t launches = 0;
     // launch_topk begins by clearing the histogram, the selection state and the output cursor,
     // so whatever the previous call left in the array is never read
-    distsim::launch_topk(static_cast<cudaStream_t>(stream), d_batch_ns, first, count, k, sc,
+    distsim::launch_topk(static_cast<cudaStream_t>(stream), d_batch_ns, first, count, k, INT64_MAX, sc,
                          d_indices, d_times, &launches);
     return cudaGetLastError() == cudaSuccess ? DISTSIM_OK : DISTSIM_E_CUDA;
 }
