@@ -27,6 +27,22 @@ namespace distsim {
 
 constexpr int kThreadBlock = 128;
 
+// Tunables (overridable at compile time for experiments).
+#ifndef DS_MINBLOCKS_WIDE
+#define DS_MINBLOCKS_WIDE 3       // resident blocks per SM asked for when pp == 16
+#endif
+#ifndef DS_MINBLOCKS_NARROW
+#define DS_MINBLOCKS_NARROW 4     // ... when pp <= 8
+#endif
+#ifndef DS_UNROLL_MAIN
+#define DS_UNROLL_MAIN 1          // unroll factor of the steady-state wave loops
+#endif
+#ifndef DS_ROLLED_TRIANGLES
+#define DS_ROLLED_TRIANGLES 0     // 1: warm-up / drain waves as predicated rolled loops
+#endif
+#define DS_PRAGMA(x) _Pragma(#x)
+#define DS_UNROLL(n) DS_PRAGMA(unroll n)
+
 template <int PP>
 struct ThreadState {
     int64_t fop[PP], bop[PP];
@@ -38,14 +54,14 @@ __device__ __forceinline__ void run_gpipe(const ThreadState<PP> &c, int m, int64
 {
 #pragma unroll
     for (int d = 0; d < PP; ++d) free_at[d] = 0;
-#pragma unroll 2
+DS_UNROLL(DS_UNROLL_MAIN)
     for (int j = 0; j < m; ++j) {
         int64_t t = free_at[0] + c.fop[0];
         free_at[0] = t;
 #pragma unroll
         for (int d = 1; d < PP; ++d) { t = max64(t, free_at[d]) + c.fop[d]; free_at[d] = t; }
     }
-#pragma unroll 2
+DS_UNROLL(DS_UNROLL_MAIN)
     for (int j = 0; j < m; ++j) {
         int64_t t = free_at[PP - 1] + c.bop[PP - 1];
         free_at[PP - 1] = t;
@@ -112,12 +128,37 @@ __device__ __forceinline__ void run_1f1b(const ThreadState<PP> &c, int m, int64_
     int64_t last_f[PP];
 #pragma unroll
     for (int d = 0; d < PP; ++d) { free_at[d] = 0; last_f[d] = 0; }
+#if DS_ROLLED_TRIANGLES
+    // warm-up wave j covers the stages d < PP - j
+    for (int j = 0; j < min(PP, m); ++j) {
+        int64_t t = 0;
+#pragma unroll
+        for (int d = 0; d < PP; ++d)
+            if (d < PP - j) { t = (d == 0 ? free_at[0] : max64(t, free_at[d])) + c.fop[d]; free_at[d] = t; last_f[d] = t; }
+    }
+DS_UNROLL(DS_UNROLL_MAIN)
+    for (int i = 0; i < m - PP; ++i) wave_1f1b<PP, 0>(c, free_at, last_f);
+    // with k waves to go, stage d still runs a forward item iff PP - d < k
+    for (int k = min(PP, m); k >= 1; --k) {
+        int64_t t = 0;
+#pragma unroll
+        for (int d = PP - 1; d >= 0; --d) {
+            t = (d == PP - 1 ? free_at[d] : max64(t, free_at[d])) + c.bop[d];
+            free_at[d] = t;
+            if (PP - d < k) {
+                const int64_t f = (d == 0 ? free_at[0] : max64(last_f[d > 0 ? d - 1 : 0], free_at[d])) + c.fop[d];
+                free_at[d] = f; last_f[d] = f;
+            }
+        }
+    }
+#else
     WarmWaves<PP, 0>::run(c, m, free_at, last_f);
     // waves i = 0 .. m-PP-1: every stage still has a forward item to pair with its backward
-#pragma unroll 2
+DS_UNROLL(DS_UNROLL_MAIN)
     for (int i = 0; i < m - PP; ++i) wave_1f1b<PP, 0>(c, free_at, last_f);
     // the last min(PP, m) waves
     TailWaves<PP, PP>::run(c, m, free_at, last_f);
+#endif
 }
 
 // Shared-memory plan of a block (offsets in int64 words from the dynamic shared base).
@@ -128,7 +169,7 @@ struct ThreadKernelSmem {
 };
 
 template <int PP, bool kBusy>
-__global__ void __launch_bounds__(kThreadBlock)
+__global__ void __launch_bounds__(kThreadBlock, (PP >= 16 ? DS_MINBLOCKS_WIDE : DS_MINBLOCKS_NARROW))
 eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t first,
                    int e_begin, int e_end, int entries_per_thread, int64_t p_lo, int64_t p_hi,
                    int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out,
@@ -137,7 +178,8 @@ eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t 
     extern __shared__ __align__(16) int64_t dsm[];
     __shared__ __align__(8) uint64_t bar;
     __shared__ int64_t xs[PP][kThreadBlock];          // per thread, per stage: bucket-lane excess X
-    const Row row = v.rows[row_index];
+    __shared__ uint16_t cs[PP + 1][kThreadBlock];      // per thread: stage bounds c_0 .. c_PP
+    const Row &row = v.rows[row_index];
     const int lp = v.tc.lp;
     const int L1 = v.tc.n_layers + 1;
 
@@ -164,12 +206,11 @@ eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t 
     const int e0 = e_begin + (int)blockIdx.y * entries_per_thread;
     const int e1 = min(e_end, e0 + entries_per_thread);
 
-    // ---- decode the partition once ---------------------------------------------------------
-    int c[PP + 1];
-    c[0] = 0; c[PP] = v.tc.n_layers;
+    // ---- decode the partition once (bounds are parked in shared memory) ----------------------
+    cs[0][threadIdx.x] = 0; cs[PP][threadIdx.x] = (uint16_t)v.tc.n_layers;
     if (v.sc.partition_mode == 0) {
 #pragma unroll
-        for (int j = 1; j < PP; ++j) c[j] = (int)((int64_t)j * v.tc.n_layers / PP);
+        for (int j = 1; j < PP; ++j) cs[j][threadIdx.x] = (uint16_t)((int64_t)j * v.tc.n_layers / PP);
     } else {
         int64_t r = part;
         int cur = 0;
@@ -182,28 +223,29 @@ eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t 
                 r -= cnt;
                 ++cur;
             }
-            c[i] = cur;
+            cs[i][threadIdx.x] = (uint16_t)cur;
         }
     }
 
     const int64_t per_entry = row.n_part * row.n_sched;
     for (int e = e0; e < e1; ++e) {                     // e: entry index inside the row
-        const Entry en = v.entries[row.entry0 + e];
+        const Entry &en = v.entries[row.entry0 + e];
         const int64_t *pf = etf + (int64_t)e * lp;
         const int64_t *pb = etb + (int64_t)e * lp;
         const int m = en.m;
         ThreadState<PP> st;
 #pragma unroll
         for (int d = 0; d < PP; ++d) {
-            st.fop[d] = pf[c[d + 1]] - pf[c[d]] + (d < PP - 1 ? p2p_cost(row, en, d) : 0);
-            st.bop[d] = pb[c[d + 1]] - pb[c[d]] + (d > 0 ? p2p_cost(row, en, d - 1) : 0);
+            const int a = cs[d][threadIdx.x], ee = cs[d + 1][threadIdx.x];
+            st.fop[d] = pf[ee] - pf[a] + (d < PP - 1 ? p2p_cost(row, en, d) : 0);
+            st.bop[d] = pb[ee] - pb[a] + (d > 0 ? p2p_cost(row, en, d - 1) : 0);
         }
         // ---- bucket-lane excess per stage (schedule independent) ------------------------
 #pragma unroll
         for (int d = 0; d < PP; ++d) {
             int64_t x = 0;
             if (row.dp > 1) {
-                const int a = c[d], ee = c[d + 1];
+                const int a = cs[d][threadIdx.x], ee = cs[d + 1][threadIdx.x];
                 const int64_t *nbe = nbt + (int64_t)ee * L1;
                 const int64_t partial = tpt[(int64_t)ee * L1 + a];
                 const int64_t n_full = nbe[a];

@@ -14,7 +14,7 @@ import os
 import numpy as np
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libdistsim.so")
+LIB_PATH = os.environ.get("DISTSIM_LIBRARY", os.path.join(_PKG, "libdistsim.so"))   # another build of the same ABI
 MAX_PP = 64
 
 OK, E_ARG, E_STATE, E_RANGE, E_CAPACITY, E_OVERFLOW, E_CUDA, E_TIMEOUT, E_UNSUPPORTED = (
