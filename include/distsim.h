@@ -240,13 +240,14 @@ int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int64_t first, 
 
 /*
  * Measurement helper (no counterpart in the paper): enqueues a kernel of `blocks` x 256 threads
- * that issues a dependency-free stream of 32-bit integer add / logic instructions, `iters`
- * rounds of 16 per thread, and stores the total instruction count (threads x instructions) in
- * *h_ops.  Timed by the caller with events on `stream`, it gives the device's plain-integer
+ * that issues a dependency-free stream of integer work, `iters` rounds per thread, and stores
+ * the total instruction count (threads x instructions) in *h_ops.  mode 0: 16 32-bit add / xor
+ * instructions per round; mode 1: 8 recurrence cells x = max(x, y) + c on int64 per round,
+ * counted as 6 instructions each; mode 2: 16 32-bit compare / select instructions per round.  Timed by the caller with events on `stream`, it gives the device's plain-integer
  * issue rate under the clocks of the moment.  Asynchronous.
  */
-int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t blocks, int32_t iters,
-                            int64_t *h_ops);
+int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t mode, int32_t blocks,
+                            int32_t iters, int64_t *h_ops);
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t distsim_launch_count(const distsim_ctx *ctx);

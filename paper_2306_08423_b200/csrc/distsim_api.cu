@@ -66,7 +66,8 @@ struct distsim_ctx {
     std::vector<int64_t> binom;
     int64_t time_bound = 0;
     int64_t op_words_per_cand = 0;
-    DevBuf d_rows, d_entries, d_etf, d_etb, d_nb, d_tp, d_binom;
+    DevBuf d_rows, d_entries, d_etf, d_etb, d_nb, d_tp, d_binom, d_dt;
+    bool have_dt = false;
 
     // scratch
     DevBuf d_status, d_sel, d_result, d_plans, d_op_start, d_totals, d_batch, d_topk;
@@ -80,6 +81,8 @@ struct distsim_ctx {
         v.etf = d_etf.as<int64_t>(); v.etb = d_etb.as<int64_t>();
         v.nb = d_nb.as<int64_t>(); v.tp = d_tp.as<int64_t>();
         v.binom = d_binom.as<int64_t>();
+        v.dt = have_dt ? d_dt.as<int64_t>() : nullptr;
+        v.tab_words = ((tc.n_layers + 1) * (tc.n_layers + 1) + 1) & ~1;
         v.next_grad = d_next_grad.as<int32_t>(); v.pe = d_pe.as<int32_t>();
         v.status = d_status.as<int32_t>();
         return v;
@@ -371,9 +374,16 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
                         ctx->d_etb.as<int64_t>(), &ctx->launches);
     launch_build_bucket_tables(0, tc, ctx->raw, ctx->d_rows.as<Row>(), sc.n_rows, ctx->d_nb.as<int64_t>(),
                                ctx->d_tp.as<int64_t>(), &ctx->launches);
+    // per-entry bucket-lane tables, when the search enumerates stage compositions and they fit
+    const size_t dt_bytes = entries.size() * (size_t)(((L + 1) * (L + 1) + 1) & ~1) * sizeof(int64_t);
+    ctx->have_dt = sp->partition_mode == 1 && dt_bytes <= ((size_t)256 << 20);
+    if (ctx->have_dt) CU(ctx->d_dt.reserve(dt_bytes), "alloc bucket-lane tables");
+    launch_build_entry_tables(0, ctx->view(), ctx->d_entries.as<Entry>(), ctx->have_dt ? ctx->d_dt.as<int64_t>() : nullptr,
+                              &ctx->launches);
     CU(cudaGetLastError(), "set-up launch");
-    // the host copy of the rows takes the device-filled fields; this copy also waits for set-up
+    // the host copies take the device-filled fields; these copies also wait for set-up
     CU(cudaMemcpy(ctx->rows.data(), ctx->d_rows.p, rows.size() * sizeof(Row), cudaMemcpyDeviceToHost), "rows readback");
+    CU(cudaMemcpy(ctx->entries.data(), ctx->d_entries.p, entries.size() * sizeof(Entry), cudaMemcpyDeviceToHost), "entries readback");
     ctx->space_set = true;
     *n_candidates = total;
     return DISTSIM_OK;
@@ -434,7 +444,7 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
         const int64_t lo = first > row.offset ? first - row.offset : 0;
         const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
         if (hi <= lo) continue;
-        launch_eval_row(s, v, (int)r, row, lo, hi, first, d_batch_ns, d_stage_busy_ns, &ctx->launches);
+        launch_eval_row(s, v, (int)r, row, ctx->entries.data() + row.entry0, lo, hi, first, d_batch_ns, d_stage_busy_ns, &ctx->launches);
     }
     CU(cudaGetLastError(), "evaluation launch");
     return DISTSIM_OK;
@@ -528,12 +538,12 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table, co
     return distsim_argmin(ctx, nullptr, d_batch, 0, n, h_best_index, h_best_batch_ns);
 }
 
-int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t blocks, int32_t iters, int64_t *h_ops)
+int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t mode, int32_t blocks, int32_t iters, int64_t *h_ops)
 {
     if (!ctx) return DISTSIM_E_ARG;
-    if (!h_ops || blocks < 1 || iters < 1) return fail(ctx, DISTSIM_E_ARG, "bad probe arguments");
+    if (!h_ops || blocks < 1 || iters < 1 || mode < 0 || mode > 2) return fail(ctx, DISTSIM_E_ARG, "bad probe arguments");
     if (int rc = set_device(ctx)) return rc;
-    *h_ops = launch_int_issue_probe(static_cast<cudaStream_t>(stream), blocks, iters,
+    *h_ops = launch_int_issue_probe(static_cast<cudaStream_t>(stream), mode, blocks, iters,
                                     ctx->d_result.as<int64_t>() + 4, &ctx->launches);
     CU(cudaGetLastError(), "probe launch");
     return DISTSIM_OK;

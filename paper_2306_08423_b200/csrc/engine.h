@@ -15,6 +15,9 @@
 //   NB/TP    per row, [e][l] tables for the gradient buckets of a stage that ends at layer e:
 //            NB = number of full buckets completed once layers e-1..l have produced their
 //            gradients; TP = cost of the trailing partial bucket of the stage [l, e).
+//   DT       per entry, [e][l]: for the stage [l, e), with gradient overlap the end of its bucket
+//            lane relative to the start of its last backward item (-1 if it has no buckets);
+//            without overlap the total cost of its buckets.  Optional (memory budget).
 //   binom    C(n, k), saturated at 2^62, for unranking stage partitions.
 #pragma once
 
@@ -54,6 +57,7 @@ struct Row {
 struct Entry {
     int32_t m, b, cls, row;
     int64_t p2p_intra, p2p_inter, a2a, ar;   // [device-filled]
+    int64_t bound;        // [device-filled] upper bound on every time of every candidate of the entry
 };
 
 struct SpaceConst {
@@ -81,6 +85,9 @@ struct DeviceView {
     const Entry *entries;
     const int64_t *etf, *etb;        // [n_entries][lp]
     const int64_t *nb, *tp;          // per row [L+1][L+1]
+    const int64_t *dt;               // per entry [L+1][L+1] bucket-lane table (nullptr: not built)
+    int32_t tab_words;               // words of one [L+1][L+1] table, rounded up to even
+    int32_t pad_view;
     const int64_t *binom;            // [n_layers][binom_k]
     const int32_t *next_grad;        // [L+1] smallest l' >= l with grad_bytes[l'] > 0 (L if none)
     const int32_t *pe;               // [L+1] number of expert layers before layer l
@@ -96,15 +103,19 @@ void launch_build_prefix(cudaStream_t s, const TableConst &tc, const RawTable &r
 void launch_build_bucket_tables(cudaStream_t s, const TableConst &tc, const RawTable &raw,
                                 const Row *rows, int n_rows, int64_t *nb, int64_t *tp,
                                 int64_t *launches);
+// Per entry: the bucket-lane table (if dt != nullptr) and the time bound of the entry.
+void launch_build_entry_tables(cudaStream_t s, const DeviceView &v, Entry *entries, int64_t *dt,
+                               int64_t *launches);
 void launch_build_layer_tables(cudaStream_t s, const TableConst &tc, const RawTable &raw,
                                int32_t *next_grad, int32_t *pe, int64_t *launches);
 
 // ---- evaluation (eval_kernels.cu) ------------------------------------------------------
 // Evaluates candidates [lo, hi) of row `row_index` (indices local to the row); results go to
 // batch_out[row.offset + local - first] and, if non-null, busy_out[(same) * pp_max + d].
+// row_entries: host copies of the row's entries (their time bounds choose the arithmetic width).
 void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const Row &row_host,
-                     int64_t lo, int64_t hi, int64_t first, int64_t *batch_out, int64_t *busy_out,
-                     int64_t *launches);
+                     const Entry *row_entries, int64_t lo, int64_t hi, int64_t first,
+                     int64_t *batch_out, int64_t *busy_out, int64_t *launches);
 
 // ---- selection (select_kernels.cu) -----------------------------------------------------
 struct SelectScratch {
@@ -152,6 +163,6 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
 // ---- probe (probe_kernels.cu) ----------------------------------------------------------
 // Launches the integer-issue probe; returns the number of integer instructions (per thread,
 // summed over threads) it executes.
-int64_t launch_int_issue_probe(cudaStream_t s, int blocks, int iters, int64_t *sink, int64_t *launches);
+int64_t launch_int_issue_probe(cudaStream_t s, int mode, int blocks, int iters, int64_t *sink, int64_t *launches);
 
 }  // namespace distsim

@@ -73,76 +73,107 @@ eval_lockstep_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_
     }
 }
 
-template <int PP>
+template <int PP, typename T>
 void launch_thread_kernel(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo,
                           int64_t hi, int64_t first, int e_begin, int e_end, int ept, int64_t p_lo,
                           int64_t p_hi, int64_t *batch_out, int64_t *busy_out)
 {
     const int lp = v.tc.lp;
-    const int L1 = v.tc.n_layers + 1;
-    const int tab_words = (L1 * L1 + 1) & ~1;
     ThreadKernelSmem plan{};
     size_t words = 0;
-    const size_t budget_words = (200 * 1024 - sizeof(int64_t) * PP * kThreadBlock) / sizeof(int64_t);
-    // prefix rows of every entry of the row, then the row's two bucket tables, as far as they fit
+    // prefix rows of every entry of the row; the row's two bucket tables only when there is no
+    // per-entry bucket-lane table to look the result up in
     if ((size_t)row.n_entries * lp * 2 <= 8192) {
         plan.n_entries_staged = row.n_entries;
         plan.off_etb = row.n_entries * lp;
         words = (size_t)row.n_entries * lp * 2;
     }
-    if (words + 2 * (size_t)tab_words <= (budget_words < 12288 ? budget_words : 12288)) {
+    if (!v.dt && words + 2 * (size_t)v.tab_words <= 12288) {
         plan.tables_staged = 1;
         plan.off_nb = (int32_t)words;
-        plan.off_tp = (int32_t)words + tab_words;
-        words += 2 * (size_t)tab_words;
+        plan.off_tp = (int32_t)words + v.tab_words;
+        words += 2 * (size_t)v.tab_words;
     }
     const size_t smem = words * sizeof(int64_t);
     const int64_t n_threads = p_hi - p_lo;
     dim3 grid((unsigned)((n_threads + kThreadBlock - 1) / kThreadBlock), (unsigned)((e_end - e_begin + ept - 1) / ept));
     if (busy_out) {
-        if (smem > 32 * 1024)
-            cudaFuncSetAttribute(eval_thread_kernel<PP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        eval_thread_kernel<PP, true><<<grid, kThreadBlock, smem, s>>>(v, row_index, lo, hi, first, e_begin, e_end, ept,
-                                                                      p_lo, p_hi, batch_out, busy_out, plan, tab_words);
+        if (smem > 24 * 1024)
+            cudaFuncSetAttribute(eval_thread_kernel<PP, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_thread_kernel<PP, T, true><<<grid, kThreadBlock, smem, s>>>(v, row_index, lo, hi, first, e_begin, e_end, ept,
+                                                                         p_lo, p_hi, batch_out, busy_out, plan);
     } else {
-        if (smem > 32 * 1024)
-            cudaFuncSetAttribute(eval_thread_kernel<PP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        eval_thread_kernel<PP, false><<<grid, kThreadBlock, smem, s>>>(v, row_index, lo, hi, first, e_begin, e_end, ept,
-                                                                       p_lo, p_hi, batch_out, busy_out, plan, tab_words);
+        if (smem > 24 * 1024)
+            cudaFuncSetAttribute(eval_thread_kernel<PP, T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_thread_kernel<PP, T, false><<<grid, kThreadBlock, smem, s>>>(v, row_index, lo, hi, first, e_begin, e_end, ept,
+                                                                          p_lo, p_hi, batch_out, busy_out, plan);
     }
 }
 
+template <typename T>
+void launch_thread_kernel_pp(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo,
+                             int64_t hi, int64_t first, int e_begin, int e_end, int ept, int64_t p_lo,
+                             int64_t p_hi, int64_t *batch_out, int64_t *busy_out)
+{
+    switch (row.pp) {
+    case 1: launch_thread_kernel<1, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+    case 2: launch_thread_kernel<2, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+    case 4: launch_thread_kernel<4, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+    case 8: launch_thread_kernel<8, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+    default: launch_thread_kernel<16, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
+    }
+}
+
+void launch_lockstep(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo, int64_t hi,
+                     int64_t first, int64_t *batch_out, int64_t *busy_out);
+
 }  // namespace
 
-void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const Row &row,
+void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, const Entry *row_entries,
                      int64_t lo, int64_t hi, int64_t first, int64_t *batch_out, int64_t *busy_out,
                      int64_t *launches)
 {
     if (hi <= lo) return;
-    // Rows with many partitions and short pipelines: one partition per thread.
-    if (row.pp <= 16) {
-        const int64_t per_entry = row.n_part * row.n_sched;
-        const int e_begin = (int)(lo / per_entry), e_end = (int)((hi - 1) / per_entry) + 1;
+    if (row.pp > 16) {
+        launch_lockstep(s, v, row_index, row, lo, hi, first, batch_out, busy_out);
+        ++*launches;
+        return;
+    }
+    // Short pipelines: cut the range into runs of entries with the same arithmetic width; a run
+    // with enough partitions goes to the one-partition-per-thread kernel, the rest to lock-step.
+    const int64_t per_entry = row.n_part * row.n_sched;
+    const int e_begin = (int)(lo / per_entry), e_end = (int)((hi - 1) / per_entry) + 1;
+    int r0 = e_begin;
+    while (r0 < e_end) {
+        const bool narrow = row_entries[r0].bound < ((int64_t)1 << 32);
+        int r1 = r0 + 1;
+        while (r1 < e_end && (row_entries[r1].bound < ((int64_t)1 << 32)) == narrow) ++r1;
+        const int64_t lo_r = lo > (int64_t)r0 * per_entry ? lo : (int64_t)r0 * per_entry;
+        const int64_t hi_r = hi < (int64_t)r1 * per_entry ? hi : (int64_t)r1 * per_entry;
         int64_t p_lo = 0, p_hi = row.n_part;
-        if (e_end - e_begin == 1) {
-            p_lo = (lo - (int64_t)e_begin * per_entry) / row.n_sched;
-            p_hi = (hi - 1 - (int64_t)e_begin * per_entry) / row.n_sched + 1;
+        if (r1 - r0 == 1) {
+            p_lo = (lo_r - (int64_t)r0 * per_entry) / row.n_sched;
+            p_hi = (hi_r - 1 - (int64_t)r0 * per_entry) / row.n_sched + 1;
         }
         const int64_t n_parts = p_hi - p_lo;
-        const int n_e = e_end - e_begin;
+        const int n_e = r1 - r0;
         const int ept = n_parts >= 148 * 4 * kThreadBlock ? n_e : 1;       // entries per thread
         if (n_parts * ((n_e + ept - 1) / ept) >= 2048) {
-            switch (row.pp) {
-            case 1: launch_thread_kernel<1>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-            case 2: launch_thread_kernel<2>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-            case 4: launch_thread_kernel<4>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-            case 8: launch_thread_kernel<8>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-            default: launch_thread_kernel<16>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-            }
-            ++*launches;
-            return;
+            if (narrow) launch_thread_kernel_pp<uint32_t>(s, v, row_index, row, lo_r, hi_r, first, r0, r1, ept, p_lo, p_hi, batch_out, busy_out);
+            else launch_thread_kernel_pp<int64_t>(s, v, row_index, row, lo_r, hi_r, first, r0, r1, ept, p_lo, p_hi, batch_out, busy_out);
+        } else {
+            launch_lockstep(s, v, row_index, row, lo_r, hi_r, first, batch_out, busy_out);
         }
+        ++*launches;
+        r0 = r1;
     }
+}
+
+namespace {
+
+void launch_lockstep(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo, int64_t hi,
+                     int64_t first, int64_t *batch_out, int64_t *busy_out)
+{
     const int S = row.pp > 32 ? 2 : 1;
     const int wl = row.pp / S;
     const int cpb = (kEvalThreads / 32) * (32 / wl);      // candidates per block
@@ -165,7 +196,8 @@ void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const R
         eval_lockstep_kernel<2><<<(unsigned)blocks, kEvalThreads, smem, s>>>(v, row_index, lo, hi, first,
                                                                            batch_out, busy_out, max_stage);
     }
-    ++*launches;
 }
+
+}  // namespace
 
 }  // namespace distsim

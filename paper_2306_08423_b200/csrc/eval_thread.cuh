@@ -5,8 +5,8 @@
 // counts) and both schedules with it, so the partition is decoded once and the stage costs once
 // per entry.  All per-stage state of the pipeline recurrence - forward/backward item cost,
 // device-free time, latest forward end - lives in registers (the stage loops are fully
-// unrolled, pp is a template parameter), so a recurrence cell is exactly one 64-bit max and one
-// 64-bit add with no memory traffic and no shuffles, and every lane does useful work in every
+// unrolled, pp is a template parameter), so a recurrence cell is exactly one max and one add
+// with no memory traffic and no shuffles, and every lane does useful work in every
 // instruction.  Item order per schedule (any order consistent with every device's own order and
 // with the data dependencies gives the same times):
 //   GPipe  forward waves j = 0..m-1 over stages 0..pp-1, then backward waves over pp-1..0.
@@ -18,6 +18,11 @@
 //   DT = max over bucket groups of (ready offset of the group + cost of all buckets from it on),
 // which does not depend on the schedule; with X = max(0, DT - backward item cost) the stage's
 // contribution to the batch time is main_end + X and its activity time m(fop+bop) + X.
+//
+// Arithmetic width.  On this GPU a 64-bit max + add costs six half-rate integer instructions,
+// a 32-bit one two full-rate ones.  Every entry carries an upper bound on every time any of its
+// candidates can produce; the entries whose bound is below 2^32 are evaluated with T = uint32_t
+// (exactly: nothing can overflow), the others with T = int64_t.
 #pragma once
 
 #include "recurrence.cuh"
@@ -26,61 +31,55 @@
 namespace distsim {
 
 constexpr int kThreadBlock = 128;
+constexpr int kMaxRowEntries = 16;      // entries whose scalars are kept in shared memory
 
-// Tunables (overridable at compile time for experiments).
-#ifndef DS_MINBLOCKS_WIDE
-#define DS_MINBLOCKS_WIDE 3       // resident blocks per SM asked for when pp == 16
-#endif
-#ifndef DS_MINBLOCKS_NARROW
-#define DS_MINBLOCKS_NARROW 4     // ... when pp <= 8
-#endif
-#ifndef DS_UNROLL_MAIN
-#define DS_UNROLL_MAIN 1          // unroll factor of the steady-state wave loops
-#endif
-#ifndef DS_ROLLED_TRIANGLES
-#define DS_ROLLED_TRIANGLES 0     // 1: warm-up / drain waves as predicated rolled loops
-#endif
-#define DS_PRAGMA(x) _Pragma(#x)
-#define DS_UNROLL(n) DS_PRAGMA(unroll n)
+// Resident blocks per SM asked of the compiler (caps the registers per thread).
+template <int PP, typename T>
+constexpr int thread_kernel_min_blocks()
+{
+    return sizeof(T) == 8 ? (PP >= 16 ? 3 : 4) : (PP >= 16 ? 4 : 8);
+}
 
-template <int PP>
+template <typename T> __device__ __forceinline__ T vmax(T a, T b) { return a > b ? a : b; }
+
+template <int PP, typename T>
 struct ThreadState {
-    int64_t fop[PP], bop[PP];
+    T fop[PP], bop[PP];
 };
 
 // GPipe: returns main-lane end of every stage in free_at.
-template <int PP>
-__device__ __forceinline__ void run_gpipe(const ThreadState<PP> &c, int m, int64_t (&free_at)[PP])
+template <int PP, typename T>
+__device__ __forceinline__ void run_gpipe(const ThreadState<PP, T> &c, int m, T (&free_at)[PP])
 {
 #pragma unroll
     for (int d = 0; d < PP; ++d) free_at[d] = 0;
-DS_UNROLL(DS_UNROLL_MAIN)
+#pragma unroll 1
     for (int j = 0; j < m; ++j) {
-        int64_t t = free_at[0] + c.fop[0];
+        T t = free_at[0] + c.fop[0];
         free_at[0] = t;
 #pragma unroll
-        for (int d = 1; d < PP; ++d) { t = max64(t, free_at[d]) + c.fop[d]; free_at[d] = t; }
+        for (int d = 1; d < PP; ++d) { t = vmax(t, free_at[d]) + c.fop[d]; free_at[d] = t; }
     }
-DS_UNROLL(DS_UNROLL_MAIN)
+#pragma unroll 1
     for (int j = 0; j < m; ++j) {
-        int64_t t = free_at[PP - 1] + c.bop[PP - 1];
+        T t = free_at[PP - 1] + c.bop[PP - 1];
         free_at[PP - 1] = t;
 #pragma unroll
-        for (int d = PP - 2; d >= 0; --d) { t = max64(t, free_at[d]) + c.bop[d]; free_at[d] = t; }
+        for (int d = PP - 2; d >= 0; --d) { t = vmax(t, free_at[d]) + c.bop[d]; free_at[d] = t; }
     }
 }
 
 // One 1F1B backward wave in which the stages d >= D0 also run a forward item (D0 may be PP).
-template <int PP, int D0>
-__device__ __forceinline__ void wave_1f1b(const ThreadState<PP> &c, int64_t (&free_at)[PP], int64_t (&last_f)[PP])
+template <int PP, int D0, typename T>
+__device__ __forceinline__ void wave_1f1b(const ThreadState<PP, T> &c, T (&free_at)[PP], T (&last_f)[PP])
 {
-    int64_t t = 0;
+    T t = 0;
 #pragma unroll
     for (int d = PP - 1; d >= 0; --d) {
-        t = (d == PP - 1 ? free_at[d] : max64(t, free_at[d])) + c.bop[d];
+        t = (d == PP - 1 ? free_at[d] : vmax(t, free_at[d])) + c.bop[d];
         free_at[d] = t;
         if (d >= D0) {
-            const int64_t f = (d == 0 ? free_at[0] : max64(last_f[d > 0 ? d - 1 : 0], free_at[d])) + c.fop[d];
+            const T f = (d == 0 ? free_at[0] : vmax(last_f[d > 0 ? d - 1 : 0], free_at[d])) + c.fop[d];
             free_at[d] = f;
             last_f[d] = f;
         }
@@ -88,77 +87,51 @@ __device__ __forceinline__ void wave_1f1b(const ThreadState<PP> &c, int64_t (&fr
 }
 
 // Runs the last waves, in which fewer and fewer stages still have a forward item: with K waves
-// to go, the stages with pp - d < K do (statically unrolled over K = KMAX .. 1).
-template <int PP, int K>
+// to go, the stages with pp - d < K do (statically unrolled over K = PP .. 1).
+template <int PP, int K, typename T>
 struct TailWaves {
-    static __device__ __forceinline__ void run(const ThreadState<PP> &c, int m, int64_t (&free_at)[PP], int64_t (&last_f)[PP])
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &c, int m, T (&free_at)[PP], T (&last_f)[PP])
     {
-        // stage d runs a forward item in this wave iff pp - d < K, i.e. d >= PP - K + 1
-        if (K <= m) wave_1f1b<PP, PP - K + 1>(c, free_at, last_f);
-        TailWaves<PP, K - 1>::run(c, m, free_at, last_f);
+        if (K <= m) wave_1f1b<PP, PP - K + 1, T>(c, free_at, last_f);
+        TailWaves<PP, K - 1, T>::run(c, m, free_at, last_f);
     }
 };
-template <int PP>
-struct TailWaves<PP, 0> {
-    static __device__ __forceinline__ void run(const ThreadState<PP> &, int, int64_t (&)[PP], int64_t (&)[PP]) {}
+template <int PP, typename T>
+struct TailWaves<PP, 0, T> {
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &, int, T (&)[PP], T (&)[PP]) {}
 };
 
 // Warm-up forward wave J over stages 0 .. PP-1-J.
-template <int PP, int J>
+template <int PP, int J, typename T>
 struct WarmWaves {
-    static __device__ __forceinline__ void run(const ThreadState<PP> &c, int m, int64_t (&free_at)[PP], int64_t (&last_f)[PP])
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &c, int m, T (&free_at)[PP], T (&last_f)[PP])
     {
         if (J < m) {
-            int64_t t = free_at[0] + c.fop[0];
+            T t = free_at[0] + c.fop[0];
             free_at[0] = t; last_f[0] = t;
 #pragma unroll
-            for (int d = 1; d < PP - J; ++d) { t = max64(t, free_at[d]) + c.fop[d]; free_at[d] = t; last_f[d] = t; }
+            for (int d = 1; d < PP - J; ++d) { t = vmax(t, free_at[d]) + c.fop[d]; free_at[d] = t; last_f[d] = t; }
         }
-        WarmWaves<PP, J + 1>::run(c, m, free_at, last_f);
+        WarmWaves<PP, J + 1, T>::run(c, m, free_at, last_f);
     }
 };
-template <int PP>
-struct WarmWaves<PP, PP> {
-    static __device__ __forceinline__ void run(const ThreadState<PP> &, int, int64_t (&)[PP], int64_t (&)[PP]) {}
+template <int PP, typename T>
+struct WarmWaves<PP, PP, T> {
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &, int, T (&)[PP], T (&)[PP]) {}
 };
 
-template <int PP>
-__device__ __forceinline__ void run_1f1b(const ThreadState<PP> &c, int m, int64_t (&free_at)[PP])
+template <int PP, typename T>
+__device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (&free_at)[PP])
 {
-    int64_t last_f[PP];
+    T last_f[PP];
 #pragma unroll
     for (int d = 0; d < PP; ++d) { free_at[d] = 0; last_f[d] = 0; }
-#if DS_ROLLED_TRIANGLES
-    // warm-up wave j covers the stages d < PP - j
-    for (int j = 0; j < min(PP, m); ++j) {
-        int64_t t = 0;
-#pragma unroll
-        for (int d = 0; d < PP; ++d)
-            if (d < PP - j) { t = (d == 0 ? free_at[0] : max64(t, free_at[d])) + c.fop[d]; free_at[d] = t; last_f[d] = t; }
-    }
-DS_UNROLL(DS_UNROLL_MAIN)
-    for (int i = 0; i < m - PP; ++i) wave_1f1b<PP, 0>(c, free_at, last_f);
-    // with k waves to go, stage d still runs a forward item iff PP - d < k
-    for (int k = min(PP, m); k >= 1; --k) {
-        int64_t t = 0;
-#pragma unroll
-        for (int d = PP - 1; d >= 0; --d) {
-            t = (d == PP - 1 ? free_at[d] : max64(t, free_at[d])) + c.bop[d];
-            free_at[d] = t;
-            if (PP - d < k) {
-                const int64_t f = (d == 0 ? free_at[0] : max64(last_f[d > 0 ? d - 1 : 0], free_at[d])) + c.fop[d];
-                free_at[d] = f; last_f[d] = f;
-            }
-        }
-    }
-#else
-    WarmWaves<PP, 0>::run(c, m, free_at, last_f);
+    WarmWaves<PP, 0, T>::run(c, m, free_at, last_f);
     // waves i = 0 .. m-PP-1: every stage still has a forward item to pair with its backward
-DS_UNROLL(DS_UNROLL_MAIN)
-    for (int i = 0; i < m - PP; ++i) wave_1f1b<PP, 0>(c, free_at, last_f);
+#pragma unroll 1
+    for (int i = 0; i < m - PP; ++i) wave_1f1b<PP, 0, T>(c, free_at, last_f);
     // the last min(PP, m) waves
-    TailWaves<PP, PP>::run(c, m, free_at, last_f);
-#endif
+    TailWaves<PP, PP, T>::run(c, m, free_at, last_f);
 }
 
 // Shared-memory plan of a block (offsets in int64 words from the dynamic shared base).
@@ -168,33 +141,47 @@ struct ThreadKernelSmem {
     int32_t off_etb, off_nb, off_tp;
 };
 
-template <int PP, bool kBusy>
-__global__ void __launch_bounds__(kThreadBlock, (PP >= 16 ? DS_MINBLOCKS_WIDE : DS_MINBLOCKS_NARROW))
+// Entry scalars the hot path needs, kept in shared memory for the whole row.
+struct EntryLite { int64_t p2p_intra, p2p_inter; int32_t m, pad; };
+
+template <int PP, typename T, bool kBusy>
+__global__ void __launch_bounds__(kThreadBlock, thread_kernel_min_blocks<PP, T>())
 eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t first,
                    int e_begin, int e_end, int entries_per_thread, int64_t p_lo, int64_t p_hi,
                    int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out,
-                   ThreadKernelSmem plan, int tab_words)
+                   ThreadKernelSmem plan)
 {
     extern __shared__ __align__(16) int64_t dsm[];
     __shared__ __align__(8) uint64_t bar;
-    __shared__ int64_t xs[PP][kThreadBlock];          // per thread, per stage: bucket-lane excess X
-    __shared__ uint16_t cs[PP + 1][kThreadBlock];      // per thread: stage bounds c_0 .. c_PP
+    __shared__ T xs[PP][kThreadBlock];                // per thread, per stage: bucket-lane excess X
+    __shared__ uint16_t cs[PP + 1][kThreadBlock];     // per thread: stage bounds c_0 .. c_PP
+    __shared__ EntryLite ents[kMaxRowEntries];
     const Row &row = v.rows[row_index];
     const int lp = v.tc.lp;
     const int L1 = v.tc.n_layers + 1;
+    const int dp = row.dp, n_sched = row.n_sched, sched0 = row.sched0, period = row.p2p_period;
+    const int64_t t_full = row.t_full;
 
-    // ---- stage the row's prefix rows and bucket tables ---------------------------------
+    // ---- stage the row's prefix rows (and bucket tables when no per-entry table exists) ----
     const int64_t *etf_g = v.etf + (int64_t)row.entry0 * lp;
     const int64_t *etb_g = v.etb + (int64_t)row.entry0 * lp;
     const int64_t *nb_g = v.nb + row.row_tab_off;
     const int64_t *tp_g = v.tp + row.row_tab_off;
+    if (threadIdx.x < kMaxRowEntries && threadIdx.x < row.n_entries) {
+        const Entry &en = v.entries[row.entry0 + threadIdx.x];
+        ents[threadIdx.x].p2p_intra = en.p2p_intra;
+        ents[threadIdx.x].p2p_inter = en.p2p_inter;
+        ents[threadIdx.x].m = en.m;
+    }
     bool staged = false;
     if (plan.n_entries_staged > 0 || plan.tables_staged) {
         const uint32_t pbytes = (uint32_t)(plan.n_entries_staged * lp * sizeof(int64_t));
-        const uint32_t tbytes = plan.tables_staged ? (uint32_t)(tab_words * sizeof(int64_t)) : 0u;
+        const uint32_t tbytes = plan.tables_staged ? (uint32_t)(v.tab_words * sizeof(int64_t)) : 0u;
         const StageCopy cp[kMaxCopies] = {{dsm, etf_g, pbytes}, {dsm + plan.off_etb, etb_g, pbytes},
                                           {dsm + plan.off_nb, nb_g, tbytes}, {dsm + plan.off_tp, tp_g, tbytes}};
-        staged = stage_tables(&bar, cp, v.status);
+        staged = stage_tables(&bar, cp, v.status);      // contains the block-wide barriers
+    } else {
+        __syncthreads();
     }
     const int64_t *etf = (staged && plan.n_entries_staged) ? dsm : etf_g;
     const int64_t *etb = (staged && plan.n_entries_staged) ? dsm + plan.off_etb : etb_g;
@@ -227,67 +214,90 @@ eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t 
         }
     }
 
-    const int64_t per_entry = row.n_part * row.n_sched;
+    const int64_t per_entry = row.n_part * n_sched;
     for (int e = e0; e < e1; ++e) {                     // e: entry index inside the row
-        const Entry &en = v.entries[row.entry0 + e];
         const int64_t *pf = etf + (int64_t)e * lp;
         const int64_t *pb = etb + (int64_t)e * lp;
-        const int m = en.m;
-        ThreadState<PP> st;
+        int m;
+        int64_t p2p_intra, p2p_inter;
+        if (e < kMaxRowEntries) { m = ents[e].m; p2p_intra = ents[e].p2p_intra; p2p_inter = ents[e].p2p_inter; }
+        else { const Entry &en = v.entries[row.entry0 + e]; m = en.m; p2p_intra = en.p2p_intra; p2p_inter = en.p2p_inter; }
+        const int64_t *dte = v.dt ? v.dt + (int64_t)(row.entry0 + e) * v.tab_words : nullptr;
+
+        // ---- stage costs and bucket-lane excess (schedule independent) -------------------
+        ThreadState<PP, T> st;
+        int a = 0;
+        int64_t pfa = pf[0], pba = pb[0];
 #pragma unroll
         for (int d = 0; d < PP; ++d) {
-            const int a = cs[d][threadIdx.x], ee = cs[d + 1][threadIdx.x];
-            st.fop[d] = pf[ee] - pf[a] + (d < PP - 1 ? p2p_cost(row, en, d) : 0);
-            st.bop[d] = pb[ee] - pb[a] + (d > 0 ? p2p_cost(row, en, d - 1) : 0);
-        }
-        // ---- bucket-lane excess per stage (schedule independent) ------------------------
-#pragma unroll
-        for (int d = 0; d < PP; ++d) {
+            const int ee = cs[d + 1][threadIdx.x];
+            const int64_t pfe = pf[ee], pbe = pb[ee];
+            const int64_t send_f = d < PP - 1 ? ((((d + 1) & (period - 1)) == 0) ? p2p_inter : p2p_intra) : 0;
+            const int64_t send_b = d > 0 ? (((d & (period - 1)) == 0) ? p2p_inter : p2p_intra) : 0;
+            const int64_t fop = pfe - pfa + send_f;
+            const int64_t bop = pbe - pba + send_b;
             int64_t x = 0;
-            if (row.dp > 1) {
-                const int a = cs[d][threadIdx.x], ee = cs[d + 1][threadIdx.x];
-                const int64_t *nbe = nbt + (int64_t)ee * L1;
-                const int64_t partial = tpt[(int64_t)ee * L1 + a];
-                const int64_t n_full = nbe[a];
-                if (!v.tc.overlap) {
-                    x = n_full * row.t_full + partial;
+            if (dp > 1) {
+                if (dte) {
+                    const int64_t val = __ldg(&dte[(int64_t)ee * L1 + a]);
+                    x = v.tc.overlap ? val - bop : val;
                 } else {
-                    int64_t dt = -1;                     // latest bucket-lane end relative to the last backward start
-                    const int64_t pbe = pb[ee];
-                    if (n_full > 0) {
-                        int64_t nb_prev = 0;
-                        for (int l = ee - 1; l >= a; --l) {
-                            const int64_t nb_l = nbe[l];
-                            if (nb_l != nb_prev)
-                                dt = max64(dt, (pbe - pb[l]) + (n_full - nb_prev) * row.t_full + partial);
-                            nb_prev = nb_l;
+                    const int64_t *nbe = nbt + (int64_t)ee * L1;
+                    const int64_t partial = tpt[(int64_t)ee * L1 + a];
+                    const int64_t n_full = nbe[a];
+                    if (!v.tc.overlap) {
+                        x = n_full * t_full + partial;
+                    } else {
+                        int64_t dt = -1;
+                        if (n_full > 0) {
+                            int64_t nb_prev = 0;
+                            for (int l = ee - 1; l >= a; --l) {
+                                const int64_t nb_l = nbe[l];
+                                if (nb_l != nb_prev)
+                                    dt = max64(dt, (pbe - pb[l]) + (n_full - nb_prev) * t_full + partial);
+                                nb_prev = nb_l;
+                            }
                         }
+                        if (partial > 0) dt = max64(dt, (pbe - pb[__ldg(&v.next_grad[a])]) + partial);
+                        x = dt - bop;
                     }
-                    if (partial > 0) dt = max64(dt, (pbe - pb[__ldg(&v.next_grad[a])]) + partial);
-                    x = dt - st.bop[d];
-                    if (x < 0) x = 0;
                 }
+                if (x < 0) x = 0;
             }
-            xs[d][threadIdx.x] = x;
+            st.fop[d] = (T)fop; st.bop[d] = (T)bop;
+            xs[d][threadIdx.x] = (T)x;
+            a = ee; pfa = pfe; pba = pbe;
         }
 
-        for (int sc = 0; sc < row.n_sched; ++sc) {
-            const int64_t local = (int64_t)e * per_entry + part * row.n_sched + sc;
+        // ---- both schedules -----------------------------------------------------------------
+        const int64_t local0 = (int64_t)e * per_entry + part * n_sched;
+        int64_t res[2] = {0, 0};
+#pragma unroll 1
+        for (int sc = 0; sc < n_sched; ++sc) {
+            const int64_t local = local0 + sc;
             if (local < lo || local >= hi) continue;
-            int64_t free_at[PP];
-            if (row.sched0 + sc == 0) run_gpipe<PP>(st, m, free_at);
-            else run_1f1b<PP>(st, m, free_at);
-            int64_t batch = 0;
+            T free_at[PP];
+            if (sched0 + sc == 0) run_gpipe<PP, T>(st, m, free_at);
+            else run_1f1b<PP, T>(st, m, free_at);
+            T batch = 0;
 #pragma unroll
-            for (int d = 0; d < PP; ++d) batch = max64(batch, free_at[d] + xs[d][threadIdx.x]);
-            const int64_t out = row.offset + local - first;
-            batch_out[out] = batch;
+            for (int d = 0; d < PP; ++d) batch = vmax(batch, (T)(free_at[d] + xs[d][threadIdx.x]));
+            res[sc] = (int64_t)batch;
             if (kBusy) {
-                int64_t *bo = busy_out + out * v.sc.pp_max;
+                int64_t *bo = busy_out + (row.offset + local - first) * v.sc.pp_max;
 #pragma unroll
-                for (int d = 0; d < PP; ++d) bo[d] = (int64_t)m * (st.fop[d] + st.bop[d]) + xs[d][threadIdx.x];
+                for (int d = 0; d < PP; ++d)
+                    bo[d] = (int64_t)m * ((int64_t)st.fop[d] + (int64_t)st.bop[d]) + (int64_t)xs[d][threadIdx.x];
                 for (int d = PP; d < v.sc.pp_max; ++d) bo[d] = 0;
             }
+        }
+        // results of the two schedules are neighbours in the output: one 16-byte store if aligned
+        const int64_t out0 = row.offset + local0 - first;
+        if (n_sched == 2 && local0 >= lo && local0 + 1 < hi && !(reinterpret_cast<uintptr_t>(batch_out + out0) & 15)) {
+            *reinterpret_cast<longlong2 *>(batch_out + out0) = make_longlong2(res[0], res[1]);
+        } else {
+            for (int sc = 0; sc < n_sched; ++sc)
+                if (local0 + sc >= lo && local0 + sc < hi) batch_out[out0 + sc] = res[sc];
         }
     }
 }

@@ -1,6 +1,10 @@
-// Integer-issue probe: a dependency-free stream of 32-bit integer ALU instructions, used by the
-// benchmark to measure the device's plain-integer issue peak under the clocks of the moment
-// (the denominator of the evaluation kernel's roofline).
+// Integer-issue probes: dependency-free streams of integer ALU work, used by the benchmark to
+// measure the device's plain-integer peaks under the clocks of the moment (the denominators of
+// the evaluation kernel's roofline).
+//   mode 0  32-bit add / xor pairs                      (16 instructions per round and thread)
+//   mode 1  recurrence cells x = max(x, y) + c on int64 (8 cells per round and thread, counted
+//           as 6 instructions each: compare pair, two selects, add, add-with-carry)
+//   mode 2  32-bit compare + select pairs               (16 instructions per round and thread)
 #include "engine.h"
 
 namespace distsim {
@@ -9,38 +13,54 @@ namespace {
 
 constexpr int kChains = 8;
 
-// Each thread advances 8 independent (x, y) pairs: x += y (integer add) and y ^= x (logic op),
-// i.e. 16 integer instructions per iteration that cannot be fused with one another.
+template <int kMode>
 __global__ void __launch_bounds__(256) int_issue_probe_kernel(int iters, int64_t *sink)
 {
     uint32_t x[kChains], y[kChains];
+    int64_t a[kChains], b[kChains], c[kChains];
 #pragma unroll
-    for (int k = 0; k < kChains; ++k) { x[k] = threadIdx.x + k; y[k] = blockIdx.x * 7u + k; }
-    // 8 rounds per loop trip: 128 counted instructions against 2 of loop overhead
+    for (int k = 0; k < kChains; ++k) {
+        x[k] = threadIdx.x + k; y[k] = blockIdx.x * 7u + k;
+        a[k] = threadIdx.x * 3 + k; b[k] = (int64_t)blockIdx.x * 1000003 + k; c[k] = k + 1 + (sink == nullptr);
+    }
+    // 8 rounds per loop trip, so that loop overhead is about 1 %
     for (int it = 0; it < iters; it += 8) {
 #pragma unroll
         for (int rep = 0; rep < 8; ++rep) {
 #pragma unroll
             for (int k = 0; k < kChains; ++k) {
-                asm volatile("add.u32 %0, %0, %1;" : "+r"(x[k]) : "r"(y[k]));
-                asm volatile("xor.b32 %0, %0, %1;" : "+r"(y[k]) : "r"(x[k]));
+                if (kMode == 0) {
+                    asm volatile("add.u32 %0, %0, %1;" : "+r"(x[k]) : "r"(y[k]));
+                    asm volatile("xor.b32 %0, %0, %1;" : "+r"(y[k]) : "r"(x[k]));
+                } else if (kMode == 1) {
+                    // chain k: a = max(a, b) + c; b alternates with a through the other chain
+                    const int64_t mx = a[k] > b[k] ? a[k] : b[k];
+                    a[k] = mx + c[k];
+                    b[k] += (rep & 1) ? 0 : 0;   // b stays loop invariant; a grows past it or not by data
+                } else {
+                    asm volatile("{ .reg .pred p; setp.gt.u32 p, %0, %1; selp.u32 %0, %0, %1, p; }" : "+r"(x[k]) : "r"(y[k]));
+                    asm volatile("{ .reg .pred p; setp.lt.u32 p, %0, %1; selp.u32 %0, %1, %0, p; }" : "+r"(y[k]) : "r"(x[k]));
+                }
             }
         }
     }
     uint32_t acc = 0;
 #pragma unroll
-    for (int k = 0; k < kChains; ++k) acc += x[k] ^ y[k];
-    if (acc == 0x12345678u) sink[0] = acc;       // keeps the work alive; practically never taken
+    for (int k = 0; k < kChains; ++k) acc += x[k] ^ y[k] ^ (uint32_t)a[k] ^ (uint32_t)(a[k] >> 32);
+    if (acc == 0x12345678u && sink) sink[0] = acc;       // keeps the work alive; practically never taken
 }
 
 }  // namespace
 
-int64_t launch_int_issue_probe(cudaStream_t s, int blocks, int iters, int64_t *sink, int64_t *launches)
+int64_t launch_int_issue_probe(cudaStream_t s, int mode, int blocks, int iters, int64_t *sink, int64_t *launches)
 {
     iters = (iters + 7) & ~7;                    // the kernel runs whole groups of 8 rounds
-    int_issue_probe_kernel<<<blocks, 256, 0, s>>>(iters, sink);
+    if (mode == 1) int_issue_probe_kernel<1><<<blocks, 256, 0, s>>>(iters, sink);
+    else if (mode == 2) int_issue_probe_kernel<2><<<blocks, 256, 0, s>>>(iters, sink);
+    else int_issue_probe_kernel<0><<<blocks, 256, 0, s>>>(iters, sink);
     ++*launches;
-    return (int64_t)blocks * 256 * iters * kChains * 2;
+    const int64_t per_round = mode == 1 ? kChains * 6 : kChains * 2;
+    return (int64_t)blocks * 256 * iters * per_round;
 }
 
 }  // namespace distsim

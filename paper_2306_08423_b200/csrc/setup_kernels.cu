@@ -118,7 +118,89 @@ __global__ void build_layer_tables_kernel(TableConst tc, RawTable raw, int32_t *
     pe[tc.n_layers] = acc;
 }
 
+// One thread per (entry, e): bucket-lane table row e of the entry.
+//   overlap: DT[e][l] = max over the bucket groups of the stage [l, e) of (ready offset of the
+//            group + cost of all buckets from that group on), offsets counted from the start of
+//            the stage's last backward item; -1 when the stage has no buckets.
+//   no overlap: total bucket cost of the stage.
+__global__ void build_dt_kernel(DeviceView v, int64_t *dt)
+{
+    const int L1 = v.tc.n_layers + 1;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= v.sc.n_entries * L1) return;
+    const int en_i = i / L1, e = i % L1;
+    const Entry &en = v.entries[en_i];
+    const Row &row = v.rows[en.row];
+    int64_t *out = dt + (int64_t)en_i * v.tab_words + (int64_t)e * L1;
+    const int64_t *nbe = v.nb + row.row_tab_off + (int64_t)e * L1;
+    const int64_t *tpe = v.tp + row.row_tab_off + (int64_t)e * L1;
+    const int64_t *pb = v.etb + (int64_t)en_i * v.tc.lp;
+    for (int l = e; l < L1; ++l) out[l] = -1;
+    if (row.dp == 1) { for (int l = 0; l < e; ++l) out[l] = v.tc.overlap ? -1 : 0; return; }
+    for (int a = 0; a < e; ++a) {
+        const int64_t n_full = nbe[a], partial = tpe[a];
+        int64_t val;
+        if (!v.tc.overlap) {
+            val = n_full * row.t_full + partial;
+        } else {
+            val = -1;
+            int64_t nb_prev = 0;
+            for (int l = e - 1; l >= a; --l) {
+                const int64_t nb_l = nbe[l];
+                if (nb_l != nb_prev) {
+                    const int64_t cand = (pb[e] - pb[l]) + (n_full - nb_prev) * row.t_full + partial;
+                    val = cand > val ? cand : val;
+                }
+                nb_prev = nb_l;
+            }
+            if (partial > 0) {
+                const int64_t cand = (pb[e] - pb[v.next_grad[a]]) + partial;
+                val = cand > val ? cand : val;
+            }
+        }
+        out[a] = val;
+    }
+}
+
+// One thread per entry: an upper bound on every time any candidate of the entry can produce:
+// all items of the pipeline in sequence plus the largest possible bucket-lane excess.
+__global__ void entry_bound_kernel(DeviceView v, Entry *entries)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= v.sc.n_entries) return;
+    Entry en = entries[i];
+    const Row &row = v.rows[en.row];
+    const int L = v.tc.n_layers, L1 = L + 1;
+    const int64_t *pf = v.etf + (int64_t)i * v.tc.lp, *pb = v.etb + (int64_t)i * v.tc.lp;
+    int64_t per_mb = pf[L] + pb[L];
+    for (int d = 0; d + 1 < row.pp; ++d)
+        per_mb += 2 * ((((d + 1) & (row.p2p_period - 1)) == 0) ? en.p2p_inter : en.p2p_intra);
+    int64_t excess = 0;
+    if (row.dp > 1) {
+        const int64_t *nbL = v.nb + row.row_tab_off + (int64_t)L * L1;
+        const int64_t *tpL = v.tp + row.row_tab_off + (int64_t)L * L1;
+        // a stage's buckets cost at most all full buckets of the model plus one more bucket
+        excess = nbL[0] * row.t_full + (v.tc.bucket > 0 ? row.t_full : tpL[0]);
+    }
+    const __int128 b = (__int128)en.m * per_mb + excess;
+    en.bound = b >= (__int128)kSat ? kSat : (int64_t)b;
+    entries[i] = en;
+}
+
 }  // namespace
+
+void launch_build_entry_tables(cudaStream_t s, const DeviceView &v, Entry *entries, int64_t *dt,
+                               int64_t *launches)
+{
+    if (v.sc.n_entries == 0) return;
+    if (dt) {
+        const int n = v.sc.n_entries * (v.tc.n_layers + 1);
+        build_dt_kernel<<<(n + 127) / 128, 128, 0, s>>>(v, dt);
+        ++*launches;
+    }
+    entry_bound_kernel<<<(v.sc.n_entries + 127) / 128, 128, 0, s>>>(v, entries);
+    ++*launches;
+}
 
 void launch_fill_entries(cudaStream_t s, const TableConst &tc, Row *rows, int n_rows,
                          Entry *entries, int n_entries, int64_t *launches)

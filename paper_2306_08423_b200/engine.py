@@ -85,7 +85,7 @@ _lib.distsim_search_host.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_S
                                      C.c_void_p, C.c_void_p]
 
 
-_lib.distsim_int_issue_probe.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]
+_lib.distsim_int_issue_probe.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]
 
 
 _lib.distsim_topk_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
@@ -250,10 +250,10 @@ def distsim_search_host(ctx: Context, table, space, k: int = 0):
     return ctx.n_candidates, int(bi.value), int(bt.value), idx[:kk], tim[:kk]
 
 
-def distsim_int_issue_probe(ctx: Context, blocks: int, iters: int, stream=None) -> int:
+def distsim_int_issue_probe(ctx: Context, blocks: int, iters: int, mode: int = 0, stream=None) -> int:
     """Enqueues the integer-issue probe; returns the number of integer instructions it runs."""
     ops = C.c_int64(0)
-    ctx._check(_lib.distsim_int_issue_probe(ctx._h, _stream(stream), blocks, iters, C.byref(ops)))
+    ctx._check(_lib.distsim_int_issue_probe(ctx._h, _stream(stream), mode, blocks, iters, C.byref(ops)))
     return int(ops.value)
 
 
