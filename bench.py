@@ -31,10 +31,14 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+from paper_2306_08423_b200 import sharding  # noqa: E402
 from paper_2306_08423_b200 import workloads as W  # noqa: E402
 
 TOP_K = 1024
-INT_OPS_PER_CELL = 6      # int64 max (compare pair + two selects) + int64 add (add, add-with-carry)
+# 32-bit integer instructions a recurrence cell (one max + one add) needs: on int64 a compare
+# pair, two selects, add and add-with-carry; on uint32 (used where an entry's time bound is
+# below 2^32) one max and one add.
+INT_OPS_PER_CELL_64, INT_OPS_PER_CELL_32 = 6, 2
 RECORD_BYTES = 40
 
 
@@ -159,7 +163,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     peaks, peak_kind = measured_peaks()
 
-    w = W.config1(seed=1 + rank)
+    w = W.config1(seed=sharding.rank_seed(1, rank))
     table, space = w.table, w.space
     n_total, cells = W.count_candidates_and_cells(table, space)
     N = table.n_devices
@@ -272,10 +276,8 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
 
     # ---- max over ranks -----------------------------------------------------------------------
-    red = torch.tensor([total_ms, sum(e2e_times) / len(e2e_times)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(red, op=dist.ReduceOp.MAX)
-    total_ms_max, e2e_s_max = red.tolist()
+    total_ms_max = sharding.max_over_ranks(total_ms, device=dev)
+    e2e_s_max = sharding.max_over_ranks(sum(e2e_times) / len(e2e_times), device=dev)
     ms_per_step = total_ms_max / args.steps
     value = world * n_total / (ms_per_step * 1e-3)
 
@@ -285,21 +287,33 @@ def run_ours(args):
         return
 
     # ---- rooflines -----------------------------------------------------------------------------
-    # integer-issue peak, measured now with a dependency-free add/xor stream
-    pe0, pe1 = ev(), ev()
-    E.distsim_int_issue_probe(ctx, 148 * 16, 2000)
-    pe0.record(stream)
-    ops = E.distsim_int_issue_probe(ctx, 148 * 16, 20000)
-    pe1.record(stream)
-    torch.cuda.synchronize()
-    int_peak_gops = ops / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
+    # integer peaks, measured now with dependency-free instruction streams
+    def probe(mode):
+        pe0, pe1 = ev(), ev()
+        E.distsim_int_issue_probe(ctx, 148 * 16, 2000, mode)
+        pe0.record(stream)
+        ops = E.distsim_int_issue_probe(ctx, 148 * 16, 20000, mode)
+        pe1.record(stream)
+        torch.cuda.synchronize()
+        return ops / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
+    int_peak_gops = probe(0)
+    cell64_peak, cell32_peak, cmpsel_peak = probe(1) / 6, probe(3) / 2, probe(2)      # G cells/s, G instr/s
+    cells_all, cells_32 = E.distsim_space_cells(ctx)
+    assert cells_all == cells
     eval_s = statistics.mean(eval_ms) * 1e-3
-    achieved_gops = cells * INT_OPS_PER_CELL / eval_s / 1e9
-    roofline = {"bound": "alu", "kernel": "eval_lockstep_kernel", "achieved": achieved_gops, "peak": int_peak_gops,
-                "unit": "Gop/s (32-bit integer instructions; 6 per recurrence cell)",
+    alg_ops = cells_32 * INT_OPS_PER_CELL_32 + (cells - cells_32) * INT_OPS_PER_CELL_64
+    achieved_gops = alg_ops / eval_s / 1e9
+    # time the recurrence cells alone would take at the measured cell rates of this device
+    cell_floor_s = (cells_32 / cell32_peak + (cells - cells_32) / cell64_peak) / 1e9
+    roofline = {"bound": "alu", "kernel": "eval_thread_kernel (+ lock-step kernel on small rows)",
+                "achieved": achieved_gops, "peak": int_peak_gops,
+                "unit": "G 32-bit integer instr/s (2 per uint32 cell, 6 per int64 cell)",
                 "frac": achieved_gops / int_peak_gops, "traffic": None,
-                "peak_kind": "measured in this run (add/xor issue probe)",
-                "ms_per_launch_set": statistics.mean(eval_ms)}
+                "peak_kind": "measured in this run: dependency-free add/xor stream",
+                "cells": cells, "cells_32bit": cells_32, "ms_per_launch_set": statistics.mean(eval_ms),
+                "cell_rate_peaks_Gcells_per_s": {"uint32": cell32_peak, "int64": cell64_peak},
+                "compare_select_peak_Ginstr_per_s": cmpsel_peak,
+                "frac_of_cell_rate_floor": cell_floor_s / eval_s}
     emit_bytes = tot * RECORD_BYTES + TOP_K * N * 24 + 8
     emit_gbs = emit_bytes / (statistics.mean(emit_ms) * 1e-3) / 1e9
     roofline_emit = {"bound": "hbm", "kernel": "emit_items_kernel (+plan, scan, devices, buckets)",
@@ -310,7 +324,8 @@ def run_ours(args):
     line = {
         "metric": "strategy_candidates_per_sec", "value": value, "unit": "candidates/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int64 (exact uint32 arithmetic inside entries whose time bound is below 2^32)",
         "data": "synthetic",
         "config": {"workload": w.name, "candidates": n_total, "recurrence_cells": cells, "devices": N,
                    "layers": table.n_layers, "top_k_emitted": TOP_K, "records_emitted": tot,

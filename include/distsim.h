@@ -219,7 +219,7 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table,
  * block on the allocator's device-wide synchronisation, a process whose whole GPU memory has
  * already been handed to a pool, or a plug-in inside a host application that forbids it.
  * This variant needs no context and calls no allocator (neither CUDA's nor any library's):
- * its radix-select scratch is a fixed array of about 18 KB that is part of the library image,
+ * its radix-select scratch is a fixed array of about 33 KB that is part of the library image,
  * present on every GPU that has loaded the library until the process exits.
  *   d_batch_ns [count] in; d_indices [k] out (first + position), d_times [k] out, nullable;
  *   result ascending by (batch time, index), identical to distsim_topk's.
@@ -243,11 +243,19 @@ int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int64_t first, 
  * that issues a dependency-free stream of integer work, `iters` rounds per thread, and stores
  * the total instruction count (threads x instructions) in *h_ops.  mode 0: 16 32-bit add / xor
  * instructions per round; mode 1: 8 recurrence cells x = max(x, y) + c on int64 per round,
- * counted as 6 instructions each; mode 2: 16 32-bit compare / select instructions per round.  Timed by the caller with events on `stream`, it gives the device's plain-integer
+ * counted as 6 instructions each; mode 2: 16 32-bit compare / select instructions per round;
+ * mode 3: 8 recurrence cells on uint32 per round, counted as 2 instructions each.  Timed by the caller with events on `stream`, it gives the device's plain-integer
  * issue rate under the clocks of the moment.  Asynchronous.
  */
 int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t mode, int32_t blocks,
                             int32_t iters, int64_t *h_ops);
+
+/*
+ * Reporting helper: recurrence cells of the current space (a candidate has 2 m pp cells, one per
+ * schedule item), and how many of them belong to entries whose time bound is below 2^32, which
+ * the engine may evaluate in 32-bit arithmetic (exactly).  Host outputs.
+ */
+int distsim_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32bit);
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t distsim_launch_count(const distsim_ctx *ctx);

@@ -91,8 +91,8 @@ struct distsim_ctx {
     {
         SelectScratch s{};
         unsigned long long *base = d_sel.as<unsigned long long>();
-        s.key = base; s.hist = base + 8; s.sel_state = base + 8 + 256;
-        s.cand_time = reinterpret_cast<int64_t *>(base + 8 + 256 + 8);
+        s.key = base; s.hist = base + 8; s.sel_state = base + 8 + 2048;
+        s.cand_time = reinterpret_cast<int64_t *>(base + 8 + 2048 + 8);
         s.cand_idx = s.cand_time + 4096;
         return s;
     }
@@ -168,7 +168,7 @@ int distsim_create(distsim_ctx **out, int cuda_device)
     ctx->device = cuda_device;
     if (cudaSetDevice(cuda_device) != cudaSuccess ||
         ctx->d_status.reserve(64) != cudaSuccess ||
-        ctx->d_sel.reserve((8 + 256 + 8 + 2 * 4096) * sizeof(int64_t)) != cudaSuccess ||
+        ctx->d_sel.reserve((8 + 2048 + 8 + 2 * 4096) * sizeof(int64_t)) != cudaSuccess ||
         ctx->d_result.reserve(64) != cudaSuccess || ctx->d_totals.reserve(64) != cudaSuccess ||
         cudaMemset(ctx->d_status.p, 0, 64) != cudaSuccess ||
         cudaMallocHost(&ctx->h_pinned, 8 * sizeof(int64_t)) != cudaSuccess) {
@@ -384,6 +384,11 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     // the host copies take the device-filled fields; these copies also wait for set-up
     CU(cudaMemcpy(ctx->rows.data(), ctx->d_rows.p, rows.size() * sizeof(Row), cudaMemcpyDeviceToHost), "rows readback");
     CU(cudaMemcpy(ctx->entries.data(), ctx->d_entries.p, entries.size() * sizeof(Entry), cudaMemcpyDeviceToHost), "entries readback");
+    // the device's per-entry bounds are tighter than the host's estimate
+    int64_t bmax = 0;
+    for (const Entry &en : ctx->entries) bmax = en.bound > bmax ? en.bound : bmax;
+    if (bmax >= kSat) return fail(ctx, DISTSIM_E_OVERFLOW, "batch-time bound does not fit 62 bits");
+    ctx->time_bound = bmax;
     ctx->space_set = true;
     *n_candidates = total;
     return DISTSIM_OK;
@@ -538,10 +543,30 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table, co
     return distsim_argmin(ctx, nullptr, d_batch, 0, n, h_best_index, h_best_batch_ns);
 }
 
+int distsim_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32bit)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!h_cells || !h_cells_32bit) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
+    __int128 total = 0, narrow = 0;
+    for (const Row &row : ctx->rows)
+        for (int e = 0; e < row.n_entries; ++e) {
+            const Entry &en = ctx->entries[row.entry0 + e];
+            const __int128 c = (__int128)2 * en.m * row.pp * row.n_part * row.n_sched;
+            total += c;
+            // 32-bit arithmetic is used where the entry's time bound allows it and the row is
+            // evaluated by the one-partition-per-thread kernel
+            if (en.bound < ((int64_t)1 << 32) && row.pp <= 16) narrow += c;
+        }
+    *h_cells = total >= (__int128)kSat ? kSat : (int64_t)total;
+    *h_cells_32bit = narrow >= (__int128)kSat ? kSat : (int64_t)narrow;
+    return DISTSIM_OK;
+}
+
 int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t mode, int32_t blocks, int32_t iters, int64_t *h_ops)
 {
     if (!ctx) return DISTSIM_E_ARG;
-    if (!h_ops || blocks < 1 || iters < 1 || mode < 0 || mode > 2) return fail(ctx, DISTSIM_E_ARG, "bad probe arguments");
+    if (!h_ops || blocks < 1 || iters < 1 || mode < 0 || mode > 3) return fail(ctx, DISTSIM_E_ARG, "bad probe arguments");
     if (int rc = set_device(ctx)) return rc;
     *h_ops = launch_int_issue_probe(static_cast<cudaStream_t>(stream), mode, blocks, iters,
                                     ctx->d_result.as<int64_t>() + 4, &ctx->launches);

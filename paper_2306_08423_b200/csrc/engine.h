@@ -120,7 +120,7 @@ void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const R
 // ---- selection (select_kernels.cu) -----------------------------------------------------
 struct SelectScratch {
     unsigned long long *key;        // [2] packed / two-pass argmin keys
-    unsigned long long *hist;       // [256] radix histogram
+    unsigned long long *hist;       // [2048] radix histogram
     unsigned long long *sel_state;  // [8] radix-select state
     int64_t *cand_time, *cand_idx;  // [4096] selected pairs before sorting
 };

@@ -5,6 +5,8 @@
 //   mode 1  recurrence cells x = max(x, y) + c on int64 (8 cells per round and thread, counted
 //           as 6 instructions each: compare pair, two selects, add, add-with-carry)
 //   mode 2  32-bit compare + select pairs               (16 instructions per round and thread)
+//   mode 3  recurrence cells x = max(x, y) + c on uint32 (8 cells per round and thread, counted
+//           as 2 instructions each)
 #include "engine.h"
 
 namespace distsim {
@@ -36,7 +38,9 @@ __global__ void __launch_bounds__(256) int_issue_probe_kernel(int iters, int64_t
                     // chain k: a = max(a, b) + c; b alternates with a through the other chain
                     const int64_t mx = a[k] > b[k] ? a[k] : b[k];
                     a[k] = mx + c[k];
-                    b[k] += (rep & 1) ? 0 : 0;   // b stays loop invariant; a grows past it or not by data
+                } else if (kMode == 3) {
+                    const uint32_t mx = x[k] > y[k] ? x[k] : y[k];
+                    x[k] = mx + (uint32_t)c[k];
                 } else {
                     asm volatile("{ .reg .pred p; setp.gt.u32 p, %0, %1; selp.u32 %0, %0, %1, p; }" : "+r"(x[k]) : "r"(y[k]));
                     asm volatile("{ .reg .pred p; setp.lt.u32 p, %0, %1; selp.u32 %0, %1, %0, p; }" : "+r"(y[k]) : "r"(x[k]));
@@ -57,9 +61,10 @@ int64_t launch_int_issue_probe(cudaStream_t s, int mode, int blocks, int iters, 
     iters = (iters + 7) & ~7;                    // the kernel runs whole groups of 8 rounds
     if (mode == 1) int_issue_probe_kernel<1><<<blocks, 256, 0, s>>>(iters, sink);
     else if (mode == 2) int_issue_probe_kernel<2><<<blocks, 256, 0, s>>>(iters, sink);
+    else if (mode == 3) int_issue_probe_kernel<3><<<blocks, 256, 0, s>>>(iters, sink);
     else int_issue_probe_kernel<0><<<blocks, 256, 0, s>>>(iters, sink);
     ++*launches;
-    const int64_t per_round = mode == 1 ? kChains * 6 : kChains * 2;
+    const int64_t per_round = mode == 1 ? kChains * 6 : kChains * 2;   // modes 0, 2: 16 = 8 x 2; mode 3: 8 x 2
     return (int64_t)blocks * 256 * iters * per_round;
 }
 

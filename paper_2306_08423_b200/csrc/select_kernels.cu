@@ -82,34 +82,40 @@ __global__ void argmin_unpack_kernel(const u64 *key, int idx_bits, int packed, i
 }
 
 // ---- top-k ---------------------------------------------------------------------------------
-// Radix select, most significant byte first: first on the time, then on the index among the
-// elements whose time equals the threshold.  `rank` is the rank still to resolve inside the
-// current group; blocks_done counts finished blocks of a pass; cursor is the output cursor.
+// Radix select with 11-bit digits, most significant first: first on the time, then (only if the
+// threshold time is shared by more elements than are still wanted) on the index among the
+// elements that have it.  `rank` is the rank still to resolve inside the current group;
+// blocks_done counts finished blocks of a pass; cursor is the output cursor.
+constexpr int kRadixBits = 11;
+constexpr int kBins = 1 << kRadixBits;
 struct SelState { u64 tprefix, tmask, rank, iprefix, imask, blocks_done, cursor, skip_index; };
 
 template <bool kIndexPhase>
 __global__ void __launch_bounds__(kSelThreads)
-radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, u64 *hist, SelState *st)
+radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, int width, bool last_time_pass,
+                  u64 *hist, SelState *st)
 {
-    __shared__ unsigned int sh[256];
+    __shared__ unsigned int sh[kBins];
+    __shared__ u64 partial[kSelThreads];
     __shared__ bool last;
     // no ties at the threshold time: every element equal to it is wanted, no index pass needed
     if (kIndexPhase && st->skip_index) return;
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) sh[i] = 0;
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) sh[i] = 0;
     __syncthreads();
     const u64 tprefix = st->tprefix, tmask = st->tmask, iprefix = st->iprefix, imask = st->imask;
+    const unsigned dmask = (1u << width) - 1u;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
         const u64 x = (u64)t[i];
         if ((x & tmask) != tprefix) continue;
         if (kIndexPhase) {
             if (((u64)i & imask) != iprefix) continue;
-            atomicAdd(&sh[((u64)i >> shift) & 255u], 1u);
+            atomicAdd(&sh[(unsigned)((u64)i >> shift) & dmask], 1u);
         } else {
-            atomicAdd(&sh[(x >> shift) & 255u], 1u);
+            atomicAdd(&sh[(unsigned)(x >> shift) & dmask], 1u);
         }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) if (sh[i]) atomicAdd(&hist[i], (u64)sh[i]);
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) if (sh[i]) atomicAdd(&hist[i], (u64)sh[i]);
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) last = atomicAdd(&st->blocks_done, 1ull) == (u64)gridDim.x - 1;
@@ -117,30 +123,40 @@ radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, u64 *hist
     if (!last) return;
     // the last block to finish picks the bin that holds the wanted rank
     __threadfence();
+    constexpr int kPer = kBins / kSelThreads;
+    u64 mine = 0;
+    for (int k = 0; k < kPer; ++k) mine += *((volatile u64 *)&hist[threadIdx.x * kPer + k]);
+    partial[threadIdx.x] = mine;
+    __syncthreads();
     if (threadIdx.x == 0) {
         u64 rank = st->rank, cum = 0, in_bin = 0;
-        int bin = 255;
-        for (int b = 0; b < 256; ++b) {
-            const u64 h = *((volatile u64 *)&hist[b]);
-            if (rank < cum + h) { bin = b; in_bin = h; break; }
+        int chunk = kSelThreads - 1;
+        for (int c = 0; c < kSelThreads; ++c) {
+            if (rank < cum + partial[c]) { chunk = c; break; }
+            cum += partial[c];
+        }
+        int bin = chunk * kPer + kPer - 1;
+        for (int k = 0; k < kPer; ++k) {
+            const u64 h = *((volatile u64 *)&hist[chunk * kPer + k]);
+            if (rank < cum + h) { bin = chunk * kPer + k; in_bin = h; break; }
             cum += h;
         }
         st->rank = rank - cum;
-        if (!kIndexPhase && shift == 0 && in_bin == rank - cum + 1) {
+        if (!kIndexPhase && last_time_pass && in_bin == rank - cum + 1) {
             // the elements equal to the threshold time are exactly the ones still needed
             st->skip_index = 1; st->iprefix = ~0ull;
         }
-        if (kIndexPhase) { st->iprefix = iprefix | ((u64)bin << shift); st->imask = imask | (255ull << shift); }
-        else { st->tprefix = tprefix | ((u64)bin << shift); st->tmask = tmask | (255ull << shift); }
+        if (kIndexPhase) { st->iprefix = iprefix | ((u64)bin << shift); st->imask = imask | ((u64)dmask << shift); }
+        else { st->tprefix = tprefix | ((u64)bin << shift); st->tmask = tmask | ((u64)dmask << shift); }
         st->blocks_done = 0;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) hist[i] = 0;
 }
 
 __global__ void sel_init_kernel(SelState *st, u64 *hist, int k)
 {
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) hist[i] = 0;
     if (threadIdx.x == 0) { SelState z = {0, 0, (u64)(k - 1), 0, 0, 0, 0, 0}; *st = z; }
 }
 
@@ -250,15 +266,17 @@ void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t co
     sel_init_kernel<<<1, 256, 0, s>>>(st, sc.hist, k);
     ++*launches;
     const int g = grid_for(count);
-    // bytes above the bound on any time are zero everywhere: start below them
-    const int tb = bits_for(time_bound);
-    for (int shift = ((tb + 7) / 8 - 1) * 8; shift >= 0; shift -= 8) {
-        radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, shift, sc.hist, st);
+    // bits above the bound on any time are zero everywhere: start below them
+    const int tb = bits_for(time_bound) > 0 ? bits_for(time_bound) : 1;
+    for (int shift = ((tb + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
+        const int width = tb - shift < kRadixBits ? tb - shift : kRadixBits;
+        radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, shift, width, shift == 0, sc.hist, st);
         ++*launches;
     }
-    const int ib = bits_for(count - 1);
-    for (int shift = ((ib + 7) / 8 - 1) * 8; shift >= 0; shift -= 8) {
-        radix_pass_kernel<true><<<g, kSelThreads, 0, s>>>(batch, count, shift, sc.hist, st);
+    const int ib = bits_for(count - 1) > 0 ? bits_for(count - 1) : 1;
+    for (int shift = ((ib + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
+        const int width = ib - shift < kRadixBits ? ib - shift : kRadixBits;
+        radix_pass_kernel<true><<<g, kSelThreads, 0, s>>>(batch, count, shift, width, false, sc.hist, st);
         ++*launches;
     }
     collect_kernel<<<g, kSelThreads, 0, s>>>(batch, count, st, k, sc.cand_time, sc.cand_idx);
@@ -274,7 +292,7 @@ void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t co
 // call neither needs a context nor touches the CUDA allocator.
 namespace {
 
-constexpr int kStaticWords = 8 + 256 + 8 + 2 * DISTSIM_TOPK_STATIC_MAX_K;      // 64-bit words
+constexpr int kStaticWords = 8 + distsim::kBins + 8 + 2 * DISTSIM_TOPK_STATIC_MAX_K;    // 64-bit words
 static __device__ __align__(256) unsigned long long g_topk_static_scratch[kStaticWords];
 
 constexpr int kMaxDevices = 64;
@@ -299,8 +317,8 @@ extern "C" int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int6
     }
     unsigned long long *base = g_static_scratch_addr[dev];
     distsim::SelectScratch sc{};
-    sc.key = base; sc.hist = base + 8; sc.sel_state = base + 8 + 256;
-    sc.cand_time = reinterpret_cast<int64_t *>(base + 8 + 256 + 8);
+    sc.key = base; sc.hist = base + 8; sc.sel_state = base + 8 + distsim::kBins;
+    sc.cand_time = reinterpret_cast<int64_t *>(base + 8 + distsim::kBins + 8);
     sc.cand_idx = sc.cand_time + DISTSIM_TOPK_STATIC_MAX_K;
     int64_t launches = 0;
     // launch_topk begins by clearing the histogram, the selection state and the output cursor,

@@ -24,7 +24,7 @@ EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error", "distsim_l
            "distsim_load_event_table", "distsim_set_space", "distsim_decode",
            "distsim_eval_strategies", "distsim_argmin", "distsim_topk",
            "distsim_emit_timelines", "distsim_search_host", "distsim_int_issue_probe",
-           "distsim_topk_static")
+           "distsim_topk_static", "distsim_space_cells")
 TOPK_STATIC_MAX_K = 1024
 
 if not os.path.exists(LIB_PATH):
@@ -90,6 +90,9 @@ _lib.distsim_int_issue_probe.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_
 
 _lib.distsim_topk_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
                                      C.c_void_p, C.c_void_p]
+
+
+_lib.distsim_space_cells.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 
 
 def _np_ptr(a: np.ndarray):
@@ -276,3 +279,10 @@ def distsim_topk_static(d_batch_ns, first: int, count: int, k: int, d_indices, d
         raise DistsimError(rc, f"k = {k} exceeds the fixed scratch (at most {TOPK_STATIC_MAX_K})")
     if rc != OK:
         raise DistsimError(rc, "distsim_topk_static failed")
+
+
+def distsim_space_cells(ctx: Context):
+    """(recurrence cells of the space, cells the engine may evaluate in 32-bit arithmetic)."""
+    a, b = C.c_int64(0), C.c_int64(0)
+    ctx._check(_lib.distsim_space_cells(ctx._h, C.byref(a), C.byref(b)))
+    return int(a.value), int(b.value)
