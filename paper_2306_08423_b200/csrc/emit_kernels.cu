@@ -5,13 +5,15 @@
 //                        while recording every item's start time into scratch, count records.
 //   emit_scan_kernel     one block: exclusive scan of the per-candidate record totals.
 //   emit_devices_kernel  per (candidate, device): record offset, activity time, utilisation.
-//   emit_items_kernel    the bandwidth-bound part.  A block owns (candidate, stage, chunk of
-//                        items, chunk of replicas).  It builds the stage's forward and backward
-//                        item templates (records relative to the item's start) in shared memory
-//                        once, then each warp streams whole items: the flat int64 words of an
-//                        item are template word + {0, 0, microbatch, start, start}, written with
-//                        fully coalesced 8-byte stores to each of the stage's mp*dp replicas
-//                        (all replicas of a stage have identical lists).
+//   emit_items_kernel    the bandwidth-bound part.  A block owns (candidate, stage, run of
+//                        consecutive items, chunk of replicas).  It builds the stage's forward
+//                        and backward item templates (records relative to the item's start) in
+//                        shared memory once.  The run's records are contiguous in memory, so the
+//                        block walks the run as one flat stream of int64 words: word x belongs to
+//                        the item found by a search in the run's offset table, and its value is
+//                        template word + {0, 0, microbatch, start, start}.  Consecutive threads
+//                        write consecutive words (full 256-byte warp stores whatever the item
+//                        size) to each of the stage's mp*dp replicas, whose lists are identical.
 //   emit_buckets_kernel  gradient-bucket records of every stage.
 #include "recurrence.cuh"
 
@@ -20,7 +22,8 @@ namespace distsim {
 namespace {
 
 constexpr int kItemThreads = 256;
-constexpr int kTileItems = 32;      // schedule items per block
+constexpr int kMaxTileItems = 128;  // most schedule items per block (a plan picks its own count)
+constexpr int kTileWords = 16384;   // target size of a block's run, in int64 words per replica
 constexpr int kTileReplicas = 16;   // replicas per block
 
 __device__ __forceinline__ int find_row(const DeviceView &v, int64_t index)
@@ -85,6 +88,10 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
         for (int d = 0; d < row.pp; ++d) { plan->stage_rec_prefix[d] = acc; acc += plan->stage_recs[d]; }
         plan->stage_rec_prefix[row.pp] = acc;
         plan->rec_total = acc * row.mp * row.dp;
+        int widest = 1;
+        for (int d = 0; d < row.pp; ++d) widest = max(widest, plan->rf[d] + plan->rb[d]);
+        const int per_tile = kTileWords / ((widest * 5 + 1) / 2);      // average item: (rf + rb) / 2 records
+        plan->tile_items = max(8, min(kMaxTileItems, per_tile));
     }
 }
 
@@ -99,7 +106,7 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
     if (index < 0 || index >= v.sc.n_candidates) {
         if ((threadIdx.x & 31) == 0) {
             plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
-            plan->mp = 1; plan->dp = 1;
+            plan->mp = 1; plan->dp = 1; plan->tile_items = 8;
             atomicCAS(v.status, 0, DISTSIM_E_RANGE);
         }
         return;
@@ -133,7 +140,7 @@ __global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /*[2]: 
         plans[i].rec_base = acc; acc += plans[i].rec_total;
         if (plans[i].ok) {
             const int64_t reps = (int64_t)plans[i].mp * plans[i].dp;
-            const int64_t tiles = (int64_t)plans[i].pp * ((2 * plans[i].m + kTileItems - 1) / kTileItems) *
+            const int64_t tiles = (int64_t)plans[i].pp * ((2 * plans[i].m + plans[i].tile_items - 1) / plans[i].tile_items) *
                                   ((reps + kTileReplicas - 1) / kTileReplicas);
             mt = max64(mt, tiles);
         }
@@ -189,12 +196,17 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
 {
     extern __shared__ __align__(16) int64_t tmpl[];     // [rf*5] forward, then [rb*5] backward
     __shared__ int64_t rep_off_s[kTileReplicas];
+    __shared__ int64_t start_s[kMaxTileItems];          // start time of each item of the run
+    __shared__ int32_t ioff[kMaxTileItems + 1];         // word offset of each item inside the run
+    __shared__ int32_t meta_s[kMaxTileItems];           // micro-batch << 1 | is-backward
+    __shared__ int64_t run_base_s;                      // word offset of the run inside the stage stream
     const int i = blockIdx.y;
     const EmitPlan &p = plans[i];
     if (!p.ok) return;
-    const int m = p.m, pp = p.pp;
-    const int reps = p.mp * p.dp;
-    const int item_chunks = (2 * m + kTileItems - 1) / kTileItems;
+    const int m = p.m, pp = p.pp, sched = p.sched, mp = p.mp;
+    const int reps = mp * p.dp;
+    const int tile_items = p.tile_items;
+    const int item_chunks = (2 * m + tile_items - 1) / tile_items;
     const int rep_chunks = (reps + kTileReplicas - 1) / kTileReplicas;
     int tile = blockIdx.x;
     if (tile >= pp * item_chunks * rep_chunks) return;
@@ -202,35 +214,50 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     const int ic = tile % item_chunks;
     const int d = tile / item_chunks;
 
-    const Row row = v.rows[p.row];
-    const Entry en = v.entries[p.entry];
+    const Row &row = v.rows[p.row];
+    const Entry &en = v.entries[p.entry];
     const int a = p.bounds[d], e = p.bounds[d + 1];
     const int rf = p.rf[d], rb = p.rb[d];
     const int64_t *pf = v.etf + (int64_t)p.entry * v.tc.lp;
     const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
     const int64_t *f = v.raw.fwd + (int64_t)en.cls * v.tc.n_layers;
     const int64_t *g = v.raw.bwd + (int64_t)en.cls * v.tc.n_layers;
-    const int per_layer = row.mp > 1 ? 2 : 1;
+    const int row_mp = row.mp, row_dp = row.dp;
+    const int per_layer = row_mp > 1 ? 2 : 1;
+    const int64_t ar = en.ar, a2a = en.a2a;
     int64_t *tf = tmpl, *tb = tmpl + (int64_t)rf * 5;
 
     // ---- item templates: records relative to the item's start --------------------------
     for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
-        const bool ex = row.dp > 1 && v.raw.expert[l];
+        const bool ex = row_dp > 1 && v.raw.expert[l];
         {   // forward: layers ascending
-            const int r = (l - a) * per_layer + (row.dp > 1 ? v.pe[l] - v.pe[a] : 0);
+            const int r = (l - a) * per_layer + (row_dp > 1 ? v.pe[l] - v.pe[a] : 0);
             int64_t t = pf[l] - pf[a];
             int64_t *w = tf + (int64_t)r * 5;
             w[0] = DISTSIM_COMPUTE_F; w[1] = l; w[2] = 0; w[3] = t; t += f[l]; w[4] = t; w += 5;
-            if (row.mp > 1) { w[0] = DISTSIM_MP_AR_F; w[1] = l; w[2] = 0; w[3] = t; t += en.ar; w[4] = t; w += 5; }
-            if (ex) { w[0] = DISTSIM_A2A_F; w[1] = l; w[2] = 0; w[3] = t; t += en.a2a; w[4] = t; }
+            if (row_mp > 1) { w[0] = DISTSIM_MP_AR_F; w[1] = l; w[2] = 0; w[3] = t; t += ar; w[4] = t; w += 5; }
+            if (ex) { w[0] = DISTSIM_A2A_F; w[1] = l; w[2] = 0; w[3] = t; t += a2a; w[4] = t; }
         }
         {   // backward: layers descending
-            const int r = (e - 1 - l) * per_layer + (row.dp > 1 ? v.pe[e] - v.pe[l + 1] : 0);
+            const int r = (e - 1 - l) * per_layer + (row_dp > 1 ? v.pe[e] - v.pe[l + 1] : 0);
             int64_t t = pb[e] - pb[l + 1];
             int64_t *w = tb + (int64_t)r * 5;
             w[0] = DISTSIM_COMPUTE_B; w[1] = l; w[2] = 0; w[3] = t; t += g[l]; w[4] = t; w += 5;
-            if (row.mp > 1) { w[0] = DISTSIM_MP_AR_B; w[1] = l; w[2] = 0; w[3] = t; t += en.ar; w[4] = t; w += 5; }
-            if (ex) { w[0] = DISTSIM_A2A_B; w[1] = l; w[2] = 0; w[3] = t; t += en.a2a; w[4] = t; }
+            if (row_mp > 1) { w[0] = DISTSIM_MP_AR_B; w[1] = l; w[2] = 0; w[3] = t; t += ar; w[4] = t; w += 5; }
+            if (ex) { w[0] = DISTSIM_A2A_B; w[1] = l; w[2] = 0; w[3] = t; t += a2a; w[4] = t; }
+        }
+    }
+    // ---- the run: its items' start times, kinds, micro-batches and word offsets ------------
+    const int s0 = ic * tile_items;
+    const int n_items = min(2 * m, s0 + tile_items) - s0;
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTileItems) {
+        const int k = threadIdx.x - 64;
+        if (k < n_items) {
+            bool bwd; int j, nf, nb;
+            item_at(sched, pp, m, d, s0 + k, bwd, j, nf, nb);
+            start_s[k] = op_start[(int64_t)i * op_words_per_cand + (int64_t)d * 2 * m + s0 + k];
+            meta_s[k] = (j << 1) | (bwd ? 1 : 0);
+            if (k == 0) run_base_s = ((int64_t)nf * rf + (int64_t)nb * rb) * 5;
         }
     }
     // word offset of every replica (r, q) of this tile relative to replica 0 of the stage
@@ -241,8 +268,8 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         int64_t off = 0;
         if (k < n_rep) {
             const int rep = rep0 + k;
-            const int r = rep / p.mp, q = rep - r * p.mp;
-            off = (int64_t)r * p.mp * p.stage_rec_prefix[pp] * 5 + (int64_t)q * p.stage_recs[d] * 5;
+            const int r = rep / mp, q = rep - r * mp;
+            off = (int64_t)r * mp * p.stage_rec_prefix[pp] * 5 + (int64_t)q * p.stage_recs[d] * 5;
         }
         rep_off_s[k] = off;
     }
@@ -259,32 +286,34 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         }
     }
     __syncthreads();
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int k = 0; k < n_items; ++k) { ioff[k] = acc; acc += ((meta_s[k] & 1) ? rb : rf) * 5; }
+        ioff[n_items] = acc;
+    }
+    __syncthreads();
 
-    // ---- stream the items of this tile -------------------------------------------------
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    const int s_end = min(2 * m, (ic + 1) * kTileItems);
+    // ---- stream the run as flat words ---------------------------------------------------------
     int64_t roff[kTileReplicas];                     // word offset of each replica of this tile
 #pragma unroll
     for (int k = 0; k < kTileReplicas; ++k) roff[k] = rep_off_s[k];
-    int64_t *stage_out = out + (p.rec_base + (int64_t)p.mp * p.stage_rec_prefix[d]) * 5;
-    const int64_t *starts = op_start + (int64_t)i * op_words_per_cand + (int64_t)d * 2 * m;
-    for (int s = ic * kTileItems + warp; s < s_end; s += n_warps) {
-        bool bwd; int j, nf, nb;
-        item_at(p.sched, pp, m, d, s, bwd, j, nf, nb);
-        const int64_t t0 = starts[s];
-        const int64_t *src = bwd ? tb : tf;
-        const int n_words = (bwd ? rb : rf) * 5;
-        int64_t *item_out = stage_out + ((int64_t)nf * rf + (int64_t)nb * rb) * 5;
-        int field = lane % 5;
-        for (int w = lane; w < n_words; w += 32) {
-            int64_t val = src[w];
-            val += field == 2 ? (int64_t)j : (field >= 3 ? t0 : 0);
-            field += 2; if (field >= 5) field -= 5;                      // (w + 32) mod 5
-            int64_t *dst = item_out + w;
-#pragma unroll
-            for (int k = 0; k < kTileReplicas; ++k)
-                if (k < n_rep) __stcs(dst + roff[k], val);
+    int64_t *run_out = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + run_base_s;
+    const int total = ioff[n_items];
+    for (int x = threadIdx.x; x < total; x += blockDim.x) {
+        int lo = 0, hi = n_items - 1;                // the item holding word x: last k with ioff[k] <= x
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (ioff[mid] <= x) lo = mid; else hi = mid - 1;
         }
+        const int w = x - ioff[lo];
+        const int meta = meta_s[lo];
+        const int field = w - (w / 5) * 5;
+        int64_t val = ((meta & 1) ? tb : tf)[w];
+        val += field == 2 ? (int64_t)(meta >> 1) : (field >= 3 ? start_s[lo] : 0);
+        int64_t *dst = run_out + x;
+#pragma unroll
+        for (int k = 0; k < kTileReplicas; ++k)
+            if (k < n_rep) __stcs(dst + roff[k], val);
     }
 }
 

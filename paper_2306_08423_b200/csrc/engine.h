@@ -140,7 +140,7 @@ struct EmitPlan {                    // per selected candidate, written by the p
     int64_t rec_total;               // records of all its devices
     int32_t row, entry, m, sched, pp, mp, dp, ok;
     int32_t bounds[DISTSIM_MAX_PP + 1];
-    int32_t pad;
+    int32_t tile_items;              // schedule items per block of the record kernel
     int32_t rf[DISTSIM_MAX_PP], rb[DISTSIM_MAX_PP];   // records of one forward / backward item
     int64_t n_buckets[DISTSIM_MAX_PP];
     int64_t stage_recs[DISTSIM_MAX_PP];               // records of one device of stage d
