@@ -393,7 +393,7 @@ def other_workloads(E, ctx, torch, dev, peaks):
     E.distsim_eval_strategies(ctx, 0, n, batch)
     top = torch.empty(w.top_k, dtype=torch.int64, device=dev)
     E.distsim_topk(ctx, batch, 0, n, w.top_k, top)
-    chunk = 32
+    chunk = 128                       # candidates per call: about 10 GB of records
     sizes = [E.distsim_emit_timelines(ctx, top[i:i + chunk], min(chunk, w.top_k - i), None, 0)
              for i in range(0, w.top_k, chunk)]
     cap = max(sizes) + 1024
@@ -401,7 +401,7 @@ def other_workloads(E, ctx, torch, dev, peaks):
     offsets = torch.empty(chunk * N + 1, dtype=torch.int64, device=dev)
     busy = torch.empty(chunk * N, dtype=torch.int64, device=dev)
     util = torch.empty(chunk * N, dtype=torch.float64, device=dev)
-    for i in range(0, 3 * chunk, chunk):                                     # warm-up
+    for i in range(0, 2 * chunk, chunk):                                     # warm-up
         E.distsim_emit_timelines(ctx, top[i:i + chunk], chunk, records, cap, offsets, busy, util)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     total = 0

@@ -12,8 +12,9 @@
 //                        block walks the run as one flat stream of int64 words: word x belongs to
 //                        the item found by a search in the run's offset table, and its value is
 //                        template word + {0, 0, microbatch, start, start}.  Consecutive threads
-//                        write consecutive words (full 256-byte warp stores whatever the item
-//                        size) to each of the stage's mp*dp replicas, whose lists are identical.
+//                        write consecutive word pairs (16-byte stores, full-width warp stores
+//                        whatever the item size) to each of the stage's mp*dp replicas, whose
+//                        lists are identical.
 //   emit_buckets_kernel  gradient-bucket records of every stage.
 #include "recurrence.cuh"
 
@@ -24,7 +25,7 @@ namespace {
 constexpr int kItemThreads = 256;
 constexpr int kMaxTileItems = 128;  // most schedule items per block (a plan picks its own count)
 constexpr int kTileWords = 16384;   // target size of a block's run, in int64 words per replica
-constexpr int kTileReplicas = 16;   // replicas per block
+constexpr int kTileReplicas = 8;    // replicas per block
 
 __device__ __forceinline__ int find_row(const DeviceView &v, int64_t index)
 {
@@ -199,7 +200,6 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     __shared__ int64_t start_s[kMaxTileItems];          // start time of each item of the run
     __shared__ int32_t ioff[kMaxTileItems + 1];         // word offset of each item inside the run
     __shared__ int32_t meta_s[kMaxTileItems];           // micro-batch << 1 | is-backward
-    __shared__ int64_t run_base_s;                      // word offset of the run inside the stage stream
     const int i = blockIdx.y;
     const EmitPlan &p = plans[i];
     if (!p.ok) return;
@@ -248,16 +248,21 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         }
     }
     // ---- the run: its items' start times, kinds, micro-batches and word offsets ------------
+    // an item's offset follows from how many forward / backward items precede it in the run
     const int s0 = ic * tile_items;
     const int n_items = min(2 * m, s0 + tile_items) - s0;
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTileItems) {
+    bool bwd0; int j0, nf0, nb0;
+    item_at(sched, pp, m, d, s0, bwd0, j0, nf0, nb0);
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTileItems + 1) {
         const int k = threadIdx.x - 64;
-        if (k < n_items) {
+        if (k <= n_items) {
             bool bwd; int j, nf, nb;
-            item_at(sched, pp, m, d, s0 + k, bwd, j, nf, nb);
-            start_s[k] = op_start[(int64_t)i * op_words_per_cand + (int64_t)d * 2 * m + s0 + k];
-            meta_s[k] = (j << 1) | (bwd ? 1 : 0);
-            if (k == 0) run_base_s = ((int64_t)nf * rf + (int64_t)nb * rb) * 5;
+            item_at(sched, pp, m, d, s0 + k, bwd, j, nf, nb);       // k == n_items: one past the run
+            ioff[k] = ((nf - nf0) * rf + (nb - nb0) * rb) * 5;
+            if (k < n_items) {
+                start_s[k] = op_start[(int64_t)i * op_words_per_cand + (int64_t)d * 2 * m + s0 + k];
+                meta_s[k] = (j << 1) | (bwd ? 1 : 0);
+            }
         }
     }
     // word offset of every replica (r, q) of this tile relative to replica 0 of the stage
@@ -286,34 +291,57 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         }
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int acc = 0;
-        for (int k = 0; k < n_items; ++k) { ioff[k] = acc; acc += ((meta_s[k] & 1) ? rb : rf) * 5; }
-        ioff[n_items] = acc;
-    }
-    __syncthreads();
 
     // ---- stream the run as flat words ---------------------------------------------------------
     int64_t roff[kTileReplicas];                     // word offset of each replica of this tile
 #pragma unroll
     for (int k = 0; k < kTileReplicas; ++k) roff[k] = rep_off_s[k];
-    int64_t *run_out = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + run_base_s;
+    int64_t *run_out = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 +
+                       ((int64_t)nf0 * rf + (int64_t)nb0 * rb) * 5;
     const int total = ioff[n_items];
-    for (int x = threadIdx.x; x < total; x += blockDim.x) {
-        int lo = 0, hi = n_items - 1;                // the item holding word x: last k with ioff[k] <= x
+    // Each pass covers 2 * blockDim.x consecutive words.  Records are 40 bytes, so a replica's
+    // copy of the run starts on an even or an odd word; to write 16 bytes at a time to both
+    // kinds, thread t prepares the words 2t-1, 2t and 2t+1 and stores the pair (2t, 2t+1) to
+    // even-based replicas and the pair (2t-1, 2t) to odd-based ones (single words at the ends).
+    unsigned odd_mask = 0;                           // bit k: replica k's copy starts on an odd word
+#pragma unroll
+    for (int k = 0; k < kTileReplicas; ++k)
+        if (((reinterpret_cast<uintptr_t>(run_out + roff[k]) >> 3) & 1) != 0) odd_mask |= 1u << k;
+    auto word = [&](int x, int it) -> int64_t {
+        const int w = x - ioff[it];
+        const int meta = meta_s[it];
+        const int field = w - (w / 5) * 5;
+        int64_t t = ((meta & 1) ? tb : tf)[w];
+        t += field == 2 ? (int64_t)(meta >> 1) : (field >= 3 ? start_s[it] : 0);
+        return t;
+    };
+    for (int x0 = 0; x0 < total; x0 += 2 * kItemThreads) {
+        const int x = x0 + 2 * threadIdx.x;          // the even word of this thread
+        if (x - 1 >= total) break;
+        int lo = 0, hi = n_items - 1;                // item holding word min(x, total-1)
+        const int xs = min(x, total - 1);
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
-            if (ioff[mid] <= x) lo = mid; else hi = mid - 1;
+            if (ioff[mid] <= xs) lo = mid; else hi = mid - 1;
         }
-        const int w = x - ioff[lo];
-        const int meta = meta_s[lo];
-        const int field = w - (w / 5) * 5;
-        int64_t val = ((meta & 1) ? tb : tf)[w];
-        val += field == 2 ? (int64_t)(meta >> 1) : (field >= 3 ? start_s[lo] : 0);
-        int64_t *dst = run_out + x;
+        const bool has_m1 = x >= 1, has_0 = x < total, has_p1 = x + 1 < total;
+        int64_t v_m1 = 0, v_0 = 0, v_p1 = 0;
+        if (has_0) v_0 = word(x, lo);
+        if (has_m1) v_m1 = word(x - 1, (has_0 && x == ioff[lo]) ? lo - 1 : lo);
+        if (has_p1) v_p1 = word(x + 1, (x + 1 == ioff[lo + 1]) ? lo + 1 : lo);
 #pragma unroll
-        for (int k = 0; k < kTileReplicas; ++k)
-            if (k < n_rep) __stcs(dst + roff[k], val);
+        for (int k = 0; k < kTileReplicas; ++k) {
+            if (k >= n_rep) continue;
+            int64_t *dst = run_out + roff[k] + x;
+            if (!((odd_mask >> k) & 1)) {            // (x, x+1) is 16-byte aligned
+                if (has_p1) __stcs(reinterpret_cast<longlong2 *>(dst), make_longlong2(v_0, v_p1));
+                else if (has_0) __stcs(dst, v_0);
+            } else {                                 // (x-1, x) is 16-byte aligned
+                if (has_m1 && has_0) __stcs(reinterpret_cast<longlong2 *>(dst - 1), make_longlong2(v_m1, v_0));
+                else if (has_0) __stcs(dst, v_0);            // x == 0: the run's first word
+                else if (has_m1) __stcs(dst - 1, v_m1);      // x == total: the run's last word
+            }
+        }
     }
 }
 
