@@ -42,6 +42,25 @@ constexpr int thread_kernel_min_blocks()
 
 template <typename T> __device__ __forceinline__ T vmax(T a, T b) { return a > b ? a : b; }
 
+#ifndef DS_CELL_FORM
+#define DS_CELL_FORM 0            // 0: max(t, free) + c;  1: max(t + c, free + c) (shorter chain)
+#endif
+#ifndef DS_UNROLL_MAIN
+#define DS_UNROLL_MAIN 2
+#endif
+#define DS_PRAGMA(x) _Pragma(#x)
+#define DS_UNROLL(n) DS_PRAGMA(unroll n)
+
+// One recurrence cell: end = max(input arrival, device free) + cost.
+template <typename T> __device__ __forceinline__ T cell(T arrival, T free_at, T cost)
+{
+#if DS_CELL_FORM == 1
+    return vmax((T)(arrival + cost), (T)(free_at + cost));
+#else
+    return (T)(vmax(arrival, free_at) + cost);
+#endif
+}
+
 template <int PP, typename T>
 struct ThreadState {
     T fop[PP], bop[PP];
@@ -53,19 +72,19 @@ __device__ __forceinline__ void run_gpipe(const ThreadState<PP, T> &c, int m, T 
 {
 #pragma unroll
     for (int d = 0; d < PP; ++d) free_at[d] = 0;
-#pragma unroll 1
+DS_UNROLL(DS_UNROLL_MAIN)
     for (int j = 0; j < m; ++j) {
         T t = free_at[0] + c.fop[0];
         free_at[0] = t;
 #pragma unroll
-        for (int d = 1; d < PP; ++d) { t = vmax(t, free_at[d]) + c.fop[d]; free_at[d] = t; }
+        for (int d = 1; d < PP; ++d) { t = cell(t, free_at[d], c.fop[d]); free_at[d] = t; }
     }
-#pragma unroll 1
+DS_UNROLL(DS_UNROLL_MAIN)
     for (int j = 0; j < m; ++j) {
         T t = free_at[PP - 1] + c.bop[PP - 1];
         free_at[PP - 1] = t;
 #pragma unroll
-        for (int d = PP - 2; d >= 0; --d) { t = vmax(t, free_at[d]) + c.bop[d]; free_at[d] = t; }
+        for (int d = PP - 2; d >= 0; --d) { t = cell(t, free_at[d], c.bop[d]); free_at[d] = t; }
     }
 }
 
@@ -76,13 +95,27 @@ __device__ __forceinline__ void wave_1f1b(const ThreadState<PP, T> &c, T (&free_
     T t = 0;
 #pragma unroll
     for (int d = PP - 1; d >= 0; --d) {
-        t = (d == PP - 1 ? free_at[d] : vmax(t, free_at[d])) + c.bop[d];
+        t = d == PP - 1 ? (T)(free_at[d] + c.bop[d]) : cell(t, free_at[d], c.bop[d]);
         free_at[d] = t;
         if (d >= D0) {
-            const T f = (d == 0 ? free_at[0] : vmax(last_f[d > 0 ? d - 1 : 0], free_at[d])) + c.fop[d];
+            const T f = d == 0 ? (T)(free_at[0] + c.fop[0]) : cell(last_f[d > 0 ? d - 1 : 0], free_at[d], c.fop[d]);
             free_at[d] = f;
             last_f[d] = f;
         }
+    }
+}
+
+// A steady-state 1F1B wave: every stage runs its backward item and then a forward item.  After
+// a forward item the device's free time IS that item's end, so inside the steady state the
+// free times are not kept separately: last_f doubles as the free time.
+template <int PP, typename T>
+__device__ __forceinline__ void wave_1f1b_steady(const ThreadState<PP, T> &c, T (&last_f)[PP])
+{
+    T t = 0;
+#pragma unroll
+    for (int d = PP - 1; d >= 0; --d) {
+        t = d == PP - 1 ? (T)(last_f[d] + c.bop[d]) : cell(t, last_f[d], c.bop[d]);
+        last_f[d] = d == 0 ? (T)(t + c.fop[0]) : cell(last_f[d > 0 ? d - 1 : 0], t, c.fop[d]);
     }
 }
 
@@ -110,7 +143,7 @@ struct WarmWaves {
             T t = free_at[0] + c.fop[0];
             free_at[0] = t; last_f[0] = t;
 #pragma unroll
-            for (int d = 1; d < PP - J; ++d) { t = vmax(t, free_at[d]) + c.fop[d]; free_at[d] = t; last_f[d] = t; }
+            for (int d = 1; d < PP - J; ++d) { t = cell(t, free_at[d], c.fop[d]); free_at[d] = t; last_f[d] = t; }
         }
         WarmWaves<PP, J + 1, T>::run(c, m, free_at, last_f);
     }
@@ -127,9 +160,14 @@ __device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (
 #pragma unroll
     for (int d = 0; d < PP; ++d) { free_at[d] = 0; last_f[d] = 0; }
     WarmWaves<PP, 0, T>::run(c, m, free_at, last_f);
-    // waves i = 0 .. m-PP-1: every stage still has a forward item to pair with its backward
-#pragma unroll 1
-    for (int i = 0; i < m - PP; ++i) wave_1f1b<PP, 0, T>(c, free_at, last_f);
+    // waves i = 0 .. m-PP-1: every stage still has a forward item to pair with its backward;
+    // entering them every stage's latest item is a forward one (free_at == last_f)
+    if (m > PP) {
+DS_UNROLL(DS_UNROLL_MAIN)
+        for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T>(c, last_f);
+#pragma unroll
+        for (int d = 0; d < PP; ++d) free_at[d] = last_f[d];
+    }
     // the last min(PP, m) waves
     TailWaves<PP, PP, T>::run(c, m, free_at, last_f);
 }
