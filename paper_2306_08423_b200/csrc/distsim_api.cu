@@ -443,14 +443,8 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
     if (int rc = set_device(ctx)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const DeviceView v = ctx->view();
-    const int64_t last = first + count;
-    for (size_t r = 0; r < ctx->rows.size(); ++r) {
-        const Row &row = ctx->rows[r];
-        const int64_t lo = first > row.offset ? first - row.offset : 0;
-        const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
-        if (hi <= lo) continue;
-        launch_eval_row(s, v, (int)r, row, ctx->entries.data() + row.entry0, lo, hi, first, d_batch_ns, d_stage_busy_ns, &ctx->launches);
-    }
+    launch_eval(s, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
+                d_batch_ns, d_stage_busy_ns, &ctx->launches);
     CU(cudaGetLastError(), "evaluation launch");
     return DISTSIM_OK;
 }

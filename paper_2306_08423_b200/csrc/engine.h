@@ -110,12 +110,24 @@ void launch_build_layer_tables(cudaStream_t s, const TableConst &tc, const RawTa
                                int32_t *next_grad, int32_t *pe, int64_t *launches);
 
 // ---- evaluation (eval_kernels.cu) ------------------------------------------------------
-// Evaluates candidates [lo, hi) of row `row_index` (indices local to the row); results go to
-// batch_out[row.offset + local - first] and, if non-null, busy_out[(same) * pp_max + d].
-// row_entries: host copies of the row's entries (their time bounds choose the arithmetic width).
-void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const Row &row_host,
-                     const Entry *row_entries, int64_t lo, int64_t hi, int64_t first,
-                     int64_t *batch_out, int64_t *busy_out, int64_t *launches);
+// One launch covers several (row, range) work items; a block finds its item from block_begin.
+struct EvalWork {
+    int32_t row;                 // row index
+    int32_t e_begin, e_end, ept; // thread kernel: entries [e_begin, e_end) of the row, per thread
+    int64_t p_lo, p_hi;          // thread kernel: partitions [p_lo, p_hi)
+    int64_t lo, hi;              // candidates [lo, hi), local to the row
+    int32_t block_begin;         // first block of the item inside the launch
+    int32_t nx;                  // thread kernel: blocks along the partition axis
+};
+constexpr int kMaxEvalWork = 24;
+struct EvalBatch {
+    int32_t n, pad;
+    EvalWork w[kMaxEvalWork];
+};
+// Evaluates candidates [first, first + count); rows / entries: host copies.  Results go to
+// batch_out[index - first] and, if non-null, busy_out[(index - first) * pp_max + d].
+void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_rows, const Entry *entries,
+                 int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out, int64_t *launches);
 
 // ---- selection (select_kernels.cu) -----------------------------------------------------
 struct SelectScratch {

@@ -1,11 +1,17 @@
 // Evaluation kernels: batch time (and optionally per-stage activity time) of a range of
-// candidates of one row.
+// candidates.
 //
+// eval_thread_kernel (eval_thread.cuh): one stage partition per thread, for rows with many
+// partitions and pp <= 16.
 // eval_lockstep_kernel: a segment of pp/S consecutive lanes evaluates one candidate, lane =
 // stage (S = 2 stages per lane when pp = 64), 32/(pp/S) candidates per warp, all segments of a
 // warp advancing through the slots of the lock-step recurrence together.  The prefix rows of
 // the entries a block touches are staged into shared memory with one bulk copy per table
 // (cp.async.bulk, completion on the block's own mbarrier, no multicast).
+//
+// A search space has a few dozen rows, many of them tiny; launching them one by one would leave
+// the device idle between kernels, so one launch carries a list of (row, range) work items and
+// every block looks up the item it belongs to.
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
 #include "eval_thread.cuh"
@@ -18,19 +24,22 @@ constexpr int kEvalThreads = 256;
 
 template <int S>
 __global__ void __launch_bounds__(kEvalThreads)
-eval_lockstep_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t first,
-                     int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out,
-                     int max_stage_entries)
+eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
+                     int64_t *__restrict__ busy_out, int smem_words)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t bar;
-    const Row row = v.rows[row_index];
+    int wi = 0;
+    while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
+    const EvalWork &wk = batch.w[wi];
+    const int64_t lo = wk.lo, hi = wk.hi;
+    const Row row = v.rows[wk.row];
     const int pp = row.pp;
     const int wl = pp / S;                         // lanes per candidate
     const int cpw = 32 / wl;                       // candidates per warp
     const int warps = blockDim.x >> 5;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t cta_first = lo + (int64_t)blockIdx.x * warps * cpw;
+    const int64_t cta_first = lo + (int64_t)((int)blockIdx.x - wk.block_begin) * warps * cpw;
     if (cta_first >= hi) return;
     const int64_t cta_last = min(hi, cta_first + (int64_t)warps * cpw) - 1;
 
@@ -39,6 +48,7 @@ eval_lockstep_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_
     const int e_hi = split_local(row, cta_last).entry;
     const int n_stage = e_hi - e_lo + 1;
     const int lp = v.tc.lp;
+    const int max_stage_entries = smem_words / (2 * lp);
     int64_t *sm_f = reinterpret_cast<int64_t *>(smem_raw);
     int64_t *sm_b = sm_f + (int64_t)max_stage_entries * lp;
     bool staged = false;
@@ -73,131 +83,165 @@ eval_lockstep_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_
     }
 }
 
-template <int PP, typename T>
-void launch_thread_kernel(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo,
-                          int64_t hi, int64_t first, int e_begin, int e_end, int ept, int64_t p_lo,
-                          int64_t p_hi, int64_t *batch_out, int64_t *busy_out)
-{
-    const int lp = v.tc.lp;
-    ThreadKernelSmem plan{};
-    size_t words = 0;
-    // prefix rows of every entry of the row; the row's two bucket tables only when there is no
-    // per-entry bucket-lane table to look the result up in
-    if ((size_t)row.n_entries * lp * 2 <= 8192) {
-        plan.n_entries_staged = row.n_entries;
-        plan.off_etb = row.n_entries * lp;
-        words = (size_t)row.n_entries * lp * 2;
-    }
-    if (!v.dt && words + 2 * (size_t)v.tab_words <= 12288) {
-        plan.tables_staged = 1;
-        plan.off_nb = (int32_t)words;
-        plan.off_tp = (int32_t)words + v.tab_words;
-        words += 2 * (size_t)v.tab_words;
-    }
-    const size_t smem = words * sizeof(int64_t);
-    const int64_t n_threads = p_hi - p_lo;
-    dim3 grid((unsigned)((n_threads + kThreadBlock - 1) / kThreadBlock), (unsigned)((e_end - e_begin + ept - 1) / ept));
-    if (busy_out) {
-        if (smem > 24 * 1024)
-            cudaFuncSetAttribute(eval_thread_kernel<PP, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        eval_thread_kernel<PP, T, true><<<grid, kThreadBlock, smem, s>>>(v, row_index, lo, hi, first, e_begin, e_end, ept,
-                                                                         p_lo, p_hi, batch_out, busy_out, plan);
-    } else {
-        if (smem > 24 * 1024)
-            cudaFuncSetAttribute(eval_thread_kernel<PP, T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        eval_thread_kernel<PP, T, false><<<grid, kThreadBlock, smem, s>>>(v, row_index, lo, hi, first, e_begin, e_end, ept,
-                                                                          p_lo, p_hi, batch_out, busy_out, plan);
-    }
-}
+// Work items collected for one kernel instance, launched when full or at the end.
+struct Pending {
+    EvalBatch batch{};
+    int blocks = 0;
+    int smem_words = 0;
+};
 
-template <typename T>
-void launch_thread_kernel_pp(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo,
-                             int64_t hi, int64_t first, int e_begin, int e_end, int ept, int64_t p_lo,
-                             int64_t p_hi, int64_t *batch_out, int64_t *busy_out)
-{
-    switch (row.pp) {
-    case 1: launch_thread_kernel<1, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-    case 2: launch_thread_kernel<2, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-    case 4: launch_thread_kernel<4, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-    case 8: launch_thread_kernel<8, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-    default: launch_thread_kernel<16, T>(s, v, row_index, row, lo, hi, first, e_begin, e_end, ept, p_lo, p_hi, batch_out, busy_out); break;
-    }
-}
-
-void launch_lockstep(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo, int64_t hi,
-                     int64_t first, int64_t *batch_out, int64_t *busy_out);
-
-}  // namespace
-
-void launch_eval_row(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, const Entry *row_entries,
-                     int64_t lo, int64_t hi, int64_t first, int64_t *batch_out, int64_t *busy_out,
-                     int64_t *launches)
-{
-    if (hi <= lo) return;
-    if (row.pp > 16) {
-        launch_lockstep(s, v, row_index, row, lo, hi, first, batch_out, busy_out);
-        ++*launches;
-        return;
-    }
-    // Short pipelines: cut the range into runs of entries with the same arithmetic width; a run
-    // with enough partitions goes to the one-partition-per-thread kernel, the rest to lock-step.
-    const int64_t per_entry = row.n_part * row.n_sched;
-    const int e_begin = (int)(lo / per_entry), e_end = (int)((hi - 1) / per_entry) + 1;
-    int r0 = e_begin;
-    while (r0 < e_end) {
-        const bool narrow = row_entries[r0].bound < ((int64_t)1 << 32);
-        int r1 = r0 + 1;
-        while (r1 < e_end && (row_entries[r1].bound < ((int64_t)1 << 32)) == narrow) ++r1;
-        const int64_t lo_r = lo > (int64_t)r0 * per_entry ? lo : (int64_t)r0 * per_entry;
-        const int64_t hi_r = hi < (int64_t)r1 * per_entry ? hi : (int64_t)r1 * per_entry;
-        int64_t p_lo = 0, p_hi = row.n_part;
-        if (r1 - r0 == 1) {
-            p_lo = (lo_r - (int64_t)r0 * per_entry) / row.n_sched;
-            p_hi = (hi_r - 1 - (int64_t)r0 * per_entry) / row.n_sched + 1;
-        }
-        const int64_t n_parts = p_hi - p_lo;
-        const int n_e = r1 - r0;
-        const int ept = n_parts >= 148 * 4 * kThreadBlock ? n_e : 1;       // entries per thread
-        if (n_parts * ((n_e + ept - 1) / ept) >= 2048) {
-            if (narrow) launch_thread_kernel_pp<uint32_t>(s, v, row_index, row, lo_r, hi_r, first, r0, r1, ept, p_lo, p_hi, batch_out, busy_out);
-            else launch_thread_kernel_pp<int64_t>(s, v, row_index, row, lo_r, hi_r, first, r0, r1, ept, p_lo, p_hi, batch_out, busy_out);
-        } else {
-            launch_lockstep(s, v, row_index, row, lo_r, hi_r, first, batch_out, busy_out);
-        }
-        ++*launches;
-        r0 = r1;
-    }
-}
-
-namespace {
-
-void launch_lockstep(cudaStream_t s, const DeviceView &v, int row_index, const Row &row, int64_t lo, int64_t hi,
-                     int64_t first, int64_t *batch_out, int64_t *busy_out)
+int lockstep_blocks(const Row &row, int64_t lo, int64_t hi)
 {
     const int S = row.pp > 32 ? 2 : 1;
-    const int wl = row.pp / S;
-    const int cpb = (kEvalThreads / 32) * (32 / wl);      // candidates per block
-    const int64_t blocks = (hi - lo + cpb - 1) / cpb;
-    // entries a block can touch: its candidates span at most this many entries
+    const int cpb = (kEvalThreads / 32) * (32 / (row.pp / S));
+    return (int)((hi - lo + cpb - 1) / cpb);
+}
+
+int lockstep_smem_words(const DeviceView &v, const Row &row)
+{
+    const int S = row.pp > 32 ? 2 : 1;
+    const int cpb = (kEvalThreads / 32) * (32 / (row.pp / S));
     const int64_t per_entry = row.n_part * row.n_sched;
     int64_t span = (cpb + per_entry - 1) / per_entry + 1;
     if (span > row.n_entries) span = row.n_entries;
-    int max_stage = (int)span;
-    size_t smem = (size_t)max_stage * v.tc.lp * sizeof(int64_t) * 2;
-    if (smem > 96 * 1024) { max_stage = 0; smem = 0; }   // too wide: read the rows from global
-    if (S == 1) {
-        if (smem > 48 * 1024)
-            cudaFuncSetAttribute(eval_lockstep_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        eval_lockstep_kernel<1><<<(unsigned)blocks, kEvalThreads, smem, s>>>(v, row_index, lo, hi, first,
-                                                                           batch_out, busy_out, max_stage);
-    } else {
-        if (smem > 48 * 1024)
-            cudaFuncSetAttribute(eval_lockstep_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        eval_lockstep_kernel<2><<<(unsigned)blocks, kEvalThreads, smem, s>>>(v, row_index, lo, hi, first,
-                                                                           batch_out, busy_out, max_stage);
+    const int64_t words = span * v.tc.lp * 2;
+    return words * (int64_t)sizeof(int64_t) > 96 * 1024 ? 0 : (int)words;     // too wide: global reads
+}
+
+template <int S>
+void flush_lockstep(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first, int64_t *batch_out,
+                    int64_t *busy_out, int64_t *launches)
+{
+    if (p.batch.n == 0) return;
+    const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
+    if (smem > 48 * 1024)
+        cudaFuncSetAttribute(eval_lockstep_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    eval_lockstep_kernel<S><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
+    ++*launches;
+    p = Pending{};
+}
+
+template <int PP, typename T, bool kBusy>
+void flush_thread(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first, int64_t *batch_out,
+                  int64_t *busy_out, int64_t *launches)
+{
+    if (p.batch.n == 0) return;
+    const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
+    if (smem > 24 * 1024)
+        cudaFuncSetAttribute(eval_thread_kernel<PP, T, kBusy>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    eval_thread_kernel<PP, T, kBusy><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out);
+    ++*launches;
+    p = Pending{};
+}
+
+// Thread-kernel instances are indexed by (log2 pp, narrow).
+template <typename T, bool kBusy>
+void flush_thread_pp(int log2pp, cudaStream_t s, const DeviceView &v, Pending &p, int64_t first,
+                     int64_t *batch_out, int64_t *busy_out, int64_t *launches)
+{
+    switch (log2pp) {
+    case 0: flush_thread<1, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
+    case 1: flush_thread<2, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
+    case 2: flush_thread<4, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
+    case 3: flush_thread<8, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
+    default: flush_thread<16, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
     }
 }
 
+void flush_thread_any(int log2pp, bool narrow, cudaStream_t s, const DeviceView &v, Pending &p, int64_t first,
+                      int64_t *batch_out, int64_t *busy_out, int64_t *launches)
+{
+    if (narrow) {
+        if (busy_out) flush_thread_pp<uint32_t, true>(log2pp, s, v, p, first, batch_out, busy_out, launches);
+        else flush_thread_pp<uint32_t, false>(log2pp, s, v, p, first, batch_out, busy_out, launches);
+    } else {
+        if (busy_out) flush_thread_pp<int64_t, true>(log2pp, s, v, p, first, batch_out, busy_out, launches);
+        else flush_thread_pp<int64_t, false>(log2pp, s, v, p, first, batch_out, busy_out, launches);
+    }
+}
+
+int ilog2(int v) { int b = 0; while ((1 << (b + 1)) <= v) ++b; return b; }
+
 }  // namespace
+
+void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_rows, const Entry *entries,
+                 int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out, int64_t *launches)
+{
+    const int64_t last = first + count;
+    Pending lock[2];                               // lock-step kernel, S = 1 and S = 2
+    Pending thr[5][2];                             // thread kernel, [log2 pp][narrow]
+    constexpr int kMaxBlocks = 1 << 30;
+
+    auto add_lockstep = [&](int r, int64_t lo, int64_t hi) {
+        const int which = rows[r].pp > 32 ? 1 : 0;
+        Pending &p = lock[which];
+        const int blocks = lockstep_blocks(rows[r], lo, hi);
+        if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - blocks) {
+            if (which) flush_lockstep<2>(s, v, p, first, batch_out, busy_out, launches);
+            else flush_lockstep<1>(s, v, p, first, batch_out, busy_out, launches);
+        }
+        EvalWork &w = p.batch.w[p.batch.n++];
+        w = EvalWork{};
+        w.row = r; w.lo = lo; w.hi = hi; w.block_begin = p.blocks;
+        p.blocks += blocks;
+        const int words = lockstep_smem_words(v, rows[r]);
+        // one dynamic size per launch: the largest any item wants (items that want none still work)
+        if (words > p.smem_words) p.smem_words = words;
+    };
+
+    for (int r = 0; r < n_rows; ++r) {
+        const Row &row = rows[r];
+        const int64_t lo = first > row.offset ? first - row.offset : 0;
+        const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
+        if (hi <= lo) continue;
+        if (row.pp > 16) { add_lockstep(r, lo, hi); continue; }
+        // Short pipelines: cut the range into runs of entries with the same arithmetic width; a
+        // run with enough partitions goes to the one-partition-per-thread kernel, the rest to
+        // the lock-step kernel.
+        const Entry *row_entries = entries + row.entry0;
+        const int64_t per_entry = row.n_part * row.n_sched;
+        const int e_begin = (int)(lo / per_entry), e_end = (int)((hi - 1) / per_entry) + 1;
+        int r0 = e_begin;
+        while (r0 < e_end) {
+            const bool narrow = row_entries[r0].bound < ((int64_t)1 << 32);
+            int r1 = r0 + 1;
+            while (r1 < e_end && (row_entries[r1].bound < ((int64_t)1 << 32)) == narrow) ++r1;
+            const int64_t lo_r = lo > (int64_t)r0 * per_entry ? lo : (int64_t)r0 * per_entry;
+            const int64_t hi_r = hi < (int64_t)r1 * per_entry ? hi : (int64_t)r1 * per_entry;
+            int64_t p_lo = 0, p_hi = row.n_part;
+            if (r1 - r0 == 1) {
+                p_lo = (lo_r - (int64_t)r0 * per_entry) / row.n_sched;
+                p_hi = (hi_r - 1 - (int64_t)r0 * per_entry) / row.n_sched + 1;
+            }
+            const int64_t n_parts = p_hi - p_lo;
+            const int n_e = r1 - r0;
+            const int ept = n_parts >= 148 * 4 * kThreadBlock ? n_e : 1;       // entries per thread
+            const int64_t nx = (n_parts + kThreadBlock - 1) / kThreadBlock;
+            const int64_t ny = (n_e + ept - 1) / ept;
+            if (n_parts * ny >= 2048 && nx * ny < kMaxBlocks) {
+                const int lg = ilog2(row.pp);
+                Pending &p = thr[lg][narrow ? 1 : 0];
+                if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - (int)(nx * ny))
+                    flush_thread_any(lg, narrow, s, v, p, first, batch_out, busy_out, launches);
+                EvalWork &w = p.batch.w[p.batch.n++];
+                w = EvalWork{};
+                w.row = r; w.e_begin = r0; w.e_end = r1; w.ept = ept; w.p_lo = p_lo; w.p_hi = p_hi;
+                w.lo = lo_r; w.hi = hi_r; w.block_begin = p.blocks; w.nx = (int)nx;
+                p.blocks += (int)(nx * ny);
+                const int words = thread_kernel_smem(row.n_entries, v.tc.lp, v.tab_words, v.dt != nullptr).words;
+                if (words > p.smem_words) p.smem_words = words;
+            } else {
+                add_lockstep(r, lo_r, hi_r);
+            }
+            r0 = r1;
+        }
+    }
+    // largest kernels first, so that the small ones fill the tail of the big ones
+    for (int lg = 4; lg >= 0; --lg)
+        for (int nw = 1; nw >= 0; --nw)
+            flush_thread_any(lg, nw == 1, s, v, thr[lg][nw], first, batch_out, busy_out, launches);
+    flush_lockstep<2>(s, v, lock[1], first, batch_out, busy_out, launches);
+    flush_lockstep<1>(s, v, lock[0], first, batch_out, busy_out, launches);
+}
 
 }  // namespace distsim

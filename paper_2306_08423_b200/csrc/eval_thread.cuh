@@ -172,23 +172,50 @@ DS_UNROLL(DS_UNROLL_MAIN)
     TailWaves<PP, PP, T>::run(c, m, free_at, last_f);
 }
 
-// Shared-memory plan of a block (offsets in int64 words from the dynamic shared base).
+// Shared-memory plan of a block (offsets in int64 words from the dynamic shared base): the
+// prefix rows of every entry of the row, and the row's two bucket tables only when there is no
+// per-entry bucket-lane table to look the result up in - each as far as it fits.
 struct ThreadKernelSmem {
     int32_t n_entries_staged;   // 0: read prefix rows from global
     int32_t tables_staged;      // 1: NB / TP tables of the row are in shared memory
     int32_t off_etb, off_nb, off_tp;
+    int32_t words;              // dynamic shared memory needed, in int64 words
 };
+__host__ __device__ inline ThreadKernelSmem thread_kernel_smem(int n_entries, int lp, int tab_words, bool have_dt)
+{
+    ThreadKernelSmem plan{};
+    int words = 0;
+    if (n_entries * lp * 2 <= 8192) {
+        plan.n_entries_staged = n_entries;
+        plan.off_etb = n_entries * lp;
+        words = n_entries * lp * 2;
+    }
+    if (!have_dt && words + 2 * tab_words <= 12288) {
+        plan.tables_staged = 1;
+        plan.off_nb = words;
+        plan.off_tp = words + tab_words;
+        words += 2 * tab_words;
+    }
+    plan.words = words;
+    return plan;
+}
 
 // Entry scalars the hot path needs, kept in shared memory for the whole row.
 struct EntryLite { int64_t p2p_intra, p2p_inter; int32_t m, pad; };
 
 template <int PP, typename T, bool kBusy>
 __global__ void __launch_bounds__(kThreadBlock, thread_kernel_min_blocks<PP, T>())
-eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t first,
-                   int e_begin, int e_end, int entries_per_thread, int64_t p_lo, int64_t p_hi,
-                   int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out,
-                   ThreadKernelSmem plan)
+eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
+                   int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out)
 {
+    // which work item (row and range) this block belongs to
+    int wi = 0;
+    while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
+    const EvalWork &wk = batch.w[wi];
+    const int row_index = wk.row, e_begin = wk.e_begin, e_end = wk.e_end, entries_per_thread = wk.ept;
+    const int64_t lo = wk.lo, hi = wk.hi, p_lo = wk.p_lo, p_hi = wk.p_hi;
+    const int local_block = (int)blockIdx.x - wk.block_begin;
+    const int block_x = local_block % wk.nx, block_y = local_block / wk.nx;
     extern __shared__ __align__(16) int64_t dsm[];
     __shared__ __align__(8) uint64_t bar;
     __shared__ T xs[PP][kThreadBlock];                // per thread, per stage: bucket-lane excess X
@@ -197,6 +224,7 @@ eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t 
     const Row &row = v.rows[row_index];
     const int lp = v.tc.lp;
     const int L1 = v.tc.n_layers + 1;
+    const ThreadKernelSmem plan = thread_kernel_smem(row.n_entries, lp, v.tab_words, v.dt != nullptr);
     const int dp = row.dp, n_sched = row.n_sched, sched0 = row.sched0, period = row.p2p_period;
     const int64_t t_full = row.t_full;
 
@@ -226,9 +254,9 @@ eval_thread_kernel(DeviceView v, int row_index, int64_t lo, int64_t hi, int64_t 
     const int64_t *nbt = (staged && plan.tables_staged) ? dsm + plan.off_nb : nb_g;
     const int64_t *tpt = (staged && plan.tables_staged) ? dsm + plan.off_tp : tp_g;
 
-    const int64_t part = p_lo + (int64_t)blockIdx.x * kThreadBlock + threadIdx.x;
+    const int64_t part = p_lo + (int64_t)block_x * kThreadBlock + threadIdx.x;
     if (part >= p_hi) return;
-    const int e0 = e_begin + (int)blockIdx.y * entries_per_thread;
+    const int e0 = e_begin + block_y * entries_per_thread;
     const int e1 = min(e_end, e0 + entries_per_thread);
 
     // ---- decode the partition once (bounds are parked in shared memory) ----------------------
