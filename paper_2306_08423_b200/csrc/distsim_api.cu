@@ -30,6 +30,8 @@ struct DevBuf {
     template <class T> T *as() const { return static_cast<T *>(p); }
 };
 
+constexpr int64_t kCompactCap = 1 << 20;     // pairs in the top-k compact buffer (16 MB)
+
 bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
 
 int64_t sat_mul(int64_t a, int64_t b)
@@ -92,8 +94,11 @@ struct distsim_ctx {
         SelectScratch s{};
         unsigned long long *base = d_sel.as<unsigned long long>();
         s.key = base; s.hist = base + 8; s.sel_state = base + 8 + 2048;
-        s.cand_time = reinterpret_cast<int64_t *>(base + 8 + 2048 + 8);
+        s.cand_time = reinterpret_cast<int64_t *>(base + 8 + 2048 + 16);
         s.cand_idx = s.cand_time + 4096;
+        s.comp_time = s.cand_idx + 4096;
+        s.comp_idx = s.comp_time + kCompactCap;
+        s.comp_cap = kCompactCap;
         return s;
     }
 };
@@ -168,7 +173,7 @@ int distsim_create(distsim_ctx **out, int cuda_device)
     ctx->device = cuda_device;
     if (cudaSetDevice(cuda_device) != cudaSuccess ||
         ctx->d_status.reserve(64) != cudaSuccess ||
-        ctx->d_sel.reserve((8 + 2048 + 8 + 2 * 4096) * sizeof(int64_t)) != cudaSuccess ||
+        ctx->d_sel.reserve((8 + 2048 + 16 + 2 * 4096 + 2 * kCompactCap) * sizeof(int64_t)) != cudaSuccess ||
         ctx->d_result.reserve(64) != cudaSuccess || ctx->d_totals.reserve(64) != cudaSuccess ||
         cudaMemset(ctx->d_status.p, 0, 64) != cudaSuccess ||
         cudaMallocHost(&ctx->h_pinned, 8 * sizeof(int64_t)) != cudaSuccess) {

@@ -133,8 +133,10 @@ void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_row
 struct SelectScratch {
     unsigned long long *key;        // [2] packed / two-pass argmin keys
     unsigned long long *hist;       // [2048] radix histogram
-    unsigned long long *sel_state;  // [8] radix-select state
+    unsigned long long *sel_state;  // [16] radix-select state
     int64_t *cand_time, *cand_idx;  // [4096] selected pairs before sorting
+    int64_t *comp_time, *comp_idx;  // [comp_cap] compact buffer of the surviving pairs (optional)
+    int64_t comp_cap;               // 0: no compact buffer
 };
 // d_result[0] = smallest time, d_result[1] = its smallest position in `batch`.
 void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t time_bound,

@@ -84,32 +84,51 @@ __global__ void argmin_unpack_kernel(const u64 *key, int idx_bits, int packed, i
 // ---- top-k ---------------------------------------------------------------------------------
 // Radix select with 11-bit digits, most significant first: first on the time, then (only if the
 // threshold time is shared by more elements than are still wanted) on the index among the
-// elements that have it.  `rank` is the rank still to resolve inside the current group;
-// blocks_done counts finished blocks of a pass; cursor is the output cursor.
+// elements that have it.  `rank` is the rank still to resolve inside the current group.
+// After the first pass only the elements whose top digit does not exceed the chosen bin can
+// still matter; they are copied to a compact (time, index) buffer and the remaining passes read
+// that buffer instead of the whole array (if they fit; otherwise everything stays on the array).
 constexpr int kRadixBits = 11;
 constexpr int kBins = 1 << kRadixBits;
-struct SelState { u64 tprefix, tmask, rank, iprefix, imask, blocks_done, cursor, skip_index; };
+struct SelState {
+    u64 tprefix, tmask, rank, iprefix, imask, blocks_done, cursor, skip_index;
+    u64 use_compact, cn;         // remaining passes read the compact buffer of cn pairs
+    u64 pad[6];
+};
+
+// The source a pass reads: the array itself (index = position) or the compact buffer.
+struct SelSource { const int64_t *t; const int64_t *idx; int64_t n; };
+__device__ __forceinline__ SelSource sel_source(const SelState *st, const int64_t *batch, int64_t count,
+                                                const SelectScratch &sc)
+{
+    if (st->use_compact) return SelSource{sc.comp_time, sc.comp_idx, (int64_t)st->cn};
+    return SelSource{batch, nullptr, count};
+}
 
 template <bool kIndexPhase>
 __global__ void __launch_bounds__(kSelThreads)
-radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, int width, bool last_time_pass,
-                  u64 *hist, SelState *st)
+radix_pass_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int shift, int width,
+                  bool last_time_pass)
 {
     __shared__ unsigned int sh[kBins];
     __shared__ u64 partial[kSelThreads];
     __shared__ bool last;
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    u64 *hist = sc.hist;
     // no ties at the threshold time: every element equal to it is wanted, no index pass needed
     if (kIndexPhase && st->skip_index) return;
     for (int i = threadIdx.x; i < kBins; i += blockDim.x) sh[i] = 0;
     __syncthreads();
+    const SelSource src = sel_source(st, batch, count, sc);
     const u64 tprefix = st->tprefix, tmask = st->tmask, iprefix = st->iprefix, imask = st->imask;
     const unsigned dmask = (1u << width) - 1u;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-        const u64 x = (u64)t[i];
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < src.n; i += (int64_t)gridDim.x * blockDim.x) {
+        const u64 x = (u64)src.t[i];
         if ((x & tmask) != tprefix) continue;
         if (kIndexPhase) {
-            if (((u64)i & imask) != iprefix) continue;
-            atomicAdd(&sh[(unsigned)((u64)i >> shift) & dmask], 1u);
+            const u64 id = src.idx ? (u64)src.idx[i] : (u64)i;
+            if ((id & imask) != iprefix) continue;
+            atomicAdd(&sh[(unsigned)(id >> shift) & dmask], 1u);
         } else {
             atomicAdd(&sh[(unsigned)(x >> shift) & dmask], 1u);
         }
@@ -149,6 +168,9 @@ radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, int width
         if (kIndexPhase) { st->iprefix = iprefix | ((u64)bin << shift); st->imask = imask | ((u64)dmask << shift); }
         else { st->tprefix = tprefix | ((u64)bin << shift); st->tmask = tmask | ((u64)dmask << shift); }
         st->blocks_done = 0;
+        // everything at or below the chosen bin may still matter: this many pairs to compact
+        // (once the compact buffer is in use, cn is its size and must stay)
+        if (!st->use_compact) st->cn = cum + in_bin;
     }
     __syncthreads();
     for (int i = threadIdx.x; i < kBins; i += blockDim.x) hist[i] = 0;
@@ -157,19 +179,46 @@ radix_pass_kernel(const int64_t *__restrict__ t, int64_t n, int shift, int width
 __global__ void sel_init_kernel(SelState *st, u64 *hist, int k)
 {
     for (int i = threadIdx.x; i < kBins; i += blockDim.x) hist[i] = 0;
-    if (threadIdx.x == 0) { SelState z = {0, 0, (u64)(k - 1), 0, 0, 0, 0, 0}; *st = z; }
+    if (threadIdx.x == 0) { SelState z{}; z.rank = (u64)(k - 1); *st = z; }
+}
+
+// After the first time pass: copies the elements whose time does not exceed the chosen top
+// digit into the compact buffer, if they fit; the last block then switches the source over.
+__global__ void __launch_bounds__(kSelThreads)
+compact_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int shift)
+{
+    __shared__ bool last;
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    const u64 cn = st->cn;
+    if (cn > (u64)sc.comp_cap) return;              // does not fit: later passes keep reading the array
+    const u64 limit = st->tprefix >> shift;         // the chosen top digit
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+        const u64 x = (u64)batch[i];
+        if ((x >> shift) <= limit) {
+            const u64 pos = atomicAdd(&st->cursor, 1ull);
+            if (pos < (u64)sc.comp_cap) { sc.comp_time[pos] = (int64_t)x; sc.comp_idx[pos] = i; }
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&st->blocks_done, 1ull) == (u64)gridDim.x - 1;
+    __syncthreads();
+    if (last && threadIdx.x == 0) { st->use_compact = 1; st->cursor = 0; st->blocks_done = 0; }
 }
 
 // Collects the k elements that are not above the threshold pair (time, index), in any order.
 __global__ void __launch_bounds__(kSelThreads)
-collect_kernel(const int64_t *__restrict__ t, int64_t n, SelState *st, int k, int64_t *ct, int64_t *ci)
+collect_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int k)
 {
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    const SelSource src = sel_source(st, batch, count, sc);
     const u64 T = st->tprefix, I = st->iprefix;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-        const u64 x = (u64)t[i];
-        if (x < T || (x == T && (u64)i <= I)) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < src.n; i += (int64_t)gridDim.x * blockDim.x) {
+        const u64 x = (u64)src.t[i];
+        const u64 id = src.idx ? (u64)src.idx[i] : (u64)i;
+        if (x < T || (x == T && id <= I)) {
             const u64 pos = atomicAdd(&st->cursor, 1ull);
-            if (pos < (u64)k) { ct[pos] = (int64_t)x; ci[pos] = i; }
+            if (pos < (u64)k) { sc.cand_time[pos] = (int64_t)x; sc.cand_idx[pos] = (int64_t)id; }
         }
     }
 }
@@ -268,18 +317,24 @@ void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t co
     const int g = grid_for(count);
     // bits above the bound on any time are zero everywhere: start below them
     const int tb = bits_for(time_bound) > 0 ? bits_for(time_bound) : 1;
+    bool first_pass = true;
     for (int shift = ((tb + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
         const int width = tb - shift < kRadixBits ? tb - shift : kRadixBits;
-        radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, shift, width, shift == 0, sc.hist, st);
+        radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, sc, shift, width, shift == 0);
         ++*launches;
+        if (first_pass && shift > 0 && sc.comp_cap > 0) {
+            compact_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc, shift);
+            ++*launches;
+        }
+        first_pass = false;
     }
     const int ib = bits_for(count - 1) > 0 ? bits_for(count - 1) : 1;
     for (int shift = ((ib + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
         const int width = ib - shift < kRadixBits ? ib - shift : kRadixBits;
-        radix_pass_kernel<true><<<g, kSelThreads, 0, s>>>(batch, count, shift, width, false, sc.hist, st);
+        radix_pass_kernel<true><<<g, kSelThreads, 0, s>>>(batch, count, sc, shift, width, false);
         ++*launches;
     }
-    collect_kernel<<<g, kSelThreads, 0, s>>>(batch, count, st, k, sc.cand_time, sc.cand_idx);
+    collect_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc, k);
     sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, k, k, first, d_indices, d_times);
     *launches += 2;
 }
@@ -292,7 +347,7 @@ void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t co
 // call neither needs a context nor touches the CUDA allocator.
 namespace {
 
-constexpr int kStaticWords = 8 + distsim::kBins + 8 + 2 * DISTSIM_TOPK_STATIC_MAX_K;    // 64-bit words
+constexpr int kStaticWords = 8 + distsim::kBins + 16 + 2 * DISTSIM_TOPK_STATIC_MAX_K;   // 64-bit words
 static __device__ __align__(256) unsigned long long g_topk_static_scratch[kStaticWords];
 
 constexpr int kMaxDevices = 64;
@@ -318,7 +373,7 @@ extern "C" int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int6
     unsigned long long *base = g_static_scratch_addr[dev];
     distsim::SelectScratch sc{};
     sc.key = base; sc.hist = base + 8; sc.sel_state = base + 8 + distsim::kBins;
-    sc.cand_time = reinterpret_cast<int64_t *>(base + 8 + distsim::kBins + 8);
+    sc.cand_time = reinterpret_cast<int64_t *>(base + 8 + distsim::kBins + 16);
     sc.cand_idx = sc.cand_time + DISTSIM_TOPK_STATIC_MAX_K;
     int64_t launches = 0;
     // launch_topk begins by clearing the histogram, the selection state and the output cursor,
