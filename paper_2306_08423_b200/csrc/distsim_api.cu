@@ -504,13 +504,13 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     launch_emit_plan(s, v, d_indices, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
                      ctx->op_words_per_cand, d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), &ctx->launches);
     CU(cudaGetLastError(), "emission planning launch");
-    CU(cudaMemcpyAsync(ctx->h_pinned, ctx->d_totals.p, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, s), "totals readback");
+    CU(cudaMemcpyAsync(ctx->h_pinned, ctx->d_totals.p, 3 * sizeof(int64_t), cudaMemcpyDeviceToHost, s), "totals readback");
     if (int rc = read_status(ctx, s)) return rc;       // synchronises
     *h_total_records = ctx->h_pinned[0];
     if (!d_records) return DISTSIM_OK;
     if (ctx->h_pinned[0] > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");
     launch_emit_records(s, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
-                        ctx->op_words_per_cand, ctx->h_pinned[1], d_records, &ctx->launches);
+                        ctx->op_words_per_cand, ctx->h_pinned[1], ctx->h_pinned[2], d_records, &ctx->launches);
     CU(cudaGetLastError(), "emission launch");
     CU(cudaStreamSynchronize(s), "emission sync");
     return DISTSIM_OK;

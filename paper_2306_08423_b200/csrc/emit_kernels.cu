@@ -120,13 +120,13 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
 }
 
 // Exclusive scan of rec_total over the selections (n is small: one block, serial per chunk).
-__global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /*[2]: records, max tiles*/)
+__global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /*[3]: records, max tiles, max bucket copies of a stage*/)
 {
     __shared__ int64_t chunk_sum[1024];
     const int t = threadIdx.x, nt = blockDim.x;
     const int per = (n + nt - 1) / nt;
     const int b = min(n, t * per), e = min(n, b + per);
-    int64_t s = 0, mt = 0;
+    int64_t s = 0, mt = 0, mb = 0;
     for (int i = b; i < e; ++i) s += plans[i].rec_total;
     chunk_sum[t] = s;
     __syncthreads();
@@ -144,9 +144,11 @@ __global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /*[2]: 
             const int64_t tiles = (int64_t)plans[i].pp * ((2 * plans[i].m + plans[i].tile_items - 1) / plans[i].tile_items) *
                                   ((reps + kTileReplicas - 1) / kTileReplicas);
             mt = max64(mt, tiles);
+            for (int d = 0; d < plans[i].pp; ++d) mb = max64(mb, plans[i].n_buckets[d] * reps);
         }
     }
     if (mt > 0) atomicMax((unsigned long long *)&totals[1], (unsigned long long)mt);
+    if (mb > 0) atomicMax((unsigned long long *)&totals[2], (unsigned long long)mb);
 }
 
 __global__ void __launch_bounds__(256)
@@ -345,37 +347,47 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     }
 }
 
-// Gradient-bucket records of stage blockIdx.x of selection blockIdx.y.  Buckets whose last byte
-// lies in the same layer share a ready time, so once the first of them has started the rest
-// follow back to back: per layer one serial step, inside a layer a closed form.
-__global__ void __launch_bounds__(256)
-emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *__restrict__ out)
+// Gradient-bucket records: one warp per (selection, stage).  Buckets whose last byte lies in the
+// same layer share a ready time, so once the first of them has started the rest follow back to
+// back: per layer one serial step (lane 0), inside a layer a closed form (all lanes).
+constexpr int kBucketWarps = 4;
+__global__ void __launch_bounds__(kBucketWarps * 32)
+emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int n, int64_t *__restrict__ out)
 {
-    __shared__ int64_t g_start[DISTSIM_MAX_LAYERS + 1];   // start of the first bucket ending in layer a+i
-    __shared__ int64_t g_first[DISTSIM_MAX_LAYERS + 1];   // number of that bucket
-    __shared__ int64_t part_start;
-    const int i = blockIdx.y, d = blockIdx.x;
+    __shared__ int64_t g_start_s[kBucketWarps][DISTSIM_MAX_LAYERS + 1];   // start of the first bucket ending in layer a+i
+    __shared__ int64_t g_first_s[kBucketWarps][DISTSIM_MAX_LAYERS + 1];   // number of that bucket
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t unit = (int64_t)blockIdx.x * kBucketWarps + warp;
+    const int i = (int)(unit / v.sc.pp_max), d = (int)(unit % v.sc.pp_max);
+    if (i >= n) return;
     const EmitPlan &p = plans[i];
     if (!p.ok || d >= p.pp || p.dp == 1) return;
     const int64_t kb = p.n_buckets[d];
     if (kb == 0) return;
-    const Row row = v.rows[p.row];
+    int64_t *g_start = g_start_s[warp], *g_first = g_first_s[warp];
+    const Row &row = v.rows[p.row];
     const int a = p.bounds[d], e = p.bounds[d + 1];
     const int L1 = v.tc.n_layers + 1;
     const int64_t *nbe = v.nb + row.row_tab_off + (int64_t)e * L1;
     const int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
     const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
-    const int64_t n_full = nbe[a];
-    if (threadIdx.x == 0) {
-        int64_t end = 0, nb_prev = 0;
-        const int64_t tbs = p.last_b_start[d], main_end = p.main_end[d];
+    const int64_t n_full = nbe[a], t_full = row.t_full;
+    int64_t part_start = 0;
+    const int64_t tbs = p.last_b_start[d], main_end = p.main_end[d];
+    // all lanes fetch the per-layer inputs (independent loads), then lane 0 runs the short chain
+    for (int l = a + lane; l < e; l += 32) {
+        g_first[l - a] = l + 1 < e ? nbe[l + 1] : 0;                       // buckets before layer l's group
+        g_start[l - a] = v.tc.overlap ? tbs + (pb[e] - pb[l]) : main_end;    // ready time of the group
+    }
+    __syncwarp();
+    if (lane == 0) {
+        int64_t end = 0;
         for (int l = e - 1; l >= a; --l) {
-            const int64_t nb_l = nbe[l], n_l = nb_l - nb_prev;
-            const int64_t ready = v.tc.overlap ? tbs + (pb[e] - pb[l]) : main_end;
-            g_first[l - a] = nb_prev;
-            g_start[l - a] = max64(end, ready);
-            if (n_l > 0) end = g_start[l - a] + n_l * row.t_full;
-            nb_prev = nb_l;
+            const int64_t nb_prev = g_first[l - a];
+            const int64_t nb_l = l > a ? g_first[l - 1 - a] : n_full;       // nb[e][l]
+            const int64_t start = max64(end, g_start[l - a]);
+            g_start[l - a] = start;
+            if (nb_l > nb_prev) end = start + (nb_l - nb_prev) * t_full;
         }
         if (part > 0) {
             const int ls = v.next_grad[a];
@@ -383,17 +395,17 @@ emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *_
             part_start = max64(end, ready);
         }
     }
-    __syncthreads();
-    const int reps = p.mp * p.dp;
-    const int rep_chunks = gridDim.z;
-    const int per = (reps + rep_chunks - 1) / rep_chunks;
-    const int rep0 = blockIdx.z * per, rep1 = min(reps, rep0 + per);
+    part_start = __shfl_sync(0xffffffffu, part_start, 0);
+    __syncwarp();
+    const int mp = p.mp, reps = mp * p.dp;
+    // the stage's bucket words are cut into gridDim.y slices; a value is computed once and
+    // written to every replica
+    const int64_t per = ((kb * 5 + gridDim.y - 1) / gridDim.y + 31) & ~(int64_t)31;
+    const int64_t w0 = (int64_t)blockIdx.y * per, w1 = min(kb * 5, w0 + per);
     const int64_t stage_words = p.stage_recs[d] * 5;
-    const int64_t replica_words = (int64_t)p.mp * p.stage_rec_prefix[p.pp] * 5;
-    const int64_t base = (p.rec_base + (int64_t)p.mp * p.stage_rec_prefix[d]) * 5 +
-                         (int64_t)p.m * (p.rf[d] + p.rb[d]) * 5;
-    const int r0 = rep0 / p.mp, q0 = rep0 - r0 * p.mp;
-    for (int64_t w = threadIdx.x; w < kb * 5; w += blockDim.x) {
+    const int64_t replica_words = (int64_t)mp * p.stage_rec_prefix[p.pp] * 5;
+    int64_t *base = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + (int64_t)p.m * (p.rf[d] + p.rb[d]) * 5;
+    for (int64_t w = w0 + lane; w < w1; w += 32) {
         const int64_t k = w / 5;
         const int field = (int)(w - k * 5);
         int64_t val;
@@ -411,17 +423,17 @@ emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *_
                     const int mid = (lo + hi + 1) >> 1;
                     if (nbe[mid] > k) lo = mid; else hi = mid - 1;
                 }
-                start = g_start[lo - a] + (k - g_first[lo - a]) * row.t_full;
-                dur = row.t_full;
+                start = g_start[lo - a] + (k - g_first[lo - a]) * t_full;
+                dur = t_full;
             }
             val = field == 3 ? start : start + dur;
         }
-        int r = r0, q = q0;
-        int64_t *dst = out + base + (int64_t)r * replica_words + (int64_t)q * stage_words + w;
-        for (int rep = rep0; rep < rep1; ++rep) {
+        int r = 0, q = 0;
+        int64_t *dst = base + w;
+        for (int rep = 0; rep < reps; ++rep) {
             __stcs(dst, val);
             dst += stage_words;
-            if (++q == p.mp) { q = 0; ++r; dst = out + base + (int64_t)r * replica_words + w; }
+            if (++q == mp) { q = 0; ++r; dst = base + w + (int64_t)r * replica_words; }
         }
     }
 }
@@ -433,7 +445,7 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
                       int64_t *launches)
 {
-    cudaMemsetAsync(d_totals, 0, 2 * sizeof(int64_t), s);
+    cudaMemsetAsync(d_totals, 0, 3 * sizeof(int64_t), s);
     emit_plan_kernel<<<(n + 3) / 4, 128, 0, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand);
     emit_scan_kernel<<<1, 1024, 0, s>>>(plans, n, d_totals);
     *launches += 2;
@@ -446,7 +458,7 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
 
 void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
                          const int64_t *op_start, int64_t op_words_per_cand, int64_t max_tiles,
-                         distsim_record *records, int64_t *launches)
+                         int64_t max_bucket_copies, distsim_record *records, int64_t *launches)
 {
     if (n == 0 || max_tiles == 0) return;
     const size_t smem = (size_t)(2 * (3 * v.tc.n_layers + 1)) * 5 * sizeof(int64_t);
@@ -460,7 +472,11 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
         v, plans, op_start, op_words_per_cand, out);
     ++*launches;
     if (v.tc.n_devices > 1) {
-        emit_buckets_kernel<<<dim3((unsigned)v.sc.pp_max, (unsigned)n, 4), 256, 0, s>>>(v, plans, out);
+        const int64_t units = (int64_t)n * v.sc.pp_max;
+        // stages with many bucket records times many replicas are cut into replica slices
+        int64_t ny = (max_bucket_copies + 4095) / 4096;
+        ny = ny < 1 ? 1 : (ny > 64 ? 64 : ny);
+        emit_buckets_kernel<<<dim3((unsigned)((units + kBucketWarps - 1) / kBucketWarps), (unsigned)ny), kBucketWarps * 32, 0, s>>>(v, plans, n, out);
         ++*launches;
     }
 }

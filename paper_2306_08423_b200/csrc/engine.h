@@ -165,14 +165,14 @@ struct EmitPlan {                    // per selected candidate, written by the p
 };
 // Plans the n selections: item start times into op_start (op_words_per_cand words each), record
 // counts, offsets / busy / util (each nullable); d_totals[0] = records, d_totals[1] = largest
-// number of item tiles of any selection.
+// number of item tiles of any selection, d_totals[2] = largest (bucket records x replicas) of any stage.
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
                       int64_t *launches);
 void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
                          const int64_t *op_start, int64_t op_words_per_cand, int64_t max_tiles,
-                         distsim_record *records, int64_t *launches);
+                         int64_t max_bucket_copies, distsim_record *records, int64_t *launches);
 
 // ---- probe (probe_kernels.cu) ----------------------------------------------------------
 // Launches the integer-issue probe; returns the number of integer instructions (per thread,
