@@ -218,6 +218,74 @@ def test_config1_full_size_sampled(E, ctx):
     check_emission(E, ctx, w, pick)
 
 
+def _flat_table(n_layers, n_devices, gpus_per_node, global_batch, space, per_layer_ns, seed):
+    """Table whose layer times do not depend on the micro-batch size, so that an entry's time
+    bound grows with m: small m fits 32 bits, large m does not."""
+    rng = np.random.default_rng(seed)
+    classes = W.event_classes(n_devices, global_batch, n_layers, space)
+    f = rng.integers(per_layer_ns // 2, per_layer_ns, n_layers)
+    g = 2 * f + rng.integers(0, 1000, n_layers)
+    return W.EventTable(
+        n_layers=n_layers, n_devices=n_devices, gpus_per_node=gpus_per_node, global_batch=global_batch,
+        seq=128, hidden=64, class_mp=[c[0] for c in classes], class_b=[c[1] for c in classes],
+        fwd_ns=np.tile(f, (len(classes), 1)), bwd_ns=np.tile(g, (len(classes), 1)),
+        layer_is_expert=(np.arange(n_layers) % 3 == 0).astype(np.uint8),
+        grad_bytes=rng.integers(1, 5 * 10**6, n_layers), dp_bucket_bytes=2 * 10**6)
+
+
+def test_rows_mixing_32_and_64_bit_entries(E, ctx):
+    # per micro-batch ~ 16 layers x 3 x 2^24 ns: the bound crosses 2^32 between m = 4 and m = 8,
+    # so one row is evaluated partly in uint32 and partly in int64 arithmetic
+    space = W.SearchSpace(mp_max=2, pp_max=8, m_list=[1, 2, 4, 8, 16], m_rule=W.M_RULE_CEIL,
+                          partition_mode=W.PARTITION_ALL)
+    table = _flat_table(16, 16, 4, 64, space, 1 << 24, 5)
+    w = W.Workload("mixed_width", table, space, 5)
+    n = load(E, ctx, w)
+    cells, cells32 = E.distsim_space_cells(ctx)
+    assert cells == W.count_candidates_and_cells(table, space)[1] and 0 < cells32 < cells
+    batch, sb = eval_all(E, ctx, n)
+    rng = np.random.default_rng(0)
+    idx = np.unique(np.concatenate([rng.integers(0, n, 4000), np.arange(0, n, max(1, n // 500)), [n - 1]]))
+    ob, obusy = oracle.eval_indices_parallel(table, space, idx, THREADS, pp_stride=space.pp_max)
+    sel = torch.from_numpy(idx).cuda()
+    assert (batch[sel].cpu().numpy() == ob).all()
+    assert (sb[sel].cpu().numpy() == obusy).all()
+    # an odd-aligned sub-range exercises the unpaired store path
+    first, count = 12345, 40001
+    out = dev(count + 1)[1:]
+    E.distsim_eval_strategies(ctx, first, count, out)
+    assert torch.equal(out, batch[first:first + count])
+    check_emission(E, ctx, w, [0, 7, int(idx[len(idx) // 2]), n - 1])
+
+
+@pytest.mark.parametrize("pp,n_layers", [(32, 34), (64, 66)])
+def test_long_pipelines_every_composition(E, ctx, pp, n_layers):
+    # lock-step kernel with all compositions: one and two stages per lane
+    space = W.SearchSpace(mp_max=1, pp_max=pp, m_list=[1, 3, 40, 70], m_rule=W.M_RULE_CEIL,
+                          partition_mode=W.PARTITION_ALL)
+    # an odd global batch admits dp = 1 only, so the space holds the pp = n_devices row alone
+    table = _flat_table(n_layers, pp, 8, 141, space, 50_000, pp)
+    w = W.Workload(f"long_{pp}", table, space, pp)
+    n = load(E, ctx, w)
+    batch, sb = eval_all(E, ctx, n)
+    cands = oracle.enumerate_at(table, space, np.arange(n))
+    assert all(c.pp == pp for c in cands)
+    idx = np.unique(np.concatenate([np.arange(0, n, 37), [n - 1]]))
+    ob, obusy = oracle.eval_indices_parallel(table, space, idx, THREADS, pp_stride=space.pp_max)
+    sel = torch.from_numpy(idx).cuda()
+    assert (batch[sel].cpu().numpy() == ob).all()
+    assert (sb[sel].cpu().numpy() == obusy).all()
+    check_emission(E, ctx, w, [int(idx[1]), int(idx[-2])])
+
+
+def test_integer_probes_run(E, ctx):
+    for mode in range(4):
+        assert E.distsim_int_issue_probe(ctx, 148, 64, mode) > 0
+    torch.cuda.synchronize()
+    with pytest.raises(E.DistsimError):
+        E.distsim_int_issue_probe(ctx, 148, 64, 9)
+
+
 def test_two_pass_argmin_for_wide_times(E, ctx):
     # times near 2^55 with a large count cannot be packed with the index into 64 bits
     w = W.random_small(3, lo=2**44, hi=2**45, partition_mode=W.PARTITION_ALL, n_layers=12, pp_max=4,
