@@ -85,6 +85,11 @@ const char *distsim_last_error(const distsim_ctx *ctx);
  *                                        event; 1: a bucket starts once the layer
  *                                        holding its last byte has finished the
  *                                        last micro-batch's backward
+ *   allreduce_profile_max                0: every all-reduce size is modelled directly;
+ *                                        k > 1: an all-reduce over n > k devices takes the
+ *                                        k-device time scaled by the per-device volume,
+ *                                        ceil(T(k) * k (n-1) / ((k-1) n))  (the paper profiles
+ *                                        up to 8 devices and extrapolates, Sec. 4.2)
  * Communication costs: ring all-reduce over n devices of S bytes
  * 2(n-1)alpha + ceil(2(n-1)S / (n beta)) (per-device volume 2(n-1)S/n, Sec. 4.2);
  * transfer alpha + ceil(S/beta); all-to-all (n-1)alpha + ceil((n-1)S/(n beta)).
@@ -104,6 +109,8 @@ typedef struct {
     const int64_t *fwd_ns, *bwd_ns;
     const uint8_t *layer_is_expert;
     const int64_t *grad_bytes;
+    int32_t allreduce_profile_max;
+    int32_t reserved;               /* must be 0 */
 } distsim_event_table;
 
 int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *h_table);

@@ -6,5 +6,5 @@ package; the CUDA engine never does, and this package imports nothing from it.
 """
 from .oracle import (  # noqa: F401
     KINDS, Candidate, OracleError, SimResult, build, count, enumerate_at, eval_indices,
-    eval_indices_parallel, ring_allreduce_ns, all_to_all_ns, p2p_ns, simulate,
+    eval_indices_parallel, ring_allreduce_ns, allreduce_ns, all_to_all_ns, p2p_ns, simulate,
 )

@@ -67,6 +67,10 @@ typedef struct {
     const int64_t *fwd_ns, *bwd_ns;       /* [n_classes][n_layers]                */
     const uint8_t *layer_is_expert;       /* [n_layers]                           */
     const int64_t *grad_bytes;            /* [n_layers], at mp = 1                */
+    int32_t allreduce_profile_max;        /* 0: every all-reduce size is modelled directly;
+                                             k > 0: all-reduces over more than k devices are
+                                             the k-device time scaled by the volume formula */
+    int32_t pad;
 } orc_table;
 
 /* The search space (paper Sec. 5: grid search over parallel degrees). */
@@ -121,6 +125,16 @@ static int list_push(orc_list *l, orc_event e)
 int64_t orc_ring_allreduce_ns(int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
 {
     return 2 * (n - 1) * alpha + cdiv(2 * (n - 1) * bytes, n * beta);
+}
+/* All-reduce event time.  The paper (Sec. 4.2) profiles all-reduces of up to 8 devices directly
+ * and, above that, takes the 8-device time and scales it by the per-device volume
+ * 2(N-1)P/N of the actual device count: T(n) = T(k) * [2(n-1)/n] / [2(k-1)/k], rounded up.
+ * Here the "profiled" times come from the ring alpha-beta form; k = 0 switches the
+ * extrapolation off (every size modelled directly). */
+int64_t orc_allreduce_ns(int64_t k, int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
+{
+    if (k <= 1 || n <= k) return orc_ring_allreduce_ns(n, bytes, alpha, beta);
+    return cdiv(orc_ring_allreduce_ns(k, bytes, alpha, beta) * k * (n - 1), (k - 1) * n);
 }
 /* Pairwise-exchange all-to-all: n-1 steps, each moving 1/n of the buffer. */
 int64_t orc_all_to_all_ns(int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
@@ -356,7 +370,7 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
     if (mp > 1) {
         int loc = loc_mp_groups(T, x);
         if (loc < 0) { e = ORC_E_LOCALITY; goto fail; }
-        AR = orc_ring_allreduce_ns(mp, 2 * act, alpha_of(T, loc), beta_of(T, loc));
+        AR = orc_allreduce_ns(T->allreduce_profile_max, mp, 2 * act, alpha_of(T, loc), beta_of(T, loc));
     }
     if (dp > 1) {
         loc_dp = loc_dp_groups(T, x);
@@ -500,7 +514,7 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                             if (ready < 0) { e = ORC_E_ARG; goto fail; }
                         }
                         const int64_t start = max64(ready, prev_end);
-                        const int64_t end = start + orc_ring_allreduce_ns(dp, hi - lo, alpha_of(T, loc_dp), beta_of(T, loc_dp));
+                        const int64_t end = start + orc_allreduce_ns(T->allreduce_profile_max, dp, hi - lo, alpha_of(T, loc_dp), beta_of(T, loc_dp));
                         if ((e = list_push(dst, (orc_event){ ORC_DP_AR, k, -1, start, end })) != ORC_OK) goto fail;
                         prev_end = end;
                     }

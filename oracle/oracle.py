@@ -37,7 +37,8 @@ class _Table(C.Structure):
                 ("dp_bucket_bytes", C.c_int64), ("dp_overlap", C.c_int32),
                 ("act_bytes_per_elem", C.c_int32), ("class_mp", C.c_void_p),
                 ("class_b", C.c_void_p), ("fwd_ns", C.c_void_p), ("bwd_ns", C.c_void_p),
-                ("layer_is_expert", C.c_void_p), ("grad_bytes", C.c_void_p)]
+                ("layer_is_expert", C.c_void_p), ("grad_bytes", C.c_void_p),
+                ("allreduce_profile_max", C.c_int32), ("pad", C.c_int32)]
 
 
 class _Space(C.Structure):
@@ -96,7 +97,7 @@ def _load():
         lib.orc_result_batch.restype = C.c_int64
         lib.orc_result_total_records.restype = C.c_int64
         lib.orc_result_n_lists.restype = C.c_int32
-        for f in (lib.orc_ring_allreduce_ns, lib.orc_all_to_all_ns, lib.orc_p2p_ns):
+        for f in (lib.orc_ring_allreduce_ns, lib.orc_all_to_all_ns, lib.orc_p2p_ns, lib.orc_allreduce_ns):
             f.restype = C.c_int64
         assert lib.orc_sizeof_candidate() == C.sizeof(_Cand)
         _lib = lib
@@ -115,7 +116,8 @@ def _table(t):
             np.ascontiguousarray(t.grad_bytes, np.int64)]
     s = _Table(t.n_layers, arrs[0].shape[0], t.n_devices, t.gpus_per_node, t.global_batch, t.seq,
                t.hidden, t.alpha_intra_ns, t.beta_intra, t.alpha_inter_ns, t.beta_inter,
-               t.dp_bucket_bytes, t.dp_overlap, t.act_bytes_per_elem, *[_ptr(a) for a in arrs])
+               t.dp_bucket_bytes, t.dp_overlap, t.act_bytes_per_elem, *[_ptr(a) for a in arrs],
+               int(getattr(t, "allreduce_profile_max", 0)), 0)
     return s, arrs
 
 
@@ -127,6 +129,10 @@ def _space(sp):
 
 def ring_allreduce_ns(n, nbytes, alpha, beta):
     return _load().orc_ring_allreduce_ns(C.c_int64(n), C.c_int64(nbytes), C.c_int64(alpha), C.c_int64(beta))
+
+
+def allreduce_ns(k, n, nbytes, alpha, beta):
+    return _load().orc_allreduce_ns(C.c_int64(k), C.c_int64(n), C.c_int64(nbytes), C.c_int64(alpha), C.c_int64(beta))
 
 
 def all_to_all_ns(n, nbytes, alpha, beta):

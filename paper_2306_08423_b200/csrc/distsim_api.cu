@@ -208,6 +208,8 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *t)
         return fail(ctx, DISTSIM_E_UNSUPPORTED, "n_devices and gpus_per_node must be powers of two");
     if (t->global_batch < 1 || t->seq < 0 || t->hidden < 0 || t->act_bytes_per_elem < 0)
         return fail(ctx, DISTSIM_E_ARG, "negative size");
+    if (t->allreduce_profile_max < 0 || t->allreduce_profile_max == 1 || t->reserved != 0)
+        return fail(ctx, DISTSIM_E_ARG, "bad allreduce_profile_max");
     if (t->alpha_intra_ns < 0 || t->alpha_inter_ns < 0 || t->beta_intra < 1 || t->beta_inter < 1 || t->dp_bucket_bytes < 0)
         return fail(ctx, DISTSIM_E_ARG, "bad link constants");
     const int64_t L = t->n_layers, K = t->n_classes;
@@ -230,7 +232,7 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *t)
     tc.hidden = t->hidden; tc.alpha_intra = t->alpha_intra_ns; tc.beta_intra = t->beta_intra;
     tc.alpha_inter = t->alpha_inter_ns; tc.beta_inter = t->beta_inter; tc.bucket = t->dp_bucket_bytes;
     tc.overlap = t->dp_overlap ? 1 : 0; tc.elem_bytes = t->act_bytes_per_elem;
-    tc.lp = (int32_t)((L + 1 + 1) & ~1); tc.pad = 0;
+    tc.lp = (int32_t)((L + 1 + 1) & ~1); tc.ar_profile_max = t->allreduce_profile_max;
     ctx->class_mp.assign(t->class_mp, t->class_mp + K);
     ctx->class_b.assign(t->class_b, t->class_b + K);
     ctx->fwd.assign(t->fwd_ns, t->fwd_ns + K * L);

@@ -38,7 +38,7 @@ struct TableConst {
     int32_t overlap;
     int32_t elem_bytes;
     int32_t lp;           // padded prefix-row length (int64 words)
-    int32_t pad;
+    int32_t ar_profile_max;   // all-reduces over more devices are extrapolated (0: never)
 };
 
 struct Row {

@@ -16,6 +16,15 @@ __device__ __forceinline__ int64_t ring_cost(int64_t n, int64_t bytes, int64_t a
     return 2 * (n - 1) * alpha + ceil_div(2 * (n - 1) * bytes, n * beta);
 }
 
+// All-reduce event time: directly modelled up to k = ar_profile_max devices; above, the k-device
+// time scaled by the per-device volume 2(n-1)S/n of the actual device count (paper Sec. 4.2).
+__device__ __forceinline__ int64_t allreduce_cost(const TableConst &tc, int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
+{
+    const int64_t k = tc.ar_profile_max;
+    if (k <= 1 || n <= k) return ring_cost(n, bytes, alpha, beta);
+    return ceil_div(ring_cost(k, bytes, alpha, beta) * k * (n - 1), (k - 1) * n);
+}
+
 // One thread per entry: the communication-event costs that depend on (mp, dp, b).
 // The first thread of each row also fills the row's full-bucket cost.
 __global__ void fill_entries_kernel(TableConst tc, Row *rows, int n_rows, Entry *entries, int n_entries)
@@ -32,7 +41,7 @@ __global__ void fill_entries_kernel(TableConst tc, Row *rows, int n_rows, Entry 
     const bool dp_inter = tc.n_devices > tc.gpus_per_node;
     en.ar = 0;
     if (row.mp > 1)
-        en.ar = ring_cost(row.mp, 2 * act, mp_inter ? tc.alpha_inter : tc.alpha_intra,
+        en.ar = allreduce_cost(tc, row.mp, 2 * act, mp_inter ? tc.alpha_inter : tc.alpha_intra,
                           mp_inter ? tc.beta_inter : tc.beta_intra);
     en.a2a = 0;
     if (row.dp > 1) {
@@ -46,7 +55,7 @@ __global__ void fill_entries_kernel(TableConst tc, Row *rows, int n_rows, Entry 
     if (i == row.entry0) {
         int64_t t_full = 0;
         if (row.dp > 1 && tc.bucket > 0)
-            t_full = ring_cost(row.dp, tc.bucket, dp_inter ? tc.alpha_inter : tc.alpha_intra,
+            t_full = allreduce_cost(tc, row.dp, tc.bucket, dp_inter ? tc.alpha_inter : tc.alpha_intra,
                                dp_inter ? tc.beta_inter : tc.beta_intra);
         rows[en.row].t_full = t_full;
     }
@@ -97,7 +106,7 @@ __global__ void build_bucket_tables_kernel(TableConst tc, RawTable raw, const Ro
         int64_t full = 0, rem = w;
         if (tc.bucket > 0) { full = w / tc.bucket; rem = w - full * tc.bucket; }
         nbr[l] = full;
-        tpr[l] = (rem > 0 && row.dp > 1) ? ring_cost(row.dp, rem, a, be) : 0;
+        tpr[l] = (rem > 0 && row.dp > 1) ? allreduce_cost(tc, row.dp, rem, a, be) : 0;
     }
     for (int l = e + 1; l < L1; ++l) { nbr[l] = 0; tpr[l] = 0; }
 }

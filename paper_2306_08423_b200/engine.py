@@ -47,7 +47,8 @@ class _Table(C.Structure):
                 ("dp_bucket_bytes", C.c_int64), ("dp_overlap", C.c_int32),
                 ("act_bytes_per_elem", C.c_int32), ("class_mp", C.c_void_p),
                 ("class_b", C.c_void_p), ("fwd_ns", C.c_void_p), ("bwd_ns", C.c_void_p),
-                ("layer_is_expert", C.c_void_p), ("grad_bytes", C.c_void_p)]
+                ("layer_is_expert", C.c_void_p), ("grad_bytes", C.c_void_p),
+                ("allreduce_profile_max", C.c_int32), ("reserved", C.c_int32)]
 
 
 class _Space(C.Structure):
@@ -106,7 +107,8 @@ def _table_struct(t):
             np.ascontiguousarray(t.grad_bytes, np.int64)]
     s = _Table(t.n_layers, arrs[0].shape[0], t.n_devices, t.gpus_per_node, t.global_batch, t.seq,
                t.hidden, t.alpha_intra_ns, t.beta_intra, t.alpha_inter_ns, t.beta_inter,
-               t.dp_bucket_bytes, t.dp_overlap, t.act_bytes_per_elem, *[_np_ptr(a) for a in arrs])
+               t.dp_bucket_bytes, t.dp_overlap, t.act_bytes_per_elem, *[_np_ptr(a) for a in arrs],
+               int(getattr(t, "allreduce_profile_max", 0)), 0)
     return s, arrs
 
 

@@ -88,6 +88,8 @@ class EventTable:
     dp_bucket_bytes: int = 25 * 2**20
     dp_overlap: int = 1
     act_bytes_per_elem: int = 2             # bf16 messages
+    allreduce_profile_max: int = 0          # k > 0: all-reduces over more than k devices are the
+                                            # k-device time scaled by the volume formula (paper Sec. 4.2)
 
     def __post_init__(self):
         self.class_mp = np.ascontiguousarray(self.class_mp, dtype=np.int32)
@@ -264,6 +266,19 @@ def config4(seed: int = 2) -> Workload:
     """Timeline emission: the 1024 fastest candidates of config 2."""
     w = config2(seed)
     return Workload("config4_emit_top1024_of_config2", w.table, w.space, seed, top_k=1024)
+
+
+def paper_grid(seed: int = 7) -> Workload:
+    """The shape of the paper's own strategy search (Sec. 5): 16 GPUs on 4 nodes, a 48-layer
+    transformer, global batch 16, every degree in {1, 2, 4, 8, 16}, with all-reduces above 8
+    devices extrapolated from the 8-device time (Sec. 4.2).  Event times are synthetic."""
+    space = SearchSpace(mp_max=16, pp_max=16, m_list=[1, 2, 4, 8, 16], m_rule=M_RULE_DIVIDES,
+                        partition_mode=PARTITION_BALANCED)
+    f1, u = _uniform_layers(SplitMix64(seed), 48, 200_000, 400_000)
+    table = build_table(per_sample_fwd_ns=f1, per_sample_bwd_extra_ns=u, n_devices=16,
+                        gpus_per_node=4, global_batch=16, seq=512, hidden=1024, space=space,
+                        allreduce_profile_max=8)
+    return Workload("paper_grid_16gpu_48layers", table, space, seed)
 
 
 CONFIGS = {0: config0, 1: config1, 2: config2, 3: config3, 4: config4}

@@ -278,6 +278,41 @@ def test_long_pipelines_every_composition(E, ctx, pp, n_layers):
     check_emission(E, ctx, w, [int(idx[1]), int(idx[-2])])
 
 
+@pytest.mark.parametrize("cfg,stride", [(1, 39_119), (2, 1), (3, 653)])
+def test_index_decoding_matches_loop_enumeration(E, ctx, cfg, stride):
+    # the library's index -> candidate mapping against the oracle's nested loops
+    w = W.CONFIGS[cfg]()
+    n = load(E, ctx, w)
+    idx = np.unique(np.concatenate([np.arange(0, n, stride), [n - 1]]))
+    for i, c in zip(idx.tolist(), oracle.enumerate_at(w.table, w.space, idx)):
+        d = E.distsim_decode(ctx, i)
+        assert (d["mp"], d["pp"], d["dp"], d["m"], d["sched"], d["bounds"]) == (c.mp, c.pp, c.dp, c.m, c.sched, c.bounds), i
+        assert d["micro_batch_size"] == -(-(w.table.global_batch // c.dp) // c.m)
+
+
+def test_paper_grid_with_extrapolated_allreduce(E, ctx):
+    # the paper's own search shape (16 GPUs, 48 layers, 15 valid (mp, pp) settings), with
+    # all-reduces above 8 devices extrapolated from the 8-device time
+    w = W.paper_grid()
+    n = load(E, ctx, w)
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    assert (batch.cpu().numpy() == ob).all() and (sb.cpu().numpy() == obusy).all()
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(n))
+    dp16 = [i for i, c in enumerate(cands) if c.dp == 16]
+    mp16 = [i for i, c in enumerate(cands) if c.mp == 16]
+    check_emission(E, ctx, w, dp16[:2] + mp16[:2] + [n // 2, n - 1])
+    # and a small irregular space where even 4- and 8-way all-reduces are extrapolated
+    w2 = W.random_small(41)
+    w2.table.allreduce_profile_max = 2
+    n2 = load(E, ctx, w2)
+    b2, s2 = eval_all(E, ctx, n2)
+    o2, ob2 = oracle.eval_indices_parallel(w2.table, w2.space, np.arange(n2), THREADS, pp_stride=w2.space.pp_max)
+    assert (b2.cpu().numpy() == o2).all() and (s2.cpu().numpy() == ob2).all()
+    check_emission(E, ctx, w2, list(range(0, n2, max(1, n2 // 12))))
+
+
 def test_integer_probes_run(E, ctx):
     for mode in range(4):
         assert E.distsim_int_issue_probe(ctx, 148, 64, mode) > 0

@@ -53,6 +53,40 @@ def test_ring_allreduce_volume_matches_paper_formula():
     assert oracle.ring_allreduce_ns(2, 301, 0, 300) == 2  # rounds up
 
 
+def test_allreduce_extrapolation_above_profiled_size():
+    # Sec. 4.2: up to k devices the all-reduce is taken as profiled; above, the k-device time is
+    # scaled by the per-device volume 2(N-1)P/N of the actual device count
+    k, a, be = 8, 10_000, 25
+    for p in (1, 4096, 26214400):
+        t8 = oracle.ring_allreduce_ns(8, p, a, be)
+        for n in (2, 4, 8):
+            assert oracle.allreduce_ns(k, n, p, a, be) == oracle.ring_allreduce_ns(n, p, a, be)
+        for n in (16, 64, 1024):
+            got = oracle.allreduce_ns(k, n, p, a, be)
+            want = t8 * (2 * (n - 1) / n) / (2 * 7 / 8)
+            assert got == -(-t8 * 8 * (n - 1) // (7 * n)) and abs(got - want) <= 1
+            assert got < 8 * t8 / 7 + 1                       # bounded: tends to T(8) * 8/7
+        assert oracle.allreduce_ns(0, 64, p, a, be) == oracle.ring_allreduce_ns(64, p, a, be)
+    # end to end: pure DP on 16 devices with one bucket
+    f, g = [5, 11, 3], [9, 20, 8]
+    grad = np.array([1000, 555, 77], np.int64)
+    T = make_table(f, g, n_devices=16, gpus_per_node=4, global_batch=16, classes=[(1, 1)], grad=grad,
+                   dp_bucket_bytes=0, dp_overlap=0, alpha_intra_ns=3, beta_intra=16, alpha_inter_ns=40,
+                   beta_inter=2, allreduce_profile_max=8)
+    r = oracle.simulate(T, Candidate(1, 1, 16, 1, 0, (0, 3)))
+    t8 = 2 * 7 * 40 + -(-2 * 7 * 1632 // (8 * 2))
+    assert r.batch_ns == sum(f) + sum(g) + -(-t8 * 8 * 15 // (7 * 16))
+
+
+def test_paper_grid_workload_shape():
+    w = W.paper_grid()
+    assert oracle.count(w.table, w.space) == 2 * sum(
+        len([m for m in (1, 2, 4, 8, 16) if (16 // dp) % m == 0])
+        for mp in (1, 2, 4, 8, 16) for pp in (1, 2, 4, 8, 16) if mp * pp <= 16 for dp in [16 // (mp * pp)])
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(oracle.count(w.table, w.space)))
+    assert len({(c.mp, c.pp) for c in cands}) == 15           # Sec. 5: 15 valid settings of 25
+
+
 def test_p2p_and_all_to_all_formulas():
     assert oracle.p2p_ns(1000, 7, 10) == 107
     assert oracle.p2p_ns(1001, 7, 10) == 108
