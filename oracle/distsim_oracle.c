@@ -50,7 +50,8 @@ enum {
     ORC_MP_AR_F = 2,   ORC_MP_AR_B = 3,
     ORC_A2A_F = 4,     ORC_A2A_B = 5,
     ORC_SEND_F = 6,    ORC_SEND_B = 7,
-    ORC_DP_AR = 8
+    ORC_DP_AR = 8,
+    ORC_JITTER_F = 9,  ORC_JITTER_B = 10   /* per-micro-batch fluctuation at the start of an item */
 };
 
 /* The event table: profiled (here: synthetic) event times per class, plus the
@@ -70,7 +71,13 @@ typedef struct {
     int32_t allreduce_profile_max;        /* 0: every all-reduce size is modelled directly;
                                              k > 0: all-reduces over more than k devices are
                                              the k-device time scaled by the volume formula */
+    int32_t n_jitter;                     /* P: number of micro-batch slots of the jitter table
+                                             (0: all micro-batches of a stage cost the same)  */
+    int32_t jitter_stages;                /* columns of the jitter tables (>= pp of any strategy) */
     int32_t pad;
+    const int64_t *jitter_fwd_ns;         /* [P][jitter_stages]: extra time of the forward item of
+                                             micro-batch j on stage d is [j mod P][d]          */
+    const int64_t *jitter_bwd_ns;         /* same for backward items                           */
 } orc_table;
 
 /* The search space (paper Sec. 5: grid search over parallel degrees). */
@@ -351,7 +358,8 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
 
     if (pp < 1 || pp > ORC_MAX_PP || mp < 1 || dp < 1 || m < 1 ||
         (int64_t)mp * pp * dp != T->n_devices || T->global_batch % dp != 0 ||
-        x->bounds[0] != 0 || x->bounds[pp] != L || (x->sched != 0 && x->sched != 1)) {
+        x->bounds[0] != 0 || x->bounds[pp] != L || (x->sched != 0 && x->sched != 1) ||
+        (T->n_jitter > 0 && (T->jitter_stages < pp || !T->jitter_fwd_ns || !T->jitter_bwd_ns))) {
         e = ORC_E_ARG; goto fail;
     }
     for (int d = 0; d < pp; ++d) if (x->bounds[d + 1] <= x->bounds[d]) { e = ORC_E_ARG; goto fail; }
@@ -387,7 +395,7 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
     ops = (orc_op *)malloc((size_t)pp * 2 * m * sizeof(orc_op));
     endF = (int64_t *)malloc((size_t)pp * m * sizeof(int64_t));
     endB = (int64_t *)malloc((size_t)pp * m * sizeof(int64_t));
-    tmp = (orc_event *)malloc((size_t)(3 * L + 1) * sizeof(orc_event));
+    tmp = (orc_event *)malloc((size_t)(3 * L + 2) * sizeof(orc_event));
     const int mp_lists = replicate ? mp : 1;
     F = (orc_list *)calloc((size_t)pp * mp_lists, sizeof(orc_list));
     if (!ops || !endF || !endB || !tmp || !F) { e = ORC_E_NOMEM; goto fail; }
@@ -435,6 +443,17 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
              * its all-reduce event (mp > 1) and its all-to-all event (expert layer,
              * dp > 1); then e_comm, the transfer to the neighbouring stage. */
             int n = 0;
+            /* Fluctuation between micro-batches (the paper's error analysis, Sec. 6.3, blames
+             * profiling fluctuation that accumulates along the stages): when a jitter table is
+             * given, the item of micro-batch j on stage d begins with a jitter event of
+             * [j mod P][d] ns, before its first computation event. */
+            if (T->n_jitter > 0) {
+                const int64_t *jt = o.is_bwd ? T->jitter_bwd_ns : T->jitter_fwd_ns;
+                const int64_t jit = jt[(int64_t)(o.mb % T->n_jitter) * T->jitter_stages + d];
+                const int first_layer = o.is_bwd ? x->bounds[d + 1] - 1 : x->bounds[d];
+                tmp[n++] = (orc_event){ o.is_bwd ? ORC_JITTER_B : ORC_JITTER_F, first_layer, o.mb, t, t + jit };
+                t += jit;
+            }
             if (!o.is_bwd) {
                 for (int l = x->bounds[d]; l < x->bounds[d + 1]; ++l) {
                     tmp[n++] = (orc_event){ ORC_COMPUTE_F, l, o.mb, t, t + f[l] }; t += f[l];

@@ -20,7 +20,7 @@ _LIB = os.path.join(_HERE, "_liborc.so")
 _MAX_PP = 64
 
 KINDS = {"COMPUTE_F": 0, "COMPUTE_B": 1, "MP_AR_F": 2, "MP_AR_B": 3, "A2A_F": 4, "A2A_B": 5,
-         "SEND_F": 6, "SEND_B": 7, "DP_AR": 8}
+         "SEND_F": 6, "SEND_B": 7, "DP_AR": 8, "JITTER_F": 9, "JITTER_B": 10}
 
 
 class OracleError(RuntimeError):
@@ -38,7 +38,9 @@ class _Table(C.Structure):
                 ("act_bytes_per_elem", C.c_int32), ("class_mp", C.c_void_p),
                 ("class_b", C.c_void_p), ("fwd_ns", C.c_void_p), ("bwd_ns", C.c_void_p),
                 ("layer_is_expert", C.c_void_p), ("grad_bytes", C.c_void_p),
-                ("allreduce_profile_max", C.c_int32), ("pad", C.c_int32)]
+                ("allreduce_profile_max", C.c_int32), ("n_jitter", C.c_int32),
+                ("jitter_stages", C.c_int32), ("pad", C.c_int32),
+                ("jitter_fwd_ns", C.c_void_p), ("jitter_bwd_ns", C.c_void_p)]
 
 
 class _Space(C.Structure):
@@ -117,7 +119,15 @@ def _table(t):
     s = _Table(t.n_layers, arrs[0].shape[0], t.n_devices, t.gpus_per_node, t.global_batch, t.seq,
                t.hidden, t.alpha_intra_ns, t.beta_intra, t.alpha_inter_ns, t.beta_inter,
                t.dp_bucket_bytes, t.dp_overlap, t.act_bytes_per_elem, *[_ptr(a) for a in arrs],
-               int(getattr(t, "allreduce_profile_max", 0)), 0)
+               int(getattr(t, "allreduce_profile_max", 0)), 0, 0, 0, None, None)
+    jf = getattr(t, "jitter_fwd_ns", None)
+    if jf is not None and np.size(jf) > 0:
+        jf = np.ascontiguousarray(jf, np.int64)
+        jb = np.ascontiguousarray(t.jitter_bwd_ns, np.int64)
+        assert jf.ndim == 2 and jf.shape == jb.shape
+        s.n_jitter, s.jitter_stages = jf.shape
+        s.jitter_fwd_ns, s.jitter_bwd_ns = _ptr(jf), _ptr(jb)
+        arrs += [jf, jb]
     return s, arrs
 
 

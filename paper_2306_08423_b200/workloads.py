@@ -90,6 +90,8 @@ class EventTable:
     act_bytes_per_elem: int = 2             # bf16 messages
     allreduce_profile_max: int = 0          # k > 0: all-reduces over more than k devices are the
                                             # k-device time scaled by the volume formula (paper Sec. 4.2)
+    jitter_fwd_ns: np.ndarray = None        # int64 [P, stages] or None: extra time of the forward
+    jitter_bwd_ns: np.ndarray = None        # (backward) item of micro-batch j on stage d is [j mod P, d]
 
     def __post_init__(self):
         self.class_mp = np.ascontiguousarray(self.class_mp, dtype=np.int32)
@@ -98,6 +100,10 @@ class EventTable:
         self.bwd_ns = np.ascontiguousarray(self.bwd_ns, dtype=np.int64)
         self.layer_is_expert = np.ascontiguousarray(self.layer_is_expert, dtype=np.uint8)
         self.grad_bytes = np.ascontiguousarray(self.grad_bytes, dtype=np.int64)
+        if self.jitter_fwd_ns is not None:
+            self.jitter_fwd_ns = np.ascontiguousarray(self.jitter_fwd_ns, dtype=np.int64)
+            self.jitter_bwd_ns = np.ascontiguousarray(self.jitter_bwd_ns, dtype=np.int64)
+            assert self.jitter_fwd_ns.ndim == 2 and self.jitter_fwd_ns.shape == self.jitter_bwd_ns.shape
         assert self.fwd_ns.shape == (self.n_classes, self.n_layers)
         assert self.bwd_ns.shape == (self.n_classes, self.n_layers)
 
@@ -279,6 +285,17 @@ def paper_grid(seed: int = 7) -> Workload:
                         gpus_per_node=4, global_batch=16, seq=512, hidden=1024, space=space,
                         allreduce_profile_max=8)
     return Workload("paper_grid_16gpu_48layers", table, space, seed)
+
+
+def add_jitter(w: Workload, slots: int, max_ns: int, seed: int = 11) -> Workload:
+    """Gives a workload a per-micro-batch jitter table: `slots` (a power of two) micro-batch
+    slots x pp_max stages of extra item time, uniform in [0, max_ns]."""
+    rng = SplitMix64(seed)
+    stages = w.space.pp_max
+    w.table.jitter_fwd_ns = np.array([[rng.randint(0, max_ns) for _ in range(stages)] for _ in range(slots)], np.int64)
+    w.table.jitter_bwd_ns = np.array([[rng.randint(0, max_ns) for _ in range(stages)] for _ in range(slots)], np.int64)
+    w.name += f"_jitter{slots}"
+    return w
 
 
 CONFIGS = {0: config0, 1: config1, 2: config2, 3: config3, 4: config4}

@@ -76,6 +76,9 @@ def longest_path_timeline(table, cand):
         for (typ, j) in stage_order(cand.sched, pp, d, m):
             evs = []
             layers = range(c[d], c[d + 1]) if typ == "F" else range(c[d + 1] - 1, c[d] - 1, -1)
+            jt = getattr(T, "jitter_fwd_ns" if typ == "F" else "jitter_bwd_ns", None)
+            if jt is not None:
+                evs.append((9 if typ == "F" else 10, layers[0], int(jt[j % len(jt)][d])))
             for l in layers:
                 evs.append((0 if typ == "F" else 1, l, f[l] if typ == "F" else g[l]))
                 if mp > 1:

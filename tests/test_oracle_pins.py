@@ -167,10 +167,13 @@ def test_single_stage_sum():
 def test_hand_worked_examples():
     rows = [l.split() for l in open(os.path.join(GOLDEN, "worked_pipeline_examples.txt"))
             if l.strip() and not l.startswith("#")]
-    assert len(rows) == 4
+    assert len(rows) == 6
     for name, p2p, sched, batch, busy0, busy1 in rows:
+        jit = {}
+        if name == "W3":
+            jit = dict(jitter_fwd_ns=np.array([[0, 0], [3, 0]]), jitter_bwd_ns=np.zeros((2, 2), np.int64))
         T = make_table([1, 1], [2, 2], n_devices=2, gpus_per_node=1, global_batch=2, classes=[(1, 1)],
-                       alpha_intra_ns=int(p2p), alpha_inter_ns=int(p2p))
+                       alpha_intra_ns=int(p2p), alpha_inter_ns=int(p2p), **jit)
         r = oracle.simulate(T, Candidate(1, 2, 1, 2, int(sched), (0, 1, 2)))
         assert r.batch_ns == int(batch), name
         assert r.busy_ns.tolist() == [int(busy0), int(busy1)]
@@ -200,6 +203,63 @@ def test_brute_force_longest_path(w):
         for d in range(c.pp):
             got = [tuple(x) for x in r.records[r.offsets[d]:r.offsets[d + 1]].tolist()]
             assert got == lanes[d], (c, d)
+
+
+# per-micro-batch jitter
+def _jittered(seed, **kw):
+    w = W.random_small(seed, n_devices=8, gpus_per_node=4, n_layers=4, global_batch=8, mp_max=2,
+                       pp_max=4, m_list=(1, 2, 3, 5), dp_bucket_bytes=700, **kw)
+    return W.add_jitter(w, 4, 900, seed)
+
+
+@pytest.mark.parametrize("seed", range(60, 66))
+def test_jitter_brute_force_longest_path(seed):
+    w = _jittered(seed, dp_overlap=seed % 2)
+    n = oracle.count(w.table, w.space)
+    for c in oracle.enumerate_at(w.table, w.space, np.arange(n)):
+        r = oracle.simulate(w.table, c, replicate=False)
+        batch, lanes = longest_path_timeline(w.table, c)
+        assert r.batch_ns == batch
+        for d in range(c.pp):
+            got = [tuple(x) for x in r.records[r.offsets[d]:r.offsets[d + 1]].tolist()]
+            assert got == lanes[d], (c, d)
+
+
+def test_jitter_special_cases():
+    import copy
+    w = _jittered(70)
+    n = oracle.count(w.table, w.space)
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(0, n, 7))
+    plain = copy.deepcopy(w.table); plain.jitter_fwd_ns = None; plain.jitter_bwd_ns = None
+    zero = copy.deepcopy(w.table); zero.jitter_fwd_ns[:] = 0; zero.jitter_bwd_ns[:] = 0
+    more = copy.deepcopy(w.table); more.jitter_fwd_ns[2, 1] += 55
+    for c in cands:
+        r0 = oracle.simulate(plain, c, replicate=False)
+        rz = oracle.simulate(zero, c, replicate=False)
+        rj = oracle.simulate(w.table, c, replicate=False)
+        # an all-zero table changes no time; it only adds one zero-length event per item
+        assert rz.batch_ns == r0.batch_ns and (rz.busy_ns == r0.busy_ns).all()
+        keep = ~np.isin(rz.records[:, 0], [9, 10])
+        assert (rz.records[keep] == r0.records).all()
+        assert (~keep).sum() == 2 * c.m * c.pp and (rz.records[~keep, 4] == rz.records[~keep, 3]).all()
+        # jitter only delays, and more jitter delays more
+        assert rj.batch_ns >= r0.batch_ns
+        assert oracle.simulate(more, c, replicate=False).batch_ns >= rj.batch_ns
+        # busy time = sum of durations on the main lane (+ bucket excess): check the main lane
+        for d in range(c.pp):
+            rec = rj.records[rj.offsets[d]:rj.offsets[d + 1]]
+            main = rec[rec[:, 0] != 8]
+            jit = main[np.isin(main[:, 0], [9, 10])]
+            want = sum(int(w.table.jitter_fwd_ns[j % 4, d]) + int(w.table.jitter_bwd_ns[j % 4, d]) for j in range(c.m))
+            assert int((jit[:, 4] - jit[:, 3]).sum()) == want
+    # constant jitter on uniform stages: the closed form with longer items
+    pp, m, tf, tb, cj = 4, 6, 7, 13, 5
+    T = make_table([tf] * pp, [tb] * pp, n_devices=pp, gpus_per_node=1, global_batch=m, classes=[(1, 1)],
+                   alpha_intra_ns=0, alpha_inter_ns=0, jitter_fwd_ns=np.full((2, pp), cj),
+                   jitter_bwd_ns=np.full((2, pp), cj))
+    for sched in (0, 1):
+        r = oracle.simulate(T, Candidate(1, pp, 1, m, sched, balanced(pp, pp)))
+        assert r.batch_ns == (m + pp - 1) * (tf + tb + 2 * cj)
 
 
 # --------------------------------------------------------------------------- #
