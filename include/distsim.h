@@ -55,7 +55,8 @@ enum {
     DISTSIM_MP_AR_F = 2,   DISTSIM_MP_AR_B = 3,     /* model-parallel all-reduce     */
     DISTSIM_A2A_F = 4,     DISTSIM_A2A_B = 5,       /* expert-layer all-to-all       */
     DISTSIM_SEND_F = 6,    DISTSIM_SEND_B = 7,      /* transfer to the neighbour     */
-    DISTSIM_DP_AR = 8                               /* gradient all-reduce bucket    */
+    DISTSIM_DP_AR = 8,                              /* gradient all-reduce bucket    */
+    DISTSIM_JITTER_F = 9,  DISTSIM_JITTER_B = 10    /* fluctuation at an item's start */
 };
 
 typedef struct distsim_ctx distsim_ctx;
@@ -90,6 +91,13 @@ const char *distsim_last_error(const distsim_ctx *ctx);
  *                                        k-device time scaled by the per-device volume,
  *                                        ceil(T(k) * k (n-1) / ((k-1) n))  (the paper profiles
  *                                        up to 8 devices and extrapolates, Sec. 4.2)
+ *   n_jitter, jitter_*                   fluctuation between micro-batches (the paper's error
+ *                                        analysis, Sec. 6.3, blames profiling fluctuation that
+ *                                        accumulates along the stages): with P = n_jitter > 0 the
+ *                                        forward (backward) item of micro-batch j on stage d
+ *                                        begins with a jitter event of jitter_fwd_ns
+ *                                        (jitter_bwd_ns) [j mod P][d] ns.  Every strategy of the
+ *                                        space must have pp <= jitter_stages.
  * Communication costs: ring all-reduce over n devices of S bytes
  * 2(n-1)alpha + ceil(2(n-1)S / (n beta)) (per-device volume 2(n-1)S/n, Sec. 4.2);
  * transfer alpha + ceil(S/beta); all-to-all (n-1)alpha + ceil((n-1)S/(n beta)).
@@ -110,7 +118,10 @@ typedef struct {
     const uint8_t *layer_is_expert;
     const int64_t *grad_bytes;
     int32_t allreduce_profile_max;
-    int32_t reserved;               /* must be 0 */
+    int32_t n_jitter;               /* P: 0, or a power of two <= 64                */
+    int32_t jitter_stages;          /* columns of the jitter tables, <= 64         */
+    int32_t reserved;               /* must be 0                                   */
+    const int64_t *jitter_fwd_ns, *jitter_bwd_ns;   /* [P][jitter_stages], NULL if P == 0 */
 } distsim_event_table;
 
 int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *h_table);

@@ -58,7 +58,7 @@ struct distsim_ctx {
     std::vector<int32_t> class_mp, class_b;
     std::vector<int64_t> fwd, bwd, grad;
     std::vector<uint8_t> expert;
-    DevBuf d_class_mp, d_class_b, d_fwd, d_bwd, d_expert, d_grad, d_next_grad, d_pe;
+    DevBuf d_class_mp, d_class_b, d_fwd, d_bwd, d_expert, d_grad, d_next_grad, d_pe, d_jit_f, d_jit_b, d_jsum;
     RawTable raw{};
 
     // space
@@ -86,6 +86,7 @@ struct distsim_ctx {
         v.dt = have_dt ? d_dt.as<int64_t>() : nullptr;
         v.tab_words = ((tc.n_layers + 1) * (tc.n_layers + 1) + 1) & ~1;
         v.next_grad = d_next_grad.as<int32_t>(); v.pe = d_pe.as<int32_t>();
+        v.jsum = tc.n_jitter > 0 ? d_jsum.as<int64_t>() : nullptr;
         v.status = d_status.as<int32_t>();
         return v;
     }
@@ -210,6 +211,16 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *t)
         return fail(ctx, DISTSIM_E_ARG, "negative size");
     if (t->allreduce_profile_max < 0 || t->allreduce_profile_max == 1 || t->reserved != 0)
         return fail(ctx, DISTSIM_E_ARG, "bad allreduce_profile_max");
+    if (t->n_jitter < 0 || t->n_jitter > 64 || (t->n_jitter & (t->n_jitter - 1)))
+        return fail(ctx, DISTSIM_E_UNSUPPORTED, "n_jitter must be 0 or a power of two <= 64");
+    if (t->n_jitter > 0) {
+        if (!t->jitter_fwd_ns || !t->jitter_bwd_ns || t->jitter_stages < 1 || t->jitter_stages > DISTSIM_MAX_PP)
+            return fail(ctx, DISTSIM_E_ARG, "bad jitter tables");
+        for (int64_t i = 0; i < (int64_t)t->n_jitter * t->jitter_stages; ++i)
+            if (t->jitter_fwd_ns[i] < 0 || t->jitter_bwd_ns[i] < 0 || t->jitter_fwd_ns[i] >= kSat / 8192 ||
+                t->jitter_bwd_ns[i] >= kSat / 8192)
+                return fail(ctx, DISTSIM_E_ARG, "jitter out of range");
+    }
     if (t->alpha_intra_ns < 0 || t->alpha_inter_ns < 0 || t->beta_intra < 1 || t->beta_inter < 1 || t->dp_bucket_bytes < 0)
         return fail(ctx, DISTSIM_E_ARG, "bad link constants");
     const int64_t L = t->n_layers, K = t->n_classes;
@@ -233,6 +244,7 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *t)
     tc.alpha_inter = t->alpha_inter_ns; tc.beta_inter = t->beta_inter; tc.bucket = t->dp_bucket_bytes;
     tc.overlap = t->dp_overlap ? 1 : 0; tc.elem_bytes = t->act_bytes_per_elem;
     tc.lp = (int32_t)((L + 1 + 1) & ~1); tc.ar_profile_max = t->allreduce_profile_max;
+    tc.n_jitter = t->n_jitter; tc.jitter_stages = t->n_jitter > 0 ? t->jitter_stages : 0;
     ctx->class_mp.assign(t->class_mp, t->class_mp + K);
     ctx->class_b.assign(t->class_b, t->class_b + K);
     ctx->fwd.assign(t->fwd_ns, t->fwd_ns + K * L);
@@ -251,6 +263,13 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *t)
     ctx->raw.class_mp = ctx->d_class_mp.as<int32_t>(); ctx->raw.class_b = ctx->d_class_b.as<int32_t>();
     ctx->raw.fwd = ctx->d_fwd.as<int64_t>(); ctx->raw.bwd = ctx->d_bwd.as<int64_t>();
     ctx->raw.expert = ctx->d_expert.as<uint8_t>(); ctx->raw.grad = ctx->d_grad.as<int64_t>();
+    ctx->raw.jit_f = ctx->raw.jit_b = nullptr;
+    if (t->n_jitter > 0) {
+        const size_t nj = (size_t)t->n_jitter * t->jitter_stages;
+        if (int rc = upload(ctx, ctx->d_jit_f, t->jitter_fwd_ns, nj, "upload jitter")) return rc;
+        if (int rc = upload(ctx, ctx->d_jit_b, t->jitter_bwd_ns, nj, "upload jitter")) return rc;
+        ctx->raw.jit_f = ctx->d_jit_f.as<int64_t>(); ctx->raw.jit_b = ctx->d_jit_b.as<int64_t>();
+    }
     launch_build_layer_tables(0, tc, ctx->raw, ctx->d_next_grad.as<int32_t>(), ctx->d_pe.as<int32_t>(), &ctx->launches);
     CU(cudaGetLastError(), "layer tables launch");
     ctx->table_loaded = true;
@@ -358,6 +377,9 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
             rows.push_back(r);
         }
     if (rows.empty()) return fail(ctx, DISTSIM_E_ARG, "the space has no valid candidate");
+    if (tc.n_jitter > 0)
+        for (const Row &r : rows)
+            if (r.pp > tc.jitter_stages) return fail(ctx, DISTSIM_E_ARG, "a strategy has more stages than the jitter tables have columns");
     if (tb >= (long double)kSat) return fail(ctx, DISTSIM_E_OVERFLOW, "batch-time bound does not fit 62 bits");
 
     ctx->rows = rows; ctx->entries = entries; ctx->binom = binom;
@@ -385,8 +407,9 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     const size_t dt_bytes = entries.size() * (size_t)(((L + 1) * (L + 1) + 1) & ~1) * sizeof(int64_t);
     ctx->have_dt = sp->partition_mode == 1 && dt_bytes <= ((size_t)256 << 20);
     if (ctx->have_dt) CU(ctx->d_dt.reserve(dt_bytes), "alloc bucket-lane tables");
+    if (tc.n_jitter > 0) CU(ctx->d_jsum.reserve(entries.size() * DISTSIM_MAX_PP * sizeof(int64_t)), "alloc jitter sums");
     launch_build_entry_tables(0, ctx->view(), ctx->d_entries.as<Entry>(), ctx->have_dt ? ctx->d_dt.as<int64_t>() : nullptr,
-                              &ctx->launches);
+                              tc.n_jitter > 0 ? ctx->d_jsum.as<int64_t>() : nullptr, &ctx->launches);
     CU(cudaGetLastError(), "set-up launch");
     // the host copies take the device-filled fields; these copies also wait for set-up
     CU(cudaMemcpy(ctx->rows.data(), ctx->d_rows.p, rows.size() * sizeof(Row), cudaMemcpyDeviceToHost), "rows readback");

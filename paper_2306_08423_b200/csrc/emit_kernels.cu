@@ -50,7 +50,7 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
     const int64_t *pf = v.etf + (int64_t)cc.entry * v.tc.lp;
     const int64_t *pb = v.etb + (int64_t)cc.entry * v.tc.lp;
     const int n_slots = 2 * (en.m + row.pp - 1);
-    const StageResult<S> R = lockstep_candidate<S, true>(v, row, en, pf, pb, cc.sched, cc.part_rank,
+    const StageResult<S> R = lockstep_candidate<S, true>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank,
                                                          seg_lane, wl, n_slots, owner ? rec : nullptr);
     if (owner) {
         const int L1 = v.tc.n_layers + 1;
@@ -60,7 +60,8 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
             const int a = R.a[k], e = R.e[k];
             const int n_layers = e - a;
             const int n_exp = v.pe[e] - v.pe[a];
-            const int64_t per_dir = (int64_t)n_layers * (row.mp > 1 ? 2 : 1) + (row.dp > 1 ? n_exp : 0);
+            const int64_t per_dir = (int64_t)n_layers * (row.mp > 1 ? 2 : 1) + (row.dp > 1 ? n_exp : 0) +
+                                    (v.tc.n_jitter > 0 ? 1 : 0);      // an item starts with its jitter event
             const int64_t rf = per_dir + (d < row.pp - 1 ? 1 : 0);
             const int64_t rb = per_dir + (d > 0 ? 1 : 0);
             int64_t kb = 0;
@@ -202,6 +203,7 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     __shared__ int64_t start_s[kMaxTileItems];          // start time of each item of the run
     __shared__ int32_t ioff[kMaxTileItems + 1];         // word offset of each item inside the run
     __shared__ int32_t meta_s[kMaxTileItems];           // micro-batch << 1 | is-backward
+    __shared__ int64_t jit_s[kMaxTileItems];            // jitter at the start of each item
     const int i = blockIdx.y;
     const EmitPlan &p = plans[i];
     if (!p.ok) return;
@@ -228,12 +230,17 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     const int per_layer = row_mp > 1 ? 2 : 1;
     const int64_t ar = en.ar, a2a = en.a2a;
     int64_t *tf = tmpl, *tb = tmpl + (int64_t)rf * 5;
+    const int jr = v.tc.n_jitter > 0 ? 1 : 0;           // record 0 of an item is its jitter event
 
-    // ---- item templates: records relative to the item's start --------------------------
+    // ---- item templates: records relative to the end of the item's jitter event ----------
+    if (jr && threadIdx.x == 32) {
+        tf[0] = DISTSIM_JITTER_F; tf[1] = a; tf[2] = 0; tf[3] = 0; tf[4] = 0;
+        tb[0] = DISTSIM_JITTER_B; tb[1] = e - 1; tb[2] = 0; tb[3] = 0; tb[4] = 0;
+    }
     for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
         const bool ex = row_dp > 1 && v.raw.expert[l];
         {   // forward: layers ascending
-            const int r = (l - a) * per_layer + (row_dp > 1 ? v.pe[l] - v.pe[a] : 0);
+            const int r = jr + (l - a) * per_layer + (row_dp > 1 ? v.pe[l] - v.pe[a] : 0);
             int64_t t = pf[l] - pf[a];
             int64_t *w = tf + (int64_t)r * 5;
             w[0] = DISTSIM_COMPUTE_F; w[1] = l; w[2] = 0; w[3] = t; t += f[l]; w[4] = t; w += 5;
@@ -241,7 +248,7 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
             if (ex) { w[0] = DISTSIM_A2A_F; w[1] = l; w[2] = 0; w[3] = t; t += a2a; w[4] = t; }
         }
         {   // backward: layers descending
-            const int r = (e - 1 - l) * per_layer + (row_dp > 1 ? v.pe[e] - v.pe[l + 1] : 0);
+            const int r = jr + (e - 1 - l) * per_layer + (row_dp > 1 ? v.pe[e] - v.pe[l + 1] : 0);
             int64_t t = pb[e] - pb[l + 1];
             int64_t *w = tb + (int64_t)r * 5;
             w[0] = DISTSIM_COMPUTE_B; w[1] = l; w[2] = 0; w[3] = t; t += g[l]; w[4] = t; w += 5;
@@ -264,6 +271,7 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
             if (k < n_items) {
                 start_s[k] = op_start[(int64_t)i * op_words_per_cand + (int64_t)d * 2 * m + s0 + k];
                 meta_s[k] = (j << 1) | (bwd ? 1 : 0);
+                jit_s[k] = jitter_of(v, bwd ? v.raw.jit_b : v.raw.jit_f, j, d);
             }
         }
     }
@@ -314,7 +322,9 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         const int meta = meta_s[it];
         const int field = w - (w / 5) * 5;
         int64_t t = ((meta & 1) ? tb : tf)[w];
-        t += field == 2 ? (int64_t)(meta >> 1) : (field >= 3 ? start_s[it] : 0);
+        // times: the jitter event runs [start, start + jitter); every later event is relative to its end
+        if (field == 2) t += (int64_t)(meta >> 1);
+        else if (field >= 3) t += start_s[it] + ((jr && w != 3) ? jit_s[it] : 0);
         return t;
     };
     for (int x0 = 0; x0 < total; x0 += 2 * kItemThreads) {

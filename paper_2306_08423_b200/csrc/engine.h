@@ -39,6 +39,8 @@ struct TableConst {
     int32_t elem_bytes;
     int32_t lp;           // padded prefix-row length (int64 words)
     int32_t ar_profile_max;   // all-reduces over more devices are extrapolated (0: never)
+    int32_t n_jitter;         // P: micro-batch slots of the jitter tables (0 or a power of two)
+    int32_t jitter_stages;    // columns of the jitter tables
 };
 
 struct Row {
@@ -74,6 +76,7 @@ struct RawTable {
     const int64_t *fwd, *bwd;        // [n_classes][n_layers]
     const uint8_t *expert;           // [n_layers]
     const int64_t *grad;             // [n_layers]
+    const int64_t *jit_f, *jit_b;    // [n_jitter][jitter_stages] extra item time (nullptr if none)
 };
 
 // Everything a kernel needs, passed by value.
@@ -91,6 +94,8 @@ struct DeviceView {
     const int64_t *binom;            // [n_layers][binom_k]
     const int32_t *next_grad;        // [L+1] smallest l' >= l with grad_bytes[l'] > 0 (L if none)
     const int32_t *pe;               // [L+1] number of expert layers before layer l
+    const int64_t *jsum;             // [n_entries][DISTSIM_MAX_PP] total jitter of the m forward and
+                                     // m backward items of a stage (nullptr without jitter)
     int32_t *status;                 // device status word: 0 ok, else first error code
 };
 
@@ -105,7 +110,7 @@ void launch_build_bucket_tables(cudaStream_t s, const TableConst &tc, const RawT
                                 int64_t *launches);
 // Per entry: the bucket-lane table (if dt != nullptr) and the time bound of the entry.
 void launch_build_entry_tables(cudaStream_t s, const DeviceView &v, Entry *entries, int64_t *dt,
-                               int64_t *launches);
+                               int64_t *jsum, int64_t *launches);
 void launch_build_layer_tables(cudaStream_t s, const TableConst &tc, const RawTable &raw,
                                int32_t *next_grad, int32_t *pe, int64_t *launches);
 

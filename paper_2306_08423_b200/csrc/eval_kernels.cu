@@ -70,7 +70,7 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     int n_slots = 2 * (en.m + pp - 1);
     n_slots = __reduce_max_sync(0xffffffffu, n_slots);
 
-    const StageResult<S> R = lockstep_candidate<S, false>(v, row, en, pf, pb, cc.sched, cc.part_rank,
+    const StageResult<S> R = lockstep_candidate<S, false>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank,
                                                           seg_lane, wl, n_slots, nullptr);
     if (!valid) return;
     const int64_t out = row.offset + local - first;
@@ -194,7 +194,7 @@ void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_row
         const int64_t lo = first > row.offset ? first - row.offset : 0;
         const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
         if (hi <= lo) continue;
-        if (row.pp > 16) { add_lockstep(r, lo, hi); continue; }
+        if (row.pp > 16 || v.tc.n_jitter > 0) { add_lockstep(r, lo, hi); continue; }   // jitter: lock-step only (for now)
         // Short pipelines: cut the range into runs of entries with the same arithmetic width; a
         // run with enough partitions goes to the one-partition-per-thread kernel, the rest to
         // the lock-step kernel.

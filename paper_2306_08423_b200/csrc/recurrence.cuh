@@ -86,20 +86,29 @@ __device__ __forceinline__ CandidateCoords split_local(const Row &row, int64_t l
     return cc;
 }
 
-// Does stage d run a forward / backward item in slot s?
-__device__ __forceinline__ void slot_activity(int sched, int pp, int m, int d, int s, bool &do_f, bool &do_b)
+// Does stage d run a forward / backward item in slot s, and of which micro-batch j?
+__device__ __forceinline__ void slot_activity(int sched, int pp, int m, int d, int s, bool &do_f, bool &do_b, int &j)
 {
     const int x = s - d;
     if (sched == 0) {
         do_f = x >= 0 && x < m;
         const int y = s - (m + 2 * pp - 2 - d);
         do_b = y >= 0 && y < m;
+        j = do_f ? x : y;
     } else {
         const int w = min(pp - d, m);
-        do_f = (x >= 0 && x < w) || (x >= 2 * w && !(x & 1) && (x >> 1) < m);
+        const bool warm = x >= 0 && x < w;
+        do_f = warm || (x >= 2 * w && !(x & 1) && (x >> 1) < m);
         const int y = s - (2 * pp - 1 - d);
         do_b = y >= 0 && !(y & 1) && (y >> 1) < m;
+        j = do_f ? (warm ? x : x >> 1) : y >> 1;
     }
+}
+
+// Extra time of the item of micro-batch j on stage d (0 without a jitter table).
+__device__ __forceinline__ int64_t jitter_of(const DeviceView &v, const int64_t *table, int j, int d)
+{
+    return v.tc.n_jitter ? __ldg(&table[(j & (v.tc.n_jitter - 1)) * v.tc.jitter_stages + d]) : 0;
 }
 
 // Gradient all-reduce buckets of one stage [a, e) on the communication lane (DP modeling).
@@ -149,7 +158,7 @@ struct StageResult {
     int a[S], e[S];              // layer range [a, e) of each owned stage
     int64_t fop[S], bop[S];      // cost of a forward / backward item incl. trailing transfer
     int64_t main_end[S];         // end of the stage's last item
-    int64_t last_b_start[S];     // start of the stage's last backward item
+    int64_t last_b_start[S];     // start of the first layer event of the stage's last backward item
     int64_t dp_end[S];           // end of the gradient-bucket lane
     int64_t busy[S];             // activity time of a device of the stage
     int64_t batch;               // max over all stages (same on every lane of the segment)
@@ -163,13 +172,14 @@ __device__ __forceinline__ int64_t p2p_cost(const Row &row, const Entry &en, int
 
 // Lock-step evaluation of one candidate by `wl` consecutive lanes (wl * S == pp), every lane of
 // the warp calling this together (lanes of other segments work on their own candidates).
-//   seg_lane   lane index inside the segment;  n_slots_warp: loop bound, uniform over the warp
+//   entry_index  global index of `en`;  seg_lane: lane index inside the segment;
+//   n_slots_warp loop bound, uniform over the warp
 //   pf, pb     the entry's forward / backward prefix rows (shared or global memory)
 //   rec        if kRecord and non-null: item start times go to rec[d * 2m + position in stage order]
 template <int S, bool kRecord>
 __device__ __forceinline__ StageResult<S> lockstep_candidate(
-    const DeviceView &v, const Row &row, const Entry &en, const int64_t *pf, const int64_t *pb,
-    int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec)
+    const DeviceView &v, const Row &row, const Entry &en, int entry_index, const int64_t *pf,
+    const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec)
 {
     StageResult<S> R;
     const int pp = row.pp, m = en.m;
@@ -199,19 +209,21 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         for (int k = 0; k < S; ++k) {
             const int d = d0 + k;
             bool do_f, do_b;
-            slot_activity(sched, pp, m, d, s, do_f, do_b);
+            int j;
+            slot_activity(sched, pp, m, d, s, do_f, do_b, j);
             if (do_f) {
                 const int64_t dep = (k == 0) ? (seg_lane == 0 ? 0 : up_f) : old_f[k > 0 ? k - 1 : 0];
                 const int64_t st = max64(dep, free_at[k]);
                 if (kRecord && rec) rec[(int64_t)d * 2 * m + n_done[k]] = st;
-                last_f[k] = free_at[k] = st + R.fop[k];
+                last_f[k] = free_at[k] = st + R.fop[k] + jitter_of(v, v.raw.jit_f, j, d);
                 ++n_done[k];
             } else if (do_b) {
                 const int64_t dep = (k == S - 1) ? (seg_lane == wl - 1 ? 0 : dn_b) : old_b[k < S - 1 ? k + 1 : 0];
                 const int64_t st = max64(dep, free_at[k]);
+                const int64_t jit = jitter_of(v, v.raw.jit_b, j, d);
                 if (kRecord && rec) rec[(int64_t)d * 2 * m + n_done[k]] = st;
-                R.last_b_start[k] = st;
-                last_b[k] = free_at[k] = st + R.bop[k];
+                R.last_b_start[k] = st + jit;
+                last_b[k] = free_at[k] = st + jit + R.bop[k];
                 ++n_done[k];
             }
         }
@@ -225,7 +237,8 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         R.main_end[k] = free_at[k];
         R.dp_end[k] = bucket_lane_end(v, row, pb, nbt, tpt, R.a[k], R.e[k], R.last_b_start[k], R.main_end[k]);
         const int64_t extra = R.dp_end[k] - R.main_end[k];
-        R.busy[k] = (int64_t)m * (R.fop[k] + R.bop[k]) + (extra > 0 ? extra : 0);
+        R.busy[k] = (int64_t)m * (R.fop[k] + R.bop[k]) + (extra > 0 ? extra : 0) +
+                    (v.jsum ? __ldg(&v.jsum[(int64_t)entry_index * DISTSIM_MAX_PP + d0 + k]) : 0);
         mx = max64(mx, max64(R.main_end[k], R.dp_end[k]));
     }
     for (int off = 1; off < wl; off <<= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, off, wl));

@@ -173,7 +173,7 @@ __global__ void build_dt_kernel(DeviceView v, int64_t *dt)
 
 // One thread per entry: an upper bound on every time any candidate of the entry can produce:
 // all items of the pipeline in sequence plus the largest possible bucket-lane excess.
-__global__ void entry_bound_kernel(DeviceView v, Entry *entries)
+__global__ void entry_bound_kernel(DeviceView v, Entry *entries, int64_t *jsum)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= v.sc.n_entries) return;
@@ -191,7 +191,26 @@ __global__ void entry_bound_kernel(DeviceView v, Entry *entries)
         // a stage's buckets cost at most all full buckets of the model plus one more bucket
         excess = nbL[0] * row.t_full + (v.tc.bucket > 0 ? row.t_full : tpL[0]);
     }
-    const __int128 b = (__int128)en.m * per_mb + excess;
+    // total jitter of a stage's items: whole cycles of the P slots plus the remainder
+    __int128 jitter_total = 0;
+    if (jsum) {
+        const int P = v.tc.n_jitter, S = v.tc.jitter_stages;
+        for (int d = 0; d < DISTSIM_MAX_PP; ++d) {
+            int64_t sum = 0;
+            if (d < row.pp) {
+                int64_t cycle = 0, rest = 0;
+                for (int p = 0; p < P; ++p) {
+                    const int64_t x = v.raw.jit_f[p * S + d] + v.raw.jit_b[p * S + d];
+                    cycle += x;
+                    if (p < en.m % P) rest += x;
+                }
+                sum = (int64_t)(en.m / P) * cycle + rest;
+            }
+            jsum[(int64_t)i * DISTSIM_MAX_PP + d] = sum;
+            jitter_total += sum;
+        }
+    }
+    const __int128 b = (__int128)en.m * per_mb + excess + jitter_total;
     en.bound = b >= (__int128)kSat ? kSat : (int64_t)b;
     entries[i] = en;
 }
@@ -199,7 +218,7 @@ __global__ void entry_bound_kernel(DeviceView v, Entry *entries)
 }  // namespace
 
 void launch_build_entry_tables(cudaStream_t s, const DeviceView &v, Entry *entries, int64_t *dt,
-                               int64_t *launches)
+                               int64_t *jsum, int64_t *launches)
 {
     if (v.sc.n_entries == 0) return;
     if (dt) {
@@ -207,7 +226,7 @@ void launch_build_entry_tables(cudaStream_t s, const DeviceView &v, Entry *entri
         build_dt_kernel<<<(n + 127) / 128, 128, 0, s>>>(v, dt);
         ++*launches;
     }
-    entry_bound_kernel<<<(v.sc.n_entries + 127) / 128, 128, 0, s>>>(v, entries);
+    entry_bound_kernel<<<(v.sc.n_entries + 127) / 128, 128, 0, s>>>(v, entries, jsum);
     ++*launches;
 }
 

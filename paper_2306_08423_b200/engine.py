@@ -48,7 +48,9 @@ class _Table(C.Structure):
                 ("act_bytes_per_elem", C.c_int32), ("class_mp", C.c_void_p),
                 ("class_b", C.c_void_p), ("fwd_ns", C.c_void_p), ("bwd_ns", C.c_void_p),
                 ("layer_is_expert", C.c_void_p), ("grad_bytes", C.c_void_p),
-                ("allreduce_profile_max", C.c_int32), ("reserved", C.c_int32)]
+                ("allreduce_profile_max", C.c_int32), ("n_jitter", C.c_int32),
+                ("jitter_stages", C.c_int32), ("reserved", C.c_int32),
+                ("jitter_fwd_ns", C.c_void_p), ("jitter_bwd_ns", C.c_void_p)]
 
 
 class _Space(C.Structure):
@@ -108,7 +110,14 @@ def _table_struct(t):
     s = _Table(t.n_layers, arrs[0].shape[0], t.n_devices, t.gpus_per_node, t.global_batch, t.seq,
                t.hidden, t.alpha_intra_ns, t.beta_intra, t.alpha_inter_ns, t.beta_inter,
                t.dp_bucket_bytes, t.dp_overlap, t.act_bytes_per_elem, *[_np_ptr(a) for a in arrs],
-               int(getattr(t, "allreduce_profile_max", 0)), 0)
+               int(getattr(t, "allreduce_profile_max", 0)), 0, 0, 0, None, None)
+    jf = getattr(t, "jitter_fwd_ns", None)
+    if jf is not None and np.size(jf) > 0:
+        jf = np.ascontiguousarray(jf, np.int64)
+        jb = np.ascontiguousarray(t.jitter_bwd_ns, np.int64)
+        s.n_jitter, s.jitter_stages = jf.shape
+        s.jitter_fwd_ns, s.jitter_bwd_ns = _np_ptr(jf), _np_ptr(jb)
+        arrs += [jf, jb]
     return s, arrs
 
 

@@ -313,6 +313,53 @@ def test_paper_grid_with_extrapolated_allreduce(E, ctx):
     check_emission(E, ctx, w2, list(range(0, n2, max(1, n2 // 12))))
 
 
+@pytest.mark.parametrize("seed", range(4))
+def test_per_microbatch_jitter_full_parity(E, ctx, seed):
+    kw = dict(dp_overlap=seed % 2, dp_bucket_bytes=3000)
+    if seed >= 2:
+        kw.update(n_devices=16, gpus_per_node=2, n_layers=9, global_batch=24, mp_max=4, pp_max=8,
+                  m_list=(1, 2, 3, 5, 6, 12), partition_mode=W.PARTITION_ALL)
+    w = W.add_jitter(W.random_small(200 + seed, **kw), 4 if seed % 2 else 1, 2500, seed)
+    n = load(E, ctx, w)
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    gb = batch.cpu().numpy()
+    assert (gb == ob).all(), np.argwhere(gb != ob)[:5]
+    assert (sb.cpu().numpy() == obusy).all()
+    rng = np.random.default_rng(seed)
+    check_emission(E, ctx, w, rng.choice(n, size=min(n, 20), replace=False).tolist())
+
+
+def test_jitter_on_benchmark_shapes(E, ctx):
+    # 256-device MoE workload (int64 times, every composition) and the long pipelines of the
+    # 1024-device workload, each with an 8-slot jitter table
+    for cfg, amp, n_sample in ((3, 200_000, 1500), (2, 5_000_000, 4176)):
+        w = W.add_jitter(W.CONFIGS[cfg](), 8, amp)
+        n = load(E, ctx, w)
+        batch, sb = eval_all(E, ctx, n)
+        idx = np.unique(np.linspace(0, n - 1, n_sample).astype(np.int64))
+        ob, obusy = oracle.eval_indices_parallel(w.table, w.space, idx, THREADS, pp_stride=w.space.pp_max)
+        sel = torch.from_numpy(idx).cuda()
+        assert (batch[sel].cpu().numpy() == ob).all()
+        assert (sb[sel].cpu().numpy() == obusy).all()
+        ki = dev(4)
+        E.distsim_topk(ctx, batch, 0, n, 4, ki)
+        check_emission(E, ctx, w, ki.cpu().numpy().tolist()[:2] + [int(idx[len(idx) // 3])])
+    # tables the engine refuses
+    import copy
+    t = copy.deepcopy(W.config0().table)
+    t.jitter_fwd_ns = np.zeros((3, 4), np.int64); t.jitter_bwd_ns = np.zeros((3, 4), np.int64)
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_load_event_table(ctx, t)
+    assert ei.value.code == E.E_UNSUPPORTED                   # slots must be a power of two
+    t.jitter_fwd_ns = np.zeros((2, 2), np.int64); t.jitter_bwd_ns = np.zeros((2, 2), np.int64)
+    E.distsim_load_event_table(ctx, t)
+    with pytest.raises(E.DistsimError) as ei:
+        E.distsim_set_space(ctx, W.config0().space)           # pp = 4 needs 4 columns
+    assert ei.value.code == E.E_ARG
+
+
 def test_integer_probes_run(E, ctx):
     for mode in range(4):
         assert E.distsim_int_issue_probe(ctx, 148, 64, mode) > 0
