@@ -127,9 +127,15 @@ void flush_thread(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first
 {
     if (p.batch.n == 0) return;
     const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
-    if (smem > 24 * 1024)
-        cudaFuncSetAttribute(eval_thread_kernel<PP, T, kBusy>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    eval_thread_kernel<PP, T, kBusy><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out);
+    if (v.tc.n_jitter > 0) {
+        if (smem > 16 * 1024)
+            cudaFuncSetAttribute(eval_thread_kernel<PP, T, kBusy, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_thread_kernel<PP, T, kBusy, true><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out);
+    } else {
+        if (smem > 24 * 1024)
+            cudaFuncSetAttribute(eval_thread_kernel<PP, T, kBusy, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_thread_kernel<PP, T, kBusy, false><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out);
+    }
     ++*launches;
     p = Pending{};
 }
@@ -194,7 +200,7 @@ void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_row
         const int64_t lo = first > row.offset ? first - row.offset : 0;
         const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
         if (hi <= lo) continue;
-        if (row.pp > 16 || v.tc.n_jitter > 0) { add_lockstep(r, lo, hi); continue; }   // jitter: lock-step only (for now)
+        if (row.pp > 16) { add_lockstep(r, lo, hi); continue; }
         // Short pipelines: cut the range into runs of entries with the same arithmetic width; a
         // run with enough partitions goes to the one-partition-per-thread kernel, the rest to
         // the lock-step kernel.

@@ -66,39 +66,56 @@ struct ThreadState {
     T fop[PP], bop[PP];
 };
 
+// Per-micro-batch jitter: extra time of the item of micro-batch j on stage d, from tables in
+// shared memory ([slot][stage], the slot count a power of two).  Every thread of a block asks
+// for the same (j, d), so the reads are broadcasts.  Without a jitter table (kJit false) the
+// accessors fold to zero at compile time.
+template <int PP, typename T, bool kJit>
+struct JitterTab {
+    const T *f, *b;
+    int mask;
+    __device__ __forceinline__ T fwd(int j, int d) const { return kJit ? f[(j & mask) * PP + d] : (T)0; }
+    __device__ __forceinline__ T bwd(int j, int d) const { return kJit ? b[(j & mask) * PP + d] : (T)0; }
+};
+
 // GPipe: returns main-lane end of every stage in free_at.
-template <int PP, typename T>
-__device__ __forceinline__ void run_gpipe(const ThreadState<PP, T> &c, int m, T (&free_at)[PP])
+template <int PP, typename T, bool kJit>
+__device__ __forceinline__ void run_gpipe(const ThreadState<PP, T> &c, int m, T (&free_at)[PP],
+                                          const JitterTab<PP, T, kJit> &jt)
 {
 #pragma unroll
     for (int d = 0; d < PP; ++d) free_at[d] = 0;
 DS_UNROLL(DS_UNROLL_MAIN)
     for (int j = 0; j < m; ++j) {
-        T t = free_at[0] + c.fop[0];
+        T t = free_at[0] + c.fop[0] + jt.fwd(j, 0);
         free_at[0] = t;
 #pragma unroll
-        for (int d = 1; d < PP; ++d) { t = cell(t, free_at[d], c.fop[d]); free_at[d] = t; }
+        for (int d = 1; d < PP; ++d) { t = cell(t, free_at[d], (T)(c.fop[d] + jt.fwd(j, d))); free_at[d] = t; }
     }
 DS_UNROLL(DS_UNROLL_MAIN)
     for (int j = 0; j < m; ++j) {
-        T t = free_at[PP - 1] + c.bop[PP - 1];
+        T t = free_at[PP - 1] + c.bop[PP - 1] + jt.bwd(j, PP - 1);
         free_at[PP - 1] = t;
 #pragma unroll
-        for (int d = PP - 2; d >= 0; --d) { t = cell(t, free_at[d], c.bop[d]); free_at[d] = t; }
+        for (int d = PP - 2; d >= 0; --d) { t = cell(t, free_at[d], (T)(c.bop[d] + jt.bwd(j, d))); free_at[d] = t; }
     }
 }
 
-// One 1F1B backward wave in which the stages d >= D0 also run a forward item (D0 may be PP).
-template <int PP, int D0, typename T>
-__device__ __forceinline__ void wave_1f1b(const ThreadState<PP, T> &c, T (&free_at)[PP], T (&last_f)[PP])
+// 1F1B backward wave i in which the stages d >= D0 also run a forward item (D0 may be PP): the
+// backward item is B(d, i), the forward item F(d, PP - d + i).
+template <int PP, int D0, typename T, bool kJit>
+__device__ __forceinline__ void wave_1f1b(const ThreadState<PP, T> &c, T (&free_at)[PP], T (&last_f)[PP],
+                                          const JitterTab<PP, T, kJit> &jt, int i)
 {
     T t = 0;
 #pragma unroll
     for (int d = PP - 1; d >= 0; --d) {
-        t = d == PP - 1 ? (T)(free_at[d] + c.bop[d]) : cell(t, free_at[d], c.bop[d]);
+        const T cb = c.bop[d] + jt.bwd(i, d);
+        t = d == PP - 1 ? (T)(free_at[d] + cb) : cell(t, free_at[d], cb);
         free_at[d] = t;
         if (d >= D0) {
-            const T f = d == 0 ? (T)(free_at[0] + c.fop[0]) : cell(last_f[d > 0 ? d - 1 : 0], free_at[d], c.fop[d]);
+            const T cf = c.fop[d] + jt.fwd(PP - d + i, d);
+            const T f = d == 0 ? (T)(free_at[0] + cf) : cell(last_f[d > 0 ? d - 1 : 0], free_at[d], cf);
             free_at[d] = f;
             last_f[d] = f;
         }
@@ -108,68 +125,79 @@ __device__ __forceinline__ void wave_1f1b(const ThreadState<PP, T> &c, T (&free_
 // A steady-state 1F1B wave: every stage runs its backward item and then a forward item.  After
 // a forward item the device's free time IS that item's end, so inside the steady state the
 // free times are not kept separately: last_f doubles as the free time.
-template <int PP, typename T>
-__device__ __forceinline__ void wave_1f1b_steady(const ThreadState<PP, T> &c, T (&last_f)[PP])
+template <int PP, typename T, bool kJit>
+__device__ __forceinline__ void wave_1f1b_steady(const ThreadState<PP, T> &c, T (&last_f)[PP],
+                                                 const JitterTab<PP, T, kJit> &jt, int i)
 {
     T t = 0;
 #pragma unroll
     for (int d = PP - 1; d >= 0; --d) {
-        t = d == PP - 1 ? (T)(last_f[d] + c.bop[d]) : cell(t, last_f[d], c.bop[d]);
-        last_f[d] = d == 0 ? (T)(t + c.fop[0]) : cell(last_f[d > 0 ? d - 1 : 0], t, c.fop[d]);
+        const T cb = c.bop[d] + jt.bwd(i, d);
+        const T cf = c.fop[d] + jt.fwd(PP - d + i, d);
+        t = d == PP - 1 ? (T)(last_f[d] + cb) : cell(t, last_f[d], cb);
+        last_f[d] = d == 0 ? (T)(t + cf) : cell(last_f[d > 0 ? d - 1 : 0], t, cf);
     }
 }
 
 // Runs the last waves, in which fewer and fewer stages still have a forward item: with K waves
-// to go, the stages with pp - d < K do (statically unrolled over K = PP .. 1).
-template <int PP, int K, typename T>
+// to go (wave i = m - K), the stages with pp - d < K do (statically unrolled over K = PP .. 1).
+template <int PP, int K, typename T, bool kJit>
 struct TailWaves {
-    static __device__ __forceinline__ void run(const ThreadState<PP, T> &c, int m, T (&free_at)[PP], T (&last_f)[PP])
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &c, int m, T (&free_at)[PP], T (&last_f)[PP],
+                                               const JitterTab<PP, T, kJit> &jt)
     {
-        if (K <= m) wave_1f1b<PP, PP - K + 1, T>(c, free_at, last_f);
-        TailWaves<PP, K - 1, T>::run(c, m, free_at, last_f);
+        if (K <= m) wave_1f1b<PP, PP - K + 1, T, kJit>(c, free_at, last_f, jt, m - K);
+        TailWaves<PP, K - 1, T, kJit>::run(c, m, free_at, last_f, jt);
     }
 };
-template <int PP, typename T>
-struct TailWaves<PP, 0, T> {
-    static __device__ __forceinline__ void run(const ThreadState<PP, T> &, int, T (&)[PP], T (&)[PP]) {}
+template <int PP, typename T, bool kJit>
+struct TailWaves<PP, 0, T, kJit> {
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &, int, T (&)[PP], T (&)[PP],
+                                               const JitterTab<PP, T, kJit> &) {}
 };
 
 // Warm-up forward wave J over stages 0 .. PP-1-J.
-template <int PP, int J, typename T>
+template <int PP, int J, typename T, bool kJit>
 struct WarmWaves {
-    static __device__ __forceinline__ void run(const ThreadState<PP, T> &c, int m, T (&free_at)[PP], T (&last_f)[PP])
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &c, int m, T (&free_at)[PP], T (&last_f)[PP],
+                                               const JitterTab<PP, T, kJit> &jt)
     {
         if (J < m) {
-            T t = free_at[0] + c.fop[0];
+            T t = free_at[0] + c.fop[0] + jt.fwd(J, 0);
             free_at[0] = t; last_f[0] = t;
 #pragma unroll
-            for (int d = 1; d < PP - J; ++d) { t = cell(t, free_at[d], c.fop[d]); free_at[d] = t; last_f[d] = t; }
+            for (int d = 1; d < PP - J; ++d) {
+                t = cell(t, free_at[d], (T)(c.fop[d] + jt.fwd(J, d)));
+                free_at[d] = t; last_f[d] = t;
+            }
         }
-        WarmWaves<PP, J + 1, T>::run(c, m, free_at, last_f);
+        WarmWaves<PP, J + 1, T, kJit>::run(c, m, free_at, last_f, jt);
     }
 };
-template <int PP, typename T>
-struct WarmWaves<PP, PP, T> {
-    static __device__ __forceinline__ void run(const ThreadState<PP, T> &, int, T (&)[PP], T (&)[PP]) {}
+template <int PP, typename T, bool kJit>
+struct WarmWaves<PP, PP, T, kJit> {
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &, int, T (&)[PP], T (&)[PP],
+                                               const JitterTab<PP, T, kJit> &) {}
 };
 
-template <int PP, typename T>
-__device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (&free_at)[PP])
+template <int PP, typename T, bool kJit>
+__device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (&free_at)[PP],
+                                         const JitterTab<PP, T, kJit> &jt)
 {
     T last_f[PP];
 #pragma unroll
     for (int d = 0; d < PP; ++d) { free_at[d] = 0; last_f[d] = 0; }
-    WarmWaves<PP, 0, T>::run(c, m, free_at, last_f);
+    WarmWaves<PP, 0, T, kJit>::run(c, m, free_at, last_f, jt);
     // waves i = 0 .. m-PP-1: every stage still has a forward item to pair with its backward;
     // entering them every stage's latest item is a forward one (free_at == last_f)
     if (m > PP) {
 DS_UNROLL(DS_UNROLL_MAIN)
-        for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T>(c, last_f);
+        for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T, kJit>(c, last_f, jt, i);
 #pragma unroll
         for (int d = 0; d < PP; ++d) free_at[d] = last_f[d];
     }
     // the last min(PP, m) waves
-    TailWaves<PP, PP, T>::run(c, m, free_at, last_f);
+    TailWaves<PP, PP, T, kJit>::run(c, m, free_at, last_f, jt);
 }
 
 // Shared-memory plan of a block (offsets in int64 words from the dynamic shared base): the
@@ -203,7 +231,9 @@ __host__ __device__ inline ThreadKernelSmem thread_kernel_smem(int n_entries, in
 // Entry scalars the hot path needs, kept in shared memory for the whole row.
 struct EntryLite { int64_t p2p_intra, p2p_inter; int32_t m, pad; };
 
-template <int PP, typename T, bool kBusy>
+constexpr int kMaxJitterSlots = 64;
+
+template <int PP, typename T, bool kBusy, bool kJit>
 __global__ void __launch_bounds__(kThreadBlock, thread_kernel_min_blocks<PP, T>())
 eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
                    int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out)
@@ -221,6 +251,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
     __shared__ T xs[PP][kThreadBlock];                // per thread, per stage: bucket-lane excess X
     __shared__ uint16_t cs[PP + 1][kThreadBlock];     // per thread: stage bounds c_0 .. c_PP
     __shared__ EntryLite ents[kMaxRowEntries];
+    __shared__ T jit_f_s[kJit ? kMaxJitterSlots * PP : 1], jit_b_s[kJit ? kMaxJitterSlots * PP : 1];
     const Row &row = v.rows[row_index];
     const int lp = v.tc.lp;
     const int L1 = v.tc.n_layers + 1;
@@ -239,6 +270,13 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
         ents[threadIdx.x].p2p_inter = en.p2p_inter;
         ents[threadIdx.x].m = en.m;
     }
+    if (kJit)
+        for (int k = threadIdx.x; k < v.tc.n_jitter * PP; k += blockDim.x) {
+            const int p = k / PP, d = k - p * PP;
+            jit_f_s[k] = (T)v.raw.jit_f[p * v.tc.jitter_stages + d];
+            jit_b_s[k] = (T)v.raw.jit_b[p * v.tc.jitter_stages + d];
+        }
+    const JitterTab<PP, T, kJit> jt{jit_f_s, jit_b_s, v.tc.n_jitter - 1};
     bool staged = false;
     if (plan.n_entries_staged > 0 || plan.tables_staged) {
         const uint32_t pbytes = (uint32_t)(plan.n_entries_staged * lp * sizeof(int64_t));
@@ -343,8 +381,8 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
             const int64_t local = local0 + sc;
             if (local < lo || local >= hi) continue;
             T free_at[PP];
-            if (sched0 + sc == 0) run_gpipe<PP, T>(st, m, free_at);
-            else run_1f1b<PP, T>(st, m, free_at);
+            if (sched0 + sc == 0) run_gpipe<PP, T, kJit>(st, m, free_at, jt);
+            else run_1f1b<PP, T, kJit>(st, m, free_at, jt);
             T batch = 0;
 #pragma unroll
             for (int d = 0; d < PP; ++d) batch = vmax(batch, (T)(free_at[d] + xs[d][threadIdx.x]));
@@ -353,7 +391,8 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
                 int64_t *bo = busy_out + (row.offset + local - first) * v.sc.pp_max;
 #pragma unroll
                 for (int d = 0; d < PP; ++d)
-                    bo[d] = (int64_t)m * ((int64_t)st.fop[d] + (int64_t)st.bop[d]) + (int64_t)xs[d][threadIdx.x];
+                    bo[d] = (int64_t)m * ((int64_t)st.fop[d] + (int64_t)st.bop[d]) + (int64_t)xs[d][threadIdx.x] +
+                            (kJit ? __ldg(&v.jsum[(int64_t)(row.entry0 + e) * DISTSIM_MAX_PP + d]) : 0);
                 for (int d = PP; d < v.sc.pp_max; ++d) bo[d] = 0;
             }
         }

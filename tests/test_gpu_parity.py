@@ -334,7 +334,8 @@ def test_per_microbatch_jitter_full_parity(E, ctx, seed):
 def test_jitter_on_benchmark_shapes(E, ctx):
     # 256-device MoE workload (int64 times, every composition) and the long pipelines of the
     # 1024-device workload, each with an 8-slot jitter table
-    for cfg, amp, n_sample in ((3, 200_000, 1500), (2, 5_000_000, 4176)):
+    # and the 64-device workload (uint32 arithmetic in the one-partition-per-thread kernel)
+    for cfg, amp, n_sample in ((3, 200_000, 1500), (2, 5_000_000, 4176), (1, 50_000, 3000)):
         w = W.add_jitter(W.CONFIGS[cfg](), 8, amp)
         n = load(E, ctx, w)
         batch, sb = eval_all(E, ctx, n)
