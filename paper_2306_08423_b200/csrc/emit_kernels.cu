@@ -327,7 +327,8 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         else if (field >= 3) t += start_s[it] + ((jr && w != 3) ? jit_s[it] : 0);
         return t;
     };
-    for (int x0 = 0; x0 < total; x0 += 2 * kItemThreads) {
+    // (x0 == total can occur: an odd-based replica's last word is then written by the thread at x == total)
+    for (int x0 = 0; x0 <= total; x0 += 2 * kItemThreads) {
         const int x = x0 + 2 * threadIdx.x;          // the even word of this thread
         if (x - 1 >= total) break;
         int lo = 0, hi = n_items - 1;                // item holding word min(x, total-1)

@@ -369,6 +369,59 @@ def test_integer_probes_run(E, ctx):
         E.distsim_int_issue_probe(ctx, 148, 64, 9)
 
 
+def _emit_chunk_and_check(E, ctx, w, top, sample_positions):
+    """Emits the selections `top` (device tensor) in one call, checks structure on the device
+    and the sampled selections record by record against the oracle."""
+    N = w.table.n_devices
+    n = top.numel()
+    offsets, busy, util = dev(n * N + 1), dev(n * N), dev(n * N, torch.float64)
+    total = E.distsim_emit_timelines(ctx, top, n, None, 0)
+    records = dev(total * 5)
+    records.fill_(-7)                                  # no field of any record is ever -7
+    assert E.distsim_emit_timelines(ctx, top, n, records, total, offsets, busy, util) == total
+    assert int((records == -7).sum()) == 0             # every word was written
+    rec = records.view(total, 5)
+    # properties that hold at any size
+    assert int(offsets[0]) == 0 and int(offsets[-1]) == total
+    assert bool((offsets[1:] >= offsets[:-1]).all())
+    assert bool(((rec[:, 0] >= 0) & (rec[:, 0] <= 10)).all())
+    assert bool((rec[:, 4] >= rec[:, 3]).all()) and bool((rec[:, 3] >= 0).all())
+    assert bool((util > 0).all()) and bool((util <= 1.0).all())
+    idx = top.cpu().numpy()
+    for pos in sample_positions:
+        c = oracle.enumerate_at(w.table, w.space, np.array([idx[pos]]))[0]
+        r = oracle.simulate(w.table, c, replicate=True)
+        lo, hi = int(offsets[pos * N]), int(offsets[(pos + 1) * N])
+        assert hi - lo == r.offsets[-1]
+        assert (offsets[pos * N: (pos + 1) * N + 1].cpu().numpy() - lo == r.offsets).all()
+        assert (rec[lo:hi].cpu().numpy() == r.records).all(), (pos, c)
+        assert (busy[pos * N: (pos + 1) * N].cpu().numpy() == r.busy_ns).all()
+        np.testing.assert_allclose(util[pos * N: (pos + 1) * N].cpu().numpy(), r.util, rtol=1e-12, atol=0)
+    return total
+
+
+def test_emission_in_the_benchmark_launch_configurations(E, ctx):
+    # (a) the search step of the benchmark: the 1024 fastest of the 64-device workload, one call
+    w = W.config1()
+    n = load(E, ctx, w)
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    top = dev(1024)
+    E.distsim_topk(ctx, batch, 0, n, 1024, top)
+    _emit_chunk_and_check(E, ctx, w, top, [0, 333, 1023])
+    del batch
+    # (b) the emission workload: the 1024 fastest of the 1024-device workload, 128 per call
+    w = W.config4()
+    n = load(E, ctx, w)
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    top = dev(w.top_k)
+    E.distsim_topk(ctx, batch, 0, n, w.top_k, top)
+    grand = 0
+    for k, i in enumerate(range(0, w.top_k, 128)):
+        grand += _emit_chunk_and_check(E, ctx, w, top[i:i + 128], [(17 * k) % 128] if k % 3 == 0 else [])
+        torch.cuda.empty_cache()
+    assert grand > 10**9                              # about 2e9 records, 8e10 bytes in all
+
+
 def test_two_pass_argmin_for_wide_times(E, ctx):
     # times near 2^55 with a large count cannot be packed with the index into 64 bits
     w = W.random_small(3, lo=2**44, hi=2**45, partition_mode=W.PARTITION_ALL, n_layers=12, pp_max=4,
