@@ -422,6 +422,23 @@ def test_emission_in_the_benchmark_launch_configurations(E, ctx):
     assert grand > 10**9                              # about 2e9 records, 8e10 bytes in all
 
 
+@pytest.mark.parametrize("cfg", [1, 3])
+def test_small_windows_agree_with_the_full_evaluation(E, ctx, cfg):
+    # a window of under 2048 partitions is evaluated by the lock-step kernel, the whole space by
+    # the one-partition-per-thread kernel: two implementations, one answer
+    w = W.CONFIGS[cfg]()
+    n = load(E, ctx, w)
+    full, fb = eval_all(E, ctx, n)
+    rng = np.random.default_rng(cfg)
+    out, ob = dev(3001), dev(3001 * ctx.pp_max)
+    for _ in range(48):
+        count = int(rng.integers(1, 3001))
+        first = int(rng.integers(0, n - count))
+        E.distsim_eval_strategies(ctx, first, count, out, ob)
+        assert torch.equal(out[:count], full[first:first + count])
+        assert torch.equal(ob[:count * ctx.pp_max].view(count, -1), fb[first:first + count])
+
+
 def test_two_pass_argmin_for_wide_times(E, ctx):
     # times near 2^55 with a large count cannot be packed with the index into 64 bits
     w = W.random_small(3, lo=2**44, hi=2**45, partition_mode=W.PARTITION_ALL, n_layers=12, pp_max=4,
