@@ -50,8 +50,11 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
     const int64_t *pf = v.etf + (int64_t)cc.entry * v.tc.lp;
     const int64_t *pb = v.etb + (int64_t)cc.entry * v.tc.lp;
     const int n_slots = 2 * (en.m + row.pp - 1);
-    const StageResult<S> R = lockstep_candidate<S, true>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank,
-                                                         seg_lane, wl, n_slots, owner ? rec : nullptr);
+    const StageResult<S> R = v.tc.n_jitter > 0
+        ? lockstep_candidate<S, true, true>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank, seg_lane, wl,
+                                            n_slots, owner ? rec : nullptr)
+        : lockstep_candidate<S, true, false>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank, seg_lane, wl,
+                                             n_slots, owner ? rec : nullptr);
     if (owner) {
         const int L1 = v.tc.n_layers + 1;
 #pragma unroll

@@ -22,7 +22,7 @@ namespace {
 
 constexpr int kEvalThreads = 256;
 
-template <int S>
+template <int S, bool kJit>
 __global__ void __launch_bounds__(kEvalThreads)
 eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
                      int64_t *__restrict__ busy_out, int smem_words)
@@ -70,7 +70,7 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     int n_slots = 2 * (en.m + pp - 1);
     n_slots = __reduce_max_sync(0xffffffffu, n_slots);
 
-    const StageResult<S> R = lockstep_candidate<S, false>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank,
+    const StageResult<S> R = lockstep_candidate<S, false, kJit>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank,
                                                           seg_lane, wl, n_slots, nullptr);
     if (!valid) return;
     const int64_t out = row.offset + local - first;
@@ -114,9 +114,15 @@ void flush_lockstep(cudaStream_t s, const DeviceView &v, Pending &p, int64_t fir
 {
     if (p.batch.n == 0) return;
     const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
-    if (smem > 48 * 1024)
-        cudaFuncSetAttribute(eval_lockstep_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    eval_lockstep_kernel<S><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
+    if (v.tc.n_jitter > 0) {
+        if (smem > 48 * 1024)
+            cudaFuncSetAttribute(eval_lockstep_kernel<S, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_lockstep_kernel<S, true><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
+    } else {
+        if (smem > 48 * 1024)
+            cudaFuncSetAttribute(eval_lockstep_kernel<S, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        eval_lockstep_kernel<S, false><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
+    }
     ++*launches;
     p = Pending{};
 }

@@ -176,7 +176,8 @@ __device__ __forceinline__ int64_t p2p_cost(const Row &row, const Entry &en, int
 //   n_slots_warp loop bound, uniform over the warp
 //   pf, pb     the entry's forward / backward prefix rows (shared or global memory)
 //   rec        if kRecord and non-null: item start times go to rec[d * 2m + position in stage order]
-template <int S, bool kRecord>
+//   kJit       the table has per-micro-batch jitter (otherwise none of its code is generated)
+template <int S, bool kRecord, bool kJit>
 __device__ __forceinline__ StageResult<S> lockstep_candidate(
     const DeviceView &v, const Row &row, const Entry &en, int entry_index, const int64_t *pf,
     const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec)
@@ -215,12 +216,12 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
                 const int64_t dep = (k == 0) ? (seg_lane == 0 ? 0 : up_f) : old_f[k > 0 ? k - 1 : 0];
                 const int64_t st = max64(dep, free_at[k]);
                 if (kRecord && rec) rec[(int64_t)d * 2 * m + n_done[k]] = st;
-                last_f[k] = free_at[k] = st + R.fop[k] + jitter_of(v, v.raw.jit_f, j, d);
+                last_f[k] = free_at[k] = st + R.fop[k] + (kJit ? jitter_of(v, v.raw.jit_f, j, d) : 0);
                 ++n_done[k];
             } else if (do_b) {
                 const int64_t dep = (k == S - 1) ? (seg_lane == wl - 1 ? 0 : dn_b) : old_b[k < S - 1 ? k + 1 : 0];
                 const int64_t st = max64(dep, free_at[k]);
-                const int64_t jit = jitter_of(v, v.raw.jit_b, j, d);
+                const int64_t jit = kJit ? jitter_of(v, v.raw.jit_b, j, d) : 0;
                 if (kRecord && rec) rec[(int64_t)d * 2 * m + n_done[k]] = st;
                 R.last_b_start[k] = st + jit;
                 last_b[k] = free_at[k] = st + jit + R.bop[k];
@@ -238,7 +239,7 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         R.dp_end[k] = bucket_lane_end(v, row, pb, nbt, tpt, R.a[k], R.e[k], R.last_b_start[k], R.main_end[k]);
         const int64_t extra = R.dp_end[k] - R.main_end[k];
         R.busy[k] = (int64_t)m * (R.fop[k] + R.bop[k]) + (extra > 0 ? extra : 0) +
-                    (v.jsum ? __ldg(&v.jsum[(int64_t)entry_index * DISTSIM_MAX_PP + d0 + k]) : 0);
+                    (kJit ? __ldg(&v.jsum[(int64_t)entry_index * DISTSIM_MAX_PP + d0 + k]) : 0);
         mx = max64(mx, max64(R.main_end[k], R.dp_end[k]));
     }
     for (int off = 1; off < wl; off <<= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, off, wl));
