@@ -40,6 +40,11 @@ TOP_K = 1024
 # below 2^32) one max and one add.
 INT_OPS_PER_CELL_64, INT_OPS_PER_CELL_32 = 6, 2
 RECORD_BYTES = 40
+# DRAM read + write bytes per step of the timed workload, from the one-pass ncu counters summarised in
+# profiles/bench_config1_dram_bytes.md.  They describe the kernels as captured: set them to None when
+# an evaluation or emission kernel changes, until the counters are taken again.
+EVAL_TRAFFIC_BYTES = 205_375_000
+EMIT_TRAFFIC_BYTES = 1_698_347_000
 
 
 def measured_peaks():
@@ -327,7 +332,10 @@ def run_ours(args):
     roofline = {"bound": "alu", "kernel": "eval_thread_kernel (+ lock-step kernel on small rows)",
                 "achieved": achieved_gops, "peak": int_peak_gops,
                 "unit": "G 32-bit integer instr/s (2 per uint32 cell, 6 per int64 cell)",
-                "frac": achieved_gops / int_peak_gops, "traffic": None,
+                "frac": achieved_gops / int_peak_gops, "traffic": EVAL_TRAFFIC_BYTES,
+                "traffic_note": "DRAM read + write bytes of the four evaluation launches of one step (ncu, one pass); "
+                                "of it 141.4e6 by the dominant launch; algorithmic: 8 B per candidate = "
+                                f"{8 * n_total} B, part of which is still in the L2 when the launches end",
                 "peak_kind": "measured in this run: dependency-free add/xor stream",
                 "cells": cells, "cells_32bit": cells_32, "ms_per_launch_set": statistics.mean(eval_ms),
                 "cell_rate_peaks_Gcells_per_s": {"uint32": cell32_peak, "int64": cell64_peak},
@@ -337,7 +345,9 @@ def run_ours(args):
     emit_gbs = emit_bytes / (statistics.mean(emit_ms) * 1e-3) / 1e9
     roofline_emit = {"bound": "hbm", "kernel": "emit_items_kernel (+plan, scan, devices, buckets)",
                      "achieved": emit_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": emit_gbs / peaks["hbm_gbs"], "traffic": None, "peak_kind": peak_kind,
+                     "frac": emit_gbs / peaks["hbm_gbs"], "traffic": EMIT_TRAFFIC_BYTES, "peak_kind": peak_kind,
+                     "traffic_note": "DRAM read + write bytes of emit_items_kernel + emit_buckets_kernel of one step "
+                                     "(ncu, one pass); the bucket-lane records are still in the L2 when they end",
                      "bytes_per_step": emit_bytes, "ms": statistics.mean(emit_ms)}
 
     line = {
