@@ -457,7 +457,10 @@ def profile_case(name):
     """Small, bounded invocations for profiler captures (no timing, no JSON line):
     eval1  - evaluation of a 2 M-candidate slice of the 64-device workload (a pp = 16 row)
     eval3  - evaluation of the whole 256-device MoE workload (650 k candidates)
-    emit4  - emission of 16 of the fastest candidates of the 1024-device workload (~1.3 GB)"""
+    emit4  - emission of 16 of the fastest candidates of the 1024-device workload (~1.9 GB)
+    emit1  - emission of the 1024 fastest candidates of the 64-device workload (~1.8 GB)
+    emit4x128 - as emit4 for 128 candidates, one call of the benchmark's size (~10 GB; for
+             one-pass launch lists only)"""
     import torch
     from paper_2306_08423_b200 import engine as E
     torch.cuda.set_device(0)
@@ -478,18 +481,19 @@ def profile_case(name):
         for _ in range(3):
             E.distsim_eval_strategies(ctx, first, count, batch)
         print(name, "best", E.distsim_argmin(ctx, batch, first, count))
-    elif name == "emit4":
-        w = W.config4()
+    elif name in ("emit4", "emit4x128", "emit1"):
+        k = {"emit4": 16, "emit4x128": 128, "emit1": TOP_K}[name]
+        w = W.config4() if name != "emit1" else W.config1()
         E.distsim_load_event_table(ctx, w.table)
         n = E.distsim_set_space(ctx, w.space)
         batch = torch.empty(n, dtype=torch.int64, device="cuda")
         E.distsim_eval_strategies(ctx, 0, n, batch)
-        top = torch.empty(16, dtype=torch.int64, device="cuda")
-        E.distsim_topk(ctx, batch, 0, n, 16, top)
-        total = E.distsim_emit_timelines(ctx, top, 16, None, 0)
+        top = torch.empty(k, dtype=torch.int64, device="cuda")
+        E.distsim_topk(ctx, batch, 0, n, k, top)
+        total = E.distsim_emit_timelines(ctx, top, k, None, 0)
         records = torch.empty(total * 5, dtype=torch.int64, device="cuda")
         for _ in range(2):
-            E.distsim_emit_timelines(ctx, top, 16, records, total)
+            E.distsim_emit_timelines(ctx, top, k, records, total)
         print(name, "records", total, "bytes", total * RECORD_BYTES)
     else:
         raise SystemExit(f"unknown profile case {name}")
@@ -505,7 +509,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-workloads", action="store_true", help="skip the per-workload summary")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
-    ap.add_argument("--profile-case", default=None, help="eval1 | eval3 | emit4: small run for ncu")
+    ap.add_argument("--profile-case", default=None, help="eval1 | eval3 | emit1 | emit4 | emit4x128: small run for ncu")
     args = ap.parse_args()
     if args.profile_case:
         profile_case(args.profile_case)

@@ -73,7 +73,8 @@ struct distsim_ctx {
 
     // scratch
     DevBuf d_status, d_sel, d_result, d_plans, d_op_start, d_totals, d_batch, d_topk;
-    int64_t *h_pinned = nullptr;          // 8 words of pinned host memory for small results
+    int64_t *h_pinned = nullptr;          // 16 words of pinned host memory for small results:
+                                          // [0..3] results, [4] status, [8..15] emission totals
 
     DeviceView view() const
     {
@@ -177,7 +178,7 @@ int distsim_create(distsim_ctx **out, int cuda_device)
         ctx->d_sel.reserve((8 + 2048 + 16 + 2 * 4096 + 2 * kCompactCap) * sizeof(int64_t)) != cudaSuccess ||
         ctx->d_result.reserve(64) != cudaSuccess || ctx->d_totals.reserve(64) != cudaSuccess ||
         cudaMemset(ctx->d_status.p, 0, 64) != cudaSuccess ||
-        cudaMallocHost(&ctx->h_pinned, 8 * sizeof(int64_t)) != cudaSuccess) {
+        cudaMallocHost(&ctx->h_pinned, 16 * sizeof(int64_t)) != cudaSuccess) {
         delete ctx;
         return DISTSIM_E_CUDA;
     }
@@ -529,13 +530,15 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     launch_emit_plan(s, v, d_indices, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
                      ctx->op_words_per_cand, d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), &ctx->launches);
     CU(cudaGetLastError(), "emission planning launch");
-    CU(cudaMemcpyAsync(ctx->h_pinned, ctx->d_totals.p, 3 * sizeof(int64_t), cudaMemcpyDeviceToHost, s), "totals readback");
+    static_assert(sizeof(EmitTotals) == 8 * sizeof(int64_t), "totals occupy the second half of the pinned words");
+    const EmitTotals *totals = reinterpret_cast<const EmitTotals *>(ctx->h_pinned + 8);
+    CU(cudaMemcpyAsync(ctx->h_pinned + 8, ctx->d_totals.p, sizeof(EmitTotals), cudaMemcpyDeviceToHost, s), "totals readback");
     if (int rc = read_status(ctx, s)) return rc;       // synchronises
-    *h_total_records = ctx->h_pinned[0];
+    *h_total_records = totals->records;
     if (!d_records) return DISTSIM_OK;
-    if (ctx->h_pinned[0] > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");
+    if (totals->records > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");
     launch_emit_records(s, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
-                        ctx->op_words_per_cand, ctx->h_pinned[1], ctx->h_pinned[2], d_records, &ctx->launches);
+                        ctx->op_words_per_cand, *totals, d_records, &ctx->launches);
     CU(cudaGetLastError(), "emission launch");
     CU(cudaStreamSynchronize(s), "emission sync");
     return DISTSIM_OK;

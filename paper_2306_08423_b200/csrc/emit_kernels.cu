@@ -8,24 +8,28 @@
 //   emit_items_kernel    the bandwidth-bound part.  A block owns (candidate, stage, run of
 //                        consecutive items, chunk of replicas).  It builds the stage's forward
 //                        and backward item templates (records relative to the item's start) in
-//                        shared memory once.  The run's records are contiguous in memory, so the
-//                        block walks the run as one flat stream of int64 words: word x belongs to
-//                        the item found by a search in the run's offset table, and its value is
-//                        template word + {0, 0, microbatch, start, start}.  Consecutive threads
-//                        write consecutive word pairs (16-byte stores, full-width warp stores
-//                        whatever the item size) to each of the stage's mp*dp replicas, whose
-//                        lists are identical.
+//                        shared memory once, then an image of the whole run: a warp per item, a
+//                        word is template word + {0, 0, microbatch, start, start}.  The stage's
+//                        mp*dp replicas hold identical lists, so the image is computed once and
+//                        written to each replica of the chunk by one bulk asynchronous copy
+//                        (cp.async.bulk shared -> global) issued by one lane per replica.
 //   emit_buckets_kernel  gradient-bucket records of every stage.
 #include "recurrence.cuh"
+#include "smem_stage.cuh"
 
 namespace distsim {
 
 namespace {
 
 constexpr int kItemThreads = 256;
-constexpr int kMaxTileItems = 128;  // most schedule items per block (a plan picks its own count)
-constexpr int kTileWords = 16384;   // target size of a block's run, in int64 words per replica
-constexpr int kTileReplicas = 8;    // replicas per block
+constexpr int kMaxTileItems = 192;  // most schedule items per block (a plan picks its own count)
+constexpr int kTileWords = 3872;    // capacity of a block's image of its run, in int64 words
+constexpr int kTileReplicas = 16;   // replicas per block
+constexpr int kBucketThreads = 128;
+constexpr int kBucketRun = 768;     // gradient buckets per shared-memory image (5 words each)
+constexpr int kBucketReplicas = 32; // replicas per block of the bucket kernel: one lane of the first warp each
+// the longest item: every layer with computation, all-reduce and all-to-all, a jitter event, a transfer
+static_assert((3 * DISTSIM_MAX_LAYERS + 2) * 5 <= kTileWords && kTileWords % 2 == 0, "an item must fit the image");
 
 __device__ __forceinline__ int find_row(const DeviceView &v, int64_t index)
 {
@@ -93,10 +97,14 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
         for (int d = 0; d < row.pp; ++d) { plan->stage_rec_prefix[d] = acc; acc += plan->stage_recs[d]; }
         plan->stage_rec_prefix[row.pp] = acc;
         plan->rec_total = acc * row.mp * row.dp;
-        int widest = 1;
-        for (int d = 0; d < row.pp; ++d) widest = max(widest, plan->rf[d] + plan->rb[d]);
-        const int per_tile = kTileWords / ((widest * 5 + 1) / 2);      // average item: (rf + rb) / 2 records
-        plan->tile_items = max(8, min(kMaxTileItems, per_tile));
+        int widest = 1, both = 2;
+        for (int d = 0; d < row.pp; ++d) {
+            widest = max(widest, max(plan->rf[d], plan->rb[d]));
+            both = max(both, plan->rf[d] + plan->rb[d]);
+        }
+        // a run of tile_items items of any mix must fit the image of kTileWords words
+        plan->tile_items = max(1, min(kMaxTileItems, kTileWords / (widest * 5)));
+        plan->tmpl_words = both * 5;
     }
 }
 
@@ -111,7 +119,7 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
     if (index < 0 || index >= v.sc.n_candidates) {
         if ((threadIdx.x & 31) == 0) {
             plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
-            plan->mp = 1; plan->dp = 1; plan->tile_items = 8;
+            plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0;
             atomicCAS(v.status, 0, DISTSIM_E_RANGE);
         }
         return;
@@ -124,13 +132,13 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
 }
 
 // Exclusive scan of rec_total over the selections (n is small: one block, serial per chunk).
-__global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /*[3]: records, max tiles, max bucket copies of a stage*/)
+__global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /* the words of EmitTotals */)
 {
     __shared__ int64_t chunk_sum[1024];
     const int t = threadIdx.x, nt = blockDim.x;
     const int per = (n + nt - 1) / nt;
     const int b = min(n, t * per), e = min(n, b + per);
-    int64_t s = 0, mt = 0, mb = 0;
+    int64_t s = 0, mt = 0, mb = 0, mw = 0, mk = 0;
     for (int i = b; i < e; ++i) s += plans[i].rec_total;
     chunk_sum[t] = s;
     __syncthreads();
@@ -148,11 +156,15 @@ __global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /*[3]: 
             const int64_t tiles = (int64_t)plans[i].pp * ((2 * plans[i].m + plans[i].tile_items - 1) / plans[i].tile_items) *
                                   ((reps + kTileReplicas - 1) / kTileReplicas);
             mt = max64(mt, tiles);
-            for (int d = 0; d < plans[i].pp; ++d) mb = max64(mb, plans[i].n_buckets[d] * reps);
+            mw = max64(mw, plans[i].tmpl_words);
+            mb = max64(mb, (int64_t)plans[i].pp * ((reps + kBucketReplicas - 1) / kBucketReplicas));
+            for (int d = 0; d < plans[i].pp; ++d) mk = max64(mk, plans[i].n_buckets[d]);
         }
     }
     if (mt > 0) atomicMax((unsigned long long *)&totals[1], (unsigned long long)mt);
     if (mb > 0) atomicMax((unsigned long long *)&totals[2], (unsigned long long)mb);
+    if (mw > 0) atomicMax((unsigned long long *)&totals[3], (unsigned long long)mw);
+    if (mk > 0) atomicMax((unsigned long long *)&totals[4], (unsigned long long)mk);
 }
 
 __global__ void __launch_bounds__(256)
@@ -201,12 +213,15 @@ __global__ void __launch_bounds__(kItemThreads)
 emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_t *__restrict__ op_start,
                   int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */)
 {
-    extern __shared__ __align__(16) int64_t tmpl[];     // [rf*5] forward, then [rb*5] backward
+    extern __shared__ __align__(16) int64_t dyn_s[];
+    int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
+    int64_t *img_b = dyn_s + kTileWords;                // the same word at img_b[x + 1]
+    int64_t *tmpl = dyn_s + 2 * kTileWords + 2;         // [rf*5] forward, then [rb*5] backward
     __shared__ int64_t rep_off_s[kTileReplicas];
     __shared__ int64_t start_s[kMaxTileItems];          // start time of each item of the run
+    __shared__ int64_t jit_s[kMaxTileItems];            // jitter at the start of each item
     __shared__ int32_t ioff[kMaxTileItems + 1];         // word offset of each item inside the run
     __shared__ int32_t meta_s[kMaxTileItems];           // micro-batch << 1 | is-backward
-    __shared__ int64_t jit_s[kMaxTileItems];            // jitter at the start of each item
     const int i = blockIdx.y;
     const EmitPlan &p = plans[i];
     if (!p.ok) return;
@@ -265,24 +280,21 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     const int n_items = min(2 * m, s0 + tile_items) - s0;
     bool bwd0; int j0, nf0, nb0;
     item_at(sched, pp, m, d, s0, bwd0, j0, nf0, nb0);
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTileItems + 1) {
-        const int k = threadIdx.x - 64;
-        if (k <= n_items) {
-            bool bwd; int j, nf, nb;
-            item_at(sched, pp, m, d, s0 + k, bwd, j, nf, nb);       // k == n_items: one past the run
-            ioff[k] = ((nf - nf0) * rf + (nb - nb0) * rb) * 5;
-            if (k < n_items) {
-                start_s[k] = op_start[(int64_t)i * op_words_per_cand + (int64_t)d * 2 * m + s0 + k];
-                meta_s[k] = (j << 1) | (bwd ? 1 : 0);
-                jit_s[k] = jitter_of(v, bwd ? v.raw.jit_b : v.raw.jit_f, j, d);
-            }
+    for (int k = threadIdx.x; k <= n_items; k += blockDim.x) {
+        bool bwd; int j, nf, nb;
+        item_at(sched, pp, m, d, s0 + k, bwd, j, nf, nb);           // k == n_items: one past the run
+        ioff[k] = ((nf - nf0) * rf + (nb - nb0) * rb) * 5;
+        if (k < n_items) {
+            start_s[k] = op_start[(int64_t)i * op_words_per_cand + (int64_t)d * 2 * m + s0 + k];
+            meta_s[k] = (j << 1) | (bwd ? 1 : 0);
+            jit_s[k] = jitter_of(v, bwd ? v.raw.jit_b : v.raw.jit_f, j, d);
         }
     }
     // word offset of every replica (r, q) of this tile relative to replica 0 of the stage
     const int rep0 = rc * kTileReplicas;
     const int n_rep = min(reps, rep0 + kTileReplicas) - rep0;
-    if (threadIdx.x >= 32 && threadIdx.x < 32 + kTileReplicas) {
-        const int k = threadIdx.x - 32;
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + kTileReplicas) {
+        const int k = threadIdx.x - 64;
         int64_t off = 0;
         if (k < n_rep) {
             const int rep = rep0 + k;
@@ -305,80 +317,77 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     }
     __syncthreads();
 
-    // ---- stream the run as flat words ---------------------------------------------------------
-    int64_t roff[kTileReplicas];                     // word offset of each replica of this tile
-#pragma unroll
-    for (int k = 0; k < kTileReplicas; ++k) roff[k] = rep_off_s[k];
-    int64_t *run_out = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 +
-                       ((int64_t)nf0 * rf + (int64_t)nb0 * rb) * 5;
-    const int total = ioff[n_items];
-    // Each pass covers 2 * blockDim.x consecutive words.  Records are 40 bytes, so a replica's
-    // copy of the run starts on an even or an odd word; to write 16 bytes at a time to both
-    // kinds, thread t prepares the words 2t-1, 2t and 2t+1 and stores the pair (2t, 2t+1) to
-    // even-based replicas and the pair (2t-1, 2t) to odd-based ones (single words at the ends).
-    unsigned odd_mask = 0;                           // bit k: replica k's copy starts on an odd word
-#pragma unroll
-    for (int k = 0; k < kTileReplicas; ++k)
-        if (((reinterpret_cast<uintptr_t>(run_out + roff[k]) >> 3) & 1) != 0) odd_mask |= 1u << k;
-    auto word = [&](int x, int it) -> int64_t {
-        const int w = x - ioff[it];
-        const int meta = meta_s[it];
-        const int field = w - (w / 5) * 5;
-        int64_t t = ((meta & 1) ? tb : tf)[w];
-        // times: the jitter event runs [start, start + jitter); every later event is relative to its end
-        if (field == 2) t += (int64_t)(meta >> 1);
-        else if (field >= 3) t += start_s[it] + ((jr && w != 3) ? jit_s[it] : 0);
-        return t;
-    };
-    // (x0 == total can occur: an odd-based replica's last word is then written by the thread at x == total)
-    for (int x0 = 0; x0 <= total; x0 += 2 * kItemThreads) {
-        const int x = x0 + 2 * threadIdx.x;          // the even word of this thread
-        if (x - 1 >= total) break;
-        int lo = 0, hi = n_items - 1;                // item holding word min(x, total-1)
-        const int xs = min(x, total - 1);
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (ioff[mid] <= xs) lo = mid; else hi = mid - 1;
-        }
-        const bool has_m1 = x >= 1, has_0 = x < total, has_p1 = x + 1 < total;
-        int64_t v_m1 = 0, v_0 = 0, v_p1 = 0;
-        if (has_0) v_0 = word(x, lo);
-        if (has_m1) v_m1 = word(x - 1, (has_0 && x == ioff[lo]) ? lo - 1 : lo);
-        if (has_p1) v_p1 = word(x + 1, (x + 1 == ioff[lo + 1]) ? lo + 1 : lo);
-#pragma unroll
-        for (int k = 0; k < kTileReplicas; ++k) {
-            if (k >= n_rep) continue;
-            int64_t *dst = run_out + roff[k] + x;
-            if (!((odd_mask >> k) & 1)) {            // (x, x+1) is 16-byte aligned
-                if (has_p1) __stcs(reinterpret_cast<longlong2 *>(dst), make_longlong2(v_0, v_p1));
-                else if (has_0) __stcs(dst, v_0);
-            } else {                                 // (x-1, x) is 16-byte aligned
-                if (has_m1 && has_0) __stcs(reinterpret_cast<longlong2 *>(dst - 1), make_longlong2(v_m1, v_0));
-                else if (has_0) __stcs(dst, v_0);            // x == 0: the run's first word
-                else if (has_m1) __stcs(dst - 1, v_m1);      // x == total: the run's last word
+    // ---- the run's image: one warp per item, a word is template word + {0, 0, j, start, start} ----
+    const int total = ioff[n_items];                 // <= kTileWords by the plan's choice of tile_items
+    {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        const int lane_field = lane - (lane / 5) * 5;
+        for (int it = warp; it < n_items; it += kItemThreads / 32) {
+            const int off = ioff[it], len = ioff[it + 1] - off;
+            const int meta = meta_s[it];
+            const int64_t *tp = (meta & 1) ? tb : tf;
+            const int64_t j = meta >> 1;
+            // the jitter event runs [start, start + jitter); every later event is relative to its end
+            const int64_t t0 = start_s[it], t1 = t0 + (jr ? jit_s[it] : 0);
+            int field = lane_field;                  // w mod 5, kept without dividing
+            for (int w = lane; w < len; w += 32) {
+                int64_t val = tp[w];
+                if (field == 2) val += j;
+                else if (field >= 3) val += (w == 3 ? t0 : t1);
+                img_a[off + w] = val;
+                img_b[off + w + 1] = val;
+                field += 2;                          // 32 mod 5
+                if (field >= 5) field -= 5;
             }
         }
     }
+    // make the image visible to the bulk-copy engine, then hand it one copy per replica
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x >= n_rep || total == 0) return;
+    // Records are 40 bytes, so a replica's copy of the run starts on a 16-byte boundary or 8 bytes
+    // past one.  Bulk copies need both ends 16-byte aligned: aligned replicas take img_a from word 0,
+    // the others take img_b (the run shifted by one word) from word 1; single words at the ends are
+    // stored directly.
+    int64_t *dst = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 +
+                   ((int64_t)nf0 * rf + (int64_t)nb0 * rb) * 5 + rep_off_s[threadIdx.x];
+    const bool odd = ((reinterpret_cast<uintptr_t>(dst) >> 3) & 1) != 0;
+    const int head = odd ? 1 : 0;                    // words stored directly before the bulk copy
+    const int bulk_words = (total - head) & ~1;
+    if (odd) __stcs(dst, img_a[0]);
+    if (bulk_words > 0) {
+        const int64_t *src = odd ? img_b + 2 : img_a;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     :: "l"(dst + head), "r"(smem_addr(src)), "r"(bulk_words * 8) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    if (head + bulk_words < total) __stcs(dst + total - 1, img_a[total - 1]);
+    // the block's shared memory must outlive the copy engine's reads of it
+    if (bulk_words > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
-// Gradient-bucket records: one warp per (selection, stage).  Buckets whose last byte lies in the
-// same layer share a ready time, so once the first of them has started the rest follow back to
-// back: per layer one serial step (lane 0), inside a layer a closed form (all lanes).
-constexpr int kBucketWarps = 4;
-__global__ void __launch_bounds__(kBucketWarps * 32)
-emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int n, int64_t *__restrict__ out)
+// Gradient-bucket records.  A block owns (selection, stage, chunk of replicas).  Buckets whose last byte lies in the same layer share a ready time, so once the
+// first of them has started the rest follow back to back: per layer one serial step (lane 0),
+// inside a layer a closed form (a thread per bucket).  The records of up to `run` buckets
+// are assembled in shared memory once and sent to every replica by a bulk copy, as in
+// emit_items_kernel.
+__global__ void __launch_bounds__(kBucketThreads)
+emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *__restrict__ out, int run /* buckets per image */)
 {
-    __shared__ int64_t g_start_s[kBucketWarps][DISTSIM_MAX_LAYERS + 1];   // start of the first bucket ending in layer a+i
-    __shared__ int64_t g_first_s[kBucketWarps][DISTSIM_MAX_LAYERS + 1];   // number of that bucket
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t unit = (int64_t)blockIdx.x * kBucketWarps + warp;
-    const int i = (int)(unit / v.sc.pp_max), d = (int)(unit % v.sc.pp_max);
-    if (i >= n) return;
-    const EmitPlan &p = plans[i];
-    if (!p.ok || d >= p.pp || p.dp == 1) return;
+    extern __shared__ __align__(16) int64_t dyn_s[];
+    int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
+    int64_t *img_b = dyn_s + run * 5 + 1;               // the same word at img_b[x + 1] (run * 5 + 1 is even)
+    __shared__ int64_t g_start[DISTSIM_MAX_LAYERS + 1];   // start of the first bucket ending in layer a+i
+    __shared__ int64_t g_first[DISTSIM_MAX_LAYERS + 1];   // number of that bucket
+    __shared__ int64_t part_start_s;
+    const EmitPlan &p = plans[blockIdx.y];
+    if (!p.ok || p.dp == 1) return;
+    const int mp = p.mp, reps = mp * p.dp;
+    const int rep_chunks = (reps + kBucketReplicas - 1) / kBucketReplicas;
+    const int d = blockIdx.x / rep_chunks, rc = blockIdx.x - d * rep_chunks;
+    if (d >= p.pp) return;
     const int64_t kb = p.n_buckets[d];
     if (kb == 0) return;
-    int64_t *g_start = g_start_s[warp], *g_first = g_first_s[warp];
     const Row &row = v.rows[p.row];
     const int a = p.bounds[d], e = p.bounds[d + 1];
     const int L1 = v.tc.n_layers + 1;
@@ -386,16 +395,15 @@ emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int n, int
     const int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
     const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
     const int64_t n_full = nbe[a], t_full = row.t_full;
-    int64_t part_start = 0;
     const int64_t tbs = p.last_b_start[d], main_end = p.main_end[d];
-    // all lanes fetch the per-layer inputs (independent loads), then lane 0 runs the short chain
-    for (int l = a + lane; l < e; l += 32) {
+    // all threads fetch the per-layer inputs (independent loads), then thread 0 runs the short chain
+    for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
         g_first[l - a] = l + 1 < e ? nbe[l + 1] : 0;                       // buckets before layer l's group
         g_start[l - a] = v.tc.overlap ? tbs + (pb[e] - pb[l]) : main_end;    // ready time of the group
     }
-    __syncwarp();
-    if (lane == 0) {
-        int64_t end = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t end = 0, part_start = 0;
         for (int l = e - 1; l >= a; --l) {
             const int64_t nb_prev = g_first[l - a];
             const int64_t nb_l = l > a ? g_first[l - 1 - a] : n_full;       // nb[e][l]
@@ -408,47 +416,58 @@ emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int n, int
             const int64_t ready = v.tc.overlap ? tbs + (pb[e] - pb[ls]) : main_end;
             part_start = max64(end, ready);
         }
+        part_start_s = part_start;
     }
-    part_start = __shfl_sync(0xffffffffu, part_start, 0);
-    __syncwarp();
-    const int mp = p.mp, reps = mp * p.dp;
-    // the stage's bucket words are cut into gridDim.y slices; a value is computed once and
-    // written to every replica
-    const int64_t per = ((kb * 5 + gridDim.y - 1) / gridDim.y + 31) & ~(int64_t)31;
-    const int64_t w0 = (int64_t)blockIdx.y * per, w1 = min(kb * 5, w0 + per);
+    __syncthreads();
+    const int64_t part_start = part_start_s;
     const int64_t stage_words = p.stage_recs[d] * 5;
     const int64_t replica_words = (int64_t)mp * p.stage_rec_prefix[p.pp] * 5;
     int64_t *base = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + (int64_t)p.m * (p.rf[d] + p.rb[d]) * 5;
-    for (int64_t w = w0 + lane; w < w1; w += 32) {
-        const int64_t k = w / 5;
-        const int field = (int)(w - k * 5);
-        int64_t val;
-        if (field == 0) val = DISTSIM_DP_AR;
-        else if (field == 1) val = k;
-        else if (field == 2) val = -1;
-        else {
+    for (int64_t k0 = 0; k0 < kb; k0 += run) {
+        const int nk = (int)min((int64_t)run, kb - k0);
+        for (int kk = threadIdx.x; kk < nk; kk += blockDim.x) {
+            const int64_t k = k0 + kk;
             int64_t start, dur;
             if (k >= n_full) { start = part_start; dur = part; }
             else {
                 // the layer whose group holds bucket k: the largest l with nb[e][l] > k
-                // (nb[e][l] grows as l decreases, and nb[e][a] = n_full > k)
+                // (nb[e][l] = g_first[l-1-a] for l > a grows as l decreases, and nb[e][a] = n_full > k)
                 int lo = a, hi = e - 1;
                 while (lo < hi) {
                     const int mid = (lo + hi + 1) >> 1;
-                    if (nbe[mid] > k) lo = mid; else hi = mid - 1;
+                    if (g_first[mid - 1 - a] > k) lo = mid; else hi = mid - 1;
                 }
                 start = g_start[lo - a] + (k - g_first[lo - a]) * t_full;
                 dur = t_full;
             }
-            val = field == 3 ? start : start + dur;
+            const int64_t rec[5] = {DISTSIM_DP_AR, k, -1, start, start + dur};
+#pragma unroll
+            for (int f = 0; f < 5; ++f) { img_a[kk * 5 + f] = rec[f]; img_b[kk * 5 + f + 1] = rec[f]; }
         }
-        int r = 0, q = 0;
-        int64_t *dst = base + w;
-        for (int rep = 0; rep < reps; ++rep) {
-            __stcs(dst, val);
-            dst += stage_words;
-            if (++q == mp) { q = 0; ++r; dst = base + w + (int64_t)r * replica_words; }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        const int total = nk * 5;
+        const int rep = rc * kBucketReplicas + threadIdx.x;
+        if (threadIdx.x < kBucketReplicas && rep < reps) {
+            const int r = rep / mp, q = rep - r * mp;
+            int64_t *dst = base + (int64_t)r * replica_words + (int64_t)q * stage_words + k0 * 5;
+            // 16-byte aligned copies take img_a from word 0, the others img_b from word 1
+            const bool odd = ((reinterpret_cast<uintptr_t>(dst) >> 3) & 1) != 0;
+            const int head = odd ? 1 : 0;
+            const int bulk_words = (total - head) & ~1;
+            if (odd) __stcs(dst, img_a[0]);
+            if (head + bulk_words < total) __stcs(dst + total - 1, img_a[total - 1]);
+            // the image is rewritten by the next run, and the block's shared memory must outlive
+            // the copy engine's reads of it
+            if (bulk_words > 0) {
+                const int64_t *src = odd ? img_b + 2 : img_a;
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                             :: "l"(dst + head), "r"(smem_addr(src)), "r"(bulk_words * 8) : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            }
         }
+        __syncthreads();
     }
 }
 
@@ -459,7 +478,7 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
                       int64_t *launches)
 {
-    cudaMemsetAsync(d_totals, 0, 3 * sizeof(int64_t), s);
+    cudaMemsetAsync(d_totals, 0, sizeof(EmitTotals), s);
     emit_plan_kernel<<<(n + 3) / 4, 128, 0, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand);
     emit_scan_kernel<<<1, 1024, 0, s>>>(plans, n, d_totals);
     *launches += 2;
@@ -471,26 +490,24 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
 }
 
 void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
-                         const int64_t *op_start, int64_t op_words_per_cand, int64_t max_tiles,
-                         int64_t max_bucket_copies, distsim_record *records, int64_t *launches)
+                         const int64_t *op_start, int64_t op_words_per_cand, const EmitTotals &t,
+                         distsim_record *records, int64_t *launches)
 {
-    if (n == 0 || max_tiles == 0) return;
-    const size_t smem = (size_t)(2 * (3 * v.tc.n_layers + 1)) * 5 * sizeof(int64_t);
-    static size_t smem_set = 0;
-    if (smem > 48 * 1024 && smem > smem_set) {
-        cudaFuncSetAttribute(emit_items_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        smem_set = smem;
-    }
+    if (n == 0 || t.item_tiles == 0) return;
+    // two images of the run, then the forward and backward item templates of the widest stage
+    const size_t smem = (size_t)(2 * kTileWords + 2 + t.tmpl_words) * sizeof(int64_t);
+    cudaFuncSetAttribute(emit_items_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int64_t *out = reinterpret_cast<int64_t *>(records);
-    emit_items_kernel<<<dim3((unsigned)max_tiles, (unsigned)n), kItemThreads, smem, s>>>(
+    emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
         v, plans, op_start, op_words_per_cand, out);
     ++*launches;
-    if (v.tc.n_devices > 1) {
-        const int64_t units = (int64_t)n * v.sc.pp_max;
-        // stages with many bucket records times many replicas are cut into replica slices
-        int64_t ny = (max_bucket_copies + 4095) / 4096;
-        ny = ny < 1 ? 1 : (ny > 64 ? 64 : ny);
-        emit_buckets_kernel<<<dim3((unsigned)((units + kBucketWarps - 1) / kBucketWarps), (unsigned)ny), kBucketWarps * 32, 0, s>>>(v, plans, n, out);
+    if (t.bucket_tiles > 0 && t.bucket_recs > 0) {
+        // an odd number of buckets per image keeps both images 16-byte aligned
+        int run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun);
+        run |= 1;
+        const size_t bsmem = (size_t)(2 * (run * 5 + 1)) * sizeof(int64_t);
+        cudaFuncSetAttribute(emit_buckets_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bsmem);
+        emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, s>>>(v, plans, out, run);
         ++*launches;
     }
 }

@@ -160,6 +160,7 @@ struct EmitPlan {                    // per selected candidate, written by the p
     int32_t row, entry, m, sched, pp, mp, dp, ok;
     int32_t bounds[DISTSIM_MAX_PP + 1];
     int32_t tile_items;              // schedule items per block of the record kernel
+    int32_t tmpl_words;              // words of the widest stage's forward + backward item templates
     int32_t rf[DISTSIM_MAX_PP], rb[DISTSIM_MAX_PP];   // records of one forward / backward item
     int64_t n_buckets[DISTSIM_MAX_PP];
     int64_t stage_recs[DISTSIM_MAX_PP];               // records of one device of stage d
@@ -168,16 +169,24 @@ struct EmitPlan {                    // per selected candidate, written by the p
     int64_t main_end[DISTSIM_MAX_PP];
     int64_t last_b_start[DISTSIM_MAX_PP];
 };
+// Totals over the planned selections (device words written by the scan kernel, read by the host).
+struct EmitTotals {
+    int64_t records;        // records of all selections
+    int64_t item_tiles;     // most item tiles of any selection
+    int64_t bucket_tiles;   // most (stage, replica chunk) tiles of any selection's bucket lanes
+    int64_t tmpl_words;     // most words of any stage's forward + backward item templates
+    int64_t bucket_recs;    // most gradient-bucket records of any stage
+    int64_t pad[3];
+};
 // Plans the n selections: item start times into op_start (op_words_per_cand words each), record
-// counts, offsets / busy / util (each nullable); d_totals[0] = records, d_totals[1] = largest
-// number of item tiles of any selection, d_totals[2] = largest (bucket records x replicas) of any stage.
+// counts, offsets / busy / util (each nullable); d_totals: the words of an EmitTotals.
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
                       int64_t *launches);
 void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
-                         const int64_t *op_start, int64_t op_words_per_cand, int64_t max_tiles,
-                         int64_t max_bucket_copies, distsim_record *records, int64_t *launches);
+                         const int64_t *op_start, int64_t op_words_per_cand, const EmitTotals &totals,
+                         distsim_record *records, int64_t *launches);
 
 // ---- probe (probe_kernels.cu) ----------------------------------------------------------
 // Launches the integer-issue probe; returns the number of integer instructions (per thread,
