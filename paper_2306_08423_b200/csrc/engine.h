@@ -60,6 +60,7 @@ struct Entry {
     int32_t m, b, cls, row;
     int64_t p2p_intra, p2p_inter, a2a, ar;   // [device-filled]
     int64_t bound;        // [device-filled] upper bound on every time of every candidate of the entry
+    int64_t rel_bound;    // [device-filled] bound + the largest shift of a relative time frame
 };
 
 struct SpaceConst {

@@ -19,6 +19,18 @@
 // which does not depend on the schedule; with X = max(0, DT - backward item cost) the stage's
 // contribution to the batch time is main_end + X and its activity time m(fop+bop) + X.
 //
+// Relative time frames (tables without jitter).  Along a wave the cell t_d = max(t_{d-1}, free_d)
+// + c_d chains a max and an add per stage.  Measuring stage d's times from the cost prefix
+// C_d = c_0 + .. + c_d (w_d = t_d - C_d) turns the wave into
+//   w_d = max(r_d + c_d, w_{d-1}),   r_d = w_d of the previous wave,
+// a single fused add-max per cell (__viaddmax_u32 on 32-bit times).  Backward waves use the
+// suffix sums of the backward costs, shifted by their total so that every value stays
+// non-negative (the entry's time bound includes that shift).  In a steady 1F1B wave - a
+// backward and a forward item per stage - the same change of variables, with
+// h_d = latest forward end of stage d - fop_d + bop_0 + .. + bop_{d-1} and fb_d = fop_d + bop_d:
+//   w_d = max(h_d + fb_d, w_{d+1}),   h_d <- max(h_{d-1} + fb_{d-1}, w_d),
+// again one fused add-max per cell.  All of it is exact integer arithmetic.
+//
 // Arithmetic width.  On this GPU a 64-bit max + add costs six half-rate integer instructions,
 // a 32-bit one two full-rate ones.  Every entry carries an upper bound on every time any of its
 // candidates can produce; the entries whose bound is below 2^32 are evaluated with T = uint32_t
@@ -44,6 +56,9 @@ template <typename T> __device__ __forceinline__ T vmax(T a, T b) { return a > b
 
 #ifndef DS_CELL_FORM
 #define DS_CELL_FORM 0            // 0: max(t, free) + c;  1: max(t + c, free + c) (shorter chain)
+#endif
+#ifndef DS_DPX
+#define DS_DPX 1
 #endif
 #ifndef DS_UNROLL_MAIN
 #define DS_UNROLL_MAIN 2
@@ -180,9 +195,65 @@ struct WarmWaves<PP, PP, T, kJit> {
                                                const JitterTab<PP, T, kJit> &) {}
 };
 
+// max(a + b, c): one instruction on 32-bit operands (the GPU's fused add-max).
+template <typename T> __device__ __forceinline__ T addmax(T a, T b, T c) { return vmax((T)(a + b), c); }
+#if DS_DPX
+template <> __device__ __forceinline__ uint32_t addmax<uint32_t>(uint32_t a, uint32_t b, uint32_t c)
+{
+    return __viaddmax_u32(a, b, c);
+}
+#endif
+
+// GPipe without jitter, in relative frames (see the header): returns main-lane ends in free_at.
+template <int PP, typename T>
+__device__ __forceinline__ void run_gpipe_rel(const ThreadState<PP, T> &c, int m, T (&free_at)[PP])
+{
+    // forward, frame w_d = t_d - (fop[0] + .. + fop[d]): r[d] holds w_d of the previous wave;
+    // wave 0 has w = 0 on every stage
+    T r[PP];
+#pragma unroll
+    for (int d = 0; d < PP; ++d) r[d] = 0;
+DS_UNROLL(DS_UNROLL_MAIN)
+    for (int j = 1; j < m; ++j) {
+        T w = r[0] + c.fop[0];
+        r[0] = w;
+#pragma unroll
+        for (int d = 1; d < PP; ++d) { w = addmax(r[d], c.fop[d], w); r[d] = w; }
+    }
+    // backward, frame w_d = t_d + (bop[0] + .. + bop[d-1]): r[d] = (device-free time of stage d)
+    // + that prefix; the stage is free at r[d] + fop[0] + .. + fop[d] after its last forward item
+    T cf = 0, pb = 0;
+#pragma unroll
+    for (int d = 0; d < PP; ++d) { cf += c.fop[d]; r[d] = (T)(r[d] + cf + pb); pb += c.bop[d]; }
+DS_UNROLL(DS_UNROLL_MAIN)
+    for (int j = 0; j < m; ++j) {
+        T w = r[PP - 1] + c.bop[PP - 1];
+        r[PP - 1] = w;
+#pragma unroll
+        for (int d = PP - 2; d >= 0; --d) { w = addmax(r[d], c.bop[d], w); r[d] = w; }
+    }
+    pb = 0;
+#pragma unroll
+    for (int d = 0; d < PP; ++d) { free_at[d] = (T)(r[d] - pb); pb += c.bop[d]; }
+}
+
+// A steady-state 1F1B wave without jitter.  fb[d] = fop[d] + bop[d];
+// h[d] = latest forward end of stage d - fop[d] + (bop[0] + .. + bop[d-1]).
+template <int PP, typename T>
+__device__ __forceinline__ void wave_1f1b_steady_rel(const T (&fb)[PP], T (&h)[PP])
+{
+    T w = 0;
+#pragma unroll
+    for (int d = PP - 1; d >= 0; --d) {
+        w = d == PP - 1 ? (T)(h[d] + fb[d]) : addmax(h[d], fb[d], w);                  // backward item
+        h[d] = d == 0 ? w : addmax(h[d > 0 ? d - 1 : 0], fb[d > 0 ? d - 1 : 0], w);   // forward item
+    }
+}
+
+// rel: the steady waves may use the relative frame (never with jitter).
 template <int PP, typename T, bool kJit>
 __device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (&free_at)[PP],
-                                         const JitterTab<PP, T, kJit> &jt)
+                                         const JitterTab<PP, T, kJit> &jt, bool rel)
 {
     T last_f[PP];
 #pragma unroll
@@ -191,8 +262,19 @@ __device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (
     // waves i = 0 .. m-PP-1: every stage still has a forward item to pair with its backward;
     // entering them every stage's latest item is a forward one (free_at == last_f)
     if (m > PP) {
+        if (kJit || !rel) {
 DS_UNROLL(DS_UNROLL_MAIN)
-        for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T, kJit>(c, last_f, jt, i);
+            for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T, kJit>(c, last_f, jt, i);
+        } else {
+            T fb[PP], pb = 0;
+#pragma unroll
+            for (int d = 0; d < PP; ++d) { fb[d] = c.fop[d] + c.bop[d]; last_f[d] = (T)(last_f[d] - c.fop[d] + pb); pb += c.bop[d]; }
+DS_UNROLL(DS_UNROLL_MAIN)
+            for (int i = 0; i < m - PP; ++i) wave_1f1b_steady_rel<PP, T>(fb, last_f);
+            pb = 0;
+#pragma unroll
+            for (int d = 0; d < PP; ++d) { last_f[d] = (T)(last_f[d] + c.fop[d] - pb); pb += c.bop[d]; }
+        }
 #pragma unroll
         for (int d = 0; d < PP; ++d) free_at[d] = last_f[d];
     }
@@ -229,7 +311,7 @@ __host__ __device__ inline ThreadKernelSmem thread_kernel_smem(int n_entries, in
 }
 
 // Entry scalars the hot path needs, kept in shared memory for the whole row.
-struct EntryLite { int64_t p2p_intra, p2p_inter; int32_t m, pad; };
+struct EntryLite { int64_t p2p_intra, p2p_inter; int32_t m, rel_fits32; };
 
 constexpr int kMaxJitterSlots = 64;
 
@@ -269,6 +351,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
         ents[threadIdx.x].p2p_intra = en.p2p_intra;
         ents[threadIdx.x].p2p_inter = en.p2p_inter;
         ents[threadIdx.x].m = en.m;
+        ents[threadIdx.x].rel_fits32 = en.rel_bound < ((int64_t)1 << 32) ? 1 : 0;
     }
     if (kJit)
         for (int k = threadIdx.x; k < v.tc.n_jitter * PP; k += blockDim.x) {
@@ -324,8 +407,13 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
         const int64_t *pb = etb + (int64_t)e * lp;
         int m;
         int64_t p2p_intra, p2p_inter;
-        if (e < kMaxRowEntries) { m = ents[e].m; p2p_intra = ents[e].p2p_intra; p2p_inter = ents[e].p2p_inter; }
-        else { const Entry &en = v.entries[row.entry0 + e]; m = en.m; p2p_intra = en.p2p_intra; p2p_inter = en.p2p_inter; }
+        bool rel = sizeof(T) == 8;      // the relative frames' shift must fit the arithmetic width as well
+        if (e < kMaxRowEntries) { m = ents[e].m; p2p_intra = ents[e].p2p_intra; p2p_inter = ents[e].p2p_inter; rel = rel || ents[e].rel_fits32; }
+        else {
+            const Entry &en = v.entries[row.entry0 + e];
+            m = en.m; p2p_intra = en.p2p_intra; p2p_inter = en.p2p_inter;
+            rel = rel || en.rel_bound < ((int64_t)1 << 32);
+        }
         const int64_t *dte = v.dt ? v.dt + (int64_t)(row.entry0 + e) * v.tab_words : nullptr;
 
         // ---- stage costs and bucket-lane excess (schedule independent) -------------------
@@ -381,8 +469,11 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
             const int64_t local = local0 + sc;
             if (local < lo || local >= hi) continue;
             T free_at[PP];
-            if (sched0 + sc == 0) run_gpipe<PP, T, kJit>(st, m, free_at, jt);
-            else run_1f1b<PP, T, kJit>(st, m, free_at, jt);
+            if (sched0 + sc == 0) {
+                if (kJit || !rel) run_gpipe<PP, T, kJit>(st, m, free_at, jt);
+                else run_gpipe_rel<PP, T>(st, m, free_at);
+            }
+            else run_1f1b<PP, T, kJit>(st, m, free_at, jt, rel);
             T batch = 0;
 #pragma unroll
             for (int d = 0; d < PP; ++d) batch = vmax(batch, (T)(free_at[d] + xs[d][threadIdx.x]));

@@ -173,6 +173,8 @@ __global__ void build_dt_kernel(DeviceView v, int64_t *dt)
 
 // One thread per entry: an upper bound on every time any candidate of the entry can produce:
 // all items of the pipeline in sequence plus the largest possible bucket-lane excess.
+// rel_bound adds one more backward pass over all stages, the largest shift of the evaluation
+// kernel's relative time frames.
 __global__ void entry_bound_kernel(DeviceView v, Entry *entries, int64_t *jsum)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -181,9 +183,12 @@ __global__ void entry_bound_kernel(DeviceView v, Entry *entries, int64_t *jsum)
     const Row &row = v.rows[en.row];
     const int L = v.tc.n_layers, L1 = L + 1;
     const int64_t *pf = v.etf + (int64_t)i * v.tc.lp, *pb = v.etb + (int64_t)i * v.tc.lp;
-    int64_t per_mb = pf[L] + pb[L];
-    for (int d = 0; d + 1 < row.pp; ++d)
-        per_mb += 2 * ((((d + 1) & (row.p2p_period - 1)) == 0) ? en.p2p_inter : en.p2p_intra);
+    int64_t per_mb = pf[L] + pb[L], frame_shift = pb[L];
+    for (int d = 0; d + 1 < row.pp; ++d) {
+        const int64_t p2p = (((d + 1) & (row.p2p_period - 1)) == 0) ? en.p2p_inter : en.p2p_intra;
+        per_mb += 2 * p2p;
+        frame_shift += p2p;
+    }
     int64_t excess = 0;
     if (row.dp > 1) {
         const int64_t *nbL = v.nb + row.row_tab_off + (int64_t)L * L1;
@@ -212,6 +217,7 @@ __global__ void entry_bound_kernel(DeviceView v, Entry *entries, int64_t *jsum)
     }
     const __int128 b = (__int128)en.m * per_mb + excess + jitter_total;
     en.bound = b >= (__int128)kSat ? kSat : (int64_t)b;
+    en.rel_bound = b + frame_shift >= (__int128)kSat ? kSat : (int64_t)(b + frame_shift);
     entries[i] = en;
 }
 
