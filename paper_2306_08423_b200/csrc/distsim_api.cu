@@ -73,6 +73,7 @@ struct distsim_ctx {
 
     // scratch
     DevBuf d_status, d_sel, d_result, d_plans, d_op_start, d_totals, d_batch, d_topk;
+    SideStream side;                      // second stream of an evaluation (lock-step launches)
     int64_t *h_pinned = nullptr;          // 16 words of pinned host memory for small results:
                                           // [0..3] results, [4] status, [8..15] emission totals
 
@@ -179,8 +180,20 @@ int distsim_create(distsim_ctx **out, int cuda_device)
         ctx->d_result.reserve(64) != cudaSuccess || ctx->d_totals.reserve(64) != cudaSuccess ||
         cudaMemset(ctx->d_status.p, 0, 64) != cudaSuccess ||
         cudaMallocHost(&ctx->h_pinned, 16 * sizeof(int64_t)) != cudaSuccess) {
-        delete ctx;
+        distsim_destroy(ctx);
         return DISTSIM_E_CUDA;
+    }
+    // the side stream is an optimisation: without it evaluations run on the caller's stream alone
+    int prio_lo = 0, prio_hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&ctx->side.side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->side.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->side.join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        if (ctx->side.fork) cudaEventDestroy(ctx->side.fork);
+        if (ctx->side.join) cudaEventDestroy(ctx->side.join);
+        if (ctx->side.side) cudaStreamDestroy(ctx->side.side);
+        ctx->side = SideStream{};
     }
     *out = ctx;
     return DISTSIM_OK;
@@ -191,6 +204,9 @@ void distsim_destroy(distsim_ctx *ctx)
     if (!ctx) return;
     cudaSetDevice(ctx->device);
     if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
+    if (ctx->side.fork) cudaEventDestroy(ctx->side.fork);
+    if (ctx->side.join) cudaEventDestroy(ctx->side.join);
+    if (ctx->side.side) cudaStreamDestroy(ctx->side.side);
     delete ctx;
 }
 
@@ -474,7 +490,7 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
     if (int rc = set_device(ctx)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const DeviceView v = ctx->view();
-    launch_eval(s, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
+    launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
                 d_batch_ns, d_stage_busy_ns, &ctx->launches);
     CU(cudaGetLastError(), "evaluation launch");
     return DISTSIM_OK;

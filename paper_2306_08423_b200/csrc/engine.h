@@ -130,10 +130,18 @@ struct EvalBatch {
     int32_t n, pad;
     EvalWork w[kMaxEvalWork];
 };
+// A second stream for the latency-bound lock-step launches of an evaluation, so that they run
+// beside the throughput-bound launches instead of after them (side == nullptr: one stream).
+struct SideStream {
+    cudaStream_t side = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
 // Evaluates candidates [first, first + count); rows / entries: host copies.  Results go to
-// batch_out[index - first] and, if non-null, busy_out[(index - first) * pp_max + d].
-void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_rows, const Entry *entries,
-                 int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out, int64_t *launches);
+// batch_out[index - first] and, if non-null, busy_out[(index - first) * pp_max + d].  All work
+// is ordered after what `s` held before the call and before what is enqueued on `s` after it.
+void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
+                 const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
+                 int64_t *launches);
 
 // ---- selection (select_kernels.cu) -----------------------------------------------------
 struct SelectScratch {

@@ -176,10 +176,23 @@ int ilog2(int v) { int b = 0; while ((1 << (b + 1)) <= v) ++b; return b; }
 
 }  // namespace
 
-void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_rows, const Entry *entries,
-                 int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out, int64_t *launches)
+void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
+                 const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
+                 int64_t *launches)
 {
     const int64_t last = first + count;
+    // lock-step launches go to the side stream, forked from `s` here and joined at the end
+    cudaStream_t ls = s;
+    bool forked = false;
+    auto lockstep_stream = [&]() {
+        if (ss.side && !forked) {
+            cudaEventRecord(ss.fork, s);
+            cudaStreamWaitEvent(ss.side, ss.fork, 0);
+            ls = ss.side;
+            forked = true;
+        }
+        return ls;
+    };
     Pending lock[2];                               // lock-step kernel, S = 1 and S = 2
     Pending thr[5][2];                             // thread kernel, [log2 pp][narrow]
     constexpr int kMaxBlocks = 1 << 30;
@@ -189,8 +202,8 @@ void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_row
         Pending &p = lock[which];
         const int blocks = lockstep_blocks(rows[r], lo, hi);
         if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - blocks) {
-            if (which) flush_lockstep<2>(s, v, p, first, batch_out, busy_out, launches);
-            else flush_lockstep<1>(s, v, p, first, batch_out, busy_out, launches);
+            if (which) flush_lockstep<2>(lockstep_stream(), v, p, first, batch_out, busy_out, launches);
+            else flush_lockstep<1>(lockstep_stream(), v, p, first, batch_out, busy_out, launches);
         }
         EvalWork &w = p.batch.w[p.batch.n++];
         w = EvalWork{};
@@ -248,12 +261,17 @@ void launch_eval(cudaStream_t s, const DeviceView &v, const Row *rows, int n_row
             r0 = r1;
         }
     }
-    // largest kernels first, so that the small ones fill the tail of the big ones
+    // the lock-step launches first, on their own stream: few blocks that run for long, beside
+    // the thread-kernel launches (largest first) that fill the rest of the device
+    if (lock[1].batch.n) flush_lockstep<2>(lockstep_stream(), v, lock[1], first, batch_out, busy_out, launches);
+    if (lock[0].batch.n) flush_lockstep<1>(lockstep_stream(), v, lock[0], first, batch_out, busy_out, launches);
     for (int lg = 4; lg >= 0; --lg)
         for (int nw = 1; nw >= 0; --nw)
             flush_thread_any(lg, nw == 1, s, v, thr[lg][nw], first, batch_out, busy_out, launches);
-    flush_lockstep<2>(s, v, lock[1], first, batch_out, busy_out, launches);
-    flush_lockstep<1>(s, v, lock[0], first, batch_out, busy_out, launches);
+    if (forked) {
+        cudaEventRecord(ss.join, ss.side);
+        cudaStreamWaitEvent(s, ss.join, 0);
+    }
 }
 
 }  // namespace distsim
