@@ -73,7 +73,7 @@ struct distsim_ctx {
 
     // scratch
     DevBuf d_status, d_sel, d_result, d_plans, d_op_start, d_totals, d_batch, d_topk;
-    SideStream side;                      // second stream of an evaluation (lock-step launches)
+    SideStream side;                      // extra streams of an evaluation (lock-step launches)
     int64_t *h_pinned = nullptr;          // 16 words of pinned host memory for small results:
                                           // [0..3] results, [4] status, [8..15] emission totals
 
@@ -156,6 +156,16 @@ int read_status(distsim_ctx *ctx, cudaStream_t s)
     return DISTSIM_OK;
 }
 
+void destroy_side(SideStream &ss)
+{
+    if (ss.fork) cudaEventDestroy(ss.fork);
+    for (int k = 0; k < 2; ++k) {
+        if (ss.join[k]) cudaEventDestroy(ss.join[k]);
+        if (ss.side[k]) cudaStreamDestroy(ss.side[k]);
+    }
+    ss = SideStream{};
+}
+
 int floor_log2(int64_t v) { int b = -1; while (v > 0) { ++b; v >>= 1; } return b; }
 
 }  // namespace
@@ -183,17 +193,16 @@ int distsim_create(distsim_ctx **out, int cuda_device)
         distsim_destroy(ctx);
         return DISTSIM_E_CUDA;
     }
-    // the side stream is an optimisation: without it evaluations run on the caller's stream alone
+    // the side streams are an optimisation: without them evaluations run on the caller's stream alone
     int prio_lo = 0, prio_hi = 0;
     if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess ||
-        cudaStreamCreateWithPriority(&ctx->side.side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&ctx->side.side[0], cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&ctx->side.side[1], cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->side.fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ctx->side.join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ctx->side.join[0], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->side.join[1], cudaEventDisableTiming) != cudaSuccess) {
         cudaGetLastError();
-        if (ctx->side.fork) cudaEventDestroy(ctx->side.fork);
-        if (ctx->side.join) cudaEventDestroy(ctx->side.join);
-        if (ctx->side.side) cudaStreamDestroy(ctx->side.side);
-        ctx->side = SideStream{};
+        destroy_side(ctx->side);
     }
     *out = ctx;
     return DISTSIM_OK;
@@ -204,9 +213,7 @@ void distsim_destroy(distsim_ctx *ctx)
     if (!ctx) return;
     cudaSetDevice(ctx->device);
     if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
-    if (ctx->side.fork) cudaEventDestroy(ctx->side.fork);
-    if (ctx->side.join) cudaEventDestroy(ctx->side.join);
-    if (ctx->side.side) cudaStreamDestroy(ctx->side.side);
+    destroy_side(ctx->side);
     delete ctx;
 }
 

@@ -130,11 +130,12 @@ struct EvalBatch {
     int32_t n, pad;
     EvalWork w[kMaxEvalWork];
 };
-// A second stream for the latency-bound lock-step launches of an evaluation, so that they run
-// beside the throughput-bound launches instead of after them (side == nullptr: one stream).
+// Two more streams for the latency-bound lock-step launches of an evaluation (one per kernel
+// instance), so that they run beside each other and beside the throughput-bound launches
+// instead of one after the other (side[0] == nullptr: everything on the caller's stream).
 struct SideStream {
-    cudaStream_t side = nullptr;
-    cudaEvent_t fork = nullptr, join = nullptr;
+    cudaStream_t side[2] = {nullptr, nullptr};
+    cudaEvent_t fork = nullptr, join[2] = {nullptr, nullptr};
 };
 // Evaluates candidates [first, first + count); rows / entries: host copies.  Results go to
 // batch_out[index - first] and, if non-null, busy_out[(index - first) * pp_max + d].  All work

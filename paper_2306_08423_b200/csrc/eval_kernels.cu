@@ -181,17 +181,13 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
                  int64_t *launches)
 {
     const int64_t last = first + count;
-    // lock-step launches go to the side stream, forked from `s` here and joined at the end
-    cudaStream_t ls = s;
-    bool forked = false;
-    auto lockstep_stream = [&]() {
-        if (ss.side && !forked) {
-            cudaEventRecord(ss.fork, s);
-            cudaStreamWaitEvent(ss.side, ss.fork, 0);
-            ls = ss.side;
-            forked = true;
-        }
-        return ls;
+    // lock-step launches go to the side streams, forked from `s` on first use and joined at the end
+    bool fork_recorded = false, forked[2] = {false, false};
+    auto lockstep_stream = [&](int which) {
+        if (!ss.side[0]) return s;
+        if (!fork_recorded) { cudaEventRecord(ss.fork, s); fork_recorded = true; }
+        if (!forked[which]) { cudaStreamWaitEvent(ss.side[which], ss.fork, 0); forked[which] = true; }
+        return ss.side[which];
     };
     Pending lock[2];                               // lock-step kernel, S = 1 and S = 2
     Pending thr[5][2];                             // thread kernel, [log2 pp][narrow]
@@ -202,8 +198,8 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
         Pending &p = lock[which];
         const int blocks = lockstep_blocks(rows[r], lo, hi);
         if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - blocks) {
-            if (which) flush_lockstep<2>(lockstep_stream(), v, p, first, batch_out, busy_out, launches);
-            else flush_lockstep<1>(lockstep_stream(), v, p, first, batch_out, busy_out, launches);
+            if (which) flush_lockstep<2>(lockstep_stream(1), v, p, first, batch_out, busy_out, launches);
+            else flush_lockstep<1>(lockstep_stream(0), v, p, first, batch_out, busy_out, launches);
         }
         EvalWork &w = p.batch.w[p.batch.n++];
         w = EvalWork{};
@@ -261,17 +257,18 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
             r0 = r1;
         }
     }
-    // the lock-step launches first, on their own stream: few blocks that run for long, beside
+    // the lock-step launches first, on their own streams: few blocks that run for long, beside
     // the thread-kernel launches (largest first) that fill the rest of the device
-    if (lock[1].batch.n) flush_lockstep<2>(lockstep_stream(), v, lock[1], first, batch_out, busy_out, launches);
-    if (lock[0].batch.n) flush_lockstep<1>(lockstep_stream(), v, lock[0], first, batch_out, busy_out, launches);
+    if (lock[1].batch.n) flush_lockstep<2>(lockstep_stream(1), v, lock[1], first, batch_out, busy_out, launches);
+    if (lock[0].batch.n) flush_lockstep<1>(lockstep_stream(0), v, lock[0], first, batch_out, busy_out, launches);
     for (int lg = 4; lg >= 0; --lg)
         for (int nw = 1; nw >= 0; --nw)
             flush_thread_any(lg, nw == 1, s, v, thr[lg][nw], first, batch_out, busy_out, launches);
-    if (forked) {
-        cudaEventRecord(ss.join, ss.side);
-        cudaStreamWaitEvent(s, ss.join, 0);
-    }
+    for (int k = 0; k < 2; ++k)
+        if (forked[k]) {
+            cudaEventRecord(ss.join[k], ss.side[k]);
+            cudaStreamWaitEvent(s, ss.join[k], 0);
+        }
 }
 
 }  // namespace distsim

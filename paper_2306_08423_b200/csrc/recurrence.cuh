@@ -91,15 +91,15 @@ __device__ __forceinline__ void slot_activity(int sched, int pp, int m, int d, i
 {
     const int x = s - d;
     if (sched == 0) {
-        do_f = x >= 0 && x < m;
         const int y = s - (m + 2 * pp - 2 - d);
-        do_b = y >= 0 && y < m;
+        do_f = (unsigned)x < (unsigned)m;
+        do_b = (unsigned)y < (unsigned)m;
         j = do_f ? x : y;
     } else {
         const int w = min(pp - d, m);
-        const bool warm = x >= 0 && x < w;
-        do_f = warm || (x >= 2 * w && !(x & 1) && (x >> 1) < m);
         const int y = s - (2 * pp - 1 - d);
+        const bool warm = (unsigned)x < (unsigned)w;
+        do_f = warm || (x >= 2 * w && !(x & 1) && (x >> 1) < m);
         do_b = y >= 0 && !(y & 1) && (y >> 1) < m;
         j = do_f ? (warm ? x : x >> 1) : y >> 1;
     }
@@ -200,6 +200,8 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
 #pragma unroll
     for (int k = 0; k < S; ++k) { last_f[k] = 0; last_b[k] = 0; free_at[k] = 0; n_done[k] = 0; }
 
+    // The lanes of a warp run forward items, backward items or nothing in the same slot, so the
+    // slot body is written without branches: one cell with selected operands per owned stage.
     for (int s = 0; s < n_slots_warp; ++s) {
         const int64_t up_f = __shfl_up_sync(0xffffffffu, last_f[S - 1], 1, wl);
         const int64_t dn_b = __shfl_down_sync(0xffffffffu, last_b[0], 1, wl);
@@ -212,21 +214,20 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
             bool do_f, do_b;
             int j;
             slot_activity(sched, pp, m, d, s, do_f, do_b, j);
-            if (do_f) {
-                const int64_t dep = (k == 0) ? (seg_lane == 0 ? 0 : up_f) : old_f[k > 0 ? k - 1 : 0];
-                const int64_t st = max64(dep, free_at[k]);
-                if (kRecord && rec) rec[(int64_t)d * 2 * m + n_done[k]] = st;
-                last_f[k] = free_at[k] = st + R.fop[k] + (kJit ? jitter_of(v, v.raw.jit_f, j, d) : 0);
-                ++n_done[k];
-            } else if (do_b) {
-                const int64_t dep = (k == S - 1) ? (seg_lane == wl - 1 ? 0 : dn_b) : old_b[k < S - 1 ? k + 1 : 0];
-                const int64_t st = max64(dep, free_at[k]);
-                const int64_t jit = kJit ? jitter_of(v, v.raw.jit_b, j, d) : 0;
-                if (kRecord && rec) rec[(int64_t)d * 2 * m + n_done[k]] = st;
-                R.last_b_start[k] = st + jit;
-                last_b[k] = free_at[k] = st + jit + R.bop[k];
-                ++n_done[k];
-            }
+            do_b = do_b && !do_f;
+            const bool act = do_f || do_b;
+            const int64_t dep_f = (k == 0) ? (seg_lane == 0 ? 0 : up_f) : old_f[k > 0 ? k - 1 : 0];
+            const int64_t dep_b = (k == S - 1) ? (seg_lane == wl - 1 ? 0 : dn_b) : old_b[k < S - 1 ? k + 1 : 0];
+            const int64_t st = max64(do_f ? dep_f : dep_b, free_at[k]);
+            int64_t jit = 0;
+            if (kJit) jit = act ? jitter_of(v, do_f ? v.raw.jit_f : v.raw.jit_b, j, d) : 0;
+            const int64_t end = st + jit + (do_f ? R.fop[k] : R.bop[k]);
+            if (kRecord && rec && act) rec[(int64_t)d * 2 * m + n_done[k]] = st;
+            if (S > 1 && !act) continue;             // a lane with several stages skips its idle ones
+            if (act) free_at[k] = end;
+            if (do_f) last_f[k] = end;
+            if (do_b) { last_b[k] = end; R.last_b_start[k] = st + jit; }
+            n_done[k] += act ? 1 : 0;
         }
     }
 
