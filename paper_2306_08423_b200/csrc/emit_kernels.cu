@@ -134,21 +134,32 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
 // Exclusive scan of rec_total over the selections (n is small: one block, serial per chunk).
 __global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /* the words of EmitTotals */)
 {
-    __shared__ int64_t chunk_sum[1024];
-    const int t = threadIdx.x, nt = blockDim.x;
+    __shared__ int64_t warp_sum[32];
+    const int t = threadIdx.x, nt = blockDim.x, lane = t & 31, warp = t >> 5;
     const int per = (n + nt - 1) / nt;
     const int b = min(n, t * per), e = min(n, b + per);
     int64_t s = 0, mt = 0, mb = 0, mw = 0, mk = 0;
     for (int i = b; i < e; ++i) s += plans[i].rec_total;
-    chunk_sum[t] = s;
+    // exclusive scan of the per-thread sums over the block: inside warps, then over the warp totals
+    int64_t incl = s;
+    for (int off = 1; off < 32; off <<= 1) {
+        const int64_t up = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
     __syncthreads();
-    if (t == 0) {
-        int64_t acc = 0;
-        for (int k = 0; k < nt; ++k) { const int64_t x = chunk_sum[k]; chunk_sum[k] = acc; acc += x; }
-        totals[0] = acc;
+    if (warp == 0) {
+        const int64_t w = lane < (nt >> 5) ? warp_sum[lane] : 0;
+        int64_t wi = w;
+        for (int off = 1; off < 32; off <<= 1) {
+            const int64_t up = __shfl_up_sync(0xffffffffu, wi, off);
+            if (lane >= off) wi += up;
+        }
+        warp_sum[lane] = wi - w;                       // exclusive
+        if (lane == 31) totals[0] = wi;
     }
     __syncthreads();
-    int64_t acc = chunk_sum[t];
+    int64_t acc = warp_sum[warp] + incl - s;
     for (int i = b; i < e; ++i) {
         plans[i].rec_base = acc; acc += plans[i].rec_total;
         if (plans[i].ok) {
