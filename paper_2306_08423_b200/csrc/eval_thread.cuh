@@ -250,10 +250,82 @@ __device__ __forceinline__ void wave_1f1b_steady_rel(const T (&fb)[PP], T (&h)[P
     }
 }
 
-// rel: the steady waves may use the relative frame (never with jitter).
+// 1F1B without jitter and with m >= PP, entirely in relative frames.
+//   warm-up   forward frame as in run_gpipe_rel: r[d] = w_d of stage d's latest forward item.
+//   then      h[d] = (end of stage d's latest forward item) - fop[d] + bop[0] + .. + bop[d-1]
+//             while the stage's latest item is a forward one ("after F"), and
+//             h[d] = (end of its latest backward item) + bop[0] + .. + bop[d-1] once it is a
+//             backward one ("after B", in the last waves); the backward item of the next wave is
+//             w_d = max(h[d] + y_d, w_{d+1}) with y_d = fop[d] + bop[d] after F and bop[d] after B.
+// Wave K of the tail (K waves to go, i = m - K): stages d >= PP-K+1 still run a forward item; a
+// stage is "after F" iff it ran one in the wave before (d >= PP-K; in the first wave, K = PP,
+// that is every stage).  Requires m >= PP: all PP warm-up waves and all PP tail waves exist.
+template <int PP, int K, typename T>
+struct TailWavesRel {
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &c, const T (&fb)[PP], int m, T (&h)[PP])
+    {
+        {
+            T w = 0;
+#pragma unroll
+            for (int d = PP - 1; d >= 0; --d) {
+                const T y = d >= PP - K ? fb[d] : c.bop[d];
+                w = d == PP - 1 ? (T)(h[d] + y) : addmax(h[d], y, w);
+                if (d >= PP - K + 1) h[d] = d == 0 ? w : addmax(h[d > 0 ? d - 1 : 0], fb[d > 0 ? d - 1 : 0], w);
+                else h[d] = w;
+            }
+        }
+        TailWavesRel<PP, K - 1, T>::run(c, fb, m, h);
+    }
+};
+template <int PP, typename T>
+struct TailWavesRel<PP, 0, T> {
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &, const T (&)[PP], int, T (&)[PP]) {}
+};
+
+// Warm-up forward wave J >= 1 over stages 0 .. PP-1-J (wave 0 leaves w = 0 everywhere).
+template <int PP, int J, typename T>
+struct WarmWavesRel {
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &c, int m, T (&r)[PP])
+    {
+        {
+            T w = r[0] + c.fop[0];
+            r[0] = w;
+#pragma unroll
+            for (int d = 1; d < PP - J; ++d) { w = addmax(r[d], c.fop[d], w); r[d] = w; }
+        }
+        WarmWavesRel<PP, J + 1, T>::run(c, m, r);
+    }
+};
+template <int PP, typename T>
+struct WarmWavesRel<PP, PP, T> {
+    static __device__ __forceinline__ void run(const ThreadState<PP, T> &, int, T (&)[PP]) {}
+};
+
+template <int PP, typename T>
+__device__ __forceinline__ void run_1f1b_rel(const ThreadState<PP, T> &c, int m, T (&free_at)[PP])
+{
+    T h[PP], fb[PP];
+#pragma unroll
+    for (int d = 0; d < PP; ++d) { h[d] = 0; fb[d] = c.fop[d] + c.bop[d]; }
+    WarmWavesRel<PP, (PP > 1 ? 1 : PP), T>::run(c, m, h);
+    // forward frame -> the frame of h: add fop[0] + .. + fop[d-1] and bop[0] + .. + bop[d-1]
+    T off = 0;
+#pragma unroll
+    for (int d = 0; d < PP; ++d) { h[d] += off; off += fb[d]; }
+    if (m > PP) {
+DS_UNROLL(DS_UNROLL_MAIN)
+        for (int i = 0; i < m - PP; ++i) wave_1f1b_steady_rel<PP, T>(fb, h);
+    }
+    TailWavesRel<PP, PP, T>::run(c, fb, m, h);
+    // every stage's latest item is now its last backward item
+    T pb = 0;
+#pragma unroll
+    for (int d = 0; d < PP; ++d) { free_at[d] = (T)(h[d] - pb); pb += c.bop[d]; }
+}
+
 template <int PP, typename T, bool kJit>
 __device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (&free_at)[PP],
-                                         const JitterTab<PP, T, kJit> &jt, bool rel)
+                                         const JitterTab<PP, T, kJit> &jt)
 {
     T last_f[PP];
 #pragma unroll
@@ -262,19 +334,8 @@ __device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (
     // waves i = 0 .. m-PP-1: every stage still has a forward item to pair with its backward;
     // entering them every stage's latest item is a forward one (free_at == last_f)
     if (m > PP) {
-        if (kJit || !rel) {
 DS_UNROLL(DS_UNROLL_MAIN)
-            for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T, kJit>(c, last_f, jt, i);
-        } else {
-            T fb[PP], pb = 0;
-#pragma unroll
-            for (int d = 0; d < PP; ++d) { fb[d] = c.fop[d] + c.bop[d]; last_f[d] = (T)(last_f[d] - c.fop[d] + pb); pb += c.bop[d]; }
-DS_UNROLL(DS_UNROLL_MAIN)
-            for (int i = 0; i < m - PP; ++i) wave_1f1b_steady_rel<PP, T>(fb, last_f);
-            pb = 0;
-#pragma unroll
-            for (int d = 0; d < PP; ++d) { last_f[d] = (T)(last_f[d] + c.fop[d] - pb); pb += c.bop[d]; }
-        }
+        for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T, kJit>(c, last_f, jt, i);
 #pragma unroll
         for (int d = 0; d < PP; ++d) free_at[d] = last_f[d];
     }
@@ -473,7 +534,8 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
                 if (kJit || !rel) run_gpipe<PP, T, kJit>(st, m, free_at, jt);
                 else run_gpipe_rel<PP, T>(st, m, free_at);
             }
-            else run_1f1b<PP, T, kJit>(st, m, free_at, jt, rel);
+            else if (kJit || !rel || m < PP) run_1f1b<PP, T, kJit>(st, m, free_at, jt);
+            else run_1f1b_rel<PP, T>(st, m, free_at);
             T batch = 0;
 #pragma unroll
             for (int d = 0; d < PP; ++d) batch = vmax(batch, (T)(free_at[d] + xs[d][threadIdx.x]));
