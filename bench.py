@@ -43,8 +43,9 @@ RECORD_BYTES = 40
 # DRAM read + write bytes per step of the timed workload, from the one-pass ncu counters summarised in
 # profiles/bench_config1_dram_bytes.md.  They describe the kernels as captured: set them to None when
 # an evaluation or emission kernel changes, until the counters are taken again.
-EVAL_TRAFFIC_BYTES = 205_375_000
-EMIT_TRAFFIC_BYTES = 1_698_347_000
+EVAL_TRAFFIC_BYTES = None
+EMIT_TRAFFIC_BYTES = None
+SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32      # issue slots: one warp instruction per scheduler and clock
 
 
 def measured_peaks():
@@ -322,6 +323,9 @@ def run_ours(args):
         return ops / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
     int_peak_gops = probe(0)
     cell64_peak, cell32_peak, cmpsel_peak = probe(1) / 6, probe(3) / 2, probe(2)      # G cells/s, G instr/s
+    cell32_fused_peak = probe(4) / 2                                                 # G cells/s, one fused add-max per cell
+    cell32_peak = max(cell32_peak, cell32_fused_peak)
+    sm_mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
     cells_all, cells_32 = E.distsim_space_cells(ctx)
     assert cells_all == cells
     eval_s = statistics.mean(eval_ms) * 1e-3
@@ -333,12 +337,20 @@ def run_ours(args):
                 "achieved": achieved_gops, "peak": int_peak_gops,
                 "unit": "G 32-bit integer instr/s (2 per uint32 cell, 6 per int64 cell)",
                 "frac": achieved_gops / int_peak_gops, "traffic": EVAL_TRAFFIC_BYTES,
-                "traffic_note": "DRAM read + write bytes of the four evaluation launches of one step (ncu, one pass); "
-                                "of it 141.4e6 by the dominant launch; algorithmic: 8 B per candidate = "
-                                f"{8 * n_total} B, part of which is still in the L2 when the launches end",
+                "traffic_note": "DRAM read + write bytes of the four evaluation launches of one step (ncu, one pass; "
+                                "null when the kernels changed after the counters were taken); algorithmic: 8 B per "
+                                f"candidate = {8 * n_total} B, part of which is still in the L2 when the launches end",
                 "peak_kind": "measured in this run: dependency-free add/xor stream",
                 "cells": cells, "cells_32bit": cells_32, "ms_per_launch_set": statistics.mean(eval_ms),
-                "cell_rate_peaks_Gcells_per_s": {"uint32": cell32_peak, "int64": cell64_peak},
+                "cell_rate_peaks_Gcells_per_s": {"uint32": cell32_peak, "uint32_fused_add_max": cell32_fused_peak,
+                                                 "int64": cell64_peak},
+                "peak_derived": {"issue_slots_Ginstr_per_s": SM_COUNT * SCHEDULERS_PER_SM * LANES * sm_mhz * 1e-3,
+                                 "half_rate_max_Gcells_per_s": SM_COUNT * SCHEDULERS_PER_SM * LANES / 2 * sm_mhz * 1e-3,
+                                 "sm_mhz": sm_mhz,
+                                 "note": "148 SMs x 4 schedulers x 32 lanes x SM clock; integer max (and the fused "
+                                         "add-max) issues at half rate, one per cell"},
+                "frac_of_derived_half_rate_max": (cells / eval_s / 1e9) /
+                                                 (SM_COUNT * SCHEDULERS_PER_SM * LANES / 2 * sm_mhz * 1e-3),
                 "compare_select_peak_Ginstr_per_s": cmpsel_peak,
                 "frac_of_cell_rate_floor": cell_floor_s / eval_s}
     emit_bytes = tot * RECORD_BYTES + TOP_K * N * 24 + 8
@@ -354,7 +366,8 @@ def run_ours(args):
         "metric": "strategy_candidates_per_sec", "value": value, "unit": "candidates/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int64 (exact uint32 arithmetic inside entries whose time bound is below 2^32)",
+        "dtype": "int64",
+        "dtype_note": "int64 nanoseconds at the boundary; exact uint32 arithmetic inside entries whose time bound is below 2^32",
         "data": "synthetic",
         "config": {"workload": w.name, "candidates": n_total, "recurrence_cells": cells, "devices": N,
                    "layers": table.n_layers, "top_k_emitted": TOP_K, "records_emitted": tot,

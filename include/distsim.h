@@ -262,8 +262,10 @@ int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int64_t first, 
  * the total instruction count (threads x instructions) in *h_ops.  mode 0: 16 32-bit add / xor
  * instructions per round; mode 1: 8 recurrence cells x = max(x, y) + c on int64 per round,
  * counted as 6 instructions each; mode 2: 16 32-bit compare / select instructions per round;
- * mode 3: 8 recurrence cells on uint32 per round, counted as 2 instructions each.  Timed by the caller with events on `stream`, it gives the device's plain-integer
- * issue rate under the clocks of the moment.  Asynchronous.
+ * mode 3: 8 recurrence cells on uint32 per round, counted as 2 instructions each; mode 4: the
+ * same cells in the form x = max(x + c, y), issued as one fused add-max instruction each (still
+ * counted as 2).  Timed by the caller with events on `stream`, it gives the device's
+ * plain-integer issue rate under the clocks of the moment.  Asynchronous.
  */
 int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t mode, int32_t blocks,
                             int32_t iters, int64_t *h_ops);

@@ -86,11 +86,12 @@ typedef struct {
     const int32_t *m_list;                /* ascending                            */
     int32_t m_rule;                       /* 0: m divides Bp; 1: any m <= Bp      */
     int32_t partition_mode;               /* 0: balanced; 1: all compositions     */
-    int32_t sched_mask;                   /* bit 0: GPipe, bit 1: 1F1B (Dapple)   */
+    int32_t sched_mask;                   /* bit 0: GPipe, bit 1: 1F1B (Dapple),
+                                             bit 2: 1F1B without gradient synchronisation */
 } orc_space;
 
 typedef struct {
-    int32_t mp, pp, dp, m, sched;         /* sched 0: GPipe, 1: 1F1B              */
+    int32_t mp, pp, dp, m, sched;         /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B */
     int32_t bounds[ORC_MAX_PP + 1];       /* c_0 .. c_pp                          */
 } orc_candidate;
 
@@ -211,7 +212,7 @@ static int64_t beta_of(const orc_table *T, int loc) { return loc ? T->beta_inter
 /*   pp ascending over powers of two <= min(pp_max, L) with mp*pp | N, dp | B; */
 /*   m ascending over the valid entries of m_list;                             */
 /*   stage partition in lexicographic order of (c_1..c_{pp-1});                */
-/*   schedule: GPipe, then 1F1B.                                               */
+/*   schedule: GPipe, then 1F1B, then asynchronous 1F1B.                       */
 /* The paper's own grid (Sec. 5) walks mp and pp over powers of two and takes  */
 /* dp = GPUs/mp/pp, dropping the invalid combinations.                         */
 
@@ -259,7 +260,7 @@ static int64_t walk_space(const orc_table *T, const orc_space *S, orc_visit_fn v
                 else
                     for (int j = 1; j < pp; ++j) x.bounds[j] = j;
                 do {
-                    for (int sc = 0; sc < 2; ++sc) {
+                    for (int sc = 0; sc < 3; ++sc) {
                         if (!(S->sched_mask & (1 << sc))) continue;
                         x.sched = sc;
                         if (visit && visit(ctx, index, &x)) return index + 1;
@@ -358,7 +359,7 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
 
     if (pp < 1 || pp > ORC_MAX_PP || mp < 1 || dp < 1 || m < 1 ||
         (int64_t)mp * pp * dp != T->n_devices || T->global_batch % dp != 0 ||
-        x->bounds[0] != 0 || x->bounds[pp] != L || (x->sched != 0 && x->sched != 1) ||
+        x->bounds[0] != 0 || x->bounds[pp] != L || x->sched < 0 || x->sched > 2 ||
         (T->n_jitter > 0 && (T->jitter_stages < pp || !T->jitter_fwd_ns || !T->jitter_bwd_ns))) {
         e = ORC_E_ARG; goto fail;
     }
@@ -406,7 +407,8 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
         if (x->sched == 0) {                      /* GPipe: all forwards, then all backwards */
             for (int j = 0; j < m; ++j) { o[k].is_bwd = 0; o[k++].mb = j; }
             for (int j = 0; j < m; ++j) { o[k].is_bwd = 1; o[k++].mb = j; }
-        } else {                                  /* 1F1B (Dapple): warm-up, then one-B-one-F */
+        } else {                                  /* 1F1B (Dapple): warm-up, then one-B-one-F;
+                                                     the asynchronous variant keeps this order */
             int w = pp - d < m ? pp - d : m;
             int nf = 0, nb = 0;
             for (; nf < w; ++nf) { o[k].is_bwd = 0; o[k++].mb = nf; }
@@ -498,6 +500,12 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                     for (int64_t i = 0; i < src->n; ++i)
                         if ((e = list_push(dst, src->ev[i])) != ORC_OK) goto fail;
                     if (dp == 1) continue;
+                    /* Asynchronous pipeline parallelism (the paper's discussion of new
+                     * algorithms in "Related Work And Discussion": the pipeline schedule
+                     * is built in the same way, only without the global synchronisation
+                     * event, usually an all-reduce): every replica updates its own
+                     * weights, so no gradient all-reduce event is appended. */
+                    if (x->sched == 2) continue;
                     /* gradient all-reduce events: the stage's gradients, in the
                      * order the backward pass produces them (last layer first),
                      * cut into buckets; each bucket is a ring all-reduce over

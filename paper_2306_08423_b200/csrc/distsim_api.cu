@@ -616,7 +616,7 @@ int distsim_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32b
 int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t mode, int32_t blocks, int32_t iters, int64_t *h_ops)
 {
     if (!ctx) return DISTSIM_E_ARG;
-    if (!h_ops || blocks < 1 || iters < 1 || mode < 0 || mode > 3) return fail(ctx, DISTSIM_E_ARG, "bad probe arguments");
+    if (!h_ops || blocks < 1 || iters < 1 || mode < 0 || mode > 4) return fail(ctx, DISTSIM_E_ARG, "bad probe arguments");
     if (int rc = set_device(ctx)) return rc;
     *h_ops = launch_int_issue_probe(static_cast<cudaStream_t>(stream), mode, blocks, iters,
                                     ctx->d_result.as<int64_t>() + 4, &ctx->launches);

@@ -7,6 +7,8 @@
 //   mode 2  32-bit compare + select pairs               (16 instructions per round and thread)
 //   mode 3  recurrence cells x = max(x, y) + c on uint32 (8 cells per round and thread, counted
 //           as 2 instructions each)
+//   mode 4  recurrence cells x = max(x + c, y) on uint32 with the fused add-max instruction
+//           (8 cells per round and thread, counted as 2 instructions each, as in mode 3)
 #include "engine.h"
 
 namespace distsim {
@@ -41,6 +43,8 @@ __global__ void __launch_bounds__(256) int_issue_probe_kernel(int iters, int64_t
                 } else if (kMode == 3) {
                     const uint32_t mx = x[k] > y[k] ? x[k] : y[k];
                     x[k] = mx + (uint32_t)c[k];
+                } else if (kMode == 4) {
+                    x[k] = __viaddmax_u32(x[k], (uint32_t)c[k], y[k]);
                 } else {
                     asm volatile("{ .reg .pred p; setp.gt.u32 p, %0, %1; selp.u32 %0, %0, %1, p; }" : "+r"(x[k]) : "r"(y[k]));
                     asm volatile("{ .reg .pred p; setp.lt.u32 p, %0, %1; selp.u32 %0, %1, %0, p; }" : "+r"(y[k]) : "r"(x[k]));
@@ -62,9 +66,10 @@ int64_t launch_int_issue_probe(cudaStream_t s, int mode, int blocks, int iters, 
     if (mode == 1) int_issue_probe_kernel<1><<<blocks, 256, 0, s>>>(iters, sink);
     else if (mode == 2) int_issue_probe_kernel<2><<<blocks, 256, 0, s>>>(iters, sink);
     else if (mode == 3) int_issue_probe_kernel<3><<<blocks, 256, 0, s>>>(iters, sink);
+    else if (mode == 4) int_issue_probe_kernel<4><<<blocks, 256, 0, s>>>(iters, sink);
     else int_issue_probe_kernel<0><<<blocks, 256, 0, s>>>(iters, sink);
     ++*launches;
-    const int64_t per_round = mode == 1 ? kChains * 6 : kChains * 2;   // modes 0, 2: 16 = 8 x 2; mode 3: 8 x 2
+    const int64_t per_round = mode == 1 ? kChains * 6 : kChains * 2;   // modes 0, 2: 16 = 8 x 2; modes 3, 4: 8 x 2
     return (int64_t)blocks * 256 * iters * per_round;
 }
 

@@ -61,7 +61,7 @@ class SearchSpace:
     m_list: np.ndarray                      # int32, ascending
     m_rule: int = M_RULE_DIVIDES
     partition_mode: int = PARTITION_BALANCED
-    sched_mask: int = 3                     # bit 0 GPipe, bit 1 1F1B
+    sched_mask: int = 3                     # bit 0 GPipe, bit 1 1F1B, bit 2 asynchronous 1F1B
 
     def __post_init__(self):
         self.m_list = np.ascontiguousarray(self.m_list, dtype=np.int32)
@@ -154,7 +154,7 @@ def space_shape(table, space):
     """Rows of the search space for reporting: a list of (mp, pp, dp, [valid m], partitions,
     schedules).  Pure counting; candidates = sum(len(ms) * partitions * schedules)."""
     rows = []
-    n_sched = bin(space.sched_mask & 3).count("1")
+    n_sched = bin(space.sched_mask & 7).count("1")
     for mp in _pow2_upto(space.mp_max):
         for pp in _pow2_upto(min(space.pp_max, table.n_layers)):
             if table.n_devices % (mp * pp):
@@ -304,11 +304,11 @@ CONFIGS = {0: config0, 1: config1, 2: config2, 3: config3, 4: config4}
 def random_small(seed: int, *, n_devices=8, gpus_per_node=4, n_layers=6, global_batch=16,
                  seq=64, hidden=32, mp_max=4, pp_max=4, m_list=(1, 2, 3, 4, 8),
                  m_rule=M_RULE_CEIL, partition_mode=PARTITION_ALL, moe=True,
-                 dp_bucket_bytes=3000, dp_overlap=1, lo=50, hi=5000) -> Workload:
+                 dp_bucket_bytes=3000, dp_overlap=1, lo=50, hi=5000, sched_mask=3) -> Workload:
     """Small irregular workload for element-by-element parity tests."""
     rng = SplitMix64(seed)
     space = SearchSpace(mp_max=mp_max, pp_max=pp_max, m_list=list(m_list), m_rule=m_rule,
-                        partition_mode=partition_mode)
+                        partition_mode=partition_mode, sched_mask=sched_mask)
     f1 = [rng.randint(lo, hi) for _ in range(n_layers)]
     u = [rng.randint(0, hi // 4) for _ in range(n_layers)]
     expert = np.array([(rng.next() & 1) if moe else 0 for _ in range(n_layers)], dtype=np.uint8)

@@ -112,7 +112,7 @@ def longest_path_timeline(table, cand):
                 preds[first_of_op[(d, "B", j)]].append(last_of_op[(d, "F", j)])
     # gradient buckets on a separate lane
     buckets = {d: [] for d in range(pp)}
-    if dp > 1:
+    if dp > 1 and cand.sched != 2:       # the asynchronous schedule has no gradient all-reduce
         a, be = ab(dp_inter)
         for d in range(pp):
             stream = [(l, ceil_div(int(T.grad_bytes[l]), mp)) for l in range(c[d + 1] - 1, c[d] - 1, -1)]

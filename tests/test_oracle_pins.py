@@ -205,6 +205,39 @@ def test_brute_force_longest_path(w):
             assert got == lanes[d], (c, d)
 
 
+# asynchronous 1F1B: the 1F1B order without the gradient all-reduce events
+@pytest.mark.parametrize("seed", range(20, 26))
+def test_async_1f1b_is_1f1b_without_gradient_allreduce(seed):
+    w = W.random_small(seed, n_devices=8, gpus_per_node=4, n_layers=4, global_batch=8, mp_max=2,
+                       pp_max=4, m_list=(1, 2, 3, 5), dp_overlap=seed % 2,
+                       dp_bucket_bytes=0 if seed % 3 == 2 else 700, sched_mask=7)
+    n = oracle.count(w.table, w.space)
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(n))
+    assert [c.sched for c in cands[:6]] == [0, 1, 2, 0, 1, 2]          # the schedule varies fastest
+    seen_dp = False
+    for i in range(0, n, 3):
+        sync, asyn = cands[i + 1], cands[i + 2]
+        assert (sync.sched, asyn.sched) == (1, 2) and sync.bounds == asyn.bounds and sync.m == asyn.m
+        r1 = oracle.simulate(w.table, sync, replicate=True)
+        r2 = oracle.simulate(w.table, asyn, replicate=True)
+        ends = []
+        for dev in range(w.table.n_devices):
+            a = r1.records[r1.offsets[dev]:r1.offsets[dev + 1]]
+            b = r2.records[r2.offsets[dev]:r2.offsets[dev + 1]]
+            main = a[a[:, 0] != 8]
+            assert (b == main).all()                                   # identical main lanes, no buckets
+            assert r2.busy_ns[dev] == int((main[:, 4] - main[:, 3]).sum())
+            ends.append(int(main[:, 4].max()))
+        assert r2.batch_ns == max(ends) <= r1.batch_ns
+        if sync.dp == 1:
+            assert r2.batch_ns == r1.batch_ns
+        else:
+            seen_dp = True
+        batch, lanes = longest_path_timeline(w.table, asyn)            # independent DAG without all-reduce nodes
+        assert batch == r2.batch_ns
+    assert seen_dp
+
+
 # per-micro-batch jitter
 def _jittered(seed, **kw):
     w = W.random_small(seed, n_devices=8, gpus_per_node=4, n_layers=4, global_batch=8, mp_max=2,
