@@ -134,8 +134,11 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *h_tabl
  * dp | global_batch; m ascending over the valid entries of m_list (m_rule 0: m
  * divides Bp = global_batch/dp; 1: any m <= Bp, micro-batch size ceil(Bp/m));
  * stage partition (partition_mode 0: the balanced one, c_j = floor(j L / pp);
- * 1: every composition, lexicographic in (c_1..c_{pp-1})); schedule GPipe then
- * 1F1B as enabled in sched_mask (bit 0 GPipe, bit 1 1F1B/Dapple).
+ * 1: every composition, lexicographic in (c_1..c_{pp-1})); schedule GPipe, 1F1B,
+ * asynchronous 1F1B as enabled in sched_mask (bit 0 GPipe, bit 1 1F1B/Dapple, bit 2
+ * asynchronous 1F1B: the 1F1B item order without gradient all-reduce events - the paper's
+ * discussion of new algorithms reads an asynchronous pipeline as the same schedule minus the
+ * global synchronisation event).
  * Candidates are never materialised: the device decodes them from the index.
  * Fails with DISTSIM_E_ARG if a needed class (mp, b) is not in the table, with
  * DISTSIM_E_OVERFLOW if the count does not fit 62 bits.  *n_candidates receives
@@ -152,7 +155,7 @@ typedef struct {
 int distsim_set_space(distsim_ctx *ctx, const distsim_space *h_space, int64_t *n_candidates);
 
 typedef struct {
-    int32_t mp, pp, dp, m, sched;   /* sched 0: GPipe, 1: 1F1B                     */
+    int32_t mp, pp, dp, m, sched;   /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B */
     int32_t micro_batch_size;       /* b = ceil(Bp / m)                            */
     int32_t class_index;            /* row of the event table                      */
     int32_t bounds[DISTSIM_MAX_PP + 1];

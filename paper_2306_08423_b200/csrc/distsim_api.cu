@@ -307,7 +307,7 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     if (!ctx->table_loaded) return fail(ctx, DISTSIM_E_STATE, "no event table loaded");
     if (sp->mp_max < 1 || sp->pp_max < 1 || sp->n_m < 1 || !sp->m_list) return fail(ctx, DISTSIM_E_ARG, "empty space");
     if (sp->pp_max > DISTSIM_MAX_PP) return fail(ctx, DISTSIM_E_ARG, "pp_max too large");
-    if ((sp->sched_mask & 3) == 0 || (sp->sched_mask & ~3)) return fail(ctx, DISTSIM_E_ARG, "bad sched_mask");
+    if ((sp->sched_mask & 7) == 0 || (sp->sched_mask & ~7)) return fail(ctx, DISTSIM_E_ARG, "bad sched_mask");
     if (sp->m_rule < 0 || sp->m_rule > 1 || sp->partition_mode < 0 || sp->partition_mode > 1)
         return fail(ctx, DISTSIM_E_ARG, "bad m_rule or partition_mode");
     for (int i = 0; i < sp->n_m; ++i) {
@@ -341,8 +341,9 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     std::vector<Entry> entries;
     int64_t total = 0, op_words = 0;
     long double tb = 0;
-    const int n_sched = (sp->sched_mask == 3) ? 2 : 1;
-    const int sched0 = (sp->sched_mask & 1) ? 0 : 1;
+    int n_sched = 0, sched_list = 0;
+    for (int id = 0; id < 3; ++id)
+        if (sp->sched_mask & (1 << id)) sched_list |= id << (2 * n_sched++);
     long double fg_max = 0;                       // largest per-class sum of layer times
     for (int k = 0; k < tc.n_classes; ++k) {
         long double s = 0;
@@ -363,7 +364,7 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
             Row r{};
             r.mp = (int32_t)mp; r.pp = (int32_t)pp; r.dp = (int32_t)dp; r.log2_mp = floor_log2(mp);
             r.entry0 = (int32_t)entries.size(); r.n_entries = 0;
-            r.n_sched = n_sched; r.sched0 = sched0;
+            r.n_sched = n_sched; r.sched_list = sched_list;
             r.p2p_period = mp >= tc.gpus_per_node ? 1 : (int32_t)(tc.gpus_per_node / mp);
             r.n_part = sp->partition_mode == 0 ? 1 : binom[(size_t)(L - 1) * bk + (pp - 1)];
             for (int i = 0; i < sp->n_m; ++i) {
@@ -464,7 +465,7 @@ int distsim_decode(distsim_ctx *ctx, int64_t index, distsim_candidate *out)
     const Entry &en = ctx->entries[row.entry0 + e];
     memset(out, 0, sizeof *out);
     out->mp = row.mp; out->pp = row.pp; out->dp = row.dp; out->m = en.m;
-    out->sched = row.sched0 + (int32_t)(rem % row.n_sched);
+    out->sched = row_sched(row, (int)(rem % row.n_sched));
     out->micro_batch_size = en.b; out->class_index = en.cls;
     const int L = ctx->tc.n_layers, pp = row.pp, bk = ctx->sc.binom_k;
     out->bounds[0] = 0; out->bounds[pp] = L;

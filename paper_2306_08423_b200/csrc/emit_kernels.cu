@@ -72,7 +72,7 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
             const int64_t rf = per_dir + (d < row.pp - 1 ? 1 : 0);
             const int64_t rb = per_dir + (d > 0 ? 1 : 0);
             int64_t kb = 0;
-            if (row.dp > 1) {
+            if (row.dp > 1 && cc.sched != 2) {              // no buckets in the asynchronous schedule
                 const int64_t *nbt = v.nb + row.row_tab_off, *tpt = v.tp + row.row_tab_off;
                 kb = nbt[(int64_t)e * L1 + a] + (tpt[(int64_t)e * L1 + a] > 0 ? 1 : 0);
             }

@@ -51,10 +51,13 @@ struct Row {
     int64_t row_tab_off;  // offset (words) of this row's NB / TP tables
     int32_t mp, pp, dp, log2_mp;
     int32_t n_entries, entry0;
-    int32_t n_sched, sched0;
+    int32_t n_sched, sched_list;   // enabled schedules in canonical order, two bits each (see row_sched)
     int32_t p2p_period;   // boundary d|d+1 is inter-node iff ((d+1) & (p2p_period-1)) == 0
     int32_t pad;
 };
+
+// Schedule id (0 GPipe, 1 1F1B, 2 asynchronous 1F1B) of position sc among a row's schedules.
+__host__ __device__ inline int row_sched(const Row &row, int sc) { return (row.sched_list >> (2 * sc)) & 3; }
 
 struct Entry {
     int32_t m, b, cls, row;

@@ -2,7 +2,7 @@
 // pp <= 16.
 //
 // A thread owns one stage partition of the row and walks the row's entries (micro-batch
-// counts) and both schedules with it, so the partition is decoded once and the stage costs once
+// counts) and schedules with it, so the partition is decoded once and the stage costs once
 // per entry.  All per-stage state of the pipeline recurrence - forward/backward item cost,
 // device-free time, latest forward end - lives in registers (the stage loops are fully
 // unrolled, pp is a template parameter), so a recurrence cell is exactly one max and one add
@@ -399,7 +399,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
     const int lp = v.tc.lp;
     const int L1 = v.tc.n_layers + 1;
     const ThreadKernelSmem plan = thread_kernel_smem(row.n_entries, lp, v.tab_words, v.dt != nullptr);
-    const int dp = row.dp, n_sched = row.n_sched, sched0 = row.sched0, period = row.p2p_period;
+    const int dp = row.dp, n_sched = row.n_sched, sched_list = row.sched_list, period = row.p2p_period;
     const int64_t t_full = row.t_full;
 
     // ---- stage the row's prefix rows (and bucket tables when no per-entry table exists) ----
@@ -522,29 +522,48 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
             a = ee; pfa = pfe; pba = pbe;
         }
 
-        // ---- both schedules -----------------------------------------------------------------
+        // ---- the row's schedules -------------------------------------------------------------
         const int64_t local0 = (int64_t)e * per_entry + part * n_sched;
-        int64_t res[2] = {0, 0};
+        int64_t res[3] = {0, 0, 0};
+        int64_t main_only = -1;            // batch time of the 1F1B main lanes alone, once known
 #pragma unroll 1
         for (int sc = 0; sc < n_sched; ++sc) {
             const int64_t local = local0 + sc;
             if (local < lo || local >= hi) continue;
-            T free_at[PP];
-            if (sched0 + sc == 0) {
-                if (kJit || !rel) run_gpipe<PP, T, kJit>(st, m, free_at, jt);
-                else run_gpipe_rel<PP, T>(st, m, free_at);
-            }
-            else if (kJit || !rel || m < PP) run_1f1b<PP, T, kJit>(st, m, free_at, jt);
-            else run_1f1b_rel<PP, T>(st, m, free_at);
-            T batch = 0;
+            const int id = (sched_list >> (2 * sc)) & 3;
+            // the asynchronous schedule is the 1F1B main lane without the gradient buckets
+            const bool with_buckets = id != 2;
+            if (id == 2 && main_only >= 0) {
+                res[sc] = main_only;
+            } else {
+                T free_at[PP];
+                if (id == 0) {
+                    if (kJit || !rel) run_gpipe<PP, T, kJit>(st, m, free_at, jt);
+                    else run_gpipe_rel<PP, T>(st, m, free_at);
+                } else {
+                    if (kJit || !rel || m < PP) run_1f1b<PP, T, kJit>(st, m, free_at, jt);
+                    else run_1f1b_rel<PP, T>(st, m, free_at);
+                }
+                T batch = 0;
+                if (with_buckets) {
 #pragma unroll
-            for (int d = 0; d < PP; ++d) batch = vmax(batch, (T)(free_at[d] + xs[d][threadIdx.x]));
-            res[sc] = (int64_t)batch;
+                    for (int d = 0; d < PP; ++d) batch = vmax(batch, (T)(free_at[d] + xs[d][threadIdx.x]));
+                }
+                if (id == 2 || (id == 1 && sc + 1 < n_sched)) {      // an asynchronous twin follows (or this is it)
+                    T plain = 0;
+#pragma unroll
+                    for (int d = 0; d < PP; ++d) plain = vmax(plain, free_at[d]);
+                    main_only = (int64_t)plain;
+                    if (id == 2) batch = plain;
+                }
+                res[sc] = (int64_t)batch;
+            }
             if (kBusy) {
                 int64_t *bo = busy_out + (row.offset + local - first) * v.sc.pp_max;
 #pragma unroll
                 for (int d = 0; d < PP; ++d)
-                    bo[d] = (int64_t)m * ((int64_t)st.fop[d] + (int64_t)st.bop[d]) + (int64_t)xs[d][threadIdx.x] +
+                    bo[d] = (int64_t)m * ((int64_t)st.fop[d] + (int64_t)st.bop[d]) +
+                            (with_buckets ? (int64_t)xs[d][threadIdx.x] : 0) +
                             (kJit ? __ldg(&v.jsum[(int64_t)(row.entry0 + e) * DISTSIM_MAX_PP + d]) : 0);
                 for (int d = PP; d < v.sc.pp_max; ++d) bo[d] = 0;
             }

@@ -59,7 +59,7 @@ __device__ __forceinline__ void partition_bounds(const DeviceView &v, int pp, in
 
 struct CandidateCoords {
     int entry;           // global entry index
-    int sched;           // 0 GPipe, 1 1F1B
+    int sched;           // 0 GPipe, 1 1F1B, 2 asynchronous 1F1B (1F1B order, no gradient all-reduce)
     int64_t part_rank;
 };
 
@@ -74,14 +74,14 @@ __device__ __forceinline__ CandidateCoords split_local(const Row &row, int64_t l
         const uint32_t rem = l32 - e * per_entry;
         cc.entry = row.entry0 + (int)e;
         cc.part_rank = rem / (uint32_t)row.n_sched;
-        cc.sched = row.sched0 + (int)(rem - (uint32_t)cc.part_rank * (uint32_t)row.n_sched);
+        cc.sched = row_sched(row, (int)(rem - (uint32_t)cc.part_rank * (uint32_t)row.n_sched));
     } else {
         const int64_t per_entry = row.n_part * row.n_sched;
         const int64_t e = local / per_entry;
         const int64_t rem = local - e * per_entry;
         cc.entry = row.entry0 + (int)e;
         cc.part_rank = rem / row.n_sched;
-        cc.sched = row.sched0 + (int)(rem - cc.part_rank * row.n_sched);
+        cc.sched = row_sched(row, (int)(rem - cc.part_rank * row.n_sched));
     }
     return cc;
 }
@@ -237,7 +237,9 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
 #pragma unroll
     for (int k = 0; k < S; ++k) {
         R.main_end[k] = free_at[k];
-        R.dp_end[k] = bucket_lane_end(v, row, pb, nbt, tpt, R.a[k], R.e[k], R.last_b_start[k], R.main_end[k]);
+        // the asynchronous schedule has no gradient all-reduce events
+        R.dp_end[k] = sched == 2 ? R.main_end[k]
+                                 : bucket_lane_end(v, row, pb, nbt, tpt, R.a[k], R.e[k], R.last_b_start[k], R.main_end[k]);
         const int64_t extra = R.dp_end[k] - R.main_end[k];
         R.busy[k] = (int64_t)m * (R.fop[k] + R.bop[k]) + (extra > 0 ? extra : 0) +
                     (kJit ? __ldg(&v.jsum[(int64_t)entry_index * DISTSIM_MAX_PP + d0 + k]) : 0);

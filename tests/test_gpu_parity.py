@@ -127,6 +127,40 @@ def test_random_small_full_parity(E, ctx, seed):
     check_emission(E, ctx, w, pick)
 
 
+@pytest.mark.parametrize("sched_mask", [7, 4, 5, 6])
+def test_asynchronous_1f1b_schedule(E, ctx, sched_mask):
+    """Spaces with the asynchronous schedule (bit 2) alone and beside the others: every candidate
+    of a small space (lock-step kernel), sampled candidates of a space with enough partitions for
+    the one-partition-per-thread kernel, emitted timelines without gradient buckets."""
+    w = W.random_small(300 + sched_mask, dp_overlap=sched_mask % 2, sched_mask=sched_mask)
+    n = load(E, ctx, w)
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    assert (batch.cpu().numpy() == ob).all() and (sb.cpu().numpy() == obusy).all()
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(n))
+    for i in range(0, n, max(1, n // 50)):
+        assert E.distsim_decode(ctx, i)["sched"] == cands[i].sched
+    pick = [i for i, c in enumerate(cands) if c.sched == 2 and c.dp > 1][:: max(1, n // 60)][:16]
+    assert pick
+    check_emission(E, ctx, w, pick + [0, n - 1])
+    # 50 388 partitions at pp = 8: the thread kernel, 32-bit and relative-frame paths included
+    w = W.random_small(310 + sched_mask, n_devices=16, gpus_per_node=4, n_layers=20, global_batch=64,
+                       mp_max=2, pp_max=8, m_list=(1, 3, 8, 16, 32), sched_mask=sched_mask,
+                       partition_mode=W.PARTITION_ALL)
+    n = load(E, ctx, w)
+    batch, sb = eval_all(E, ctx, n)
+    rng = np.random.default_rng(sched_mask)
+    idx = np.unique(np.concatenate([rng.integers(0, n, 3000), [0, n - 1]]))
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, idx, THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    sel = torch.from_numpy(idx).cuda()
+    assert (batch[sel].cpu().numpy() == ob).all()
+    assert (sb[sel].cpu().numpy() == obusy).all()
+    bi, bt = E.distsim_argmin(ctx, batch, 0, n)
+    assert oracle.eval_indices(w.table, w.space, np.array([bi]))[0][0] == bt == int(batch.min().item())
+
+
 def test_ranges_straddle_rows_and_empty(E, ctx):
     w = W.random_small(7, partition_mode=W.PARTITION_ALL)
     n = load(E, ctx, w)
