@@ -174,6 +174,18 @@ void flush_thread_any(int log2pp, bool narrow, cudaStream_t s, const DeviceView 
 
 int ilog2(int v) { int b = 0; while ((1 << (b + 1)) <= v) ++b; return b; }
 
+// The shared-memory budget of the kernel instance that evaluates rows of this pp and arithmetic width.
+int thread_budget_words(int pp, bool narrow, bool jitter)
+{
+    switch (ilog2(pp)) {
+    case 0: return narrow ? thread_kernel_budget_words<1, uint32_t>(jitter) : thread_kernel_budget_words<1, int64_t>(jitter);
+    case 1: return narrow ? thread_kernel_budget_words<2, uint32_t>(jitter) : thread_kernel_budget_words<2, int64_t>(jitter);
+    case 2: return narrow ? thread_kernel_budget_words<4, uint32_t>(jitter) : thread_kernel_budget_words<4, int64_t>(jitter);
+    case 3: return narrow ? thread_kernel_budget_words<8, uint32_t>(jitter) : thread_kernel_budget_words<8, int64_t>(jitter);
+    default: return narrow ? thread_kernel_budget_words<16, uint32_t>(jitter) : thread_kernel_budget_words<16, int64_t>(jitter);
+    }
+}
+
 }  // namespace
 
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
@@ -249,7 +261,9 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
                 w.row = r; w.e_begin = r0; w.e_end = r1; w.ept = ept; w.p_lo = p_lo; w.p_hi = p_hi;
                 w.lo = lo_r; w.hi = hi_r; w.block_begin = p.blocks; w.nx = (int)nx;
                 p.blocks += (int)(nx * ny);
-                const int words = thread_kernel_smem(row.n_entries, v.tc.lp, v.tab_words, v.dt != nullptr).words;
+                const int binom_words = v.sc.partition_mode ? v.tc.n_layers * v.sc.binom_k : 0;
+                const int words = thread_kernel_smem(row.n_entries, v.tc.lp, v.tab_words, v.dt != nullptr, binom_words,
+                                                     thread_budget_words(row.pp, narrow, v.tc.n_jitter > 0)).words;
                 if (words > p.smem_words) p.smem_words = words;
             } else {
                 add_lockstep(r, lo_r, hi_r);

@@ -344,28 +344,60 @@ DS_UNROLL(DS_UNROLL_MAIN)
 }
 
 // Shared-memory plan of a block (offsets in int64 words from the dynamic shared base): the
-// prefix rows of every entry of the row, and the row's two bucket tables only when there is no
-// per-entry bucket-lane table to look the result up in - each as far as it fits.
+// prefix rows of every entry of the row; then, when per-entry bucket-lane tables exist, the
+// binomial table of the unranking and the bucket-lane tables of the row's last entries (as many
+// as the budget allows: the entries with the most micro-batches come last); otherwise the row's
+// two bucket tables - each as far as it fits.
 struct ThreadKernelSmem {
     int32_t n_entries_staged;   // 0: read prefix rows from global
     int32_t tables_staged;      // 1: NB / TP tables of the row are in shared memory
-    int32_t off_etb, off_nb, off_tp;
+    int32_t n_dt_staged;        // bucket-lane tables of the row's last n_dt_staged entries are in shared memory
+    int32_t binom_staged;       // 1: the binomial table is in shared memory
+    int32_t off_etb, off_nb, off_tp, off_dt, off_binom;
     int32_t words;              // dynamic shared memory needed, in int64 words
 };
-__host__ __device__ inline ThreadKernelSmem thread_kernel_smem(int n_entries, int lp, int tab_words, bool have_dt)
+// Dynamic shared memory (int64 words) a block may use without lowering the number of resident
+// blocks the kernel is compiled for: an SM's 228 KB, less 1 KB per block, less the kernel's
+// static arrays.
+template <int PP, typename T>
+__host__ __device__ constexpr int thread_kernel_budget_words(bool jitter)
+{
+    const int per_block = 233472 / thread_kernel_min_blocks<PP, T>() - 1024;
+    const int fixed = PP * kThreadBlock * (int)sizeof(T) + (PP + 1) * kThreadBlock * 2 + 16 * 24 + 256 +
+                      (jitter ? 2 * 64 * PP * (int)sizeof(T) : 0);
+    return (per_block - fixed) / 8 > 0 ? (per_block - fixed) / 8 : 0;
+}
+__host__ __device__ inline ThreadKernelSmem thread_kernel_smem(int n_entries, int lp, int tab_words, bool have_dt,
+                                                               int binom_words, int budget_words)
 {
     ThreadKernelSmem plan{};
     int words = 0;
-    if (n_entries * lp * 2 <= 8192) {
+    if (n_entries * lp * 2 <= 8192 && n_entries * lp * 2 <= budget_words) {
         plan.n_entries_staged = n_entries;
         plan.off_etb = n_entries * lp;
         words = n_entries * lp * 2;
     }
-    if (!have_dt && words + 2 * tab_words <= 12288) {
-        plan.tables_staged = 1;
-        plan.off_nb = words;
-        plan.off_tp = words + tab_words;
-        words += 2 * tab_words;
+    if (!have_dt) {
+        if (words + 2 * tab_words <= 12288 && words + 2 * tab_words <= budget_words) {
+            plan.tables_staged = 1;
+            plan.off_nb = words;
+            plan.off_tp = words + tab_words;
+            words += 2 * tab_words;
+        }
+    } else {
+        // bulk copies move multiples of 16 bytes: an odd-sized binomial table stays in global memory
+        if (binom_words > 0 && !(binom_words & 1) && words + binom_words <= budget_words) {
+            plan.binom_staged = 1;
+            plan.off_binom = words;
+            words += binom_words;
+        }
+        int k = tab_words > 0 ? (budget_words - words) / tab_words : 0;
+        if (k > n_entries) k = n_entries;
+        if (k > 0 && (int64_t)k * tab_words * 8 < (1 << 20)) {       // one bulk copy, one barrier transaction count
+            plan.n_dt_staged = k;
+            plan.off_dt = words;
+            words += k * tab_words;
+        }
     }
     plan.words = words;
     return plan;
@@ -398,7 +430,9 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
     const Row &row = v.rows[row_index];
     const int lp = v.tc.lp;
     const int L1 = v.tc.n_layers + 1;
-    const ThreadKernelSmem plan = thread_kernel_smem(row.n_entries, lp, v.tab_words, v.dt != nullptr);
+    const int binom_words = v.sc.partition_mode ? v.tc.n_layers * v.sc.binom_k : 0;
+    const ThreadKernelSmem plan = thread_kernel_smem(row.n_entries, lp, v.tab_words, v.dt != nullptr, binom_words,
+                                                     thread_kernel_budget_words<PP, T>(kJit));
     const int dp = row.dp, n_sched = row.n_sched, sched_list = row.sched_list, period = row.p2p_period;
     const int64_t t_full = row.t_full;
 
@@ -422,15 +456,24 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
         }
     const JitterTab<PP, T, kJit> jt{jit_f_s, jit_b_s, v.tc.n_jitter - 1};
     bool staged = false;
-    if (plan.n_entries_staged > 0 || plan.tables_staged) {
+    const int dt_first = row.n_entries - plan.n_dt_staged;      // first entry whose bucket-lane table is staged
+    if (plan.n_entries_staged > 0 || plan.tables_staged || plan.n_dt_staged > 0 || plan.binom_staged) {
         const uint32_t pbytes = (uint32_t)(plan.n_entries_staged * lp * sizeof(int64_t));
         const uint32_t tbytes = plan.tables_staged ? (uint32_t)(v.tab_words * sizeof(int64_t)) : 0u;
+        const uint32_t dbytes = (uint32_t)(plan.n_dt_staged * v.tab_words * sizeof(int64_t));
+        const uint32_t bbytes = plan.binom_staged ? (uint32_t)(binom_words * sizeof(int64_t)) : 0u;
+        const int64_t *dt_g = v.dt ? v.dt + (int64_t)(row.entry0 + dt_first) * v.tab_words : nullptr;
+        // with per-entry bucket-lane tables the row's NB / TP tables are not needed here
         const StageCopy cp[kMaxCopies] = {{dsm, etf_g, pbytes}, {dsm + plan.off_etb, etb_g, pbytes},
-                                          {dsm + plan.off_nb, nb_g, tbytes}, {dsm + plan.off_tp, tp_g, tbytes}};
+                                          v.dt ? StageCopy{dsm + plan.off_dt, dt_g, dbytes}
+                                               : StageCopy{dsm + plan.off_nb, nb_g, tbytes},
+                                          v.dt ? StageCopy{dsm + plan.off_binom, v.binom, bbytes}
+                                               : StageCopy{dsm + plan.off_tp, tp_g, tbytes}};
         staged = stage_tables(&bar, cp, v.status);      // contains the block-wide barriers
     } else {
         __syncthreads();
     }
+    const int64_t *binom_p = (staged && plan.binom_staged) ? dsm + plan.off_binom : v.binom;
     const int64_t *etf = (staged && plan.n_entries_staged) ? dsm : etf_g;
     const int64_t *etb = (staged && plan.n_entries_staged) ? dsm + plan.off_etb : etb_g;
     const int64_t *nbt = (staged && plan.tables_staged) ? dsm + plan.off_nb : nb_g;
@@ -453,7 +496,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
         for (int i = 1; i < PP; ++i) {
             ++cur;
             while (true) {
-                const int64_t cnt = __ldg(&v.binom[(int64_t)(v.tc.n_layers - 1 - cur) * v.sc.binom_k + (PP - 1 - i)]);
+                const int64_t cnt = binom_p[(v.tc.n_layers - 1 - cur) * v.sc.binom_k + (PP - 1 - i)];
                 if (r < cnt) break;
                 r -= cnt;
                 ++cur;
@@ -475,7 +518,10 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
             m = en.m; p2p_intra = en.p2p_intra; p2p_inter = en.p2p_inter;
             rel = rel || en.rel_bound < ((int64_t)1 << 32);
         }
-        const int64_t *dte = v.dt ? v.dt + (int64_t)(row.entry0 + e) * v.tab_words : nullptr;
+        const int64_t *dte = nullptr;
+        if (v.dt)
+            dte = (staged && e >= dt_first) ? dsm + plan.off_dt + (e - dt_first) * v.tab_words
+                                            : v.dt + (int64_t)(row.entry0 + e) * v.tab_words;
 
         // ---- stage costs and bucket-lane excess (schedule independent) -------------------
         ThreadState<PP, T> st;
@@ -492,7 +538,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
             int64_t x = 0;
             if (dp > 1) {
                 if (dte) {
-                    const int64_t val = __ldg(&dte[(int64_t)ee * L1 + a]);
+                    const int64_t val = dte[ee * L1 + a];
                     x = v.tc.overlap ? val - bop : val;
                 } else {
                     const int64_t *nbe = nbt + (int64_t)ee * L1;
