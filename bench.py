@@ -470,6 +470,7 @@ def profile_case(name):
     """Small, bounded invocations for profiler captures (no timing, no JSON line):
     eval1  - evaluation of a 2 M-candidate slice of the 64-device workload (a pp = 16 row, m = 16 and 32)
     eval1m128 - the m = 128 entry of the same row (1 M candidates, 4.0e9 cells)
+    eval1m1 - the m = 1 entry of the same row (1 M candidates: unranking and set-up only)
     eval3  - evaluation of the whole 256-device MoE workload (650 k candidates)
     emit4  - emission of 16 of the fastest candidates of the 1024-device workload (~1.9 GB)
     emit1  - emission of the 1024 fastest candidates of the 64-device workload (~1.8 GB)
@@ -479,7 +480,7 @@ def profile_case(name):
     from paper_2306_08423_b200 import engine as E
     torch.cuda.set_device(0)
     ctx = E.Context(0)
-    if name in ("eval1", "eval1m128", "eval3"):
+    if name in ("eval1", "eval1m1", "eval1m128", "eval3"):
         w = W.config1() if name != "eval3" else W.config3()
         E.distsim_load_event_table(ctx, w.table)
         n = E.distsim_set_space(ctx, w.space)
@@ -490,7 +491,7 @@ def profile_case(name):
             off = 0
             for mp, pp, dp, ms, parts, n_sched in W.space_shape(w.table, w.space):
                 if (mp, pp) == (1, 16):
-                    e0, ne = (4, 2) if name == "eval1" else (ms.index(128), 1)
+                    e0, ne = (4, 2) if name == "eval1" else (ms.index(128 if name == "eval1m128" else 1), 1)
                     first, count = off + e0 * parts * n_sched, ne * parts * n_sched
                 off += len(ms) * parts * n_sched
         batch = torch.empty(count, dtype=torch.int64, device="cuda")
@@ -525,7 +526,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-workloads", action="store_true", help="skip the per-workload summary")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
-    ap.add_argument("--profile-case", default=None, help="eval1 | eval1m128 | eval3 | emit1 | emit4 | emit4x128: small run for ncu")
+    ap.add_argument("--profile-case", default=None, help="eval1 | eval1m1 | eval1m128 | eval3 | emit1 | emit4 | emit4x128: small run for ncu")
     args = ap.parse_args()
     if args.profile_case:
         profile_case(args.profile_case)

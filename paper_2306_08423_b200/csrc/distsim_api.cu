@@ -68,8 +68,8 @@ struct distsim_ctx {
     std::vector<int64_t> binom;
     int64_t time_bound = 0;
     int64_t op_words_per_cand = 0;
-    DevBuf d_rows, d_entries, d_etf, d_etb, d_nb, d_tp, d_binom, d_dt;
-    bool have_dt = false;
+    DevBuf d_rows, d_entries, d_etf, d_etb, d_nb, d_tp, d_binom, d_dt, d_pfb32, d_dt32;
+    bool have_dt = false, have_narrow = false;
 
     // scratch
     DevBuf d_status, d_sel, d_result, d_plans, d_op_start, d_totals, d_batch, d_topk;
@@ -87,6 +87,9 @@ struct distsim_ctx {
         v.binom = d_binom.as<int64_t>();
         v.dt = have_dt ? d_dt.as<int64_t>() : nullptr;
         v.tab_words = ((tc.n_layers + 1) * (tc.n_layers + 1) + 1) & ~1;
+        v.tab_words32 = ((tc.n_layers + 1) * (tc.n_layers + 1) + 3) & ~3;
+        v.pfb32 = have_narrow ? d_pfb32.as<uint2>() : nullptr;
+        v.dt32 = have_narrow && have_dt ? d_dt32.as<uint32_t>() : nullptr;
         v.next_grad = d_next_grad.as<int32_t>(); v.pe = d_pe.as<int32_t>();
         v.jsum = tc.n_jitter > 0 ? d_jsum.as<int64_t>() : nullptr;
         v.status = d_status.as<int32_t>();
@@ -316,6 +319,7 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     }
     if (int rc = set_device(ctx)) return rc;
     ctx->space_set = false;
+    ctx->have_narrow = false;
     const TableConst &tc = ctx->tc;
     const int L = tc.n_layers;
     const int64_t N = tc.n_devices, B = tc.global_batch;
@@ -435,6 +439,16 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     if (tc.n_jitter > 0) CU(ctx->d_jsum.reserve(entries.size() * DISTSIM_MAX_PP * sizeof(int64_t)), "alloc jitter sums");
     launch_build_entry_tables(0, ctx->view(), ctx->d_entries.as<Entry>(), ctx->have_dt ? ctx->d_dt.as<int64_t>() : nullptr,
                               tc.n_jitter > 0 ? ctx->d_jsum.as<int64_t>() : nullptr, &ctx->launches);
+    // 32-bit copies for the entries that are evaluated in 32-bit arithmetic
+    ctx->have_narrow = false;
+    {
+        const size_t t32 = (size_t)(((L + 1) * (L + 1) + 3) & ~3);
+        CU(ctx->d_pfb32.reserve(entries.size() * tc.lp * sizeof(uint2)), "alloc 32-bit prefix rows");
+        if (ctx->have_dt) CU(ctx->d_dt32.reserve(entries.size() * t32 * sizeof(uint32_t)), "alloc 32-bit bucket-lane tables");
+        launch_build_narrow_tables(0, ctx->view(), ctx->d_pfb32.as<uint2>(),
+                                   ctx->have_dt ? ctx->d_dt32.as<uint32_t>() : nullptr, &ctx->launches);
+        ctx->have_narrow = true;
+    }
     CU(cudaGetLastError(), "set-up launch");
     // the host copies take the device-filled fields; these copies also wait for set-up
     CU(cudaMemcpy(ctx->rows.data(), ctx->d_rows.p, rows.size() * sizeof(Row), cudaMemcpyDeviceToHost), "rows readback");

@@ -94,7 +94,11 @@ struct DeviceView {
     const int64_t *nb, *tp;          // per row [L+1][L+1]
     const int64_t *dt;               // per entry [L+1][L+1] bucket-lane table (nullptr: not built)
     int32_t tab_words;               // words of one [L+1][L+1] table, rounded up to even
-    int32_t pad_view;
+    int32_t tab_words32;             // 32-bit words of one dt32 table, rounded up to a multiple of 4
+    const uint2 *pfb32;              // [n_entries][lp] (forward, backward) prefix sums of the entries whose
+                                     // time bound is below 2^32 (zeros for the others); nullptr: not built
+    const uint32_t *dt32;            // [n_entries][tab_words32] bucket-lane tables of those entries, negative
+                                     // values stored as 0 (nullptr: not built)
     const int64_t *binom;            // [n_layers][binom_k]
     const int32_t *next_grad;        // [L+1] smallest l' >= l with grad_bytes[l'] > 0 (L if none)
     const int32_t *pe;               // [L+1] number of expert layers before layer l
@@ -111,6 +115,10 @@ void launch_build_prefix(cudaStream_t s, const TableConst &tc, const RawTable &r
                          int64_t *launches);
 void launch_build_bucket_tables(cudaStream_t s, const TableConst &tc, const RawTable &raw,
                                 const Row *rows, int n_rows, int64_t *nb, int64_t *tp,
+                                int64_t *launches);
+// 32-bit copies of the prefix rows and bucket-lane tables for the entries whose time bound is
+// below 2^32 (after launch_build_entry_tables: reads the entries' bounds).  dt32 may be null.
+void launch_build_narrow_tables(cudaStream_t s, const DeviceView &v, uint2 *pfb32, uint32_t *dt32,
                                 int64_t *launches);
 // Per entry: the bucket-lane table (if dt != nullptr) and the time bound of the entry.
 void launch_build_entry_tables(cudaStream_t s, const DeviceView &v, Entry *entries, int64_t *dt,

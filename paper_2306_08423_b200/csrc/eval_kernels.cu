@@ -262,8 +262,11 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
                 w.lo = lo_r; w.hi = hi_r; w.block_begin = p.blocks; w.nx = (int)nx;
                 p.blocks += (int)(nx * ny);
                 const int binom_words = v.sc.partition_mode ? v.tc.n_layers * v.sc.binom_k : 0;
-                const int words = thread_kernel_smem(row.n_entries, v.tc.lp, v.tab_words, v.dt != nullptr, binom_words,
-                                                     thread_budget_words(row.pp, narrow, v.tc.n_jitter > 0)).words;
+                const int budget = thread_budget_words(row.pp, narrow, v.tc.n_jitter > 0);
+                const bool use32 = narrow && v.pfb32 != nullptr && (row.dp == 1 || v.dt32 != nullptr);   // as in the kernel
+                const int words =
+                    use32 ? thread_kernel_smem32(row.n_entries, v.tc.lp, v.tab_words32, v.dt32 != nullptr, binom_words, budget).words
+                          : thread_kernel_smem(row.n_entries, v.tc.lp, v.tab_words, v.dt != nullptr, binom_words, budget).words;
                 if (words > p.smem_words) p.smem_words = words;
             } else {
                 add_lockstep(r, lo_r, hi_r);

@@ -403,6 +403,37 @@ __host__ __device__ inline ThreadKernelSmem thread_kernel_smem(int n_entries, in
     return plan;
 }
 
+// The same plan for a launch in 32-bit arithmetic, which reads the 32-bit copies of the tables:
+// one (forward, backward) prefix row per entry (lp words), the binomial table, and the 32-bit
+// bucket-lane tables (tab_words32 / 2 words each) of the row's last entries.
+__host__ __device__ inline ThreadKernelSmem thread_kernel_smem32(int n_entries, int lp, int tab_words32, bool have_dt,
+                                                                 int binom_words, int budget_words)
+{
+    ThreadKernelSmem plan{};
+    int words = 0;
+    if (n_entries * lp <= 8192 && n_entries * lp <= budget_words) {
+        plan.n_entries_staged = n_entries;
+        words = n_entries * lp;                      // lp is even: the next table stays 16-byte aligned
+    }
+    if (binom_words > 0 && !(binom_words & 1) && words + binom_words <= budget_words) {
+        plan.binom_staged = 1;
+        plan.off_binom = words;
+        words += binom_words;
+    }
+    if (have_dt) {
+        const int tw = tab_words32 / 2;
+        int k = (budget_words - words) / tw;
+        if (k > n_entries) k = n_entries;
+        if (k > 0 && (int64_t)k * tw * 8 < (1 << 20)) {
+            plan.n_dt_staged = k;
+            plan.off_dt = words;
+            words += k * tw;
+        }
+    }
+    plan.words = words;
+    return plan;
+}
+
 // Entry scalars the hot path needs, kept in shared memory for the whole row.
 struct EntryLite { int64_t p2p_intra, p2p_inter; int32_t m, rel_fits32; };
 
@@ -431,8 +462,13 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
     const int lp = v.tc.lp;
     const int L1 = v.tc.n_layers + 1;
     const int binom_words = v.sc.partition_mode ? v.tc.n_layers * v.sc.binom_k : 0;
-    const ThreadKernelSmem plan = thread_kernel_smem(row.n_entries, lp, v.tab_words, v.dt != nullptr, binom_words,
-                                                     thread_kernel_budget_words<PP, T>(kJit));
+    // 32-bit arithmetic reads 32-bit copies of the prefix rows and bucket-lane tables
+    const bool use32 = sizeof(T) == 4 && v.pfb32 != nullptr && (row.dp == 1 || v.dt32 != nullptr);
+    const ThreadKernelSmem plan =
+        use32 ? thread_kernel_smem32(row.n_entries, lp, v.tab_words32, v.dt32 != nullptr, binom_words,
+                                     thread_kernel_budget_words<PP, T>(kJit))
+              : thread_kernel_smem(row.n_entries, lp, v.tab_words, v.dt != nullptr, binom_words,
+                                   thread_kernel_budget_words<PP, T>(kJit));
     const int dp = row.dp, n_sched = row.n_sched, sched_list = row.sched_list, period = row.p2p_period;
     const int64_t t_full = row.t_full;
 
@@ -457,7 +493,17 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
     const JitterTab<PP, T, kJit> jt{jit_f_s, jit_b_s, v.tc.n_jitter - 1};
     bool staged = false;
     const int dt_first = row.n_entries - plan.n_dt_staged;      // first entry whose bucket-lane table is staged
-    if (plan.n_entries_staged > 0 || plan.tables_staged || plan.n_dt_staged > 0 || plan.binom_staged) {
+    if (use32) {
+        const uint32_t pbytes = (uint32_t)(plan.n_entries_staged * lp * sizeof(uint2));
+        const uint32_t bbytes = plan.binom_staged ? (uint32_t)(binom_words * sizeof(int64_t)) : 0u;
+        const uint32_t dbytes = (uint32_t)(plan.n_dt_staged * v.tab_words32 * sizeof(uint32_t));
+        const uint32_t *dt_g = v.dt32 ? v.dt32 + (int64_t)(row.entry0 + dt_first) * v.tab_words32 : nullptr;
+        const StageCopy cp[kMaxCopies] = {{dsm, v.pfb32 + (int64_t)row.entry0 * lp, pbytes},
+                                          {dsm + plan.off_binom, v.binom, bbytes},
+                                          {dsm + plan.off_dt, dt_g, dbytes}, {nullptr, nullptr, 0u}};
+        if (pbytes + bbytes + dbytes > 0) staged = stage_tables(&bar, cp, v.status);
+        else __syncthreads();
+    } else if (plan.n_entries_staged > 0 || plan.tables_staged || plan.n_dt_staged > 0 || plan.binom_staged) {
         const uint32_t pbytes = (uint32_t)(plan.n_entries_staged * lp * sizeof(int64_t));
         const uint32_t tbytes = plan.tables_staged ? (uint32_t)(v.tab_words * sizeof(int64_t)) : 0u;
         const uint32_t dbytes = (uint32_t)(plan.n_dt_staged * v.tab_words * sizeof(int64_t));
@@ -507,8 +553,6 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
 
     const int64_t per_entry = row.n_part * n_sched;
     for (int e = e0; e < e1; ++e) {                     // e: entry index inside the row
-        const int64_t *pf = etf + (int64_t)e * lp;
-        const int64_t *pb = etb + (int64_t)e * lp;
         int m;
         int64_t p2p_intra, p2p_inter;
         bool rel = sizeof(T) == 8;      // the relative frames' shift must fit the arithmetic width as well
@@ -518,54 +562,87 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
             m = en.m; p2p_intra = en.p2p_intra; p2p_inter = en.p2p_inter;
             rel = rel || en.rel_bound < ((int64_t)1 << 32);
         }
-        const int64_t *dte = nullptr;
-        if (v.dt)
-            dte = (staged && e >= dt_first) ? dsm + plan.off_dt + (e - dt_first) * v.tab_words
-                                            : v.dt + (int64_t)(row.entry0 + e) * v.tab_words;
 
         // ---- stage costs and bucket-lane excess (schedule independent) -------------------
         ThreadState<PP, T> st;
-        int a = 0;
-        int64_t pfa = pf[0], pba = pb[0];
+        if (use32) {
+            // everything of this entry fits 32 bits: packed prefix rows, 32-bit table values
+            const uint2 *pr = (staged && plan.n_entries_staged) ? reinterpret_cast<const uint2 *>(dsm) + e * lp
+                                                                : v.pfb32 + (int64_t)(row.entry0 + e) * lp;
+            const uint32_t *d32 = nullptr;
+            if (v.dt32)
+                d32 = (staged && e >= dt_first)
+                          ? reinterpret_cast<const uint32_t *>(dsm + plan.off_dt) + (e - dt_first) * v.tab_words32
+                          : v.dt32 + (int64_t)(row.entry0 + e) * v.tab_words32;
+            const uint32_t p_in = (uint32_t)p2p_intra, p_out = (uint32_t)p2p_inter;
+            uint2 prev = pr[0];
+            int a = 0;
 #pragma unroll
-        for (int d = 0; d < PP; ++d) {
-            const int ee = cs[d + 1][threadIdx.x];
-            const int64_t pfe = pf[ee], pbe = pb[ee];
-            const int64_t send_f = d < PP - 1 ? ((((d + 1) & (period - 1)) == 0) ? p2p_inter : p2p_intra) : 0;
-            const int64_t send_b = d > 0 ? (((d & (period - 1)) == 0) ? p2p_inter : p2p_intra) : 0;
-            const int64_t fop = pfe - pfa + send_f;
-            const int64_t bop = pbe - pba + send_b;
-            int64_t x = 0;
-            if (dp > 1) {
-                if (dte) {
-                    const int64_t val = dte[ee * L1 + a];
-                    x = v.tc.overlap ? val - bop : val;
-                } else {
-                    const int64_t *nbe = nbt + (int64_t)ee * L1;
-                    const int64_t partial = tpt[(int64_t)ee * L1 + a];
-                    const int64_t n_full = nbe[a];
-                    if (!v.tc.overlap) {
-                        x = n_full * t_full + partial;
-                    } else {
-                        int64_t dt = -1;
-                        if (n_full > 0) {
-                            int64_t nb_prev = 0;
-                            for (int l = ee - 1; l >= a; --l) {
-                                const int64_t nb_l = nbe[l];
-                                if (nb_l != nb_prev)
-                                    dt = max64(dt, (pbe - pb[l]) + (n_full - nb_prev) * t_full + partial);
-                                nb_prev = nb_l;
-                            }
-                        }
-                        if (partial > 0) dt = max64(dt, (pbe - pb[__ldg(&v.next_grad[a])]) + partial);
-                        x = dt - bop;
-                    }
+            for (int d = 0; d < PP; ++d) {
+                const int ee = cs[d + 1][threadIdx.x];
+                const uint2 cur = pr[ee];
+                const uint32_t send_f = d < PP - 1 ? ((((d + 1) & (period - 1)) == 0) ? p_out : p_in) : 0u;
+                const uint32_t send_b = d > 0 ? (((d & (period - 1)) == 0) ? p_out : p_in) : 0u;
+                const uint32_t fop = cur.x - prev.x + send_f;
+                const uint32_t bop = cur.y - prev.y + send_b;
+                uint32_t x = 0;
+                if (dp > 1) {
+                    const uint32_t val = d32[ee * L1 + a];
+                    x = v.tc.overlap ? max(val, bop) - bop : val;
                 }
-                if (x < 0) x = 0;
+                st.fop[d] = (T)fop; st.bop[d] = (T)bop;
+                xs[d][threadIdx.x] = (T)x;
+                a = ee; prev = cur;
             }
-            st.fop[d] = (T)fop; st.bop[d] = (T)bop;
-            xs[d][threadIdx.x] = (T)x;
-            a = ee; pfa = pfe; pba = pbe;
+        } else {
+            const int64_t *pf = etf + (int64_t)e * lp;
+            const int64_t *pb = etb + (int64_t)e * lp;
+            const int64_t *dte = nullptr;
+            if (v.dt)
+                dte = (staged && e >= dt_first) ? dsm + plan.off_dt + (e - dt_first) * v.tab_words
+                                                : v.dt + (int64_t)(row.entry0 + e) * v.tab_words;
+            int a = 0;
+            int64_t pfa = pf[0], pba = pb[0];
+#pragma unroll
+            for (int d = 0; d < PP; ++d) {
+                const int ee = cs[d + 1][threadIdx.x];
+                const int64_t pfe = pf[ee], pbe = pb[ee];
+                const int64_t send_f = d < PP - 1 ? ((((d + 1) & (period - 1)) == 0) ? p2p_inter : p2p_intra) : 0;
+                const int64_t send_b = d > 0 ? (((d & (period - 1)) == 0) ? p2p_inter : p2p_intra) : 0;
+                const int64_t fop = pfe - pfa + send_f;
+                const int64_t bop = pbe - pba + send_b;
+                int64_t x = 0;
+                if (dp > 1) {
+                    if (dte) {
+                        const int64_t val = dte[ee * L1 + a];
+                        x = v.tc.overlap ? val - bop : val;
+                    } else {
+                        const int64_t *nbe = nbt + (int64_t)ee * L1;
+                        const int64_t partial = tpt[(int64_t)ee * L1 + a];
+                        const int64_t n_full = nbe[a];
+                        if (!v.tc.overlap) {
+                            x = n_full * t_full + partial;
+                        } else {
+                            int64_t dt = -1;
+                            if (n_full > 0) {
+                                int64_t nb_prev = 0;
+                                for (int l = ee - 1; l >= a; --l) {
+                                    const int64_t nb_l = nbe[l];
+                                    if (nb_l != nb_prev)
+                                        dt = max64(dt, (pbe - pb[l]) + (n_full - nb_prev) * t_full + partial);
+                                    nb_prev = nb_l;
+                                }
+                            }
+                            if (partial > 0) dt = max64(dt, (pbe - pb[__ldg(&v.next_grad[a])]) + partial);
+                            x = dt - bop;
+                        }
+                    }
+                    if (x < 0) x = 0;
+                }
+                st.fop[d] = (T)fop; st.bop[d] = (T)bop;
+                xs[d][threadIdx.x] = (T)x;
+                a = ee; pfa = pfe; pba = pbe;
+            }
         }
 
         // ---- the row's schedules -------------------------------------------------------------

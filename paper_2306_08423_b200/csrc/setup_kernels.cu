@@ -221,7 +221,41 @@ __global__ void entry_bound_kernel(DeviceView v, Entry *entries, int64_t *jsum)
     entries[i] = en;
 }
 
+// One thread per (entry, word): 32-bit copies of the entry's prefix rows and bucket-lane table.
+// Every value of an entry is at most the entry's time bound, so for a bound below 2^32 the copy
+// is exact; the table's "no buckets" marker (-1) becomes 0, which the evaluation treats alike.
+__global__ void narrow_tables_kernel(DeviceView v, uint2 *pfb32, uint32_t *dt32)
+{
+    const int lp = v.tc.lp, t32 = v.tab_words32, n_tab = (v.tc.n_layers + 1) * (v.tc.n_layers + 1);
+    const int per_entry = lp + (dt32 ? t32 : 0);
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)v.sc.n_entries * per_entry) return;
+    const int en = (int)(i / per_entry), k = (int)(i - (int64_t)en * per_entry);
+    const bool narrow = v.entries[en].bound < ((int64_t)1 << 32);
+    if (k < lp) {
+        uint2 out = make_uint2(0u, 0u);
+        if (narrow) out = make_uint2((uint32_t)v.etf[(int64_t)en * lp + k], (uint32_t)v.etb[(int64_t)en * lp + k]);
+        pfb32[(int64_t)en * lp + k] = out;
+    } else {
+        const int w = k - lp;
+        uint32_t out = 0;
+        if (narrow && w < n_tab) {
+            const int64_t val = v.dt[(int64_t)en * v.tab_words + w];
+            out = val > 0 ? (uint32_t)val : 0u;
+        }
+        dt32[(int64_t)en * t32 + w] = out;
+    }
+}
+
 }  // namespace
+
+void launch_build_narrow_tables(cudaStream_t s, const DeviceView &v, uint2 *pfb32, uint32_t *dt32, int64_t *launches)
+{
+    if (v.sc.n_entries == 0 || !pfb32) return;
+    const int64_t n = (int64_t)v.sc.n_entries * (v.tc.lp + (dt32 ? v.tab_words32 : 0));
+    narrow_tables_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(v, pfb32, dt32);
+    ++*launches;
+}
 
 void launch_build_entry_tables(cudaStream_t s, const DeviceView &v, Entry *entries, int64_t *dt,
                                int64_t *jsum, int64_t *launches)
