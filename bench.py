@@ -43,8 +43,8 @@ RECORD_BYTES = 40
 # DRAM read + write bytes per step of the timed workload, from the one-pass ncu counters summarised in
 # profiles/bench_config1_dram_bytes.md.  They describe the kernels as captured: set them to None when
 # an evaluation or emission kernel changes, until the counters are taken again.
-EVAL_TRAFFIC_BYTES = 214_797_000
-EMIT_TRAFFIC_BYTES = 1_696_308_000
+EVAL_TRAFFIC_BYTES = 214_772_224
+EMIT_TRAFFIC_BYTES = 1_696_515_072
 SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32      # issue slots: one warp instruction per scheduler and clock
 
 
@@ -333,14 +333,18 @@ def run_ours(args):
     achieved_gops = alg_ops / eval_s / 1e9
     # time the recurrence cells alone would take at the measured cell rates of this device
     cell_floor_s = (cells_32 / cell32_peak + (cells - cells_32) / cell64_peak) / 1e9
+    issue_peak_gops = SM_COUNT * SCHEDULERS_PER_SM * LANES * sm_mhz * 1e-3
     roofline = {"bound": "alu", "kernel": "eval_thread_kernel (+ lock-step kernel on small rows)",
-                "achieved": achieved_gops, "peak": int_peak_gops,
-                "unit": "G 32-bit integer instr/s (2 per uint32 cell, 6 per int64 cell)",
-                "frac": achieved_gops / int_peak_gops, "traffic": EVAL_TRAFFIC_BYTES,
+                "achieved": achieved_gops, "peak": issue_peak_gops,
+                "unit": "G 32-bit integer operations/s (2 per uint32 cell: max and add; 6 per int64 cell)",
+                "frac": achieved_gops / issue_peak_gops, "traffic": EVAL_TRAFFIC_BYTES,
                 "traffic_note": "DRAM read + write bytes of the four evaluation launches of one step (ncu, one pass; "
                                 "null when the kernels changed after the counters were taken); algorithmic: 8 B per "
                                 f"candidate = {8 * n_total} B, part of which is still in the L2 when the launches end",
-                "peak_kind": "measured in this run: dependency-free add/xor stream",
+                "peak_kind": "derived: 148 SMs x 4 schedulers x 32 lanes x SM clock sampled during the run (one "
+                             "instruction per scheduler and clock); a uint32 cell's max and add fuse into one "
+                             "add-max instruction that issues at half rate, so this is also the cell bound x 2",
+                "add_xor_probe_Ginstr_per_s": int_peak_gops, "frac_of_add_xor_probe": achieved_gops / int_peak_gops,
                 "cells": cells, "cells_32bit": cells_32, "ms_per_launch_set": statistics.mean(eval_ms),
                 "cell_rate_peaks_Gcells_per_s": {"uint32": cell32_peak, "uint32_fused_add_max": cell32_fused_peak,
                                                  "int64": cell64_peak},
