@@ -215,7 +215,12 @@ typedef struct { int64_t kind, layer, microbatch, start_ns, end_ns; } distsim_re
  *                                  intervals) and busy / batch time
  *   h_total_records                out (host): records needed
  * If capacity_records is too small nothing is written to d_records and the call
- * returns DISTSIM_E_CAPACITY with *h_total_records set.  Synchronises `stream`.
+ * returns DISTSIM_E_CAPACITY with *h_total_records set.  The call synchronises `stream` once,
+ * after planning, to size the output (that is when *h_total_records, d_offsets, d_busy_ns and
+ * d_util are final); the record kernels are then enqueued and the call returns without waiting
+ * for them: d_records is complete when the work enqueued on `stream` so far has finished.  The
+ * context's planning scratch is reused by the next call, so issue a context's calls on one
+ * stream or order them yourself.
  */
 int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indices, int32_t n,
                            distsim_record *d_records, int64_t capacity_records,

@@ -22,7 +22,7 @@ namespace distsim {
 namespace {
 
 constexpr int kItemThreads = 256;
-constexpr int kMaxTileItems = 192;  // most schedule items per block (a plan picks its own count)
+constexpr int kMaxTileItems = 256;  // most schedule items per block (a plan picks its own count)
 constexpr int kTileWords = 3872;    // capacity of a block's image of its run, in int64 words
 constexpr int kTileReplicas = 16;   // replicas per block
 constexpr int kBucketThreads = 128;
@@ -103,7 +103,9 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
             both = max(both, plan->rf[d] + plan->rb[d]);
         }
         // a run of tile_items items of any mix must fit the image of kTileWords words
-        plan->tile_items = max(1, min(kMaxTileItems, kTileWords / (widest * 5)));
+        const int cap = max(1, min(kMaxTileItems, kTileWords / (widest * 5)));
+        const int n_chunks = (2 * en.m + cap - 1) / cap;          // equal runs rather than full ones and a rest
+        plan->tile_items = (2 * en.m + n_chunks - 1) / n_chunks;
         plan->tmpl_words = both * 5;
     }
 }
