@@ -161,6 +161,37 @@ def test_asynchronous_1f1b_schedule(E, ctx, sched_mask):
     assert oracle.eval_indices(w.table, w.space, np.array([bi]))[0][0] == bt == int(batch.min().item())
 
 
+@pytest.mark.parametrize("case", range(12))
+def test_randomised_spaces_sampled_parity(E, ctx, case):
+    """Randomly drawn clusters, layer counts, micro-batch lists (around m = pp, where the
+    recurrence changes form), duration scales (time bounds far below, around and above 2^32, so
+    rows mix 32-bit and 64-bit entries), bucket sizes, overlap modes, schedule masks and jitter:
+    sampled candidates and their per-stage activity times against the oracle."""
+    rng = np.random.default_rng(4000 + case)
+    hi = int(rng.choice([5000, 400_000, 30_000_000, 400_000_000]))
+    ms = sorted(set(int(x) for x in rng.choice([1, 2, 3, 4, 7, 8, 9, 15, 16, 17, 24, 31, 32, 33, 48, 64], size=6)))
+    w = W.random_small(2000 + case, n_devices=int(rng.choice([16, 32, 64])), gpus_per_node=int(rng.choice([2, 4, 8])),
+                       n_layers=int(rng.choice([17, 20, 24])), global_batch=int(rng.choice([64, 96, 128])),
+                       mp_max=int(rng.choice([1, 2, 4])), pp_max=int(rng.choice([4, 8, 16, 16])), m_list=tuple(ms),
+                       partition_mode=W.PARTITION_ALL, dp_overlap=int(rng.integers(0, 2)),
+                       dp_bucket_bytes=int(rng.choice([0, 3000, 100_000])), lo=50, hi=hi,
+                       moe=bool(rng.integers(0, 2)), sched_mask=int(rng.choice([3, 3, 7, 2, 5])))
+    if case % 4 == 3:
+        w = W.add_jitter(w, 4, hi // 7 + 1, case)
+    if W.count_candidates_and_cells(w.table, w.space)[0] < 10:
+        pytest.skip("the draw gave an empty space")
+    n = load(E, ctx, w)
+    batch, sb = eval_all(E, ctx, n, busy=n * ctx.pp_max < 2e8)
+    idx = np.unique(np.concatenate([rng.integers(0, n, 1500), [0, n - 1]]))
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, idx, THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    sel = torch.from_numpy(idx).cuda()
+    gb = batch[sel].cpu().numpy()
+    assert (gb == ob).all(), idx[np.argwhere(gb != ob)[:5, 0]]
+    if sb is not None:
+        assert (sb[sel].cpu().numpy() == obusy).all()
+
+
 def test_ranges_straddle_rows_and_empty(E, ctx):
     w = W.random_small(7, partition_mode=W.PARTITION_ALL)
     n = load(E, ctx, w)
