@@ -47,7 +47,7 @@ constexpr int kMaxRowEntries = 16;      // entries whose scalars are kept in sha
 
 // Resident blocks per SM asked of the compiler (caps the registers per thread).
 template <int PP, typename T>
-constexpr int thread_kernel_min_blocks()
+__host__ __device__ constexpr int thread_kernel_min_blocks()
 {
     return sizeof(T) == 8 ? (PP >= 16 ? 3 : 4) : (PP >= 16 ? 4 : 8);
 }

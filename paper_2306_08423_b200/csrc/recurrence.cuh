@@ -170,21 +170,38 @@ __device__ __forceinline__ int64_t p2p_cost(const Row &row, const Entry &en, int
     return (((d + 1) & (row.p2p_period - 1)) == 0) ? en.p2p_inter : en.p2p_intra;
 }
 
-// Lock-step evaluation of one candidate by `wl` consecutive lanes (wl * S == pp), every lane of
-// the warp calling this together (lanes of other segments work on their own candidates).
+// Two warps that evaluate one candidate together (pp = 64, a stage per lane): per slot the
+// boundary lanes hand the neighbouring warp their latest forward / backward end through shared
+// memory, double-buffered by slot parity, with one named barrier of the 64 threads per slot.
+struct PairLink {
+    int64_t *xf, *xb;            // [2] each: forward end of stage 31, backward end of stage 32
+    int64_t *xm;                 // [2]: each warp's maximum for the final reduction
+    int bar_id;                  // named barrier of the pair (1 .. 15)
+    int half;                    // 0: stages 0 .. 31, 1: stages 32 .. 63
+};
+__device__ __forceinline__ void pair_barrier(int id)
+{
+    asm volatile("bar.sync %0, 64;" :: "r"(id) : "memory");
+}
+
+// Lock-step evaluation of one candidate by `wl` consecutive lanes (wl * S == pp; with kPair by
+// the 2 x 32 lanes of two warps, S == 1), every lane of the warp calling this together (lanes
+// of other segments work on their own candidates).
 //   entry_index  global index of `en`;  seg_lane: lane index inside the segment;
-//   n_slots_warp loop bound, uniform over the warp
+//   n_slots_warp loop bound, uniform over the warp (and over both warps of a pair)
 //   pf, pb     the entry's forward / backward prefix rows (shared or global memory)
 //   rec        if kRecord and non-null: item start times go to rec[d * 2m + position in stage order]
 //   kJit       the table has per-micro-batch jitter (otherwise none of its code is generated)
-template <int S, bool kRecord, bool kJit>
+template <int S, bool kRecord, bool kJit, bool kPair = false>
 __device__ __forceinline__ StageResult<S> lockstep_candidate(
     const DeviceView &v, const Row &row, const Entry &en, int entry_index, const int64_t *pf,
-    const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec)
+    const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec,
+    PairLink link = PairLink{})
 {
+    static_assert(!kPair || S == 1, "a pair of warps owns one stage per lane");
     StageResult<S> R;
     const int pp = row.pp, m = en.m;
-    const int d0 = seg_lane * S;
+    const int d0 = (kPair ? link.half * 32 + seg_lane : seg_lane) * S;
     int bounds[S + 1];
     partition_bounds<S>(v, pp, part_rank, d0, bounds);
 #pragma unroll
@@ -203,8 +220,16 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
     // The lanes of a warp run forward items, backward items or nothing in the same slot, so the
     // slot body is written without branches: one cell with selected operands per owned stage.
     for (int s = 0; s < n_slots_warp; ++s) {
-        const int64_t up_f = __shfl_up_sync(0xffffffffu, last_f[S - 1], 1, wl);
-        const int64_t dn_b = __shfl_down_sync(0xffffffffu, last_b[0], 1, wl);
+        int64_t up_f = __shfl_up_sync(0xffffffffu, last_f[S - 1], 1, wl);
+        int64_t dn_b = __shfl_down_sync(0xffffffffu, last_b[0], 1, wl);
+        if (kPair) {
+            const int buf = s & 1;
+            if (link.half == 0 && seg_lane == 31) link.xf[buf] = last_f[0];
+            if (link.half == 1 && seg_lane == 0) link.xb[buf] = last_b[0];
+            pair_barrier(link.bar_id);
+            if (link.half == 1 && seg_lane == 0) up_f = link.xf[buf];
+            if (link.half == 0 && seg_lane == 31) dn_b = link.xb[buf];
+        }
         int64_t old_f[S], old_b[S];
 #pragma unroll
         for (int k = 0; k < S; ++k) { old_f[k] = last_f[k]; old_b[k] = last_b[k]; }
@@ -216,8 +241,8 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
             slot_activity(sched, pp, m, d, s, do_f, do_b, j);
             do_b = do_b && !do_f;
             const bool act = do_f || do_b;
-            const int64_t dep_f = (k == 0) ? (seg_lane == 0 ? 0 : up_f) : old_f[k > 0 ? k - 1 : 0];
-            const int64_t dep_b = (k == S - 1) ? (seg_lane == wl - 1 ? 0 : dn_b) : old_b[k < S - 1 ? k + 1 : 0];
+            const int64_t dep_f = (k == 0) ? (d == 0 ? 0 : up_f) : old_f[k > 0 ? k - 1 : 0];
+            const int64_t dep_b = (k == S - 1) ? (d == pp - 1 ? 0 : dn_b) : old_b[k < S - 1 ? k + 1 : 0];
             const int64_t st = max64(do_f ? dep_f : dep_b, free_at[k]);
             int64_t jit = 0;
             if (kJit) jit = act ? jitter_of(v, do_f ? v.raw.jit_f : v.raw.jit_b, j, d) : 0;
@@ -246,6 +271,11 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         mx = max64(mx, max64(R.main_end[k], R.dp_end[k]));
     }
     for (int off = 1; off < wl; off <<= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, off, wl));
+    if (kPair) {
+        if (seg_lane == 0) link.xm[link.half] = mx;
+        pair_barrier(link.bar_id);
+        mx = max64(link.xm[0], link.xm[1]);
+    }
     R.batch = mx;
     return R;
 }
