@@ -25,16 +25,25 @@
 //   w_d = max(r_d + c_d, w_{d-1}),   r_d = w_d of the previous wave,
 // a single fused add-max per cell (__viaddmax_u32 on 32-bit times).  Backward waves use the
 // suffix sums of the backward costs, shifted by their total so that every value stays
-// non-negative (the entry's time bound includes that shift).  In a steady 1F1B wave - a
+// non-negative (entries whose time bound plus that shift does not fit 32 bits keep the plain
+// form in 32-bit arithmetic).  In a steady 1F1B wave - a
 // backward and a forward item per stage - the same change of variables, with
 // h_d = latest forward end of stage d - fop_d + bop_0 + .. + bop_{d-1} and fb_d = fop_d + bop_d:
 //   w_d = max(h_d + fb_d, w_{d+1}),   h_d <- max(h_{d-1} + fb_{d-1}, w_d),
 // again one fused add-max per cell.  All of it is exact integer arithmetic.
 //
-// Arithmetic width.  On this GPU a 64-bit max + add costs six half-rate integer instructions,
-// a 32-bit one two full-rate ones.  Every entry carries an upper bound on every time any of its
+// Arithmetic width.  On this GPU a 64-bit max + add costs six integer instructions, a 32-bit
+// one two (one when fused).  Every entry carries an upper bound on every time any of its
 // candidates can produce; the entries whose bound is below 2^32 are evaluated with T = uint32_t
 // (exactly: nothing can overflow), the others with T = int64_t.
+//
+// Tables.  Before the recurrence of an entry a thread works out its pp stage costs and
+// bucket-lane excesses; for entries with few micro-batches that part outweighs the cells.  The
+// block therefore stages what it reads in shared memory with bulk copies: the prefix rows of
+// the row's entries, the binomial table of the unranking and the bucket-lane tables of as many
+// of the row's last entries as fit the budget that keeps the kernel's resident blocks per SM.
+// The 32-bit instance reads 32-bit copies of the tables (forward and backward prefix packed
+// into one 8-byte word), which halves the shared memory and the arithmetic of that part.
 #pragma once
 
 #include "recurrence.cuh"
