@@ -24,6 +24,10 @@
  *   pipeline lists as d*MP + m_p; DP modeling duplicates them DP times, so the
  *   replica index r is outermost).  node(rank) = rank / G.
  *
+ * Schedules: GPipe, 1F1B (Dapple), asynchronous 1F1B (no gradient all-reduce) and, for
+ * candidates given explicitly, interleaved 1F1B over v model chunks per device (see the
+ * comment above orc_simulate).
+ *
  * Pins for every function here live in tests/test_oracle_pins.py (closed
  * forms, invariants, brute-force longest path, hand-worked examples, printed
  * counts from the paper).  The paper's measured accuracy against real clusters
@@ -91,8 +95,11 @@ typedef struct {
 } orc_space;
 
 typedef struct {
-    int32_t mp, pp, dp, m, sched;         /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B */
-    int32_t bounds[ORC_MAX_PP + 1];       /* c_0 .. c_pp                          */
+    int32_t mp, pp, dp, m, sched;         /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B,
+                                             3: interleaved 1F1B (simulated when given
+                                             explicitly; the search space does not enumerate it) */
+    int32_t bounds[ORC_MAX_PP + 1];       /* c_0 .. c_P, P = pp (P = pp * v for sched 3)  */
+    int32_t v;                            /* sched 3: model chunks per device (0 or 1 otherwise) */
 } orc_candidate;
 
 typedef struct { int64_t kind, layer, mb, start, end; } orc_event;
@@ -192,13 +199,15 @@ static int loc_dp_groups(const orc_table *T, const orc_candidate *x)
         }
     return cur;
 }
-static int loc_boundary(const orc_table *T, const orc_candidate *x, int64_t d)
+/* Transfer from pipeline device da to pipeline device db (db = da + 1 between neighbouring
+ * stages; the interleaved schedule also sends from the last device back to the first). */
+static int loc_transfer(const orc_table *T, const orc_candidate *x, int64_t da, int64_t db)
 {
     int cur = -2;
     for (int64_t r = 0; r < x->dp; ++r)
         for (int64_t q = 0; q < x->mp; ++q) {
-            int inter = rank_of(x, r, d, q) / T->gpus_per_node !=
-                        rank_of(x, r, d + 1, q) / T->gpus_per_node;
+            int inter = rank_of(x, r, da, q) / T->gpus_per_node !=
+                        rank_of(x, r, db, q) / T->gpus_per_node;
             cur = merge_loc(cur, inter);
         }
     return cur;
@@ -298,7 +307,7 @@ int orc_enumerate_at(const orc_table *T, const orc_space *S, const int64_t *sort
 /* ------------------------------------------------------------------------- */
 /* The simulation of one candidate.                                           */
 
-typedef struct { int32_t is_bwd, mb; } orc_op;
+typedef struct { int32_t is_bwd, mb, chunk; } orc_op;
 
 static int find_class(const orc_table *T, int64_t mp, int64_t b)
 {
@@ -339,6 +348,21 @@ static int64_t union_measure(const orc_list *l)
 }
 
 /*
+ * Interleaved 1F1B (sched 3; the paper names further scheduling algorithms as input to the same
+ * pipeline modeling, Sec. 4.3 "the pipeline schedule generated from the pipeline algorithm",
+ * and cites Megatron-LM, whose interleaved schedule this is).  Every device holds v model
+ * chunks: the model is cut into P = pp * v virtual stages, virtual stage s = c * pp + d being
+ * chunk c of device d, so consecutive virtual stages sit on consecutive devices and the last
+ * device sends to the first between chunks.  A device runs its m * v forward and m * v backward
+ * items in this order (m must be a multiple of pp): the k-th forward item is chunk
+ * (k / pp) mod v of micro-batch (k / (pp v)) pp + k mod pp, the k-th backward item the same
+ * with chunk v - 1 - (k / pp) mod v; device d first runs min(m v, 2 (pp - d - 1) + (v - 1) pp)
+ * forward items (all of them when m = pp), then alternates one forward, one backward, and
+ * finishes with the remaining backward items.  Dependencies, events, transfers and the
+ * device-is-busy rule are those of Algorithm 1, with virtual stages in the place of stages.
+ * Gradient buckets are cut per chunk (each chunk's gradients in backward order), chunks in the
+ * order their last micro-batch's backward runs (v - 1 first), on the device's one lane.
+ *
  * orc_simulate
  *   replicate    1: keep a list for every one of the N devices;
  *                0: keep only the device (r=0, q=0) of every stage (pp lists).
@@ -356,14 +380,17 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
     int64_t *endF = NULL, *endB = NULL;
     orc_event *tmp = NULL;
     const int pp = x->pp, mp = x->mp, dp = x->dp, m = x->m, L = T->n_layers;
+    const int v = x->sched == 3 ? x->v : 1;      /* model chunks per device               */
+    const int P = pp * v;                        /* virtual stages                         */
 
-    if (pp < 1 || pp > ORC_MAX_PP || mp < 1 || dp < 1 || m < 1 ||
+    if (pp < 1 || pp > ORC_MAX_PP || mp < 1 || dp < 1 || m < 1 || v < 1 || P > ORC_MAX_PP ||
         (int64_t)mp * pp * dp != T->n_devices || T->global_batch % dp != 0 ||
-        x->bounds[0] != 0 || x->bounds[pp] != L || x->sched < 0 || x->sched > 2 ||
+        x->bounds[0] != 0 || x->bounds[P] != L || x->sched < 0 || x->sched > 3 ||
+        (x->sched == 3 && (m % pp != 0 || T->n_jitter > 0)) ||
         (T->n_jitter > 0 && (T->jitter_stages < pp || !T->jitter_fwd_ns || !T->jitter_bwd_ns))) {
         e = ORC_E_ARG; goto fail;
     }
-    for (int d = 0; d < pp; ++d) if (x->bounds[d + 1] <= x->bounds[d]) { e = ORC_E_ARG; goto fail; }
+    for (int s = 0; s < P; ++s) if (x->bounds[s + 1] <= x->bounds[s]) { e = ORC_E_ARG; goto fail; }
 
     /* ---- Step 1: events and their elapsed times (MP modeling) ------------- */
     const int64_t Bp = T->global_batch / dp;
@@ -386,25 +413,47 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
         if (loc_dp < 0) { e = ORC_E_LOCALITY; goto fail; }
         A2A = orc_all_to_all_ns(dp, act, alpha_of(T, loc_dp), beta_of(T, loc_dp));
     }
-    for (int d = 0; d + 1 < pp; ++d) {
-        int loc = loc_boundary(T, x, d);
+    /* P2P[s]: transfer between virtual stages s and s + 1, i.e. between devices s mod pp and
+     * (s + 1) mod pp */
+    for (int s = 0; s + 1 < P; ++s) {
+        int loc = loc_transfer(T, x, s % pp, (s + 1) % pp);
         if (loc < 0) { e = ORC_E_LOCALITY; goto fail; }
-        P2P[d] = orc_p2p_ns(act, alpha_of(T, loc), beta_of(T, loc));
+        P2P[s] = orc_p2p_ns(act, alpha_of(T, loc), beta_of(T, loc));
     }
 
     /* ---- Step 2: the pipeline schedule S(D, L, M) -------------------------- */
-    ops = (orc_op *)malloc((size_t)pp * 2 * m * sizeof(orc_op));
-    endF = (int64_t *)malloc((size_t)pp * m * sizeof(int64_t));
-    endB = (int64_t *)malloc((size_t)pp * m * sizeof(int64_t));
+    const int n_ops = 2 * m * v;                 /* items of one device                    */
+    ops = (orc_op *)malloc((size_t)pp * n_ops * sizeof(orc_op));
+    endF = (int64_t *)malloc((size_t)P * m * sizeof(int64_t));      /* [virtual stage][micro-batch] */
+    endB = (int64_t *)malloc((size_t)P * m * sizeof(int64_t));
     tmp = (orc_event *)malloc((size_t)(3 * L + 2) * sizeof(orc_event));
     const int mp_lists = replicate ? mp : 1;
     F = (orc_list *)calloc((size_t)pp * mp_lists, sizeof(orc_list));
     if (!ops || !endF || !endB || !tmp || !F) { e = ORC_E_NOMEM; goto fail; }
-    for (int64_t i = 0; i < (int64_t)pp * m; ++i) endF[i] = endB[i] = -1;
+    for (int64_t i = 0; i < (int64_t)P * m; ++i) endF[i] = endB[i] = -1;
     for (int d = 0; d < pp; ++d) {
-        orc_op *o = ops + (int64_t)d * 2 * m;
+        orc_op *o = ops + (int64_t)d * n_ops;
         int k = 0;
-        if (x->sched == 0) {                      /* GPipe: all forwards, then all backwards */
+        for (int i = 0; i < n_ops; ++i) o[i].chunk = 0;
+        if (x->sched == 3) {                      /* interleaved 1F1B over v chunks        */
+            const int total = m * v;
+            int warm = (pp - d - 1) * 2 + (v - 1) * pp;
+            if (m == pp || warm > total) warm = total;
+            int nf = 0, nb = 0;
+            for (int step = 0; step < 2 * total; ++step) {
+                /* warm-up forwards; then forward, backward alternately; then the backwards left */
+                int is_b;
+                if (nf < warm) is_b = 0;
+                else if (nf < total) is_b = ((step - warm) & 1);
+                else is_b = 1;
+                const int idx = is_b ? nb++ : nf++;
+                const int c = (idx / pp) % v;
+                o[k].is_bwd = is_b;
+                o[k].chunk = is_b ? v - 1 - c : c;
+                o[k].mb = (idx / (pp * v)) * pp + idx % pp;
+                ++k;
+            }
+        } else if (x->sched == 0) {               /* GPipe: all forwards, then all backwards */
             for (int j = 0; j < m; ++j) { o[k].is_bwd = 0; o[k++].mb = j; }
             for (int j = 0; j < m; ++j) { o[k].is_bwd = 1; o[k++].mb = j; }
         } else {                                  /* 1F1B (Dapple): warm-up, then one-B-one-F;
@@ -423,24 +472,28 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
     {
         int32_t head[ORC_MAX_PP];
         int64_t device_free[ORC_MAX_PP];
-        int64_t remaining = (int64_t)pp * 2 * m;
+        int64_t remaining = (int64_t)pp * n_ops;
         for (int d = 0; d < pp; ++d) { head[d] = 0; device_free[d] = 0; }
         while (remaining > 0) {
-            /* first_available: the first stage whose next item has its data ready */
+            /* first_available: the first device whose next item has its data ready; the item
+             * belongs to virtual stage vs = chunk * pp + d (vs = d without chunks) */
             int pick = -1; int64_t t = 0;
             for (int s = 0; s < pp && pick < 0; ++s) {
                 int d = reverse_scan ? pp - 1 - s : s;
-                if (head[d] == 2 * m) continue;
-                orc_op o = ops[(int64_t)d * 2 * m + head[d]];
+                if (head[d] == n_ops) continue;
+                orc_op o = ops[(int64_t)d * n_ops + head[d]];
+                const int vs = o.chunk * pp + d;
                 int64_t dep;
-                if (!o.is_bwd) dep = d == 0 ? 0 : endF[(int64_t)(d - 1) * m + o.mb];
-                else dep = d == pp - 1 ? endF[(int64_t)d * m + o.mb] : endB[(int64_t)(d + 1) * m + o.mb];
+                if (!o.is_bwd) dep = vs == 0 ? 0 : endF[(int64_t)(vs - 1) * m + o.mb];
+                else dep = vs == P - 1 ? endF[(int64_t)vs * m + o.mb] : endB[(int64_t)(vs + 1) * m + o.mb];
                 if (dep < 0) continue;
                 pick = d; t = max64(device_free[d], dep);
             }
             if (pick < 0) { e = ORC_E_DEADLOCK; goto fail; }
             const int d = pick;
-            const orc_op o = ops[(int64_t)d * 2 * m + head[d]];
+            const orc_op o = ops[(int64_t)d * n_ops + head[d]];
+            const int vs = o.chunk * pp + d;
+            const int la = x->bounds[vs], le = x->bounds[vs + 1];   /* the item's layers [la, le) */
             /* e <- MAP[l]: the stage's layers, each a computation event followed by
              * its all-reduce event (mp > 1) and its all-to-all event (expert layer,
              * dp > 1); then e_comm, the transfer to the neighbouring stage. */
@@ -452,26 +505,26 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
             if (T->n_jitter > 0) {
                 const int64_t *jt = o.is_bwd ? T->jitter_bwd_ns : T->jitter_fwd_ns;
                 const int64_t jit = jt[(int64_t)(o.mb % T->n_jitter) * T->jitter_stages + d];
-                const int first_layer = o.is_bwd ? x->bounds[d + 1] - 1 : x->bounds[d];
+                const int first_layer = o.is_bwd ? le - 1 : la;
                 tmp[n++] = (orc_event){ o.is_bwd ? ORC_JITTER_B : ORC_JITTER_F, first_layer, o.mb, t, t + jit };
                 t += jit;
             }
             if (!o.is_bwd) {
-                for (int l = x->bounds[d]; l < x->bounds[d + 1]; ++l) {
+                for (int l = la; l < le; ++l) {
                     tmp[n++] = (orc_event){ ORC_COMPUTE_F, l, o.mb, t, t + f[l] }; t += f[l];
                     if (mp > 1) { tmp[n++] = (orc_event){ ORC_MP_AR_F, l, o.mb, t, t + AR }; t += AR; }
                     if (T->layer_is_expert[l] && dp > 1) { tmp[n++] = (orc_event){ ORC_A2A_F, l, o.mb, t, t + A2A }; t += A2A; }
                 }
-                if (d < pp - 1) { tmp[n++] = (orc_event){ ORC_SEND_F, x->bounds[d + 1] - 1, o.mb, t, t + P2P[d] }; t += P2P[d]; }
-                endF[(int64_t)d * m + o.mb] = t;
+                if (vs < P - 1) { tmp[n++] = (orc_event){ ORC_SEND_F, le - 1, o.mb, t, t + P2P[vs] }; t += P2P[vs]; }
+                endF[(int64_t)vs * m + o.mb] = t;
             } else {
-                for (int l = x->bounds[d + 1] - 1; l >= x->bounds[d]; --l) {
+                for (int l = le - 1; l >= la; --l) {
                     tmp[n++] = (orc_event){ ORC_COMPUTE_B, l, o.mb, t, t + g[l] }; t += g[l];
                     if (mp > 1) { tmp[n++] = (orc_event){ ORC_MP_AR_B, l, o.mb, t, t + AR }; t += AR; }
                     if (T->layer_is_expert[l] && dp > 1) { tmp[n++] = (orc_event){ ORC_A2A_B, l, o.mb, t, t + A2A }; t += A2A; }
                 }
-                if (d > 0) { tmp[n++] = (orc_event){ ORC_SEND_B, x->bounds[d], o.mb, t, t + P2P[d - 1] }; t += P2P[d - 1]; }
-                endB[(int64_t)d * m + o.mb] = t;
+                if (vs > 0) { tmp[n++] = (orc_event){ ORC_SEND_B, la, o.mb, t, t + P2P[vs - 1] }; t += P2P[vs - 1]; }
+                endB[(int64_t)vs * m + o.mb] = t;
             }
             device_free[d] = t;
             for (int q = 0; q < mp_lists; ++q)          /* every device of the MP group */
@@ -511,39 +564,45 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                      * cut into buckets; each bucket is a ring all-reduce over
                      * the dp replicas on a separate communication lane. */
                     const int64_t main_end = src->n ? src->ev[src->n - 1].end : 0;
-                    int64_t W = 0;
-                    for (int l = x->bounds[d]; l < x->bounds[d + 1]; ++l) W += cdiv(T->grad_bytes[l], mp);
-                    if (W == 0) continue;
-                    const int64_t bucket = T->dp_bucket_bytes > 0 ? T->dp_bucket_bytes : W;
-                    const int64_t nb = cdiv(W, bucket);
-                    int64_t prev_end = 0;
-                    for (int64_t k = 0; k < nb; ++k) {
-                        const int64_t lo = k * bucket;
-                        const int64_t hi = lo + bucket < W ? lo + bucket : W;
-                        int64_t ready = main_end;
-                        if (T->dp_overlap) {
-                            /* the layer holding the bucket's last byte (position hi-1) */
-                            int64_t pos = 0; int last = -1;
-                            for (int l = x->bounds[d + 1] - 1; l >= x->bounds[d]; --l) {
-                                int64_t gl = cdiv(T->grad_bytes[l], mp);
-                                if (hi - 1 >= pos && hi - 1 < pos + gl) { last = l; break; }
-                                pos += gl;
+                    int64_t prev_end = 0, kb = 0;      /* the device's one lane; bucket numbers run on */
+                    /* one gradient stream per model chunk (one stream without chunks), the
+                     * chunks in the order their last backward runs: chunk v - 1 first */
+                    for (int c = v - 1; c >= 0; --c) {
+                        const int vs = c * pp + d;
+                        const int la = x->bounds[vs], le = x->bounds[vs + 1];
+                        int64_t W = 0;
+                        for (int l = la; l < le; ++l) W += cdiv(T->grad_bytes[l], mp);
+                        if (W == 0) continue;
+                        const int64_t bucket = T->dp_bucket_bytes > 0 ? T->dp_bucket_bytes : W;
+                        const int64_t nb = cdiv(W, bucket);
+                        for (int64_t k = 0; k < nb; ++k) {
+                            const int64_t lo = k * bucket;
+                            const int64_t hi = lo + bucket < W ? lo + bucket : W;
+                            int64_t ready = main_end;
+                            if (T->dp_overlap) {
+                                /* the layer holding the bucket's last byte (position hi-1) */
+                                int64_t pos = 0; int last = -1;
+                                for (int l = le - 1; l >= la; --l) {
+                                    int64_t gl = cdiv(T->grad_bytes[l], mp);
+                                    if (hi - 1 >= pos && hi - 1 < pos + gl) { last = l; break; }
+                                    pos += gl;
+                                }
+                                /* ready when that layer's backward events of the LAST
+                                 * microbatch's backward pass have all finished */
+                                ready = -1;
+                                for (int64_t i = 0; i < src->n; ++i) {
+                                    const orc_event *ev = &src->ev[i];
+                                    if (ev->layer == last && ev->mb == m - 1 &&
+                                        (ev->kind == ORC_COMPUTE_B || ev->kind == ORC_MP_AR_B || ev->kind == ORC_A2A_B))
+                                        ready = max64(ready, ev->end);
+                                }
+                                if (ready < 0) { e = ORC_E_ARG; goto fail; }
                             }
-                            /* ready when that layer's backward events of the LAST
-                             * microbatch's backward pass have all finished */
-                            ready = -1;
-                            for (int64_t i = 0; i < src->n; ++i) {
-                                const orc_event *v = &src->ev[i];
-                                if (v->layer == last && v->mb == m - 1 &&
-                                    (v->kind == ORC_COMPUTE_B || v->kind == ORC_MP_AR_B || v->kind == ORC_A2A_B))
-                                    ready = max64(ready, v->end);
-                            }
-                            if (ready < 0) { e = ORC_E_ARG; goto fail; }
+                            const int64_t start = max64(ready, prev_end);
+                            const int64_t end = start + orc_allreduce_ns(T->allreduce_profile_max, dp, hi - lo, alpha_of(T, loc_dp), beta_of(T, loc_dp));
+                            if ((e = list_push(dst, (orc_event){ ORC_DP_AR, kb++, -1, start, end })) != ORC_OK) goto fail;
+                            prev_end = end;
                         }
-                        const int64_t start = max64(ready, prev_end);
-                        const int64_t end = start + orc_allreduce_ns(T->allreduce_profile_max, dp, hi - lo, alpha_of(T, loc_dp), beta_of(T, loc_dp));
-                        if ((e = list_push(dst, (orc_event){ ORC_DP_AR, k, -1, start, end })) != ORC_OK) goto fail;
-                        prev_end = end;
                     }
                 }
     }

@@ -51,7 +51,7 @@ class _Space(C.Structure):
 
 class _Cand(C.Structure):
     _fields_ = [("mp", C.c_int32), ("pp", C.c_int32), ("dp", C.c_int32), ("m", C.c_int32),
-                ("sched", C.c_int32), ("bounds", C.c_int32 * (_MAX_PP + 1))]
+                ("sched", C.c_int32), ("bounds", C.c_int32 * (_MAX_PP + 1)), ("v", C.c_int32)]
 
 
 @dataclass
@@ -62,11 +62,13 @@ class Candidate:
     m: int
     sched: int
     bounds: tuple
+    v: int = 1               # model chunks per device (interleaved 1F1B, sched 3)
 
     def _c(self) -> _Cand:
         c = _Cand(self.mp, self.pp, self.dp, self.m, self.sched)
-        for i, v in enumerate(self.bounds):
-            c.bounds[i] = v
+        for i, b in enumerate(self.bounds):
+            c.bounds[i] = b
+        c.v = self.v
         return c
 
 

@@ -31,10 +31,29 @@ def stage_order(sched, pp, d, m):
     return order
 
 
+def interleaved_order(pp, v, d, m):
+    """('F'|'B', j, chunk) in the order device d runs them under interleaved 1F1B: micro-batches
+    go in groups of pp; a group passes chunk 0, 1, .. forward and v-1, v-2, .. backward.  The
+    device launches forwards until the first micro-batch can have come back to it through all
+    later devices and chunks (all of them when there is a single group), then alternates."""
+    fseq = [(c, g * pp + i) for g in range(m // pp) for c in range(v) for i in range(pp)]
+    bseq = [(c, g * pp + i) for g in range(m // pp) for c in reversed(range(v)) for i in range(pp)]
+    warm = len(fseq) if m == pp else min(len(fseq), 2 * (pp - d - 1) + (v - 1) * pp)
+    order = [("F", j, c) for (c, j) in fseq[:warm]]
+    rest_f, b = fseq[warm:], list(bseq)
+    while rest_f:
+        c, j = rest_f.pop(0); order.append(("F", j, c))
+        c, j = b.pop(0); order.append(("B", j, c))
+    order += [("B", j, c) for (c, j) in b]
+    return order
+
+
 def longest_path_timeline(table, cand):
     """Returns (batch_ns, {stage d: [(kind, layer, mb, start, end), ...] main lane then buckets})."""
     T = table
     pp, mp, dp, m = cand.pp, cand.mp, cand.dp, cand.m
+    v = cand.v if cand.sched == 3 else 1       # model chunks per device
+    P = pp * v                                  # virtual stages; stage vs = chunk * pp + device
     c = cand.bounds
     G = T.gpus_per_node
     Bp = T.global_batch // dp
@@ -62,8 +81,8 @@ def longest_path_timeline(table, cand):
         a, be = ab(dp_inter)
         A2A = (dp - 1) * a + ceil_div((dp - 1) * act, dp * be)
     P2P = []
-    for d in range(pp - 1):
-        a, be = ab(rank(0, d, 0) // G != rank(0, d + 1, 0) // G)
+    for vs in range(P - 1):
+        a, be = ab(rank(0, vs % pp, 0) // G != rank(0, (vs + 1) % pp, 0) // G)
         P2P.append(a + ceil_div(act, be))
 
     # nodes: id -> (duration, [predecessor ids]); names are tuples
@@ -73,9 +92,12 @@ def longest_path_timeline(table, cand):
     lane = {d: [] for d in range(pp)}
     for d in range(pp):
         prev = None
-        for (typ, j) in stage_order(cand.sched, pp, d, m):
+        items = (interleaved_order(pp, v, d, m) if cand.sched == 3
+                 else [(typ, j, 0) for (typ, j) in stage_order(cand.sched, pp, d, m)])
+        for (typ, j, ch) in items:
             evs = []
-            layers = range(c[d], c[d + 1]) if typ == "F" else range(c[d + 1] - 1, c[d] - 1, -1)
+            vs = ch * pp + d
+            layers = range(c[vs], c[vs + 1]) if typ == "F" else range(c[vs + 1] - 1, c[vs] - 1, -1)
             jt = getattr(T, "jitter_fwd_ns" if typ == "F" else "jitter_bwd_ns", None)
             if jt is not None:
                 evs.append((9 if typ == "F" else 10, layers[0], int(jt[j % len(jt)][d])))
@@ -85,58 +107,61 @@ def longest_path_timeline(table, cand):
                     evs.append((2 if typ == "F" else 3, l, AR))
                 if T.layer_is_expert[l] and dp > 1:
                     evs.append((4 if typ == "F" else 5, l, A2A))
-            if typ == "F" and d < pp - 1:
-                evs.append((6, c[d + 1] - 1, P2P[d]))
-            if typ == "B" and d > 0:
-                evs.append((7, c[d], P2P[d - 1]))
+            if typ == "F" and vs < P - 1:
+                evs.append((6, c[vs + 1] - 1, P2P[vs]))
+            if typ == "B" and vs > 0:
+                evs.append((7, c[vs], P2P[vs - 1]))
             for i, (kind, l, du) in enumerate(evs):
-                nid = (d, typ, j, i)
+                nid = (vs, typ, j, i)
                 dur[nid] = du
                 preds[nid] = [prev] if prev is not None else []
                 label[nid] = (kind, l, j)
                 lane[d].append(nid)
                 if i == 0:
-                    first_of_op[(d, typ, j)] = nid
+                    first_of_op[(vs, typ, j)] = nid
                 if typ == "B" and j == m - 1 and kind in (1, 3, 5):
                     layer_done[(d, l)] = nid
                 prev = nid
-            last_of_op[(d, typ, j)] = prev
-    # data edges
-    for d in range(pp):
+            last_of_op[(vs, typ, j)] = prev
+    # data edges between neighbouring (virtual) stages
+    for vs in range(P):
         for j in range(m):
-            if d > 0:
-                preds[first_of_op[(d, "F", j)]].append(last_of_op[(d - 1, "F", j)])
-            if d < pp - 1:
-                preds[first_of_op[(d, "B", j)]].append(last_of_op[(d + 1, "B", j)])
+            if vs > 0:
+                preds[first_of_op[(vs, "F", j)]].append(last_of_op[(vs - 1, "F", j)])
+            if vs < P - 1:
+                preds[first_of_op[(vs, "B", j)]].append(last_of_op[(vs + 1, "B", j)])
             else:
-                preds[first_of_op[(d, "B", j)]].append(last_of_op[(d, "F", j)])
+                preds[first_of_op[(vs, "B", j)]].append(last_of_op[(vs, "F", j)])
     # gradient buckets on a separate lane
     buckets = {d: [] for d in range(pp)}
     if dp > 1 and cand.sched != 2:       # the asynchronous schedule has no gradient all-reduce
         a, be = ab(dp_inter)
         for d in range(pp):
-            stream = [(l, ceil_div(int(T.grad_bytes[l]), mp)) for l in range(c[d + 1] - 1, c[d] - 1, -1)]
-            W = sum(x[1] for x in stream)
-            if W == 0:
-                continue
-            size = T.dp_bucket_bytes if T.dp_bucket_bytes > 0 else W
-            k, lo, prevb = 0, 0, None
-            while lo < W:
-                hi = min(W, lo + size)
-                pos, owner = 0, None
-                for (l, gl) in stream:
-                    if pos <= hi - 1 < pos + gl:
-                        owner = l
-                    pos += gl
-                nid = (d, "G", k, 0)
-                dur[nid] = 2 * (dp - 1) * a + ceil_div(2 * (dp - 1) * (hi - lo), dp * be)
-                ready = layer_done[(d, owner)] if T.dp_overlap else lane[d][-1]
-                preds[nid] = [ready] + ([prevb] if prevb is not None else [])
-                label[nid] = (8, k, -1)
-                buckets[d].append(nid)
-                prevb = nid
-                k += 1
-                lo = hi
+            k, prevb = 0, None                  # one lane per device; bucket numbers run on over the chunks
+            for ch in reversed(range(v)):       # a stream per chunk, the chunk whose last backward runs first first
+                vs = ch * pp + d
+                stream = [(l, ceil_div(int(T.grad_bytes[l]), mp)) for l in range(c[vs + 1] - 1, c[vs] - 1, -1)]
+                W = sum(x[1] for x in stream)
+                if W == 0:
+                    continue
+                size = T.dp_bucket_bytes if T.dp_bucket_bytes > 0 else W
+                lo = 0
+                while lo < W:
+                    hi = min(W, lo + size)
+                    pos, owner = 0, None
+                    for (l, gl) in stream:
+                        if pos <= hi - 1 < pos + gl:
+                            owner = l
+                        pos += gl
+                    nid = (d, "G", k, 0)
+                    dur[nid] = 2 * (dp - 1) * a + ceil_div(2 * (dp - 1) * (hi - lo), dp * be)
+                    ready = layer_done[(d, owner)] if T.dp_overlap else lane[d][-1]
+                    preds[nid] = [ready] + ([prevb] if prevb is not None else [])
+                    label[nid] = (8, k, -1)
+                    buckets[d].append(nid)
+                    prevb = nid
+                    k += 1
+                    lo = hi
 
     sys.setrecursionlimit(max(10000, 4 * len(dur) + 1000))
 

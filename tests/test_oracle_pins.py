@@ -238,6 +238,84 @@ def test_async_1f1b_is_1f1b_without_gradient_allreduce(seed):
     assert seen_dp
 
 
+# interleaved 1F1B (v model chunks per device): simulated for candidates given explicitly
+@pytest.mark.parametrize("pp,v,groups", [(2, 2, 1), (2, 2, 3), (2, 4, 2), (4, 2, 1), (4, 3, 2), (8, 2, 3), (8, 4, 1), (16, 2, 2)])
+def test_interleaved_uniform_closed_form(pp, v, groups):
+    # Uniform virtual stages, no communication cost: the schedule's bubble is (pp - 1) items of
+    # one chunk, 1 / v of the plain pipeline's: batch = (m v + pp - 1)(t_f + t_b) with per-chunk
+    # item times.  Any slip in the item order shows up as a longer batch or a deadlock.
+    tf, tb, per, m = 7, 13, 2, pp * groups
+    L = pp * v * per
+    T = make_table([tf] * L, [tb] * L, n_devices=pp, gpus_per_node=1, global_batch=m,
+                   classes=[(1, 1)], alpha_intra_ns=0, alpha_inter_ns=0)
+    r = oracle.simulate(T, Candidate(1, pp, 1, m, 3, tuple(j * per for j in range(pp * v + 1)), v))
+    assert r.batch_ns == (m * v + pp - 1) * per * (tf + tb)
+    assert (r.busy_ns == m * v * per * (tf + tb)).all()
+    # the same model on the plain pipeline (v times longer stages) has the v times larger bubble
+    plain = oracle.simulate(T, Candidate(1, pp, 1, m, 1, balanced(L, pp)))
+    assert plain.batch_ns == (m + pp - 1) * v * per * (tf + tb) > r.batch_ns
+
+
+def _interleaved_cases():
+    for seed in range(12):
+        rng = np.random.default_rng(700 + seed)
+        pp, v = [(2, 2), (2, 3), (4, 2)][seed % 3]
+        mp = 1 + seed % 2
+        dp = [1, 2][(seed // 2) % 2]
+        m = pp * int(rng.integers(1, 3))
+        P = pp * v
+        L = P + int(rng.integers(0, 4))
+        cuts = sorted(rng.choice(np.arange(1, L), size=P - 1, replace=False).tolist())
+        w = W.random_small(800 + seed, n_devices=pp * mp * dp, gpus_per_node=2, n_layers=L,
+                           global_batch=dp * m * int(rng.integers(1, 3)), mp_max=2, pp_max=4, m_list=(m,),
+                           dp_overlap=seed % 2, dp_bucket_bytes=0 if seed % 5 == 4 else 700)
+        yield w, Candidate(mp, pp, dp, m, 3, (0, *cuts, L), v)
+
+
+@pytest.mark.parametrize("w,cand", list(_interleaved_cases()), ids=lambda x: getattr(x, "name", None))
+def test_interleaved_brute_force_and_invariants(w, cand):
+    T = w.table
+    r = oracle.simulate(T, cand, replicate=False)
+    batch, lanes = longest_path_timeline(T, cand)          # independent DAG over virtual stages
+    assert r.batch_ns == batch
+    for d in range(cand.pp):
+        got = [tuple(x) for x in r.records[r.offsets[d]:r.offsets[d + 1]].tolist()]
+        assert got == lanes[d], (cand, d)
+    # the scan order of first_available does not matter; replicas are identical
+    assert oracle.simulate(T, cand, replicate=False, reverse_scan=True).batch_ns == r.batch_ns
+    full = oracle.simulate(T, cand, replicate=True)
+    assert full.batch_ns == r.batch_ns
+    for rr in range(cand.dp):
+        for d in range(cand.pp):
+            for q in range(cand.mp):
+                dev = (rr * cand.pp + d) * cand.mp + q
+                a = full.records[full.offsets[dev]:full.offsets[dev + 1]]
+                assert (a == r.records[r.offsets[d]:r.offsets[d + 1]]).all()
+    # every device's main lane is serial and holds each (chunk, micro-batch) item once
+    for d in range(cand.pp):
+        a = r.records[r.offsets[d]:r.offsets[d + 1]]
+        main = a[a[:, 0] != 8]
+        assert (main[1:, 3] >= main[:-1, 4]).all()
+        comp_f = main[main[:, 0] == 0]
+        layers_d = [l for c in range(cand.v) for l in range(cand.bounds[c * cand.pp + d], cand.bounds[c * cand.pp + d + 1])]
+        assert sorted(set(comp_f[:, 1].tolist())) == sorted(layers_d)
+        assert len(comp_f) == cand.m * len(layers_d)
+        if not T.dp_overlap or cand.dp == 1:
+            assert r.busy_ns[d] == int((a[:, 4] - a[:, 3]).sum())
+    assert r.batch_ns >= int(r.busy_ns.max())
+
+
+def test_interleaved_rejects_what_the_schedule_does_not_define():
+    T = make_table([5] * 8, [9] * 8, n_devices=2, gpus_per_node=2, global_batch=6, classes=[(1, 1), (1, 2), (1, 3)],
+                   alpha_intra_ns=1, alpha_inter_ns=1, beta_intra=1, beta_inter=1)
+    ok = Candidate(1, 2, 1, 6, 3, (0, 2, 4, 6, 8), 2)
+    assert oracle.simulate(T, ok).batch_ns > 0
+    with pytest.raises(Exception):
+        oracle.simulate(T, Candidate(1, 2, 1, 3, 3, (0, 2, 4, 6, 8), 2))      # m is not a multiple of pp
+    with pytest.raises(Exception):
+        oracle.simulate(T, Candidate(1, 2, 1, 6, 3, (0, 4, 8), 2))            # bounds for pp stages, not pp * v
+
+
 # per-micro-batch jitter
 def _jittered(seed, **kw):
     w = W.random_small(seed, n_devices=8, gpus_per_node=4, n_layers=4, global_batch=8, mp_max=2,
