@@ -392,7 +392,7 @@ def run_ours(args):
 
     if world == 1:
         if not args.no_workloads:
-            line["workloads"] = other_workloads(E, ctx, torch, dev, peaks)
+            line["workloads"] = other_workloads(E, ctx, torch, dev, peaks, cell32_peak, cell64_peak)
         if not args.no_cpu:
             import oracle
             oracle.build()
@@ -409,7 +409,7 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def other_workloads(E, ctx, torch, dev, peaks):
+def other_workloads(E, ctx, torch, dev, peaks, cell32_peak, cell64_peak):
     """Evaluation rate on the other search workloads and emission rate on the 1024 fastest
     candidates of the 1024-device workload (device-resident, CUDA events)."""
     out = {}
@@ -430,8 +430,12 @@ def other_workloads(E, ctx, torch, dev, peaks):
             if it >= 3:
                 times.append(e0.elapsed_time(e1) * 1e-3)
         t = statistics.median(times)
-        out[w.name] = {"candidates": n, "cells": cells, "eval_ms": t * 1e3, "candidates_per_sec": n / t,
-                       "events_per_sec": cells / t, "best_index": best[0], "best_batch_ns": best[1]}
+        _, cells_32 = E.distsim_space_cells(ctx)
+        # time the cells alone would take at this device's measured 32-bit / 64-bit cell rates
+        floor_s = (cells_32 / cell32_peak + (cells - cells_32) / cell64_peak) / 1e9
+        out[w.name] = {"candidates": n, "cells": cells, "cells_32bit": cells_32, "eval_ms": t * 1e3,
+                       "candidates_per_sec": n / t, "events_per_sec": cells / t,
+                       "frac_of_cell_rate_floor": floor_s / t, "best_index": best[0], "best_batch_ns": best[1]}
     # emission: still loaded with the 1024-device workload?  reload it to be explicit
     w = W.config4()
     n, _ = W.count_candidates_and_cells(w.table, w.space)
