@@ -352,6 +352,50 @@ DS_UNROLL(DS_UNROLL_MAIN)
     TailWaves<PP, PP, T, kJit>::run(c, m, free_at, last_f, jt);
 }
 
+// The same schedule with the warm-up and last waves as loops over the wave number (the set of
+// stages that run a forward item is tested per stage at run time) instead of one unrolled copy
+// per wave: an eighth of the code.  Used for the few entries of a table without jitter that
+// cannot take the relative form (m < pp, or a time bound too close to 2^32), where a smaller
+// kernel is worth more than their speed.
+template <int PP, typename T>
+__device__ __forceinline__ void run_1f1b_compact(const ThreadState<PP, T> &c, int m, T (&free_at)[PP])
+{
+    T last_f[PP];
+#pragma unroll
+    for (int d = 0; d < PP; ++d) { free_at[d] = 0; last_f[d] = 0; }
+    const int n_edge = min(PP, m);
+#pragma unroll 1
+    for (int J = 0; J < n_edge; ++J) {           // warm-up wave J: forward items on stages 0 .. PP-1-J
+        T t = 0;
+#pragma unroll
+        for (int d = 0; d < PP; ++d)
+            if (d < PP - J) {
+                t = d == 0 ? (T)(free_at[0] + c.fop[0]) : cell(t, free_at[d], c.fop[d]);
+                free_at[d] = t; last_f[d] = t;
+            }
+    }
+    const JitterTab<PP, T, false> none{nullptr, nullptr, 0};
+    if (m > PP) {
+#pragma unroll 1
+        for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T, false>(c, last_f, none, i);
+#pragma unroll
+        for (int d = 0; d < PP; ++d) free_at[d] = last_f[d];
+    }
+#pragma unroll 1
+    for (int K = n_edge; K >= 1; --K) {          // K waves to go: stages d >= PP-K+1 still run a forward item
+        T t = 0;
+#pragma unroll
+        for (int d = PP - 1; d >= 0; --d) {
+            t = d == PP - 1 ? (T)(free_at[d] + c.bop[d]) : cell(t, free_at[d], c.bop[d]);
+            free_at[d] = t;
+            if (d >= PP - K + 1) {
+                const T f = d == 0 ? (T)(t + c.fop[0]) : cell(last_f[d > 0 ? d - 1 : 0], t, c.fop[d]);
+                free_at[d] = f; last_f[d] = f;
+            }
+        }
+    }
+}
+
 // Shared-memory plan of a block (offsets in int64 words from the dynamic shared base): the
 // prefix rows of every entry of the row; then, when per-entry bucket-lane tables exist, the
 // binomial table of the unranking and the bucket-lane tables of the row's last entries (as many
@@ -673,7 +717,8 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
                     if (kJit || !rel) run_gpipe<PP, T, kJit>(st, m, free_at, jt);
                     else run_gpipe_rel<PP, T>(st, m, free_at);
                 } else {
-                    if (kJit || !rel || m < PP) run_1f1b<PP, T, kJit>(st, m, free_at, jt);
+                    if (kJit) run_1f1b<PP, T, kJit>(st, m, free_at, jt);
+                    else if (!rel || m < PP) run_1f1b_compact<PP, T>(st, m, free_at);
                     else run_1f1b_rel<PP, T>(st, m, free_at);
                 }
                 T batch = 0;
