@@ -58,7 +58,7 @@ constexpr int kMaxRowEntries = 16;      // entries whose scalars are kept in sha
 template <int PP, typename T>
 __host__ __device__ constexpr int thread_kernel_min_blocks()
 {
-    return sizeof(T) == 8 ? (PP >= 16 ? 3 : 4) : (PP >= 16 ? 4 : 8);
+    return sizeof(T) == 8 ? (PP >= 16 ? 3 : 4) : (PP >= 16 ? 5 : 8);
 }
 
 template <typename T> __device__ __forceinline__ T vmax(T a, T b) { return a > b ? a : b; }
