@@ -43,8 +43,8 @@ RECORD_BYTES = 40
 # DRAM read + write bytes per step of the timed workload, from the one-pass ncu counters summarised in
 # profiles/bench_config1_dram_bytes.md.  They describe the kernels as captured: set them to None when
 # an evaluation or emission kernel changes, until the counters are taken again.
-EVAL_TRAFFIC_BYTES = 214_723_840
-EMIT_TRAFFIC_BYTES = 1_696_231_424
+EVAL_TRAFFIC_BYTES = 198_050_304
+EMIT_TRAFFIC_BYTES = 1_696_420_864
 SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32      # issue slots: one warp instruction per scheduler and clock
 
 
