@@ -192,6 +192,24 @@ def test_randomised_spaces_sampled_parity(E, ctx, case):
         assert (sb[sel].cpu().numpy() == obusy).all()
 
 
+def test_many_layers(E, ctx):
+    """200 layers: tables too large to stage in shared memory (bucket-lane tables and binomials
+    are read from global memory), long item templates and one-item runs in emission."""
+    w = W.random_small(77, n_devices=8, gpus_per_node=4, n_layers=200, global_batch=32, mp_max=2, pp_max=4,
+                       m_list=(1, 3, 4, 8), partition_mode=W.PARTITION_ALL, dp_bucket_bytes=30_000, hi=3000)
+    n = load(E, ctx, w)
+    assert n > 10**6
+    batch, sb = eval_all(E, ctx, n)
+    rng = np.random.default_rng(77)
+    idx = np.unique(np.concatenate([rng.integers(0, n, 400), [0, n - 1]]))
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, idx, THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    sel = torch.from_numpy(idx).cuda()
+    assert (batch[sel].cpu().numpy() == ob).all()
+    assert (sb[sel].cpu().numpy() == obusy).all()
+    check_emission(E, ctx, w, [int(idx[0]), int(idx[len(idx) // 2]), int(idx[-1])])
+
+
 def test_ranges_straddle_rows_and_empty(E, ctx):
     w = W.random_small(7, partition_mode=W.PARTITION_ALL)
     n = load(E, ctx, w)
