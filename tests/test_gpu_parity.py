@@ -210,6 +210,22 @@ def test_many_layers(E, ctx):
     check_emission(E, ctx, w, [int(idx[0]), int(idx[len(idx) // 2]), int(idx[-1])])
 
 
+def test_many_microbatches(E, ctx):
+    """m = 1000 and 4096 (the largest the interface takes): thousands of lock-step slots, item
+    runs spanning many blocks in emission."""
+    w = W.random_small(78, n_devices=8, gpus_per_node=4, n_layers=9, global_batch=8192, mp_max=2, pp_max=8,
+                       m_list=(1000, 4096), m_rule=W.M_RULE_CEIL, partition_mode=W.PARTITION_BALANCED,
+                       dp_bucket_bytes=3000, hi=900)
+    n = load(E, ctx, w)
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    assert (batch.cpu().numpy() == ob).all() and (sb.cpu().numpy() == obusy).all()
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(n))
+    pick = [i for i, c in enumerate(cands) if c.pp == 8][:2] + [i for i, c in enumerate(cands) if c.m == 4096 and c.pp == 2][:1]
+    check_emission(E, ctx, w, pick)
+
+
 def test_ranges_straddle_rows_and_empty(E, ctx):
     w = W.random_small(7, partition_mode=W.PARTITION_ALL)
     n = load(E, ctx, w)
