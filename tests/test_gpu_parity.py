@@ -226,6 +226,26 @@ def test_many_microbatches(E, ctx):
     check_emission(E, ctx, w, pick)
 
 
+@pytest.mark.parametrize("n_devices,n_layers,batch", [(1, 1, 1), (1, 3, 4), (2, 1, 2), (2, 2, 6), (4, 3, 4)])
+def test_degenerate_shapes(E, ctx, n_devices, n_layers, batch):
+    """One device, one layer, one sample: spaces of a handful of candidates, every candidate
+    evaluated, selected (k = whole range) and emitted."""
+    w = W.random_small(90 + n_devices + n_layers, n_devices=n_devices, gpus_per_node=min(2, n_devices),
+                       n_layers=n_layers, global_batch=batch, mp_max=4, pp_max=4, m_list=(1, 2, 3, 4),
+                       partition_mode=W.PARTITION_ALL, dp_bucket_bytes=0, hi=300)
+    n = load(E, ctx, w)
+    assert 1 <= n < 200
+    batch_t, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices(w.table, w.space, np.arange(n), replicate=True, pp_stride=w.space.pp_max)
+    assert (batch_t.cpu().numpy() == ob).all() and (sb.cpu().numpy() == obusy).all()
+    order = np.lexsort((np.arange(n), ob))
+    assert E.distsim_argmin(ctx, batch_t, 0, n) == (order[0], ob[order[0]])
+    ki, kt = dev(n), dev(n)
+    E.distsim_topk(ctx, batch_t, 0, n, n, ki, kt)
+    assert (ki.cpu().numpy() == order).all() and (kt.cpu().numpy() == ob[order]).all()
+    check_emission(E, ctx, w, list(range(n)))
+
+
 def test_ranges_straddle_rows_and_empty(E, ctx):
     w = W.random_small(7, partition_mode=W.PARTITION_ALL)
     n = load(E, ctx, w)
