@@ -228,7 +228,9 @@ def distsim_emit_timelines(ctx: Context, d_indices, n: int, d_records, capacity_
                            d_offsets=None, d_busy_ns=None, d_util=None, stream=None) -> int:
     """Returns the number of records needed; raises DistsimError(E_CAPACITY) if
     ``d_records`` is given but too small.  ``d_records`` is an int64 tensor of
-    at least ``5 * capacity_records`` elements (or None for a sizing pass)."""
+    at least ``5 * capacity_records`` elements (or None for a sizing pass).  Offsets, busy
+    times and utilisations are final on return; the records are written in stream order
+    (complete once the work enqueued on the stream has finished)."""
     pi = _dev_ptr(d_indices, "int64", n, "d_indices")
     pr = _dev_ptr(d_records, "int64", 5 * capacity_records, "d_records")
     nn = n * ctx.n_devices
