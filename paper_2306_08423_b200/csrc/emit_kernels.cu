@@ -23,7 +23,9 @@ namespace {
 
 constexpr int kItemThreads = 256;
 constexpr int kMaxTileItems = 256;  // most schedule items per block (a plan picks its own count)
-constexpr int kTileWords = 3872;    // capacity of a block's image of its run, in int64 words
+constexpr int kTileWords = 3872;    // largest capacity of a block's image of its run, in int64 words
+constexpr int kRunWords = 3872;     // run length the plans aim at (three blocks per SM; shorter runs
+                                    // measured slower: the per-block set-up weighs more)
 constexpr int kTileReplicas = 16;   // replicas per block
 constexpr int kBucketThreads = 128;
 constexpr int kBucketRun = 768;     // gradient buckets per shared-memory image (5 words each)
@@ -103,9 +105,11 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
             both = max(both, plan->rf[d] + plan->rb[d]);
         }
         // a run of tile_items items of any mix must fit the image of kTileWords words
-        const int cap = max(1, min(kMaxTileItems, kTileWords / (widest * 5)));
+        // a run aims at kRunWords words (small images: more blocks per SM), holds at least one item
+        const int cap = max(1, min(kMaxTileItems, kRunWords / (widest * 5)));
         const int n_chunks = (2 * en.m + cap - 1) / cap;          // equal runs rather than full ones and a rest
         plan->tile_items = (2 * en.m + n_chunks - 1) / n_chunks;
+        plan->run_words = plan->tile_items * widest * 5;          // no run of this selection is longer
         plan->tmpl_words = both * 5;
     }
 }
@@ -121,7 +125,7 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
     if (index < 0 || index >= v.sc.n_candidates) {
         if ((threadIdx.x & 31) == 0) {
             plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
-            plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0;
+            plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
             atomicCAS(v.status, 0, DISTSIM_E_RANGE);
         }
         return;
@@ -140,7 +144,7 @@ __global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /* the 
     const int t = threadIdx.x, nt = blockDim.x, lane = t & 31, warp = t >> 5;
     const int per = (n + nt - 1) / nt;
     const int b = min(n, t * per), e = min(n, b + per);
-    int64_t s = 0, mt = 0, mb = 0, mw = 0, mk = 0;
+    int64_t s = 0, mt = 0, mb = 0, mw = 0, mk = 0, mr = 0;
     for (int i = b; i < e; ++i) s += plans[i].rec_total;
     // exclusive scan of the per-thread sums over the block: inside warps, then over the warp totals
     int64_t incl = s;
@@ -170,6 +174,7 @@ __global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /* the 
                                   ((reps + kTileReplicas - 1) / kTileReplicas);
             mt = max64(mt, tiles);
             mw = max64(mw, plans[i].tmpl_words);
+            mr = max64(mr, plans[i].run_words);
             mb = max64(mb, (int64_t)plans[i].pp * ((reps + kBucketReplicas - 1) / kBucketReplicas));
             for (int d = 0; d < plans[i].pp; ++d) mk = max64(mk, plans[i].n_buckets[d]);
         }
@@ -178,6 +183,7 @@ __global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /* the 
     if (mb > 0) atomicMax((unsigned long long *)&totals[2], (unsigned long long)mb);
     if (mw > 0) atomicMax((unsigned long long *)&totals[3], (unsigned long long)mw);
     if (mk > 0) atomicMax((unsigned long long *)&totals[4], (unsigned long long)mk);
+    if (mr > 0) atomicMax((unsigned long long *)&totals[5], (unsigned long long)mr);
 }
 
 __global__ void __launch_bounds__(256)
@@ -224,12 +230,13 @@ __device__ __forceinline__ void item_at(int sched, int pp, int m, int d, int s, 
 
 __global__ void __launch_bounds__(kItemThreads)
 emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_t *__restrict__ op_start,
-                  int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */)
+                  int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */,
+                  int cap /* words of one image: even, at least the longest run of any selection */)
 {
     extern __shared__ __align__(16) int64_t dyn_s[];
     int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
-    int64_t *img_b = dyn_s + kTileWords;                // the same word at img_b[x + 1]
-    int64_t *tmpl = dyn_s + 2 * kTileWords + 2;         // [rf*5] forward, then [rb*5] backward
+    int64_t *img_b = dyn_s + cap;                       // the same word at img_b[x + 1]
+    int64_t *tmpl = dyn_s + 2 * cap + 2;                // [rf*5] forward, then [rb*5] backward
     __shared__ int64_t rep_off_s[kTileReplicas];
     __shared__ int64_t start_s[kMaxTileItems];          // start time of each item of the run
     __shared__ int64_t jit_s[kMaxTileItems];            // jitter at the start of each item
@@ -331,7 +338,7 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     __syncthreads();
 
     // ---- the run's image: one warp per item, a word is template word + {0, 0, j, start, start} ----
-    const int total = ioff[n_items];                 // <= kTileWords by the plan's choice of tile_items
+    const int total = ioff[n_items];                 // <= cap by the plans' choice of tile_items
     {
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         const int lane_field = lane - (lane / 5) * 5;
@@ -508,11 +515,12 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
 {
     if (n == 0 || t.item_tiles == 0) return;
     // two images of the run, then the forward and backward item templates of the widest stage
-    const size_t smem = (size_t)(2 * kTileWords + 2 + t.tmpl_words) * sizeof(int64_t);
+    const int cap = (int)((t.run_words + 1) & ~(int64_t)1);
+    const size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
     cudaFuncSetAttribute(emit_items_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int64_t *out = reinterpret_cast<int64_t *>(records);
     emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
-        v, plans, op_start, op_words_per_cand, out);
+        v, plans, op_start, op_words_per_cand, out, cap);
     ++*launches;
     if (t.bucket_tiles > 0 && t.bucket_recs > 0) {
         // an odd number of buckets per image keeps both images 16-byte aligned

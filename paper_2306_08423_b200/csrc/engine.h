@@ -182,6 +182,7 @@ struct EmitPlan {                    // per selected candidate, written by the p
     int32_t bounds[DISTSIM_MAX_PP + 1];
     int32_t tile_items;              // schedule items per block of the record kernel
     int32_t tmpl_words;              // words of the widest stage's forward + backward item templates
+    int32_t run_words;               // upper bound on the words of any run of items of this selection
     int32_t rf[DISTSIM_MAX_PP], rb[DISTSIM_MAX_PP];   // records of one forward / backward item
     int64_t n_buckets[DISTSIM_MAX_PP];
     int64_t stage_recs[DISTSIM_MAX_PP];               // records of one device of stage d
@@ -197,7 +198,8 @@ struct EmitTotals {
     int64_t bucket_tiles;   // most (stage, replica chunk) tiles of any selection's bucket lanes
     int64_t tmpl_words;     // most words of any stage's forward + backward item templates
     int64_t bucket_recs;    // most gradient-bucket records of any stage
-    int64_t pad[3];
+    int64_t run_words;      // most words of any run of items (capacity of the record kernel's images)
+    int64_t pad[2];
 };
 // Plans the n selections: item start times into op_start (op_words_per_cand words each), record
 // counts, offsets / busy / util (each nullable); d_totals: the words of an EmitTotals.
