@@ -92,7 +92,7 @@ const char *distsim_last_error(const distsim_ctx *ctx);
  *                                        ceil(T(k) * k (n-1) / ((k-1) n))  (the paper profiles
  *                                        up to 8 devices and extrapolates, Sec. 4.2)
  *   n_jitter, jitter_*                   fluctuation between micro-batches (the paper's error
- *                                        analysis, Sec. 6.3, blames profiling fluctuation that
+ *                                        analysis, Sec. 5.3, blames profiling fluctuation that
  *                                        accumulates along the stages): with P = n_jitter > 0 the
  *                                        forward (backward) item of micro-batch j on stage d
  *                                        begins with a jitter event of jitter_fwd_ns
@@ -127,7 +127,7 @@ typedef struct {
 int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *h_table);
 
 /*
- * The search space (paper Sec. 5: grid over parallel degrees with dp =
+ * The search space (paper Sec. 6: grid over parallel degrees with dp =
  * GPUs/mp/pp, invalid combinations dropped).  Candidates are numbered in this
  * canonical order, outermost first: mp ascending over powers of two <= mp_max;
  * pp ascending over powers of two <= min(pp_max, n_layers) with mp*pp | N and
@@ -178,7 +178,7 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
                             int64_t *d_batch_ns, int64_t *d_stage_busy_ns);
 
 /*
- * Best strategy of a range (paper Sec. 5: the grid search keeps the fastest):
+ * Best strategy of a range (paper Sec. 6: the grid search keeps the fastest):
  * smallest d_batch_ns[i], ties to the smallest index.  d_batch_ns[i] belongs to
  * candidate first + i.  Results go to host memory; the call synchronises `stream`.
  */

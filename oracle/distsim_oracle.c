@@ -84,7 +84,7 @@ typedef struct {
     const int64_t *jitter_bwd_ns;         /* same for backward items                           */
 } orc_table;
 
-/* The search space (paper Sec. 5: grid search over parallel degrees). */
+/* The search space (paper Sec. 6: grid search over parallel degrees). */
 typedef struct {
     int32_t mp_max, pp_max, n_m;
     const int32_t *m_list;                /* ascending                            */
@@ -222,7 +222,7 @@ static int64_t beta_of(const orc_table *T, int loc) { return loc ? T->beta_inter
 /*   m ascending over the valid entries of m_list;                             */
 /*   stage partition in lexicographic order of (c_1..c_{pp-1});                */
 /*   schedule: GPipe, then 1F1B, then asynchronous 1F1B.                       */
-/* The paper's own grid (Sec. 5) walks mp and pp over powers of two and takes  */
+/* The paper's own grid (Sec. 6) walks mp and pp over powers of two and takes  */
 /* dp = GPUs/mp/pp, dropping the invalid combinations.                         */
 
 static int valid_m(const orc_space *S, int64_t Bp, int64_t m)
@@ -366,7 +366,7 @@ static int64_t union_measure(const orc_list *l)
  * orc_simulate
  *   replicate    1: keep a list for every one of the N devices;
  *                0: keep only the device (r=0, q=0) of every stage (pp lists).
- *   reverse_scan 0: first_available scans stages 0..pp-1; 1: pp-1..0.  The
+ *   reverse_scan 0: the pick step scans stages 0..pp-1; 1: pp-1..0.  The
  *                result must not depend on it (each item's start depends only
  *                on its two predecessors).
  */
@@ -475,8 +475,9 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
         int64_t remaining = (int64_t)pp * n_ops;
         for (int d = 0; d < pp; ++d) { head[d] = 0; device_free[d] = 0; }
         while (remaining > 0) {
-            /* first_available: the first device whose next item has its data ready; the item
-             * belongs to virtual stage vs = chunk * pp + d (vs = d without chunks) */
+            /* Pick step of Algorithm 1 (Sec. 4.3): the first device whose next schedule item
+             * has its input data ready and its micro-batch matched; the item belongs to virtual
+             * stage vs = chunk * pp + d (vs = d without chunks) */
             int pick = -1; int64_t t = 0;
             for (int s = 0; s < pp && pick < 0; ++s) {
                 int d = reverse_scan ? pp - 1 - s : s;
@@ -494,11 +495,12 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
             const orc_op o = ops[(int64_t)d * n_ops + head[d]];
             const int vs = o.chunk * pp + d;
             const int la = x->bounds[vs], le = x->bounds[vs + 1];   /* the item's layers [la, le) */
-            /* e <- MAP[l]: the stage's layers, each a computation event followed by
-             * its all-reduce event (mp > 1) and its all-to-all event (expert layer,
-             * dp > 1); then e_comm, the transfer to the neighbouring stage. */
+            /* Look-up step of Algorithm 1: the events MP modeling mapped the item's layers to -
+             * per layer a computation event, then its all-reduce event (mp > 1) and its
+             * all-to-all event (expert layer, dp > 1) - followed by the communication event of
+             * the item, the transfer to the neighbouring stage. */
             int n = 0;
-            /* Fluctuation between micro-batches (the paper's error analysis, Sec. 6.3, blames
+            /* Fluctuation between micro-batches (the paper's error analysis, Sec. 5.3, blames
              * profiling fluctuation that accumulates along the stages): when a jitter table is
              * given, the item of micro-batch j on stage d begins with a jitter event of
              * [j mod P][d] ns, before its first computation event. */
@@ -530,7 +532,7 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
             for (int q = 0; q < mp_lists; ++q)          /* every device of the MP group */
                 for (int i = 0; i < n; ++i)
                     if ((e = list_push(&F[d * mp_lists + q], tmp[i])) != ORC_OK) goto fail;
-            ++head[d]; --remaining;                      /* S <- S - st */
+            ++head[d]; --remaining;                      /* the item leaves the schedule */
         }
     }
 

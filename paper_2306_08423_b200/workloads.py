@@ -11,7 +11,7 @@ degree and micro-batch size, i.e. the operator's parameters and input shape that
 key an event - it gives each layer's forward and backward computation time in
 integer nanoseconds, plus the alpha-beta constants that replace profiled
 communication events.  The workloads below stand in for the paper's BERT-Large /
-GPT-2 / T5 / BERT-exLarge / 145B-GPT profiles (Sec. 6-7), which are not
+GPT-2 / T5 / BERT-exLarge / 145B-GPT profiles (Sec. 5-6), which are not
 available; shapes, sizes and value distributions follow the five benchmark
 configurations.
 
@@ -275,7 +275,7 @@ def config4(seed: int = 2) -> Workload:
 
 
 def paper_grid(seed: int = 7) -> Workload:
-    """The shape of the paper's own strategy search (Sec. 5): 16 GPUs on 4 nodes, a 48-layer
+    """The shape of the paper's own strategy search (Sec. 6): 16 GPUs on 4 nodes, a 48-layer
     transformer, global batch 16, every degree in {1, 2, 4, 8, 16}, with all-reduces above 8
     devices extrapolated from the 8-device time (Sec. 4.2).  Event times are synthetic."""
     space = SearchSpace(mp_max=16, pp_max=16, m_list=[1, 2, 4, 8, 16], m_rule=M_RULE_DIVIDES,

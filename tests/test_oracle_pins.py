@@ -84,7 +84,7 @@ def test_paper_grid_workload_shape():
         len([m for m in (1, 2, 4, 8, 16) if (16 // dp) % m == 0])
         for mp in (1, 2, 4, 8, 16) for pp in (1, 2, 4, 8, 16) if mp * pp <= 16 for dp in [16 // (mp * pp)])
     cands = oracle.enumerate_at(w.table, w.space, np.arange(oracle.count(w.table, w.space)))
-    assert len({(c.mp, c.pp) for c in cands}) == 15           # Sec. 5: 15 valid settings of 25
+    assert len({(c.mp, c.pp) for c in cands}) == 15           # Sec. 6: 15 valid settings of 25
 
 
 def test_p2p_and_all_to_all_formulas():
@@ -281,7 +281,7 @@ def test_interleaved_brute_force_and_invariants(w, cand):
     for d in range(cand.pp):
         got = [tuple(x) for x in r.records[r.offsets[d]:r.offsets[d + 1]].tolist()]
         assert got == lanes[d], (cand, d)
-    # the scan order of first_available does not matter; replicas are identical
+    # the scan order of the pick step (Algorithm 1) does not matter; replicas are identical
     assert oracle.simulate(T, cand, replicate=False, reverse_scan=True).batch_ns == r.batch_ns
     full = oracle.simulate(T, cand, replicate=True)
     assert full.batch_ns == r.batch_ns
@@ -414,6 +414,82 @@ def test_busy_equals_sum_of_durations_without_overlap():
             assert r.busy_ns[d] == int((rec[:, 4] - rec[:, 3]).sum())
 
 
+def _coverage_measure(rec):
+    """Measure of the union of the records' [start, end) intervals by a coverage count over the
+    distinct end points (no sorting of intervals, no merging)."""
+    pts = np.unique(np.concatenate([rec[:, 3], rec[:, 4]]))
+    diff = np.zeros(len(pts) + 1, np.int64)
+    np.add.at(diff, np.searchsorted(pts, rec[:, 3]), 1)
+    np.add.at(diff, np.searchsorted(pts, rec[:, 4]), -1)
+    covered = np.cumsum(diff)[:-1] > 0                      # segment [pts[i], pts[i+1])
+    return int((np.diff(pts) * covered[:-1]).sum())
+
+
+def _merge_that_forgets_the_running_end(rec):
+    """The plausible mistake in an interval merge: the running end is overwritten by the next
+    interval's end instead of the later of the two."""
+    iv = sorted((int(s), int(e)) for s, e in rec[:, 3:5])
+    total, lo, hi = 0, iv[0][0], iv[0][1]
+    for s, e in iv[1:]:
+        if s > hi:
+            total += hi - lo; lo, hi = s, e
+        else:
+            hi = e
+    return total + hi - lo
+
+
+def test_busy_is_the_union_of_intervals_when_buckets_overlap_the_main_lane():
+    # Sec. 3.2 activity time under DP modeling with overlapped buckets (dp > 1): buckets start
+    # inside main-lane events, so the union is smaller than the sum of the durations.
+    n_nested = n_strict = 0
+    for w, c in _cases(range(70, 82), dp_overlap=1, dp_bucket_bytes=900, n_layers=6):
+        if c.dp == 1 or c.sched == 2:
+            continue
+        r = oracle.simulate(w.table, c, replicate=False)
+        for d in range(c.pp):
+            rec = r.records[r.offsets[d]:r.offsets[d + 1]]
+            main, bk = rec[rec[:, 0] != 8], rec[rec[:, 0] == 8]
+            want = _coverage_measure(rec)
+            assert r.busy_ns[d] == want, (c, d)
+            # the same on a boolean time grid when it is small enough
+            if rec[:, 4].max() < 4_000_000:
+                grid = np.zeros(int(rec[:, 4].max()), bool)
+                for s, e in rec[:, 3:5]:
+                    grid[s:e] = True
+                assert int(grid.sum()) == want
+            # main lane without gaps after its first event, bucket lane busy after the main lane
+            # ends: activity = sum of the main-lane durations + what the buckets add past its end
+            main_sum = int((main[:, 4] - main[:, 3]).sum())
+            dp_end = int(bk[:, 4].max()) if len(bk) else 0
+            assert r.busy_ns[d] == main_sum + max(0, dp_end - int(main[:, 4].max())), (c, d)
+            n_strict += r.busy_ns[d] < int((rec[:, 4] - rec[:, 3]).sum())
+            n_nested += _merge_that_forgets_the_running_end(rec) != want
+    assert n_strict >= 10 and n_nested >= 5      # the cases do exercise overlap and nesting
+
+
+def test_hand_worked_bucket_overlap_examples():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "worked_bucket_overlap_examples.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) == 4
+    for name, sched, overlap, batch, *busy in rows:
+        if name == "W4":
+            T = make_table([1, 1], [10, 10], n_devices=2, gpus_per_node=1, global_batch=2, classes=[(1, 1)],
+                           grad=np.array([100, 200], np.int64), dp_bucket_bytes=100, dp_overlap=int(overlap),
+                           alpha_intra_ns=50, beta_intra=1, alpha_inter_ns=1, beta_inter=100)
+            c = Candidate(1, 1, 2, 1, int(sched), (0, 2))
+        else:
+            T = make_table([1, 1], [2, 2], n_devices=4, gpus_per_node=2, global_batch=4, classes=[(1, 1)],
+                           grad=np.array([100, 200], np.int64), dp_bucket_bytes=100, dp_overlap=int(overlap),
+                           alpha_intra_ns=7, beta_intra=1, alpha_inter_ns=1, beta_inter=100)
+            c = Candidate(1, 2, 2, 2, int(sched), (0, 1, 2))
+        r = oracle.simulate(T, c, replicate=False)
+        assert r.batch_ns == int(batch), (name, sched)
+        assert r.busy_ns.tolist() == [int(x) for x in busy], (name, sched)
+        assert r.util.tolist() == [int(x) / int(batch) for x in busy]
+        full = oracle.simulate(T, c, replicate=True)
+        assert full.busy_ns.tolist() == [int(busy[(k // c.mp) % c.pp]) for k in range(T.n_devices)]
+
+
 def test_main_lane_is_serial_and_bucket_lane_is_serial():
     for w, c in _cases(range(40, 44)):
         r = oracle.simulate(w.table, c, replicate=False)
@@ -499,7 +575,7 @@ def test_bucket_chain_properties():
 # enumeration pins
 
 def test_paper_grid_has_15_valid_settings():
-    # Sec. 5: degrees {1,2,4,8,16} on 16 GPUs -> 15 valid (mp, pp) settings, dp = GPUs/mp/pp
+    # Sec. 6: degrees {1,2,4,8,16} on 16 GPUs -> 15 valid (mp, pp) settings, dp = GPUs/mp/pp
     sp = W.SearchSpace(mp_max=16, pp_max=16, m_list=[1], sched_mask=1)
     T = make_table([1] * 48, [1] * 48, n_devices=16, gpus_per_node=4, global_batch=16, classes=[(1, 1)])
     n = oracle.count(T, sp)
@@ -510,7 +586,7 @@ def test_paper_grid_has_15_valid_settings():
 
 
 def test_paper_per_stage_example_item_counts():
-    # Sec. 6.4: "2m4p1d", 4 micro-batches -> 32 forward and backward items, 4 (each) per GPU
+    # Sec. 5.4: "2m4p1d", 4 micro-batches -> 32 forward and backward items, 4 (each) per GPU
     T = make_table([5] * 8, [9] * 8, n_devices=8, gpus_per_node=4, global_batch=4, classes=[(2, 1)],
                    seq=4, hidden=4)
     for sched in (0, 1):
@@ -525,7 +601,7 @@ def test_paper_per_stage_example_item_counts():
             assert nf == 4 and nb == 4
             tot_f += nf; tot_b += nb
         assert tot_f == 32 and tot_b == 32
-        # the two GPUs of an MP group behave identically (Sec. 6.4)
+        # the two GPUs of an MP group behave identically (Sec. 5.4)
         for k in range(0, 8, 2):
             assert (r.records[r.offsets[k]:r.offsets[k + 1]] == r.records[r.offsets[k + 1]:r.offsets[k + 2]]).all()
 
