@@ -63,8 +63,9 @@ def oracle_sample_rate(w, n_total, sample, threads):
     import oracle
     idx = np.unique(np.linspace(0, n_total - 1, sample).astype(np.int64))
     t0 = time.perf_counter()
-    oracle.eval_indices_parallel(w.table, w.space, idx, threads, replicate=False)
+    values, _ = oracle.eval_indices_parallel(w.table, w.space, idx, threads, replicate=False)
     dt = time.perf_counter() - t0
+    oracle_sample_rate.last = (idx, values)            # what the oracle computed, for the caller to compare
     return len(idx) / dt, dt, len(idx)
 
 
@@ -313,11 +314,14 @@ def run_ours(args):
 
     # ---- rooflines -----------------------------------------------------------------------------
     # integer peaks, measured now with dependency-free instruction streams
+    from paper_2306_08423_b200 import probes
+    sink = torch.zeros(1, dtype=torch.int64, device=dev)
+
     def probe(mode):
         pe0, pe1 = ev(), ev()
-        E.distsim_int_issue_probe(ctx, 148 * 16, 2000, mode)
+        probes.distsim_bench_int_issue_probe(148 * 16, 2000, mode, sink)
         pe0.record(stream)
-        ops = E.distsim_int_issue_probe(ctx, 148 * 16, 20000, mode)
+        ops = probes.distsim_bench_int_issue_probe(148 * 16, 20000, mode, sink)
         pe1.record(stream)
         torch.cuda.synchronize()
         return ops / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
@@ -326,7 +330,7 @@ def run_ours(args):
     cell32_fused_peak = probe(4) / 2                                                 # G cells/s, one fused add-max per cell
     cell32_peak = max(cell32_peak, cell32_fused_peak)
     sm_mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
-    cells_all, cells_32 = E.distsim_space_cells(ctx)
+    cells_all, cells_32 = E.distsim_testing_space_cells(ctx)
     assert cells_all == cells
     eval_s = statistics.mean(eval_ms) * 1e-3
     alg_ops = cells_32 * INT_OPS_PER_CELL_32 + (cells - cells_32) * INT_OPS_PER_CELL_64
@@ -390,6 +394,7 @@ def run_ours(args):
         "gpu_launches": launches, "clocks": clocks,
     }
 
+    failed = False
     if world == 1:
         if not args.no_workloads:
             line["workloads"] = other_workloads(E, ctx, torch, dev, peaks, cell32_peak, cell64_peak)
@@ -403,10 +408,21 @@ def run_ours(args):
             rate, dt, ns = oracle_sample_rate(w, n_total, sample, threads)
             line["cpu_baseline"] = {"value": rate, "unit": "candidates/s", "cores": threads, "kind": "oracle",
                                     "sample": f"{ns} evenly strided candidates of {n_total}, {dt:.1f} s"}
+            # the batch array the timed steps wrote, against the oracle's values at the same indices
+            o_idx, o_val = oracle_sample_rate.last
+            got = batch[torch.from_numpy(o_idx).to(dev)].cpu().numpy()
+            mismatches = int((got != o_val).sum())
+            o_order = np.lexsort((o_idx, o_val))
+            line["verified"] = {"candidates": int(len(o_idx)), "mismatches": mismatches,
+                                "best_not_above_sample_minimum": bool(best[1] <= int(o_val[o_order[0]])),
+                                "what": "batch times of the timed steps vs the CPU oracle, bit-exact"}
+            failed = mismatches != 0 or not line["verified"]["best_not_above_sample_minimum"]
     ctx.close()
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+    if world == 1 and not args.no_cpu and failed:
+        sys.exit(1)
 
 
 def other_workloads(E, ctx, torch, dev, peaks, cell32_peak, cell64_peak):
@@ -430,7 +446,7 @@ def other_workloads(E, ctx, torch, dev, peaks, cell32_peak, cell64_peak):
             if it >= 3:
                 times.append(e0.elapsed_time(e1) * 1e-3)
         t = statistics.median(times)
-        _, cells_32 = E.distsim_space_cells(ctx)
+        _, cells_32 = E.distsim_testing_space_cells(ctx)
         # time the cells alone would take at this device's measured 32-bit / 64-bit cell rates
         floor_s = (cells_32 / cell32_peak + (cells - cells_32) / cell64_peak) / 1e9
         out[w.name] = {"candidates": n, "cells": cells, "cells_32bit": cells_32, "eval_ms": t * 1e3,
@@ -480,6 +496,8 @@ def profile_case(name):
     eval1m128 - the m = 128 entry of the same row (1 M candidates, 4.0e9 cells)
     eval1m1 - the m = 1 entry of the same row (1 M candidates: unranking and set-up only)
     eval3  - evaluation of the whole 256-device MoE workload (650 k candidates)
+    eval2  - evaluation of the whole 1024-device workload (4 176 candidates, long pipelines)
+    eval2pp64 - the pp = 64 rows of the same workload (lock-step kernel, two warps per candidate)
     emit4  - emission of 16 of the fastest candidates of the 1024-device workload (~1.9 GB)
     emit1  - emission of the 1024 fastest candidates of the 64-device workload (~1.8 GB)
     emit4x128 - as emit4 for 128 candidates, one call of the benchmark's size (~10 GB; for
@@ -488,12 +506,19 @@ def profile_case(name):
     from paper_2306_08423_b200 import engine as E
     torch.cuda.set_device(0)
     ctx = E.Context(0)
-    if name in ("eval1", "eval1m1", "eval1m128", "eval3"):
-        w = W.config1() if name != "eval3" else W.config3()
+    if name in ("eval1", "eval1m1", "eval1m128", "eval3", "eval2", "eval2pp64"):
+        w = {"eval3": W.config3, "eval2": W.config2, "eval2pp64": W.config2}.get(name, W.config1)()
         E.distsim_load_event_table(ctx, w.table)
         n = E.distsim_set_space(ctx, w.space)
         first, count = 0, n
-        if name != "eval3":
+        if name == "eval2pp64":
+            # the first pp = 64 row (mp = 1): 256 micro-batch counts x 2 schedules
+            off = 0
+            for mp, pp, dp, ms, parts, n_sched in W.space_shape(w.table, w.space):
+                if (mp, pp) == (1, 64):
+                    first, count = off, len(ms) * parts * n_sched
+                off += len(ms) * parts * n_sched
+        elif name in ("eval1", "eval1m1", "eval1m128"):
             # whole entries of the (mp = 1, pp = 16) row, 980 628 candidates each:
             # eval1 m = 16 and 32, eval1m128 m = 128
             off = 0
@@ -534,7 +559,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-workloads", action="store_true", help="skip the per-workload summary")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
-    ap.add_argument("--profile-case", default=None, help="eval1 | eval1m1 | eval1m128 | eval3 | emit1 | emit4 | emit4x128: small run for ncu")
+    ap.add_argument("--profile-case", default=None, help="eval1 | eval1m1 | eval1m128 | eval2 | eval2pp64 | eval3 | emit1 | emit4 | emit4x128: small run for ncu")
     args = ap.parse_args()
     if args.profile_case:
         profile_case(args.profile_case)

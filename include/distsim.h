@@ -23,6 +23,14 @@
  *   - All times are int64 nanoseconds.  A context is not thread-safe: use one
  *     per host thread.
  *   - There is no CPU fallback: without a CUDA device distsim_create fails.
+ *   - DISTSIM_E_TIMEOUT.  Kernels stage their tables into shared memory with bulk copies and
+ *     wait for them a bounded number of times.  A block whose wait gives up reads the same
+ *     tables from global memory instead, so its results are exact.  The stall is reported by
+ *     the next synchronising call (distsim_argmin, distsim_emit_timelines), which still writes
+ *     all its outputs and then returns DISTSIM_E_TIMEOUT: the code tells the caller that the
+ *     device's copy engine stalled, not that the outputs are wrong.  Only if a block's second,
+ *     equally bounded wait gives up too (a copy may then still be in flight) does that call
+ *     write nothing; distsim_last_error says which of the two happened.
  */
 #ifndef DISTSIM_H
 #define DISTSIM_H
@@ -45,7 +53,7 @@ enum {
     DISTSIM_E_CAPACITY = -4,   /* caller's output buffer too small                  */
     DISTSIM_E_OVERFLOW = -5,   /* a time or count bound does not fit 62 bits        */
     DISTSIM_E_CUDA = -6,       /* a CUDA runtime call failed                        */
-    DISTSIM_E_TIMEOUT = -7,    /* a bounded device-side wait gave up                */
+    DISTSIM_E_TIMEOUT = -7,    /* a bounded device-side wait gave up (see below)    */
     DISTSIM_E_UNSUPPORTED = -8 /* e.g. degrees that are not powers of two           */
 };
 
@@ -215,7 +223,9 @@ typedef struct { int64_t kind, layer, microbatch, start_ns, end_ns; } distsim_re
  *                                  intervals) and busy / batch time
  *   h_total_records                out (host): records needed
  * If capacity_records is too small nothing is written to d_records and the call
- * returns DISTSIM_E_CAPACITY with *h_total_records set.  The call synchronises `stream` once,
+ * returns DISTSIM_E_CAPACITY with *h_total_records set.  The indices are read from device
+ * memory so that the output of distsim_topk feeds this call without a trip through the host.
+ * The call synchronises `stream` once,
  * after planning, to size the output (that is when *h_total_records, d_offsets, d_busy_ns and
  * d_util are final); the record kernels are then enqueued and the call returns without waiting
  * for them: d_records is complete when the work enqueued on `stream` so far has finished.  The
@@ -226,6 +236,19 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
                            distsim_record *d_records, int64_t capacity_records,
                            int64_t *d_offsets, int64_t *d_busy_ns, double *d_util,
                            int64_t *h_total_records);
+
+/*
+ * Order-sensitive 64-bit checksum of every device's record stream (the paper has no counterpart:
+ * a way to check emitted timelines, e.g. after they have been moved, without comparing gigabytes).
+ * List k holds the records [d_offsets[k], d_offsets[k+1]) of d_records, as written by
+ * distsim_emit_timelines (n_lists = n * N).  With w_0 .. w_{5r-1} the int64 words of its r
+ * records in order, d_checksums[k] = sum over i of mix(w_i + (i + 1) * 0x9E3779B97F4A7C15) modulo
+ * 2^64, where mix(z) is the SplitMix64 finaliser: z ^= z >> 30; z *= 0xBF58476D1CE4E5B9;
+ * z ^= z >> 27; z *= 0x94D049BB133111EB; z ^= z >> 31.
+ *   d_records, d_offsets [n_lists + 1] in; d_checksums [n_lists] out.  Asynchronous on `stream`.
+ */
+int distsim_checksum_timelines(distsim_ctx *ctx, void *stream, const distsim_record *d_records,
+                               const int64_t *d_offsets, int64_t n_lists, uint64_t *d_checksums);
 
 /*
  * Whole search from host memory: loads the table and space, evaluates every
@@ -263,30 +286,6 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table,
 #define DISTSIM_TOPK_STATIC_MAX_K 1024
 int distsim_topk_static(void *stream, const int64_t *d_batch_ns, int64_t first, int64_t count,
                         int32_t k, int64_t *d_indices, int64_t *d_times);
-
-/*
- * Measurement helper (no counterpart in the paper): enqueues a kernel of `blocks` x 256 threads
- * that issues a dependency-free stream of integer work, `iters` rounds per thread, and stores
- * the total instruction count (threads x instructions) in *h_ops.  mode 0: 16 32-bit add / xor
- * instructions per round; mode 1: 8 recurrence cells x = max(x, y) + c on int64 per round,
- * counted as 6 instructions each; mode 2: 16 32-bit compare / select instructions per round;
- * mode 3: 8 recurrence cells on uint32 per round, counted as 2 instructions each; mode 4: the
- * same cells in the form x = max(x + c, y), issued as one fused add-max instruction each (still
- * counted as 2).  Timed by the caller with events on `stream`, it gives the device's
- * plain-integer issue rate under the clocks of the moment.  Asynchronous.
- */
-int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t mode, int32_t blocks,
-                            int32_t iters, int64_t *h_ops);
-
-/*
- * Reporting helper: recurrence cells of the current space (a candidate has 2 m pp cells, one per
- * schedule item), and how many of them belong to entries whose time bound is below 2^32, which
- * the engine may evaluate in 32-bit arithmetic (exactly).  Host outputs.
- */
-int distsim_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32bit);
-
-/* Number of kernels this context has launched so far (for launch accounting). */
-int64_t distsim_launch_count(const distsim_ctx *ctx);
 
 #ifdef __cplusplus
 }

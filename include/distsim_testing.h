@@ -1,0 +1,40 @@
+/*
+ * distsim_testing.h -- hooks into a context for the test-suite and the benchmark's accounting.
+ * They are exported by the engine's library because they need the context, but they are not
+ * part of its stable ABI; the paper has no counterpart for any of them.
+ */
+#ifndef DISTSIM_TESTING_H
+#define DISTSIM_TESTING_H
+
+#include <stdint.h>
+
+#include "distsim.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/*
+ * Sets how often the evaluation kernels poll, in their FIRST wait, for the bulk copies that
+ * stage tables into shared memory (default 65 536).  With 0 that wait gives up at once: every
+ * block takes the path a stalled copy engine would force - it records the stall, waits for the
+ * copy once more with the full limit (so nothing is in flight when the block goes on) and reads
+ * its tables from global memory.  Results stay exact; the next synchronising call returns
+ * DISTSIM_E_TIMEOUT after writing its outputs.  Nothing hangs, traps or faults in either setting.
+ */
+int distsim_testing_set_stage_wait_polls(distsim_ctx *ctx, int32_t polls);
+
+/* Number of kernels this context has launched so far (launch accounting of the benchmark). */
+int64_t distsim_testing_launch_count(const distsim_ctx *ctx);
+
+/*
+ * Recurrence cells of the current space (a candidate has 2 m pp cells, one per schedule item),
+ * and how many of them belong to entries that the engine evaluates in 32-bit arithmetic
+ * (exactly: their time bound is below 2^32).  Host outputs.
+ */
+int distsim_testing_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32bit);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DISTSIM_TESTING_H */

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "engine.h"
+#include "../../include/distsim_testing.h"
 
 using namespace distsim;
 
@@ -68,6 +69,7 @@ struct distsim_ctx {
     std::vector<int64_t> binom;
     int64_t time_bound = 0;
     int64_t op_words_per_cand = 0;
+    int32_t stage_polls = 1 << 16;        // polls of the first wait for staged tables
     DevBuf d_rows, d_entries, d_etf, d_etb, d_nb, d_tp, d_binom, d_dt, d_pfb32, d_dt32;
     bool have_dt = false, have_narrow = false;
 
@@ -93,6 +95,7 @@ struct distsim_ctx {
         v.next_grad = d_next_grad.as<int32_t>(); v.pe = d_pe.as<int32_t>();
         v.jsum = tc.n_jitter > 0 ? d_jsum.as<int64_t>() : nullptr;
         v.status = d_status.as<int32_t>();
+        v.stage_polls = stage_polls;
         return v;
     }
     SelectScratch select_scratch() const
@@ -142,8 +145,14 @@ int upload(distsim_ctx *ctx, DevBuf &b, const T *src, size_t n, const char *what
     return DISTSIM_OK;
 }
 
-// Reads and clears the device status word; synchronises the stream.
-int read_status(distsim_ctx *ctx, cudaStream_t s)
+const char *const kTimeoutText =
+    "a bounded device-side wait for a bulk copy gave up; the affected blocks read their tables from "
+    "global memory instead, so the outputs are exact and have been written";
+
+// Reads and clears the device status word; synchronises the stream.  A wait that gave up while
+// the copy still completed before its block went on is advisory: *stalled is set and DISTSIM_OK
+// returned, so that the caller can finish its work and report DISTSIM_E_TIMEOUT with valid outputs.
+int read_status(distsim_ctx *ctx, cudaStream_t s, bool *stalled)
 {
     int32_t *st = reinterpret_cast<int32_t *>(ctx->h_pinned + 4);
     CU(cudaMemcpyAsync(st, ctx->d_status.p, sizeof(int32_t), cudaMemcpyDeviceToHost, s), "status read");
@@ -151,8 +160,9 @@ int read_status(distsim_ctx *ctx, cudaStream_t s)
     const int32_t code = *st;
     if (code != 0) {
         cudaMemsetAsync(ctx->d_status.p, 0, sizeof(int32_t), s);
-        if (code == DISTSIM_E_TIMEOUT)
-            return fail(ctx, code, "a bounded device-side wait gave up (the affected blocks read their tables from global memory instead)");
+        if (code == DISTSIM_E_TIMEOUT) { *stalled = true; return DISTSIM_OK; }
+        if (code == kStatusCopyPending)
+            return fail(ctx, DISTSIM_E_TIMEOUT, "a bulk copy into shared memory never completed: results computed on this device since may be wrong");
         if (code == DISTSIM_E_RANGE) return fail(ctx, code, "candidate index out of range");
         return fail(ctx, code, "device reported an error");
     }
@@ -222,7 +232,7 @@ void distsim_destroy(distsim_ctx *ctx)
 
 const char *distsim_last_error(const distsim_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
-int64_t distsim_launch_count(const distsim_ctx *ctx) { return ctx ? ctx->launches : 0; }
+int64_t distsim_testing_launch_count(const distsim_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
 int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *t)
 {
@@ -530,10 +540,11 @@ int distsim_argmin(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, in
     launch_argmin(s, d_batch_ns, count, ctx->time_bound, ctx->select_scratch(), ctx->d_result.as<int64_t>(), &ctx->launches);
     CU(cudaGetLastError(), "argmin launch");
     CU(cudaMemcpyAsync(ctx->h_pinned, ctx->d_result.p, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, s), "argmin readback");
-    if (int rc = read_status(ctx, s)) return rc;          // synchronises
+    bool stalled = false;
+    if (int rc = read_status(ctx, s, &stalled)) return rc;          // synchronises
     *h_best_batch_ns = ctx->h_pinned[0];
     *h_best_index = first + ctx->h_pinned[1];
-    return DISTSIM_OK;
+    return stalled ? fail(ctx, DISTSIM_E_TIMEOUT, kTimeoutText) : DISTSIM_OK;
 }
 
 int distsim_topk(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int64_t first,
@@ -571,14 +582,29 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     static_assert(sizeof(EmitTotals) == 8 * sizeof(int64_t), "totals occupy the second half of the pinned words");
     const EmitTotals *totals = reinterpret_cast<const EmitTotals *>(ctx->h_pinned + 8);
     CU(cudaMemcpyAsync(ctx->h_pinned + 8, ctx->d_totals.p, sizeof(EmitTotals), cudaMemcpyDeviceToHost, s), "totals readback");
-    if (int rc = read_status(ctx, s)) return rc;       // synchronises
+    bool stalled = false;
+    if (int rc = read_status(ctx, s, &stalled)) return rc;       // synchronises
     *h_total_records = totals->records;
-    if (!d_records) return DISTSIM_OK;
-    if (totals->records > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");
-    launch_emit_records(s, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
-                        ctx->op_words_per_cand, *totals, d_records, &ctx->launches);
-    CU(cudaGetLastError(), "emission launch");
-    return DISTSIM_OK;                                 // the records are written in stream order
+    if (d_records) {
+        if (totals->records > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");
+        launch_emit_records(s, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
+                            ctx->op_words_per_cand, *totals, d_records, &ctx->launches);
+        CU(cudaGetLastError(), "emission launch");
+    }
+    // the records are written in stream order
+    return stalled ? fail(ctx, DISTSIM_E_TIMEOUT, kTimeoutText) : DISTSIM_OK;
+}
+
+int distsim_checksum_timelines(distsim_ctx *ctx, void *stream, const distsim_record *d_records,
+                               const int64_t *d_offsets, int64_t n_lists, uint64_t *d_checksums)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!d_records || !d_offsets || !d_checksums) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (n_lists < 0) return fail(ctx, DISTSIM_E_ARG, "negative list count");
+    if (int rc = set_device(ctx)) return rc;
+    launch_checksum_lists(static_cast<cudaStream_t>(stream), d_records, d_offsets, n_lists, d_checksums, &ctx->launches);
+    CU(cudaGetLastError(), "checksum launch");
+    return DISTSIM_OK;
 }
 
 int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table, const distsim_space *h_space,
@@ -607,7 +633,7 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table, co
     return distsim_argmin(ctx, nullptr, d_batch, 0, n, h_best_index, h_best_batch_ns);
 }
 
-int distsim_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32bit)
+int distsim_testing_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32bit)
 {
     if (!ctx) return DISTSIM_E_ARG;
     if (!h_cells || !h_cells_32bit) return fail(ctx, DISTSIM_E_ARG, "null argument");
@@ -627,14 +653,11 @@ int distsim_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32b
     return DISTSIM_OK;
 }
 
-int distsim_int_issue_probe(distsim_ctx *ctx, void *stream, int32_t mode, int32_t blocks, int32_t iters, int64_t *h_ops)
+int distsim_testing_set_stage_wait_polls(distsim_ctx *ctx, int32_t polls)
 {
     if (!ctx) return DISTSIM_E_ARG;
-    if (!h_ops || blocks < 1 || iters < 1 || mode < 0 || mode > 4) return fail(ctx, DISTSIM_E_ARG, "bad probe arguments");
-    if (int rc = set_device(ctx)) return rc;
-    *h_ops = launch_int_issue_probe(static_cast<cudaStream_t>(stream), mode, blocks, iters,
-                                    ctx->d_result.as<int64_t>() + 4, &ctx->launches);
-    CU(cudaGetLastError(), "probe launch");
+    if (polls < 0) return fail(ctx, DISTSIM_E_ARG, "negative poll count");
+    ctx->stage_polls = polls;
     return DISTSIM_OK;
 }
 

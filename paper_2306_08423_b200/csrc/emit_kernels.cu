@@ -491,7 +491,50 @@ emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *_
     }
 }
 
+// Order-sensitive 64-bit checksum of every device's record stream: the sum over the stream's
+// words w_i (five per record, i counted from the start of the device's list) of
+// mix(w_i + (i + 1) * 0x9E3779B97F4A7C15) modulo 2^64, mix being the SplitMix64 finaliser.  Moving,
+// dropping or altering a word changes the sum.  One block per list.
+__device__ __forceinline__ uint64_t mix64(uint64_t z)
+{
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+__global__ void __launch_bounds__(256)
+checksum_lists_kernel(const int64_t *__restrict__ words, const int64_t *__restrict__ offsets, int64_t n_lists,
+                      unsigned long long *__restrict__ out)
+{
+    __shared__ unsigned long long part[8];
+    for (int64_t list = blockIdx.x; list < n_lists; list += gridDim.x) {
+        const int64_t w0 = offsets[list] * 5, n = (offsets[list + 1] - offsets[list]) * 5;
+        unsigned long long acc = 0;
+        for (int64_t i = threadIdx.x; i < n; i += blockDim.x)
+            acc += mix64((uint64_t)__ldcs(words + w0 + i) + (uint64_t)(i + 1) * 0x9E3779B97F4A7C15ull);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long sum = 0;
+            for (int k = 0; k < 8; ++k) sum += part[k];
+            out[list] = sum;
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace
+
+void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const int64_t *offsets, int64_t n_lists,
+                           uint64_t *out, int64_t *launches)
+{
+    if (n_lists <= 0) return;
+    const unsigned grid = (unsigned)(n_lists < (1 << 20) ? n_lists : (1 << 20));
+    checksum_lists_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const int64_t *>(records), offsets, n_lists,
+                                               reinterpret_cast<unsigned long long *>(out));
+    ++*launches;
+}
 
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand,
@@ -517,7 +560,7 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
     // two images of the run, then the forward and backward item templates of the widest stage
     const int cap = (int)((t.run_words + 1) & ~(int64_t)1);
     const size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
-    cudaFuncSetAttribute(emit_items_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_items_kernel), smem);
     int64_t *out = reinterpret_cast<int64_t *>(records);
     emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
         v, plans, op_start, op_words_per_cand, out, cap);
@@ -527,7 +570,7 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
         int run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun);
         run |= 1;
         const size_t bsmem = (size_t)(2 * (run * 5 + 1)) * sizeof(int64_t);
-        cudaFuncSetAttribute(emit_buckets_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bsmem);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_buckets_kernel), bsmem);
         emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, s>>>(v, plans, out, run);
         ++*launches;
     }

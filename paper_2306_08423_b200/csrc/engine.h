@@ -24,11 +24,17 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+#include <vector>
+
 #include "../../include/distsim.h"
 
 namespace distsim {
 
 constexpr int64_t kSat = (int64_t)1 << 62;
+// Device status word beyond the DISTSIM_E_* codes: a block gave up waiting for a bulk copy twice
+// and may have left with the copy still in flight.
+constexpr int32_t kStatusCopyPending = -70;
 
 struct TableConst {
     int32_t n_layers, n_classes, n_devices, gpus_per_node;
@@ -105,7 +111,33 @@ struct DeviceView {
     const int64_t *jsum;             // [n_entries][DISTSIM_MAX_PP] total jitter of the m forward and
                                      // m backward items of a stage (nullptr without jitter)
     int32_t *status;                 // device status word: 0 ok, else first error code
+    int32_t stage_polls;             // polls of the first wait for staged tables (the drain wait keeps its own limit)
 };
+
+// A kernel's limit on dynamic shared memory is an attribute of (kernel, device): raise it when a
+// launch needs more than this process has asked for so far on the current device, not on every
+// launch.  `kernel` is the address of the __global__ function.
+inline cudaError_t ensure_dynamic_smem(const void *kernel, size_t bytes)
+{
+    struct Granted { const void *kernel; int device; size_t bytes; };
+    static std::mutex mu;
+    static std::vector<Granted> granted;
+    if (bytes == 0) return cudaSuccess;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (Granted &g : granted)
+        if (g.kernel == kernel && g.device == dev) {
+            if (bytes <= g.bytes) return cudaSuccess;
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+            if (e == cudaSuccess) g.bytes = bytes;
+            return e;
+        }
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) granted.push_back(Granted{kernel, dev, bytes});
+    return e;
+}
 
 // ---- set-up kernels (setup_kernels.cu) -------------------------------------------------
 void launch_fill_entries(cudaStream_t s, const TableConst &tc, Row *rows, int n_rows,
@@ -207,13 +239,11 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
                       int64_t *launches);
+// out[k] = order-sensitive checksum of the records [offsets[k], offsets[k + 1]).
+void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const int64_t *offsets, int64_t n_lists,
+                           uint64_t *out, int64_t *launches);
 void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
                          const int64_t *op_start, int64_t op_words_per_cand, const EmitTotals &totals,
                          distsim_record *records, int64_t *launches);
-
-// ---- probe (probe_kernels.cu) ----------------------------------------------------------
-// Launches the integer-issue probe; returns the number of integer instructions (per thread,
-// summed over threads) it executes.
-int64_t launch_int_issue_probe(cudaStream_t s, int mode, int blocks, int iters, int64_t *sink, int64_t *launches);
 
 }  // namespace distsim

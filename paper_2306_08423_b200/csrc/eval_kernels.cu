@@ -5,10 +5,9 @@
 // partitions and pp <= 16.
 // eval_lockstep_kernel: a segment of pp consecutive lanes evaluates one candidate, lane = stage,
 // 32/pp candidates per warp, all segments of a warp advancing through the slots of the
-// lock-step recurrence together; for pp = 64 two warps share a candidate and exchange the two
-// boundary values per slot through shared memory (one named barrier of 64 threads per slot).  The prefix rows of
-// the entries a block touches are staged into shared memory with one bulk copy per table
-// (cp.async.bulk, completion on the block's own mbarrier, no multicast).
+// lock-step recurrence together; for pp = 64 a lane owns two neighbouring stages and a warp one
+// candidate.  The prefix rows of the entries a block touches are staged into shared memory with
+// one bulk copy per table (cp.async.bulk, completion on the block's own mbarrier, no multicast).
 //
 // A search space has a few dozen rows, many of them tiny; launching them one by one would leave
 // the device idle between kernels, so one launch carries a list of (row, range) work items and
@@ -23,24 +22,23 @@ namespace {
 
 constexpr int kEvalThreads = 256;
 
-template <bool kPair, bool kJit>
+template <int S, bool kJit>
 __global__ void __launch_bounds__(kEvalThreads)
 eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
                      int64_t *__restrict__ busy_out, int smem_words)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t bar;
-    __shared__ int64_t pair_x[kEvalThreads / 64][6];       // per pair of warps: xf[2], xb[2], xm[2]
     int wi = 0;
     while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
     const EvalWork &wk = batch.w[wi];
     const int64_t lo = wk.lo, hi = wk.hi;
     const Row row = v.rows[wk.row];
     const int pp = row.pp;
-    const int wl = kPair ? 32 : pp;                // lanes of a warp per candidate
+    const int wl = pp / S;                         // lanes of a warp per candidate
     const int warps = blockDim.x >> 5;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int cpb = kPair ? warps / 2 : warps * (32 / wl);     // candidates per block
+    const int cpb = warps * (32 / wl);             // candidates per block
     const int64_t cta_first = lo + (int64_t)((int)blockIdx.x - wk.block_begin) * cpb;
     if (cta_first >= hi) return;                   // the whole block leaves: no barrier is left waiting
     const int64_t cta_last = min(hi, cta_first + (int64_t)cpb) - 1;
@@ -57,39 +55,31 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     if (max_stage_entries > 0 && n_stage <= max_stage_entries) {
         const uint32_t bytes = (uint32_t)(n_stage * lp * sizeof(int64_t));
         staged = stage_two_tables(&bar, sm_f, v.etf + (int64_t)e_lo * lp, sm_b,
-                                  v.etb + (int64_t)e_lo * lp, bytes, v.status);
+                                  v.etb + (int64_t)e_lo * lp, bytes, v.status, v.stage_polls);
     }
 
-    const int seg = kPair ? 0 : lane / wl, seg_lane = lane - seg * wl;
-    int64_t local = cta_first + (kPair ? warp >> 1 : warp * (32 / wl) + seg);
+    const int seg = lane / wl, seg_lane = lane - seg * wl;
+    int64_t local = cta_first + warp * (32 / wl) + seg;
     const bool valid = local < hi;
-    if (!valid) local = hi - 1;                    // idle segments (and pairs) shadow a real candidate
+    if (!valid) local = hi - 1;                    // idle segments shadow a real candidate
     const CandidateCoords cc = split_local(row, local);
     const Entry en = v.entries[cc.entry];
     const int64_t *pf = staged ? sm_f + (int64_t)(cc.entry - e_lo) * lp : v.etf + (int64_t)cc.entry * lp;
     const int64_t *pb = staged ? sm_b + (int64_t)(cc.entry - e_lo) * lp : v.etb + (int64_t)cc.entry * lp;
 
-    // both warps of a pair hold the same candidate, hence the same number of slots
     int n_slots = 2 * (en.m + pp - 1);
     n_slots = __reduce_max_sync(0xffffffffu, n_slots);
 
-    PairLink link{};
-    if (kPair) {
-        int64_t *x = pair_x[warp >> 1];
-        link.xf = x; link.xb = x + 2; link.xm = x + 4;
-        link.bar_id = 1 + (warp >> 1);
-        link.half = warp & 1;
-    }
-    const StageResult<1> R = lockstep_candidate<1, false, kJit, kPair>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank,
-                                                                  seg_lane, wl, n_slots, nullptr, link);
+    const StageResult<S> R = lockstep_candidate<S, false, kJit>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank,
+                                                                seg_lane, wl, n_slots, nullptr);
     if (!valid) return;
     const int64_t out = row.offset + local - first;
-    const int d = (kPair ? link.half * 32 : 0) + seg_lane;
-    if (d == 0) batch_out[out] = R.batch;
+    if (seg_lane == 0) batch_out[out] = R.batch;
     if (busy_out) {
         int64_t *bo = busy_out + out * v.sc.pp_max;
-        bo[d] = R.busy[0];
-        for (int z = pp + d; z < v.sc.pp_max; z += pp) bo[z] = 0;
+#pragma unroll
+        for (int k = 0; k < S; ++k) bo[seg_lane * S + k] = R.busy[k];
+        for (int z = pp + seg_lane; z < v.sc.pp_max; z += wl) bo[z] = 0;
     }
 }
 
@@ -100,10 +90,10 @@ struct Pending {
     int smem_words = 0;
 };
 
-// Candidates per block of the lock-step kernel: 32 / pp per warp, half a candidate per warp at pp = 64.
+// Candidates per block of the lock-step kernel: 32 / pp per warp, one per warp (two stages per lane) at pp = 64.
 int lockstep_cpb(const Row &row)
 {
-    return row.pp > 32 ? (kEvalThreads / 32) / 2 : (kEvalThreads / 32) * (32 / row.pp);
+    return row.pp > 32 ? kEvalThreads / 32 : (kEvalThreads / 32) * (32 / row.pp);
 }
 
 int lockstep_blocks(const Row &row, int64_t lo, int64_t hi)
@@ -122,20 +112,18 @@ int lockstep_smem_words(const DeviceView &v, const Row &row)
     return words * (int64_t)sizeof(int64_t) > 96 * 1024 ? 0 : (int)words;     // too wide: global reads
 }
 
-template <bool kPair>
+template <int S>
 void flush_lockstep(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first, int64_t *batch_out,
                     int64_t *busy_out, int64_t *launches)
 {
     if (p.batch.n == 0) return;
     const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
     if (v.tc.n_jitter > 0) {
-        if (smem > 48 * 1024)
-            cudaFuncSetAttribute(eval_lockstep_kernel<kPair, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        eval_lockstep_kernel<kPair, true><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_lockstep_kernel<S, true>), smem);
+        eval_lockstep_kernel<S, true><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
     } else {
-        if (smem > 48 * 1024)
-            cudaFuncSetAttribute(eval_lockstep_kernel<kPair, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        eval_lockstep_kernel<kPair, false><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_lockstep_kernel<S, false>), smem);
+        eval_lockstep_kernel<S, false><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
     }
     ++*launches;
     p = Pending{};
@@ -148,12 +136,10 @@ void flush_thread(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first
     if (p.batch.n == 0) return;
     const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
     if (v.tc.n_jitter > 0) {
-        if (smem > 16 * 1024)
-            cudaFuncSetAttribute(eval_thread_kernel<PP, T, kBusy, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_thread_kernel<PP, T, kBusy, true>), smem);
         eval_thread_kernel<PP, T, kBusy, true><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out);
     } else {
-        if (smem > 24 * 1024)
-            cudaFuncSetAttribute(eval_thread_kernel<PP, T, kBusy, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_thread_kernel<PP, T, kBusy, false>), smem);
         eval_thread_kernel<PP, T, kBusy, false><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out);
     }
     ++*launches;
@@ -224,8 +210,8 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
         Pending &p = lock[which];
         const int blocks = lockstep_blocks(rows[r], lo, hi);
         if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - blocks) {
-            if (which) flush_lockstep<true>(lockstep_stream(1), v, p, first, batch_out, busy_out, launches);
-            else flush_lockstep<false>(lockstep_stream(0), v, p, first, batch_out, busy_out, launches);
+            if (which) flush_lockstep<2>(lockstep_stream(1), v, p, first, batch_out, busy_out, launches);
+            else flush_lockstep<1>(lockstep_stream(0), v, p, first, batch_out, busy_out, launches);
         }
         EvalWork &w = p.batch.w[p.batch.n++];
         w = EvalWork{};
@@ -290,8 +276,8 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
     }
     // the lock-step launches first, on their own streams: few blocks that run for long, beside
     // the thread-kernel launches (largest first) that fill the rest of the device
-    if (lock[1].batch.n) flush_lockstep<true>(lockstep_stream(1), v, lock[1], first, batch_out, busy_out, launches);
-    if (lock[0].batch.n) flush_lockstep<false>(lockstep_stream(0), v, lock[0], first, batch_out, busy_out, launches);
+    if (lock[1].batch.n) flush_lockstep<2>(lockstep_stream(1), v, lock[1], first, batch_out, busy_out, launches);
+    if (lock[0].batch.n) flush_lockstep<1>(lockstep_stream(0), v, lock[0], first, batch_out, busy_out, launches);
     for (int lg = 4; lg >= 0; --lg)
         for (int nw = 1; nw >= 0; --nw)
             flush_thread_any(lg, nw == 1, s, v, thr[lg][nw], first, batch_out, busy_out, launches);

@@ -63,26 +63,10 @@ __host__ __device__ constexpr int thread_kernel_min_blocks()
 
 template <typename T> __device__ __forceinline__ T vmax(T a, T b) { return a > b ? a : b; }
 
-#ifndef DS_CELL_FORM
-#define DS_CELL_FORM 0            // 0: max(t, free) + c;  1: max(t + c, free + c) (shorter chain)
-#endif
-#ifndef DS_DPX
-#define DS_DPX 1
-#endif
-#ifndef DS_UNROLL_MAIN
-#define DS_UNROLL_MAIN 2
-#endif
-#define DS_PRAGMA(x) _Pragma(#x)
-#define DS_UNROLL(n) DS_PRAGMA(unroll n)
-
 // One recurrence cell: end = max(input arrival, device free) + cost.
 template <typename T> __device__ __forceinline__ T cell(T arrival, T free_at, T cost)
 {
-#if DS_CELL_FORM == 1
-    return vmax((T)(arrival + cost), (T)(free_at + cost));
-#else
     return (T)(vmax(arrival, free_at) + cost);
-#endif
 }
 
 template <int PP, typename T>
@@ -109,14 +93,14 @@ __device__ __forceinline__ void run_gpipe(const ThreadState<PP, T> &c, int m, T 
 {
 #pragma unroll
     for (int d = 0; d < PP; ++d) free_at[d] = 0;
-DS_UNROLL(DS_UNROLL_MAIN)
+#pragma unroll 2
     for (int j = 0; j < m; ++j) {
         T t = free_at[0] + c.fop[0] + jt.fwd(j, 0);
         free_at[0] = t;
 #pragma unroll
         for (int d = 1; d < PP; ++d) { t = cell(t, free_at[d], (T)(c.fop[d] + jt.fwd(j, d))); free_at[d] = t; }
     }
-DS_UNROLL(DS_UNROLL_MAIN)
+#pragma unroll 2
     for (int j = 0; j < m; ++j) {
         T t = free_at[PP - 1] + c.bop[PP - 1] + jt.bwd(j, PP - 1);
         free_at[PP - 1] = t;
@@ -206,12 +190,10 @@ struct WarmWaves<PP, PP, T, kJit> {
 
 // max(a + b, c): one instruction on 32-bit operands (the GPU's fused add-max).
 template <typename T> __device__ __forceinline__ T addmax(T a, T b, T c) { return vmax((T)(a + b), c); }
-#if DS_DPX
 template <> __device__ __forceinline__ uint32_t addmax<uint32_t>(uint32_t a, uint32_t b, uint32_t c)
 {
     return __viaddmax_u32(a, b, c);
 }
-#endif
 
 // GPipe without jitter, in relative frames (see the header): returns main-lane ends in free_at.
 template <int PP, typename T>
@@ -222,7 +204,7 @@ __device__ __forceinline__ void run_gpipe_rel(const ThreadState<PP, T> &c, int m
     T r[PP];
 #pragma unroll
     for (int d = 0; d < PP; ++d) r[d] = 0;
-DS_UNROLL(DS_UNROLL_MAIN)
+#pragma unroll 2
     for (int j = 1; j < m; ++j) {
         T w = r[0] + c.fop[0];
         r[0] = w;
@@ -234,7 +216,7 @@ DS_UNROLL(DS_UNROLL_MAIN)
     T cf = 0, pb = 0;
 #pragma unroll
     for (int d = 0; d < PP; ++d) { cf += c.fop[d]; r[d] = (T)(r[d] + cf + pb); pb += c.bop[d]; }
-DS_UNROLL(DS_UNROLL_MAIN)
+#pragma unroll 2
     for (int j = 0; j < m; ++j) {
         T w = r[PP - 1] + c.bop[PP - 1];
         r[PP - 1] = w;
@@ -322,7 +304,7 @@ __device__ __forceinline__ void run_1f1b_rel(const ThreadState<PP, T> &c, int m,
 #pragma unroll
     for (int d = 0; d < PP; ++d) { h[d] += off; off += fb[d]; }
     if (m > PP) {
-DS_UNROLL(DS_UNROLL_MAIN)
+#pragma unroll 2
         for (int i = 0; i < m - PP; ++i) wave_1f1b_steady_rel<PP, T>(fb, h);
     }
     TailWavesRel<PP, PP, T>::run(c, fb, m, h);
@@ -343,7 +325,7 @@ __device__ __forceinline__ void run_1f1b(const ThreadState<PP, T> &c, int m, T (
     // waves i = 0 .. m-PP-1: every stage still has a forward item to pair with its backward;
     // entering them every stage's latest item is a forward one (free_at == last_f)
     if (m > PP) {
-DS_UNROLL(DS_UNROLL_MAIN)
+#pragma unroll 2
         for (int i = 0; i < m - PP; ++i) wave_1f1b_steady<PP, T, kJit>(c, last_f, jt, i);
 #pragma unroll
         for (int d = 0; d < PP; ++d) free_at[d] = last_f[d];
@@ -554,7 +536,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
         const StageCopy cp[kMaxCopies] = {{dsm, v.pfb32 + (int64_t)row.entry0 * lp, pbytes},
                                           {dsm + plan.off_binom, v.binom, bbytes},
                                           {dsm + plan.off_dt, dt_g, dbytes}, {nullptr, nullptr, 0u}};
-        if (pbytes + bbytes + dbytes > 0) staged = stage_tables(&bar, cp, v.status);
+        if (pbytes + bbytes + dbytes > 0) staged = stage_tables(&bar, cp, v.status, v.stage_polls);
         else __syncthreads();
     } else if (plan.n_entries_staged > 0 || plan.tables_staged || plan.n_dt_staged > 0 || plan.binom_staged) {
         const uint32_t pbytes = (uint32_t)(plan.n_entries_staged * lp * sizeof(int64_t));
@@ -568,7 +550,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
                                                : StageCopy{dsm + plan.off_nb, nb_g, tbytes},
                                           v.dt ? StageCopy{dsm + plan.off_binom, v.binom, bbytes}
                                                : StageCopy{dsm + plan.off_tp, tp_g, tbytes}};
-        staged = stage_tables(&bar, cp, v.status);      // contains the block-wide barriers
+        staged = stage_tables(&bar, cp, v.status, v.stage_polls);      // contains the block-wide barriers
     } else {
         __syncthreads();
     }
@@ -700,7 +682,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
 
         // ---- the row's schedules -------------------------------------------------------------
         const int64_t local0 = (int64_t)e * per_entry + part * n_sched;
-        int64_t res[3] = {0, 0, 0};
+        int64_t res0 = 0, res1 = 0, res2 = 0;      // result per schedule position (scalars: no indexed local array)
         int64_t main_only = -1;            // batch time of the 1F1B main lanes alone, once known
 #pragma unroll 1
         for (int sc = 0; sc < n_sched; ++sc) {
@@ -709,8 +691,9 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
             const int id = (sched_list >> (2 * sc)) & 3;
             // the asynchronous schedule is the 1F1B main lane without the gradient buckets
             const bool with_buckets = id != 2;
+            int64_t res_sc;
             if (id == 2 && main_only >= 0) {
-                res[sc] = main_only;
+                res_sc = main_only;
             } else {
                 T free_at[PP];
                 if (id == 0) {
@@ -733,8 +716,9 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
                     main_only = (int64_t)plain;
                     if (id == 2) batch = plain;
                 }
-                res[sc] = (int64_t)batch;
+                res_sc = (int64_t)batch;
             }
+            if (sc == 0) res0 = res_sc; else if (sc == 1) res1 = res_sc; else res2 = res_sc;
             if (kBusy) {
                 int64_t *bo = busy_out + (row.offset + local - first) * v.sc.pp_max;
 #pragma unroll
@@ -748,10 +732,11 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
         // results of the two schedules are neighbours in the output: one 16-byte store if aligned
         const int64_t out0 = row.offset + local0 - first;
         if (n_sched == 2 && local0 >= lo && local0 + 1 < hi && !(reinterpret_cast<uintptr_t>(batch_out + out0) & 15)) {
-            *reinterpret_cast<longlong2 *>(batch_out + out0) = make_longlong2(res[0], res[1]);
+            *reinterpret_cast<longlong2 *>(batch_out + out0) = make_longlong2(res0, res1);
         } else {
-            for (int sc = 0; sc < n_sched; ++sc)
-                if (local0 + sc >= lo && local0 + sc < hi) batch_out[out0 + sc] = res[sc];
+            if (local0 >= lo && local0 < hi) batch_out[out0] = res0;
+            if (n_sched > 1 && local0 + 1 >= lo && local0 + 1 < hi) batch_out[out0 + 1] = res1;
+            if (n_sched > 2 && local0 + 2 >= lo && local0 + 2 < hi) batch_out[out0 + 2] = res2;
         }
     }
 }

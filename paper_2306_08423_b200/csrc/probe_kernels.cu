@@ -9,9 +9,13 @@
 //           as 2 instructions each)
 //   mode 4  recurrence cells x = max(x + c, y) on uint32 with the fused add-max instruction
 //           (8 cells per round and thread, counted as 2 instructions each, as in mode 3)
-#include "engine.h"
+//
+// This file is a library of its own (libdistsim_bench.so, declared in include/distsim_bench.h):
+// measurement code stays out of the engine's library.
+#include <cuda_runtime.h>
+#include <stdint.h>
 
-namespace distsim {
+#include "../../include/distsim_bench.h"
 
 namespace {
 
@@ -60,17 +64,18 @@ __global__ void __launch_bounds__(256) int_issue_probe_kernel(int iters, int64_t
 
 }  // namespace
 
-int64_t launch_int_issue_probe(cudaStream_t s, int mode, int blocks, int iters, int64_t *sink, int64_t *launches)
+extern "C" int distsim_bench_int_issue_probe(void *stream, int32_t mode, int32_t blocks, int32_t iters,
+                                             int64_t *d_sink, int64_t *h_ops)
 {
+    if (!h_ops || !d_sink || blocks < 1 || iters < 1 || mode < 0 || mode > 4) return -1;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
     iters = (iters + 7) & ~7;                    // the kernel runs whole groups of 8 rounds
-    if (mode == 1) int_issue_probe_kernel<1><<<blocks, 256, 0, s>>>(iters, sink);
-    else if (mode == 2) int_issue_probe_kernel<2><<<blocks, 256, 0, s>>>(iters, sink);
-    else if (mode == 3) int_issue_probe_kernel<3><<<blocks, 256, 0, s>>>(iters, sink);
-    else if (mode == 4) int_issue_probe_kernel<4><<<blocks, 256, 0, s>>>(iters, sink);
-    else int_issue_probe_kernel<0><<<blocks, 256, 0, s>>>(iters, sink);
-    ++*launches;
+    if (mode == 1) int_issue_probe_kernel<1><<<blocks, 256, 0, s>>>(iters, d_sink);
+    else if (mode == 2) int_issue_probe_kernel<2><<<blocks, 256, 0, s>>>(iters, d_sink);
+    else if (mode == 3) int_issue_probe_kernel<3><<<blocks, 256, 0, s>>>(iters, d_sink);
+    else if (mode == 4) int_issue_probe_kernel<4><<<blocks, 256, 0, s>>>(iters, d_sink);
+    else int_issue_probe_kernel<0><<<blocks, 256, 0, s>>>(iters, d_sink);
     const int64_t per_round = mode == 1 ? kChains * 6 : kChains * 2;   // modes 0, 2: 16 = 8 x 2; modes 3, 4: 8 x 2
-    return (int64_t)blocks * 256 * iters * per_round;
+    *h_ops = (int64_t)blocks * 256 * iters * per_round;
+    return cudaGetLastError() == cudaSuccess ? 0 : -6;
 }
-
-}  // namespace distsim

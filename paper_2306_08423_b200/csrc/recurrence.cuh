@@ -14,8 +14,8 @@
 // all items finish within 2(m + pp - 1) slots, a stage runs at most one item per slot in its
 // schedule's order, and when an item runs, the *most recent* forward (backward) item finished
 // by the previous (next) stage before this slot is exactly the one it depends on.  So a lane
-// that owns a stage keeps only `last_f` and `last_b` (end of its latest forward / backward
-// item) and `free_at`; per slot it fetches the neighbour's value with one shuffle each way.
+// that owns a stage keeps only the end of its latest item and fetches the neighbour's with a
+// shuffle per slot (see lockstep_candidate).
 #pragma once
 
 #include "engine.h"
@@ -86,23 +86,26 @@ __device__ __forceinline__ CandidateCoords split_local(const Row &row, int64_t l
     return cc;
 }
 
-// Does stage d run a forward / backward item in slot s, and of which micro-batch j?
-__device__ __forceinline__ void slot_activity(int sched, int pp, int m, int d, int s, bool &do_f, bool &do_b, int &j)
+// A stage's place in the lock-step slots, in a form both schedules share: the forward items
+// j < w run in slot d + j and the others in slot d + 2j; the backward item j runs in slot
+// b0 + (j << sh).  GPipe: w = m, b0 = m + 2pp - 2 - d, sh = 0; 1F1B: w = min(pp - d, m),
+// b0 = 2pp - 1 - d, sh = 1.  A stage never has a forward and a backward item in one slot.
+struct SlotPlan { int w, b0, sh; };
+__device__ __forceinline__ SlotPlan slot_plan(int sched, int pp, int m, int d)
 {
-    const int x = s - d;
-    if (sched == 0) {
-        const int y = s - (m + 2 * pp - 2 - d);
-        do_f = (unsigned)x < (unsigned)m;
-        do_b = (unsigned)y < (unsigned)m;
-        j = do_f ? x : y;
-    } else {
-        const int w = min(pp - d, m);
-        const int y = s - (2 * pp - 1 - d);
-        const bool warm = (unsigned)x < (unsigned)w;
-        do_f = warm || (x >= 2 * w && !(x & 1) && (x >> 1) < m);
-        do_b = y >= 0 && !(y & 1) && (y >> 1) < m;
-        j = do_f ? (warm ? x : x >> 1) : y >> 1;
-    }
+    SlotPlan sp;
+    if (sched == 0) { sp.w = m; sp.b0 = m + 2 * pp - 2 - d; sp.sh = 0; }
+    else { sp.w = min(pp - d, m); sp.b0 = 2 * pp - 1 - d; sp.sh = 1; }
+    return sp;
+}
+// Does stage d run a forward / backward item in slot s, and of which micro-batch j?
+__device__ __forceinline__ void slot_activity(const SlotPlan &sp, int m, int d, int s, bool &do_f, bool &do_b, int &j)
+{
+    const int x = s - d, y = s - sp.b0;
+    const bool warm = (unsigned)x < (unsigned)sp.w;
+    do_f = warm || (x >= 2 * sp.w && !(x & 1) && (x >> 1) < m);
+    do_b = y >= 0 && !(y & sp.sh) && (y >> sp.sh) < m;
+    j = do_f ? (warm ? x : x >> 1) : y >> sp.sh;
 }
 
 // Extra time of the item of micro-batch j on stage d (0 without a jitter table).
@@ -170,89 +173,91 @@ __device__ __forceinline__ int64_t p2p_cost(const Row &row, const Entry &en, int
     return (((d + 1) & (row.p2p_period - 1)) == 0) ? en.p2p_inter : en.p2p_intra;
 }
 
-// Two warps that evaluate one candidate together (pp = 64, a stage per lane): per slot the
-// boundary lanes hand the neighbouring warp their latest forward / backward end through shared
-// memory, double-buffered by slot parity, with one named barrier of the 64 threads per slot.
-struct PairLink {
-    int64_t *xf, *xb;            // [2] each: forward end of stage 31, backward end of stage 32
-    int64_t *xm;                 // [2]: each warp's maximum for the final reduction
-    int bar_id;                  // named barrier of the pair (1 .. 15)
-    int half;                    // 0: stages 0 .. 31, 1: stages 32 .. 63
-};
-__device__ __forceinline__ void pair_barrier(int id)
+__device__ __forceinline__ int64_t shfl_idx64(int64_t x, int src_lane)
 {
-    asm volatile("bar.sync %0, 64;" :: "r"(id) : "memory");
+    const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)x, src_lane);
+    const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)((uint64_t)x >> 32), src_lane);
+    return (int64_t)(((uint64_t)hi << 32) | lo);
 }
 
-// Lock-step evaluation of one candidate by `wl` consecutive lanes (wl * S == pp; with kPair by
-// the 2 x 32 lanes of two warps, S == 1), every lane of the warp calling this together (lanes
-// of other segments work on their own candidates).
+// Lock-step evaluation of one candidate by `wl` consecutive lanes (wl * S == pp), every lane of
+// the warp calling this together (lanes of other segments work on their own candidates).
 //   entry_index  global index of `en`;  seg_lane: lane index inside the segment;
-//   n_slots_warp loop bound, uniform over the warp (and over both warps of a pair)
+//   n_slots_warp loop bound, uniform over the warp
 //   pf, pb     the entry's forward / backward prefix rows (shared or global memory)
 //   rec        if kRecord and non-null: item start times go to rec[d * 2m + position in stage order]
 //   kJit       the table has per-micro-batch jitter (otherwise none of its code is generated)
-template <int S, bool kRecord, bool kJit, bool kPair = false>
+// Per stage the only state is t, the end of the stage's latest item (= when its device is free).
+// When an item runs, the item it takes its input from ran on the neighbouring stage in the slot
+// before, or (the first forward item after a 1F1B warm-up) is still that stage's latest item; so
+// the input's arrival is the neighbour's t as of the previous slot, and a slot is
+//   t = max(neighbour's t, t) + cost
+// with the neighbour chosen by the kind of item (previous stage for a forward item, next stage
+// for a backward one, the stage itself - a no-op - when it idles or has no such neighbour: the
+// first stage's forward items and the last stage's backward items wait for their own device only).
+// One stage per lane fetches exactly that value with one indexed shuffle per slot.
+template <int S, bool kRecord, bool kJit>
 __device__ __forceinline__ StageResult<S> lockstep_candidate(
     const DeviceView &v, const Row &row, const Entry &en, int entry_index, const int64_t *pf,
-    const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec,
-    PairLink link = PairLink{})
+    const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec)
 {
-    static_assert(!kPair || S == 1, "a pair of warps owns one stage per lane");
     StageResult<S> R;
     const int pp = row.pp, m = en.m;
-    const int d0 = (kPair ? link.half * 32 + seg_lane : seg_lane) * S;
+    const int d0 = seg_lane * S;
     int bounds[S + 1];
     partition_bounds<S>(v, pp, part_rank, d0, bounds);
+    SlotPlan sp[S];
 #pragma unroll
     for (int k = 0; k < S; ++k) {
         const int d = d0 + k;
         R.a[k] = bounds[k]; R.e[k] = bounds[k + 1];
         R.fop[k] = pf[R.e[k]] - pf[R.a[k]] + (d < pp - 1 ? p2p_cost(row, en, d) : 0);
         R.bop[k] = pb[R.e[k]] - pb[R.a[k]] + (d > 0 ? p2p_cost(row, en, d - 1) : 0);
-        R.last_b_start[k] = 0;
+        sp[k] = slot_plan(sched, pp, m, d);
     }
-    int64_t last_f[S], last_b[S], free_at[S];
+    int64_t t[S];
     int n_done[S];
 #pragma unroll
-    for (int k = 0; k < S; ++k) { last_f[k] = 0; last_b[k] = 0; free_at[k] = 0; n_done[k] = 0; }
+    for (int k = 0; k < S; ++k) { t[k] = 0; n_done[k] = 0; }
+    const int lane = threadIdx.x & 31;
 
-    // The lanes of a warp run forward items, backward items or nothing in the same slot, so the
-    // slot body is written without branches: one cell with selected operands per owned stage.
     for (int s = 0; s < n_slots_warp; ++s) {
-        int64_t up_f = __shfl_up_sync(0xffffffffu, last_f[S - 1], 1, wl);
-        int64_t dn_b = __shfl_down_sync(0xffffffffu, last_b[0], 1, wl);
-        if (kPair) {
-            const int buf = s & 1;
-            if (link.half == 0 && seg_lane == 31) link.xf[buf] = last_f[0];
-            if (link.half == 1 && seg_lane == 0) link.xb[buf] = last_b[0];
-            pair_barrier(link.bar_id);
-            if (link.half == 1 && seg_lane == 0) up_f = link.xf[buf];
-            if (link.half == 0 && seg_lane == 31) dn_b = link.xb[buf];
-        }
-        int64_t old_f[S], old_b[S];
-#pragma unroll
-        for (int k = 0; k < S; ++k) { old_f[k] = last_f[k]; old_b[k] = last_b[k]; }
-#pragma unroll
-        for (int k = 0; k < S; ++k) {
-            const int d = d0 + k;
+        if (S == 1) {
             bool do_f, do_b;
             int j;
-            slot_activity(sched, pp, m, d, s, do_f, do_b, j);
-            do_b = do_b && !do_f;
-            const bool act = do_f || do_b;
-            const int64_t dep_f = (k == 0) ? (d == 0 ? 0 : up_f) : old_f[k > 0 ? k - 1 : 0];
-            const int64_t dep_b = (k == S - 1) ? (d == pp - 1 ? 0 : dn_b) : old_b[k < S - 1 ? k + 1 : 0];
-            const int64_t st = max64(do_f ? dep_f : dep_b, free_at[k]);
-            int64_t jit = 0;
-            if (kJit) jit = act ? jitter_of(v, do_f ? v.raw.jit_f : v.raw.jit_b, j, d) : 0;
-            const int64_t end = st + jit + (do_f ? R.fop[k] : R.bop[k]);
-            if (kRecord && rec && act) rec[(int64_t)d * 2 * m + n_done[k]] = st;
-            if (S > 1 && !act) continue;             // a lane with several stages skips its idle ones
-            if (act) free_at[k] = end;
-            if (do_f) last_f[k] = end;
-            if (do_b) { last_b[k] = end; R.last_b_start[k] = st + jit; }
-            n_done[k] += act ? 1 : 0;
+            slot_activity(sp[0], m, d0, s, do_f, do_b, j);
+            const int src = lane - ((do_f && d0 > 0) ? 1 : 0) + ((do_b && d0 < pp - 1) ? 1 : 0);
+            const int64_t dep = shfl_idx64(t[0], src);
+            int64_t cost = do_f ? R.fop[0] : (do_b ? R.bop[0] : 0);
+            const int64_t st = max64(dep, t[0]);
+            if (kJit) cost += (do_f || do_b) ? jitter_of(v, do_f ? v.raw.jit_f : v.raw.jit_b, j, d0) : 0;
+            if (kRecord && rec && (do_f || do_b)) rec[(int64_t)d0 * 2 * m + n_done[0]] = st;
+            if (kRecord) n_done[0] += (do_f || do_b) ? 1 : 0;
+            t[0] = st + cost;
+        } else {
+            // several stages per lane: the lane's first (last) stage takes the previous (next)
+            // lane's last (first) stage, the others their neighbour inside the lane
+            const int64_t up_f = __shfl_up_sync(0xffffffffu, t[S - 1], 1, wl);
+            const int64_t dn_b = __shfl_down_sync(0xffffffffu, t[0], 1, wl);
+            int64_t old[S];
+#pragma unroll
+            for (int k = 0; k < S; ++k) old[k] = t[k];
+#pragma unroll
+            for (int k = 0; k < S; ++k) {
+                const int d = d0 + k;
+                bool do_f, do_b;
+                int j;
+                slot_activity(sp[k], m, d, s, do_f, do_b, j);
+                const int64_t dep_f = (k == 0) ? (d == 0 ? 0 : up_f) : old[k > 0 ? k - 1 : 0];
+                const int64_t dep_b = (k == S - 1) ? (d == pp - 1 ? 0 : dn_b) : old[k < S - 1 ? k + 1 : 0];
+                const int64_t dep = do_f ? dep_f : (do_b ? dep_b : 0);
+                int64_t cost = do_f ? R.fop[k] : (do_b ? R.bop[k] : 0);
+                const int64_t st = max64(dep, old[k]);
+                if (kJit) cost += (do_f || do_b) ? jitter_of(v, do_f ? v.raw.jit_f : v.raw.jit_b, j, d) : 0;
+                if (kRecord && rec && (do_f || do_b)) rec[(int64_t)d * 2 * m + n_done[k]] = st;
+                if (kRecord) n_done[k] += (do_f || do_b) ? 1 : 0;
+                t[k] = st + cost;
+            }
         }
     }
 
@@ -261,7 +266,10 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
     int64_t mx = 0;
 #pragma unroll
     for (int k = 0; k < S; ++k) {
-        R.main_end[k] = free_at[k];
+        R.main_end[k] = t[k];
+        // every stage's last item is the backward item of the last micro-batch; its first layer
+        // event starts one backward item cost before its end
+        R.last_b_start[k] = t[k] - R.bop[k];
         // the asynchronous schedule has no gradient all-reduce events
         R.dp_end[k] = sched == 2 ? R.main_end[k]
                                  : bucket_lane_end(v, row, pb, nbt, tpt, R.a[k], R.e[k], R.last_b_start[k], R.main_end[k]);
@@ -271,11 +279,6 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         mx = max64(mx, max64(R.main_end[k], R.dp_end[k]));
     }
     for (int off = 1; off < wl; off <<= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, off, wl));
-    if (kPair) {
-        if (seg_lane == 0) link.xm[link.half] = mx;
-        pair_barrier(link.bar_id);
-        mx = max64(link.xm[0], link.xm[1]);
-    }
     R.batch = mx;
     return R;
 }

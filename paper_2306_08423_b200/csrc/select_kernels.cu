@@ -300,12 +300,8 @@ void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t co
                  int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
                  int64_t *launches)
 {
-    static bool attr_set = false;
     const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
-    if (!attr_set) {
-        cudaFuncSetAttribute(sort_pairs_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem);
-        attr_set = true;
-    }
+    ensure_dynamic_smem(reinterpret_cast<const void *>(&sort_pairs_kernel), sort_smem);     // per device
     if (count <= kSortMax) {
         sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(batch, nullptr, (int)count, k, first, d_indices, d_times);
         ++*launches;

@@ -3,9 +3,11 @@
 // One thread arms the block's mbarrier with the expected byte count and issues the copies
 // (cp.async.bulk global -> shared of the issuing block, no multicast); every thread then waits
 // on the barrier's phase with a bounded number of polls.  If the wait gives up, the block records
-// DISTSIM_E_TIMEOUT in the status word and reads the tables from global memory instead; it
-// polls once more (again bounded) before leaving so that no copy is still in flight when the
-// block's shared memory is released.
+// DISTSIM_E_TIMEOUT in the status word and reads the tables from global memory instead (the same
+// values, so results stay exact); it polls once more (again bounded) before going on so that no
+// copy is still in flight when the block's shared memory is released.  Should that second wait
+// give up as well, the status word takes kStatusCopyPending: the block may leave with a copy in
+// flight and nothing computed on the device afterwards can be trusted.
 // Requirements: sources and destinations 16-byte aligned, sizes multiples of 16 bytes.
 #pragma once
 
@@ -38,7 +40,9 @@ struct StageCopy { void *dst; const void *src; uint32_t bytes; };
 // them.  Must be called once per block, by every thread.  Returns true when the shared copies
 // are usable by the whole block.
 constexpr int kMaxCopies = 4;
-__device__ __forceinline__ bool stage_tables(uint64_t *bar_ptr, const StageCopy (&c)[kMaxCopies], int32_t *status)
+constexpr int kDrainPolls = 1 << 16;
+__device__ __forceinline__ bool stage_tables(uint64_t *bar_ptr, const StageCopy (&c)[kMaxCopies], int32_t *status,
+                                             int first_polls)
 {
     const uint32_t bar = smem_addr(bar_ptr);
     if (threadIdx.x == 0) {
@@ -60,10 +64,11 @@ __device__ __forceinline__ bool stage_tables(uint64_t *bar_ptr, const StageCopy 
                     :: "r"(smem_addr(c[i].dst)), "l"(c[i].src), "r"(c[i].bytes), "r"(bar) : "memory");
     }
     // each try_wait already blocks for a bounded, implementation-defined time
-    bool ok = mbar_poll(bar, 0, 1 << 16);
+    bool ok = mbar_poll(bar, 0, first_polls);
     if (!ok) {
         atomicCAS(status, 0, DISTSIM_E_TIMEOUT);
-        mbar_poll(bar, 0, 1 << 16);          // drain before the block can exit
+        if (!mbar_poll(bar, 0, kDrainPolls))                  // drain before the block can exit
+            atomicMin(status, kStatusCopyPending);
     }
     // the block must agree: a table that one thread could not see is read from global by all
     ok = __syncthreads_and(ok);
@@ -72,10 +77,10 @@ __device__ __forceinline__ bool stage_tables(uint64_t *bar_ptr, const StageCopy 
 
 __device__ __forceinline__ bool stage_two_tables(uint64_t *bar_ptr, void *dst_a, const void *src_a,
                                                  void *dst_b, const void *src_b, uint32_t bytes,
-                                                 int32_t *status)
+                                                 int32_t *status, int first_polls)
 {
     const StageCopy c[kMaxCopies] = {{dst_a, src_a, bytes}, {dst_b, src_b, bytes}, {nullptr, nullptr, 0}, {nullptr, nullptr, 0}};
-    return stage_tables(bar_ptr, c, status);
+    return stage_tables(bar_ptr, c, status, first_polls);
 }
 
 }  // namespace distsim

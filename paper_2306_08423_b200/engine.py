@@ -20,11 +20,14 @@ MAX_PP = 64
 OK, E_ARG, E_STATE, E_RANGE, E_CAPACITY, E_OVERFLOW, E_CUDA, E_TIMEOUT, E_UNSUPPORTED = (
     0, -1, -2, -3, -4, -5, -6, -7, -8)
 
-EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error", "distsim_launch_count",
+EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error",
            "distsim_load_event_table", "distsim_set_space", "distsim_decode",
            "distsim_eval_strategies", "distsim_argmin", "distsim_topk",
-           "distsim_emit_timelines", "distsim_search_host", "distsim_int_issue_probe",
-           "distsim_topk_static", "distsim_space_cells")
+           "distsim_emit_timelines", "distsim_checksum_timelines", "distsim_search_host",
+           "distsim_topk_static")
+# hooks of include/distsim_testing.h (test-suite and benchmark accounting; not the stable ABI)
+TESTING_EXPORTS = ("distsim_testing_set_stage_wait_polls", "distsim_testing_launch_count",
+                   "distsim_testing_space_cells")
 TOPK_STATIC_MAX_K = 1024
 
 if not os.path.exists(LIB_PATH):
@@ -70,8 +73,9 @@ _lib.distsim_destroy.argtypes = [C.c_void_p]
 _lib.distsim_destroy.restype = None
 _lib.distsim_last_error.argtypes = [C.c_void_p]
 _lib.distsim_last_error.restype = C.c_char_p
-_lib.distsim_launch_count.argtypes = [C.c_void_p]
-_lib.distsim_launch_count.restype = C.c_int64
+_lib.distsim_testing_launch_count.argtypes = [C.c_void_p]
+_lib.distsim_testing_launch_count.restype = C.c_int64
+_lib.distsim_testing_set_stage_wait_polls.argtypes = [C.c_void_p, C.c_int32]
 _lib.distsim_load_event_table.argtypes = [C.c_void_p, C.POINTER(_Table)]
 _lib.distsim_set_space.argtypes = [C.c_void_p, C.POINTER(_Space), C.POINTER(C.c_int64)]
 _lib.distsim_decode.argtypes = [C.c_void_p, C.c_int64, C.POINTER(_Candidate)]
@@ -83,19 +87,17 @@ _lib.distsim_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c
 _lib.distsim_emit_timelines.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                         C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.POINTER(C.c_int64)]
+_lib.distsim_checksum_timelines.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
 _lib.distsim_search_host.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_Space), C.c_int32,
                                      C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                                      C.c_void_p, C.c_void_p]
-
-
-_lib.distsim_int_issue_probe.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]
 
 
 _lib.distsim_topk_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
                                      C.c_void_p, C.c_void_p]
 
 
-_lib.distsim_space_cells.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+_lib.distsim_testing_space_cells.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 
 
 def _np_ptr(a: np.ndarray):
@@ -176,7 +178,7 @@ class Context:
 
     @property
     def launch_count(self) -> int:
-        return int(_lib.distsim_launch_count(self._h))
+        return int(_lib.distsim_testing_launch_count(self._h))
 
 
 def distsim_load_event_table(ctx: Context, table) -> None:
@@ -212,7 +214,12 @@ def distsim_eval_strategies(ctx: Context, first: int, count: int, d_batch_ns,
 def distsim_argmin(ctx: Context, d_batch_ns, first: int, count: int, stream=None):
     pb = _dev_ptr(d_batch_ns, "int64", count, "d_batch_ns")
     bi, bt = C.c_int64(0), C.c_int64(0)
-    ctx._check(_lib.distsim_argmin(ctx._h, _stream(stream), pb, first, count, C.byref(bi), C.byref(bt)))
+    rc = _lib.distsim_argmin(ctx._h, _stream(stream), pb, first, count, C.byref(bi), C.byref(bt))
+    if rc == E_TIMEOUT and b"outputs are exact" in _lib.distsim_last_error(ctx._h):
+        e = DistsimError(rc, _lib.distsim_last_error(ctx._h).decode())
+        e.result = (int(bi.value), int(bt.value))       # the outputs were written before the code was returned
+        raise e
+    ctx._check(rc)
     return int(bi.value), int(bt.value)
 
 
@@ -230,7 +237,9 @@ def distsim_emit_timelines(ctx: Context, d_indices, n: int, d_records, capacity_
     ``d_records`` is given but too small.  ``d_records`` is an int64 tensor of
     at least ``5 * capacity_records`` elements (or None for a sizing pass).  Offsets, busy
     times and utilisations are final on return; the records are written in stream order
-    (complete once the work enqueued on the stream has finished)."""
+    (complete once the work enqueued on the stream has finished).  A DistsimError with code
+    E_TIMEOUT that carries ``total_records`` reports a stalled table copy: all outputs were
+    written and are exact."""
     pi = _dev_ptr(d_indices, "int64", n, "d_indices")
     pr = _dev_ptr(d_records, "int64", 5 * capacity_records, "d_records")
     nn = n * ctx.n_devices
@@ -240,12 +249,22 @@ def distsim_emit_timelines(ctx: Context, d_indices, n: int, d_records, capacity_
     total = C.c_int64(0)
     rc = _lib.distsim_emit_timelines(ctx._h, _stream(stream), pi, n, pr, capacity_records, po, pbz, pu,
                                      C.byref(total))
-    if rc == E_CAPACITY:
+    if rc == E_CAPACITY or (rc == E_TIMEOUT and b"outputs are exact" in _lib.distsim_last_error(ctx._h)):
         e = DistsimError(rc, _lib.distsim_last_error(ctx._h).decode())
         e.total_records = int(total.value)
         raise e
     ctx._check(rc)
     return int(total.value)
+
+
+def distsim_checksum_timelines(ctx: Context, d_records, d_offsets, n_lists: int, d_checksums, stream=None) -> None:
+    """Order-sensitive 64-bit checksum of each of the ``n_lists`` record streams delimited by
+    ``d_offsets`` into ``d_checksums`` (an int64 tensor holding the 64-bit sums' bit patterns)."""
+    total = 0 if n_lists == 0 else 1
+    pr = _dev_ptr(d_records, "int64", total, "d_records")
+    po = _dev_ptr(d_offsets, "int64", n_lists + 1, "d_offsets")
+    pc = _dev_ptr(d_checksums, "int64", n_lists, "d_checksums")
+    ctx._check(_lib.distsim_checksum_timelines(ctx._h, _stream(stream), pr, po, n_lists, pc))
 
 
 def distsim_search_host(ctx: Context, table, space, k: int = 0):
@@ -264,13 +283,6 @@ def distsim_search_host(ctx: Context, table, space, k: int = 0):
     ctx.pp_max = int(space.pp_max)
     kk = min(k, ctx.n_candidates, 4096)
     return ctx.n_candidates, int(bi.value), int(bt.value), idx[:kk], tim[:kk]
-
-
-def distsim_int_issue_probe(ctx: Context, blocks: int, iters: int, mode: int = 0, stream=None) -> int:
-    """Enqueues the integer-issue probe; returns the number of integer instructions it runs."""
-    ops = C.c_int64(0)
-    ctx._check(_lib.distsim_int_issue_probe(ctx._h, _stream(stream), mode, blocks, iters, C.byref(ops)))
-    return int(ops.value)
 
 
 def distsim_topk_static(d_batch_ns, first: int, count: int, k: int, d_indices, d_times=None,
@@ -294,8 +306,18 @@ def distsim_topk_static(d_batch_ns, first: int, count: int, k: int, d_indices, d
         raise DistsimError(rc, "distsim_topk_static failed")
 
 
-def distsim_space_cells(ctx: Context):
-    """(recurrence cells of the space, cells the engine may evaluate in 32-bit arithmetic)."""
+def distsim_testing_space_cells(ctx: Context):
+    """(recurrence cells of the space, cells the engine evaluates in 32-bit arithmetic)."""
     a, b = C.c_int64(0), C.c_int64(0)
-    ctx._check(_lib.distsim_space_cells(ctx._h, C.byref(a), C.byref(b)))
+    ctx._check(_lib.distsim_testing_space_cells(ctx._h, C.byref(a), C.byref(b)))
     return int(a.value), int(b.value)
+
+
+def distsim_testing_launch_count(ctx: Context) -> int:
+    return ctx.launch_count
+
+
+def distsim_testing_set_stage_wait_polls(ctx: Context, polls: int) -> None:
+    """Polls of the evaluation kernels' first wait for their staged tables (0: give up at once
+    and take the global-memory path; the library's default is 65 536)."""
+    ctx._check(_lib.distsim_testing_set_stage_wait_polls(ctx._h, polls))

@@ -6,30 +6,42 @@ import re
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def _declared():
-    text = open(os.path.join(ROOT, "include", "distsim.h")).read()
+def _declared(header):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(distsim_[a-z_0-9]+)\s*\(", text)))
 
 
-def test_library_exports_every_declared_symbol():
-    from paper_2306_08423_b200.build import build
-    lib = ctypes.CDLL(build())
-    names = _declared()
+def test_every_header_is_covered():
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["distsim.h", "distsim_bench.h", "distsim_testing.h"]
+
+
+def test_libraries_export_every_declared_symbol():
+    from paper_2306_08423_b200 import build as B
+    lib = ctypes.CDLL(B.build())
+    names = _declared("distsim.h")
     assert {"distsim_load_event_table", "distsim_eval_strategies", "distsim_emit_timelines",
             "distsim_argmin"} <= set(names)
-    for name in names:
+    for name in names + _declared("distsim_testing.h"):
         assert hasattr(lib, name), name
+    bench = ctypes.CDLL(B.BENCH_LIB)
+    for name in _declared("distsim_bench.h"):
+        assert hasattr(bench, name), name
+        assert not hasattr(lib, name), f"{name}: measurement code inside the engine's library"
 
 
-def test_binding_names_match_header():
+def test_binding_names_match_headers():
     from paper_2306_08423_b200.build import build
     build()
-    from paper_2306_08423_b200 import engine
-    assert sorted(engine.EXPORTS) == _declared()
-    for name in engine.EXPORTS:
-        if name not in ("distsim_create", "distsim_destroy", "distsim_last_error", "distsim_launch_count"):
+    from paper_2306_08423_b200 import engine, probes
+    assert sorted(engine.EXPORTS) == _declared("distsim.h")
+    assert sorted(engine.TESTING_EXPORTS) == _declared("distsim_testing.h")
+    assert sorted(probes.EXPORTS) == _declared("distsim_bench.h")
+    for name in engine.EXPORTS + engine.TESTING_EXPORTS:
+        if name not in ("distsim_create", "distsim_destroy", "distsim_last_error"):
             assert callable(getattr(engine, name)), name
+    for name in probes.EXPORTS:
+        assert callable(getattr(probes, name)), name
 
 
 def test_create_fails_loudly_without_a_gpu():

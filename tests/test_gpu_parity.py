@@ -50,6 +50,25 @@ def eval_all(E, ctx, n, busy=True):
     return batch, (sb.view(n, ctx.pp_max) if busy else None)
 
 
+def stream_checksum(rec):
+    """The order-sensitive checksum distsim_checksum_timelines defines, of one record list
+    (int64 [r, 5]), restated with numpy."""
+    with np.errstate(over="ignore"):
+        wds = rec.reshape(-1).astype(np.uint64)
+        z = wds + np.arange(1, wds.size + 1, dtype=np.uint64) * np.uint64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+        z = z ^ (z >> np.uint64(31))
+        return int(z.sum(dtype=np.uint64))
+
+
+def device_checksums(E, ctx, records, offsets, n_lists):
+    out = dev(max(1, n_lists))
+    E.distsim_checksum_timelines(ctx, records, offsets, n_lists, out)
+    torch.cuda.synchronize()
+    return out.cpu().numpy()[:n_lists].view(np.uint64)
+
+
 def check_emission(E, ctx, w, indices):
     """Emits the given candidates and compares every record with the oracle."""
     N = w.table.n_devices
@@ -65,6 +84,7 @@ def check_emission(E, ctx, w, indices):
     rec = records.cpu().numpy()[: total * 5].reshape(total, 5)
     off = offsets.cpu().numpy(); bz = busy.cpu().numpy(); ut = util.cpu().numpy()
     assert off[0] == 0 and off[-1] == total
+    sums = device_checksums(E, ctx, records, offsets, n * N)
     order = np.argsort(np.asarray(indices), kind="stable")
     cands = oracle.enumerate_at(w.table, w.space, np.asarray(indices)[order])
     for pos, c in zip(order, cands):
@@ -77,6 +97,8 @@ def check_emission(E, ctx, w, indices):
             raise AssertionError(f"{c}: record {bad}: got {got[bad]}, want {r.records[bad]}")
         assert (bz[pos * N: pos * N + N] == r.busy_ns).all(), c
         np.testing.assert_allclose(ut[pos * N: pos * N + N], r.util, rtol=1e-12, atol=0)
+        for k in (0, N // 2, N - 1):              # the stream checksum of some of its devices
+            assert int(sums[pos * N + k]) == stream_checksum(r.records[r.offsets[k]:r.offsets[k + 1]]), (c, k)
     return total
 
 
@@ -337,6 +359,87 @@ def test_config1_full_size_sampled(E, ctx):
     check_emission(E, ctx, w, pick)
 
 
+def test_config3_every_candidate(E, ctx):
+    """All 650 420 candidates of the 256-device MoE workload against the oracle."""
+    w = W.config3()
+    n = load(E, ctx, w)
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    ob, _ = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS, replicate=False)
+    gb = batch.cpu().numpy()
+    assert (gb == ob).all(), np.argwhere(gb != ob)[:5]
+    order = np.lexsort((np.arange(n), ob))
+    assert E.distsim_argmin(ctx, batch, 0, n) == (order[0], ob[order[0]])
+    ki, kt = dev(1024), dev(1024)
+    E.distsim_topk(ctx, batch, 0, n, 1024, ki, kt)
+    assert (ki.cpu().numpy() == order[:1024]).all() and (kt.cpu().numpy() == ob[order[:1024]]).all()
+
+
+def stratified_indices(table, space, per_cell, seed):
+    """Indices that hit every (row, micro-batch count, schedule) cell of a space with up to
+    `per_cell` partitions each - the first and the last partition among them, hence both ends of
+    every row."""
+    rng = np.random.default_rng(seed)
+    out, off = [], 0
+    for mp, pp, dp, ms, parts, n_sched in W.space_shape(table, space):
+        for e in range(len(ms)):
+            if parts <= per_cell:
+                p = np.arange(parts, dtype=np.int64)
+            else:
+                p = np.unique(np.concatenate([[0, parts - 1], rng.integers(0, parts, per_cell - 2)])).astype(np.int64)
+            for sc in range(n_sched):
+                out.append(off + (e * parts + p) * n_sched + sc)
+        off += len(ms) * parts * n_sched
+    return np.unique(np.concatenate(out)), off
+
+
+def test_config1_stratified_million(E, ctx):
+    """More than a million candidates of the 64-device workload, drawn so that every (row,
+    micro-batch count, schedule) cell and both ends of every row are compared with the oracle."""
+    w = W.config1()
+    n = load(E, ctx, w)
+    idx, total = stratified_indices(w.table, w.space, 10000, 11)
+    assert total == n == 38_838_764 and len(idx) >= 1_000_000 and idx[0] == 0 and idx[-1] == n - 1
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    ob, _ = oracle.eval_indices_parallel(w.table, w.space, idx, THREADS, replicate=False)
+    gb = batch[torch.from_numpy(idx).cuda()].cpu().numpy()
+    assert (gb == ob).all(), idx[np.argwhere(gb != ob)[:5, 0]]
+
+
+def test_stalled_table_copies_fall_back_exactly(E, ctx):
+    """The kernels' first wait for their staged tables is made to give up at once (a host-set poll
+    limit of 0; the second wait keeps its limit, so every copy has landed before its block goes
+    on and nothing hangs): every block then reads its tables from global memory.  Results must be
+    bit-exact, and the next synchronising call must still deliver its outputs while returning
+    DISTSIM_E_TIMEOUT."""
+    for cfg, k in ((1, 64), (3, 64), (2, 16)):      # thread kernel in 32- and 64-bit arithmetic, lock-step kernel
+        w = W.CONFIGS[cfg]()
+        n = load(E, ctx, w)
+        want, wb = eval_all(E, ctx, n)
+        best = E.distsim_argmin(ctx, want, 0, n)
+        E.distsim_testing_set_stage_wait_polls(ctx, 0)
+        try:
+            got, gbz = eval_all(E, ctx, n)
+            assert torch.equal(got, want) and torch.equal(gbz, wb)
+            with pytest.raises(E.DistsimError) as ei:
+                E.distsim_argmin(ctx, got, 0, n)
+            assert ei.value.code == E.E_TIMEOUT and ei.value.result == best
+            assert E.distsim_argmin(ctx, got, 0, n) == best          # the status word was cleared
+            # emission after a stalled evaluation: outputs complete, code reported once
+            got2, _ = eval_all(E, ctx, n, busy=False)
+            top = dev(k)
+            E.distsim_topk(ctx, got2, 0, n, k, top)
+            N = w.table.n_devices
+            off = dev(k * N + 1)
+            with pytest.raises(E.DistsimError) as ei:
+                E.distsim_emit_timelines(ctx, top, k, None, 0, off)
+            assert ei.value.code == E.E_TIMEOUT and ei.value.total_records == int(off[-1]) > 0
+        finally:
+            E.distsim_testing_set_stage_wait_polls(ctx, 1 << 16)
+        again, _ = eval_all(E, ctx, n, busy=False)
+        assert torch.equal(again, want)
+        assert E.distsim_argmin(ctx, again, 0, n) == best
+
+
 def _flat_table(n_layers, n_devices, gpus_per_node, global_batch, space, per_layer_ns, seed):
     """Table whose layer times do not depend on the micro-batch size, so that an entry's time
     bound grows with m: small m fits 32 bits, large m does not."""
@@ -360,7 +463,7 @@ def test_rows_mixing_32_and_64_bit_entries(E, ctx):
     table = _flat_table(16, 16, 4, 64, space, 1 << 24, 5)
     w = W.Workload("mixed_width", table, space, 5)
     n = load(E, ctx, w)
-    cells, cells32 = E.distsim_space_cells(ctx)
+    cells, cells32 = E.distsim_testing_space_cells(ctx)
     assert cells == W.count_candidates_and_cells(table, space)[1] and 0 < cells32 < cells
     batch, sb = eval_all(E, ctx, n)
     rng = np.random.default_rng(0)
@@ -480,12 +583,14 @@ def test_jitter_on_benchmark_shapes(E, ctx):
     assert ei.value.code == E.E_ARG
 
 
-def test_integer_probes_run(E, ctx):
-    for mode in range(4):
-        assert E.distsim_int_issue_probe(ctx, 148, 64, mode) > 0
+def test_integer_probes_run():
+    from paper_2306_08423_b200 import probes
+    sink = dev(1)
+    for mode in range(5):
+        assert probes.distsim_bench_int_issue_probe(148, 64, mode, sink) > 0
     torch.cuda.synchronize()
-    with pytest.raises(E.DistsimError):
-        E.distsim_int_issue_probe(ctx, 148, 64, 9)
+    with pytest.raises(RuntimeError):
+        probes.distsim_bench_int_issue_probe(148, 64, 9, sink)
 
 
 def _emit_chunk_and_check(E, ctx, w, top, sample_positions):
@@ -507,9 +612,12 @@ def _emit_chunk_and_check(E, ctx, w, top, sample_positions):
     assert bool((rec[:, 4] >= rec[:, 3]).all()) and bool((rec[:, 3] >= 0).all())
     assert bool((util > 0).all()) and bool((util <= 1.0).all())
     idx = top.cpu().numpy()
+    sums = device_checksums(E, ctx, records, offsets, n * N)
     for pos in sample_positions:
         c = oracle.enumerate_at(w.table, w.space, np.array([idx[pos]]))[0]
         r = oracle.simulate(w.table, c, replicate=True)
+        want = [stream_checksum(r.records[r.offsets[k]:r.offsets[k + 1]]) for k in range(N)]
+        assert sums[pos * N: (pos + 1) * N].tolist() == want, (pos, c)
         lo, hi = int(offsets[pos * N]), int(offsets[(pos + 1) * N])
         assert hi - lo == r.offsets[-1]
         assert (offsets[pos * N: (pos + 1) * N + 1].cpu().numpy() - lo == r.offsets).all()
@@ -536,7 +644,7 @@ def test_emission_in_the_benchmark_launch_configurations(E, ctx):
     E.distsim_topk(ctx, batch, 0, n, w.top_k, top)
     grand = 0
     for k, i in enumerate(range(0, w.top_k, 128)):
-        grand += _emit_chunk_and_check(E, ctx, w, top[i:i + 128], [(17 * k) % 128] if k % 3 == 0 else [])
+        grand += _emit_chunk_and_check(E, ctx, w, top[i:i + 128], [(17 * k) % 128])
         torch.cuda.empty_cache()
     assert grand > 10**9                              # about 2e9 records, 8e10 bytes in all
 

@@ -33,8 +33,15 @@ def test_static_topk_matches_context_topk_twice_in_a_row():
             E.distsim_topk(ctx, arr, first, n, k, want_i, want_t)
             got_i = torch.full((k,), -1, dtype=torch.int64, device="cuda")
             got_t = torch.full((k,), -1, dtype=torch.int64, device="cuda")
+            torch.cuda.synchronize()
+            free_before, _ = torch.cuda.mem_get_info()
             E.distsim_topk_static(arr, first, n, k, got_i, got_t)
             torch.cuda.synchronize()
+            free_after, _ = torch.cuda.mem_get_info()
+            if arr is second:
+                # the call allocates nothing: by its second use (the first one may load the
+                # kernels' code) the device's free memory is the same before and after
+                assert free_after == free_before
             assert torch.equal(got_i, want_i) and torch.equal(got_t, want_t)    # integers: bit-exact
             st, si = torch.sort(arr, stable=True)
             assert torch.equal(got_t, st[:k]) and torch.equal(got_i, si[:k] + first)
