@@ -495,6 +495,7 @@ def profile_case(name):
     eval1  - evaluation of a 2 M-candidate slice of the 64-device workload (a pp = 16 row, m = 16 and 32)
     eval1m128 - the m = 128 entry of the same row (1 M candidates, 4.0e9 cells)
     eval1m1 - the m = 1 entry of the same row (1 M candidates: unranking and set-up only)
+    eval0  - evaluation of the whole tiny workload (88 candidates)
     eval3  - evaluation of the whole 256-device MoE workload (650 k candidates)
     eval2  - evaluation of the whole 1024-device workload (4 176 candidates, long pipelines)
     eval2pp64 - the pp = 64 rows of the same workload (lock-step kernel, two warps per candidate)
@@ -506,8 +507,8 @@ def profile_case(name):
     from paper_2306_08423_b200 import engine as E
     torch.cuda.set_device(0)
     ctx = E.Context(0)
-    if name in ("eval1", "eval1m1", "eval1m128", "eval3", "eval2", "eval2pp64"):
-        w = {"eval3": W.config3, "eval2": W.config2, "eval2pp64": W.config2}.get(name, W.config1)()
+    if name in ("eval0", "eval1", "eval1m1", "eval1m128", "eval3", "eval2", "eval2pp64"):
+        w = {"eval0": W.config0, "eval3": W.config3, "eval2": W.config2, "eval2pp64": W.config2}.get(name, W.config1)()
         E.distsim_load_event_table(ctx, w.table)
         n = E.distsim_set_space(ctx, w.space)
         first, count = 0, n
@@ -559,7 +560,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-workloads", action="store_true", help="skip the per-workload summary")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
-    ap.add_argument("--profile-case", default=None, help="eval1 | eval1m1 | eval1m128 | eval2 | eval2pp64 | eval3 | emit1 | emit4 | emit4x128: small run for ncu")
+    ap.add_argument("--profile-case", default=None, help="eval0 | eval1 | eval1m1 | eval1m128 | eval2 | eval2pp64 | eval3 | emit1 | emit4 | emit4x128: small run for ncu")
     args = ap.parse_args()
     if args.profile_case:
         profile_case(args.profile_case)

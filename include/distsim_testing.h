@@ -24,6 +24,16 @@ extern "C" {
  */
 int distsim_testing_set_stage_wait_polls(distsim_ctx *ctx, int32_t polls);
 
+/*
+ * Host arithmetic of the evaluation launches (no device involved): cuts the candidates [lo, hi)
+ * of a row with pp stages into pieces of at most max_blocks blocks of the long-pipeline kernel,
+ * as the library does before it launches (so that no range, however large, overflows a grid).
+ * Returns the number of pieces (or DISTSIM_E_ARG) and writes the first max_pieces of them:
+ * h_lo[i], h_hi[i] the piece's candidates, h_blocks[i] its blocks.
+ */
+int64_t distsim_testing_lockstep_pieces(int32_t pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
+                                        int64_t *h_lo, int64_t *h_hi, int32_t *h_blocks);
+
 /* Number of kernels this context has launched so far (launch accounting of the benchmark). */
 int64_t distsim_testing_launch_count(const distsim_ctx *ctx);
 

@@ -172,7 +172,7 @@ int read_status(distsim_ctx *ctx, cudaStream_t s, bool *stalled)
 void destroy_side(SideStream &ss)
 {
     if (ss.fork) cudaEventDestroy(ss.fork);
-    for (int k = 0; k < 2; ++k) {
+    for (int k = 0; k < 1; ++k) {
         if (ss.join[k]) cudaEventDestroy(ss.join[k]);
         if (ss.side[k]) cudaStreamDestroy(ss.side[k]);
     }
@@ -206,14 +206,12 @@ int distsim_create(distsim_ctx **out, int cuda_device)
         distsim_destroy(ctx);
         return DISTSIM_E_CUDA;
     }
-    // the side streams are an optimisation: without them evaluations run on the caller's stream alone
+    // the side stream is an optimisation: without it evaluations run on the caller's stream alone
     int prio_lo = 0, prio_hi = 0;
     if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess ||
         cudaStreamCreateWithPriority(&ctx->side.side[0], cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
-        cudaStreamCreateWithPriority(&ctx->side.side[1], cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->side.fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ctx->side.join[0], cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ctx->side.join[1], cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ctx->side.join[0], cudaEventDisableTiming) != cudaSuccess) {
         cudaGetLastError();
         destroy_side(ctx->side);
     }
@@ -651,6 +649,15 @@ int distsim_testing_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_c
     *h_cells = total >= (__int128)kSat ? kSat : (int64_t)total;
     *h_cells_32bit = narrow >= (__int128)kSat ? kSat : (int64_t)narrow;
     return DISTSIM_OK;
+}
+
+int64_t distsim_testing_lockstep_pieces(int32_t pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
+                                        int64_t *h_lo, int64_t *h_hi, int32_t *h_blocks)
+{
+    if (pp < 1 || pp > DISTSIM_MAX_PP || (pp & (pp - 1)) || lo < 0 || hi < lo || max_blocks < 1 || max_pieces < 0 ||
+        (max_pieces > 0 && (!h_lo || !h_hi || !h_blocks)))
+        return DISTSIM_E_ARG;
+    return lockstep_pieces(pp, lo, hi, max_blocks, max_pieces, h_lo, h_hi, h_blocks);
 }
 
 int distsim_testing_set_stage_wait_polls(distsim_ctx *ctx, int32_t polls)

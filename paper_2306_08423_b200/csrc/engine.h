@@ -173,12 +173,12 @@ struct EvalBatch {
     int32_t n, pad;
     EvalWork w[kMaxEvalWork];
 };
-// Two more streams for the latency-bound lock-step launches of an evaluation (one per kernel
-// instance), so that they run beside each other and beside the throughput-bound launches
-// instead of one after the other (side[0] == nullptr: everything on the caller's stream).
+// One more stream for the latency-bound lock-step launch of an evaluation, so that it runs
+// beside the throughput-bound launches instead of before them (side[0] == nullptr: everything
+// on the caller's stream).
 struct SideStream {
-    cudaStream_t side[2] = {nullptr, nullptr};
-    cudaEvent_t fork = nullptr, join[2] = {nullptr, nullptr};
+    cudaStream_t side[1] = {nullptr};
+    cudaEvent_t fork = nullptr, join[1] = {nullptr};
 };
 // Evaluates candidates [first, first + count); rows / entries: host copies.  Results go to
 // batch_out[index - first] and, if non-null, busy_out[(index - first) * pp_max + d].  All work
@@ -186,6 +186,10 @@ struct SideStream {
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
                  int64_t *launches);
+// Cuts candidates [lo, hi) of a row of pp stages into pieces of at most max_blocks lock-step
+// blocks each; returns the number of pieces and writes the first max_pieces of them.
+int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
+                        int64_t *piece_lo, int64_t *piece_hi, int32_t *piece_blocks);
 
 // ---- selection (select_kernels.cu) -----------------------------------------------------
 struct SelectScratch {

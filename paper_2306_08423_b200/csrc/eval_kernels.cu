@@ -12,6 +12,8 @@
 // A search space has a few dozen rows, many of them tiny; launching them one by one would leave
 // the device idle between kernels, so one launch carries a list of (row, range) work items and
 // every block looks up the item it belongs to.
+#include <vector>
+
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
 #include "eval_thread.cuh"
@@ -20,26 +22,24 @@ namespace distsim {
 
 namespace {
 
-constexpr int kEvalThreads = 256;
+// Threads per block of the lock-step kernel.  Blocks are small so that the long candidates of
+// a row (many micro-batches: hundreds of slots) spread over all SMs instead of sharing a few.
+constexpr int kEvalThreads = 64;
 
+// The part of a block's work that depends on the number of stages a lane owns.
 template <int S, bool kJit>
-__global__ void __launch_bounds__(kEvalThreads)
-eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
-                     int64_t *__restrict__ busy_out, int smem_words)
+__device__ __forceinline__ void lockstep_block(const DeviceView &v, const EvalWork &wk, const Row &row, int local_block,
+                                               int64_t first, int64_t *__restrict__ batch_out,
+                                               int64_t *__restrict__ busy_out, int smem_words,
+                                               unsigned char *smem_raw, uint64_t *bar)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t bar;
-    int wi = 0;
-    while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
-    const EvalWork &wk = batch.w[wi];
     const int64_t lo = wk.lo, hi = wk.hi;
-    const Row row = v.rows[wk.row];
     const int pp = row.pp;
     const int wl = pp / S;                         // lanes of a warp per candidate
     const int warps = blockDim.x >> 5;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int cpb = warps * (32 / wl);             // candidates per block
-    const int64_t cta_first = lo + (int64_t)((int)blockIdx.x - wk.block_begin) * cpb;
+    const int64_t cta_first = lo + (int64_t)local_block * cpb;
     if (cta_first >= hi) return;                   // the whole block leaves: no barrier is left waiting
     const int64_t cta_last = min(hi, cta_first + (int64_t)cpb) - 1;
 
@@ -54,7 +54,7 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     bool staged = false;
     if (max_stage_entries > 0 && n_stage <= max_stage_entries) {
         const uint32_t bytes = (uint32_t)(n_stage * lp * sizeof(int64_t));
-        staged = stage_two_tables(&bar, sm_f, v.etf + (int64_t)e_lo * lp, sm_b,
+        staged = stage_two_tables(bar, sm_f, v.etf + (int64_t)e_lo * lp, sm_b,
                                   v.etb + (int64_t)e_lo * lp, bytes, v.status, v.stage_polls);
     }
 
@@ -83,6 +83,24 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     }
 }
 
+template <bool kJit>
+__global__ void __launch_bounds__(kEvalThreads)
+eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
+                     int64_t *__restrict__ busy_out, int smem_words)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bar;
+    int wi = 0;
+    while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
+    const EvalWork &wk = batch.w[wi];
+    const Row row = v.rows[wk.row];
+    // A row's candidates grow in micro-batch count, hence in slots, with their index: its last
+    // blocks are the long ones and take the first block numbers, so that they start first.
+    const int local_block = wk.nx - 1 - ((int)blockIdx.x - wk.block_begin);
+    if (row.pp > 32) lockstep_block<2, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar);
+    else lockstep_block<1, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar);
+}
+
 // Work items collected for one kernel instance, launched when full or at the end.
 struct Pending {
     EvalBatch batch{};
@@ -90,16 +108,12 @@ struct Pending {
     int smem_words = 0;
 };
 
+constexpr int kMaxBlocks = 1 << 30;                // blocks of one launch
+
 // Candidates per block of the lock-step kernel: 32 / pp per warp, one per warp (two stages per lane) at pp = 64.
 int lockstep_cpb(const Row &row)
 {
     return row.pp > 32 ? kEvalThreads / 32 : (kEvalThreads / 32) * (32 / row.pp);
-}
-
-int lockstep_blocks(const Row &row, int64_t lo, int64_t hi)
-{
-    const int cpb = lockstep_cpb(row);
-    return (int)((hi - lo + cpb - 1) / cpb);
 }
 
 int lockstep_smem_words(const DeviceView &v, const Row &row)
@@ -112,18 +126,17 @@ int lockstep_smem_words(const DeviceView &v, const Row &row)
     return words * (int64_t)sizeof(int64_t) > 96 * 1024 ? 0 : (int)words;     // too wide: global reads
 }
 
-template <int S>
 void flush_lockstep(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first, int64_t *batch_out,
                     int64_t *busy_out, int64_t *launches)
 {
     if (p.batch.n == 0) return;
     const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
     if (v.tc.n_jitter > 0) {
-        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_lockstep_kernel<S, true>), smem);
-        eval_lockstep_kernel<S, true><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_lockstep_kernel<true>), smem);
+        eval_lockstep_kernel<true><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
     } else {
-        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_lockstep_kernel<S, false>), smem);
-        eval_lockstep_kernel<S, false><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_lockstep_kernel<false>), smem);
+        eval_lockstep_kernel<false><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
     }
     ++*launches;
     p = Pending{};
@@ -188,38 +201,49 @@ int thread_budget_words(int pp, bool narrow, bool jitter)
 
 }  // namespace
 
+// Cuts candidates [lo, hi) of a row of `pp` stages into pieces of at most max_blocks blocks of the
+// lock-step kernel each (block counts are computed in 64 bits: a range of billions of candidates
+// must not overflow a launch's grid).  Returns the number of pieces; the first max_pieces are
+// written.
+int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
+                        int64_t *piece_lo, int64_t *piece_hi, int32_t *piece_blocks)
+{
+    Row row{};
+    row.pp = pp;
+    const int64_t cpb = lockstep_cpb(row);
+    const int64_t per_piece = max_blocks * cpb;            // candidates
+    int64_t n = 0;
+    for (int64_t a = lo; a < hi; a += per_piece, ++n) {
+        const int64_t b = hi - a < per_piece ? hi : a + per_piece;
+        if (n < max_pieces) {
+            piece_lo[n] = a; piece_hi[n] = b;
+            piece_blocks[n] = (int32_t)((b - a + cpb - 1) / cpb);
+        }
+    }
+    return n;
+}
+
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
                  int64_t *launches)
 {
     const int64_t last = first + count;
-    // lock-step launches go to the side streams, forked from `s` on first use and joined at the end
-    bool fork_recorded = false, forked[2] = {false, false};
-    auto lockstep_stream = [&](int which) {
-        if (!ss.side[0]) return s;
-        if (!fork_recorded) { cudaEventRecord(ss.fork, s); fork_recorded = true; }
-        if (!forked[which]) { cudaStreamWaitEvent(ss.side[which], ss.fork, 0); forked[which] = true; }
-        return ss.side[which];
-    };
-    Pending lock[2];                               // lock-step kernel: a warp segment, or a pair of warps, per candidate
-    Pending thr[5][2];                             // thread kernel, [log2 pp][narrow]
-    constexpr int kMaxBlocks = 1 << 30;
+    struct ThreadItem { EvalWork w; int lg; bool narrow; int blocks, words; };
+    std::vector<EvalWork> lock_items;              // lock-step kernel
+    std::vector<int> lock_words;
+    std::vector<ThreadItem> thread_items;          // one-partition-per-thread kernel
+    constexpr int64_t kPieceBlocks = 1 << 24;
 
     auto add_lockstep = [&](int r, int64_t lo, int64_t hi) {
-        const int which = rows[r].pp > 32 ? 1 : 0;
-        Pending &p = lock[which];
-        const int blocks = lockstep_blocks(rows[r], lo, hi);
-        if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - blocks) {
-            if (which) flush_lockstep<2>(lockstep_stream(1), v, p, first, batch_out, busy_out, launches);
-            else flush_lockstep<1>(lockstep_stream(0), v, p, first, batch_out, busy_out, launches);
+        for (int64_t a = lo; a < hi;) {
+            int64_t pl, ph; int32_t blocks;
+            lockstep_pieces(rows[r].pp, a, hi, kPieceBlocks, 1, &pl, &ph, &blocks);
+            EvalWork w{};
+            w.row = r; w.lo = pl; w.hi = ph; w.nx = blocks;
+            lock_items.push_back(w);
+            lock_words.push_back(lockstep_smem_words(v, rows[r]));
+            a = ph;
         }
-        EvalWork &w = p.batch.w[p.batch.n++];
-        w = EvalWork{};
-        w.row = r; w.lo = lo; w.hi = hi; w.block_begin = p.blocks;
-        p.blocks += blocks;
-        const int words = lockstep_smem_words(v, rows[r]);
-        // one dynamic size per launch: the largest any item wants (items that want none still work)
-        if (words > p.smem_words) p.smem_words = words;
     };
 
     for (int r = 0; r < n_rows; ++r) {
@@ -252,40 +276,66 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
             const int64_t nx = (n_parts + kThreadBlock - 1) / kThreadBlock;
             const int64_t ny = (n_e + ept - 1) / ept;
             if (n_parts * ny >= 2048 && nx * ny < kMaxBlocks) {
-                const int lg = ilog2(row.pp);
-                Pending &p = thr[lg][narrow ? 1 : 0];
-                if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - (int)(nx * ny))
-                    flush_thread_any(lg, narrow, s, v, p, first, batch_out, busy_out, launches);
-                EvalWork &w = p.batch.w[p.batch.n++];
-                w = EvalWork{};
+                ThreadItem it{};
+                it.lg = ilog2(row.pp); it.narrow = narrow; it.blocks = (int)(nx * ny);
+                EvalWork &w = it.w;
                 w.row = r; w.e_begin = r0; w.e_end = r1; w.ept = ept; w.p_lo = p_lo; w.p_hi = p_hi;
-                w.lo = lo_r; w.hi = hi_r; w.block_begin = p.blocks; w.nx = (int)nx;
-                p.blocks += (int)(nx * ny);
+                w.lo = lo_r; w.hi = hi_r; w.nx = (int)nx;
                 const int binom_words = v.sc.partition_mode ? v.tc.n_layers * v.sc.binom_k : 0;
                 const int budget = thread_budget_words(row.pp, narrow, v.tc.n_jitter > 0);
                 const bool use32 = narrow && v.pfb32 != nullptr && (row.dp == 1 || v.dt32 != nullptr);   // as in the kernel
-                const int words =
+                it.words =
                     use32 ? thread_kernel_smem32(row.n_entries, v.tc.lp, v.tab_words32, v.dt32 != nullptr, binom_words, budget).words
                           : thread_kernel_smem(row.n_entries, v.tc.lp, v.tab_words, v.dt != nullptr, binom_words, budget).words;
-                if (words > p.smem_words) p.smem_words = words;
+                thread_items.push_back(it);
             } else {
                 add_lockstep(r, lo_r, hi_r);
             }
             r0 = r1;
         }
     }
-    // the lock-step launches first, on their own streams: few blocks that run for long, beside
-    // the thread-kernel launches (largest first) that fill the rest of the device
-    if (lock[1].batch.n) flush_lockstep<2>(lockstep_stream(1), v, lock[1], first, batch_out, busy_out, launches);
-    if (lock[0].batch.n) flush_lockstep<1>(lockstep_stream(0), v, lock[0], first, batch_out, busy_out, launches);
+
+    // The lock-step launches (few warps that run for long) go first, on a high-priority side
+    // stream forked from `s` and joined to it at the end, so that they run beside the
+    // thread-kernel launches (largest first) that fill the rest of the device.  Without
+    // thread-kernel work there is nothing to run beside: everything goes to `s` directly.
+    const bool use_side = ss.side[0] != nullptr && !thread_items.empty() && !lock_items.empty();
+    cudaStream_t ls = s;
+    if (use_side) {
+        cudaEventRecord(ss.fork, s);
+        cudaStreamWaitEvent(ss.side[0], ss.fork, 0);
+        ls = ss.side[0];
+    }
+    Pending p;
+    for (size_t i = 0; i < lock_items.size(); ++i) {
+        if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - lock_items[i].nx)
+            flush_lockstep(ls, v, p, first, batch_out, busy_out, launches);
+        EvalWork &w = p.batch.w[p.batch.n++];
+        w = lock_items[i];
+        w.block_begin = p.blocks;
+        p.blocks += w.nx;
+        // one dynamic size per launch: the largest any item wants (items that want none still work)
+        if (lock_words[i] > p.smem_words) p.smem_words = lock_words[i];
+    }
+    flush_lockstep(ls, v, p, first, batch_out, busy_out, launches);
     for (int lg = 4; lg >= 0; --lg)
-        for (int nw = 1; nw >= 0; --nw)
-            flush_thread_any(lg, nw == 1, s, v, thr[lg][nw], first, batch_out, busy_out, launches);
-    for (int k = 0; k < 2; ++k)
-        if (forked[k]) {
-            cudaEventRecord(ss.join[k], ss.side[k]);
-            cudaStreamWaitEvent(s, ss.join[k], 0);
+        for (int nw = 1; nw >= 0; --nw) {
+            for (const ThreadItem &it : thread_items) {
+                if (it.lg != lg || it.narrow != (nw == 1)) continue;
+                if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - it.blocks)
+                    flush_thread_any(lg, nw == 1, s, v, p, first, batch_out, busy_out, launches);
+                EvalWork &w = p.batch.w[p.batch.n++];
+                w = it.w;
+                w.block_begin = p.blocks;
+                p.blocks += it.blocks;
+                if (it.words > p.smem_words) p.smem_words = it.words;
+            }
+            flush_thread_any(lg, nw == 1, s, v, p, first, batch_out, busy_out, launches);
         }
+    if (use_side) {
+        cudaEventRecord(ss.join[0], ss.side[0]);
+        cudaStreamWaitEvent(s, ss.join[0], 0);
+    }
 }
 
 }  // namespace distsim

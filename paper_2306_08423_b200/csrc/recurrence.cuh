@@ -271,8 +271,16 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         // event starts one backward item cost before its end
         R.last_b_start[k] = t[k] - R.bop[k];
         // the asynchronous schedule has no gradient all-reduce events
-        R.dp_end[k] = sched == 2 ? R.main_end[k]
-                                 : bucket_lane_end(v, row, pb, nbt, tpt, R.a[k], R.e[k], R.last_b_start[k], R.main_end[k]);
+        if (sched == 2 || row.dp == 1) {
+            R.dp_end[k] = R.main_end[k];
+        } else if (v.dt) {
+            // per-entry bucket-lane table: the lane's end relative to the start of the last
+            // backward item (overlap; negative: no buckets) or the buckets' total cost
+            const int64_t val = __ldg(&v.dt[(int64_t)entry_index * v.tab_words + R.e[k] * (v.tc.n_layers + 1) + R.a[k]]);
+            R.dp_end[k] = v.tc.overlap ? (val < 0 ? R.main_end[k] : R.last_b_start[k] + val) : R.main_end[k] + val;
+        } else {
+            R.dp_end[k] = bucket_lane_end(v, row, pb, nbt, tpt, R.a[k], R.e[k], R.last_b_start[k], R.main_end[k]);
+        }
         const int64_t extra = R.dp_end[k] - R.main_end[k];
         R.busy[k] = (int64_t)m * (R.fop[k] + R.bop[k]) + (extra > 0 ? extra : 0) +
                     (kJit ? __ldg(&v.jsum[(int64_t)entry_index * DISTSIM_MAX_PP + d0 + k]) : 0);

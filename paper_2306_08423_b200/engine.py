@@ -27,7 +27,7 @@ EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error",
            "distsim_topk_static")
 # hooks of include/distsim_testing.h (test-suite and benchmark accounting; not the stable ABI)
 TESTING_EXPORTS = ("distsim_testing_set_stage_wait_polls", "distsim_testing_launch_count",
-                   "distsim_testing_space_cells")
+                   "distsim_testing_space_cells", "distsim_testing_lockstep_pieces")
 TOPK_STATIC_MAX_K = 1024
 
 if not os.path.exists(LIB_PATH):
@@ -76,6 +76,9 @@ _lib.distsim_last_error.restype = C.c_char_p
 _lib.distsim_testing_launch_count.argtypes = [C.c_void_p]
 _lib.distsim_testing_launch_count.restype = C.c_int64
 _lib.distsim_testing_set_stage_wait_polls.argtypes = [C.c_void_p, C.c_int32]
+_lib.distsim_testing_lockstep_pieces.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
+                                                 C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.distsim_testing_lockstep_pieces.restype = C.c_int64
 _lib.distsim_load_event_table.argtypes = [C.c_void_p, C.POINTER(_Table)]
 _lib.distsim_set_space.argtypes = [C.c_void_p, C.POINTER(_Space), C.POINTER(C.c_int64)]
 _lib.distsim_decode.argtypes = [C.c_void_p, C.c_int64, C.POINTER(_Candidate)]
@@ -311,6 +314,17 @@ def distsim_testing_space_cells(ctx: Context):
     a, b = C.c_int64(0), C.c_int64(0)
     ctx._check(_lib.distsim_testing_space_cells(ctx._h, C.byref(a), C.byref(b)))
     return int(a.value), int(b.value)
+
+
+def distsim_testing_lockstep_pieces(pp: int, lo: int, hi: int, max_blocks: int, max_pieces: int = 64):
+    """(number of pieces, [(lo, hi, blocks) of the first max_pieces])."""
+    a, b = np.zeros(max(1, max_pieces), np.int64), np.zeros(max(1, max_pieces), np.int64)
+    c = np.zeros(max(1, max_pieces), np.int32)
+    n = int(_lib.distsim_testing_lockstep_pieces(pp, lo, hi, max_blocks, max_pieces, _np_ptr(a), _np_ptr(b), _np_ptr(c)))
+    if n < 0:
+        raise DistsimError(n, "bad arguments")
+    k = min(n, max_pieces)
+    return n, list(zip(a[:k].tolist(), b[:k].tolist(), c[:k].tolist()))
 
 
 def distsim_testing_launch_count(ctx: Context) -> int:

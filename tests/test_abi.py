@@ -53,3 +53,21 @@ def test_create_fails_loudly_without_a_gpu():
     with pytest.raises(engine.DistsimError) as ei:
         engine.Context(0)
     assert ei.value.code == engine.E_CUDA
+
+
+def test_long_pipeline_ranges_are_cut_into_launchable_pieces():
+    # host arithmetic only: block counts in 64 bits, pieces cover the range exactly once
+    from paper_2306_08423_b200 import engine
+    for pp, cpb in ((64, 2), (32, 2), (16, 4), (1, 64)):
+        for lo, hi in ((0, 1), (5, 5), (3, 1000), (0, 8_600_000_000), (7, 2**40 + 11)):
+            max_blocks = 1 << 24
+            n, pieces = engine.distsim_testing_lockstep_pieces(pp, lo, hi, max_blocks, 4096)
+            assert n == -(-(hi - lo) // (max_blocks * cpb))
+            pos = lo
+            for a, b, blocks in pieces:
+                assert a == pos and a < b <= hi and blocks == -(-(b - a) // cpb) and 1 <= blocks <= max_blocks
+                pos = b
+            if n <= 4096:
+                assert pos == (hi if hi > lo else lo)
+    with __import__("pytest").raises(engine.DistsimError):
+        engine.distsim_testing_lockstep_pieces(3, 0, 10, 16)
