@@ -98,14 +98,22 @@ __device__ __forceinline__ SlotPlan slot_plan(int sched, int pp, int m, int d)
     else { sp.w = min(pp - d, m); sp.b0 = 2 * pp - 1 - d; sp.sh = 1; }
     return sp;
 }
-// Does stage d run a forward / backward item in slot s, and of which micro-batch j?
-__device__ __forceinline__ void slot_activity(const SlotPlan &sp, int m, int d, int s, bool &do_f, bool &do_b, int &j)
+// Activity of a stage over the kChunk slots s0 .. s0 + kChunk - 1 as bit masks (bit i: slot
+// s0 + i): `fwd` the slots with a forward item, `bwd` those with a backward item.  Computed once
+// per chunk, so that the slots themselves only test a bit.
+constexpr int kChunk = 16;
+__device__ __forceinline__ uint32_t slot_range_mask(int lo_slot, int hi_slot, int s0)
 {
-    const int x = s - d, y = s - sp.b0;
-    const bool warm = (unsigned)x < (unsigned)sp.w;
-    do_f = warm || (x >= 2 * sp.w && !(x & 1) && (x >> 1) < m);
-    do_b = y >= 0 && !(y & sp.sh) && (y >> sp.sh) < m;
-    j = do_f ? (warm ? x : x >> 1) : y >> sp.sh;
+    const int lo = min(max(lo_slot - s0, 0), kChunk), hi = min(max(hi_slot - s0, 0), kChunk);
+    return hi > lo ? (1u << hi) - (1u << lo) : 0u;
+}
+__device__ __forceinline__ void chunk_activity(const SlotPlan &sp, int m, int d, int s0, uint32_t &fwd, uint32_t &bwd)
+{
+    // bits of the slots whose distance from slot `from` is even
+    auto alternate = [&](int from) { return ((from - s0) & 1) ? 0xAAAAAAAAu : 0x55555555u; };
+    fwd = slot_range_mask(d, d + sp.w, s0) |                                          // d + j, j < w
+          (slot_range_mask(d + 2 * sp.w, d + 2 * m - 1, s0) & alternate(d));          // d + 2j, w <= j < m
+    bwd = slot_range_mask(sp.b0, sp.b0 + ((m - 1) << sp.sh) + 1, s0) & (sp.sh ? alternate(sp.b0) : 0xFFFFFFFFu);
 }
 
 // Extra time of the item of micro-batch j on stage d (0 without a jitter table).
@@ -216,47 +224,59 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         sp[k] = slot_plan(sched, pp, m, d);
     }
     int64_t t[S];
-    int n_done[S];
+    int n_f[S], n_b[S];                  // forward / backward items done: the next item's micro-batch
 #pragma unroll
-    for (int k = 0; k < S; ++k) { t[k] = 0; n_done[k] = 0; }
+    for (int k = 0; k < S; ++k) { t[k] = 0; n_f[k] = 0; n_b[k] = 0; }
     const int lane = threadIdx.x & 31;
+    // where a forward (backward) item's input comes from: the previous (next) lane, or the lane
+    // itself when there is no such stage (one stage per lane)
+    const int src_f = d0 > 0 ? lane - 1 : lane, src_b = d0 < pp - 1 ? lane + 1 : lane;
 
-    for (int s = 0; s < n_slots_warp; ++s) {
-        if (S == 1) {
-            bool do_f, do_b;
-            int j;
-            slot_activity(sp[0], m, d0, s, do_f, do_b, j);
-            const int src = lane - ((do_f && d0 > 0) ? 1 : 0) + ((do_b && d0 < pp - 1) ? 1 : 0);
-            const int64_t dep = shfl_idx64(t[0], src);
-            int64_t cost = do_f ? R.fop[0] : (do_b ? R.bop[0] : 0);
-            const int64_t st = max64(dep, t[0]);
-            if (kJit) cost += (do_f || do_b) ? jitter_of(v, do_f ? v.raw.jit_f : v.raw.jit_b, j, d0) : 0;
-            if (kRecord && rec && (do_f || do_b)) rec[(int64_t)d0 * 2 * m + n_done[0]] = st;
-            if (kRecord) n_done[0] += (do_f || do_b) ? 1 : 0;
-            t[0] = st + cost;
-        } else {
-            // several stages per lane: the lane's first (last) stage takes the previous (next)
-            // lane's last (first) stage, the others their neighbour inside the lane
-            const int64_t up_f = __shfl_up_sync(0xffffffffu, t[S - 1], 1, wl);
-            const int64_t dn_b = __shfl_down_sync(0xffffffffu, t[0], 1, wl);
-            int64_t old[S];
+    for (int s0 = 0; s0 < n_slots_warp; s0 += kChunk) {
+        uint32_t fm[S], bm[S];
 #pragma unroll
-            for (int k = 0; k < S; ++k) old[k] = t[k];
+        for (int k = 0; k < S; ++k) chunk_activity(sp[k], m, d0 + k, s0, fm[k], bm[k]);
 #pragma unroll
-            for (int k = 0; k < S; ++k) {
-                const int d = d0 + k;
-                bool do_f, do_b;
-                int j;
-                slot_activity(sp[k], m, d, s, do_f, do_b, j);
-                const int64_t dep_f = (k == 0) ? (d == 0 ? 0 : up_f) : old[k > 0 ? k - 1 : 0];
-                const int64_t dep_b = (k == S - 1) ? (d == pp - 1 ? 0 : dn_b) : old[k < S - 1 ? k + 1 : 0];
-                const int64_t dep = do_f ? dep_f : (do_b ? dep_b : 0);
-                int64_t cost = do_f ? R.fop[k] : (do_b ? R.bop[k] : 0);
-                const int64_t st = max64(dep, old[k]);
-                if (kJit) cost += (do_f || do_b) ? jitter_of(v, do_f ? v.raw.jit_f : v.raw.jit_b, j, d) : 0;
-                if (kRecord && rec && (do_f || do_b)) rec[(int64_t)d * 2 * m + n_done[k]] = st;
-                if (kRecord) n_done[k] += (do_f || do_b) ? 1 : 0;
-                t[k] = st + cost;
+        for (int i = 0; i < kChunk; ++i) {
+            if (S == 1) {
+                const bool do_f = (fm[0] >> i) & 1u, do_b = (bm[0] >> i) & 1u;
+                int64_t cost = do_f ? R.fop[0] : (do_b ? R.bop[0] : 0);
+                if (kJit) {
+                    if (do_f) cost += jitter_of(v, v.raw.jit_f, n_f[0], d0);
+                    if (do_b) cost += jitter_of(v, v.raw.jit_b, n_b[0], d0);
+                }
+                const int64_t dep = shfl_idx64(t[0], do_f ? src_f : (do_b ? src_b : lane));
+                const int64_t own = t[0] + cost, via = dep + cost;       // both ready before the compare ends
+                const bool late = dep > t[0];
+                t[0] = late ? via : own;
+                if (kRecord && rec && (do_f || do_b)) rec[(int64_t)d0 * 2 * m + n_f[0] + n_b[0]] = t[0] - cost;
+                if (kRecord || kJit) { n_f[0] += do_f ? 1 : 0; n_b[0] += do_b ? 1 : 0; }
+            } else {
+                // several stages per lane: the lane's first (last) stage takes the previous (next)
+                // lane's last (first) stage, the others their neighbour inside the lane
+                const int64_t up_f = __shfl_up_sync(0xffffffffu, t[S - 1], 1, wl);
+                const int64_t dn_b = __shfl_down_sync(0xffffffffu, t[0], 1, wl);
+                int64_t old[S];
+#pragma unroll
+                for (int k = 0; k < S; ++k) old[k] = t[k];
+#pragma unroll
+                for (int k = 0; k < S; ++k) {
+                    const int d = d0 + k;
+                    const bool do_f = (fm[k] >> i) & 1u, do_b = (bm[k] >> i) & 1u;
+                    int64_t cost = do_f ? R.fop[k] : (do_b ? R.bop[k] : 0);
+                    if (kJit) {
+                        if (do_f) cost += jitter_of(v, v.raw.jit_f, n_f[k], d);
+                        if (do_b) cost += jitter_of(v, v.raw.jit_b, n_b[k], d);
+                    }
+                    const int64_t dep_f = (k == 0) ? (d == 0 ? 0 : up_f) : old[k > 0 ? k - 1 : 0];
+                    const int64_t dep_b = (k == S - 1) ? (d == pp - 1 ? 0 : dn_b) : old[k < S - 1 ? k + 1 : 0];
+                    const int64_t dep = do_f ? dep_f : (do_b ? dep_b : 0);
+                    const int64_t own = old[k] + cost, via = dep + cost;
+                    const bool late = dep > old[k];
+                    t[k] = late ? via : own;
+                    if (kRecord && rec && (do_f || do_b)) rec[(int64_t)d * 2 * m + n_f[k] + n_b[k]] = t[k] - cost;
+                    if (kRecord || kJit) { n_f[k] += do_f ? 1 : 0; n_b[k] += do_b ? 1 : 0; }
+                }
             }
         }
     }
