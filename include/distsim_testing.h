@@ -34,6 +34,15 @@ int distsim_testing_set_stage_wait_polls(distsim_ctx *ctx, int32_t polls);
 int64_t distsim_testing_lockstep_pieces(int32_t pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
                                         int64_t *h_lo, int64_t *h_hi, int32_t *h_blocks);
 
+/*
+ * Phase timing of distsim_eval_select for the benchmark: with enable != 0 the call records CUDA
+ * events on its stream before the evaluation launches, after them and after the selection
+ * launches; distsim_testing_last_phase_ms returns the two durations of the most recent such
+ * call (it must have completed: distsim_eval_select synchronises before it returns).
+ */
+int distsim_testing_time_phases(distsim_ctx *ctx, int32_t enable);
+int distsim_testing_last_phase_ms(distsim_ctx *ctx, float *h_eval_ms, float *h_select_ms);
+
 /* Number of kernels this context has launched so far (launch accounting of the benchmark). */
 int64_t distsim_testing_launch_count(const distsim_ctx *ctx);
 

@@ -70,6 +70,8 @@ struct distsim_ctx {
     int64_t time_bound = 0;
     int64_t op_words_per_cand = 0;
     int32_t stage_polls = 1 << 16;        // polls of the first wait for staged tables
+    cudaEvent_t phase_ev[3] = {nullptr, nullptr, nullptr};   // timing of distsim_eval_select's phases (hook)
+    bool phase_timing = false, phase_valid = false;
     DevBuf d_rows, d_entries, d_etf, d_etb, d_nb, d_tp, d_binom, d_dt, d_pfb32, d_dt32;
     bool have_dt = false, have_narrow = false;
 
@@ -223,6 +225,7 @@ void distsim_destroy(distsim_ctx *ctx)
 {
     if (!ctx) return;
     cudaSetDevice(ctx->device);
+    for (cudaEvent_t e : ctx->phase_ev) if (e) cudaEventDestroy(e);
     if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
     destroy_side(ctx->side);
     delete ctx;
@@ -521,9 +524,47 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const DeviceView v = ctx->view();
     launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
-                d_batch_ns, d_stage_busy_ns, &ctx->launches);
+                d_batch_ns, d_stage_busy_ns, FusedSelect{}, &ctx->launches);
     CU(cudaGetLastError(), "evaluation launch");
     return DISTSIM_OK;
+}
+
+int distsim_eval_select(distsim_ctx *ctx, void *stream, int64_t first, int64_t count, int64_t *d_batch_ns,
+                        int32_t k, int64_t *d_indices, int64_t *d_times, int64_t *h_best_index,
+                        int64_t *h_best_batch_ns)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
+    if (!d_batch_ns || !h_best_index || !h_best_batch_ns) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (first < 0 || count < 1 || first > ctx->sc.n_candidates || count > ctx->sc.n_candidates - first)
+        return fail(ctx, DISTSIM_E_RANGE, "candidate range outside the space");
+    if (k < 0 || k > 4096 || k > count || (k > 0 && !d_indices))
+        return fail(ctx, DISTSIM_E_ARG, "k must be in [0, min(count, 4096)] and d_indices non-null for k > 0");
+    if (int rc = set_device(ctx)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const DeviceView v = ctx->view();
+    const SelectScratch sc = ctx->select_scratch();
+    const FusedSelect fs = begin_fused_select(s, count, k, ctx->time_bound, sc, &ctx->launches);
+    if (ctx->phase_timing) cudaEventRecord(ctx->phase_ev[0], s);
+    launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
+                d_batch_ns, nullptr, fs, &ctx->launches);
+    CU(cudaGetLastError(), "evaluation launch");
+    if (ctx->phase_timing) cudaEventRecord(ctx->phase_ev[1], s);
+    if (fs.enabled) {
+        finish_fused_argmin(s, fs, sc, ctx->d_result.as<int64_t>(), &ctx->launches);
+        if (k > 0) finish_fused_topk(s, fs, d_batch_ns, first, count, k, ctx->time_bound, sc, d_indices, d_times, &ctx->launches);
+    } else {
+        launch_argmin(s, d_batch_ns, count, ctx->time_bound, sc, ctx->d_result.as<int64_t>(), &ctx->launches);
+        if (k > 0) launch_topk(s, d_batch_ns, first, count, k, ctx->time_bound, sc, d_indices, d_times, &ctx->launches);
+    }
+    CU(cudaGetLastError(), "selection launch");
+    if (ctx->phase_timing) { cudaEventRecord(ctx->phase_ev[2], s); ctx->phase_valid = true; }
+    CU(cudaMemcpyAsync(ctx->h_pinned, ctx->d_result.p, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, s), "argmin readback");
+    bool stalled = false;
+    if (int rc = read_status(ctx, s, &stalled)) return rc;          // synchronises
+    *h_best_batch_ns = ctx->h_pinned[0];
+    *h_best_index = first + ctx->h_pinned[1];
+    return stalled ? fail(ctx, DISTSIM_E_TIMEOUT, kTimeoutText) : DISTSIM_OK;
 }
 
 int distsim_argmin(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int64_t first,
@@ -618,17 +659,21 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table, co
     *h_n_candidates = n;
     CU(ctx->d_batch.reserve((size_t)n * sizeof(int64_t)), "alloc batch times");
     int64_t *d_batch = ctx->d_batch.as<int64_t>();
-    if (int rc = distsim_eval_strategies(ctx, nullptr, 0, n, d_batch, nullptr)) return rc;
+    if (k > n) k = (int32_t)n;
+    if (k > 4096) k = 4096;
+    int64_t *d_idx = nullptr;
     if (k > 0) {
-        if (k > n) k = (int32_t)n;
-        if (k > 4096) k = 4096;
         CU(ctx->d_topk.reserve((size_t)2 * k * sizeof(int64_t)), "alloc top-k");
-        int64_t *d_idx = ctx->d_topk.as<int64_t>();
-        if (int rc = distsim_topk(ctx, nullptr, d_batch, 0, n, k, d_idx, d_idx + k)) return rc;
-        CU(cudaMemcpyAsync(h_topk_indices, d_idx, (size_t)k * sizeof(int64_t), cudaMemcpyDeviceToHost, 0), "top-k readback");
-        CU(cudaMemcpyAsync(h_topk_times, d_idx + k, (size_t)k * sizeof(int64_t), cudaMemcpyDeviceToHost, 0), "top-k readback");
+        d_idx = ctx->d_topk.as<int64_t>();
     }
-    return distsim_argmin(ctx, nullptr, d_batch, 0, n, h_best_index, h_best_batch_ns);
+    const int rc = distsim_eval_select(ctx, nullptr, 0, n, d_batch, k, d_idx, d_idx ? d_idx + k : nullptr,
+                                       h_best_index, h_best_batch_ns);          // synchronises
+    if (rc != DISTSIM_OK && rc != DISTSIM_E_TIMEOUT) return rc;
+    if (k > 0) {
+        CU(cudaMemcpy(h_topk_indices, d_idx, (size_t)k * sizeof(int64_t), cudaMemcpyDeviceToHost), "top-k readback");
+        CU(cudaMemcpy(h_topk_times, d_idx + k, (size_t)k * sizeof(int64_t), cudaMemcpyDeviceToHost), "top-k readback");
+    }
+    return rc;
 }
 
 int distsim_testing_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_cells_32bit)
@@ -658,6 +703,27 @@ int64_t distsim_testing_lockstep_pieces(int32_t pp, int64_t lo, int64_t hi, int6
         (max_pieces > 0 && (!h_lo || !h_hi || !h_blocks)))
         return DISTSIM_E_ARG;
     return lockstep_pieces(pp, lo, hi, max_blocks, max_pieces, h_lo, h_hi, h_blocks);
+}
+
+int distsim_testing_time_phases(distsim_ctx *ctx, int32_t enable)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (int rc = set_device(ctx)) return rc;
+    if (enable && !ctx->phase_ev[0])
+        for (cudaEvent_t &e : ctx->phase_ev) CU(cudaEventCreate(&e), "event create");
+    ctx->phase_timing = enable != 0;
+    ctx->phase_valid = false;
+    return DISTSIM_OK;
+}
+
+int distsim_testing_last_phase_ms(distsim_ctx *ctx, float *h_eval_ms, float *h_select_ms)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!h_eval_ms || !h_select_ms) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (!ctx->phase_valid) return fail(ctx, DISTSIM_E_STATE, "no timed distsim_eval_select call yet");
+    CU(cudaEventElapsedTime(h_eval_ms, ctx->phase_ev[0], ctx->phase_ev[1]), "event time");
+    CU(cudaEventElapsedTime(h_select_ms, ctx->phase_ev[1], ctx->phase_ev[2]), "event time");
+    return DISTSIM_OK;
 }
 
 int distsim_testing_set_stage_wait_polls(distsim_ctx *ctx, int32_t polls)

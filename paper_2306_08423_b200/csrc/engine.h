@@ -180,12 +180,22 @@ struct SideStream {
     cudaStream_t side[1] = {nullptr};
     cudaEvent_t fork = nullptr, join[1] = {nullptr};
 };
+// Selection folded into an evaluation (enabled != 0): every result also enters a running
+// minimum of the packed key (time << idx_bits | position in the output) and the histogram of
+// the first radix-select digit (time >> shift) & (2^width - 1), so that neither the best
+// candidate nor the first pass of the k fastest needs to read the results again.
+constexpr int kSelectBins = 2048;                 // bins of a radix-select digit (11 bits)
+struct FusedSelect {
+    unsigned long long *key;                      // packed minimum (all ones: none yet)
+    unsigned long long *hist;                     // [kSelectBins]
+    int32_t idx_bits, shift, width, enabled;
+};
 // Evaluates candidates [first, first + count); rows / entries: host copies.  Results go to
 // batch_out[index - first] and, if non-null, busy_out[(index - first) * pp_max + d].  All work
 // is ordered after what `s` held before the call and before what is enqueued on `s` after it.
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
-                 int64_t *launches);
+                 const FusedSelect &fs, int64_t *launches);
 // Cuts candidates [lo, hi) of a row of pp stages into pieces of at most max_blocks lock-step
 // blocks each; returns the number of pieces and writes the first max_pieces of them.
 int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
@@ -203,6 +213,19 @@ struct SelectScratch {
 // d_result[0] = smallest time, d_result[1] = its smallest position in `batch`.
 void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t time_bound,
                    const SelectScratch &sc, int64_t *d_result, int64_t *launches);
+// Selection folded into an evaluation of `count` results whose times are below time_bound:
+// clears the key and the histogram, initialises the radix select for rank k and returns what the
+// evaluation kernels need (enabled = 0 when time and position do not fit one 64-bit key, or
+// the array is small enough to be sorted directly).
+FusedSelect begin_fused_select(cudaStream_t s, int64_t count, int k, int64_t time_bound, const SelectScratch &sc,
+                               int64_t *launches);
+// After the evaluation: d_result[0] = smallest time, d_result[1] = its smallest position.
+void finish_fused_argmin(cudaStream_t s, const FusedSelect &fs, const SelectScratch &sc, int64_t *d_result,
+                         int64_t *launches);
+// After the evaluation: the k fastest, continuing from the histogram the evaluation filled.
+void finish_fused_topk(cudaStream_t s, const FusedSelect &fs, const int64_t *batch, int64_t first, int64_t count, int k,
+                       int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
+                       int64_t *launches);
 // time_bound: an upper bound on every element of `batch` (INT64_MAX if unknown).
 void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
                  int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,

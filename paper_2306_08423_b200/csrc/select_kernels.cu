@@ -105,42 +105,13 @@ __device__ __forceinline__ SelSource sel_source(const SelState *st, const int64_
     return SelSource{batch, nullptr, count};
 }
 
+// Run by one whole block once a digit's histogram is complete: picks the bin that holds the
+// wanted rank, narrows the prefix / mask to it and clears the histogram for the next digit.
 template <bool kIndexPhase>
-__global__ void __launch_bounds__(kSelThreads)
-radix_pass_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int shift, int width,
-                  bool last_time_pass)
+__device__ __forceinline__ void pick_bin(SelState *st, u64 *hist, u64 *partial /* shared, [kSelThreads] */, int shift,
+                                         unsigned dmask, bool last_time_pass)
 {
-    __shared__ unsigned int sh[kBins];
-    __shared__ u64 partial[kSelThreads];
-    __shared__ bool last;
-    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
-    u64 *hist = sc.hist;
-    // no ties at the threshold time: every element equal to it is wanted, no index pass needed
-    if (kIndexPhase && st->skip_index) return;
-    for (int i = threadIdx.x; i < kBins; i += blockDim.x) sh[i] = 0;
-    __syncthreads();
-    const SelSource src = sel_source(st, batch, count, sc);
     const u64 tprefix = st->tprefix, tmask = st->tmask, iprefix = st->iprefix, imask = st->imask;
-    const unsigned dmask = (1u << width) - 1u;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < src.n; i += (int64_t)gridDim.x * blockDim.x) {
-        const u64 x = (u64)src.t[i];
-        if ((x & tmask) != tprefix) continue;
-        if (kIndexPhase) {
-            const u64 id = src.idx ? (u64)src.idx[i] : (u64)i;
-            if ((id & imask) != iprefix) continue;
-            atomicAdd(&sh[(unsigned)(id >> shift) & dmask], 1u);
-        } else {
-            atomicAdd(&sh[(unsigned)(x >> shift) & dmask], 1u);
-        }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < kBins; i += blockDim.x) if (sh[i]) atomicAdd(&hist[i], (u64)sh[i]);
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) last = atomicAdd(&st->blocks_done, 1ull) == (u64)gridDim.x - 1;
-    __syncthreads();
-    if (!last) return;
-    // the last block to finish picks the bin that holds the wanted rank
     __threadfence();
     constexpr int kPer = kBins / kSelThreads;
     u64 mine = 0;
@@ -176,10 +147,56 @@ radix_pass_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratc
     for (int i = threadIdx.x; i < kBins; i += blockDim.x) hist[i] = 0;
 }
 
+template <bool kIndexPhase>
+__global__ void __launch_bounds__(kSelThreads)
+radix_pass_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int shift, int width,
+                  bool last_time_pass)
+{
+    __shared__ unsigned int sh[kBins];
+    __shared__ u64 partial[kSelThreads];
+    __shared__ bool last;
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    u64 *hist = sc.hist;
+    // no ties at the threshold time: every element equal to it is wanted, no index pass needed
+    if (kIndexPhase && st->skip_index) return;
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) sh[i] = 0;
+    __syncthreads();
+    const SelSource src = sel_source(st, batch, count, sc);
+    const u64 tprefix = st->tprefix, tmask = st->tmask, iprefix = st->iprefix, imask = st->imask;
+    const unsigned dmask = (1u << width) - 1u;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < src.n; i += (int64_t)gridDim.x * blockDim.x) {
+        const u64 x = (u64)src.t[i];
+        if ((x & tmask) != tprefix) continue;
+        if (kIndexPhase) {
+            const u64 id = src.idx ? (u64)src.idx[i] : (u64)i;
+            if ((id & imask) != iprefix) continue;
+            atomicAdd(&sh[(unsigned)(id >> shift) & dmask], 1u);
+        } else {
+            atomicAdd(&sh[(unsigned)(x >> shift) & dmask], 1u);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) if (sh[i]) atomicAdd(&hist[i], (u64)sh[i]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&st->blocks_done, 1ull) == (u64)gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    pick_bin<kIndexPhase>(st, hist, partial, shift, dmask, last_time_pass);
+}
+
 __global__ void sel_init_kernel(SelState *st, u64 *hist, int k)
 {
     for (int i = threadIdx.x; i < kBins; i += blockDim.x) hist[i] = 0;
     if (threadIdx.x == 0) { SelState z{}; z.rank = (u64)(k - 1); *st = z; }
+}
+
+// The pick step alone, for a first digit whose histogram an evaluation has filled.
+__global__ void __launch_bounds__(kSelThreads)
+radix_pick_kernel(SelectScratch sc, int shift, int width, bool last_time_pass)
+{
+    __shared__ u64 partial[kSelThreads];
+    pick_bin<false>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, partial, shift, (1u << width) - 1u, last_time_pass);
 }
 
 // After the first time pass: copies the elements whose time does not exceed the chosen top
@@ -296,27 +313,34 @@ void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t 
     ++*launches;
 }
 
-void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
-                 int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
-                 int64_t *launches)
+namespace {
+
+// Bits of the times that the radix select looks at, and its first digit.
+struct TimeDigits { int tb, shift0, width0; };
+TimeDigits time_digits(int64_t time_bound)
+{
+    TimeDigits d;
+    // bits above the bound on any time are zero everywhere: start below them
+    d.tb = bits_for(time_bound) > 0 ? bits_for(time_bound) : 1;
+    d.shift0 = ((d.tb + kRadixBits - 1) / kRadixBits - 1) * kRadixBits;
+    d.width0 = d.tb - d.shift0 < kRadixBits ? d.tb - d.shift0 : kRadixBits;
+    return d;
+}
+
+// The radix select for more than kSortMax elements.  first_digit_done: the histogram of the first
+// digit has been filled already (by an evaluation), only its bin is still to be picked.
+void select_passes(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k, int64_t time_bound,
+                   const SelectScratch &sc, bool first_digit_done, int64_t *d_indices, int64_t *d_times,
+                   int64_t *launches)
 {
     const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
-    ensure_dynamic_smem(reinterpret_cast<const void *>(&sort_pairs_kernel), sort_smem);     // per device
-    if (count <= kSortMax) {
-        sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(batch, nullptr, (int)count, k, first, d_indices, d_times);
-        ++*launches;
-        return;
-    }
-    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
-    sel_init_kernel<<<1, 256, 0, s>>>(st, sc.hist, k);
-    ++*launches;
     const int g = grid_for(count);
-    // bits above the bound on any time are zero everywhere: start below them
-    const int tb = bits_for(time_bound) > 0 ? bits_for(time_bound) : 1;
+    const TimeDigits td = time_digits(time_bound);
     bool first_pass = true;
-    for (int shift = ((tb + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
-        const int width = tb - shift < kRadixBits ? tb - shift : kRadixBits;
-        radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, sc, shift, width, shift == 0);
+    for (int shift = td.shift0; shift >= 0; shift -= kRadixBits) {
+        const int width = td.tb - shift < kRadixBits ? td.tb - shift : kRadixBits;
+        if (first_pass && first_digit_done) radix_pick_kernel<<<1, kSelThreads, 0, s>>>(sc, shift, width, shift == 0);
+        else radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, sc, shift, width, shift == 0);
         ++*launches;
         if (first_pass && shift > 0 && sc.comp_cap > 0) {
             compact_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc, shift);
@@ -333,6 +357,60 @@ void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t co
     collect_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc, k);
     sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, k, k, first, d_indices, d_times);
     *launches += 2;
+}
+
+}  // namespace
+
+void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
+                 int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
+                 int64_t *launches)
+{
+    const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
+    ensure_dynamic_smem(reinterpret_cast<const void *>(&sort_pairs_kernel), sort_smem);     // per device
+    if (count <= kSortMax) {
+        sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(batch, nullptr, (int)count, k, first, d_indices, d_times);
+        ++*launches;
+        return;
+    }
+    sel_init_kernel<<<1, 256, 0, s>>>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, k);
+    ++*launches;
+    select_passes(s, batch, first, count, k, time_bound, sc, false, d_indices, d_times, launches);
+}
+
+FusedSelect begin_fused_select(cudaStream_t s, int64_t count, int k, int64_t time_bound, const SelectScratch &sc,
+                               int64_t *launches)
+{
+    static_assert(kBins == kSelectBins, "the evaluation kernels fill the radix select's histogram");
+    FusedSelect fs{};
+    fs.key = sc.key; fs.hist = sc.hist;
+    fs.idx_bits = bits_for(count - 1) > 0 ? bits_for(count - 1) : 1;
+    const TimeDigits td = time_digits(time_bound);
+    fs.shift = td.shift0; fs.width = td.width0;
+    // folded in when time and position fit one key and the array is too long to be sorted directly
+    fs.enabled = (bits_for(time_bound) + fs.idx_bits <= 63 && count > kSortMax) ? 1 : 0;
+    if (fs.enabled) {
+        cudaMemsetAsync(sc.key, 0xFF, 2 * sizeof(u64), s);
+        sel_init_kernel<<<1, 256, 0, s>>>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, k > 0 ? k : 1);
+        ++*launches;
+    }
+    return fs;
+}
+
+void finish_fused_argmin(cudaStream_t s, const FusedSelect &fs, const SelectScratch &sc, int64_t *d_result,
+                         int64_t *launches)
+{
+    argmin_unpack_kernel<<<1, 32, 0, s>>>(sc.key, fs.idx_bits, 1, d_result);
+    ++*launches;
+}
+
+void finish_fused_topk(cudaStream_t s, const FusedSelect &fs, const int64_t *batch, int64_t first, int64_t count, int k,
+                       int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
+                       int64_t *launches)
+{
+    (void)fs;
+    const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
+    ensure_dynamic_smem(reinterpret_cast<const void *>(&sort_pairs_kernel), sort_smem);     // per device
+    select_passes(s, batch, first, count, k, time_bound, sc, true, d_indices, d_times, launches);
 }
 
 }  // namespace distsim

@@ -22,12 +22,13 @@ OK, E_ARG, E_STATE, E_RANGE, E_CAPACITY, E_OVERFLOW, E_CUDA, E_TIMEOUT, E_UNSUPP
 
 EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error",
            "distsim_load_event_table", "distsim_set_space", "distsim_decode",
-           "distsim_eval_strategies", "distsim_argmin", "distsim_topk",
+           "distsim_eval_strategies", "distsim_eval_select", "distsim_argmin", "distsim_topk",
            "distsim_emit_timelines", "distsim_checksum_timelines", "distsim_search_host",
            "distsim_topk_static")
 # hooks of include/distsim_testing.h (test-suite and benchmark accounting; not the stable ABI)
 TESTING_EXPORTS = ("distsim_testing_set_stage_wait_polls", "distsim_testing_launch_count",
-                   "distsim_testing_space_cells", "distsim_testing_lockstep_pieces")
+                   "distsim_testing_space_cells", "distsim_testing_lockstep_pieces",
+                   "distsim_testing_time_phases", "distsim_testing_last_phase_ms")
 TOPK_STATIC_MAX_K = 1024
 
 if not os.path.exists(LIB_PATH):
@@ -79,10 +80,14 @@ _lib.distsim_testing_set_stage_wait_polls.argtypes = [C.c_void_p, C.c_int32]
 _lib.distsim_testing_lockstep_pieces.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
                                                  C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.distsim_testing_lockstep_pieces.restype = C.c_int64
+_lib.distsim_testing_time_phases.argtypes = [C.c_void_p, C.c_int32]
+_lib.distsim_testing_last_phase_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_float)]
 _lib.distsim_load_event_table.argtypes = [C.c_void_p, C.POINTER(_Table)]
 _lib.distsim_set_space.argtypes = [C.c_void_p, C.POINTER(_Space), C.POINTER(C.c_int64)]
 _lib.distsim_decode.argtypes = [C.c_void_p, C.c_int64, C.POINTER(_Candidate)]
 _lib.distsim_eval_strategies.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
+_lib.distsim_eval_select.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int32,
+                                     C.c_void_p, C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 _lib.distsim_argmin.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                 C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 _lib.distsim_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
@@ -214,6 +219,23 @@ def distsim_eval_strategies(ctx: Context, first: int, count: int, d_batch_ns,
     ctx._check(_lib.distsim_eval_strategies(ctx._h, _stream(stream), first, count, pb, ps))
 
 
+def distsim_eval_select(ctx: Context, first: int, count: int, d_batch_ns, k: int = 0, d_indices=None,
+                        d_times=None, stream=None):
+    """Evaluation with the best candidate and the k fastest folded in; returns (best index, best
+    batch time).  Synchronises."""
+    pb = _dev_ptr(d_batch_ns, "int64", count, "d_batch_ns")
+    pi = _dev_ptr(d_indices, "int64", k, "d_indices")
+    pt = _dev_ptr(d_times, "int64", k, "d_times")
+    bi, bt = C.c_int64(0), C.c_int64(0)
+    rc = _lib.distsim_eval_select(ctx._h, _stream(stream), first, count, pb, k, pi, pt, C.byref(bi), C.byref(bt))
+    if rc == E_TIMEOUT and b"outputs are exact" in _lib.distsim_last_error(ctx._h):
+        e = DistsimError(rc, _lib.distsim_last_error(ctx._h).decode())
+        e.result = (int(bi.value), int(bt.value))
+        raise e
+    ctx._check(rc)
+    return int(bi.value), int(bt.value)
+
+
 def distsim_argmin(ctx: Context, d_batch_ns, first: int, count: int, stream=None):
     pb = _dev_ptr(d_batch_ns, "int64", count, "d_batch_ns")
     bi, bt = C.c_int64(0), C.c_int64(0)
@@ -325,6 +347,17 @@ def distsim_testing_lockstep_pieces(pp: int, lo: int, hi: int, max_blocks: int, 
         raise DistsimError(n, "bad arguments")
     k = min(n, max_pieces)
     return n, list(zip(a[:k].tolist(), b[:k].tolist(), c[:k].tolist()))
+
+
+def distsim_testing_time_phases(ctx: Context, enable: bool) -> None:
+    ctx._check(_lib.distsim_testing_time_phases(ctx._h, 1 if enable else 0))
+
+
+def distsim_testing_last_phase_ms(ctx: Context):
+    """(evaluation ms, selection ms) of the most recent timed distsim_eval_select call."""
+    a, b = C.c_float(0), C.c_float(0)
+    ctx._check(_lib.distsim_testing_last_phase_ms(ctx._h, C.byref(a), C.byref(b)))
+    return float(a.value), float(b.value)
 
 
 def distsim_testing_launch_count(ctx: Context) -> int:

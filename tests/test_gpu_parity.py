@@ -666,6 +666,58 @@ def test_small_windows_agree_with_the_full_evaluation(E, ctx, cfg):
         assert torch.equal(ob[:count * ctx.pp_max].view(count, -1), fb[first:first + count])
 
 
+def _check_eval_select(E, ctx, first, count, k):
+    want = dev(count)
+    E.distsim_eval_strategies(ctx, first, count, want)
+    wi, wt = dev(max(1, k)), dev(max(1, k))
+    if k:
+        E.distsim_topk(ctx, want, first, count, k, wi, wt)
+    best = E.distsim_argmin(ctx, want, first, count)
+    got = dev(count); got.fill_(-1)
+    gi, gt = dev(max(1, k)), dev(max(1, k))
+    assert E.distsim_eval_select(ctx, first, count, got, k, gi if k else None, gt if k else None) == best
+    torch.cuda.synchronize()
+    assert torch.equal(got, want)
+    if k:
+        assert torch.equal(gi, wi) and torch.equal(gt, wt)
+    return want
+
+
+def test_eval_select_matches_separate_calls(E, ctx):
+    """Evaluation with the best candidate and the k fastest folded into its kernels against the
+    separate calls, which the other tests compare with the oracle: thread kernel in 32- and 64-bit
+    arithmetic, lock-step kernel, sub-ranges, short arrays, ties, times too wide to pack."""
+    for cfg, k in ((1, 1024), (3, 1024), (2, 1024), (0, 10)):
+        w = W.CONFIGS[cfg]()
+        n = load(E, ctx, w)
+        _check_eval_select(E, ctx, 0, n, k)
+        _check_eval_select(E, ctx, 0, n, 0)
+        if n > 10_000:
+            rng = np.random.default_rng(cfg)
+            for _ in range(3):
+                first = int(rng.integers(0, n - 9000))
+                count = int(rng.integers(4097, min(n - first, 3_000_000)))
+                _check_eval_select(E, ctx, first, count, int(rng.integers(1, 4097)))
+            _check_eval_select(E, ctx, 12345, 4000, 77)                # short: sorted directly
+    # coarse times: many ties at the threshold, resolved by index
+    space = W.SearchSpace(mp_max=2, pp_max=8, m_list=[1, 2, 4, 8, 16], m_rule=W.M_RULE_CEIL,
+                          partition_mode=W.PARTITION_ALL)
+    table = _flat_table(16, 16, 4, 64, space, 3, 5)                    # layer times of 1 or 2 ns
+    table.grad_bytes[:] = 0
+    w = W.Workload("ties", table, space, 5)
+    n = load(E, ctx, w)
+    full = _check_eval_select(E, ctx, 0, n, 4096)
+    assert int((full == full.min()).sum()) > 1
+    ob, _ = oracle.eval_indices_parallel(table, space, np.arange(0, n, 97), THREADS)
+    assert (full[::97].cpu().numpy() == ob).all()
+    # times near 2^45: time and position do not fit one key, the calls fall back to separate passes
+    w = W.random_small(3, lo=2**44, hi=2**45, partition_mode=W.PARTITION_ALL, n_layers=16, pp_max=4,
+                       m_list=(1, 2, 4, 8))
+    n = load(E, ctx, w)
+    assert n > 4096
+    _check_eval_select(E, ctx, 0, n, 500)
+
+
 def test_two_pass_argmin_for_wide_times(E, ctx):
     # times near 2^55 with a large count cannot be packed with the index into 64 bits
     w = W.random_small(3, lo=2**44, hi=2**45, partition_mode=W.PARTITION_ALL, n_layers=12, pp_max=4,
