@@ -186,18 +186,21 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
                             int64_t *d_batch_ns, int64_t *d_stage_busy_ns);
 
 /*
- * Evaluation with the selection folded in (paper Sec. 6: the grid search keeps the fastest):
+ * Evaluation and selection in one call (paper Sec. 6: the grid search keeps the fastest):
  * evaluates candidates [first, first + count) like distsim_eval_strategies and returns the best
- * candidate and the k fastest like distsim_argmin and distsim_topk.  The evaluation kernels keep
- * the running minimum of (batch time, index) and the histogram of the selection's first digit
- * while they write the batch times, so the best candidate costs no further pass over the array
- * and the k fastest one pass less.
+ * candidate and the k fastest like distsim_argmin and distsim_topk.  For a long range the
+ * selection reads the batch times little more than once: a strided sample of them gives a time
+ * that at least k candidates do not exceed, one pass then finds the best candidate and gathers
+ * the candidates up to that time, and the k fastest are selected among those few.
  *   d_batch_ns [count] out;  k in [0, min(count, 4096)], 0: no top-k;
  *   d_indices [k] out, d_times [k] out (nullable): ascending by (batch time, index);
- *   h_best_index, h_best_batch_ns: host out.  Synchronises `stream`.
+ *   d_best [2] out, nullable (device): batch time and index of the best candidate;
+ *   h_best_index, h_best_batch_ns: host out, both or neither.  With host outputs the call
+ *   synchronises `stream`; without them it is asynchronous, and a stalled table copy
+ *   (DISTSIM_E_TIMEOUT, see above) is reported by the next synchronising call instead.
  */
 int distsim_eval_select(distsim_ctx *ctx, void *stream, int64_t first, int64_t count, int64_t *d_batch_ns,
-                        int32_t k, int64_t *d_indices, int64_t *d_times, int64_t *h_best_index,
+                        int32_t k, int64_t *d_indices, int64_t *d_times, int64_t *d_best, int64_t *h_best_index,
                         int64_t *h_best_batch_ns);
 
 /*

@@ -76,7 +76,7 @@ struct distsim_ctx {
     bool have_dt = false, have_narrow = false;
 
     // scratch
-    DevBuf d_status, d_sel, d_result, d_plans, d_op_start, d_totals, d_batch, d_topk;
+    DevBuf d_status, d_sel, d_result, d_plans, d_plan_sums, d_op_start, d_totals, d_batch, d_topk;
     SideStream side;                      // extra streams of an evaluation (lock-step launches)
     int64_t *h_pinned = nullptr;          // 16 words of pinned host memory for small results:
                                           // [0..3] results, [4] status, [8..15] emission totals
@@ -524,18 +524,18 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const DeviceView v = ctx->view();
     launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
-                d_batch_ns, d_stage_busy_ns, FusedSelect{}, &ctx->launches);
+                d_batch_ns, d_stage_busy_ns, &ctx->launches);
     CU(cudaGetLastError(), "evaluation launch");
     return DISTSIM_OK;
 }
 
 int distsim_eval_select(distsim_ctx *ctx, void *stream, int64_t first, int64_t count, int64_t *d_batch_ns,
-                        int32_t k, int64_t *d_indices, int64_t *d_times, int64_t *h_best_index,
+                        int32_t k, int64_t *d_indices, int64_t *d_times, int64_t *d_best, int64_t *h_best_index,
                         int64_t *h_best_batch_ns)
 {
     if (!ctx) return DISTSIM_E_ARG;
     if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
-    if (!d_batch_ns || !h_best_index || !h_best_batch_ns) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (!d_batch_ns || (!h_best_index != !h_best_batch_ns)) return fail(ctx, DISTSIM_E_ARG, "null argument");
     if (first < 0 || count < 1 || first > ctx->sc.n_candidates || count > ctx->sc.n_candidates - first)
         return fail(ctx, DISTSIM_E_RANGE, "candidate range outside the space");
     if (k < 0 || k > 4096 || k > count || (k > 0 && !d_indices))
@@ -544,21 +544,22 @@ int distsim_eval_select(distsim_ctx *ctx, void *stream, int64_t first, int64_t c
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const DeviceView v = ctx->view();
     const SelectScratch sc = ctx->select_scratch();
-    const FusedSelect fs = begin_fused_select(s, count, k, ctx->time_bound, sc, &ctx->launches);
     if (ctx->phase_timing) cudaEventRecord(ctx->phase_ev[0], s);
     launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
-                d_batch_ns, nullptr, fs, &ctx->launches);
+                d_batch_ns, nullptr, &ctx->launches);
     CU(cudaGetLastError(), "evaluation launch");
     if (ctx->phase_timing) cudaEventRecord(ctx->phase_ev[1], s);
-    if (fs.enabled) {
-        finish_fused_argmin(s, fs, sc, ctx->d_result.as<int64_t>(), &ctx->launches);
-        if (k > 0) finish_fused_topk(s, fs, d_batch_ns, first, count, k, ctx->time_bound, sc, d_indices, d_times, &ctx->launches);
-    } else {
-        launch_argmin(s, d_batch_ns, count, ctx->time_bound, sc, ctx->d_result.as<int64_t>(), &ctx->launches);
-        if (k > 0) launch_topk(s, d_batch_ns, first, count, k, ctx->time_bound, sc, d_indices, d_times, &ctx->launches);
-    }
+    const bool want_best = d_best || h_best_index;
+    launch_select(s, d_batch_ns, first, count, k, ctx->time_bound, sc, want_best ? ctx->d_result.as<int64_t>() : nullptr,
+                  d_indices, d_times, &ctx->launches);
     CU(cudaGetLastError(), "selection launch");
+    if (d_best) {
+        // (batch time, position) -> (batch time, candidate index)
+        CU(cudaMemcpyAsync(d_best, ctx->d_result.p, 2 * sizeof(int64_t), cudaMemcpyDeviceToDevice, s), "best copy");
+        launch_add_scalar(s, d_best + 1, first, &ctx->launches);
+    }
     if (ctx->phase_timing) { cudaEventRecord(ctx->phase_ev[2], s); ctx->phase_valid = true; }
+    if (!h_best_index) return DISTSIM_OK;              // nothing goes to the host: no synchronisation
     CU(cudaMemcpyAsync(ctx->h_pinned, ctx->d_result.p, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, s), "argmin readback");
     bool stalled = false;
     if (int rc = read_status(ctx, s, &stalled)) return rc;          // synchronises
@@ -614,9 +615,10 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     CU(ctx->d_plans.reserve((size_t)n * sizeof(EmitPlan)), "alloc emission plans");
     CU(ctx->d_op_start.reserve((size_t)n * ctx->op_words_per_cand * sizeof(int64_t)), "alloc item start times");
+    CU(ctx->d_plan_sums.reserve((size_t)n * kEmitSumWords * sizeof(int64_t)), "alloc plan summaries");
     const DeviceView v = ctx->view();
     launch_emit_plan(s, v, d_indices, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
-                     ctx->op_words_per_cand, d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), &ctx->launches);
+                     ctx->op_words_per_cand, ctx->d_plan_sums.as<int64_t>(), d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), &ctx->launches);
     CU(cudaGetLastError(), "emission planning launch");
     static_assert(sizeof(EmitTotals) == 8 * sizeof(int64_t), "totals occupy the second half of the pinned words");
     const EmitTotals *totals = reinterpret_cast<const EmitTotals *>(ctx->h_pinned + 8);
@@ -666,7 +668,7 @@ int distsim_search_host(distsim_ctx *ctx, const distsim_event_table *h_table, co
         CU(ctx->d_topk.reserve((size_t)2 * k * sizeof(int64_t)), "alloc top-k");
         d_idx = ctx->d_topk.as<int64_t>();
     }
-    const int rc = distsim_eval_select(ctx, nullptr, 0, n, d_batch, k, d_idx, d_idx ? d_idx + k : nullptr,
+    const int rc = distsim_eval_select(ctx, nullptr, 0, n, d_batch, k, d_idx, d_idx ? d_idx + k : nullptr, nullptr,
                                        h_best_index, h_best_batch_ns);          // synchronises
     if (rc != DISTSIM_OK && rc != DISTSIM_E_TIMEOUT) return rc;
     if (k > 0) {

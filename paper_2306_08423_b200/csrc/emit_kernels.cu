@@ -2,8 +2,8 @@
 // selected candidates, plus per-device activity time and utilisation.
 //
 //   emit_plan_kernel     one warp per selected candidate: decode it, run the lock-step recurrence
-//                        while recording every item's start time into scratch, count records.
-//   emit_scan_kernel     one block: exclusive scan of the per-candidate record totals.
+//                        while recording every item's start time into scratch, count records; the
+//                        last block to finish scans the per-candidate record totals.
 //   emit_devices_kernel  per (candidate, device): record offset, activity time, utilisation.
 //   emit_items_kernel    the bandwidth-bound part.  A block owns (candidate, stage, run of
 //                        consecutive items, chunk of replicas).  It builds the stage's forward
@@ -13,7 +13,8 @@
 //                        mp*dp replicas hold identical lists, so the image is computed once and
 //                        written to each replica of the chunk by one bulk asynchronous copy
 //                        (cp.async.bulk shared -> global) issued by one lane per replica.
-//   emit_buckets_kernel  gradient-bucket records of every stage.
+//                        The blocks of the same launch beyond the item tiles write the
+//                        gradient-bucket records of every stage (emit_buckets_block).
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
 
@@ -27,7 +28,6 @@ constexpr int kTileWords = 3872;    // largest capacity of a block's image of it
 constexpr int kRunWords = 3872;     // run length the plans aim at (three blocks per SM; shorter runs
                                     // measured slower: the per-block set-up weighs more)
 constexpr int kTileReplicas = 16;   // replicas per block
-constexpr int kBucketThreads = 128;
 constexpr int kBucketRun = 768;     // gradient buckets per shared-memory image (5 words each)
 constexpr int kBucketReplicas = 32; // replicas per block of the bucket kernel: one lane of the first warp each
 // the longest item: every layer with computation, all-reduce and all-to-all, a jitter event, a transfer
@@ -43,9 +43,14 @@ __device__ __forceinline__ int find_row(const DeviceView &v, int64_t index)
     return lo;
 }
 
+// Words of a selection's summary: what the scan over all selections needs of its plan.
+enum { kSumRecords = 0, kSumItemTiles, kSumBucketTiles, kSumTmplWords, kSumBucketRecs, kSumRunWords, kSumWords = 8 };
+static_assert(kSumWords == kEmitSumWords, "the context sizes the summaries");
+
 template <int S>
 __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &row, int row_index,
-                                               int64_t index, EmitPlan *plan, int64_t *rec)
+                                               int64_t index, EmitPlan *plan, int64_t *rec, const int64_t *binom,
+                                               int64_t *sum /* the selection's words of the summary the scan reads */)
 {
     const int lane = threadIdx.x & 31;
     const int wl = row.pp / S;
@@ -58,9 +63,14 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
     const int n_slots = 2 * (en.m + row.pp - 1);
     const StageResult<S> R = v.tc.n_jitter > 0
         ? lockstep_candidate<S, true, true>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank, seg_lane, wl,
-                                            n_slots, owner ? rec : nullptr)
+                                            n_slots, owner ? rec : nullptr, binom)
         : lockstep_candidate<S, true, false>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank, seg_lane, wl,
-                                             n_slots, owner ? rec : nullptr);
+                                             n_slots, owner ? rec : nullptr, binom);
+    // per stage: records of a forward / backward item, gradient buckets, records of one device;
+    // their prefix over the stages and the widest item by shuffles over the lanes that own stages
+    int64_t recs[S];
+    int widest = 1, both = 2;
+    int64_t lane_recs = 0;
     if (owner) {
         const int L1 = v.tc.n_layers + 1;
 #pragma unroll
@@ -78,32 +88,49 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
                 const int64_t *nbt = v.nb + row.row_tab_off, *tpt = v.tp + row.row_tab_off;
                 kb = nbt[(int64_t)e * L1 + a] + (tpt[(int64_t)e * L1 + a] > 0 ? 1 : 0);
             }
+            recs[k] = (int64_t)en.m * (rf + rb) + kb;
+            lane_recs += recs[k];
+            widest = max(widest, (int)max(rf, rb));
+            both = max(both, (int)(rf + rb));
             plan->bounds[d] = a;
             if (d == row.pp - 1) plan->bounds[row.pp] = e;
             plan->rf[d] = (int32_t)rf; plan->rb[d] = (int32_t)rb;
             plan->n_buckets[d] = kb;
-            plan->stage_recs[d] = (int64_t)en.m * (rf + rb) + kb;
+            plan->stage_recs[d] = recs[k];
             plan->busy[d] = R.busy[k];
             plan->main_end[d] = R.main_end[k];
             plan->last_b_start[d] = R.last_b_start[k];
         }
-        if (lane == 0) {
-            plan->index = index; plan->batch_ns = R.batch;
-            plan->row = row_index; plan->entry = cc.entry; plan->m = en.m; plan->sched = cc.sched;
-            plan->pp = row.pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1;
-        }
     }
-    __syncwarp();
+    int64_t incl = lane_recs;                      // lanes that own no stage contribute nothing
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int64_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    const int64_t total = __shfl_sync(0xffffffffu, incl, 31);
+    int64_t most_buckets = 0;
+    if (owner) {
+#pragma unroll
+        for (int k = 0; k < S; ++k) most_buckets = max64(most_buckets, recs[k] - (int64_t)en.m * (plan->rf[seg_lane * S + k] + plan->rb[seg_lane * S + k]));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        widest = max(widest, __shfl_xor_sync(0xffffffffu, widest, o));
+        both = max(both, __shfl_xor_sync(0xffffffffu, both, o));
+        most_buckets = max64(most_buckets, __shfl_xor_sync(0xffffffffu, most_buckets, o));
+    }
+    if (owner) {
+        int64_t acc = incl - lane_recs;
+#pragma unroll
+        for (int k = 0; k < S; ++k) { plan->stage_rec_prefix[seg_lane * S + k] = acc; acc += recs[k]; }
+    }
     if (lane == 0) {
-        int64_t acc = 0;
-        for (int d = 0; d < row.pp; ++d) { plan->stage_rec_prefix[d] = acc; acc += plan->stage_recs[d]; }
-        plan->stage_rec_prefix[row.pp] = acc;
-        plan->rec_total = acc * row.mp * row.dp;
-        int widest = 1, both = 2;
-        for (int d = 0; d < row.pp; ++d) {
-            widest = max(widest, max(plan->rf[d], plan->rb[d]));
-            both = max(both, plan->rf[d] + plan->rb[d]);
-        }
+        plan->index = index; plan->batch_ns = R.batch;
+        plan->row = row_index; plan->entry = cc.entry; plan->m = en.m; plan->sched = cc.sched;
+        plan->pp = row.pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1;
+        plan->stage_rec_prefix[row.pp] = total;
+        plan->rec_total = total * row.mp * row.dp;
         // a run of tile_items items of any mix must fit the image of kTileWords words
         // a run aims at kRunWords words (small images: more blocks per SM), holds at least one item
         const int cap = max(1, min(kMaxTileItems, kRunWords / (widest * 5)));
@@ -111,41 +138,31 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
         plan->tile_items = (2 * en.m + n_chunks - 1) / n_chunks;
         plan->run_words = plan->tile_items * widest * 5;          // no run of this selection is longer
         plan->tmpl_words = both * 5;
+        const int64_t reps = (int64_t)row.mp * row.dp;
+        sum[kSumRecords] = plan->rec_total;
+        sum[kSumItemTiles] = (int64_t)row.pp * ((2 * en.m + plan->tile_items - 1) / plan->tile_items) *
+                             ((reps + kTileReplicas - 1) / kTileReplicas);
+        sum[kSumBucketTiles] = (int64_t)row.pp * ((reps + kBucketReplicas - 1) / kBucketReplicas);
+        sum[kSumTmplWords] = plan->tmpl_words;
+        sum[kSumBucketRecs] = most_buckets;
+        sum[kSumRunWords] = plan->run_words;
     }
 }
 
-__global__ void __launch_bounds__(128)
-emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitPlan *plans,
-                 int64_t *op_start, int64_t op_words_per_cand)
-{
-    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (i >= n) return;
-    EmitPlan *plan = plans + i;
-    const int64_t index = indices[i];
-    if (index < 0 || index >= v.sc.n_candidates) {
-        if ((threadIdx.x & 31) == 0) {
-            plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
-            plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
-            atomicCAS(v.status, 0, DISTSIM_E_RANGE);
-        }
-        return;
-    }
-    const int r = find_row(v, index);
-    const Row row = v.rows[r];
-    int64_t *rec = op_start + (int64_t)i * op_words_per_cand;
-    if (row.pp > 32) plan_candidate<2>(v, row, r, index, plan, rec);
-    else plan_candidate<1>(v, row, r, index, plan, rec);
-}
-
-// Exclusive scan of rec_total over the selections (n is small: one block, serial per chunk).
-__global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /* the words of EmitTotals */)
+// Totals over all selections and the exclusive scan of their record counts, by one block, from
+// the selections' summaries.
+__device__ __forceinline__ void scan_plans(EmitPlan *plans, const int64_t *sums, int n, int64_t *totals /* the words of EmitTotals */)
 {
     __shared__ int64_t warp_sum[32];
     const int t = threadIdx.x, nt = blockDim.x, lane = t & 31, warp = t >> 5;
     const int per = (n + nt - 1) / nt;
     const int b = min(n, t * per), e = min(n, b + per);
-    int64_t s = 0, mt = 0, mb = 0, mw = 0, mk = 0, mr = 0;
-    for (int i = b; i < e; ++i) s += plans[i].rec_total;
+    int64_t s = 0, mx[kSumWords] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int i = b; i < e; ++i) {
+        s += __ldcg(&sums[(int64_t)i * kSumWords + kSumRecords]);
+#pragma unroll
+        for (int w = kSumItemTiles; w <= kSumRunWords; ++w) mx[w] = max64(mx[w], __ldcg(&sums[(int64_t)i * kSumWords + w]));
+    }
     // exclusive scan of the per-thread sums over the block: inside warps, then over the warp totals
     int64_t incl = s;
     for (int off = 1; off < 32; off <<= 1) {
@@ -166,24 +183,49 @@ __global__ void emit_scan_kernel(EmitPlan *plans, int n, int64_t *totals /* the 
     }
     __syncthreads();
     int64_t acc = warp_sum[warp] + incl - s;
-    for (int i = b; i < e; ++i) {
-        plans[i].rec_base = acc; acc += plans[i].rec_total;
-        if (plans[i].ok) {
-            const int64_t reps = (int64_t)plans[i].mp * plans[i].dp;
-            const int64_t tiles = (int64_t)plans[i].pp * ((2 * plans[i].m + plans[i].tile_items - 1) / plans[i].tile_items) *
-                                  ((reps + kTileReplicas - 1) / kTileReplicas);
-            mt = max64(mt, tiles);
-            mw = max64(mw, plans[i].tmpl_words);
-            mr = max64(mr, plans[i].run_words);
-            mb = max64(mb, (int64_t)plans[i].pp * ((reps + kBucketReplicas - 1) / kBucketReplicas));
-            for (int d = 0; d < plans[i].pp; ++d) mk = max64(mk, plans[i].n_buckets[d]);
+    for (int i = b; i < e; ++i) { plans[i].rec_base = acc; acc += __ldcg(&sums[(int64_t)i * kSumWords + kSumRecords]); }
+    // totals[1..5]: item tiles, bucket tiles, template words, bucket records, run words (the order of the summary)
+#pragma unroll
+    for (int w = kSumItemTiles; w <= kSumRunWords; ++w)
+        if (mx[w] > 0) atomicMax((unsigned long long *)&totals[w], (unsigned long long)mx[w]);
+}
+
+// One warp per selection plans it; the last block to finish then scans the plans (totals[6]
+// counts the finished blocks; the totals are cleared before the launch).
+constexpr int kPlanBinomWords = 512;
+__global__ void __launch_bounds__(128)
+emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitPlan *plans,
+                 int64_t *op_start, int64_t op_words_per_cand, int64_t *sums, int64_t *totals)
+{
+    __shared__ int64_t binom_s[kPlanBinomWords];
+    __shared__ bool last;
+    const int64_t *binom = stage_binom(v, binom_s, kPlanBinomWords);
+    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (i < n) {
+        EmitPlan *plan = plans + i;
+        const int64_t index = indices[i];
+        if (index < 0 || index >= v.sc.n_candidates) {
+            if ((threadIdx.x & 31) == 0) {
+                plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
+                plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
+                for (int w = 0; w < kSumWords; ++w) sums[(int64_t)i * kSumWords + w] = 0;
+                atomicCAS(v.status, 0, DISTSIM_E_RANGE);
+            }
+        } else {
+            const int r = find_row(v, index);
+            const Row row = v.rows[r];
+            int64_t *rec = op_start + (int64_t)i * op_words_per_cand;
+            if (row.pp > 32) plan_candidate<2>(v, row, r, index, plan, rec, binom, sums + (int64_t)i * kSumWords);
+            else plan_candidate<1>(v, row, r, index, plan, rec, binom, sums + (int64_t)i * kSumWords);
         }
     }
-    if (mt > 0) atomicMax((unsigned long long *)&totals[1], (unsigned long long)mt);
-    if (mb > 0) atomicMax((unsigned long long *)&totals[2], (unsigned long long)mb);
-    if (mw > 0) atomicMax((unsigned long long *)&totals[3], (unsigned long long)mw);
-    if (mk > 0) atomicMax((unsigned long long *)&totals[4], (unsigned long long)mk);
-    if (mr > 0) atomicMax((unsigned long long *)&totals[5], (unsigned long long)mr);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd((unsigned long long *)&totals[6], 1ull) == (unsigned long long)gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    scan_plans(plans, sums, n, totals);
 }
 
 __global__ void __launch_bounds__(256)
@@ -228,12 +270,123 @@ __device__ __forceinline__ void item_at(int sched, int pp, int m, int d, int s, 
     } else { bwd = true; j = s - m; nf = m; nb = s - m; }
 }
 
+// Gradient-bucket records.  A block owns (selection, stage, chunk of replicas).  Buckets whose last byte lies in the same layer share a ready time, so once the
+// first of them has started the rest follow back to back: per layer one serial step (lane 0),
+// inside a layer a closed form (a thread per bucket).  The records of up to `run` buckets
+// are assembled in shared memory once and sent to every replica by a bulk copy, as in
+// emit_items_kernel.
+// The blocks of the record kernel beyond its item tiles run this (tile: the block's number among them).
+__device__ __forceinline__ void emit_buckets_block(const DeviceView &v, const EmitPlan &p, int tile,
+                                                   int64_t *__restrict__ out, int run /* buckets per image */,
+                                                   int64_t *dyn_s)
+{
+    int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
+    int64_t *img_b = dyn_s + run * 5 + 1;               // the same word at img_b[x + 1] (run * 5 + 1 is even)
+    int64_t *g_start = img_b + run * 5 + 1;             // [L + 1] start of the first bucket ending in layer a+i
+    int64_t *g_first = g_start + DISTSIM_MAX_LAYERS + 1;  // [L + 1] number of that bucket
+    __shared__ int64_t part_start_s;
+    if (!p.ok || p.dp == 1) return;
+    const int mp = p.mp, reps = mp * p.dp;
+    const int rep_chunks = (reps + kBucketReplicas - 1) / kBucketReplicas;
+    const int d = tile / rep_chunks, rc = tile - d * rep_chunks;
+    if (d >= p.pp) return;
+    const int64_t kb = p.n_buckets[d];
+    if (kb == 0) return;
+    const Row &row = v.rows[p.row];
+    const int a = p.bounds[d], e = p.bounds[d + 1];
+    const int L1 = v.tc.n_layers + 1;
+    const int64_t *nbe = v.nb + row.row_tab_off + (int64_t)e * L1;
+    const int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
+    const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
+    const int64_t n_full = nbe[a], t_full = row.t_full;
+    const int64_t tbs = p.last_b_start[d], main_end = p.main_end[d];
+    // all threads fetch the per-layer inputs (independent loads), then thread 0 runs the short chain
+    for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
+        g_first[l - a] = l + 1 < e ? nbe[l + 1] : 0;                       // buckets before layer l's group
+        g_start[l - a] = v.tc.overlap ? tbs + (pb[e] - pb[l]) : main_end;    // ready time of the group
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t end = 0, part_start = 0;
+        for (int l = e - 1; l >= a; --l) {
+            const int64_t nb_prev = g_first[l - a];
+            const int64_t nb_l = l > a ? g_first[l - 1 - a] : n_full;       // nb[e][l]
+            const int64_t start = max64(end, g_start[l - a]);
+            g_start[l - a] = start;
+            if (nb_l > nb_prev) end = start + (nb_l - nb_prev) * t_full;
+        }
+        if (part > 0) {
+            const int ls = v.next_grad[a];
+            const int64_t ready = v.tc.overlap ? tbs + (pb[e] - pb[ls]) : main_end;
+            part_start = max64(end, ready);
+        }
+        part_start_s = part_start;
+    }
+    __syncthreads();
+    const int64_t part_start = part_start_s;
+    const int64_t stage_words = p.stage_recs[d] * 5;
+    const int64_t replica_words = (int64_t)mp * p.stage_rec_prefix[p.pp] * 5;
+    int64_t *base = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + (int64_t)p.m * (p.rf[d] + p.rb[d]) * 5;
+    for (int64_t k0 = 0; k0 < kb; k0 += run) {
+        const int nk = (int)min((int64_t)run, kb - k0);
+        for (int kk = threadIdx.x; kk < nk; kk += blockDim.x) {
+            const int64_t k = k0 + kk;
+            int64_t start, dur;
+            if (k >= n_full) { start = part_start; dur = part; }
+            else {
+                // the layer whose group holds bucket k: the largest l with nb[e][l] > k
+                // (nb[e][l] = g_first[l-1-a] for l > a grows as l decreases, and nb[e][a] = n_full > k)
+                int lo = a, hi = e - 1;
+                while (lo < hi) {
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (g_first[mid - 1 - a] > k) lo = mid; else hi = mid - 1;
+                }
+                start = g_start[lo - a] + (k - g_first[lo - a]) * t_full;
+                dur = t_full;
+            }
+            const int64_t rec[5] = {DISTSIM_DP_AR, k, -1, start, start + dur};
+#pragma unroll
+            for (int f = 0; f < 5; ++f) { img_a[kk * 5 + f] = rec[f]; img_b[kk * 5 + f + 1] = rec[f]; }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        const int total = nk * 5;
+        const int rep = rc * kBucketReplicas + threadIdx.x;
+        if (threadIdx.x < kBucketReplicas && rep < reps) {
+            const int r = rep / mp, q = rep - r * mp;
+            int64_t *dst = base + (int64_t)r * replica_words + (int64_t)q * stage_words + k0 * 5;
+            // 16-byte aligned copies take img_a from word 0, the others img_b from word 1
+            const bool odd = ((reinterpret_cast<uintptr_t>(dst) >> 3) & 1) != 0;
+            const int head = odd ? 1 : 0;
+            const int bulk_words = (total - head) & ~1;
+            if (odd) __stcs(dst, img_a[0]);
+            if (head + bulk_words < total) __stcs(dst + total - 1, img_a[total - 1]);
+            // the image is rewritten by the next run, and the block's shared memory must outlive
+            // the copy engine's reads of it
+            if (bulk_words > 0) {
+                const int64_t *src = odd ? img_b + 2 : img_a;
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                             :: "l"(dst + head), "r"(smem_addr(src)), "r"(bulk_words * 8) : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            }
+        }
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(kItemThreads)
 emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_t *__restrict__ op_start,
                   int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */,
-                  int cap /* words of one image: even, at least the longest run of any selection */)
+                  int cap /* words of one image: even, at least the longest run of any selection */,
+                  int item_tiles /* blocks (per selection) beyond these write gradient-bucket records */,
+                  int bucket_run /* buckets per image of those blocks */)
 {
     extern __shared__ __align__(16) int64_t dyn_s[];
+    if ((int)blockIdx.x >= item_tiles) {
+        emit_buckets_block(v, plans[blockIdx.y], (int)blockIdx.x - item_tiles, out, bucket_run, dyn_s);
+        return;
+    }
     int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
     int64_t *img_b = dyn_s + cap;                       // the same word at img_b[x + 1]
     int64_t *tmpl = dyn_s + 2 * cap + 2;                // [rf*5] forward, then [rb*5] backward
@@ -386,111 +539,6 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     if (bulk_words > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
-// Gradient-bucket records.  A block owns (selection, stage, chunk of replicas).  Buckets whose last byte lies in the same layer share a ready time, so once the
-// first of them has started the rest follow back to back: per layer one serial step (lane 0),
-// inside a layer a closed form (a thread per bucket).  The records of up to `run` buckets
-// are assembled in shared memory once and sent to every replica by a bulk copy, as in
-// emit_items_kernel.
-__global__ void __launch_bounds__(kBucketThreads)
-emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *__restrict__ out, int run /* buckets per image */)
-{
-    extern __shared__ __align__(16) int64_t dyn_s[];
-    int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
-    int64_t *img_b = dyn_s + run * 5 + 1;               // the same word at img_b[x + 1] (run * 5 + 1 is even)
-    __shared__ int64_t g_start[DISTSIM_MAX_LAYERS + 1];   // start of the first bucket ending in layer a+i
-    __shared__ int64_t g_first[DISTSIM_MAX_LAYERS + 1];   // number of that bucket
-    __shared__ int64_t part_start_s;
-    const EmitPlan &p = plans[blockIdx.y];
-    if (!p.ok || p.dp == 1) return;
-    const int mp = p.mp, reps = mp * p.dp;
-    const int rep_chunks = (reps + kBucketReplicas - 1) / kBucketReplicas;
-    const int d = blockIdx.x / rep_chunks, rc = blockIdx.x - d * rep_chunks;
-    if (d >= p.pp) return;
-    const int64_t kb = p.n_buckets[d];
-    if (kb == 0) return;
-    const Row &row = v.rows[p.row];
-    const int a = p.bounds[d], e = p.bounds[d + 1];
-    const int L1 = v.tc.n_layers + 1;
-    const int64_t *nbe = v.nb + row.row_tab_off + (int64_t)e * L1;
-    const int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
-    const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
-    const int64_t n_full = nbe[a], t_full = row.t_full;
-    const int64_t tbs = p.last_b_start[d], main_end = p.main_end[d];
-    // all threads fetch the per-layer inputs (independent loads), then thread 0 runs the short chain
-    for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
-        g_first[l - a] = l + 1 < e ? nbe[l + 1] : 0;                       // buckets before layer l's group
-        g_start[l - a] = v.tc.overlap ? tbs + (pb[e] - pb[l]) : main_end;    // ready time of the group
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int64_t end = 0, part_start = 0;
-        for (int l = e - 1; l >= a; --l) {
-            const int64_t nb_prev = g_first[l - a];
-            const int64_t nb_l = l > a ? g_first[l - 1 - a] : n_full;       // nb[e][l]
-            const int64_t start = max64(end, g_start[l - a]);
-            g_start[l - a] = start;
-            if (nb_l > nb_prev) end = start + (nb_l - nb_prev) * t_full;
-        }
-        if (part > 0) {
-            const int ls = v.next_grad[a];
-            const int64_t ready = v.tc.overlap ? tbs + (pb[e] - pb[ls]) : main_end;
-            part_start = max64(end, ready);
-        }
-        part_start_s = part_start;
-    }
-    __syncthreads();
-    const int64_t part_start = part_start_s;
-    const int64_t stage_words = p.stage_recs[d] * 5;
-    const int64_t replica_words = (int64_t)mp * p.stage_rec_prefix[p.pp] * 5;
-    int64_t *base = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + (int64_t)p.m * (p.rf[d] + p.rb[d]) * 5;
-    for (int64_t k0 = 0; k0 < kb; k0 += run) {
-        const int nk = (int)min((int64_t)run, kb - k0);
-        for (int kk = threadIdx.x; kk < nk; kk += blockDim.x) {
-            const int64_t k = k0 + kk;
-            int64_t start, dur;
-            if (k >= n_full) { start = part_start; dur = part; }
-            else {
-                // the layer whose group holds bucket k: the largest l with nb[e][l] > k
-                // (nb[e][l] = g_first[l-1-a] for l > a grows as l decreases, and nb[e][a] = n_full > k)
-                int lo = a, hi = e - 1;
-                while (lo < hi) {
-                    const int mid = (lo + hi + 1) >> 1;
-                    if (g_first[mid - 1 - a] > k) lo = mid; else hi = mid - 1;
-                }
-                start = g_start[lo - a] + (k - g_first[lo - a]) * t_full;
-                dur = t_full;
-            }
-            const int64_t rec[5] = {DISTSIM_DP_AR, k, -1, start, start + dur};
-#pragma unroll
-            for (int f = 0; f < 5; ++f) { img_a[kk * 5 + f] = rec[f]; img_b[kk * 5 + f + 1] = rec[f]; }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncthreads();
-        const int total = nk * 5;
-        const int rep = rc * kBucketReplicas + threadIdx.x;
-        if (threadIdx.x < kBucketReplicas && rep < reps) {
-            const int r = rep / mp, q = rep - r * mp;
-            int64_t *dst = base + (int64_t)r * replica_words + (int64_t)q * stage_words + k0 * 5;
-            // 16-byte aligned copies take img_a from word 0, the others img_b from word 1
-            const bool odd = ((reinterpret_cast<uintptr_t>(dst) >> 3) & 1) != 0;
-            const int head = odd ? 1 : 0;
-            const int bulk_words = (total - head) & ~1;
-            if (odd) __stcs(dst, img_a[0]);
-            if (head + bulk_words < total) __stcs(dst + total - 1, img_a[total - 1]);
-            // the image is rewritten by the next run, and the block's shared memory must outlive
-            // the copy engine's reads of it
-            if (bulk_words > 0) {
-                const int64_t *src = odd ? img_b + 2 : img_a;
-                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                             :: "l"(dst + head), "r"(smem_addr(src)), "r"(bulk_words * 8) : "memory");
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            }
-        }
-        __syncthreads();
-    }
-}
-
 // Order-sensitive 64-bit checksum of every device's record stream: the sum over the stream's
 // words w_i (five per record, i counted from the start of the device's list) of
 // mix(w_i + (i + 1) * 0x9E3779B97F4A7C15) modulo 2^64, mix being the SplitMix64 finaliser.  Moving,
@@ -537,14 +585,13 @@ void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const 
 }
 
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
-                      EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand,
+                      EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
                       int64_t *launches)
 {
     cudaMemsetAsync(d_totals, 0, sizeof(EmitTotals), s);
-    emit_plan_kernel<<<(n + 3) / 4, 128, 0, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand);
-    emit_scan_kernel<<<1, 1024, 0, s>>>(plans, n, d_totals);
-    *launches += 2;
+    emit_plan_kernel<<<(n + 3) / 4, 128, 0, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand, sums, d_totals);
+    ++*launches;
     if (offsets || busy || util) {
         const int64_t total = (int64_t)n * v.tc.n_devices + 1;
         emit_devices_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(v, plans, n, offsets, busy, util, d_totals);
@@ -559,21 +606,21 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
     if (n == 0 || t.item_tiles == 0) return;
     // two images of the run, then the forward and backward item templates of the widest stage
     const int cap = (int)((t.run_words + 1) & ~(int64_t)1);
-    const size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
+    size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
+    // the blocks beyond the item tiles write the gradient-bucket records of a (stage, replica chunk):
+    // an odd number of buckets per image keeps both images 16-byte aligned
+    int run = 0, bucket_tiles = 0;
+    if (t.bucket_tiles > 0 && t.bucket_recs > 0) {
+        run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun) | 1;
+        bucket_tiles = (int)t.bucket_tiles;
+        const size_t bsmem = (size_t)(2 * (run * 5 + 1) + 2 * (DISTSIM_MAX_LAYERS + 1)) * sizeof(int64_t);
+        if (bsmem > smem) smem = bsmem;
+    }
     ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_items_kernel), smem);
     int64_t *out = reinterpret_cast<int64_t *>(records);
-    emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
-        v, plans, op_start, op_words_per_cand, out, cap);
+    emit_items_kernel<<<dim3((unsigned)(t.item_tiles + bucket_tiles), (unsigned)n), kItemThreads, smem, s>>>(
+        v, plans, op_start, op_words_per_cand, out, cap, (int)t.item_tiles, run);
     ++*launches;
-    if (t.bucket_tiles > 0 && t.bucket_recs > 0) {
-        // an odd number of buckets per image keeps both images 16-byte aligned
-        int run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun);
-        run |= 1;
-        const size_t bsmem = (size_t)(2 * (run * 5 + 1)) * sizeof(int64_t);
-        ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_buckets_kernel), bsmem);
-        emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, s>>>(v, plans, out, run);
-        ++*launches;
-    }
 }
 
 }  // namespace distsim

@@ -180,22 +180,12 @@ struct SideStream {
     cudaStream_t side[1] = {nullptr};
     cudaEvent_t fork = nullptr, join[1] = {nullptr};
 };
-// Selection folded into an evaluation (enabled != 0): every result also enters a running
-// minimum of the packed key (time << idx_bits | position in the output) and the histogram of
-// the first radix-select digit (time >> shift) & (2^width - 1), so that neither the best
-// candidate nor the first pass of the k fastest needs to read the results again.
-constexpr int kSelectBins = 2048;                 // bins of a radix-select digit (11 bits)
-struct FusedSelect {
-    unsigned long long *key;                      // packed minimum (all ones: none yet)
-    unsigned long long *hist;                     // [kSelectBins]
-    int32_t idx_bits, shift, width, enabled;
-};
 // Evaluates candidates [first, first + count); rows / entries: host copies.  Results go to
 // batch_out[index - first] and, if non-null, busy_out[(index - first) * pp_max + d].  All work
 // is ordered after what `s` held before the call and before what is enqueued on `s` after it.
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
-                 const FusedSelect &fs, int64_t *launches);
+                 int64_t *launches);
 // Cuts candidates [lo, hi) of a row of pp stages into pieces of at most max_blocks lock-step
 // blocks each; returns the number of pieces and writes the first max_pieces of them.
 int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
@@ -213,19 +203,16 @@ struct SelectScratch {
 // d_result[0] = smallest time, d_result[1] = its smallest position in `batch`.
 void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t time_bound,
                    const SelectScratch &sc, int64_t *d_result, int64_t *launches);
-// Selection folded into an evaluation of `count` results whose times are below time_bound:
-// clears the key and the histogram, initialises the radix select for rank k and returns what the
-// evaluation kernels need (enabled = 0 when time and position do not fit one 64-bit key, or
-// the array is small enough to be sorted directly).
-FusedSelect begin_fused_select(cudaStream_t s, int64_t count, int k, int64_t time_bound, const SelectScratch &sc,
-                               int64_t *launches);
-// After the evaluation: d_result[0] = smallest time, d_result[1] = its smallest position.
-void finish_fused_argmin(cudaStream_t s, const FusedSelect &fs, const SelectScratch &sc, int64_t *d_result,
-                         int64_t *launches);
-// After the evaluation: the k fastest, continuing from the histogram the evaluation filled.
-void finish_fused_topk(cudaStream_t s, const FusedSelect &fs, const int64_t *batch, int64_t first, int64_t count, int k,
-                       int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
-                       int64_t *launches);
+// The best element and the k fastest of a long array in little more than one pass over it: a
+// strided sample gives a threshold that at least k elements do not exceed (the k-th smallest of
+// a subset is never below the k-th smallest of the whole); one pass then takes the minimum of
+// the packed (time, position) key and copies the elements up to the threshold to the compact
+// buffer, and the selection proper runs on that buffer.  d_result (nullable): [0] smallest
+// time, [1] its smallest position.  k == 0: the best element only.
+void launch_select(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k, int64_t time_bound,
+                   const SelectScratch &sc, int64_t *d_result, int64_t *d_indices, int64_t *d_times,
+                   int64_t *launches);
+void launch_add_scalar(cudaStream_t s, int64_t *d_word, int64_t value, int64_t *launches);    // *d_word += value
 // time_bound: an upper bound on every element of `batch` (INT64_MAX if unknown).
 void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
                  int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
@@ -261,9 +248,11 @@ struct EmitTotals {
     int64_t pad[2];
 };
 // Plans the n selections: item start times into op_start (op_words_per_cand words each), record
-// counts, offsets / busy / util (each nullable); d_totals: the words of an EmitTotals.
+// counts, offsets / busy / util (each nullable); sums: scratch of kEmitSumWords words per
+// selection; d_totals: the words of an EmitTotals.
+constexpr int kEmitSumWords = 8;
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
-                      EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand,
+                      EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
                       int64_t *launches);
 // out[k] = order-sensitive checksum of the records [offsets[k], offsets[k + 1]).

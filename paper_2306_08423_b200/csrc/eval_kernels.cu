@@ -25,13 +25,14 @@ namespace {
 // Threads per block of the lock-step kernel.  Blocks are small so that the long candidates of
 // a row (many micro-batches: hundreds of slots) spread over all SMs instead of sharing a few.
 constexpr int kEvalThreads = 64;
+constexpr int kLockstepBinomWords = 512;          // binomial tables up to this size are copied to shared memory
 
 // The part of a block's work that depends on the number of stages a lane owns.
 template <int S, bool kJit>
 __device__ __forceinline__ void lockstep_block(const DeviceView &v, const EvalWork &wk, const Row &row, int local_block,
                                                int64_t first, int64_t *__restrict__ batch_out,
                                                int64_t *__restrict__ busy_out, int smem_words,
-                                               unsigned char *smem_raw, uint64_t *bar, const FusedSelect &fs)
+                                               unsigned char *smem_raw, uint64_t *bar, const int64_t *binom)
 {
     const int64_t lo = wk.lo, hi = wk.hi;
     const int pp = row.pp;
@@ -71,23 +72,9 @@ __device__ __forceinline__ void lockstep_block(const DeviceView &v, const EvalWo
     n_slots = __reduce_max_sync(0xffffffffu, n_slots);
 
     const StageResult<S> R = lockstep_candidate<S, false, kJit>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank,
-                                                                seg_lane, wl, n_slots, nullptr);
-    const int64_t out = row.offset + local - first;
-    if (fs.enabled) {
-        // selection folded in: the warp's smallest packed key, one histogram count per candidate
-        unsigned long long key = ~0ull;
-        if (valid && seg_lane == 0) {
-            key = ((unsigned long long)R.batch << fs.idx_bits) | (unsigned long long)out;
-            atomicAdd(&fs.hist[(uint32_t)((unsigned long long)R.batch >> fs.shift) & ((1u << fs.width) - 1u)], 1ull);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
-            key = other < key ? other : key;
-        }
-        if (lane == 0 && key != ~0ull) atomicMin(fs.key, key);
-    }
+                                                                seg_lane, wl, n_slots, nullptr, binom);
     if (!valid) return;
+    const int64_t out = row.offset + local - first;
     if (seg_lane == 0) batch_out[out] = R.batch;
     if (busy_out) {
         int64_t *bo = busy_out + out * v.sc.pp_max;
@@ -100,10 +87,12 @@ __device__ __forceinline__ void lockstep_block(const DeviceView &v, const EvalWo
 template <bool kJit>
 __global__ void __launch_bounds__(kEvalThreads)
 eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
-                     int64_t *__restrict__ busy_out, int smem_words, FusedSelect fs)
+                     int64_t *__restrict__ busy_out, int smem_words)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t bar;
+    __shared__ int64_t binom_s[kLockstepBinomWords];
+    const int64_t *binom = stage_binom(v, binom_s, kLockstepBinomWords);
     int wi = 0;
     while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
     const EvalWork &wk = batch.w[wi];
@@ -111,8 +100,8 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     // A row's candidates grow in micro-batch count, hence in slots, with their index: its last
     // blocks are the long ones and take the first block numbers, so that they start first.
     const int local_block = wk.nx - 1 - ((int)blockIdx.x - wk.block_begin);
-    if (row.pp > 32) lockstep_block<2, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar, fs);
-    else lockstep_block<1, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar, fs);
+    if (row.pp > 32) lockstep_block<2, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar, binom);
+    else lockstep_block<1, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar, binom);
 }
 
 // Work items collected for one kernel instance, launched when full or at the end.
@@ -141,16 +130,16 @@ int lockstep_smem_words(const DeviceView &v, const Row &row)
 }
 
 void flush_lockstep(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first, int64_t *batch_out,
-                    int64_t *busy_out, const FusedSelect &fs, int64_t *launches)
+                    int64_t *busy_out, int64_t *launches)
 {
     if (p.batch.n == 0) return;
     const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
     if (v.tc.n_jitter > 0) {
         ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_lockstep_kernel<true>), smem);
-        eval_lockstep_kernel<true><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words, fs);
+        eval_lockstep_kernel<true><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
     } else {
         ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_lockstep_kernel<false>), smem);
-        eval_lockstep_kernel<false><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words, fs);
+        eval_lockstep_kernel<false><<<p.blocks, kEvalThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, p.smem_words);
     }
     ++*launches;
     p = Pending{};
@@ -158,16 +147,16 @@ void flush_lockstep(cudaStream_t s, const DeviceView &v, Pending &p, int64_t fir
 
 template <int PP, typename T, bool kBusy>
 void flush_thread(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first, int64_t *batch_out,
-                  int64_t *busy_out, const FusedSelect &fs, int64_t *launches)
+                  int64_t *busy_out, int64_t *launches)
 {
     if (p.batch.n == 0) return;
     const size_t smem = (size_t)p.smem_words * sizeof(int64_t);
     if (v.tc.n_jitter > 0) {
         ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_thread_kernel<PP, T, kBusy, true>), smem);
-        eval_thread_kernel<PP, T, kBusy, true><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out, fs);
+        eval_thread_kernel<PP, T, kBusy, true><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out);
     } else {
         ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_thread_kernel<PP, T, kBusy, false>), smem);
-        eval_thread_kernel<PP, T, kBusy, false><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out, fs);
+        eval_thread_kernel<PP, T, kBusy, false><<<p.blocks, kThreadBlock, smem, s>>>(v, p.batch, first, batch_out, busy_out);
     }
     ++*launches;
     p = Pending{};
@@ -176,40 +165,40 @@ void flush_thread(cudaStream_t s, const DeviceView &v, Pending &p, int64_t first
 // Thread-kernel instances are indexed by (log2 pp, narrow).
 template <typename T, bool kBusy>
 void flush_thread_pp(int log2pp, cudaStream_t s, const DeviceView &v, Pending &p, int64_t first,
-                     int64_t *batch_out, int64_t *busy_out, const FusedSelect &fs, int64_t *launches)
+                     int64_t *batch_out, int64_t *busy_out, int64_t *launches)
 {
     switch (log2pp) {
-    case 0: flush_thread<1, T, kBusy>(s, v, p, first, batch_out, busy_out, fs, launches); break;
-    case 1: flush_thread<2, T, kBusy>(s, v, p, first, batch_out, busy_out, fs, launches); break;
-    case 2: flush_thread<4, T, kBusy>(s, v, p, first, batch_out, busy_out, fs, launches); break;
-    case 3: flush_thread<8, T, kBusy>(s, v, p, first, batch_out, busy_out, fs, launches); break;
-    default: flush_thread<16, T, kBusy>(s, v, p, first, batch_out, busy_out, fs, launches); break;
+    case 0: flush_thread<1, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
+    case 1: flush_thread<2, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
+    case 2: flush_thread<4, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
+    case 3: flush_thread<8, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
+    default: flush_thread<16, T, kBusy>(s, v, p, first, batch_out, busy_out, launches); break;
     }
 }
 
 void flush_thread_any(int log2pp, bool narrow, cudaStream_t s, const DeviceView &v, Pending &p, int64_t first,
-                      int64_t *batch_out, int64_t *busy_out, const FusedSelect &fs, int64_t *launches)
+                      int64_t *batch_out, int64_t *busy_out, int64_t *launches)
 {
     if (narrow) {
-        if (busy_out) flush_thread_pp<uint32_t, true>(log2pp, s, v, p, first, batch_out, busy_out, fs, launches);
-        else flush_thread_pp<uint32_t, false>(log2pp, s, v, p, first, batch_out, busy_out, fs, launches);
+        if (busy_out) flush_thread_pp<uint32_t, true>(log2pp, s, v, p, first, batch_out, busy_out, launches);
+        else flush_thread_pp<uint32_t, false>(log2pp, s, v, p, first, batch_out, busy_out, launches);
     } else {
-        if (busy_out) flush_thread_pp<int64_t, true>(log2pp, s, v, p, first, batch_out, busy_out, fs, launches);
-        else flush_thread_pp<int64_t, false>(log2pp, s, v, p, first, batch_out, busy_out, fs, launches);
+        if (busy_out) flush_thread_pp<int64_t, true>(log2pp, s, v, p, first, batch_out, busy_out, launches);
+        else flush_thread_pp<int64_t, false>(log2pp, s, v, p, first, batch_out, busy_out, launches);
     }
 }
 
 int ilog2(int v) { int b = 0; while ((1 << (b + 1)) <= v) ++b; return b; }
 
 // The shared-memory budget of the kernel instance that evaluates rows of this pp and arithmetic width.
-int thread_budget_words(int pp, bool narrow, bool jitter, bool select_hist)
+int thread_budget_words(int pp, bool narrow, bool jitter)
 {
     switch (ilog2(pp)) {
-    case 0: return narrow ? thread_kernel_budget_words<1, uint32_t>(jitter, select_hist) : thread_kernel_budget_words<1, int64_t>(jitter, select_hist);
-    case 1: return narrow ? thread_kernel_budget_words<2, uint32_t>(jitter, select_hist) : thread_kernel_budget_words<2, int64_t>(jitter, select_hist);
-    case 2: return narrow ? thread_kernel_budget_words<4, uint32_t>(jitter, select_hist) : thread_kernel_budget_words<4, int64_t>(jitter, select_hist);
-    case 3: return narrow ? thread_kernel_budget_words<8, uint32_t>(jitter, select_hist) : thread_kernel_budget_words<8, int64_t>(jitter, select_hist);
-    default: return narrow ? thread_kernel_budget_words<16, uint32_t>(jitter, select_hist) : thread_kernel_budget_words<16, int64_t>(jitter, select_hist);
+    case 0: return narrow ? thread_kernel_budget_words<1, uint32_t>(jitter) : thread_kernel_budget_words<1, int64_t>(jitter);
+    case 1: return narrow ? thread_kernel_budget_words<2, uint32_t>(jitter) : thread_kernel_budget_words<2, int64_t>(jitter);
+    case 2: return narrow ? thread_kernel_budget_words<4, uint32_t>(jitter) : thread_kernel_budget_words<4, int64_t>(jitter);
+    case 3: return narrow ? thread_kernel_budget_words<8, uint32_t>(jitter) : thread_kernel_budget_words<8, int64_t>(jitter);
+    default: return narrow ? thread_kernel_budget_words<16, uint32_t>(jitter) : thread_kernel_budget_words<16, int64_t>(jitter);
     }
 }
 
@@ -239,12 +228,9 @@ int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int6
 
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
-                 const FusedSelect &fs_in, int64_t *launches)
+                 int64_t *launches)
 {
     const int64_t last = first + count;
-    // the selection is folded into the instances without per-stage activity output
-    FusedSelect fs = fs_in;
-    if (busy_out) fs.enabled = 0;
     struct ThreadItem { EvalWork w; int lg; bool narrow; int blocks, words; };
     std::vector<EvalWork> lock_items;              // lock-step kernel
     std::vector<int> lock_words;
@@ -289,8 +275,7 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
             }
             const int64_t n_parts = p_hi - p_lo;
             const int n_e = r1 - r0;
-            // entries per thread (a block's 16-bit histogram counters hold 128 threads x 160 entries x 3 schedules)
-            const int ept = n_parts >= 148 * 4 * kThreadBlock ? (n_e < 160 ? n_e : 160) : 1;
+            const int ept = n_parts >= 148 * 4 * kThreadBlock ? n_e : 1;       // entries per thread
             const int64_t nx = (n_parts + kThreadBlock - 1) / kThreadBlock;
             const int64_t ny = (n_e + ept - 1) / ept;
             if (n_parts * ny >= 2048 && nx * ny < kMaxBlocks) {
@@ -300,7 +285,7 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
                 w.row = r; w.e_begin = r0; w.e_end = r1; w.ept = ept; w.p_lo = p_lo; w.p_hi = p_hi;
                 w.lo = lo_r; w.hi = hi_r; w.nx = (int)nx;
                 const int binom_words = v.sc.partition_mode ? v.tc.n_layers * v.sc.binom_k : 0;
-                const int budget = thread_budget_words(row.pp, narrow, v.tc.n_jitter > 0, busy_out == nullptr);
+                const int budget = thread_budget_words(row.pp, narrow, v.tc.n_jitter > 0);
                 const bool use32 = narrow && v.pfb32 != nullptr && (row.dp == 1 || v.dt32 != nullptr);   // as in the kernel
                 it.words =
                     use32 ? thread_kernel_smem32(row.n_entries, v.tc.lp, v.tab_words32, v.dt32 != nullptr, binom_words, budget).words
@@ -327,7 +312,7 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
     Pending p;
     for (size_t i = 0; i < lock_items.size(); ++i) {
         if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - lock_items[i].nx)
-            flush_lockstep(ls, v, p, first, batch_out, busy_out, fs, launches);
+            flush_lockstep(ls, v, p, first, batch_out, busy_out, launches);
         EvalWork &w = p.batch.w[p.batch.n++];
         w = lock_items[i];
         w.block_begin = p.blocks;
@@ -335,20 +320,20 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
         // one dynamic size per launch: the largest any item wants (items that want none still work)
         if (lock_words[i] > p.smem_words) p.smem_words = lock_words[i];
     }
-    flush_lockstep(ls, v, p, first, batch_out, busy_out, fs, launches);
+    flush_lockstep(ls, v, p, first, batch_out, busy_out, launches);
     for (int lg = 4; lg >= 0; --lg)
         for (int nw = 1; nw >= 0; --nw) {
             for (const ThreadItem &it : thread_items) {
                 if (it.lg != lg || it.narrow != (nw == 1)) continue;
                 if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - it.blocks)
-                    flush_thread_any(lg, nw == 1, s, v, p, first, batch_out, busy_out, fs, launches);
+                    flush_thread_any(lg, nw == 1, s, v, p, first, batch_out, busy_out, launches);
                 EvalWork &w = p.batch.w[p.batch.n++];
                 w = it.w;
                 w.block_begin = p.blocks;
                 p.blocks += it.blocks;
                 if (it.words > p.smem_words) p.smem_words = it.words;
             }
-            flush_thread_any(lg, nw == 1, s, v, p, first, batch_out, busy_out, fs, launches);
+            flush_thread_any(lg, nw == 1, s, v, p, first, batch_out, busy_out, launches);
         }
     if (use_side) {
         cudaEventRecord(ss.join[0], ss.side[0]);

@@ -395,11 +395,11 @@ struct ThreadKernelSmem {
 // blocks the kernel is compiled for: an SM's 228 KB, less 1 KB per block, less the kernel's
 // static arrays.
 template <int PP, typename T>
-__host__ __device__ constexpr int thread_kernel_budget_words(bool jitter, bool select_hist)
+__host__ __device__ constexpr int thread_kernel_budget_words(bool jitter)
 {
     const int per_block = 233472 / thread_kernel_min_blocks<PP, T>() - 1024;
     const int fixed = PP * kThreadBlock * (int)sizeof(T) + (PP + 1) * kThreadBlock * 2 + 16 * 24 + 256 +
-                      (jitter ? 2 * 64 * PP * (int)sizeof(T) : 0) + (select_hist ? kSelectBins * 2 + 64 : 0);
+                      (jitter ? 2 * 64 * PP * (int)sizeof(T) : 0);
     return (per_block - fixed) / 8 > 0 ? (per_block - fixed) / 8 : 0;
 }
 __host__ __device__ inline ThreadKernelSmem thread_kernel_smem(int n_entries, int lp, int tab_words, bool have_dt,
@@ -477,7 +477,7 @@ constexpr int kMaxJitterSlots = 64;
 template <int PP, typename T, bool kBusy, bool kJit>
 __global__ void __launch_bounds__(kThreadBlock, thread_kernel_min_blocks<PP, T>())
 eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
-                   int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out, FusedSelect fs)
+                   int64_t *__restrict__ batch_out, int64_t *__restrict__ busy_out)
 {
     // which work item (row and range) this block belongs to
     int wi = 0;
@@ -493,15 +493,6 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
     __shared__ uint16_t cs[PP + 1][kThreadBlock];     // per thread: stage bounds c_0 .. c_PP
     __shared__ EntryLite ents[kMaxRowEntries];
     __shared__ T jit_f_s[kJit ? kMaxJitterSlots * PP : 1], jit_b_s[kJit ? kMaxJitterSlots * PP : 1];
-    // Selection folded into the evaluation (instances without per-stage activity output): the
-    // block's histogram of the first radix-select digit, two 16-bit counters per word (a block
-    // produces fewer than 65 536 results), and the warps' smallest packed keys.
-    __shared__ uint32_t sel_hist[kBusy ? 1 : kSelectBins / 2];
-    __shared__ unsigned long long sel_min[kBusy ? 1 : kThreadBlock / 32];
-    const bool select = !kBusy && fs.enabled;
-    if (select)
-        for (int k = threadIdx.x; k < kSelectBins / 2; k += blockDim.x) sel_hist[k] = 0;
-    unsigned long long best_key = ~0ull;
     const Row &row = v.rows[row_index];
     const int lp = v.tc.lp;
     const int L1 = v.tc.n_layers + 1;
@@ -510,9 +501,9 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
     const bool use32 = sizeof(T) == 4 && v.pfb32 != nullptr && (row.dp == 1 || v.dt32 != nullptr);
     const ThreadKernelSmem plan =
         use32 ? thread_kernel_smem32(row.n_entries, lp, v.tab_words32, v.dt32 != nullptr, binom_words,
-                                     thread_kernel_budget_words<PP, T>(kJit, !kBusy))
+                                     thread_kernel_budget_words<PP, T>(kJit))
               : thread_kernel_smem(row.n_entries, lp, v.tab_words, v.dt != nullptr, binom_words,
-                                   thread_kernel_budget_words<PP, T>(kJit, !kBusy));
+                                   thread_kernel_budget_words<PP, T>(kJit));
     const int dp = row.dp, n_sched = row.n_sched, sched_list = row.sched_list, period = row.p2p_period;
     const int64_t t_full = row.t_full;
 
@@ -570,7 +561,7 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
     const int64_t *tpt = (staged && plan.tables_staged) ? dsm + plan.off_tp : tp_g;
 
     const int64_t part = p_lo + (int64_t)block_x * kThreadBlock + threadIdx.x;
-    if (part < p_hi) {                                   // (idle threads still join the block's epilogue)
+    if (part >= p_hi) return;
     const int e0 = e_begin + block_y * entries_per_thread;
     const int e1 = min(e_end, e0 + entries_per_thread);
 
@@ -746,36 +737,6 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
             if (local0 >= lo && local0 < hi) batch_out[out0] = res0;
             if (n_sched > 1 && local0 + 1 >= lo && local0 + 1 < hi) batch_out[out0 + 1] = res1;
             if (n_sched > 2 && local0 + 2 >= lo && local0 + 2 < hi) batch_out[out0 + 2] = res2;
-        }
-        if (select) {
-#pragma unroll
-            for (int sc = 0; sc < 3; ++sc) {
-                if (sc >= n_sched || local0 + sc < lo || local0 + sc >= hi) continue;
-                const unsigned long long tm = (unsigned long long)(sc == 0 ? res0 : (sc == 1 ? res1 : res2));
-                const unsigned long long key = (tm << fs.idx_bits) | (unsigned long long)(out0 + sc);
-                best_key = key < best_key ? key : best_key;
-                const uint32_t bin = (uint32_t)(tm >> fs.shift) & ((1u << fs.width) - 1u);
-                atomicAdd(&sel_hist[bin >> 1], 1u << ((bin & 1u) * 16));
-            }
-        }
-    }
-    }
-    if (!kBusy && fs.enabled) {                          // block-uniform
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best_key, o);
-            best_key = other < best_key ? other : best_key;
-        }
-        if ((threadIdx.x & 31) == 0) sel_min[threadIdx.x >> 5] = best_key;
-        __syncthreads();                                 // the block's histogram is complete as well
-        if (threadIdx.x == 0) {
-            for (int w = 1; w < kThreadBlock / 32; ++w) best_key = sel_min[w] < best_key ? sel_min[w] : best_key;
-            if (best_key != ~0ull) atomicMin(fs.key, best_key);
-        }
-        for (int k = threadIdx.x; k < kSelectBins / 2; k += blockDim.x) {
-            const uint32_t w = sel_hist[k];
-            if (w & 0xFFFFu) atomicAdd(&fs.hist[2 * k], (unsigned long long)(w & 0xFFFFu));
-            if (w >> 16) atomicAdd(&fs.hist[2 * k + 1], (unsigned long long)(w >> 16));
         }
     }
 }

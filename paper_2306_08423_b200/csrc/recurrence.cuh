@@ -28,8 +28,9 @@ __device__ __forceinline__ int64_t max64(int64_t a, int64_t b) { return a > b ? 
 // Balanced mode: c_j = floor(j L / pp).  All-compositions mode: the (pp-1)-subsets of
 // {1..L-1} in lexicographic order, decoded with the combinatorial number system: position i
 // takes the smallest value c whose block of C(L-1-c, pp-1-i) completions contains the rank.
+// `binom`: the binomial table, in global memory (v.binom) or a block's copy of it in shared memory.
 template <int S>
-__device__ __forceinline__ void partition_bounds(const DeviceView &v, int pp, int64_t part_rank,
+__device__ __forceinline__ void partition_bounds(const DeviceView &v, const int64_t *binom, int pp, int64_t part_rank,
                                                  int d0, int (&out)[S + 1])
 {
     const int L = v.tc.n_layers;
@@ -47,7 +48,7 @@ __device__ __forceinline__ void partition_bounds(const DeviceView &v, int pp, in
         ++c;
         const int kk = pp - 1 - i;
         while (true) {
-            const int64_t cnt = __ldg(&v.binom[(int64_t)(L - 1 - c) * v.sc.binom_k + kk]);
+            const int64_t cnt = binom[(int64_t)(L - 1 - c) * v.sc.binom_k + kk];
             if (r < cnt) break;
             r -= cnt;
             ++c;
@@ -55,6 +56,19 @@ __device__ __forceinline__ void partition_bounds(const DeviceView &v, int pp, in
 #pragma unroll
         for (int k = 0; k <= S; ++k) if (i == d0 + k) out[k] = c;
     }
+}
+
+// Copies the binomial table into shared memory when it fits `cap_words` (decoding a partition
+// walks it with dependent loads); returns the table to use.  Every thread of the block calls it;
+// contains a block-wide barrier.
+__device__ __forceinline__ const int64_t *stage_binom(const DeviceView &v, int64_t *smem, int cap_words)
+{
+    const int words = v.sc.partition_mode ? v.tc.n_layers * v.sc.binom_k : 0;
+    const bool fits = words > 0 && words <= cap_words;
+    if (fits)
+        for (int i = threadIdx.x; i < words; i += blockDim.x) smem[i] = __ldg(&v.binom[i]);
+    __syncthreads();
+    return fits ? smem : v.binom;
 }
 
 struct CandidateCoords {
@@ -194,6 +208,7 @@ __device__ __forceinline__ int64_t shfl_idx64(int64_t x, int src_lane)
 //   n_slots_warp loop bound, uniform over the warp
 //   pf, pb     the entry's forward / backward prefix rows (shared or global memory)
 //   rec        if kRecord and non-null: item start times go to rec[d * 2m + position in stage order]
+//   binom      the binomial table of the partition decoding (global, or the block's shared copy)
 //   kJit       the table has per-micro-batch jitter (otherwise none of its code is generated)
 // Per stage the only state is t, the end of the stage's latest item (= when its device is free).
 // When an item runs, the item it takes its input from ran on the neighbouring stage in the slot
@@ -207,13 +222,14 @@ __device__ __forceinline__ int64_t shfl_idx64(int64_t x, int src_lane)
 template <int S, bool kRecord, bool kJit>
 __device__ __forceinline__ StageResult<S> lockstep_candidate(
     const DeviceView &v, const Row &row, const Entry &en, int entry_index, const int64_t *pf,
-    const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec)
+    const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec,
+    const int64_t *binom)
 {
     StageResult<S> R;
     const int pp = row.pp, m = en.m;
     const int d0 = seg_lane * S;
     int bounds[S + 1];
-    partition_bounds<S>(v, pp, part_rank, d0, bounds);
+    partition_bounds<S>(v, binom, pp, part_rank, d0, bounds);
     SlotPlan sp[S];
 #pragma unroll
     for (int k = 0; k < S; ++k) {

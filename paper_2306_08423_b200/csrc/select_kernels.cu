@@ -93,44 +93,93 @@ constexpr int kBins = 1 << kRadixBits;
 struct SelState {
     u64 tprefix, tmask, rank, iprefix, imask, blocks_done, cursor, skip_index;
     u64 use_compact, cn;         // remaining passes read the compact buffer of cn pairs
-    u64 pad[6];
+    u64 stride;                  // > 1: the passes read every stride-th element of the array (sampling phase)
+    u64 k;                       // elements wanted
+    u64 threshold;               // sampled selection: a time that at least k elements do not exceed
+    u64 tmin;                    // sampled selection: smallest time of the array
+    u64 small;                   // sampled selection: the candidates fit one sort (n_cand of them)
+    u64 n_cand;
 };
 
 // The source a pass reads: the array itself (index = position) or the compact buffer.
-struct SelSource { const int64_t *t; const int64_t *idx; int64_t n; };
+struct SelSource { const int64_t *t; const int64_t *idx; int64_t n; int64_t stride; };
 __device__ __forceinline__ SelSource sel_source(const SelState *st, const int64_t *batch, int64_t count,
                                                 const SelectScratch &sc)
 {
-    if (st->use_compact) return SelSource{sc.comp_time, sc.comp_idx, (int64_t)st->cn};
-    return SelSource{batch, nullptr, count};
+    if (st->use_compact) return SelSource{sc.comp_time, sc.comp_idx, (int64_t)st->cn, 1};
+    if (st->stride > 1) return SelSource{batch, nullptr, (count + (int64_t)st->stride - 1) / (int64_t)st->stride, (int64_t)st->stride};
+    return SelSource{batch, nullptr, count, 1};
 }
 
-// Run by one whole block once a digit's histogram is complete: picks the bin that holds the
-// wanted rank, narrows the prefix / mask to it and clears the histogram for the next digit.
+// Run by one whole block once a histogram is complete: finds the bin that holds rank `rank`.
+// On thread 0 (only) the results are valid after the call: the bin, the number of elements in
+// the bins before it and in it.  Ends with a block-wide barrier.
+struct PickedBin { int bin; u64 before, in_bin; };
+__device__ __forceinline__ PickedBin find_bin(u64 rank, const u64 *hist, u64 *partial /* shared, [kSelThreads] */)
+{
+    __threadfence();
+    constexpr int kPer = kBins / kSelThreads;
+    u64 mine = 0;
+    for (int k = 0; k < kPer; ++k) mine += *((volatile const u64 *)&hist[threadIdx.x * kPer + k]);
+    partial[threadIdx.x] = mine;
+    __syncthreads();
+    // chunk (a thread's kPer bins) that holds the wanted rank: exclusive scan of the chunk sums by
+    // the first warp, each lane taking kSelThreads / 32 consecutive chunks
+    __shared__ int chunk_s;
+    __shared__ u64 cum_s;
+    if (threadIdx.x < 32) {
+        constexpr int kEach = kSelThreads / 32;
+        u64 sum = 0;
+        for (int c = 0; c < kEach; ++c) sum += partial[threadIdx.x * kEach + c];
+        u64 incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const u64 up = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)threadIdx.x >= o) incl += up;
+        }
+        const u64 total = __shfl_sync(0xffffffffu, incl, 31);
+        const bool mine_has = rank >= incl - sum && rank < incl;
+        const unsigned who = __ballot_sync(0xffffffffu, mine_has);
+        if (who == 0 && threadIdx.x == 0) { chunk_s = kSelThreads - 1; cum_s = total - partial[kSelThreads - 1]; }   // rank beyond the data
+        if (mine_has) {
+            u64 cum = incl - sum;
+            int chunk = threadIdx.x * kEach + kEach - 1;
+            for (int c = 0; c < kEach; ++c) {
+                const u64 pc = partial[threadIdx.x * kEach + c];
+                if (rank < cum + pc) { chunk = threadIdx.x * kEach + c; break; }
+                cum += pc;
+            }
+            chunk_s = chunk; cum_s = cum;
+        }
+    }
+    __syncthreads();
+    PickedBin p{0, 0, 0};
+    if (threadIdx.x == 0) {
+        u64 cum = cum_s;
+        const int chunk = chunk_s;
+        p.bin = chunk * kPer + kPer - 1;
+        for (int k = 0; k < kPer; ++k) {
+            const u64 h = *((volatile const u64 *)&hist[chunk * kPer + k]);
+            if (rank < cum + h) { p.bin = chunk * kPer + k; p.in_bin = h; break; }
+            cum += h;
+        }
+        p.before = cum;
+    }
+    return p;
+}
+
+// The pick step of a radix pass: narrows the prefix / mask to the bin that holds the wanted
+// rank and clears the histogram for the next digit.
 template <bool kIndexPhase>
 __device__ __forceinline__ void pick_bin(SelState *st, u64 *hist, u64 *partial /* shared, [kSelThreads] */, int shift,
                                          unsigned dmask, bool last_time_pass)
 {
     const u64 tprefix = st->tprefix, tmask = st->tmask, iprefix = st->iprefix, imask = st->imask;
-    __threadfence();
-    constexpr int kPer = kBins / kSelThreads;
-    u64 mine = 0;
-    for (int k = 0; k < kPer; ++k) mine += *((volatile u64 *)&hist[threadIdx.x * kPer + k]);
-    partial[threadIdx.x] = mine;
-    __syncthreads();
+    const u64 rank = st->rank;
+    const PickedBin p = find_bin(rank, hist, partial);
     if (threadIdx.x == 0) {
-        u64 rank = st->rank, cum = 0, in_bin = 0;
-        int chunk = kSelThreads - 1;
-        for (int c = 0; c < kSelThreads; ++c) {
-            if (rank < cum + partial[c]) { chunk = c; break; }
-            cum += partial[c];
-        }
-        int bin = chunk * kPer + kPer - 1;
-        for (int k = 0; k < kPer; ++k) {
-            const u64 h = *((volatile u64 *)&hist[chunk * kPer + k]);
-            if (rank < cum + h) { bin = chunk * kPer + k; in_bin = h; break; }
-            cum += h;
-        }
+        const u64 cum = p.before, in_bin = p.in_bin;
+        const int bin = p.bin;
         st->rank = rank - cum;
         if (!kIndexPhase && last_time_pass && in_bin == rank - cum + 1) {
             // the elements equal to the threshold time are exactly the ones still needed
@@ -165,7 +214,7 @@ radix_pass_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratc
     const u64 tprefix = st->tprefix, tmask = st->tmask, iprefix = st->iprefix, imask = st->imask;
     const unsigned dmask = (1u << width) - 1u;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < src.n; i += (int64_t)gridDim.x * blockDim.x) {
-        const u64 x = (u64)src.t[i];
+        const u64 x = (u64)src.t[i * src.stride];
         if ((x & tmask) != tprefix) continue;
         if (kIndexPhase) {
             const u64 id = src.idx ? (u64)src.idx[i] : (u64)i;
@@ -185,18 +234,75 @@ radix_pass_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratc
     pick_bin<kIndexPhase>(st, hist, partial, shift, dmask, last_time_pass);
 }
 
-__global__ void sel_init_kernel(SelState *st, u64 *hist, int k)
+__global__ void sel_init_kernel(SelState *st, u64 *hist, int k, int64_t stride, u64 *key /* nullable: [2], set to all ones */)
 {
     for (int i = threadIdx.x; i < kBins; i += blockDim.x) hist[i] = 0;
-    if (threadIdx.x == 0) { SelState z{}; z.rank = (u64)(k - 1); *st = z; }
+    if (key && threadIdx.x < 2) key[threadIdx.x] = ~0ull;
+    if (threadIdx.x == 0) {
+        SelState z{};
+        z.rank = (u64)(k - 1); z.k = (u64)k; z.stride = (u64)stride; z.tmin = ~0ull;
+        *st = z;
+    }
 }
 
-// The pick step alone, for a first digit whose histogram an evaluation has filled.
+// The one pass over a long array (after the sampling phase has left, in tprefix, a time that at
+// least k elements do not exceed): the minimum of the packed (time, position) key, and every
+// element up to the threshold copied to the compact buffer.  The last block to finish resets the
+// selection state for the selection proper, which then reads the compact buffer - or, should
+// the elements not fit it (masses of ties), the array itself.
 __global__ void __launch_bounds__(kSelThreads)
-radix_pick_kernel(SelectScratch sc, int shift, int width, bool last_time_pass)
+scan_select_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int idx_bits, int want_min,
+                   int want_compact)
 {
-    __shared__ u64 partial[kSelThreads];
-    pick_bin<false>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, partial, shift, (1u << width) - 1u, last_time_pass);
+    __shared__ bool last;
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    const u64 threshold = want_compact ? st->tprefix : 0;
+    u64 best = ~0ull, xmin = ~0ull;
+    // eight independent loads in flight per thread; elements up to the threshold are few (about k
+    // times the sampling stride out of the whole array), so each takes its own atomic
+    constexpr int kUnroll = 8;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < count; i0 += step * kUnroll) {
+        u64 x[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int64_t i = i0 + u * step;
+            x[u] = i < count ? (u64)__ldcs(batch + i) : ~0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int64_t i = i0 + u * step;
+            if (i >= count) continue;
+            xmin = x[u] < xmin ? x[u] : xmin;
+            if (want_min) {
+                const u64 key = (x[u] << idx_bits) | (u64)i;
+                best = key < best ? key : best;
+            }
+            if (want_compact && x[u] <= threshold) {
+                const u64 pos = atomicAdd(&st->cursor, 1ull);
+                if (pos < (u64)sc.comp_cap) { sc.comp_time[pos] = (int64_t)x[u]; sc.comp_idx[pos] = i; }
+            }
+        }
+    }
+    if (want_min) {
+        best = block_min_u64(best);
+        if (threadIdx.x == 0 && best != ~0ull) atomicMin(sc.key, best);
+    }
+    if (!want_compact) return;
+    xmin = block_min_u64(xmin);
+    if (threadIdx.x == 0 && xmin != ~0ull) atomicMin(&st->tmin, xmin);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&st->blocks_done, 1ull) == (u64)gridDim.x - 1;
+    __syncthreads();
+    if (last && threadIdx.x == 0) {
+        const u64 n = *((volatile u64 *)&st->cursor);
+        st->use_compact = n <= (u64)sc.comp_cap ? 1 : 0;
+        st->cn = n;
+        st->threshold = threshold;
+        st->tprefix = 0; st->tmask = 0; st->iprefix = 0; st->imask = 0; st->skip_index = 0;
+        st->rank = st->k - 1; st->stride = 0; st->cursor = 0; st->blocks_done = 0;
+    }
 }
 
 // After the first time pass: copies the elements whose time does not exceed the chosen top
@@ -223,11 +329,14 @@ compact_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch s
     if (last && threadIdx.x == 0) { st->use_compact = 1; st->cursor = 0; st->blocks_done = 0; }
 }
 
-// Collects the k elements that are not above the threshold pair (time, index), in any order.
+// Collects the elements that are not above the threshold pair (time, index), at most k of them,
+// in any order.  only_small: the refined path of the sampled selection - nothing to do unless its
+// candidates fit one sort.
 __global__ void __launch_bounds__(kSelThreads)
-collect_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int k)
+collect_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int k, int only_small)
 {
     SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    if (only_small && !st->small) return;
     const SelSource src = sel_source(st, batch, count, sc);
     const u64 T = st->tprefix, I = st->iprefix;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < src.n; i += (int64_t)gridDim.x * blockDim.x) {
@@ -240,23 +349,10 @@ collect_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch s
     }
 }
 
-// One block sorts up to 4096 (time, index) pairs ascending (bitonic network in shared memory)
-// and writes the first k.  Also the whole top-k for arrays of at most 4096 elements.
-constexpr int kSortMax = 4096;
-__global__ void __launch_bounds__(1024)
-sort_pairs_kernel(const int64_t *__restrict__ ct, const int64_t *__restrict__ ci, int n_in, int k,
-                  int64_t first, int64_t *out_idx, int64_t *out_time)
+// Bitonic sort of np2 (a power of two) (time, index) pairs in shared memory, ascending, by the
+// whole block.
+__device__ __forceinline__ void bitonic_sort_pairs(int64_t *st, int64_t *si, int np2)
 {
-    extern __shared__ __align__(16) unsigned char sm[];
-    int64_t *st = reinterpret_cast<int64_t *>(sm);
-    int64_t *si = st + kSortMax;
-    int np2 = 1;
-    while (np2 < n_in) np2 <<= 1;
-    for (int i = threadIdx.x; i < np2; i += blockDim.x) {
-        st[i] = i < n_in ? ct[i] : INT64_MAX;
-        si[i] = i < n_in ? (ci ? ci[i] : (int64_t)i) : INT64_MAX;
-    }
-    __syncthreads();
     for (int size = 2; size <= np2; size <<= 1)
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
             for (int i = threadIdx.x; i < np2 / 2; i += blockDim.x) {
@@ -271,9 +367,148 @@ sort_pairs_kernel(const int64_t *__restrict__ ct, const int64_t *__restrict__ ci
             }
             __syncthreads();
         }
+}
+
+// One block sorts up to 4096 (time, index) pairs ascending (bitonic network in shared memory)
+// and writes the first k.  Also the whole top-k for arrays of at most 4096 elements.
+// state != nullptr: the refined path of the sampled selection - the number of pairs is the
+// state's n_cand, and there is nothing to do unless the candidates fit (state->small).
+constexpr int kSortMax = 4096;
+__global__ void __launch_bounds__(1024)
+sort_pairs_kernel(const int64_t *__restrict__ ct, const int64_t *__restrict__ ci, int n_in, int k,
+                  int64_t first, int64_t *out_idx, int64_t *out_time, const SelState *state)
+{
+    extern __shared__ __align__(16) unsigned char sm[];
+    int64_t *st = reinterpret_cast<int64_t *>(sm);
+    int64_t *si = st + kSortMax;
+    if (state) {
+        if (!state->small) return;
+        n_in = (int)state->n_cand;
+    }
+    int np2 = 1;
+    while (np2 < n_in) np2 <<= 1;
+    for (int i = threadIdx.x; i < np2; i += blockDim.x) {
+        st[i] = i < n_in ? ct[i] : INT64_MAX;
+        si[i] = i < n_in ? (ci ? ci[i] : (int64_t)i) : INT64_MAX;
+    }
+    __syncthreads();
+    bitonic_sort_pairs(st, si, np2);
     for (int i = threadIdx.x; i < k; i += blockDim.x) {
         out_idx[i] = first + si[i];
         if (out_time) out_time[i] = st[i];
+    }
+}
+
+// Sampled selection, after the one pass over the array: the compact buffer holds the cn elements
+// between the array's smallest time and the sample's threshold.  One histogram over that range
+// (2048 bins of equal width, a power of two) finds a cut that at least k of them do not exceed;
+// if those candidates fit one sort (the usual case: about k plus one bin's worth), `small` is
+// set and collect + sort finish the selection; otherwise the general kernel below does.
+__global__ void __launch_bounds__(kSelThreads)
+refine_kernel(SelectScratch sc)
+{
+    __shared__ unsigned int sh[kBins];
+    __shared__ u64 partial[kSelThreads];
+    __shared__ bool last;
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    if (!st->use_compact) return;                      // the elements did not fit: `small` stays 0
+    const u64 tmin = st->tmin, range = st->threshold - tmin;
+    const int shift = range >> kRadixBits ? 64 - __clzll((long long)range) - kRadixBits : 0;     // (range >> shift) < 2048
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) sh[i] = 0;
+    __syncthreads();
+    const int64_t n = (int64_t)st->cn;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        atomicAdd(&sh[(unsigned)(((u64)sc.comp_time[i] - tmin) >> shift)], 1u);
+    __syncthreads();
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) if (sh[i]) atomicAdd(&sc.hist[i], (u64)sh[i]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&st->blocks_done, 1ull) == (u64)gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    const PickedBin p = find_bin(st->k - 1, sc.hist, partial);
+    if (threadIdx.x == 0) {
+        // candidates: everything up to the upper edge of the chosen bin, any index
+        st->tprefix = tmin + (((u64)p.bin + 1) << shift) - 1;
+        st->iprefix = ~0ull;
+        st->n_cand = p.before + p.in_bin;
+        st->small = p.before + p.in_bin <= (u64)kSortMax ? 1 : 0;
+        st->blocks_done = 0; st->cursor = 0;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) sc.hist[i] = 0;
+}
+
+// The general selection by one block, for the rare inputs the refined path cannot finish
+// (masses of equal times): a radix select over all time digits, then over the index digits among
+// the elements with the threshold time, on the compact buffer or, if that overflowed, the array
+// itself; then the k winners are sorted.  Slow on long inputs, exact on all.
+__global__ void __launch_bounds__(kSelThreads)
+general_select_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int k, int tb, int ib,
+                      int64_t first, int64_t *out_idx, int64_t *out_time)
+{
+    extern __shared__ __align__(16) unsigned char sm[];
+    int64_t *pt = reinterpret_cast<int64_t *>(sm);          // [kSortMax] winners' times
+    int64_t *pi = pt + kSortMax;                            // [kSortMax] winners' indices
+    u64 *h = reinterpret_cast<u64 *>(pi + kSortMax);        // [kBins]
+    __shared__ u64 partial[kSelThreads];
+    __shared__ PickedBin picked;
+    __shared__ unsigned int n_won;
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    if (st->small) return;
+    const SelSource src = sel_source(st, batch, count, sc);
+    u64 tprefix = 0, tmask = 0, iprefix = 0, imask = 0, rank = (u64)(k - 1);
+    bool skip_index = false;
+    for (int phase = 0; phase < 2; ++phase) {              // 0: time digits, 1: index digits
+        const int bits = phase == 0 ? tb : ib;
+        if (phase == 1 && skip_index) break;
+        for (int shift = ((bits + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
+            const int width = bits - shift < kRadixBits ? bits - shift : kRadixBits;
+            const unsigned dmask = (1u << width) - 1u;
+            for (int i = threadIdx.x; i < kBins; i += blockDim.x) h[i] = 0;
+            __syncthreads();
+            for (int64_t i = threadIdx.x; i < src.n; i += blockDim.x) {
+                const u64 x = (u64)src.t[i];
+                if ((x & tmask) != tprefix) continue;
+                if (phase == 0) { atomicAdd(&h[(unsigned)(x >> shift) & dmask], 1ull); continue; }
+                const u64 id = src.idx ? (u64)src.idx[i] : (u64)i;
+                if ((id & imask) == iprefix) atomicAdd(&h[(unsigned)(id >> shift) & dmask], 1ull);
+            }
+            __syncthreads();
+            const PickedBin p = find_bin(rank, h, partial);
+            if (threadIdx.x == 0) picked = p;
+            __syncthreads();
+            rank -= picked.before;
+            if (phase == 0) {
+                tprefix |= (u64)picked.bin << shift; tmask |= (u64)dmask << shift;
+                // the elements equal to the threshold time are exactly the ones still needed
+                if (shift == 0 && picked.in_bin == rank + 1) skip_index = true;
+            } else {
+                iprefix |= (u64)picked.bin << shift; imask |= (u64)dmask << shift;
+            }
+            __syncthreads();
+        }
+    }
+    if (skip_index) iprefix = ~0ull;
+    if (threadIdx.x == 0) n_won = 0;
+    __syncthreads();
+    for (int64_t i = threadIdx.x; i < src.n; i += blockDim.x) {
+        const u64 x = (u64)src.t[i];
+        const u64 id = src.idx ? (u64)src.idx[i] : (u64)i;
+        if (x < tprefix || (x == tprefix && id <= iprefix)) {
+            const unsigned pos = atomicAdd(&n_won, 1u);
+            if (pos < (unsigned)k) { pt[pos] = (int64_t)x; pi[pos] = (int64_t)id; }
+        }
+    }
+    __syncthreads();
+    int np2 = 1;
+    while (np2 < k) np2 <<= 1;
+    for (int i = k + threadIdx.x; i < np2; i += blockDim.x) { pt[i] = INT64_MAX; pi[i] = INT64_MAX; }
+    __syncthreads();
+    bitonic_sort_pairs(pt, pi, np2);
+    for (int i = threadIdx.x; i < k; i += blockDim.x) {
+        out_idx[i] = first + pi[i];
+        if (out_time) out_time[i] = pt[i];
     }
 }
 
@@ -284,9 +519,12 @@ int bits_for(int64_t v)       // number of bits needed to represent v >= 0
     return b;
 }
 
+// Blocks for a pass over n elements: two elements per thread while that fits eight blocks per SM
+// (short passes are bound by the latency of a thread's loads, not by their number), the
+// blocks striding over the rest.
 int grid_for(int64_t n)
 {
-    int64_t g = (n + kSelThreads * 8 - 1) / (kSelThreads * 8);
+    int64_t g = (n + kSelThreads * 2 - 1) / (kSelThreads * 2);
     if (g < 1) g = 1;
     if (g > 148 * 8) g = 148 * 8;
     return (int)g;
@@ -315,102 +553,127 @@ void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t 
 
 namespace {
 
-// Bits of the times that the radix select looks at, and its first digit.
-struct TimeDigits { int tb, shift0, width0; };
-TimeDigits time_digits(int64_t time_bound)
+// Bits of the times that the radix select looks at.
+int time_bits(int64_t time_bound)
 {
-    TimeDigits d;
     // bits above the bound on any time are zero everywhere: start below them
-    d.tb = bits_for(time_bound) > 0 ? bits_for(time_bound) : 1;
-    d.shift0 = ((d.tb + kRadixBits - 1) / kRadixBits - 1) * kRadixBits;
-    d.width0 = d.tb - d.shift0 < kRadixBits ? d.tb - d.shift0 : kRadixBits;
-    return d;
+    return bits_for(time_bound) > 0 ? bits_for(time_bound) : 1;
 }
 
-// The radix select for more than kSortMax elements.  first_digit_done: the histogram of the first
-// digit has been filled already (by an evaluation), only its bin is still to be picked.
-void select_passes(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k, int64_t time_bound,
-                   const SelectScratch &sc, bool first_digit_done, int64_t *d_indices, int64_t *d_times,
-                   int64_t *launches)
+// Radix passes over all time digits (most significant first) of the current source.
+void time_passes(cudaStream_t s, const int64_t *batch, int64_t count, int64_t n_source, int64_t time_bound,
+                 const SelectScratch &sc, bool compact_after_first, int64_t *launches)
 {
-    const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
-    const int g = grid_for(count);
-    const TimeDigits td = time_digits(time_bound);
+    const int g = grid_for(n_source);
+    const int tb = time_bits(time_bound);
     bool first_pass = true;
-    for (int shift = td.shift0; shift >= 0; shift -= kRadixBits) {
-        const int width = td.tb - shift < kRadixBits ? td.tb - shift : kRadixBits;
-        if (first_pass && first_digit_done) radix_pick_kernel<<<1, kSelThreads, 0, s>>>(sc, shift, width, shift == 0);
-        else radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, sc, shift, width, shift == 0);
+    for (int shift = ((tb + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
+        const int width = tb - shift < kRadixBits ? tb - shift : kRadixBits;
+        radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, sc, shift, width, shift == 0);
         ++*launches;
-        if (first_pass && shift > 0 && sc.comp_cap > 0) {
-            compact_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc, shift);
+        if (compact_after_first && first_pass && shift > 0 && sc.comp_cap > 0) {
+            compact_kernel<<<grid_for(count), kSelThreads, 0, s>>>(batch, count, sc, shift);
             ++*launches;
         }
         first_pass = false;
     }
+}
+
+// Index passes, collection and the final sort of the k winners.
+void finish_passes(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int64_t n_source, int k,
+                   const SelectScratch &sc, int64_t *d_indices, int64_t *d_times, int64_t *launches)
+{
+    const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
+    const int g = grid_for(n_source);
     const int ib = bits_for(count - 1) > 0 ? bits_for(count - 1) : 1;
     for (int shift = ((ib + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
         const int width = ib - shift < kRadixBits ? ib - shift : kRadixBits;
         radix_pass_kernel<true><<<g, kSelThreads, 0, s>>>(batch, count, sc, shift, width, false);
         ++*launches;
     }
-    collect_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc, k);
-    sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, k, k, first, d_indices, d_times);
+    collect_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc, k, 0);
+    sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, k, k, first, d_indices, d_times, nullptr);
     *launches += 2;
 }
 
+constexpr int64_t kSampledMin = (int64_t)1 << 20;     // arrays at least this long are sampled first
+
 }  // namespace
+
+namespace {
+__global__ void add_scalar_kernel(int64_t *word, int64_t value) { if (threadIdx.x == 0 && blockIdx.x == 0) *word += value; }
+}  // namespace
+void launch_add_scalar(cudaStream_t s, int64_t *d_word, int64_t value, int64_t *launches)
+{
+    add_scalar_kernel<<<1, 32, 0, s>>>(d_word, value);
+    ++*launches;
+}
 
 void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
                  int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
                  int64_t *launches)
 {
+    launch_select(s, batch, first, count, k, time_bound, sc, nullptr, d_indices, d_times, launches);
+}
+
+void launch_select(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k, int64_t time_bound,
+                   const SelectScratch &sc, int64_t *d_result, int64_t *d_indices, int64_t *d_times,
+                   int64_t *launches)
+{
     const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
     ensure_dynamic_smem(reinterpret_cast<const void *>(&sort_pairs_kernel), sort_smem);     // per device
-    if (count <= kSortMax) {
-        sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(batch, nullptr, (int)count, k, first, d_indices, d_times);
+    const int idx_bits = bits_for(count - 1) > 0 ? bits_for(count - 1) : 1;
+    const bool packed = bits_for(time_bound) + idx_bits <= 63;
+    const bool sampled = k > 0 && count >= kSampledMin && sc.comp_cap > 0;
+    if (!sampled) {
+        // short arrays (or no compact buffer): the best element and the selection as separate passes
+        if (d_result) launch_argmin(s, batch, count, time_bound, sc, d_result, launches);
+        if (k == 0) return;
+        if (count <= kSortMax) {
+            sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(batch, nullptr, (int)count, k, first, d_indices, d_times, nullptr);
+            ++*launches;
+            return;
+        }
+        sel_init_kernel<<<1, 256, 0, s>>>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, k, 0, nullptr);
         ++*launches;
+        time_passes(s, batch, count, count, time_bound, sc, true, launches);
+        finish_passes(s, batch, first, count, count, k, sc, d_indices, d_times, launches);
         return;
     }
-    sel_init_kernel<<<1, 256, 0, s>>>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, k);
+    // 1. the k-th smallest time of a strided sample: about 2^16 elements, but a stride small enough
+    //    for the expected k * stride elements up to that time to fit the compact buffer four times
+    int64_t stride = count >> 16;
+    if (stride > sc.comp_cap / (4 * (int64_t)k)) stride = sc.comp_cap / (4 * (int64_t)k);
+    if (stride < 64) stride = 64;
+    const int64_t n_sample = (count + stride - 1) / stride;
+    const bool min_here = d_result != nullptr && packed;
+    sel_init_kernel<<<1, 256, 0, s>>>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, k, stride,
+                                      min_here ? sc.key : nullptr);
     ++*launches;
-    select_passes(s, batch, first, count, k, time_bound, sc, false, d_indices, d_times, launches);
-}
-
-FusedSelect begin_fused_select(cudaStream_t s, int64_t count, int k, int64_t time_bound, const SelectScratch &sc,
-                               int64_t *launches)
-{
-    static_assert(kBins == kSelectBins, "the evaluation kernels fill the radix select's histogram");
-    FusedSelect fs{};
-    fs.key = sc.key; fs.hist = sc.hist;
-    fs.idx_bits = bits_for(count - 1) > 0 ? bits_for(count - 1) : 1;
-    const TimeDigits td = time_digits(time_bound);
-    fs.shift = td.shift0; fs.width = td.width0;
-    // folded in when time and position fit one key and the array is too long to be sorted directly
-    fs.enabled = (bits_for(time_bound) + fs.idx_bits <= 63 && count > kSortMax) ? 1 : 0;
-    if (fs.enabled) {
-        cudaMemsetAsync(sc.key, 0xFF, 2 * sizeof(u64), s);
-        sel_init_kernel<<<1, 256, 0, s>>>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, k > 0 ? k : 1);
+    time_passes(s, batch, count, n_sample, time_bound, sc, false, launches);
+    // 2. one pass: minimum of the packed key, elements up to that time into the compact buffer
+    scan_select_kernel<<<grid_for(count), kSelThreads, 0, s>>>(batch, count, sc, idx_bits, min_here ? 1 : 0, 1);
+    ++*launches;
+    if (min_here) {
+        argmin_unpack_kernel<<<1, 32, 0, s>>>(sc.key, idx_bits, 1, d_result);
         ++*launches;
+    } else if (d_result) {
+        launch_argmin(s, batch, count, time_bound, sc, d_result, launches);     // times too wide to pack
     }
-    return fs;
-}
-
-void finish_fused_argmin(cudaStream_t s, const FusedSelect &fs, const SelectScratch &sc, int64_t *d_result,
-                         int64_t *launches)
-{
-    argmin_unpack_kernel<<<1, 32, 0, s>>>(sc.key, fs.idx_bits, 1, d_result);
-    ++*launches;
-}
-
-void finish_fused_topk(cudaStream_t s, const FusedSelect &fs, const int64_t *batch, int64_t first, int64_t count, int k,
-                       int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
-                       int64_t *launches)
-{
-    (void)fs;
-    const size_t sort_smem = (size_t)kSortMax * 2 * sizeof(int64_t);
-    ensure_dynamic_smem(reinterpret_cast<const void *>(&sort_pairs_kernel), sort_smem);     // per device
-    select_passes(s, batch, first, count, k, time_bound, sc, true, d_indices, d_times, launches);
+    // 3. the selection proper on the compact buffer (about k * stride pairs when the sample is
+    //    representative; the grid is sized for that, the kernels stride over whatever there is):
+    //    one histogram over its range of times cuts it down to what one sort takes
+    const int64_t n_expect = (int64_t)k * stride * 4 < count ? (int64_t)k * stride * 4 : count;
+    SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
+    refine_kernel<<<grid_for(n_expect), kSelThreads, 0, s>>>(sc);
+    collect_kernel<<<grid_for(n_expect), kSelThreads, 0, s>>>(batch, count, sc, kSortMax, 1);
+    sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, 0, k, first, d_indices, d_times, st);
+    // ... and the general kernel for what that path cannot finish (it returns at once otherwise)
+    const size_t gen_smem = sort_smem + (size_t)kBins * sizeof(u64);
+    ensure_dynamic_smem(reinterpret_cast<const void *>(&general_select_kernel), gen_smem);
+    general_select_kernel<<<1, kSelThreads, gen_smem, s>>>(batch, count, sc, k, time_bits(time_bound), idx_bits, first,
+                                                          d_indices, d_times);
+    *launches += 4;
 }
 
 }  // namespace distsim

@@ -87,7 +87,7 @@ _lib.distsim_set_space.argtypes = [C.c_void_p, C.POINTER(_Space), C.POINTER(C.c_
 _lib.distsim_decode.argtypes = [C.c_void_p, C.c_int64, C.POINTER(_Candidate)]
 _lib.distsim_eval_strategies.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
 _lib.distsim_eval_select.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int32,
-                                     C.c_void_p, C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+                                     C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 _lib.distsim_argmin.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                 C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 _lib.distsim_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
@@ -220,20 +220,23 @@ def distsim_eval_strategies(ctx: Context, first: int, count: int, d_batch_ns,
 
 
 def distsim_eval_select(ctx: Context, first: int, count: int, d_batch_ns, k: int = 0, d_indices=None,
-                        d_times=None, stream=None):
-    """Evaluation with the best candidate and the k fastest folded in; returns (best index, best
-    batch time).  Synchronises."""
+                        d_times=None, d_best=None, stream=None, to_host: bool = True):
+    """Evaluation with the best candidate and the k fastest in one call.  With ``to_host`` it
+    synchronises and returns (best index, best batch time); without, it is asynchronous, returns
+    None, and ``d_best`` (int64 [2] on the device: batch time, index) receives the best candidate."""
     pb = _dev_ptr(d_batch_ns, "int64", count, "d_batch_ns")
     pi = _dev_ptr(d_indices, "int64", k, "d_indices")
     pt = _dev_ptr(d_times, "int64", k, "d_times")
+    pd = _dev_ptr(d_best, "int64", 2, "d_best")
     bi, bt = C.c_int64(0), C.c_int64(0)
-    rc = _lib.distsim_eval_select(ctx._h, _stream(stream), first, count, pb, k, pi, pt, C.byref(bi), C.byref(bt))
+    rc = _lib.distsim_eval_select(ctx._h, _stream(stream), first, count, pb, k, pi, pt, pd,
+                                  C.byref(bi) if to_host else None, C.byref(bt) if to_host else None)
     if rc == E_TIMEOUT and b"outputs are exact" in _lib.distsim_last_error(ctx._h):
         e = DistsimError(rc, _lib.distsim_last_error(ctx._h).decode())
         e.result = (int(bi.value), int(bt.value))
         raise e
     ctx._check(rc)
-    return int(bi.value), int(bt.value)
+    return (int(bi.value), int(bt.value)) if to_host else None
 
 
 def distsim_argmin(ctx: Context, d_batch_ns, first: int, count: int, stream=None):

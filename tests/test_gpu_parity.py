@@ -680,6 +680,15 @@ def _check_eval_select(E, ctx, first, count, k):
     assert torch.equal(got, want)
     if k:
         assert torch.equal(gi, wi) and torch.equal(gt, wt)
+    # without host outputs: asynchronous, the best candidate goes to device memory
+    got.fill_(-1); gi.fill_(-1); gt.fill_(-1)
+    d_best = dev(2)
+    assert E.distsim_eval_select(ctx, first, count, got, k, gi if k else None, gt if k else None, d_best,
+                                 to_host=False) is None
+    torch.cuda.synchronize()
+    assert torch.equal(got, want) and tuple(d_best.tolist()) == (best[1], best[0])
+    if k:
+        assert torch.equal(gi, wi) and torch.equal(gt, wt)
     return want
 
 
