@@ -170,10 +170,18 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     peaks, peak_kind = measured_peaks()
 
-    w = W.config1(seed=sharding.rank_seed(1, rank))
+    # weak: every rank runs its own search (seed 1 + rank).  shard: the ranks split ONE search
+    # (seed 1) into contiguous candidate ranges, select among their own candidates, exchange only
+    # their short lists of winners (one all-gather of 2 x 1024 words) and emit a slice of the
+    # merged winners each; no other traffic between GPUs.
+    shard = args.mode == "shard"
+    w = W.config1(seed=1 if shard else sharding.rank_seed(1, rank))
     table, space = w.table, w.space
     n_total, cells = W.count_candidates_and_cells(table, space)
     N = table.n_devices
+    my_first, my_count = sharding.shard_range(n_total, rank, world) if shard else (0, n_total)
+    emit_first, emit_n = sharding.shard_range(TOP_K, rank, world) if shard else (0, TOP_K)
+    k_loc = min(TOP_K, my_count)
     ctx = E.Context(local)
     stream = torch.cuda.current_stream()
 
@@ -182,19 +190,33 @@ def run_ours(args):
 
     E.distsim_load_event_table(ctx, table)
     assert E.distsim_set_space(ctx, space) == n_total
-    batch = torch.empty(n_total, dtype=torch.int64, device=dev)
+    d_best = torch.empty(2, dtype=torch.int64, device=dev)                  # (batch time, index) of this rank's best candidate
+    batch = torch.empty(my_count, dtype=torch.int64, device=dev)
     top_i = torch.empty(TOP_K, dtype=torch.int64, device=dev)
     top_t = torch.empty(TOP_K, dtype=torch.int64, device=dev)
-    offsets = torch.empty(TOP_K * N + 1, dtype=torch.int64, device=dev)
-    busy = torch.empty(TOP_K * N, dtype=torch.int64, device=dev)
-    util = torch.empty(TOP_K * N, dtype=torch.float64, device=dev)
-    d_best = torch.empty(2, dtype=torch.int64, device=dev)                  # (batch time, index) of the best candidate
+    merging = shard and world > 1
+    loc_i = torch.full((TOP_K,), torch.iinfo(torch.int64).max, dtype=torch.int64, device=dev) if merging else top_i
+    loc_t = torch.full((TOP_K,), torch.iinfo(torch.int64).max, dtype=torch.int64, device=dev) if merging else top_t
+    offsets = torch.empty(emit_n * N + 1, dtype=torch.int64, device=dev)
+    busy = torch.empty(emit_n * N, dtype=torch.int64, device=dev)
+    util = torch.empty(emit_n * N, dtype=torch.float64, device=dev)
+
+    def search():
+        """Evaluation, best candidate and the 1024 fastest in one asynchronous call; with the
+        search split over ranks, the ranks' lists are gathered and merged on every rank."""
+        E.distsim_eval_select(ctx, my_first, my_count, batch, k_loc, loc_i[:k_loc], loc_t[:k_loc], d_best, to_host=False)
+        if merging:
+            gt, gi = sharding.gather_topk_lists(loc_t, loc_i)
+            E.distsim_merge_topk(ctx, gt, gi, gt.numel(), TOP_K, top_i, top_t)
+
+    def emit(rec, cap):
+        return E.distsim_emit_timelines(ctx, top_i[emit_first:emit_first + emit_n], emit_n, rec, cap, offsets, busy, util)
+
     flush = torch.empty(256 * 2**20, dtype=torch.uint8, device=dev)          # > L2 (126 MB)
 
-    # sizing pass (untimed): how many records the 1024 fastest need
-    E.distsim_eval_strategies(ctx, 0, n_total, batch)
-    E.distsim_topk(ctx, batch, 0, n_total, TOP_K, top_i, top_t)
-    total_records = E.distsim_emit_timelines(ctx, top_i, TOP_K, None, 0)
+    # sizing pass (untimed): how many records this rank's share of the 1024 fastest needs
+    search()
+    total_records = emit(None, 0)
     capacity = total_records + total_records // 8 + 1024
     records = torch.empty(capacity * 5, dtype=torch.int64, device=dev)
 
@@ -202,12 +224,12 @@ def run_ours(args):
         e0, e1, e2, e3 = (ev(), ev(), ev(), ev()) if timers is not None else (None,) * 4
         if timers is not None:
             e0.record(stream)
-        # evaluation, best candidate and the 1024 fastest in one asynchronous call (it records
-        # events around its evaluation and its selection launches itself), then their timelines
-        E.distsim_eval_select(ctx, 0, n_total, batch, TOP_K, top_i, top_t, d_best, to_host=False)
+        # the search (the library records events around its evaluation and its selection
+        # launches itself), then the winners' timelines
+        search()
         if timers is not None:
             e2.record(stream)
-        tot = E.distsim_emit_timelines(ctx, top_i, TOP_K, records, capacity, offsets, busy, util)
+        tot = emit(records, capacity)
         if timers is not None:
             e3.record(stream)
             timers.append((e0, e1, e2, e3))
@@ -241,7 +263,7 @@ def run_ours(args):
         flush.fill_(1)                         # evict L2 between timed iterations
     barrier()
     launches = ctx.launch_count - launches0
-    best = (int(best[1]), int(best[0]))               # (index, batch time) of the last timed step
+    best = (int(top_i[0]), int(top_t[0]))             # (index, batch time): head of the (merged) list of the last timed step
     # keep the clock sampler running through the end-to-end loop as well
     step_ms = [t[0].elapsed_time(t[3]) for t in timers]
     eval_ms = [p[0] for p in phases]
@@ -252,9 +274,9 @@ def run_ours(args):
     # ---- end to end through host buffers ----------------------------------------------------
     h_top_i = torch.empty(TOP_K, dtype=torch.int64).pin_memory()
     h_top_t = torch.empty(TOP_K, dtype=torch.int64).pin_memory()
-    h_off = torch.empty(TOP_K * N + 1, dtype=torch.int64).pin_memory()
-    h_busy = torch.empty(TOP_K * N, dtype=torch.int64).pin_memory()
-    h_util = torch.empty(TOP_K * N, dtype=torch.float64).pin_memory()
+    h_off = torch.empty(emit_n * N + 1, dtype=torch.int64).pin_memory()
+    h_busy = torch.empty(emit_n * N, dtype=torch.int64).pin_memory()
+    h_util = torch.empty(emit_n * N, dtype=torch.float64).pin_memory()
     h_rec = torch.empty(capacity * 5, dtype=torch.int64).pin_memory()
     h2d = sum(a.nbytes for a in (table.class_mp, table.class_b, table.fwd_ns, table.bwd_ns,
                                  table.layer_is_expert, table.grad_bytes, space.m_list)) + 128
@@ -262,8 +284,8 @@ def run_ours(args):
     def e2e_step():
         E.distsim_load_event_table(ctx, table)                    # host -> device
         E.distsim_set_space(ctx, space)
-        best = E.distsim_eval_select(ctx, 0, n_total, batch, TOP_K, top_i, top_t)      # best -> host
-        tot = E.distsim_emit_timelines(ctx, top_i, TOP_K, records, capacity, offsets, busy, util)
+        search()
+        tot = emit(records, capacity)
         h_top_i.copy_(top_i, non_blocking=True); h_top_t.copy_(top_t, non_blocking=True)
         h_off.copy_(offsets, non_blocking=True); h_busy.copy_(busy, non_blocking=True)
         h_util.copy_(util, non_blocking=True)
@@ -275,8 +297,8 @@ def run_ours(args):
         """As e2e_step, but the multi-GB record buffer stays on the device."""
         E.distsim_load_event_table(ctx, table)
         E.distsim_set_space(ctx, space)
-        E.distsim_eval_select(ctx, 0, n_total, batch, TOP_K, top_i, top_t)
-        E.distsim_emit_timelines(ctx, top_i, TOP_K, records, capacity, offsets, busy, util)
+        search()
+        emit(records, capacity)
         h_top_i.copy_(top_i, non_blocking=True); h_top_t.copy_(top_t, non_blocking=True)
         h_off.copy_(offsets, non_blocking=True); h_busy.copy_(busy, non_blocking=True)
         h_util.copy_(util, non_blocking=True)
@@ -305,7 +327,9 @@ def run_ours(args):
     total_ms_max = sharding.max_over_ranks(total_ms, device=dev)
     e2e_s_max = sharding.max_over_ranks(sum(e2e_times) / len(e2e_times), device=dev)
     ms_per_step = total_ms_max / args.steps
-    value = world * n_total / (ms_per_step * 1e-3)
+    job_candidates = n_total if shard else world * n_total           # candidates the whole job evaluates per step
+    job_cells = cells if shard else world * cells
+    value = job_candidates / (ms_per_step * 1e-3)
 
     if rank != 0:
         if world > 1:
@@ -332,6 +356,10 @@ def run_ours(args):
     sm_mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
     cells_all, cells_32 = E.distsim_testing_space_cells(ctx)
     assert cells_all == cells
+    if merging:
+        # this rank evaluated its slice only: its share of the cells, taken as the share of the
+        # candidates (rank 0's slice holds the short pipelines, so the fraction below is indicative)
+        cells, cells_32 = int(cells * my_count / n_total), int(cells_32 * my_count / n_total)
     eval_s = statistics.mean(eval_ms) * 1e-3
     alg_ops = cells_32 * INT_OPS_PER_CELL_32 + (cells - cells_32) * INT_OPS_PER_CELL_64
     achieved_gops = alg_ops / eval_s / 1e9
@@ -361,7 +389,7 @@ def run_ours(args):
                                                  (SM_COUNT * SCHEDULERS_PER_SM * LANES / 2 * sm_mhz * 1e-3),
                 "compare_select_peak_Ginstr_per_s": cmpsel_peak,
                 "frac_of_cell_rate_floor": cell_floor_s / eval_s}
-    emit_bytes = tot * RECORD_BYTES + TOP_K * N * 24 + 8
+    emit_bytes = tot * RECORD_BYTES + emit_n * N * 24 + 8
     emit_gbs = emit_bytes / (statistics.mean(emit_ms) * 1e-3) / 1e9
     roofline_emit = {"bound": "hbm", "kernel": "emit_items_kernel (+plan, scan, devices, buckets)",
                      "achieved": emit_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -373,23 +401,26 @@ def run_ours(args):
     line = {
         "metric": "strategy_candidates_per_sec", "value": value, "unit": "candidates/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "higher_is_better": True, "scaling": "strong" if shard else "weak", "vs_baseline": None,
         "dtype": "int64",
         "dtype_note": "int64 nanoseconds at the boundary; exact uint32 arithmetic inside entries whose time bound is below 2^32",
         "data": "synthetic",
-        "config": {"workload": w.name, "candidates": n_total, "recurrence_cells": cells, "devices": N,
+        "config": {"workload": w.name, "candidates": n_total, "recurrence_cells": job_cells // (1 if shard else world), "devices": N,
                    "layers": table.n_layers, "top_k_emitted": TOP_K, "records_emitted": tot,
-                   "l2": "256 MB flush between timed iterations", "seed": "1 + rank"},
-        "events_per_sec": world * cells / (ms_per_step * 1e-3),
+                   "l2": "256 MB flush between timed iterations",
+                   "seed": "1 on every rank" if shard else "1 + rank",
+                   "mode": "one search split over the ranks by candidate range; 2 x 1024-word lists all-gathered and merged"
+                           if shard else "one search per rank"},
+        "events_per_sec": job_cells / (ms_per_step * 1e-3),
         "phase_ms": {"eval": statistics.mean(eval_ms), "argmin_topk": statistics.mean(sel_ms),
                      "emit": statistics.mean(emit_ms)},
-        "eval_only": {"candidates_per_sec": n_total / eval_s, "events_per_sec": cells / eval_s},
+        "eval_only": {"candidates_per_sec": my_count / eval_s, "events_per_sec": cells / eval_s},
         "best": {"index": best[0], "batch_ns": best[1]},
         "roofline": roofline, "roofline_emit": roofline_emit,
-        "e2e": {"value": world * n_total / e2e_s_max, "unit": "candidates/s", "h2d_bytes_per_step": h2d,
+        "e2e": {"value": job_candidates / e2e_s_max, "unit": "candidates/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s_max * 1e3,
                 "note": "includes downloading every emitted record over PCIe",
-                "records_left_on_device": {"value": world * n_total / results_only_s, "unit": "candidates/s",
+                "records_left_on_device": {"value": job_candidates / results_only_s, "unit": "candidates/s",
                                            "ms_per_step": results_only_s * 1e3}},
         "gpu_launches": launches, "clocks": clocks,
     }
@@ -586,6 +617,8 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--mode", choices=["weak", "shard"], default="weak",
+                    help="N > 1: weak = one search per rank; shard = one search split over the ranks")
     ap.add_argument("--no-workloads", action="store_true", help="skip the per-workload summary")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--profile-case", default=None, help="eval0 | eval1 | eval1m1 | eval1m128 | eval2 | eval2pp64 | eval3 | emit1 | emit4 | emit4x128: small run for ncu")

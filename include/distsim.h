@@ -222,6 +222,17 @@ int distsim_argmin(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, in
 int distsim_topk(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int64_t first,
                  int64_t count, int32_t k, int64_t *d_indices, int64_t *d_times);
 
+/*
+ * The k smallest of n given (batch time, candidate index) pairs, ascending by (time, index):
+ * the merge step of a search whose candidate range was split over several GPUs (Sec. 6: the
+ * candidates are independent, so every GPU selects among its own and only these short lists
+ * are exchanged).  d_times_in, d_indices_in [n]: the gathered lists, times and indices >= 0;
+ * d_indices [k] out, d_times [k] out (nullable).  Requires 1 <= k <= min(n, 4096).
+ * Asynchronous on `stream`.
+ */
+int distsim_merge_topk(distsim_ctx *ctx, void *stream, const int64_t *d_times_in, const int64_t *d_indices_in,
+                       int64_t n, int32_t k, int64_t *d_indices, int64_t *d_times);
+
 /* One timeline record: event `kind` of `layer` for micro-batch `microbatch`
  * occupying [start_ns, end_ns) on its device.  For transfers, `layer` is the
  * stage's boundary layer; for gradient buckets it is the bucket number and

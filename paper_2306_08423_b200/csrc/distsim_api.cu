@@ -602,6 +602,19 @@ int distsim_topk(distsim_ctx *ctx, void *stream, const int64_t *d_batch_ns, int6
     return DISTSIM_OK;
 }
 
+int distsim_merge_topk(distsim_ctx *ctx, void *stream, const int64_t *d_times_in, const int64_t *d_indices_in,
+                       int64_t n, int32_t k, int64_t *d_indices, int64_t *d_times)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!d_times_in || !d_indices_in || !d_indices) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (k < 1 || k > 4096 || k > n) return fail(ctx, DISTSIM_E_ARG, "k must be in [1, min(n, 4096)]");
+    if (int rc = set_device(ctx)) return rc;
+    launch_merge_pairs(static_cast<cudaStream_t>(stream), d_times_in, d_indices_in, n, k, ctx->select_scratch(),
+                       d_indices, d_times, &ctx->launches);
+    CU(cudaGetLastError(), "merge launch");
+    return DISTSIM_OK;
+}
+
 int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indices, int32_t n,
                            distsim_record *d_records, int64_t capacity_records, int64_t *d_offsets,
                            int64_t *d_busy_ns, double *d_util, int64_t *h_total_records)

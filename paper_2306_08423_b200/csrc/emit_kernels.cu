@@ -13,8 +13,7 @@
 //                        mp*dp replicas hold identical lists, so the image is computed once and
 //                        written to each replica of the chunk by one bulk asynchronous copy
 //                        (cp.async.bulk shared -> global) issued by one lane per replica.
-//                        The blocks of the same launch beyond the item tiles write the
-//                        gradient-bucket records of every stage (emit_buckets_block).
+//   emit_buckets_kernel  gradient-bucket records of every stage.
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
 
@@ -275,7 +274,7 @@ __device__ __forceinline__ void item_at(int sched, int pp, int m, int d, int s, 
 // inside a layer a closed form (a thread per bucket).  The records of up to `run` buckets
 // are assembled in shared memory once and sent to every replica by a bulk copy, as in
 // emit_items_kernel.
-// The blocks of the record kernel beyond its item tiles run this (tile: the block's number among them).
+// The work of one block (tile: its number inside the selection).
 __device__ __forceinline__ void emit_buckets_block(const DeviceView &v, const EmitPlan &p, int tile,
                                                    int64_t *__restrict__ out, int run /* buckets per image */,
                                                    int64_t *dyn_s)
@@ -375,18 +374,22 @@ __device__ __forceinline__ void emit_buckets_block(const DeviceView &v, const Em
     }
 }
 
+// Gradient-bucket records: a launch of its own with small blocks (measured: as extra blocks of
+// the item launch they take the places of item blocks and cost more than they save).
+constexpr int kBucketThreads = 128;
+__global__ void __launch_bounds__(kBucketThreads)
+emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *__restrict__ out, int run /* buckets per image */)
+{
+    extern __shared__ __align__(16) int64_t dyn_b[];
+    emit_buckets_block(v, plans[blockIdx.y], (int)blockIdx.x, out, run, dyn_b);
+}
+
 __global__ void __launch_bounds__(kItemThreads)
 emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_t *__restrict__ op_start,
                   int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */,
-                  int cap /* words of one image: even, at least the longest run of any selection */,
-                  int item_tiles /* blocks (per selection) beyond these write gradient-bucket records */,
-                  int bucket_run /* buckets per image of those blocks */)
+                  int cap /* words of one image: even, at least the longest run of any selection */)
 {
     extern __shared__ __align__(16) int64_t dyn_s[];
-    if ((int)blockIdx.x >= item_tiles) {
-        emit_buckets_block(v, plans[blockIdx.y], (int)blockIdx.x - item_tiles, out, bucket_run, dyn_s);
-        return;
-    }
     int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
     int64_t *img_b = dyn_s + cap;                       // the same word at img_b[x + 1]
     int64_t *tmpl = dyn_s + 2 * cap + 2;                // [rf*5] forward, then [rb*5] backward
@@ -606,21 +609,20 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
     if (n == 0 || t.item_tiles == 0) return;
     // two images of the run, then the forward and backward item templates of the widest stage
     const int cap = (int)((t.run_words + 1) & ~(int64_t)1);
-    size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
-    // the blocks beyond the item tiles write the gradient-bucket records of a (stage, replica chunk):
-    // an odd number of buckets per image keeps both images 16-byte aligned
-    int run = 0, bucket_tiles = 0;
-    if (t.bucket_tiles > 0 && t.bucket_recs > 0) {
-        run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun) | 1;
-        bucket_tiles = (int)t.bucket_tiles;
-        const size_t bsmem = (size_t)(2 * (run * 5 + 1) + 2 * (DISTSIM_MAX_LAYERS + 1)) * sizeof(int64_t);
-        if (bsmem > smem) smem = bsmem;
-    }
+    const size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
     ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_items_kernel), smem);
     int64_t *out = reinterpret_cast<int64_t *>(records);
-    emit_items_kernel<<<dim3((unsigned)(t.item_tiles + bucket_tiles), (unsigned)n), kItemThreads, smem, s>>>(
-        v, plans, op_start, op_words_per_cand, out, cap, (int)t.item_tiles, run);
+    emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
+        v, plans, op_start, op_words_per_cand, out, cap);
     ++*launches;
+    if (t.bucket_tiles > 0 && t.bucket_recs > 0) {
+        // an odd number of buckets per image keeps both images 16-byte aligned
+        const int run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun) | 1;
+        const size_t bsmem = (size_t)(2 * (run * 5 + 1) + 2 * (DISTSIM_MAX_LAYERS + 1)) * sizeof(int64_t);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_buckets_kernel), bsmem);
+        emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, s>>>(v, plans, out, run);
+        ++*launches;
+    }
 }
 
 }  // namespace distsim

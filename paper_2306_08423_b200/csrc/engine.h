@@ -212,6 +212,9 @@ void launch_argmin(cudaStream_t s, const int64_t *batch, int64_t count, int64_t 
 void launch_select(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k, int64_t time_bound,
                    const SelectScratch &sc, int64_t *d_result, int64_t *d_indices, int64_t *d_times,
                    int64_t *launches);
+// The k smallest of n given (time, index) pairs, ascending (merging the lists of several ranks).
+void launch_merge_pairs(cudaStream_t s, const int64_t *times, const int64_t *indices, int64_t n, int k,
+                        const SelectScratch &sc, int64_t *d_indices, int64_t *d_times, int64_t *launches);
 void launch_add_scalar(cudaStream_t s, int64_t *d_word, int64_t value, int64_t *launches);    // *d_word += value
 // time_bound: an upper bound on every element of `batch` (INT64_MAX if unknown).
 void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,

@@ -609,6 +609,28 @@ void launch_add_scalar(cudaStream_t s, int64_t *d_word, int64_t value, int64_t *
     ++*launches;
 }
 
+namespace {
+__global__ void merge_init_kernel(SelState *st, int64_t n)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) { SelState z{}; z.use_compact = 1; z.cn = (u64)n; *st = z; }
+}
+}  // namespace
+
+void launch_merge_pairs(cudaStream_t s, const int64_t *times, const int64_t *indices, int64_t n, int k,
+                        const SelectScratch &sc, int64_t *d_indices, int64_t *d_times, int64_t *launches)
+{
+    // the general selection kernel, reading the given pairs in the place of the compact buffer
+    SelectScratch src = sc;
+    src.comp_time = const_cast<int64_t *>(times);
+    src.comp_idx = const_cast<int64_t *>(indices);
+    src.comp_cap = n;
+    merge_init_kernel<<<1, 32, 0, s>>>(reinterpret_cast<SelState *>(sc.sel_state), n);
+    const size_t gen_smem = (size_t)kSortMax * 2 * sizeof(int64_t) + (size_t)kBins * sizeof(u64);
+    ensure_dynamic_smem(reinterpret_cast<const void *>(&general_select_kernel), gen_smem);
+    general_select_kernel<<<1, kSelThreads, gen_smem, s>>>(nullptr, n, src, k, 63, 63, 0, d_indices, d_times);
+    *launches += 2;
+}
+
 void launch_topk(cudaStream_t s, const int64_t *batch, int64_t first, int64_t count, int k,
                  int64_t time_bound, const SelectScratch &sc, int64_t *d_indices, int64_t *d_times,
                  int64_t *launches)

@@ -23,6 +23,7 @@ OK, E_ARG, E_STATE, E_RANGE, E_CAPACITY, E_OVERFLOW, E_CUDA, E_TIMEOUT, E_UNSUPP
 EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error",
            "distsim_load_event_table", "distsim_set_space", "distsim_decode",
            "distsim_eval_strategies", "distsim_eval_select", "distsim_argmin", "distsim_topk",
+           "distsim_merge_topk",
            "distsim_emit_timelines", "distsim_checksum_timelines", "distsim_search_host",
            "distsim_topk_static")
 # hooks of include/distsim_testing.h (test-suite and benchmark accounting; not the stable ABI)
@@ -92,6 +93,8 @@ _lib.distsim_argmin.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C
                                 C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 _lib.distsim_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
                               C.c_void_p, C.c_void_p]
+_lib.distsim_merge_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32,
+                                    C.c_void_p, C.c_void_p]
 _lib.distsim_emit_timelines.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                         C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.POINTER(C.c_int64)]
@@ -257,6 +260,16 @@ def distsim_topk(ctx: Context, d_batch_ns, first: int, count: int, k: int, d_ind
     pi = _dev_ptr(d_indices, "int64", k, "d_indices")
     pt = _dev_ptr(d_times, "int64", k, "d_times")
     ctx._check(_lib.distsim_topk(ctx._h, _stream(stream), pb, first, count, k, pi, pt))
+
+
+def distsim_merge_topk(ctx: Context, d_times_in, d_indices_in, n: int, k: int, d_indices, d_times=None,
+                       stream=None) -> None:
+    """The k smallest of n given (time, index) pairs, ascending: merges the lists of several ranks."""
+    pt = _dev_ptr(d_times_in, "int64", n, "d_times_in")
+    pi = _dev_ptr(d_indices_in, "int64", n, "d_indices_in")
+    po = _dev_ptr(d_indices, "int64", k, "d_indices")
+    pq = _dev_ptr(d_times, "int64", k, "d_times")
+    ctx._check(_lib.distsim_merge_topk(ctx._h, _stream(stream), pt, pi, n, k, po, pq))
 
 
 def distsim_emit_timelines(ctx: Context, d_indices, n: int, d_records, capacity_records: int,

@@ -40,6 +40,24 @@ def merge_argmin(best_index: int, best_batch_ns: int, group=None):
     return i, t
 
 
+def gather_topk_lists(local_times, local_indices, group=None):
+    """Every rank's (times, indices) top-k list, concatenated in rank order on every rank.  The
+    lists are torch tensors of equal length on all ranks (CPU tensors under gloo, device tensors
+    under NCCL); a rank with fewer than k candidates pads with (INT64_MAX, INT64_MAX) pairs.
+    The k smallest of the result (smallest time, ties to the smallest index) are the global
+    top-k: every global winner is a winner of its own rank's slice."""
+    import torch
+    import torch.distributed as dist
+    if not dist.is_available() or not dist.is_initialized():
+        return local_times, local_indices
+    world = dist.get_world_size(group)
+    pair = torch.stack([local_times, local_indices])                 # [2, k]
+    out = [torch.empty_like(pair) for _ in range(world)]
+    dist.all_gather(out, pair, group=group)
+    both = torch.cat(out, dim=1)
+    return both[0].contiguous(), both[1].contiguous()
+
+
 def max_over_ranks(value: float, device=None, group=None) -> float:
     """Largest value over the ranks (used for device-timed durations)."""
     import torch

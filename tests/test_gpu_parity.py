@@ -727,6 +727,33 @@ def test_eval_select_matches_separate_calls(E, ctx):
     _check_eval_select(E, ctx, 0, n, 500)
 
 
+def test_merged_rank_lists_equal_the_global_topk(E, ctx):
+    """One search split over 1, 2, 3 and 8 slices (as sharding.shard_range gives them to ranks):
+    every slice evaluated and selected on its own, the slices' lists merged by distsim_merge_topk,
+    against the selection over the whole range."""
+    from paper_2306_08423_b200 import sharding
+    for cfg, k in ((3, 1024), (0, 7), (2, 300)):
+        w = W.CONFIGS[cfg]()
+        n = load(E, ctx, w)
+        full, wi, wt = dev(n), dev(k), dev(k)
+        best = E.distsim_eval_select(ctx, 0, n, full, k, wi, wt)
+        for world in (1, 2, 3, 8):
+            lists_t, lists_i, bests = [], [], []
+            for rank in range(world):
+                first, count = sharding.shard_range(n, rank, world)
+                kk = min(k, count)
+                part, li, lt = dev(count), dev(k), dev(k)
+                li.fill_(torch.iinfo(torch.int64).max); lt.fill_(torch.iinfo(torch.int64).max)     # padding of short slices
+                bests.append(E.distsim_eval_select(ctx, first, count, part, kk, li[:kk], lt[:kk]))
+                lists_t.append(lt); lists_i.append(li)
+            gt, gi = torch.cat(lists_t), torch.cat(lists_i)
+            mi, mt = dev(k), dev(k)
+            E.distsim_merge_topk(ctx, gt, gi, gt.numel(), k, mi, mt)
+            torch.cuda.synchronize()
+            assert torch.equal(mi, wi) and torch.equal(mt, wt), (cfg, world)
+            assert min((t, i) for i, t in bests) == (best[1], best[0])
+
+
 def test_two_pass_argmin_for_wide_times(E, ctx):
     # times near 2^55 with a large count cannot be packed with the index into 64 bits
     w = W.random_small(3, lo=2**44, hi=2**45, partition_mode=W.PARTITION_ALL, n_layers=12, pp_max=4,

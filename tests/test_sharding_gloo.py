@@ -37,11 +37,20 @@ def _worker(rank, world, port, out):
         n = oracle.count(w.table, w.space)
         first, count = sharding.shard_range(n, rank, world)
         batch, _ = oracle.eval_indices(w.table, w.space, np.arange(first, first + count))
-        k = int(np.lexsort((np.arange(count), batch))[0])
+        local_order = np.lexsort((np.arange(count), batch))
+        k = int(local_order[0])
         best = sharding.merge_argmin(first + k, int(batch[k]))
+        # the ranks' lists of their 10 fastest, gathered; their 10 smallest are the global 10 fastest
+        import torch
+        kk = 10
+        lt = torch.from_numpy(batch[local_order[:kk]].copy())
+        li = torch.from_numpy((first + local_order[:kk]).astype(np.int64))
+        gt, gi = sharding.gather_topk_lists(lt, li)
+        sel = np.lexsort((gi.numpy(), gt.numpy()))[:kk]
+        merged = (gi.numpy()[sel].tolist(), gt.numpy()[sel].tolist())
         slowest = sharding.max_over_ranks(float(rank + 1))
         empty = sharding.merge_argmin(-1 if rank else 5, 0 if rank else 42)   # one rank has nothing
-        out.put((rank, best, slowest, empty))
+        out.put((rank, best, slowest, empty, merged))
     finally:
         dist.destroy_process_group()
 
@@ -63,7 +72,9 @@ def test_two_ranks_merge_their_winners():
     w = W.config0()
     batch, _ = oracle.eval_indices(w.table, w.space, np.arange(88))
     want = int(np.lexsort((np.arange(88), batch))[0])
-    for rank, best, slowest, empty in results:
+    order = np.lexsort((np.arange(88), batch))[:10]
+    for rank, best, slowest, empty, merged in results:
+        assert merged == (order.tolist(), batch[order].tolist())
         assert best == (want, int(batch[want]))
         assert slowest == 2.0
         assert empty == (5, 42)
