@@ -574,7 +574,7 @@ def profile_case(name):
         if name == "eval2pp64":
             # the first pp = 64 row (mp = 1): 256 micro-batch counts x 2 schedules
             off = 0
-            for mp, pp, dp, ms, parts, n_sched in W.space_shape(w.table, w.space):
+            for mp, pp, dp, ms, parts, n_sched, _v in W.space_shape(w.table, w.space):
                 if (mp, pp) == (1, 64):
                     first, count = off, len(ms) * parts * n_sched
                 off += len(ms) * parts * n_sched
@@ -582,7 +582,7 @@ def profile_case(name):
             # whole entries of the (mp = 1, pp = 16) row, 980 628 candidates each:
             # eval1 m = 16 and 32, eval1m128 m = 128
             off = 0
-            for mp, pp, dp, ms, parts, n_sched in W.space_shape(w.table, w.space):
+            for mp, pp, dp, ms, parts, n_sched, _v in W.space_shape(w.table, w.space):
                 if (mp, pp) == (1, 16):
                     e0, ne = (4, 2) if name == "eval1" else (ms.index(128 if name == "eval1m128" else 1), 1)
                     first, count = off + e0 * parts * n_sched, ne * parts * n_sched

@@ -91,7 +91,9 @@ typedef struct {
     int32_t m_rule;                       /* 0: m divides Bp; 1: any m <= Bp      */
     int32_t partition_mode;               /* 0: balanced; 1: all compositions     */
     int32_t sched_mask;                   /* bit 0: GPipe, bit 1: 1F1B (Dapple),
-                                             bit 2: 1F1B without gradient synchronisation */
+                                             bit 2: 1F1B without gradient synchronisation,
+                                             bit 3: interleaved 1F1B with v = 2, 4, .. v_max chunks */
+    int32_t v_max;                        /* largest number of model chunks per device (bit 3)    */
 } orc_space;
 
 typedef struct {
@@ -222,6 +224,11 @@ static int64_t beta_of(const orc_table *T, int loc) { return loc ? T->beta_inter
 /*   m ascending over the valid entries of m_list;                             */
 /*   stage partition in lexicographic order of (c_1..c_{pp-1});                */
 /*   schedule: GPipe, then 1F1B, then asynchronous 1F1B.                       */
+/* With bit 3 of sched_mask every (mp, pp) with pp >= 2 is followed, for       */
+/* v = 2, 4, .. <= v_max with pp*v <= min(64, L), by the interleaved 1F1B       */
+/* candidates of v chunks per device: m ascending over the valid entries that  */
+/* are multiples of pp, then the partition of the L layers into pp*v virtual    */
+/* stages (balanced, or every composition in lexicographic order).             */
 /* The paper's own grid (Sec. 6) walks mp and pp over powers of two and takes  */
 /* dp = GPUs/mp/pp, dropping the invalid combinations.                         */
 
@@ -276,6 +283,28 @@ static int64_t walk_space(const orc_table *T, const orc_space *S, orc_visit_fn v
                         ++index;
                     }
                 } while (S->partition_mode == 1 && next_partition(x.bounds, (int)pp, L));
+            }
+            /* interleaved 1F1B: candidates with v chunks per device, P = pp * v virtual stages */
+            if (!(S->sched_mask & 8) || pp < 2) continue;
+            for (int64_t v = 2; v <= S->v_max && pp * v <= ORC_MAX_PP && pp * v <= L; v *= 2) {
+                const int P = (int)(pp * v);
+                for (int mi = 0; mi < S->n_m; ++mi) {
+                    int64_t m = S->m_list[mi];
+                    if (!valid_m(S, Bp, m) || m % pp != 0) continue;
+                    orc_candidate x;
+                    memset(&x, 0, sizeof x);
+                    x.mp = (int32_t)mp; x.pp = (int32_t)pp; x.dp = (int32_t)dp; x.m = (int32_t)m;
+                    x.sched = 3; x.v = (int32_t)v;
+                    x.bounds[0] = 0; x.bounds[P] = L;
+                    if (S->partition_mode == 0)
+                        for (int j = 1; j < P; ++j) x.bounds[j] = (int32_t)((int64_t)j * L / P);
+                    else
+                        for (int j = 1; j < P; ++j) x.bounds[j] = j;
+                    do {
+                        if (visit && visit(ctx, index, &x)) return index + 1;
+                        ++index;
+                    } while (S->partition_mode == 1 && next_partition(x.bounds, P, L));
+                }
             }
         }
     return index;

@@ -46,7 +46,7 @@ class _Table(C.Structure):
 class _Space(C.Structure):
     _fields_ = [("mp_max", C.c_int32), ("pp_max", C.c_int32), ("n_m", C.c_int32),
                 ("m_list", C.c_void_p), ("m_rule", C.c_int32), ("partition_mode", C.c_int32),
-                ("sched_mask", C.c_int32)]
+                ("sched_mask", C.c_int32), ("v_max", C.c_int32)]
 
 
 class _Cand(C.Structure):
@@ -136,7 +136,7 @@ def _table(t):
 def _space(sp):
     ml = np.ascontiguousarray(sp.m_list, np.int32)
     return _Space(sp.mp_max, sp.pp_max, ml.shape[0], _ptr(ml), sp.m_rule, sp.partition_mode,
-                  sp.sched_mask), ml
+                  sp.sched_mask, int(getattr(sp, "v_max", 0))), ml
 
 
 def ring_allreduce_ns(n, nbytes, alpha, beta):
@@ -170,7 +170,8 @@ def enumerate_at(table, space, indices) -> list:
     e = _load().orc_enumerate_at(C.byref(t), C.byref(s), _ptr(idx), C.c_int64(idx.shape[0]), out)
     if e:
         raise OracleError(e)
-    return [Candidate(c.mp, c.pp, c.dp, c.m, c.sched, tuple(c.bounds[: c.pp + 1]))
+    return [Candidate(c.mp, c.pp, c.dp, c.m, c.sched, tuple(c.bounds[: c.pp * (c.v if c.sched == 3 else 1) + 1]),
+                      c.v if c.sched == 3 else 1)
             for c in out[: idx.shape[0]]]
 
 

@@ -61,7 +61,9 @@ class SearchSpace:
     m_list: np.ndarray                      # int32, ascending
     m_rule: int = M_RULE_DIVIDES
     partition_mode: int = PARTITION_BALANCED
-    sched_mask: int = 3                     # bit 0 GPipe, bit 1 1F1B, bit 2 asynchronous 1F1B
+    sched_mask: int = 3                     # bit 0 GPipe, bit 1 1F1B, bit 2 asynchronous 1F1B,
+                                            # bit 3 interleaved 1F1B with v = 2, 4, .. v_max chunks per device
+    v_max: int = 0
 
     def __post_init__(self):
         self.m_list = np.ascontiguousarray(self.m_list, dtype=np.int32)
@@ -152,9 +154,13 @@ def event_classes(n_devices: int, global_batch: int, n_layers: int, space: Searc
 
 def space_shape(table, space):
     """Rows of the search space for reporting: a list of (mp, pp, dp, [valid m], partitions,
-    schedules).  Pure counting; candidates = sum(len(ms) * partitions * schedules)."""
+    schedules, v) in canonical order; v = 1 for the plain schedules, the number of model chunks
+    per device for a row of interleaved candidates (which has one schedule and partitions the
+    layers into pp * v virtual stages).  Pure counting; candidates = sum(len(ms) * partitions *
+    schedules)."""
     rows = []
     n_sched = bin(space.sched_mask & 7).count("1")
+    v_max = int(getattr(space, "v_max", 0)) if space.sched_mask & 8 else 0
     for mp in _pow2_upto(space.mp_max):
         for pp in _pow2_upto(min(space.pp_max, table.n_layers)):
             if table.n_devices % (mp * pp):
@@ -165,20 +171,29 @@ def space_shape(table, space):
             bp = table.global_batch // dp
             ms = [m for m in space.m_list.tolist()
                   if 1 <= m <= bp and (space.m_rule == M_RULE_CEIL or bp % m == 0)]
-            if not ms:
+            if ms and n_sched:
+                parts = 1 if space.partition_mode == PARTITION_BALANCED else math.comb(table.n_layers - 1, pp - 1)
+                rows.append((mp, pp, dp, ms, parts, n_sched, 1))
+            if pp < 2:
                 continue
-            parts = 1 if space.partition_mode == PARTITION_BALANCED else math.comb(table.n_layers - 1, pp - 1)
-            rows.append((mp, pp, dp, ms, parts, n_sched))
+            for v in _pow2_upto(v_max):
+                if v < 2 or pp * v > min(64, table.n_layers):
+                    continue
+                mv = [m for m in ms if m % pp == 0]
+                if not mv:
+                    continue
+                parts = 1 if space.partition_mode == PARTITION_BALANCED else math.comb(table.n_layers - 1, pp * v - 1)
+                rows.append((mp, pp, dp, mv, parts, 1, v))
     return rows
 
 
 def count_candidates_and_cells(table, space):
-    """(candidates, recurrence cells) of a space; a candidate has 2 * m * pp cells (one per
-    schedule item: forward and backward of every micro-batch on every stage)."""
+    """(candidates, recurrence cells) of a space; a candidate has 2 * m * pp * v cells (one per
+    schedule item: forward and backward of every micro-batch on every (virtual) stage)."""
     cands = cells = 0
-    for mp, pp, dp, ms, parts, n_sched in space_shape(table, space):
+    for mp, pp, dp, ms, parts, n_sched, v in space_shape(table, space):
         cands += len(ms) * parts * n_sched
-        cells += sum(2 * m * pp for m in ms) * parts * n_sched
+        cells += sum(2 * m * pp * v for m in ms) * parts * n_sched
     return cands, cells
 
 
@@ -304,11 +319,11 @@ CONFIGS = {0: config0, 1: config1, 2: config2, 3: config3, 4: config4}
 def random_small(seed: int, *, n_devices=8, gpus_per_node=4, n_layers=6, global_batch=16,
                  seq=64, hidden=32, mp_max=4, pp_max=4, m_list=(1, 2, 3, 4, 8),
                  m_rule=M_RULE_CEIL, partition_mode=PARTITION_ALL, moe=True,
-                 dp_bucket_bytes=3000, dp_overlap=1, lo=50, hi=5000, sched_mask=3) -> Workload:
+                 dp_bucket_bytes=3000, dp_overlap=1, lo=50, hi=5000, sched_mask=3, v_max=0) -> Workload:
     """Small irregular workload for element-by-element parity tests."""
     rng = SplitMix64(seed)
     space = SearchSpace(mp_max=mp_max, pp_max=pp_max, m_list=list(m_list), m_rule=m_rule,
-                        partition_mode=partition_mode, sched_mask=sched_mask)
+                        partition_mode=partition_mode, sched_mask=sched_mask, v_max=v_max)
     f1 = [rng.randint(lo, hi) for _ in range(n_layers)]
     u = [rng.randint(0, hi // 4) for _ in range(n_layers)]
     expert = np.array([(rng.next() & 1) if moe else 0 for _ in range(n_layers)], dtype=np.uint8)

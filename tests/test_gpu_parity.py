@@ -380,7 +380,7 @@ def stratified_indices(table, space, per_cell, seed):
     every row."""
     rng = np.random.default_rng(seed)
     out, off = [], 0
-    for mp, pp, dp, ms, parts, n_sched in W.space_shape(table, space):
+    for mp, pp, dp, ms, parts, n_sched, _v in W.space_shape(table, space):
         for e in range(len(ms)):
             if parts <= per_cell:
                 p = np.arange(parts, dtype=np.int64)

@@ -645,6 +645,47 @@ def test_canonical_order_against_python_loops():
         assert [(c.mp, c.pp, c.dp, c.m, c.sched, c.bounds) for c in got] == expect
 
 
+def test_canonical_order_with_interleaved_rows():
+    # every (mp, pp) is followed by its interleaved candidates: v ascending over powers of two, m
+    # among the multiples of pp, partitions of the layers into pp * v virtual stages in
+    # lexicographic order
+    for mask, mode in ((15, W.PARTITION_ALL), (8, W.PARTITION_ALL), (11, W.PARTITION_BALANCED)):
+        w = W.random_small(5, n_devices=8, gpus_per_node=4, n_layers=9, global_batch=16, mp_max=2, pp_max=4,
+                           m_list=(1, 2, 4, 6, 8), partition_mode=mode, sched_mask=mask, v_max=4)
+        T, sp = w.table, w.space
+        L = T.n_layers
+        expect = []
+        for mp in (1, 2):
+            for pp in (1, 2, 4):
+                dp = T.n_devices // (mp * pp)
+                if T.global_batch % dp:
+                    continue
+                bp = T.global_batch // dp
+                ms = [m for m in sp.m_list.tolist() if m <= bp]
+                parts = (lambda P: [balanced(L, P)] if mode == W.PARTITION_BALANCED else
+                         [(0, *c, L) for c in itertools.combinations(range(1, L), P - 1)])
+                for m in ms:
+                    for b in parts(pp):
+                        for sc in (0, 1, 2):
+                            if mask & (1 << sc):
+                                expect.append((mp, pp, dp, m, sc, b, 1))
+                if pp >= 2:
+                    for v in (2, 4):
+                        if pp * v > L:
+                            continue
+                        for m in ms:
+                            if m % pp == 0:
+                                expect += [(mp, pp, dp, m, 3, b, v) for b in parts(pp * v)]
+        n = oracle.count(T, sp)
+        assert n == len(expect) == W.count_candidates_and_cells(T, sp)[0] and any(e[4] == 3 for e in expect)
+        got = oracle.enumerate_at(T, sp, np.arange(n))
+        assert [(c.mp, c.pp, c.dp, c.m, c.sched, c.bounds, c.v) for c in got] == expect
+        # and the enumerated interleaved candidates simulate like the same candidates given explicitly
+        for c in [c for c in got if c.sched == 3][::7]:
+            b, _ = oracle.eval_indices(T, sp, np.array([got.index(c)]))
+            assert b[0] == oracle.simulate(T, c, replicate=False, want_records=False).batch_ns
+
+
 def test_candidate_counts_of_the_benchmark_spaces():
     assert oracle.count(W.config1().table, W.config1().space) == 38_838_764
     assert oracle.count(W.config3().table, W.config3().space) == 650_420
