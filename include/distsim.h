@@ -147,6 +147,14 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *h_tabl
  * asynchronous 1F1B: the 1F1B item order without gradient all-reduce events - the paper's
  * discussion of new algorithms reads an asynchronous pipeline as the same schedule minus the
  * global synchronisation event).
+ * Bit 3 of sched_mask adds the interleaved 1F1B schedule (Sec. 4.3 takes the pipeline algorithm's
+ * schedule as Algorithm 1's input; the paper builds on Megatron-LM, whose interleaved schedule
+ * this is): every (mp, pp) with pp >= 2 is followed, for v = 2, 4, .. <= v_max with
+ * pp*v <= min(DISTSIM_MAX_PP, L), by the candidates whose devices hold v model chunks each -
+ * m ascending over the valid entries that are multiples of pp, then the partition of the layers
+ * into pp*v virtual stages (virtual stage c*pp + d is chunk c of device d).  Such candidates have
+ * schedule id 3; tables with per-micro-batch jitter do not combine with them
+ * (DISTSIM_E_UNSUPPORTED).
  * Candidates are never materialised: the device decodes them from the index.
  * Fails with DISTSIM_E_ARG if a needed class (mp, b) is not in the table, with
  * DISTSIM_E_OVERFLOW if the count does not fit 62 bits.  *n_candidates receives
@@ -158,15 +166,17 @@ typedef struct {
     int32_t m_rule;
     int32_t partition_mode;
     int32_t sched_mask;
+    int32_t v_max;                  /* interleaved 1F1B (sched_mask bit 3): chunks per device up to v_max */
 } distsim_space;
 
 int distsim_set_space(distsim_ctx *ctx, const distsim_space *h_space, int64_t *n_candidates);
 
 typedef struct {
-    int32_t mp, pp, dp, m, sched;   /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B */
+    int32_t mp, pp, dp, m, sched;   /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B, 3: interleaved 1F1B */
     int32_t micro_batch_size;       /* b = ceil(Bp / m)                            */
     int32_t class_index;            /* row of the event table                      */
-    int32_t bounds[DISTSIM_MAX_PP + 1];
+    int32_t bounds[DISTSIM_MAX_PP + 1];   /* c_0 .. c_pp (c_0 .. c_{pp*v} for sched 3) */
+    int32_t v;                      /* model chunks per device (1 unless sched 3)  */
 } distsim_candidate;
 
 /* Host-side decode of one index, for reporting (the device decodes on its own). */

@@ -166,6 +166,7 @@ int read_status(distsim_ctx *ctx, cudaStream_t s, bool *stalled)
         if (code == kStatusCopyPending)
             return fail(ctx, DISTSIM_E_TIMEOUT, "a bulk copy into shared memory never completed: results computed on this device since may be wrong");
         if (code == DISTSIM_E_RANGE) return fail(ctx, code, "candidate index out of range");
+        if (code == DISTSIM_E_UNSUPPORTED) return fail(ctx, code, "timelines of interleaved 1F1B candidates are not emitted");
         return fail(ctx, code, "device reported an error");
     }
     return DISTSIM_OK;
@@ -321,7 +322,11 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     if (!ctx->table_loaded) return fail(ctx, DISTSIM_E_STATE, "no event table loaded");
     if (sp->mp_max < 1 || sp->pp_max < 1 || sp->n_m < 1 || !sp->m_list) return fail(ctx, DISTSIM_E_ARG, "empty space");
     if (sp->pp_max > DISTSIM_MAX_PP) return fail(ctx, DISTSIM_E_ARG, "pp_max too large");
-    if ((sp->sched_mask & 7) == 0 || (sp->sched_mask & ~7)) return fail(ctx, DISTSIM_E_ARG, "bad sched_mask");
+    if ((sp->sched_mask & 15) == 0 || (sp->sched_mask & ~15)) return fail(ctx, DISTSIM_E_ARG, "bad sched_mask");
+    if ((sp->sched_mask & 8) && (sp->v_max < 2 || sp->v_max > DISTSIM_MAX_PP / 2))
+        return fail(ctx, DISTSIM_E_ARG, "interleaved schedule needs 2 <= v_max <= 32");
+    if ((sp->sched_mask & 8) && ctx->tc.n_jitter > 0)
+        return fail(ctx, DISTSIM_E_UNSUPPORTED, "the interleaved schedule does not combine with per-micro-batch jitter");
     if (sp->m_rule < 0 || sp->m_rule > 1 || sp->partition_mode < 0 || sp->partition_mode > 1)
         return fail(ctx, DISTSIM_E_ARG, "bad m_rule or partition_mode");
     for (int i = 0; i < sp->n_m; ++i) {
@@ -341,7 +346,11 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     // binomials C(n, k), n < L, k < binom_k, saturated
     int pp_cap = 1;
     while (pp_cap * 2 <= sp->pp_max && pp_cap * 2 <= L) pp_cap *= 2;
-    const int bk = pp_cap;
+    int bk = pp_cap;                                // most (virtual) stages of any candidate
+    if (sp->sched_mask & 8)
+        for (int pp = 2; pp <= pp_cap; pp *= 2)
+            for (int vc = 2; vc <= sp->v_max && pp * vc <= DISTSIM_MAX_PP && pp * vc <= L; vc *= 2)
+                if (pp * vc > bk) bk = pp * vc;
     std::vector<int64_t> binom((size_t)L * bk, 0);
     for (int n = 0; n < L; ++n)
         for (int k = 0; k < bk; ++k) {
@@ -376,45 +385,53 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
             const int64_t dp = N / (mp * pp);
             if (B % dp) continue;
             const int64_t Bp = B / dp;
-            Row r{};
-            r.mp = (int32_t)mp; r.pp = (int32_t)pp; r.dp = (int32_t)dp; r.log2_mp = floor_log2(mp);
-            r.entry0 = (int32_t)entries.size(); r.n_entries = 0;
-            r.n_sched = n_sched; r.sched_list = sched_list;
-            r.p2p_period = mp >= tc.gpus_per_node ? 1 : (int32_t)(tc.gpus_per_node / mp);
-            r.n_part = sp->partition_mode == 0 ? 1 : binom[(size_t)(L - 1) * bk + (pp - 1)];
-            for (int i = 0; i < sp->n_m; ++i) {
-                const int64_t m = sp->m_list[i];
-                if (m > Bp) continue;
-                if (sp->m_rule == 0 && Bp % m) continue;
-                const int64_t b = (Bp + m - 1) / m;
-                auto it = class_of.find(std::make_pair((int)mp, (int)b));
-                if (it == class_of.end()) {
-                    char msg[128];
-                    snprintf(msg, sizeof msg, "event class (mp=%lld, b=%lld) is not in the table", (long long)mp, (long long)b);
-                    return fail(ctx, DISTSIM_E_ARG, msg);
+            // the row of the plain schedules, then one row of interleaved candidates per chunk count
+            for (int64_t vc = 1; vc <= (((sp->sched_mask & 8) && pp >= 2) ? sp->v_max : 1); vc *= 2) {
+                if (vc == 1 && n_sched == 0) continue;
+                const int64_t P = pp * vc;              // (virtual) stages
+                if (vc > 1 && (P > DISTSIM_MAX_PP || P > L)) break;
+                Row r{};
+                r.mp = (int32_t)mp; r.pp = (int32_t)pp; r.dp = (int32_t)dp; r.log2_mp = floor_log2(mp);
+                r.v = (int32_t)vc;
+                r.entry0 = (int32_t)entries.size(); r.n_entries = 0;
+                r.n_sched = vc == 1 ? n_sched : 1; r.sched_list = vc == 1 ? sched_list : 3;
+                r.p2p_period = mp >= tc.gpus_per_node ? 1 : (int32_t)(tc.gpus_per_node / mp);
+                r.n_part = sp->partition_mode == 0 ? 1 : binom[(size_t)(L - 1) * bk + (P - 1)];
+                for (int i = 0; i < sp->n_m; ++i) {
+                    const int64_t m = sp->m_list[i];
+                    if (m > Bp) continue;
+                    if (sp->m_rule == 0 && Bp % m) continue;
+                    if (vc > 1 && m % pp) continue;     // the interleaved order needs whole groups of pp micro-batches
+                    const int64_t b = (Bp + m - 1) / m;
+                    auto it = class_of.find(std::make_pair((int)mp, (int)b));
+                    if (it == class_of.end()) {
+                        char msg[128];
+                        snprintf(msg, sizeof msg, "event class (mp=%lld, b=%lld) is not in the table", (long long)mp, (long long)b);
+                        return fail(ctx, DISTSIM_E_ARG, msg);
+                    }
+                    Entry en{};
+                    en.m = (int32_t)m; en.b = (int32_t)b; en.cls = it->second; en.row = (int32_t)rows.size();
+                    entries.push_back(en);
+                    ++r.n_entries;
+                    if (2 * m * P > op_words) op_words = 2 * m * P;
+                    // generous upper bound on any batch time of this entry: every item in sequence
+                    const long double act = (long double)b * tc.seq * tc.hidden * tc.elem_bytes;
+                    const long double comm = 2.0L * mp * a_max + 4.0L * act / b_min + 2 + dp * a_max + act / b_min + 2;
+                    const long double p2p = a_max + act / b_min + 2;
+                    const long double nbk = (tc.bucket > 0 ? gsum / tc.bucket + L + 1 : L + 1) + vc;
+                    const long double bsz = tc.bucket > 0 ? (long double)tc.bucket : gsum;
+                    const long double e_bound = (long double)m * (fg_max + 2.0L * L * comm + 2.0L * P * p2p) +
+                                                nbk * (2.0L * dp * a_max + 2.0L * bsz / b_min + 2);
+                    if (e_bound > tb) tb = e_bound;
                 }
-                Entry en{};
-                en.m = (int32_t)m; en.b = (int32_t)b; en.cls = it->second; en.row = (int32_t)rows.size();
-                entries.push_back(en);
-                ++r.n_entries;
-                if (2 * m * pp > op_words) op_words = 2 * m * pp;
-                // generous upper bound on any batch time of this entry: every item in sequence
-                const long double act = (long double)b * tc.seq * tc.hidden * tc.elem_bytes;
-                const long double comm = 2.0L * mp * a_max + 4.0L * act / b_min + 2 + dp * a_max + act / b_min + 2;
-                const long double p2p = a_max + act / b_min + 2;
-                const long double nbk = tc.bucket > 0 ? gsum / tc.bucket + L + 1 : L + 1;
-                const long double bsz = tc.bucket > 0 ? (long double)tc.bucket : gsum;
-                const long double e_bound = (long double)m * (fg_max + 2.0L * L * comm + 2.0L * pp * p2p) +
-                                            nbk * (2.0L * dp * a_max + 2.0L * bsz / b_min + 2);
-                if (e_bound > tb) tb = e_bound;
+                if (r.n_entries == 0) continue;
+                r.size = sat_mul(sat_mul(r.n_part, r.n_entries), r.n_sched);
+                r.offset = total;
+                r.row_tab_off = (int64_t)rows.size() * (((L + 1) * (L + 1) + 1) & ~1);   // even: 16-byte aligned tables
+                total = sat_add(total, r.size);
+                if (r.n_part >= kSat || total >= kSat) return fail(ctx, DISTSIM_E_OVERFLOW, "candidate count does not fit 62 bits");
+                rows.push_back(r);
             }
-            if (r.n_entries == 0) continue;
-            r.size = sat_mul(sat_mul(r.n_part, r.n_entries), r.n_sched);
-            r.offset = total;
-            r.row_tab_off = (int64_t)rows.size() * (((L + 1) * (L + 1) + 1) & ~1);   // even: 16-byte aligned tables
-            total = sat_add(total, r.size);
-            if (r.n_part >= kSat || total >= kSat) return fail(ctx, DISTSIM_E_OVERFLOW, "candidate count does not fit 62 bits");
-            rows.push_back(r);
         }
     if (rows.empty()) return fail(ctx, DISTSIM_E_ARG, "the space has no valid candidate");
     if (tc.n_jitter > 0)
@@ -492,7 +509,8 @@ int distsim_decode(distsim_ctx *ctx, int64_t index, distsim_candidate *out)
     out->mp = row.mp; out->pp = row.pp; out->dp = row.dp; out->m = en.m;
     out->sched = row_sched(row, (int)(rem % row.n_sched));
     out->micro_batch_size = en.b; out->class_index = en.cls;
-    const int L = ctx->tc.n_layers, pp = row.pp, bk = ctx->sc.binom_k;
+    out->v = row.v;
+    const int L = ctx->tc.n_layers, pp = row.pp * row.v /* (virtual) stages */, bk = ctx->sc.binom_k;
     out->bounds[0] = 0; out->bounds[pp] = L;
     if (ctx->sc.partition_mode == 0) {
         for (int j = 1; j < pp; ++j) out->bounds[j] = (int32_t)((int64_t)j * L / pp);
@@ -700,11 +718,11 @@ int distsim_testing_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_c
     for (const Row &row : ctx->rows)
         for (int e = 0; e < row.n_entries; ++e) {
             const Entry &en = ctx->entries[row.entry0 + e];
-            const __int128 c = (__int128)2 * en.m * row.pp * row.n_part * row.n_sched;
+            const __int128 c = (__int128)2 * en.m * row.pp * row.v * row.n_part * row.n_sched;
             total += c;
             // 32-bit arithmetic is used where the entry's time bound allows it and the row is
             // evaluated by the one-partition-per-thread kernel
-            if (en.bound < ((int64_t)1 << 32) && row.pp <= 16) narrow += c;
+            if (en.bound < ((int64_t)1 << 32) && row.pp <= 16 && row.v == 1) narrow += c;
         }
     *h_cells = total >= (__int128)kSat ? kSat : (int64_t)total;
     *h_cells_32bit = narrow >= (__int128)kSat ? kSat : (int64_t)narrow;

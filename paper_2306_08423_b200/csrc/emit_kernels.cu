@@ -213,9 +213,19 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
         } else {
             const int r = find_row(v, index);
             const Row row = v.rows[r];
+            if (row.v > 1) {
+                // timelines of interleaved candidates are not emitted (their evaluation is)
+                if ((threadIdx.x & 31) == 0) {
+                    plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
+                    plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
+                    for (int w = 0; w < kSumWords; ++w) sums[(int64_t)i * kSumWords + w] = 0;
+                    atomicCAS(v.status, 0, DISTSIM_E_UNSUPPORTED);
+                }
+            } else {
             int64_t *rec = op_start + (int64_t)i * op_words_per_cand;
             if (row.pp > 32) plan_candidate<2>(v, row, r, index, plan, rec, binom, sums + (int64_t)i * kSumWords);
             else plan_candidate<1>(v, row, r, index, plan, rec, binom, sums + (int64_t)i * kSumWords);
+            }
         }
     }
     __threadfence();

@@ -59,10 +59,11 @@ struct Row {
     int32_t n_entries, entry0;
     int32_t n_sched, sched_list;   // enabled schedules in canonical order, two bits each (see row_sched)
     int32_t p2p_period;   // boundary d|d+1 is inter-node iff ((d+1) & (p2p_period-1)) == 0
-    int32_t pad;
+    int32_t v;            // model chunks per device: 1, or > 1 for a row of interleaved 1F1B candidates
+                          // (one schedule, id 3; partitions into pp * v virtual stages)
 };
 
-// Schedule id (0 GPipe, 1 1F1B, 2 asynchronous 1F1B) of position sc among a row's schedules.
+// Schedule id (0 GPipe, 1 1F1B, 2 asynchronous 1F1B, 3 interleaved 1F1B) of position sc among a row's schedules.
 __host__ __device__ inline int row_sched(const Row &row, int sc) { return (row.sched_list >> (2 * sc)) & 3; }
 
 struct Entry {

@@ -17,6 +17,7 @@
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
 #include "eval_thread.cuh"
+#include "interleaved.cuh"
 
 namespace distsim {
 
@@ -235,6 +236,8 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
     std::vector<EvalWork> lock_items;              // lock-step kernel
     std::vector<int> lock_words;
     std::vector<ThreadItem> thread_items;          // one-partition-per-thread kernel
+    std::vector<EvalWork> ilv_items;               // interleaved 1F1B kernel (a candidate per warp)
+    int ilv_words = 0;
     constexpr int64_t kPieceBlocks = 1 << 24;
 
     auto add_lockstep = [&](int r, int64_t lo, int64_t hi) {
@@ -254,6 +257,18 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
         const int64_t lo = first > row.offset ? first - row.offset : 0;
         const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
         if (hi <= lo) continue;
+        if (row.v > 1) {
+            constexpr int64_t cpb = kIlvThreads / 32;
+            for (int64_t a = lo; a < hi; a += kPieceBlocks * cpb) {
+                EvalWork w{};
+                w.row = r; w.lo = a; w.hi = hi - a < kPieceBlocks * cpb ? hi : a + kPieceBlocks * cpb;
+                w.nx = (int)((w.hi - w.lo + cpb - 1) / cpb);
+                ilv_items.push_back(w);
+            }
+            const int words = interleaved_words(row.pp, row.v);
+            if (words > ilv_words) ilv_words = words;
+            continue;
+        }
         if (row.pp > 16) { add_lockstep(r, lo, hi); continue; }
         // Short pipelines: cut the range into runs of entries with the same arithmetic width; a
         // run with enough partitions goes to the one-partition-per-thread kernel, the rest to
@@ -321,6 +336,23 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
         if (lock_words[i] > p.smem_words) p.smem_words = lock_words[i];
     }
     flush_lockstep(ls, v, p, first, batch_out, busy_out, launches);
+    // interleaved candidates: a kernel of their own, on the caller's stream
+    auto flush_interleaved = [&]() {
+        if (p.batch.n == 0) return;
+        const size_t smem = (size_t)(kIlvThreads / 32) * ilv_words * sizeof(int64_t);
+        ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_interleaved_kernel), smem);
+        eval_interleaved_kernel<<<p.blocks, kIlvThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, ilv_words);
+        ++*launches;
+        p = Pending{};
+    };
+    for (const EvalWork &item : ilv_items) {
+        if (p.batch.n == kMaxEvalWork || p.blocks > kMaxBlocks - item.nx) flush_interleaved();
+        EvalWork &w = p.batch.w[p.batch.n++];
+        w = item;
+        w.block_begin = p.blocks;
+        p.blocks += w.nx;
+    }
+    flush_interleaved();
     for (int lg = 4; lg >= 0; --lg)
         for (int nw = 1; nw >= 0; --nw) {
             for (const ThreadItem &it : thread_items) {

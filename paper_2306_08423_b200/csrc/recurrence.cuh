@@ -136,44 +136,67 @@ __device__ __forceinline__ int64_t jitter_of(const DeviceView &v, const int64_t 
     return v.tc.n_jitter ? __ldg(&table[(j & (v.tc.n_jitter - 1)) * v.tc.jitter_stages + d]) : 0;
 }
 
-// Gradient all-reduce buckets of one stage [a, e) on the communication lane (DP modeling).
-// `tb` is the start of the stage's last backward item, `main_end` the end of the main lane.
-// pb: the entry's backward prefix row; nbt/tpt: the row's bucket tables.  Returns the end of the
-// last bucket (main_end when the stage sends no gradients).
-__device__ __forceinline__ int64_t bucket_lane_end(const DeviceView &v, const Row &row,
-                                                   const int64_t *pb, const int64_t *nbt,
-                                                   const int64_t *tpt, int a, int e, int64_t tb,
-                                                   int64_t main_end)
+// Gradient all-reduce buckets of one stage [a, e) appended to a communication lane (DP modeling).
+// `tb` is the start of the stage's last backward item, `main_end` the end of the device's main
+// lane, `end` the end of the lane's buckets so far (0: none yet).  pb: the entry's backward prefix
+// row; nbt/tpt: the row's bucket tables.  Returns the lane's new end and sets `any` if the stage
+// has a bucket; visit(start, end) is called for every run of buckets that follow each other
+// without a gap.
+template <class Visit>
+__device__ __forceinline__ int64_t bucket_lane_chain(const DeviceView &v, const Row &row,
+                                                     const int64_t *pb, const int64_t *nbt,
+                                                     const int64_t *tpt, int a, int e, int64_t tb,
+                                                     int64_t main_end, int64_t end, bool &any, Visit visit)
 {
-    if (row.dp == 1) return main_end;
     const int L1 = v.tc.n_layers + 1;
     const int64_t *nbe = nbt + (int64_t)e * L1;
     const int64_t part = __ldg(&tpt[(int64_t)e * L1 + a]);
     if (!v.tc.overlap) {
         const int64_t full = __ldg(&nbe[a]);
-        if (full == 0 && part == 0) return main_end;
-        return main_end + full * row.t_full + part;
+        if (full == 0 && part == 0) return end;
+        any = true;
+        const int64_t start = max64(end, main_end);
+        visit(start, start + full * row.t_full + part);
+        return start + full * row.t_full + part;
     }
     // a bucket is ready when the layer holding its last byte has finished its backward
     // composite in the last backward item; buckets then run back to back
-    int64_t end = 0;
-    bool any = false;
     const int64_t pbe = pb[e];
     if (v.tc.bucket > 0) {
         int64_t nb_prev = 0;                   // nb[e][l+1]
         for (int l = e - 1; l >= a; --l) {
             const int64_t nb_l = __ldg(&nbe[l]);
             const int64_t n_l = nb_l - nb_prev; // full buckets whose last byte lies in layer l
-            if (n_l > 0) { end = max64(end, tb + (pbe - pb[l])) + n_l * row.t_full; any = true; }
+            if (n_l > 0) {
+                const int64_t start = max64(end, tb + (pbe - pb[l]));
+                end = start + n_l * row.t_full;
+                visit(start, end);
+                any = true;
+            }
             nb_prev = nb_l;
         }
     }
     if (part > 0) {
         // the trailing bucket ends in the stage's first layer that has any gradient bytes
         const int lstar = __ldg(&v.next_grad[a]);
-        end = max64(end, tb + (pbe - pb[lstar])) + part;
+        const int64_t start = max64(end, tb + (pbe - pb[lstar]));
+        end = start + part;
+        visit(start, end);
         any = true;
     }
+    return end;
+}
+
+// The same for a device with one stage: the end of its bucket lane (main_end when the stage
+// sends no gradients).
+__device__ __forceinline__ int64_t bucket_lane_end(const DeviceView &v, const Row &row,
+                                                   const int64_t *pb, const int64_t *nbt,
+                                                   const int64_t *tpt, int a, int e, int64_t tb,
+                                                   int64_t main_end)
+{
+    if (row.dp == 1) return main_end;
+    bool any = false;
+    const int64_t end = bucket_lane_chain(v, row, pb, nbt, tpt, a, e, tb, main_end, 0, any, [](int64_t, int64_t) {});
     return any ? end : main_end;
 }
 

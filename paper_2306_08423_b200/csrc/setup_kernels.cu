@@ -186,15 +186,18 @@ __global__ void entry_bound_kernel(DeviceView v, Entry *entries, int64_t *jsum)
     int64_t per_mb = pf[L] + pb[L], frame_shift = pb[L];
     for (int d = 0; d + 1 < row.pp; ++d) {
         const int64_t p2p = (((d + 1) & (row.p2p_period - 1)) == 0) ? en.p2p_inter : en.p2p_intra;
-        per_mb += 2 * p2p;
+        per_mb += 2 * p2p * row.v;                  // once per model chunk
         frame_shift += p2p;
     }
+    // interleaved candidates: the last device sends to the first between chunks
+    if (row.v > 1) per_mb += 2 * (row.v - 1) * (en.p2p_inter > en.p2p_intra ? en.p2p_inter : en.p2p_intra);
     int64_t excess = 0;
     if (row.dp > 1) {
         const int64_t *nbL = v.nb + row.row_tab_off + (int64_t)L * L1;
         const int64_t *tpL = v.tp + row.row_tab_off + (int64_t)L * L1;
-        // a stage's buckets cost at most all full buckets of the model plus one more bucket
-        excess = nbL[0] * row.t_full + (v.tc.bucket > 0 ? row.t_full : tpL[0]);
+        // a device's buckets cost at most all full buckets of the model plus one more bucket per
+        // model chunk it holds
+        excess = nbL[0] * row.t_full + row.v * (v.tc.bucket > 0 ? row.t_full : tpL[0]);
     }
     // total jitter of a stage's items: whole cycles of the P slots plus the remainder
     __int128 jitter_total = 0;

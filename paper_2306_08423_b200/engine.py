@@ -61,13 +61,13 @@ class _Table(C.Structure):
 class _Space(C.Structure):
     _fields_ = [("mp_max", C.c_int32), ("pp_max", C.c_int32), ("n_m", C.c_int32),
                 ("m_list", C.c_void_p), ("m_rule", C.c_int32), ("partition_mode", C.c_int32),
-                ("sched_mask", C.c_int32)]
+                ("sched_mask", C.c_int32), ("v_max", C.c_int32)]
 
 
 class _Candidate(C.Structure):
     _fields_ = [("mp", C.c_int32), ("pp", C.c_int32), ("dp", C.c_int32), ("m", C.c_int32),
                 ("sched", C.c_int32), ("micro_batch_size", C.c_int32), ("class_index", C.c_int32),
-                ("bounds", C.c_int32 * (MAX_PP + 1))]
+                ("bounds", C.c_int32 * (MAX_PP + 1)), ("v", C.c_int32)]
 
 
 _lib.distsim_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
@@ -137,7 +137,7 @@ def _table_struct(t):
 def _space_struct(sp):
     ml = np.ascontiguousarray(sp.m_list, np.int32)
     return _Space(sp.mp_max, sp.pp_max, ml.shape[0], _np_ptr(ml), sp.m_rule, sp.partition_mode,
-                  sp.sched_mask), ml
+                  sp.sched_mask, int(getattr(sp, "v_max", 0))), ml
 
 
 def _dev_ptr(t, dtype_name: str, min_elems: int, what: str):
@@ -212,7 +212,7 @@ def distsim_decode(ctx: Context, index: int) -> dict:
     c = _Candidate()
     ctx._check(_lib.distsim_decode(ctx._h, index, C.byref(c)))
     return dict(mp=c.mp, pp=c.pp, dp=c.dp, m=c.m, sched=c.sched, micro_batch_size=c.micro_batch_size,
-                class_index=c.class_index, bounds=tuple(c.bounds[: c.pp + 1]))
+                class_index=c.class_index, bounds=tuple(c.bounds[: c.pp * c.v + 1]), v=c.v)
 
 
 def distsim_eval_strategies(ctx: Context, first: int, count: int, d_batch_ns,
