@@ -69,6 +69,7 @@ struct distsim_ctx {
     std::vector<int64_t> binom;
     int64_t time_bound = 0;
     int64_t op_words_per_cand = 0;
+    int ilv_words = 0;                    // shared-memory words a warp needs for the interleaved rows
     int32_t stage_polls = 1 << 16;        // polls of the first wait for staged tables
     cudaEvent_t phase_ev[3] = {nullptr, nullptr, nullptr};   // timing of distsim_eval_select's phases (hook)
     bool phase_timing = false, phase_valid = false;
@@ -166,7 +167,6 @@ int read_status(distsim_ctx *ctx, cudaStream_t s, bool *stalled)
         if (code == kStatusCopyPending)
             return fail(ctx, DISTSIM_E_TIMEOUT, "a bulk copy into shared memory never completed: results computed on this device since may be wrong");
         if (code == DISTSIM_E_RANGE) return fail(ctx, code, "candidate index out of range");
-        if (code == DISTSIM_E_UNSUPPORTED) return fail(ctx, code, "timelines of interleaved 1F1B candidates are not emitted");
         return fail(ctx, code, "device reported an error");
     }
     return DISTSIM_OK;
@@ -442,6 +442,9 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     ctx->rows = rows; ctx->entries = entries; ctx->binom = binom;
     ctx->time_bound = (int64_t)tb + 1;
     ctx->op_words_per_cand = op_words;
+    ctx->ilv_words = 0;
+    for (const Row &r : rows)
+        if (r.v > 1 && interleaved_words_of(r.pp, r.v) > ctx->ilv_words) ctx->ilv_words = interleaved_words_of(r.pp, r.v);
     SpaceConst &sc = ctx->sc;
     sc.n_rows = (int32_t)rows.size(); sc.n_entries = (int32_t)entries.size();
     sc.pp_max = sp->pp_max; sc.partition_mode = sp->partition_mode; sc.binom_k = bk; sc.pad = 0;
@@ -649,7 +652,8 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     CU(ctx->d_plan_sums.reserve((size_t)n * kEmitSumWords * sizeof(int64_t)), "alloc plan summaries");
     const DeviceView v = ctx->view();
     launch_emit_plan(s, v, d_indices, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
-                     ctx->op_words_per_cand, ctx->d_plan_sums.as<int64_t>(), d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), &ctx->launches);
+                     ctx->op_words_per_cand, ctx->d_plan_sums.as<int64_t>(), d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), ctx->ilv_words,
+                     &ctx->launches);
     CU(cudaGetLastError(), "emission planning launch");
     static_assert(sizeof(EmitTotals) == 8 * sizeof(int64_t), "totals occupy the second half of the pinned words");
     const EmitTotals *totals = reinterpret_cast<const EmitTotals *>(ctx->h_pinned + 8);

@@ -16,6 +16,7 @@
 //   emit_buckets_kernel  gradient-bucket records of every stage.
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
+#include "interleaved.cuh"
 
 namespace distsim {
 
@@ -127,7 +128,7 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
     if (lane == 0) {
         plan->index = index; plan->batch_ns = R.batch;
         plan->row = row_index; plan->entry = cc.entry; plan->m = en.m; plan->sched = cc.sched;
-        plan->pp = row.pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1;
+        plan->pp = row.pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1; plan->v = 1;
         plan->stage_rec_prefix[row.pp] = total;
         plan->rec_total = total * row.mp * row.dp;
         // a run of tile_items items of any mix must fit the image of kTileWords words
@@ -142,6 +143,85 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
         sum[kSumItemTiles] = (int64_t)row.pp * ((2 * en.m + plan->tile_items - 1) / plan->tile_items) *
                              ((reps + kTileReplicas - 1) / kTileReplicas);
         sum[kSumBucketTiles] = (int64_t)row.pp * ((reps + kBucketReplicas - 1) / kBucketReplicas);
+        sum[kSumTmplWords] = plan->tmpl_words;
+        sum[kSumBucketRecs] = most_buckets;
+        sum[kSumRunWords] = plan->run_words;
+    }
+}
+
+// The same for a candidate of the interleaved schedule (a lane per device, v chunks each): A is
+// the warp's shared memory for the evaluation.  Record counts, bounds and last backward starts
+// are kept per virtual stage c * pp + d, the rest per device.
+__device__ __forceinline__ void plan_interleaved(const DeviceView &v, const Row &row, int row_index, int64_t index,
+                                                 EmitPlan *plan, int64_t *rec, const int64_t *binom, int64_t *sum,
+                                                 const IlvArrays &A)
+{
+    const int lane = threadIdx.x & 31;
+    const int pp = row.pp, vch = row.v, P = pp * vch;
+    const CandidateCoords cc = split_local(row, index - row.offset);
+    const Entry en = v.entries[cc.entry];
+    const IlvResult R = interleaved_candidate(v, row, en, cc, binom, A, rec);
+    const int L1 = v.tc.n_layers + 1;
+    int widest = 1, both = 0;
+    int64_t dev_recs = 0, dev_buckets = 0;
+    if (lane < pp) {
+        const int d = lane;
+        for (int c = 0; c < vch; ++c) {
+            const int s = c * pp + d;
+            const int a = A.bounds[s], e = A.bounds[s + 1];
+            const int64_t per_dir = (int64_t)(e - a) * (row.mp > 1 ? 2 : 1) + (row.dp > 1 ? v.pe[e] - v.pe[a] : 0);
+            const int64_t rf = per_dir + (s < P - 1 ? 1 : 0);
+            const int64_t rb = per_dir + (s > 0 ? 1 : 0);
+            int64_t kb = 0;
+            if (row.dp > 1) {
+                const int64_t *nbt = v.nb + row.row_tab_off, *tpt = v.tp + row.row_tab_off;
+                kb = nbt[(int64_t)e * L1 + a] + (tpt[(int64_t)e * L1 + a] > 0 ? 1 : 0);
+            }
+            plan->bounds[s] = a;
+            if (s == P - 1) plan->bounds[P] = e;
+            plan->rf[s] = (int32_t)rf; plan->rb[s] = (int32_t)rb;
+            plan->last_b_start[s] = A.last_b[s];
+            dev_recs += (int64_t)en.m * (rf + rb) + kb;
+            dev_buckets += kb;
+            widest = max(widest, (int)max(rf, rb));
+            both += (int)(rf + rb);
+        }
+        plan->n_buckets[d] = dev_buckets;
+        plan->stage_recs[d] = dev_recs;
+        plan->busy[d] = R.busy;
+        plan->main_end[d] = R.main_end;
+    }
+    int64_t incl = dev_recs, most_buckets = dev_buckets;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int64_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    const int64_t total = __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        widest = max(widest, __shfl_xor_sync(0xffffffffu, widest, o));
+        both = max(both, __shfl_xor_sync(0xffffffffu, both, o));
+        most_buckets = max64(most_buckets, __shfl_xor_sync(0xffffffffu, most_buckets, o));
+    }
+    if (lane < pp) plan->stage_rec_prefix[lane] = incl - dev_recs;
+    if (lane == 0) {
+        plan->index = index; plan->batch_ns = R.batch;
+        plan->row = row_index; plan->entry = cc.entry; plan->m = en.m; plan->sched = 3;
+        plan->pp = pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1; plan->v = vch;
+        plan->stage_rec_prefix[pp] = total;
+        plan->rec_total = total * row.mp * row.dp;
+        const int n_items = 2 * en.m * vch;                       // items of a device
+        const int cap = max(1, min(kMaxTileItems, kRunWords / (widest * 5)));
+        const int n_chunks = (n_items + cap - 1) / cap;
+        plan->tile_items = (n_items + n_chunks - 1) / n_chunks;
+        plan->run_words = plan->tile_items * widest * 5;
+        plan->tmpl_words = both * 5;                              // the templates of all chunks of the widest device
+        const int64_t reps = (int64_t)row.mp * row.dp;
+        sum[kSumRecords] = plan->rec_total;
+        sum[kSumItemTiles] = (int64_t)pp * ((n_items + plan->tile_items - 1) / plan->tile_items) *
+                             ((reps + kTileReplicas - 1) / kTileReplicas);
+        sum[kSumBucketTiles] = (int64_t)pp * ((reps + kBucketReplicas - 1) / kBucketReplicas);
         sum[kSumTmplWords] = plan->tmpl_words;
         sum[kSumBucketRecs] = most_buckets;
         sum[kSumRunWords] = plan->run_words;
@@ -194,8 +274,10 @@ __device__ __forceinline__ void scan_plans(EmitPlan *plans, const int64_t *sums,
 constexpr int kPlanBinomWords = 512;
 __global__ void __launch_bounds__(128)
 emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitPlan *plans,
-                 int64_t *op_start, int64_t op_words_per_cand, int64_t *sums, int64_t *totals)
+                 int64_t *op_start, int64_t op_words_per_cand, int64_t *sums, int64_t *totals,
+                 int ilv_words /* shared-memory words per warp for interleaved candidates */)
 {
+    extern __shared__ __align__(16) int64_t plan_dyn[];
     __shared__ int64_t binom_s[kPlanBinomWords];
     __shared__ bool last;
     const int64_t *binom = stage_binom(v, binom_s, kPlanBinomWords);
@@ -205,7 +287,7 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
         const int64_t index = indices[i];
         if (index < 0 || index >= v.sc.n_candidates) {
             if ((threadIdx.x & 31) == 0) {
-                plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
+                plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0; plan->v = 1;
                 plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
                 for (int w = 0; w < kSumWords; ++w) sums[(int64_t)i * kSumWords + w] = 0;
                 atomicCAS(v.status, 0, DISTSIM_E_RANGE);
@@ -213,14 +295,10 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
         } else {
             const int r = find_row(v, index);
             const Row row = v.rows[r];
+            int64_t *rec_i = op_start + (int64_t)i * op_words_per_cand;
             if (row.v > 1) {
-                // timelines of interleaved candidates are not emitted (their evaluation is)
-                if ((threadIdx.x & 31) == 0) {
-                    plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0;
-                    plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
-                    for (int w = 0; w < kSumWords; ++w) sums[(int64_t)i * kSumWords + w] = 0;
-                    atomicCAS(v.status, 0, DISTSIM_E_UNSUPPORTED);
-                }
+                plan_interleaved(v, row, r, index, plan, rec_i, binom, sums + (int64_t)i * kSumWords,
+                                 interleaved_arrays(plan_dyn + (int64_t)(threadIdx.x >> 5) * ilv_words, row.pp, row.v));
             } else {
             int64_t *rec = op_start + (int64_t)i * op_words_per_cand;
             if (row.pp > 32) plan_candidate<2>(v, row, r, index, plan, rec, binom, sums + (int64_t)i * kSumWords);
@@ -293,94 +371,108 @@ __device__ __forceinline__ void emit_buckets_block(const DeviceView &v, const Em
     int64_t *img_b = dyn_s + run * 5 + 1;               // the same word at img_b[x + 1] (run * 5 + 1 is even)
     int64_t *g_start = img_b + run * 5 + 1;             // [L + 1] start of the first bucket ending in layer a+i
     int64_t *g_first = g_start + DISTSIM_MAX_LAYERS + 1;  // [L + 1] number of that bucket
-    __shared__ int64_t part_start_s;
+    __shared__ int64_t part_start_s, lane_end_s;
     if (!p.ok || p.dp == 1) return;
     const int mp = p.mp, reps = mp * p.dp;
     const int rep_chunks = (reps + kBucketReplicas - 1) / kBucketReplicas;
     const int d = tile / rep_chunks, rc = tile - d * rep_chunks;
     if (d >= p.pp) return;
-    const int64_t kb = p.n_buckets[d];
-    if (kb == 0) return;
+    if (p.n_buckets[d] == 0) return;
     const Row &row = v.rows[p.row];
-    const int a = p.bounds[d], e = p.bounds[d + 1];
     const int L1 = v.tc.n_layers + 1;
-    const int64_t *nbe = v.nb + row.row_tab_off + (int64_t)e * L1;
-    const int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
     const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
-    const int64_t n_full = nbe[a], t_full = row.t_full;
-    const int64_t tbs = p.last_b_start[d], main_end = p.main_end[d];
-    // all threads fetch the per-layer inputs (independent loads), then thread 0 runs the short chain
-    for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
-        g_first[l - a] = l + 1 < e ? nbe[l + 1] : 0;                       // buckets before layer l's group
-        g_start[l - a] = v.tc.overlap ? tbs + (pb[e] - pb[l]) : main_end;    // ready time of the group
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int64_t end = 0, part_start = 0;
-        for (int l = e - 1; l >= a; --l) {
-            const int64_t nb_prev = g_first[l - a];
-            const int64_t nb_l = l > a ? g_first[l - 1 - a] : n_full;       // nb[e][l]
-            const int64_t start = max64(end, g_start[l - a]);
-            g_start[l - a] = start;
-            if (nb_l > nb_prev) end = start + (nb_l - nb_prev) * t_full;
-        }
-        if (part > 0) {
-            const int ls = v.next_grad[a];
-            const int64_t ready = v.tc.overlap ? tbs + (pb[e] - pb[ls]) : main_end;
-            part_start = max64(end, ready);
-        }
-        part_start_s = part_start;
-    }
-    __syncthreads();
-    const int64_t part_start = part_start_s;
+    const int64_t t_full = row.t_full, main_end = p.main_end[d];
     const int64_t stage_words = p.stage_recs[d] * 5;
     const int64_t replica_words = (int64_t)mp * p.stage_rec_prefix[p.pp] * 5;
-    int64_t *base = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + (int64_t)p.m * (p.rf[d] + p.rb[d]) * 5;
-    for (int64_t k0 = 0; k0 < kb; k0 += run) {
-        const int nk = (int)min((int64_t)run, kb - k0);
-        for (int kk = threadIdx.x; kk < nk; kk += blockDim.x) {
-            const int64_t k = k0 + kk;
-            int64_t start, dur;
-            if (k >= n_full) { start = part_start; dur = part; }
-            else {
-                // the layer whose group holds bucket k: the largest l with nb[e][l] > k
-                // (nb[e][l] = g_first[l-1-a] for l > a grows as l decreases, and nb[e][a] = n_full > k)
-                int lo = a, hi = e - 1;
-                while (lo < hi) {
-                    const int mid = (lo + hi + 1) >> 1;
-                    if (g_first[mid - 1 - a] > k) lo = mid; else hi = mid - 1;
+    // the device's bucket records follow its main-lane records
+    int64_t *base = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + (p.stage_recs[d] - p.n_buckets[d]) * 5;
+    if (threadIdx.x == 0) lane_end_s = 0;
+    int64_t kb0 = 0;                                    // buckets of the chunks already written
+    // one gradient stream per model chunk the device holds (one without chunks), the last chunk
+    // first, all on the device's one lane
+    for (int c = p.v - 1; c >= 0; --c) {
+        const int s = c * p.pp + d;                     // (virtual) stage
+        const int a = p.bounds[s], e = p.bounds[s + 1];
+        const int64_t *nbe = v.nb + row.row_tab_off + (int64_t)e * L1;
+        const int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
+        const int64_t n_full = nbe[a];
+        const int64_t kb = n_full + (part > 0 ? 1 : 0);
+        if (kb == 0) continue;
+        const int64_t tbs = p.last_b_start[s];
+        __syncthreads();                                // the previous chunk's reads of g_start / g_first are done
+        // all threads fetch the per-layer inputs (independent loads), then thread 0 runs the short chain
+        for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
+            g_first[l - a] = l + 1 < e ? nbe[l + 1] : 0;                       // buckets before layer l's group
+            g_start[l - a] = v.tc.overlap ? tbs + (pb[e] - pb[l]) : main_end;    // ready time of the group
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int64_t end = lane_end_s, part_start = 0;
+            for (int l = e - 1; l >= a; --l) {
+                const int64_t nb_prev = g_first[l - a];
+                const int64_t nb_l = l > a ? g_first[l - 1 - a] : n_full;       // nb[e][l]
+                const int64_t start = max64(end, g_start[l - a]);
+                g_start[l - a] = start;
+                if (nb_l > nb_prev) end = start + (nb_l - nb_prev) * t_full;
+            }
+            if (part > 0) {
+                const int ls = v.next_grad[a];
+                const int64_t ready = v.tc.overlap ? tbs + (pb[e] - pb[ls]) : main_end;
+                part_start = max64(end, ready);
+                end = part_start + part;
+            }
+            part_start_s = part_start;
+            lane_end_s = end;
+        }
+        __syncthreads();
+        const int64_t part_start = part_start_s;
+        for (int64_t k0 = 0; k0 < kb; k0 += run) {
+            const int nk = (int)min((int64_t)run, kb - k0);
+            for (int kk = threadIdx.x; kk < nk; kk += blockDim.x) {
+                const int64_t k = k0 + kk;
+                int64_t start, dur;
+                if (k >= n_full) { start = part_start; dur = part; }
+                else {
+                    // the layer whose group holds bucket k: the largest l with nb[e][l] > k
+                    // (nb[e][l] = g_first[l-1-a] for l > a grows as l decreases, and nb[e][a] = n_full > k)
+                    int lo = a, hi = e - 1;
+                    while (lo < hi) {
+                        const int mid = (lo + hi + 1) >> 1;
+                        if (g_first[mid - 1 - a] > k) lo = mid; else hi = mid - 1;
+                    }
+                    start = g_start[lo - a] + (k - g_first[lo - a]) * t_full;
+                    dur = t_full;
                 }
-                start = g_start[lo - a] + (k - g_first[lo - a]) * t_full;
-                dur = t_full;
-            }
-            const int64_t rec[5] = {DISTSIM_DP_AR, k, -1, start, start + dur};
+                const int64_t rec[5] = {DISTSIM_DP_AR, kb0 + k, -1, start, start + dur};
 #pragma unroll
-            for (int f = 0; f < 5; ++f) { img_a[kk * 5 + f] = rec[f]; img_b[kk * 5 + f + 1] = rec[f]; }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncthreads();
-        const int total = nk * 5;
-        const int rep = rc * kBucketReplicas + threadIdx.x;
-        if (threadIdx.x < kBucketReplicas && rep < reps) {
-            const int r = rep / mp, q = rep - r * mp;
-            int64_t *dst = base + (int64_t)r * replica_words + (int64_t)q * stage_words + k0 * 5;
-            // 16-byte aligned copies take img_a from word 0, the others img_b from word 1
-            const bool odd = ((reinterpret_cast<uintptr_t>(dst) >> 3) & 1) != 0;
-            const int head = odd ? 1 : 0;
-            const int bulk_words = (total - head) & ~1;
-            if (odd) __stcs(dst, img_a[0]);
-            if (head + bulk_words < total) __stcs(dst + total - 1, img_a[total - 1]);
-            // the image is rewritten by the next run, and the block's shared memory must outlive
-            // the copy engine's reads of it
-            if (bulk_words > 0) {
-                const int64_t *src = odd ? img_b + 2 : img_a;
-                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                             :: "l"(dst + head), "r"(smem_addr(src)), "r"(bulk_words * 8) : "memory");
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                for (int f = 0; f < 5; ++f) { img_a[kk * 5 + f] = rec[f]; img_b[kk * 5 + f + 1] = rec[f]; }
             }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncthreads();
+            const int total = nk * 5;
+            const int rep = rc * kBucketReplicas + threadIdx.x;
+            if (threadIdx.x < kBucketReplicas && rep < reps) {
+                const int r = rep / mp, q = rep - r * mp;
+                int64_t *dst = base + (int64_t)r * replica_words + (int64_t)q * stage_words + (kb0 + k0) * 5;
+                // 16-byte aligned copies take img_a from word 0, the others img_b from word 1
+                const bool odd = ((reinterpret_cast<uintptr_t>(dst) >> 3) & 1) != 0;
+                const int head = odd ? 1 : 0;
+                const int bulk_words = (total - head) & ~1;
+                if (odd) __stcs(dst, img_a[0]);
+                if (head + bulk_words < total) __stcs(dst + total - 1, img_a[total - 1]);
+                // the image is rewritten by the next run, and the block's shared memory must outlive
+                // the copy engine's reads of it
+                if (bulk_words > 0) {
+                    const int64_t *src = odd ? img_b + 2 : img_a;
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                 :: "l"(dst + head), "r"(smem_addr(src)), "r"(bulk_words * 8) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                }
+            }
+            __syncthreads();
         }
-        __syncthreads();
+        kb0 += kb;
     }
 }
 
@@ -394,6 +486,39 @@ emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *_
     emit_buckets_block(v, plans[blockIdx.y], (int)blockIdx.x, out, run, dyn_b);
 }
 
+// Interleaved 1F1B: position `pos` in device d's order -> (is backward, chunk, micro-batch, forward
+// and backward items before it); see interleaved.cuh for the order.
+__device__ __forceinline__ void interleaved_item_at(int pp, int vch, int m, int d, int pos, bool &bwd, int &c, int &j,
+                                                    int &nf, int &nb)
+{
+    const int total = m * vch;
+    int warm = (pp - d - 1) * 2 + (vch - 1) * pp;
+    if (m == pp || warm > total) warm = total;
+    if (pos < warm) { bwd = false; nf = pos; nb = 0; }
+    else if (pos - warm < 2 * (total - warm)) { const int t = pos - warm; bwd = t & 1; nf = warm + (t + 1) / 2; nb = t / 2; }
+    else { bwd = true; nf = total; nb = pos - total; }
+    const int idx = bwd ? nb : nf;
+    const int c0 = (idx / pp) % vch;
+    c = bwd ? vch - 1 - c0 : c0;
+    j = (idx / (pp * vch)) * pp + idx % pp;
+}
+// ... and the words of the records of the device's first nf forward and nb backward items: of the
+// first n forward items, chunk c has (n / (pp v)) pp + clamp(n mod (pp v) - c pp, 0, pp); the
+// backward items take the chunks in reverse.
+__device__ __forceinline__ int64_t interleaved_words_before(const EmitPlan &p, int d, int nf, int nb)
+{
+    const int pp = p.pp, vch = p.v, cyc = pp * vch;
+    const int qf = nf / cyc, rf_ = nf - qf * cyc, qb = nb / cyc, rb_ = nb - qb * cyc;
+    int64_t recs = 0;
+    for (int c = 0; c < vch; ++c) {
+        const int s = c * pp + d;
+        const int cf = qf * pp + min(max(rf_ - c * pp, 0), pp);
+        const int cb = qb * pp + min(max(rb_ - (vch - 1 - c) * pp, 0), pp);
+        recs += (int64_t)cf * p.rf[s] + (int64_t)cb * p.rb[s];
+    }
+    return recs * 5;
+}
+
 __global__ void __launch_bounds__(kItemThreads)
 emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_t *__restrict__ op_start,
                   int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */,
@@ -402,19 +527,22 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     extern __shared__ __align__(16) int64_t dyn_s[];
     int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
     int64_t *img_b = dyn_s + cap;                       // the same word at img_b[x + 1]
-    int64_t *tmpl = dyn_s + 2 * cap + 2;                // [rf*5] forward, then [rb*5] backward
+    int64_t *tmpl = dyn_s + 2 * cap + 2;                // per chunk: [rf*5] forward, then [rb*5] backward
     __shared__ int64_t rep_off_s[kTileReplicas];
     __shared__ int64_t start_s[kMaxTileItems];          // start time of each item of the run
     __shared__ int64_t jit_s[kMaxTileItems];            // jitter at the start of each item
     __shared__ int32_t ioff[kMaxTileItems + 1];         // word offset of each item inside the run
-    __shared__ int32_t meta_s[kMaxTileItems];           // micro-batch << 1 | is-backward
+    __shared__ int32_t meta_s[kMaxTileItems];           // micro-batch << 6 | chunk << 1 | is-backward
+    __shared__ int32_t toff_s[DISTSIM_MAX_PP / 2][2];   // word offset of each chunk's forward / backward template
+    __shared__ int64_t run_base_s;                      // words of the device's records before the run
     const int i = blockIdx.y;
     const EmitPlan &p = plans[i];
     if (!p.ok) return;
-    const int m = p.m, pp = p.pp, sched = p.sched, mp = p.mp;
+    const int m = p.m, pp = p.pp, sched = p.sched, mp = p.mp, vch = p.v, P = pp * vch;
     const int reps = mp * p.dp;
     const int tile_items = p.tile_items;
-    const int item_chunks = (2 * m + tile_items - 1) / tile_items;
+    const int dev_items = 2 * m * vch;                  // items of a device
+    const int item_chunks = (dev_items + tile_items - 1) / tile_items;
     const int rep_chunks = (reps + kTileReplicas - 1) / kTileReplicas;
     int tile = blockIdx.x;
     if (tile >= pp * item_chunks * rep_chunks) return;
@@ -424,8 +552,6 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
 
     const Row &row = v.rows[p.row];
     const Entry &en = v.entries[p.entry];
-    const int a = p.bounds[d], e = p.bounds[d + 1];
-    const int rf = p.rf[d], rb = p.rb[d];
     const int64_t *pf = v.etf + (int64_t)p.entry * v.tc.lp;
     const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
     const int64_t *f = v.raw.fwd + (int64_t)en.cls * v.tc.n_layers;
@@ -433,46 +559,85 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     const int row_mp = row.mp, row_dp = row.dp;
     const int per_layer = row_mp > 1 ? 2 : 1;
     const int64_t ar = en.ar, a2a = en.a2a;
-    int64_t *tf = tmpl, *tb = tmpl + (int64_t)rf * 5;
     const int jr = v.tc.n_jitter > 0 ? 1 : 0;           // record 0 of an item is its jitter event
 
-    // ---- item templates: records relative to the end of the item's jitter event ----------
-    if (jr && threadIdx.x == 32) {
-        tf[0] = DISTSIM_JITTER_F; tf[1] = a; tf[2] = 0; tf[3] = 0; tf[4] = 0;
-        tb[0] = DISTSIM_JITTER_B; tb[1] = e - 1; tb[2] = 0; tb[3] = 0; tb[4] = 0;
-    }
-    for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
-        const bool ex = row_dp > 1 && v.raw.expert[l];
-        {   // forward: layers ascending
-            const int r = jr + (l - a) * per_layer + (row_dp > 1 ? v.pe[l] - v.pe[a] : 0);
-            int64_t t = pf[l] - pf[a];
-            int64_t *w = tf + (int64_t)r * 5;
-            w[0] = DISTSIM_COMPUTE_F; w[1] = l; w[2] = 0; w[3] = t; t += f[l]; w[4] = t; w += 5;
-            if (row_mp > 1) { w[0] = DISTSIM_MP_AR_F; w[1] = l; w[2] = 0; w[3] = t; t += ar; w[4] = t; w += 5; }
-            if (ex) { w[0] = DISTSIM_A2A_F; w[1] = l; w[2] = 0; w[3] = t; t += a2a; w[4] = t; }
+    // ---- item templates: records relative to the end of the item's jitter event; one pair of
+    //      templates per model chunk of the device (one without chunks) ----------------------
+    int tmpl_acc = 0;
+    for (int c = 0; c < vch; ++c) {
+        const int s = c * pp + d;                       // (virtual) stage
+        const int a = p.bounds[s], e = p.bounds[s + 1];
+        const int rf = p.rf[s], rb = p.rb[s];
+        int64_t *tf = tmpl + tmpl_acc, *tb = tf + (int64_t)rf * 5;
+        if (threadIdx.x == 0) { toff_s[c][0] = tmpl_acc; toff_s[c][1] = tmpl_acc + rf * 5; }
+        tmpl_acc += (rf + rb) * 5;
+        if (jr && threadIdx.x == 32) {
+            tf[0] = DISTSIM_JITTER_F; tf[1] = a; tf[2] = 0; tf[3] = 0; tf[4] = 0;
+            tb[0] = DISTSIM_JITTER_B; tb[1] = e - 1; tb[2] = 0; tb[3] = 0; tb[4] = 0;
         }
-        {   // backward: layers descending
-            const int r = jr + (e - 1 - l) * per_layer + (row_dp > 1 ? v.pe[e] - v.pe[l + 1] : 0);
-            int64_t t = pb[e] - pb[l + 1];
-            int64_t *w = tb + (int64_t)r * 5;
-            w[0] = DISTSIM_COMPUTE_B; w[1] = l; w[2] = 0; w[3] = t; t += g[l]; w[4] = t; w += 5;
-            if (row_mp > 1) { w[0] = DISTSIM_MP_AR_B; w[1] = l; w[2] = 0; w[3] = t; t += ar; w[4] = t; w += 5; }
-            if (ex) { w[0] = DISTSIM_A2A_B; w[1] = l; w[2] = 0; w[3] = t; t += a2a; w[4] = t; }
+        for (int l = a + threadIdx.x; l < e; l += blockDim.x) {
+            const bool ex = row_dp > 1 && v.raw.expert[l];
+            {   // forward: layers ascending
+                const int r = jr + (l - a) * per_layer + (row_dp > 1 ? v.pe[l] - v.pe[a] : 0);
+                int64_t t = pf[l] - pf[a];
+                int64_t *w = tf + (int64_t)r * 5;
+                w[0] = DISTSIM_COMPUTE_F; w[1] = l; w[2] = 0; w[3] = t; t += f[l]; w[4] = t; w += 5;
+                if (row_mp > 1) { w[0] = DISTSIM_MP_AR_F; w[1] = l; w[2] = 0; w[3] = t; t += ar; w[4] = t; w += 5; }
+                if (ex) { w[0] = DISTSIM_A2A_F; w[1] = l; w[2] = 0; w[3] = t; t += a2a; w[4] = t; }
+            }
+            {   // backward: layers descending
+                const int r = jr + (e - 1 - l) * per_layer + (row_dp > 1 ? v.pe[e] - v.pe[l + 1] : 0);
+                int64_t t = pb[e] - pb[l + 1];
+                int64_t *w = tb + (int64_t)r * 5;
+                w[0] = DISTSIM_COMPUTE_B; w[1] = l; w[2] = 0; w[3] = t; t += g[l]; w[4] = t; w += 5;
+                if (row_mp > 1) { w[0] = DISTSIM_MP_AR_B; w[1] = l; w[2] = 0; w[3] = t; t += ar; w[4] = t; w += 5; }
+                if (ex) { w[0] = DISTSIM_A2A_B; w[1] = l; w[2] = 0; w[3] = t; t += a2a; w[4] = t; }
+            }
+        }
+        if (threadIdx.x == 0) {
+            if (s < P - 1) {
+                int64_t *w = tf + (int64_t)(rf - 1) * 5;
+                const int64_t t = pf[e] - pf[a];
+                w[0] = DISTSIM_SEND_F; w[1] = e - 1; w[2] = 0; w[3] = t;
+                w[4] = t + (vch > 1 ? virtual_p2p_cost(v, row, en, s) : p2p_cost(row, en, d));
+            }
+            if (s > 0) {
+                int64_t *w = tb + (int64_t)(rb - 1) * 5;
+                const int64_t t = pb[e] - pb[a];
+                w[0] = DISTSIM_SEND_B; w[1] = a; w[2] = 0; w[3] = t;
+                w[4] = t + (vch > 1 ? virtual_p2p_cost(v, row, en, s - 1) : p2p_cost(row, en, d - 1));
+            }
         }
     }
     // ---- the run: its items' start times, kinds, micro-batches and word offsets ------------
-    // an item's offset follows from how many forward / backward items precede it in the run
+    // an item's offset follows from how many forward / backward items (of each chunk) precede it
     const int s0 = ic * tile_items;
-    const int n_items = min(2 * m, s0 + tile_items) - s0;
-    bool bwd0; int j0, nf0, nb0;
-    item_at(sched, pp, m, d, s0, bwd0, j0, nf0, nb0);
+    const int n_items = min(dev_items, s0 + tile_items) - s0;
+    int64_t base0;                                       // words of the device's records before the run
+    {
+        bool bwd0; int c0, j0, nf0, nb0;
+        if (vch > 1) {
+            interleaved_item_at(pp, vch, m, d, s0, bwd0, c0, j0, nf0, nb0);
+            base0 = interleaved_words_before(p, d, nf0, nb0);
+        } else {
+            item_at(sched, pp, m, d, s0, bwd0, j0, nf0, nb0);
+            base0 = ((int64_t)nf0 * p.rf[d] + (int64_t)nb0 * p.rb[d]) * 5;
+        }
+    }
     for (int k = threadIdx.x; k <= n_items; k += blockDim.x) {
-        bool bwd; int j, nf, nb;
-        item_at(sched, pp, m, d, s0 + k, bwd, j, nf, nb);           // k == n_items: one past the run
-        ioff[k] = ((nf - nf0) * rf + (nb - nb0) * rb) * 5;
+        bool bwd; int c = 0, j, nf, nb;
+        int64_t before;
+        if (vch > 1) {
+            interleaved_item_at(pp, vch, m, d, s0 + k, bwd, c, j, nf, nb);     // k == n_items: one past the run
+            before = interleaved_words_before(p, d, nf, nb);
+        } else {
+            item_at(sched, pp, m, d, s0 + k, bwd, j, nf, nb);
+            before = ((int64_t)nf * p.rf[d] + (int64_t)nb * p.rb[d]) * 5;
+        }
+        ioff[k] = (int)(before - base0);
         if (k < n_items) {
-            start_s[k] = op_start[(int64_t)i * op_words_per_cand + (int64_t)d * 2 * m + s0 + k];
-            meta_s[k] = (j << 1) | (bwd ? 1 : 0);
+            start_s[k] = op_start[(int64_t)i * op_words_per_cand + (int64_t)d * dev_items + s0 + k];
+            meta_s[k] = (j << 6) | (c << 1) | (bwd ? 1 : 0);
             jit_s[k] = jitter_of(v, bwd ? v.raw.jit_b : v.raw.jit_f, j, d);
         }
     }
@@ -489,18 +654,7 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         }
         rep_off_s[k] = off;
     }
-    if (threadIdx.x == 0) {
-        if (d < pp - 1) {
-            int64_t *w = tf + (int64_t)(rf - 1) * 5;
-            const int64_t t = pf[e] - pf[a];
-            w[0] = DISTSIM_SEND_F; w[1] = e - 1; w[2] = 0; w[3] = t; w[4] = t + p2p_cost(row, en, d);
-        }
-        if (d > 0) {
-            int64_t *w = tb + (int64_t)(rb - 1) * 5;
-            const int64_t t = pb[e] - pb[a];
-            w[0] = DISTSIM_SEND_B; w[1] = a; w[2] = 0; w[3] = t; w[4] = t + p2p_cost(row, en, d - 1);
-        }
-    }
+    if (threadIdx.x == 0) run_base_s = base0;
     __syncthreads();
 
     // ---- the run's image: one warp per item, a word is template word + {0, 0, j, start, start} ----
@@ -511,8 +665,8 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
         for (int it = warp; it < n_items; it += kItemThreads / 32) {
             const int off = ioff[it], len = ioff[it + 1] - off;
             const int meta = meta_s[it];
-            const int64_t *tp = (meta & 1) ? tb : tf;
-            const int64_t j = meta >> 1;
+            const int64_t *tp = tmpl + toff_s[(meta >> 1) & 31][meta & 1];
+            const int64_t j = meta >> 6;
             // the jitter event runs [start, start + jitter); every later event is relative to its end
             const int64_t t0 = start_s[it], t1 = t0 + (jr ? jit_s[it] : 0);
             int field = lane_field;                  // w mod 5, kept without dividing
@@ -535,8 +689,7 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     // past one.  Bulk copies need both ends 16-byte aligned: aligned replicas take img_a from word 0,
     // the others take img_b (the run shifted by one word) from word 1; single words at the ends are
     // stored directly.
-    int64_t *dst = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 +
-                   ((int64_t)nf0 * rf + (int64_t)nb0 * rb) * 5 + rep_off_s[threadIdx.x];
+    int64_t *dst = out + (p.rec_base + (int64_t)mp * p.stage_rec_prefix[d]) * 5 + run_base_s + rep_off_s[threadIdx.x];
     const bool odd = ((reinterpret_cast<uintptr_t>(dst) >> 3) & 1) != 0;
     const int head = odd ? 1 : 0;                    // words stored directly before the bulk copy
     const int bulk_words = (total - head) & ~1;
@@ -597,13 +750,18 @@ void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const 
     ++*launches;
 }
 
+int interleaved_words_of(int pp, int v) { return interleaved_words(pp, v); }
+
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,
-                      int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
+                      int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals, int ilv_words,
                       int64_t *launches)
 {
     cudaMemsetAsync(d_totals, 0, sizeof(EmitTotals), s);
-    emit_plan_kernel<<<(n + 3) / 4, 128, 0, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand, sums, d_totals);
+    const size_t plan_smem = (size_t)4 * ilv_words * sizeof(int64_t);
+    ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_plan_kernel), plan_smem);
+    emit_plan_kernel<<<(n + 3) / 4, 128, plan_smem, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand, sums, d_totals,
+                                                     ilv_words);
     ++*launches;
     if (offsets || busy || util) {
         const int64_t total = (int64_t)n * v.tc.n_devices + 1;

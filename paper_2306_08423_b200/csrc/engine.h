@@ -229,17 +229,19 @@ struct EmitPlan {                    // per selected candidate, written by the p
     int64_t rec_base;                // first record of the selection (after the scan)
     int64_t rec_total;               // records of all its devices
     int32_t row, entry, m, sched, pp, mp, dp, ok;
-    int32_t bounds[DISTSIM_MAX_PP + 1];
+    int32_t v, pad;                  // model chunks per device (1 unless interleaved 1F1B); then the arrays
+                                     // indexed "per stage" below are per virtual stage c * pp + d where noted
+    int32_t bounds[DISTSIM_MAX_PP + 1];              // per (virtual) stage
     int32_t tile_items;              // schedule items per block of the record kernel
     int32_t tmpl_words;              // words of the widest stage's forward + backward item templates
     int32_t run_words;               // upper bound on the words of any run of items of this selection
-    int32_t rf[DISTSIM_MAX_PP], rb[DISTSIM_MAX_PP];   // records of one forward / backward item
-    int64_t n_buckets[DISTSIM_MAX_PP];
+    int32_t rf[DISTSIM_MAX_PP], rb[DISTSIM_MAX_PP];   // records of one forward / backward item, per (virtual) stage
+    int64_t n_buckets[DISTSIM_MAX_PP];                // per device
     int64_t stage_recs[DISTSIM_MAX_PP];               // records of one device of stage d
     int64_t stage_rec_prefix[DISTSIM_MAX_PP + 1];
     int64_t busy[DISTSIM_MAX_PP];
     int64_t main_end[DISTSIM_MAX_PP];
-    int64_t last_b_start[DISTSIM_MAX_PP];
+    int64_t last_b_start[DISTSIM_MAX_PP];             // per (virtual) stage
 };
 // Totals over the planned selections (device words written by the scan kernel, read by the host).
 struct EmitTotals {
@@ -258,7 +260,9 @@ constexpr int kEmitSumWords = 8;
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
+                      int ilv_words /* shared-memory words a warp needs for the space's interleaved rows (0: none) */,
                       int64_t *launches);
+int interleaved_words_of(int pp, int v);           // those words for one row
 // out[k] = order-sensitive checksum of the records [offsets[k], offsets[k + 1]).
 void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const int64_t *offsets, int64_t n_lists,
                            uint64_t *out, int64_t *launches);

@@ -105,6 +105,36 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     else lockstep_block<1, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar, binom);
 }
 
+// Interleaved 1F1B candidates: a candidate per warp (interleaved.cuh).
+__global__ void __launch_bounds__(kIlvThreads)
+eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
+                        int64_t *__restrict__ busy_out, int words_per_warp)
+{
+    extern __shared__ __align__(16) int64_t ilv_s[];
+    __shared__ int64_t binom_s[512];
+    const int64_t *binom = stage_binom(v, binom_s, 512);
+    int wi = 0;
+    while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
+    const EvalWork &wk = batch.w[wi];
+    const Row row = v.rows[wk.row];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int64_t local = wk.lo + (int64_t)((int)blockIdx.x - wk.block_begin) * (kIlvThreads / 32) + warp;
+    const bool valid = local < wk.hi;
+    if (!valid) local = wk.hi - 1;                 // an idle warp shadows a real candidate
+    const CandidateCoords cc = split_local(row, local);
+    const Entry en = v.entries[cc.entry];
+    const IlvArrays A = interleaved_arrays(ilv_s + (int64_t)warp * words_per_warp, row.pp, row.v);
+    const IlvResult R = interleaved_candidate(v, row, en, cc, binom, A, nullptr);
+    if (!valid) return;
+    const int64_t out = row.offset + local - first;
+    if (lane == 0) batch_out[out] = R.batch;
+    if (busy_out) {
+        int64_t *bo = busy_out + out * v.sc.pp_max;
+        if (lane < row.pp) bo[lane] = R.busy;
+        for (int z = row.pp + lane; z < v.sc.pp_max; z += 32) bo[z] = 0;
+    }
+}
+
 // Work items collected for one kernel instance, launched when full or at the end.
 struct Pending {
     EvalBatch batch{};

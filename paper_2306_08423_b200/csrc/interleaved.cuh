@@ -51,35 +51,44 @@ __device__ __forceinline__ int64_t virtual_p2p_cost(const DeviceView &v, const R
     return row.mp * row.pp <= v.tc.gpus_per_node ? en.p2p_intra : en.p2p_inter;
 }
 
-__global__ void __launch_bounds__(kIlvThreads)
-eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
-                        int64_t *__restrict__ busy_out, int words_per_warp)
+// A candidate's arrays in the shared memory of its warp (see interleaved_words).
+struct IlvArrays {
+    int64_t *ring_f, *ring_b, *cost, *last_b, *tail;
+    int *cnt_f, *cnt_b, *bounds;
+    int kt;
+};
+__device__ __forceinline__ IlvArrays interleaved_arrays(int64_t *base, int pp, int vch)
 {
-    extern __shared__ __align__(16) int64_t ilv_s[];
-    __shared__ int64_t binom_s[512];
-    const int64_t *binom = stage_binom(v, binom_s, 512);
-    int wi = 0;
-    while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
-    const EvalWork &wk = batch.w[wi];
-    const Row row = v.rows[wk.row];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int64_t local = wk.lo + (int64_t)((int)blockIdx.x - wk.block_begin) * (kIlvThreads / 32) + warp;
-    const bool valid = local < wk.hi;
-    if (!valid) local = wk.hi - 1;                 // an idle warp shadows a real candidate
-    const CandidateCoords cc = split_local(row, local);
-    const Entry en = v.entries[cc.entry];
+    const int P = pp * vch;
+    IlvArrays A;
+    A.ring_f = base;
+    A.ring_b = A.ring_f + P * pp;
+    A.cost = A.ring_b + P * pp;                    // [2 s]: forward item of virtual stage s, [2 s + 1]: backward
+    A.last_b = A.cost + 2 * P;                     // start of the last backward item (micro-batch m - 1)
+    A.kt = interleaved_tail_items(pp, vch);
+    A.tail = A.last_b + P;                         // [device][item mod kt][start, end]
+    A.cnt_f = reinterpret_cast<int *>(A.tail + 2 * pp * A.kt);
+    A.cnt_b = A.cnt_f + P;
+    A.bounds = A.cnt_b + P;
+    return A;
+}
+
+// What a lane knows of its device after the evaluation.
+struct IlvResult { int64_t main_end, dp_end, busy, batch; };
+
+// Evaluates one interleaved candidate by the calling warp (all 32 lanes; lane d < pp owns device
+// d).  A: the warp's arrays; afterwards A.bounds, A.cost and A.last_b describe the candidate.
+// rec (nullable): item start times go to rec[d * 2 m v + position in the device's order].
+__device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, const Row &row, const Entry &en,
+                                                           const CandidateCoords &cc, const int64_t *binom,
+                                                           const IlvArrays &A, int64_t *rec)
+{
+    const int lane = threadIdx.x & 31;
     const int pp = row.pp, vch = row.v, P = pp * vch, m = en.m, L = v.tc.n_layers;
     const int log_pp = 31 - __clz(pp), log_v = 31 - __clz(vch);
-
-    int64_t *ring_f = ilv_s + (int64_t)warp * words_per_warp;
-    int64_t *ring_b = ring_f + P * pp;
-    int64_t *cost = ring_b + P * pp;               // [2 s]: forward item of virtual stage s, [2 s + 1]: backward
-    int64_t *last_b = cost + 2 * P;                // start of the last backward item (micro-batch m - 1)
-    const int kt = interleaved_tail_items(pp, vch);
-    int64_t *tail = last_b + P;                    // [device][item mod kt][start, end]
-    int *cnt_f = reinterpret_cast<int *>(tail + 2 * pp * kt);
-    int *cnt_b = cnt_f + P;
-    int *bounds = cnt_b + P;
+    int64_t *ring_f = A.ring_f, *ring_b = A.ring_b, *cost = A.cost, *last_b = A.last_b, *tail = A.tail;
+    int *cnt_f = A.cnt_f, *cnt_b = A.cnt_b, *bounds = A.bounds;
+    const int kt = A.kt;
 
     // ---- the partition into P virtual stages --------------------------------------------------
     if (v.sc.partition_mode == 0) {
@@ -152,6 +161,7 @@ eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *_
             free_at = start + cost[2 * s + (is_b ? 1 : 0)];
             int64_t *slot = tail + 2 * (d * kt + (n_f + n_b) % kt);
             slot[0] = start; slot[1] = free_at;
+            if (rec) rec[(int64_t)d * 2 * total + n_f + n_b] = start;
             if (is_b) {
                 ring_b[s * pp + (j & (pp - 1))] = free_at;
                 cnt_b[s] = j + 1;
@@ -169,7 +179,7 @@ eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *_
 
     // ---- gradient buckets: one stream per chunk, the chunk whose backward finishes first (the
     //      last one) first, chained on the device's one lane; then the reduction --------------
-    int64_t finish = 0, busy = 0;
+    IlvResult R{0, 0, 0, 0};
     if (d < pp) {
         const int64_t main_end = free_at;
         int64_t dp_end = main_end, extra = 0;       // extra: time the buckets run while the main lane is idle
@@ -195,21 +205,15 @@ eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *_
             }
             if (any) dp_end = end;
         }
-        for (int c = 0; c < vch; ++c) busy += (int64_t)m * (cost[2 * (c * pp + d)] + cost[2 * (c * pp + d) + 1]);
-        busy += extra;
-        finish = max64(main_end, dp_end);
+        for (int c = 0; c < vch; ++c) R.busy += (int64_t)m * (cost[2 * (c * pp + d)] + cost[2 * (c * pp + d) + 1]);
+        R.busy += extra;
+        R.main_end = main_end; R.dp_end = dp_end;
     }
-    int64_t mx = finish;
+    int64_t mx = max64(R.main_end, R.dp_end);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (!valid) return;
-    const int64_t out = row.offset + local - first;
-    if (lane == 0) batch_out[out] = mx;
-    if (busy_out) {
-        int64_t *bo = busy_out + out * v.sc.pp_max;
-        if (lane < pp) bo[lane] = busy;
-        for (int z = pp + lane; z < v.sc.pp_max; z += 32) bo[z] = 0;
-    }
+    R.batch = mx;
+    return R;
 }
 
 }  // namespace distsim

@@ -223,6 +223,10 @@ def test_interleaved_1f1b_every_candidate(E, ctx, case):
         assert (out.cpu().numpy() == ob[first:first + count]).all()
     cells, _ = E.distsim_testing_space_cells(ctx)
     assert cells == W.count_candidates_and_cells(w.table, w.space)[1]
+    # every record of the timelines of interleaved candidates (and some of the others beside them)
+    ilv = [i for i, c in enumerate(cands) if c.sched == 3]
+    pick = ilv[:: max(1, len(ilv) // 14)][:14] + [ilv[-1], 0, n - 1]
+    check_emission(E, ctx, w, pick)
 
 
 def test_interleaved_1f1b_on_the_64_device_shape(E, ctx):
@@ -242,12 +246,9 @@ def test_interleaved_1f1b_on_the_64_device_shape(E, ctx):
     assert (gb == ob).all(), idx[np.argwhere(gb != ob)[:5, 0]]
     bi, bt = E.distsim_argmin(ctx, batch, 0, n)
     assert oracle.eval_indices(w.table, w.space, np.array([bi]))[0][0] == bt == int(batch.min().item())
-    # timelines of interleaved candidates are refused for now, with a clear code; the rest still emits
-    ilv = int(idx[[c.sched == 3 for c in cands].index(True)])
-    with pytest.raises(E.DistsimError) as ei:
-        E.distsim_emit_timelines(ctx, torch.tensor([0, ilv], dtype=torch.int64, device="cuda"), 2, None, 0)
-    assert ei.value.code == E.E_UNSUPPORTED
-    check_emission(E, ctx, w, [0, int(idx[3])] if cands[3].sched != 3 else [0])
+    # timelines: interleaved candidates with few and many micro-batches, one of the others beside them
+    ilv = [int(i) for i, c in zip(idx, cands) if c.sched == 3]
+    check_emission(E, ctx, w, [ilv[0], ilv[len(ilv) // 2], ilv[-1], 0])
 
 
 @pytest.mark.parametrize("case", range(12))
