@@ -663,7 +663,7 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     *h_total_records = totals->records;
     if (d_records) {
         if (totals->records > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");
-        launch_emit_records(s, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
+        launch_emit_records(s, ctx->side, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
                             ctx->op_words_per_cand, *totals, d_records, &ctx->launches);
         CU(cudaGetLastError(), "emission launch");
     }

@@ -770,7 +770,7 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
     }
 }
 
-void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
+void launch_emit_records(cudaStream_t s, const SideStream &ss, const DeviceView &v, int n, const EmitPlan *plans,
                          const int64_t *op_start, int64_t op_words_per_cand, const EmitTotals &t,
                          distsim_record *records, int64_t *launches)
 {
@@ -780,17 +780,27 @@ void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitP
     const size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
     ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_items_kernel), smem);
     int64_t *out = reinterpret_cast<int64_t *>(records);
-    emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
-        v, plans, op_start, op_words_per_cand, out, cap);
-    ++*launches;
     if (t.bucket_tiles > 0 && t.bucket_recs > 0) {
         // an odd number of buckets per image keeps both images 16-byte aligned
         const int run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun) | 1;
         const size_t bsmem = (size_t)(2 * (run * 5 + 1) + 2 * (DISTSIM_MAX_LAYERS + 1)) * sizeof(int64_t);
         ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_buckets_kernel), bsmem);
-        emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, s>>>(v, plans, out, run);
+        // the bucket records are few and their blocks wait more than they write: on the side
+        // stream they run beside the item kernel (both only read the plans and write disjoint records)
+        cudaStream_t bs = s;
+        if (ss.side[0]) {
+            cudaEventRecord(ss.fork, s);                 // recorded before the item kernel below is enqueued
+            cudaStreamWaitEvent(ss.side[0], ss.fork, 0);
+            bs = ss.side[0];
+        }
+        emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, bs>>>(v, plans, out, run);
         ++*launches;
+        if (ss.side[0]) cudaEventRecord(ss.join[0], ss.side[0]);
     }
+    emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
+        v, plans, op_start, op_words_per_cand, out, cap);
+    ++*launches;
+    if (t.bucket_tiles > 0 && t.bucket_recs > 0 && ss.side[0]) cudaStreamWaitEvent(s, ss.join[0], 0);
 }
 
 }  // namespace distsim

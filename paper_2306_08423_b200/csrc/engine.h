@@ -266,7 +266,7 @@ int interleaved_words_of(int pp, int v);           // those words for one row
 // out[k] = order-sensitive checksum of the records [offsets[k], offsets[k + 1]).
 void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const int64_t *offsets, int64_t n_lists,
                            uint64_t *out, int64_t *launches);
-void launch_emit_records(cudaStream_t s, const DeviceView &v, int n, const EmitPlan *plans,
+void launch_emit_records(cudaStream_t s, const SideStream &ss, const DeviceView &v, int n, const EmitPlan *plans,
                          const int64_t *op_start, int64_t op_words_per_cand, const EmitTotals &totals,
                          distsim_record *records, int64_t *launches);
 
