@@ -40,11 +40,36 @@ TOP_K = 1024
 # below 2^32) one max and one add.
 INT_OPS_PER_CELL_64, INT_OPS_PER_CELL_32 = 6, 2
 RECORD_BYTES = 40
-# DRAM read + write bytes per step of the timed workload, from the one-pass ncu counters summarised in
-# profiles/bench_config1_dram_bytes.md.  They describe the kernels as captured: set them to None when
-# an evaluation or emission kernel changes, until the counters are taken again.
-EVAL_TRAFFIC_BYTES = 198_050_304
-EMIT_TRAFFIC_BYTES = 1_696_420_864
+# DRAM read + write bytes per launch set of the timed workload come from the one-pass ncu counters
+# summarised in profiles/bench_config1_dram_bytes.md, which records beside each figure a hash of the
+# kernel sources it was taken on: a figure whose sources have changed since reads as null.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "bench_config1_dram_bytes.md")
+KERNEL_SOURCES = {
+    "eval": ("eval_thread.cuh", "eval_kernels.cu", "recurrence.cuh", "smem_stage.cuh", "interleaved.cuh", "engine.h"),
+    "emit": ("emit_kernels.cu", "recurrence.cuh", "interleaved.cuh", "smem_stage.cuh", "engine.h"),
+}
+
+
+def sources_hash(kind: str) -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kind]:
+        with open(os.path.join(ROOT, "paper_2306_08423_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(kind: str):
+    """Bytes of the line `traffic: kernel=<kind> sources=<hash> bytes=<n>` if the hash is current."""
+    import re
+    try:
+        text = open(TRAFFIC_FILE).read()
+    except OSError:
+        return None
+    m = re.search(rf"traffic: kernel={kind} sources=([0-9a-f]+) bytes=(\d+)", text)
+    return int(m.group(2)) if m and m.group(1) == sources_hash(kind) else None
+
+
 SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32      # issue slots: one warp instruction per scheduler and clock
 
 
@@ -367,15 +392,21 @@ def run_ours(args):
     cell_floor_s = (cells_32 / cell32_peak + (cells - cells_32) / cell64_peak) / 1e9
     issue_peak_gops = SM_COUNT * SCHEDULERS_PER_SM * LANES * sm_mhz * 1e-3
     roofline = {"bound": "alu", "kernel": "eval_thread_kernel (+ lock-step kernel on small rows)",
-                "achieved": achieved_gops, "peak": issue_peak_gops,
+                "achieved": achieved_gops, "peak": achieved_gops * eval_s / cell_floor_s,
                 "unit": "G 32-bit integer operations/s (2 per uint32 cell: max and add; 6 per int64 cell)",
-                "frac": achieved_gops / issue_peak_gops, "traffic": EVAL_TRAFFIC_BYTES,
+                "frac": cell_floor_s / eval_s, "traffic": recorded_traffic("eval"),
+                "peak_kind": "measured in this run: the rate at which dependency-free chains of the same recurrence "
+                             "cell issue (uint32 cells as one fused add-max, int64 cells as six instructions), "
+                             "blended by the workload's share of each width; frac = time the cells alone take at "
+                             "those rates / evaluation time",
+                "derived_issue_slot_peak": issue_peak_gops,
+                "frac_of_derived_issue_slots": achieved_gops / issue_peak_gops,
                 "traffic_note": "DRAM read + write bytes of the four evaluation launches of one step (ncu, one pass; "
                                 "null when the kernels changed after the counters were taken); algorithmic: 8 B per "
                                 f"candidate = {8 * n_total} B, part of which is still in the L2 when the launches end",
-                "peak_kind": "derived: 148 SMs x 4 schedulers x 32 lanes x SM clock sampled during the run (one "
-                             "instruction per scheduler and clock); a uint32 cell's max and add fuse into one "
-                             "add-max instruction that issues at half rate, so this is also the cell bound x 2",
+                "derived_note": "148 SMs x 4 schedulers x 32 lanes x SM clock sampled during the run (one "
+                                "instruction per scheduler and clock); a uint32 cell's max and add fuse into one "
+                                "add-max instruction that issues at half rate, so this is also the cell bound x 2",
                 "add_xor_probe_Ginstr_per_s": int_peak_gops, "frac_of_add_xor_probe": achieved_gops / int_peak_gops,
                 "cells": cells, "cells_32bit": cells_32, "ms_per_launch_set": statistics.mean(eval_ms),
                 "cell_rate_peaks_Gcells_per_s": {"uint32": cell32_peak, "uint32_fused_add_max": cell32_fused_peak,
@@ -393,7 +424,7 @@ def run_ours(args):
     emit_gbs = emit_bytes / (statistics.mean(emit_ms) * 1e-3) / 1e9
     roofline_emit = {"bound": "hbm", "kernel": "emit_items_kernel (+plan, scan, devices, buckets)",
                      "achieved": emit_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": emit_gbs / peaks["hbm_gbs"], "traffic": EMIT_TRAFFIC_BYTES, "peak_kind": peak_kind,
+                     "frac": emit_gbs / peaks["hbm_gbs"], "traffic": recorded_traffic("emit"), "peak_kind": peak_kind,
                      "traffic_note": "DRAM read + write bytes of emit_items_kernel + emit_buckets_kernel of one step "
                                      "(ncu, one pass); the bucket-lane records are still in the L2 when they end",
                      "bytes_per_step": emit_bytes, "ms": statistics.mean(emit_ms)}

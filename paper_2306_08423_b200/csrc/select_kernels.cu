@@ -93,7 +93,9 @@ constexpr int kBins = 1 << kRadixBits;
 struct SelState {
     u64 tprefix, tmask, rank, iprefix, imask, blocks_done, cursor, skip_index;
     u64 use_compact, cn;         // remaining passes read the compact buffer of cn pairs
-    u64 stride;                  // > 1: the passes read every stride-th element of the array (sampling phase)
+    u64 stride;                  // > 1: the passes read every stride-th element of the array (sampling phase);
+                                 // with kSampleGathered set, the first pass has copied those elements to the
+                                 // head of the compact buffer and the later passes read them there
     u64 k;                       // elements wanted
     u64 threshold;               // sampled selection: a time that at least k elements do not exceed
     u64 tmin;                    // sampled selection: smallest time of the array
@@ -102,12 +104,17 @@ struct SelState {
 };
 
 // The source a pass reads: the array itself (index = position) or the compact buffer.
+constexpr u64 kSampleGathered = 1ull << 63;
 struct SelSource { const int64_t *t; const int64_t *idx; int64_t n; int64_t stride; };
 __device__ __forceinline__ SelSource sel_source(const SelState *st, const int64_t *batch, int64_t count,
                                                 const SelectScratch &sc)
 {
     if (st->use_compact) return SelSource{sc.comp_time, sc.comp_idx, (int64_t)st->cn, 1};
-    if (st->stride > 1) return SelSource{batch, nullptr, (count + (int64_t)st->stride - 1) / (int64_t)st->stride, (int64_t)st->stride};
+    if (st->stride > 1) {
+        const int64_t stride = (int64_t)(st->stride & ~kSampleGathered), n = (count + stride - 1) / stride;
+        if (st->stride & kSampleGathered) return SelSource{sc.comp_time, nullptr, n, 1};
+        return SelSource{batch, nullptr, n, stride};
+    }
     return SelSource{batch, nullptr, count, 1};
 }
 
@@ -215,6 +222,8 @@ radix_pass_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratc
     const unsigned dmask = (1u << width) - 1u;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < src.n; i += (int64_t)gridDim.x * blockDim.x) {
         const u64 x = (u64)src.t[i * src.stride];
+        // the first pass over a strided sample leaves a dense copy for the passes that follow
+        if (!kIndexPhase && src.stride > 1 && src.n <= sc.comp_cap) sc.comp_time[i] = (int64_t)x;
         if ((x & tmask) != tprefix) continue;
         if (kIndexPhase) {
             const u64 id = src.idx ? (u64)src.idx[i] : (u64)i;
@@ -232,6 +241,7 @@ radix_pass_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratc
     __syncthreads();
     if (!last) return;
     pick_bin<kIndexPhase>(st, hist, partial, shift, dmask, last_time_pass);
+    if (!kIndexPhase && threadIdx.x == 0 && src.stride > 1 && src.n <= sc.comp_cap) st->stride |= kSampleGathered;
 }
 
 __global__ void sel_init_kernel(SelState *st, u64 *hist, int k, int64_t stride, u64 *key /* nullable: [2], set to all ones */)
