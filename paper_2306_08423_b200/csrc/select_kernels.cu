@@ -262,43 +262,73 @@ __global__ void sel_init_kernel(SelState *st, u64 *hist, int k, int64_t stride, 
 // the elements not fit it (masses of ties), the array itself.
 __global__ void __launch_bounds__(kSelThreads)
 scan_select_kernel(const int64_t *__restrict__ batch, int64_t count, SelectScratch sc, int idx_bits, int want_min,
-                   int want_compact)
+                   int want_compact, int low_bits /* time bits the sampling passes left open */)
 {
     __shared__ bool last;
+    // Elements up to the threshold are few (about k times the sampling stride out of the whole
+    // array, a few hundred per block), but one counter in global memory cannot take an atomic
+    // for each: a block collects its own in shared memory and takes one range of the compact
+    // buffer at its end; what does not fit the block's buffer goes there directly.
+    constexpr int kHeld = 512;
+    __shared__ int64_t held_t[kHeld], held_i[kHeld];
+    __shared__ unsigned int n_held;
+    __shared__ u64 held_base;
+    if (threadIdx.x == 0) n_held = 0;
+    __syncthreads();
     SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
-    const u64 threshold = want_compact ? st->tprefix : 0;
-    u64 best = ~0ull, xmin = ~0ull;
-    // eight independent loads in flight per thread; elements up to the threshold are few (about k
-    // times the sampling stride out of the whole array), so each takes its own atomic
-    constexpr int kUnroll = 8;
+    const u64 threshold = want_compact ? (st->tprefix | ((1ull << low_bits) - 1ull)) : 0;
+    // A thread meets its elements in ascending position, so "strictly smaller" keeps the first
+    // of equal times: (xmin, imin) is the thread's smallest (time, position) pair.
+    u64 xmin = ~0ull;
+    int64_t imin = 0;
+    auto consider = [&](u64 x, int64_t i) {
+        if (x < xmin) { xmin = x; imin = i; }
+        if (want_compact && x <= threshold) {
+            const unsigned int h = atomicAdd(&n_held, 1u);
+            if (h < (unsigned)kHeld) { held_t[h] = (int64_t)x; held_i[h] = i; }
+            else {
+                const u64 pos = atomicAdd(&st->cursor, 1ull);
+                if (pos < (u64)sc.comp_cap) { sc.comp_time[pos] = (int64_t)x; sc.comp_idx[pos] = i; }
+            }
+        }
+    };
+    // 16-byte loads of pairs (the array from its first 16-byte boundary on), four of them in
+    // flight per thread; the element before that boundary and an odd last one go to one thread
+    const int64_t head = (count > 0 && (reinterpret_cast<uintptr_t>(batch) & 15)) ? 1 : 0;
+    const int64_t n_pairs = (count - head) >> 1;
+    const bool edges = blockIdx.x == 0 && threadIdx.x == 0;
+    if (edges && head) consider((u64)batch[0], 0);
+    const longlong2 *pairs = reinterpret_cast<const longlong2 *>(batch + head);
+    constexpr int kUnroll = 4;
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < count; i0 += step * kUnroll) {
-        u64 x[kUnroll];
+    for (int64_t p0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p0 < n_pairs; p0 += step * kUnroll) {
+        longlong2 x[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            const int64_t i = i0 + u * step;
-            x[u] = i < count ? (u64)__ldcs(batch + i) : ~0ull;
+            const int64_t p = p0 + u * step;
+            if (p < n_pairs) x[u] = __ldcs(pairs + p);
         }
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            const int64_t i = i0 + u * step;
-            if (i >= count) continue;
-            xmin = x[u] < xmin ? x[u] : xmin;
-            if (want_min) {
-                const u64 key = (x[u] << idx_bits) | (u64)i;
-                best = key < best ? key : best;
-            }
-            if (want_compact && x[u] <= threshold) {
-                const u64 pos = atomicAdd(&st->cursor, 1ull);
-                if (pos < (u64)sc.comp_cap) { sc.comp_time[pos] = (int64_t)x[u]; sc.comp_idx[pos] = i; }
-            }
+            const int64_t p = p0 + u * step;
+            if (p >= n_pairs) break;
+            consider((u64)x[u].x, head + 2 * p);
+            consider((u64)x[u].y, head + 2 * p + 1);
         }
     }
+    if (edges && head + 2 * n_pairs < count) consider((u64)batch[count - 1], count - 1);
     if (want_min) {
+        u64 best = xmin != ~0ull ? (xmin << idx_bits) | (u64)imin : ~0ull;
         best = block_min_u64(best);
         if (threadIdx.x == 0 && best != ~0ull) atomicMin(sc.key, best);
     }
     if (!want_compact) return;
+    __syncthreads();
+    const unsigned int n_mine = n_held < (unsigned)kHeld ? n_held : (unsigned)kHeld;
+    if (threadIdx.x == 0 && n_mine) held_base = atomicAdd(&st->cursor, (u64)n_mine);
+    __syncthreads();
+    for (unsigned int h = threadIdx.x; h < n_mine; h += blockDim.x)
+        if (held_base + h < (u64)sc.comp_cap) { sc.comp_time[held_base + h] = held_t[h]; sc.comp_idx[held_base + h] = held_i[h]; }
     xmin = block_min_u64(xmin);
     if (threadIdx.x == 0 && xmin != ~0ull) atomicMin(&st->tmin, xmin);
     __threadfence();
@@ -375,7 +405,27 @@ __device__ __forceinline__ void bitonic_sort_pairs(int64_t *st, int64_t *si, int
                     const int64_t y = si[a]; si[a] = si[b]; si[b] = y;
                 }
             }
-            __syncthreads();
+            // a step of stride <= 32 exchanges inside aligned groups of 64 elements, each the work
+            // of one warp (comparator i belongs to thread i mod 1024, group to warp i / 32 mod 32)
+            const int next = stride > 1 ? stride >> 1 : size;
+            if (stride >= 64 || next >= 64) __syncthreads(); else __syncwarp();
+        }
+}
+
+// The same on packed keys (time << idx_bits | index): half the shared-memory traffic.
+__device__ __forceinline__ void bitonic_sort_keys(u64 *key, int np2)
+{
+    for (int size = 2; size <= np2; size <<= 1)
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int i = threadIdx.x; i < np2 / 2; i += blockDim.x) {
+                const int a = 2 * i - (i & (stride - 1));
+                const int b = a + stride;
+                const bool up = (a & size) == 0;
+                const u64 x = key[a], y = key[b];
+                if ((x > y) == up) { key[a] = y; key[b] = x; }
+            }
+            const int next = stride > 1 ? stride >> 1 : size;
+            if (stride >= 64 || next >= 64) __syncthreads(); else __syncwarp();
         }
 }
 
@@ -386,7 +436,8 @@ __device__ __forceinline__ void bitonic_sort_pairs(int64_t *st, int64_t *si, int
 constexpr int kSortMax = 4096;
 __global__ void __launch_bounds__(1024)
 sort_pairs_kernel(const int64_t *__restrict__ ct, const int64_t *__restrict__ ci, int n_in, int k,
-                  int64_t first, int64_t *out_idx, int64_t *out_time, const SelState *state)
+                  int64_t first, int64_t *out_idx, int64_t *out_time, const SelState *state,
+                  int idx_bits /* > 0: time and index fit one 64-bit key with this many index bits */)
 {
     extern __shared__ __align__(16) unsigned char sm[];
     int64_t *st = reinterpret_cast<int64_t *>(sm);
@@ -395,8 +446,20 @@ sort_pairs_kernel(const int64_t *__restrict__ ct, const int64_t *__restrict__ ci
         if (!state->small) return;
         n_in = (int)state->n_cand;
     }
-    int np2 = 1;
+    int np2 = 64;                        // whole groups of 64 (see the sort's barriers)
     while (np2 < n_in) np2 <<= 1;
+    if (idx_bits > 0) {
+        u64 *key = reinterpret_cast<u64 *>(sm);
+        for (int i = threadIdx.x; i < np2; i += blockDim.x)
+            key[i] = i < n_in ? ((u64)ct[i] << idx_bits) | (u64)(ci ? ci[i] : (int64_t)i) : ~0ull;
+        __syncthreads();
+        bitonic_sort_keys(key, np2);
+        for (int i = threadIdx.x; i < k; i += blockDim.x) {
+            out_idx[i] = first + (int64_t)(key[i] & ((1ull << idx_bits) - 1ull));
+            if (out_time) out_time[i] = (int64_t)(key[i] >> idx_bits);
+        }
+        return;
+    }
     for (int i = threadIdx.x; i < np2; i += blockDim.x) {
         st[i] = i < n_in ? ct[i] : INT64_MAX;
         si[i] = i < n_in ? (ci ? ci[i] : (int64_t)i) : INT64_MAX;
@@ -571,13 +634,15 @@ int time_bits(int64_t time_bound)
 }
 
 // Radix passes over all time digits (most significant first) of the current source.
+// min_shift > 0 leaves the digits below that bit open: the prefix found is then the top of a
+// range of times, not one time.
 void time_passes(cudaStream_t s, const int64_t *batch, int64_t count, int64_t n_source, int64_t time_bound,
-                 const SelectScratch &sc, bool compact_after_first, int64_t *launches)
+                 const SelectScratch &sc, bool compact_after_first, int64_t *launches, int min_shift = 0)
 {
     const int g = grid_for(n_source);
     const int tb = time_bits(time_bound);
     bool first_pass = true;
-    for (int shift = ((tb + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= 0; shift -= kRadixBits) {
+    for (int shift = ((tb + kRadixBits - 1) / kRadixBits - 1) * kRadixBits; shift >= min_shift; shift -= kRadixBits) {
         const int width = tb - shift < kRadixBits ? tb - shift : kRadixBits;
         radix_pass_kernel<false><<<g, kSelThreads, 0, s>>>(batch, count, sc, shift, width, shift == 0);
         ++*launches;
@@ -602,7 +667,7 @@ void finish_passes(cudaStream_t s, const int64_t *batch, int64_t first, int64_t 
         ++*launches;
     }
     collect_kernel<<<g, kSelThreads, 0, s>>>(batch, count, sc, k, 0);
-    sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, k, k, first, d_indices, d_times, nullptr);
+    sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, k, k, first, d_indices, d_times, nullptr, 0);
     *launches += 2;
 }
 
@@ -662,7 +727,7 @@ void launch_select(cudaStream_t s, const int64_t *batch, int64_t first, int64_t 
         if (d_result) launch_argmin(s, batch, count, time_bound, sc, d_result, launches);
         if (k == 0) return;
         if (count <= kSortMax) {
-            sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(batch, nullptr, (int)count, k, first, d_indices, d_times, nullptr);
+            sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(batch, nullptr, (int)count, k, first, d_indices, d_times, nullptr, 0);
             ++*launches;
             return;
         }
@@ -682,9 +747,13 @@ void launch_select(cudaStream_t s, const int64_t *batch, int64_t first, int64_t 
     sel_init_kernel<<<1, 256, 0, s>>>(reinterpret_cast<SelState *>(sc.sel_state), sc.hist, k, stride,
                                       min_here ? sc.key : nullptr);
     ++*launches;
-    time_passes(s, batch, count, n_sample, time_bound, sc, false, launches);
+    //    The last digit of the times is left open when there are two digits above it: the threshold
+    //    is then the top of the 2048-wide range of times that holds the sample's k-th smallest -
+    //    still a time that k elements do not exceed, for one pass over the sample less.
+    const int low_bits = time_bits(time_bound) > 2 * kRadixBits ? kRadixBits : 0;
+    time_passes(s, batch, count, n_sample, time_bound, sc, false, launches, low_bits);
     // 2. one pass: minimum of the packed key, elements up to that time into the compact buffer
-    scan_select_kernel<<<grid_for(count), kSelThreads, 0, s>>>(batch, count, sc, idx_bits, min_here ? 1 : 0, 1);
+    scan_select_kernel<<<grid_for(count), kSelThreads, 0, s>>>(batch, count, sc, idx_bits, min_here ? 1 : 0, 1, low_bits);
     ++*launches;
     if (min_here) {
         argmin_unpack_kernel<<<1, 32, 0, s>>>(sc.key, idx_bits, 1, d_result);
@@ -697,9 +766,11 @@ void launch_select(cudaStream_t s, const int64_t *batch, int64_t first, int64_t 
     //    one histogram over its range of times cuts it down to what one sort takes
     const int64_t n_expect = (int64_t)k * stride * 4 < count ? (int64_t)k * stride * 4 : count;
     SelState *st = reinterpret_cast<SelState *>(sc.sel_state);
-    refine_kernel<<<grid_for(n_expect), kSelThreads, 0, s>>>(sc);
-    collect_kernel<<<grid_for(n_expect), kSelThreads, 0, s>>>(batch, count, sc, kSortMax, 1);
-    sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, 0, k, first, d_indices, d_times, st);
+    const int g_small = grid_for(n_expect) < 148 ? grid_for(n_expect) : 148;     // a block's histogram costs more than its elements
+    refine_kernel<<<g_small, kSelThreads, 0, s>>>(sc);
+    collect_kernel<<<g_small, kSelThreads, 0, s>>>(batch, count, sc, kSortMax, 1);
+    sort_pairs_kernel<<<1, 1024, sort_smem, s>>>(sc.cand_time, sc.cand_idx, 0, k, first, d_indices, d_times, st,
+                                         packed ? idx_bits : 0);
     // ... and the general kernel for what that path cannot finish (it returns at once otherwise)
     const size_t gen_smem = sort_smem + (size_t)kBins * sizeof(u64);
     ensure_dynamic_smem(reinterpret_cast<const void *>(&general_select_kernel), gen_smem);

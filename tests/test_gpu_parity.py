@@ -840,6 +840,19 @@ def test_two_pass_argmin_for_wide_times(E, ctx):
     E.distsim_topk(ctx, big, 0, big.numel(), k, ki, kt)
     st, si = torch.sort(big, stable=True)
     assert (kt == st[:k]).all() and (ki == si[:k]).all()
+    # the one pass over a long array reads 16-byte pairs: arrays that start off a 16-byte
+    # boundary, of odd and even length, with distinct times so that the refined path is taken
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    distinct = torch.randperm((1 << 21) + 3, generator=gen, device="cuda").to(torch.int64) * 1000 + 17
+    for off, length in ((1, (1 << 21) + 1), (1, 1 << 21), (0, (1 << 21) + 1), (2, 1 << 21)):
+        view = distinct[off:off + length]
+        st, si = torch.sort(view, stable=True)
+        for k in (1, 1024, 4096):
+            ki, kt = dev(k), dev(k)
+            E.distsim_topk(ctx, view, 0, length, k, ki, kt)
+            assert (kt == st[:k]).all() and (ki == si[:k]).all(), (off, length, k)
+        bi, bt = E.distsim_argmin(ctx, view, 0, length)
+        assert (bt, bi) == (int(st[0]), int(si[0]))
 
 
 def test_api_errors(E, ctx):
