@@ -226,16 +226,19 @@ def run_ours(args):
     busy = torch.empty(emit_n * N, dtype=torch.int64, device=dev)
     util = torch.empty(emit_n * N, dtype=torch.float64, device=dev)
 
+    loc_i_k, loc_t_k = loc_i[:k_loc], loc_t[:k_loc]                  # views made once, outside the timed steps
+    top_mine = top_i[emit_first:emit_first + emit_n]
+
     def search():
         """Evaluation, best candidate and the 1024 fastest in one asynchronous call; with the
         search split over ranks, the ranks' lists are gathered and merged on every rank."""
-        E.distsim_eval_select(ctx, my_first, my_count, batch, k_loc, loc_i[:k_loc], loc_t[:k_loc], d_best, to_host=False)
+        E.distsim_eval_select(ctx, my_first, my_count, batch, k_loc, loc_i_k, loc_t_k, d_best, to_host=False)
         if merging:
             gt, gi = sharding.gather_topk_lists(loc_t, loc_i)
             E.distsim_merge_topk(ctx, gt, gi, gt.numel(), TOP_K, top_i, top_t)
 
     def emit(rec, cap):
-        return E.distsim_emit_timelines(ctx, top_i[emit_first:emit_first + emit_n], emit_n, rec, cap, offsets, busy, util)
+        return E.distsim_emit_timelines(ctx, top_mine, emit_n, rec, cap, offsets, busy, util)
 
     flush = torch.empty(256 * 2**20, dtype=torch.uint8, device=dev)          # > L2 (126 MB)
 

@@ -79,6 +79,7 @@ struct distsim_ctx {
     // scratch
     DevBuf d_status, d_sel, d_result, d_plans, d_plan_sums, d_op_start, d_totals, d_batch, d_topk;
     SideStream side;                      // extra streams of an evaluation (lock-step launches)
+    cudaEvent_t planned = nullptr;        // recorded behind the emission-planning kernel
     int64_t *h_pinned = nullptr;          // 16 words of pinned host memory for small results:
                                           // [0..3] results, [4] status, [8..15] emission totals
 
@@ -155,12 +156,17 @@ const char *const kTimeoutText =
 // Reads and clears the device status word; synchronises the stream.  A wait that gave up while
 // the copy still completed before its block went on is advisory: *stalled is set and DISTSIM_OK
 // returned, so that the caller can finish its work and report DISTSIM_E_TIMEOUT with valid outputs.
+int take_status(distsim_ctx *ctx, cudaStream_t s, int32_t code, bool *stalled);
 int read_status(distsim_ctx *ctx, cudaStream_t s, bool *stalled)
 {
     int32_t *st = reinterpret_cast<int32_t *>(ctx->h_pinned + 4);
     CU(cudaMemcpyAsync(st, ctx->d_status.p, sizeof(int32_t), cudaMemcpyDeviceToHost, s), "status read");
     CU(cudaStreamSynchronize(s), "status sync");
-    const int32_t code = *st;
+    return take_status(ctx, s, *st, stalled);
+}
+// Acts on a status word read from the device (and clears the device's copy if it is set).
+int take_status(distsim_ctx *ctx, cudaStream_t s, int32_t code, bool *stalled)
+{
     if (code != 0) {
         cudaMemsetAsync(ctx->d_status.p, 0, sizeof(int32_t), s);
         if (code == DISTSIM_E_TIMEOUT) { *stalled = true; return DISTSIM_OK; }
@@ -204,8 +210,9 @@ int distsim_create(distsim_ctx **out, int cuda_device)
         ctx->d_status.reserve(64) != cudaSuccess ||
         ctx->d_sel.reserve((8 + 2048 + 16 + 2 * 4096 + 2 * kCompactCap) * sizeof(int64_t)) != cudaSuccess ||
         ctx->d_result.reserve(64) != cudaSuccess || ctx->d_totals.reserve(64) != cudaSuccess ||
-        cudaMemset(ctx->d_status.p, 0, 64) != cudaSuccess ||
-        cudaMallocHost(&ctx->h_pinned, 16 * sizeof(int64_t)) != cudaSuccess) {
+        cudaMemset(ctx->d_status.p, 0, 64) != cudaSuccess || cudaMemset(ctx->d_totals.p, 0, 64) != cudaSuccess ||
+        cudaHostAlloc(&ctx->h_pinned, 16 * sizeof(int64_t), cudaHostAllocMapped) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->planned, cudaEventDisableTiming) != cudaSuccess) {
         distsim_destroy(ctx);
         return DISTSIM_E_CUDA;
     }
@@ -227,6 +234,7 @@ void distsim_destroy(distsim_ctx *ctx)
     if (!ctx) return;
     cudaSetDevice(ctx->device);
     for (cudaEvent_t e : ctx->phase_ev) if (e) cudaEventDestroy(e);
+    if (ctx->planned) cudaEventDestroy(ctx->planned);
     if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
     destroy_side(ctx->side);
     delete ctx;
@@ -653,13 +661,15 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     const DeviceView v = ctx->view();
     launch_emit_plan(s, v, d_indices, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
                      ctx->op_words_per_cand, ctx->d_plan_sums.as<int64_t>(), d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), ctx->ilv_words,
-                     &ctx->launches);
+                     ctx->h_pinned + 8, ctx->planned, &ctx->launches);
     CU(cudaGetLastError(), "emission planning launch");
+    // The planning kernel's last block writes the totals and the status word straight into the
+    // pinned words; the host waits for that kernel only, not for the per-device words behind it.
     static_assert(sizeof(EmitTotals) == 8 * sizeof(int64_t), "totals occupy the second half of the pinned words");
     const EmitTotals *totals = reinterpret_cast<const EmitTotals *>(ctx->h_pinned + 8);
-    CU(cudaMemcpyAsync(ctx->h_pinned + 8, ctx->d_totals.p, sizeof(EmitTotals), cudaMemcpyDeviceToHost, s), "totals readback");
+    CU(cudaEventSynchronize(ctx->planned), "planning sync");
     bool stalled = false;
-    if (int rc = read_status(ctx, s, &stalled)) return rc;       // synchronises
+    if (int rc = take_status(ctx, s, (int32_t)ctx->h_pinned[8 + 7], &stalled)) return rc;
     *h_total_records = totals->records;
     if (d_records) {
         if (totals->records > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");

@@ -33,14 +33,20 @@ constexpr int kBucketReplicas = 32; // replicas per block of the bucket kernel: 
 // the longest item: every layer with computation, all-reduce and all-to-all, a jitter event, a transfer
 static_assert((3 * DISTSIM_MAX_LAYERS + 2) * 5 <= kTileWords && kTileWords % 2 == 0, "an item must fit the image");
 
+// The row that holds candidate `index`.  Every lane of the warp calls this with the same index;
+// the lanes look at 32 rows at a time (the rows' offsets ascend from 0).
 __device__ __forceinline__ int find_row(const DeviceView &v, int64_t index)
 {
-    int lo = 0, hi = v.sc.n_rows - 1;
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (v.rows[mid].offset <= index) lo = mid; else hi = mid - 1;
+    const int lane = threadIdx.x & 31;
+    int found = 0;
+    for (int base = 0; base < v.sc.n_rows; base += 32) {
+        const int r = base + lane;
+        const bool at_or_before = r < v.sc.n_rows && __ldg(&v.rows[r].offset) <= index;
+        const unsigned int mask = __ballot_sync(0xffffffffu, at_or_before);
+        if (!mask) break;
+        found = base + 31 - __clz(mask);
     }
-    return lo;
+    return found;
 }
 
 // Words of a selection's summary: what the scan over all selections needs of its plan.
@@ -61,14 +67,19 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
     const int64_t *pf = v.etf + (int64_t)cc.entry * v.tc.lp;
     const int64_t *pb = v.etb + (int64_t)cc.entry * v.tc.lp;
     const int n_slots = 2 * (en.m + row.pp - 1);
+    // times of an entry whose bound is below 2^32 fit 32 bits: half the instructions per slot
+    const bool narrow = S == 1 && v.tc.n_jitter == 0 && en.bound < ((int64_t)1 << 32);
     const StageResult<S> R = v.tc.n_jitter > 0
         ? lockstep_candidate<S, true, true>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank, seg_lane, wl,
                                             n_slots, owner ? rec : nullptr, binom)
+        : narrow
+        ? lockstep_candidate<S, true, false, uint32_t>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank, seg_lane,
+                                                       wl, n_slots, owner ? rec : nullptr, binom)
         : lockstep_candidate<S, true, false>(v, row, en, cc.entry, pf, pb, cc.sched, cc.part_rank, seg_lane, wl,
                                              n_slots, owner ? rec : nullptr, binom);
     // per stage: records of a forward / backward item, gradient buckets, records of one device;
     // their prefix over the stages and the widest item by shuffles over the lanes that own stages
-    int64_t recs[S];
+    int64_t recs[S], kbs[S];
     int widest = 1, both = 2;
     int64_t lane_recs = 0;
     if (owner) {
@@ -89,6 +100,7 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
                 kb = nbt[(int64_t)e * L1 + a] + (tpt[(int64_t)e * L1 + a] > 0 ? 1 : 0);
             }
             recs[k] = (int64_t)en.m * (rf + rb) + kb;
+            kbs[k] = kb;
             lane_recs += recs[k];
             widest = max(widest, (int)max(rf, rb));
             both = max(both, (int)(rf + rb));
@@ -112,7 +124,7 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
     int64_t most_buckets = 0;
     if (owner) {
 #pragma unroll
-        for (int k = 0; k < S; ++k) most_buckets = max64(most_buckets, recs[k] - (int64_t)en.m * (plan->rf[seg_lane * S + k] + plan->rb[seg_lane * S + k]));
+        for (int k = 0; k < S; ++k) most_buckets = max64(most_buckets, kbs[k]);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -237,6 +249,7 @@ __device__ __forceinline__ void scan_plans(EmitPlan *plans, const int64_t *sums,
     const int per = (n + nt - 1) / nt;
     const int b = min(n, t * per), e = min(n, b + per);
     int64_t s = 0, mx[kSumWords] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll 4
     for (int i = b; i < e; ++i) {
         s += __ldcg(&sums[(int64_t)i * kSumWords + kSumRecords]);
 #pragma unroll
@@ -259,9 +272,11 @@ __device__ __forceinline__ void scan_plans(EmitPlan *plans, const int64_t *sums,
         }
         warp_sum[lane] = wi - w;                       // exclusive
         if (lane == 31) totals[0] = wi;
+        if (lane >= kSumItemTiles && lane <= kSumRunWords) totals[lane] = 0;      // maxima: from zero
     }
     __syncthreads();
     int64_t acc = warp_sum[warp] + incl - s;
+#pragma unroll 4
     for (int i = b; i < e; ++i) { plans[i].rec_base = acc; acc += __ldcg(&sums[(int64_t)i * kSumWords + kSumRecords]); }
     // totals[1..5]: item tiles, bucket tiles, template words, bucket records, run words (the order of the summary)
 #pragma unroll
@@ -270,12 +285,14 @@ __device__ __forceinline__ void scan_plans(EmitPlan *plans, const int64_t *sums,
 }
 
 // One warp per selection plans it; the last block to finish then scans the plans (totals[6]
-// counts the finished blocks; the totals are cleared before the launch).
+// counts the finished blocks: zero before the first launch, and the last block leaves it zero).
 constexpr int kPlanBinomWords = 512;
 __global__ void __launch_bounds__(128)
 emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitPlan *plans,
                  int64_t *op_start, int64_t op_words_per_cand, int64_t *sums, int64_t *totals,
-                 int ilv_words /* shared-memory words per warp for interleaved candidates */)
+                 int ilv_words /* shared-memory words per warp for interleaved candidates */,
+                 int64_t *h_totals /* nullable; host memory the device can write: the totals' words, then
+                                      (word 7) the device status word as this kernel leaves it */)
 {
     extern __shared__ __align__(16) int64_t plan_dyn[];
     __shared__ int64_t binom_s[kPlanBinomWords];
@@ -312,7 +329,16 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
     __syncthreads();
     if (!last) return;
     __threadfence();
+    if (threadIdx.x == 0) totals[6] = 0;               // the next launch counts its blocks from zero
     scan_plans(plans, sums, n, totals);
+    if (!h_totals) return;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        // the host reads these once an event recorded behind this kernel has completed
+        for (int w = 0; w <= kSumRunWords; ++w) h_totals[w] = __ldcg(&totals[w]);
+        h_totals[7] = (int64_t)*((volatile int32_t *)v.status);
+        __threadfence_system();
+    }
 }
 
 __global__ void __launch_bounds__(256)
@@ -755,14 +781,14 @@ int interleaved_words_of(int pp, int v) { return interleaved_words(pp, v); }
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals, int ilv_words,
-                      int64_t *launches)
+                      int64_t *h_totals, cudaEvent_t planned, int64_t *launches)
 {
-    cudaMemsetAsync(d_totals, 0, sizeof(EmitTotals), s);
     const size_t plan_smem = (size_t)4 * ilv_words * sizeof(int64_t);
     ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_plan_kernel), plan_smem);
     emit_plan_kernel<<<(n + 3) / 4, 128, plan_smem, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand, sums, d_totals,
-                                                     ilv_words);
+                                                     ilv_words, h_totals);
     ++*launches;
+    if (planned) cudaEventRecord(planned, s);       // the host can go on while the per-device words are written
     if (offsets || busy || util) {
         const int64_t total = (int64_t)n * v.tc.n_devices + 1;
         emit_devices_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(v, plans, n, offsets, busy, util, d_totals);
@@ -780,27 +806,32 @@ void launch_emit_records(cudaStream_t s, const SideStream &ss, const DeviceView 
     const size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
     ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_items_kernel), smem);
     int64_t *out = reinterpret_cast<int64_t *>(records);
-    if (t.bucket_tiles > 0 && t.bucket_recs > 0) {
+    const bool buckets = t.bucket_tiles > 0 && t.bucket_recs > 0;
+    // The bucket records are few and their blocks wait more than they write: on the side stream
+    // they run beside the item kernel (both only read the plans and write disjoint records).  The
+    // fork event is recorded before the item kernel is enqueued, the item kernel goes first.
+    const bool beside = buckets && ss.side[0];
+    if (beside) cudaEventRecord(ss.fork, s);
+    emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
+        v, plans, op_start, op_words_per_cand, out, cap);
+    ++*launches;
+    if (buckets) {
         // an odd number of buckets per image keeps both images 16-byte aligned
         const int run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun) | 1;
         const size_t bsmem = (size_t)(2 * (run * 5 + 1) + 2 * (DISTSIM_MAX_LAYERS + 1)) * sizeof(int64_t);
         ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_buckets_kernel), bsmem);
-        // the bucket records are few and their blocks wait more than they write: on the side
-        // stream they run beside the item kernel (both only read the plans and write disjoint records)
         cudaStream_t bs = s;
-        if (ss.side[0]) {
-            cudaEventRecord(ss.fork, s);                 // recorded before the item kernel below is enqueued
+        if (beside) {
             cudaStreamWaitEvent(ss.side[0], ss.fork, 0);
             bs = ss.side[0];
         }
         emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, bs>>>(v, plans, out, run);
         ++*launches;
-        if (ss.side[0]) cudaEventRecord(ss.join[0], ss.side[0]);
+        if (beside) {
+            cudaEventRecord(ss.join[0], ss.side[0]);
+            cudaStreamWaitEvent(s, ss.join[0], 0);
+        }
     }
-    emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
-        v, plans, op_start, op_words_per_cand, out, cap);
-    ++*launches;
-    if (t.bucket_tiles > 0 && t.bucket_recs > 0 && ss.side[0]) cudaStreamWaitEvent(s, ss.join[0], 0);
 }
 
 }  // namespace distsim

@@ -261,6 +261,9 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals,
                       int ilv_words /* shared-memory words a warp needs for the space's interleaved rows (0: none) */,
+                      int64_t *h_totals /* nullable: host memory the device can write; receives the totals' words
+                                           and, in word 7, the device status word after planning */,
+                      cudaEvent_t planned /* nullable: recorded behind the planning kernel */,
                       int64_t *launches);
 int interleaved_words_of(int pp, int v);           // those words for one row
 // out[k] = order-sensitive checksum of the records [offsets[k], offsets[k + 1]).

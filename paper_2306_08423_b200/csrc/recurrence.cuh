@@ -224,6 +224,17 @@ __device__ __forceinline__ int64_t shfl_idx64(int64_t x, int src_lane)
     const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)((uint64_t)x >> 32), src_lane);
     return (int64_t)(((uint64_t)hi << 32) | lo);
 }
+// Stores `value` at `where` on the lanes where `on` holds: a predicated store, so that the slots
+// of the lock-step form stay free of branches.
+__device__ __forceinline__ void store_if(bool on, int64_t *where, int64_t value)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.s32 p, %0, 0;\n\t@p st.global.b64 [%1], %2;\n\t}"
+                 :: "r"((int)on), "l"(where), "l"(value) : "memory");
+}
+// The state word of the lock-step form in either width (uint32_t: entries whose time bound is
+// below 2^32, one shuffle and single-word compares per slot).
+__device__ __forceinline__ int64_t shfl_idx(int64_t x, int src_lane) { return shfl_idx64(x, src_lane); }
+__device__ __forceinline__ uint32_t shfl_idx(uint32_t x, int src_lane) { return __shfl_sync(0xffffffffu, x, src_lane); }
 
 // Lock-step evaluation of one candidate by `wl` consecutive lanes (wl * S == pp), every lane of
 // the warp calling this together (lanes of other segments work on their own candidates).
@@ -242,7 +253,9 @@ __device__ __forceinline__ int64_t shfl_idx64(int64_t x, int src_lane)
 // for a backward one, the stage itself - a no-op - when it idles or has no such neighbour: the
 // first stage's forward items and the last stage's backward items wait for their own device only).
 // One stage per lane fetches exactly that value with one indexed shuffle per slot.
-template <int S, bool kRecord, bool kJit>
+//   T          type of the times inside the slots: int64_t, or uint32_t when the entry's time
+//              bound is below 2^32 (exact: no time of the candidate can reach the bound)
+template <int S, bool kRecord, bool kJit, class T = int64_t>
 __device__ __forceinline__ StageResult<S> lockstep_candidate(
     const DeviceView &v, const Row &row, const Entry &en, int entry_index, const int64_t *pf,
     const int64_t *pb, int sched, int64_t part_rank, int seg_lane, int wl, int n_slots_warp, int64_t *rec,
@@ -262,10 +275,16 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         R.bop[k] = pb[R.e[k]] - pb[R.a[k]] + (d > 0 ? p2p_cost(row, en, d - 1) : 0);
         sp[k] = slot_plan(sched, pp, m, d);
     }
-    int64_t t[S];
+    T t[S], fop[S], bop[S];
     int n_f[S], n_b[S];                  // forward / backward items done: the next item's micro-batch
+    int64_t *rp[S];                      // where the next item's start goes (a stage's items are consecutive)
+    const bool recording = kRecord && rec != nullptr;
 #pragma unroll
-    for (int k = 0; k < S; ++k) { t[k] = 0; n_f[k] = 0; n_b[k] = 0; }
+    for (int k = 0; k < S; ++k) {
+        t[k] = 0; n_f[k] = 0; n_b[k] = 0;
+        fop[k] = (T)R.fop[k]; bop[k] = (T)R.bop[k];
+        rp[k] = (kRecord && rec) ? rec + (int64_t)(d0 + k) * 2 * m : nullptr;
+    }
     const int lane = threadIdx.x & 31;
     // where a forward (backward) item's input comes from: the previous (next) lane, or the lane
     // itself when there is no such stage (one stage per lane)
@@ -279,42 +298,50 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
         for (int i = 0; i < kChunk; ++i) {
             if (S == 1) {
                 const bool do_f = (fm[0] >> i) & 1u, do_b = (bm[0] >> i) & 1u;
-                int64_t cost = do_f ? R.fop[0] : (do_b ? R.bop[0] : 0);
+                T cost = do_f ? fop[0] : (do_b ? bop[0] : (T)0);
                 if (kJit) {
-                    if (do_f) cost += jitter_of(v, v.raw.jit_f, n_f[0], d0);
-                    if (do_b) cost += jitter_of(v, v.raw.jit_b, n_b[0], d0);
+                    if (do_f) cost += (T)jitter_of(v, v.raw.jit_f, n_f[0], d0);
+                    if (do_b) cost += (T)jitter_of(v, v.raw.jit_b, n_b[0], d0);
                 }
-                const int64_t dep = shfl_idx64(t[0], do_f ? src_f : (do_b ? src_b : lane));
-                const int64_t own = t[0] + cost, via = dep + cost;       // both ready before the compare ends
+                const T dep = shfl_idx(t[0], do_f ? src_f : (do_b ? src_b : lane));
+                const T own = t[0] + cost, via = dep + cost;             // both ready before the compare ends
                 const bool late = dep > t[0];
+                if (kRecord) {
+                    const bool item = recording && (do_f || do_b);
+                    store_if(item, rp[0], (int64_t)(late ? dep : t[0]));
+                    rp[0] += item ? 1 : 0;
+                }
                 t[0] = late ? via : own;
-                if (kRecord && rec && (do_f || do_b)) rec[(int64_t)d0 * 2 * m + n_f[0] + n_b[0]] = t[0] - cost;
-                if (kRecord || kJit) { n_f[0] += do_f ? 1 : 0; n_b[0] += do_b ? 1 : 0; }
+                if (kJit) { n_f[0] += do_f ? 1 : 0; n_b[0] += do_b ? 1 : 0; }
             } else {
                 // several stages per lane: the lane's first (last) stage takes the previous (next)
                 // lane's last (first) stage, the others their neighbour inside the lane
-                const int64_t up_f = __shfl_up_sync(0xffffffffu, t[S - 1], 1, wl);
-                const int64_t dn_b = __shfl_down_sync(0xffffffffu, t[0], 1, wl);
-                int64_t old[S];
+                const T up_f = __shfl_up_sync(0xffffffffu, t[S - 1], 1, wl);
+                const T dn_b = __shfl_down_sync(0xffffffffu, t[0], 1, wl);
+                T old[S];
 #pragma unroll
                 for (int k = 0; k < S; ++k) old[k] = t[k];
 #pragma unroll
                 for (int k = 0; k < S; ++k) {
                     const int d = d0 + k;
                     const bool do_f = (fm[k] >> i) & 1u, do_b = (bm[k] >> i) & 1u;
-                    int64_t cost = do_f ? R.fop[k] : (do_b ? R.bop[k] : 0);
+                    T cost = do_f ? fop[k] : (do_b ? bop[k] : (T)0);
                     if (kJit) {
-                        if (do_f) cost += jitter_of(v, v.raw.jit_f, n_f[k], d);
-                        if (do_b) cost += jitter_of(v, v.raw.jit_b, n_b[k], d);
+                        if (do_f) cost += (T)jitter_of(v, v.raw.jit_f, n_f[k], d);
+                        if (do_b) cost += (T)jitter_of(v, v.raw.jit_b, n_b[k], d);
                     }
-                    const int64_t dep_f = (k == 0) ? (d == 0 ? 0 : up_f) : old[k > 0 ? k - 1 : 0];
-                    const int64_t dep_b = (k == S - 1) ? (d == pp - 1 ? 0 : dn_b) : old[k < S - 1 ? k + 1 : 0];
-                    const int64_t dep = do_f ? dep_f : (do_b ? dep_b : 0);
-                    const int64_t own = old[k] + cost, via = dep + cost;
+                    const T dep_f = (k == 0) ? (d == 0 ? (T)0 : up_f) : old[k > 0 ? k - 1 : 0];
+                    const T dep_b = (k == S - 1) ? (d == pp - 1 ? (T)0 : dn_b) : old[k < S - 1 ? k + 1 : 0];
+                    const T dep = do_f ? dep_f : (do_b ? dep_b : (T)0);
+                    const T own = old[k] + cost, via = dep + cost;
                     const bool late = dep > old[k];
+                    if (kRecord) {
+                        const bool item = recording && (do_f || do_b);
+                        store_if(item, rp[k], (int64_t)(late ? dep : old[k]));
+                        rp[k] += item ? 1 : 0;
+                    }
                     t[k] = late ? via : own;
-                    if (kRecord && rec && (do_f || do_b)) rec[(int64_t)d * 2 * m + n_f[k] + n_b[k]] = t[k] - cost;
-                    if (kRecord || kJit) { n_f[k] += do_f ? 1 : 0; n_b[k] += do_b ? 1 : 0; }
+                    if (kJit) { n_f[k] += do_f ? 1 : 0; n_b[k] += do_b ? 1 : 0; }
                 }
             }
         }
@@ -325,10 +352,10 @@ __device__ __forceinline__ StageResult<S> lockstep_candidate(
     int64_t mx = 0;
 #pragma unroll
     for (int k = 0; k < S; ++k) {
-        R.main_end[k] = t[k];
+        R.main_end[k] = (int64_t)t[k];
         // every stage's last item is the backward item of the last micro-batch; its first layer
         // event starts one backward item cost before its end
-        R.last_b_start[k] = t[k] - R.bop[k];
+        R.last_b_start[k] = (int64_t)t[k] - R.bop[k];
         // the asynchronous schedule has no gradient all-reduce events
         if (sched == 2 || row.dp == 1) {
             R.dp_end[k] = R.main_end[k];
