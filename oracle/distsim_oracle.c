@@ -92,14 +92,14 @@ typedef struct {
     int32_t partition_mode;               /* 0: balanced; 1: all compositions     */
     int32_t sched_mask;                   /* bit 0: GPipe, bit 1: 1F1B (Dapple),
                                              bit 2: 1F1B without gradient synchronisation,
-                                             bit 3: interleaved 1F1B with v = 2, 4, .. v_max chunks */
+                                             bit 3: interleaved 1F1B with v = 2, 4, .. v_max chunks,
+                                             bit 4: bidirectional pipelines */
     int32_t v_max;                        /* largest number of model chunks per device (bit 3)    */
 } orc_space;
 
 typedef struct {
     int32_t mp, pp, dp, m, sched;         /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B,
-                                             3: interleaved 1F1B (simulated when given
-                                             explicitly; the search space does not enumerate it) */
+                                             3: interleaved 1F1B, 4: bidirectional pipelines */
     int32_t bounds[ORC_MAX_PP + 1];       /* c_0 .. c_P, P = pp (P = pp * v for sched 3)  */
     int32_t v;                            /* sched 3: model chunks per device (0 or 1 otherwise) */
 } orc_candidate;
@@ -201,6 +201,22 @@ static int loc_dp_groups(const orc_table *T, const orc_candidate *x)
         }
     return cur;
 }
+/* Bidirectional pipelines: the weights of stage s live on device s (pipeline "down") and on
+ * device pp - 1 - s (pipeline "up") of every replica; their gradients are reduced over those
+ * 2 dp devices. */
+static int loc_mirror_group(const orc_table *T, const orc_candidate *x, int64_t d)
+{
+    int cur = -2;
+    for (int64_t q = 0; q < x->mp; ++q) {
+        int inter = 0;
+        int64_t n0 = rank_of(x, 0, d, q) / T->gpus_per_node;
+        for (int64_t r = 0; r < x->dp; ++r)
+            if (rank_of(x, r, d, q) / T->gpus_per_node != n0 ||
+                rank_of(x, r, x->pp - 1 - d, q) / T->gpus_per_node != n0) inter = 1;
+        cur = merge_loc(cur, inter);
+    }
+    return cur;
+}
 /* Transfer from pipeline device da to pipeline device db (db = da + 1 between neighbouring
  * stages; the interleaved schedule also sends from the last device back to the first). */
 static int loc_transfer(const orc_table *T, const orc_candidate *x, int64_t da, int64_t db)
@@ -229,6 +245,9 @@ static int64_t beta_of(const orc_table *T, int loc) { return loc ? T->beta_inter
 /* candidates of v chunks per device: m ascending over the valid entries that  */
 /* are multiples of pp, then the partition of the L layers into pp*v virtual    */
 /* stages (balanced, or every composition in lexicographic order).             */
+/* With bit 4 every (mp, pp) with pp >= 2 is then followed by the candidates of */
+/* the bidirectional schedule: m ascending over the valid even entries, the    */
+/* partition into pp stages as for the plain schedules.                        */
 /* The paper's own grid (Sec. 6) walks mp and pp over powers of two and takes  */
 /* dp = GPUs/mp/pp, dropping the invalid combinations.                         */
 
@@ -285,8 +304,8 @@ static int64_t walk_space(const orc_table *T, const orc_space *S, orc_visit_fn v
                 } while (S->partition_mode == 1 && next_partition(x.bounds, (int)pp, L));
             }
             /* interleaved 1F1B: candidates with v chunks per device, P = pp * v virtual stages */
-            if (!(S->sched_mask & 8) || pp < 2) continue;
-            for (int64_t v = 2; v <= S->v_max && pp * v <= ORC_MAX_PP && pp * v <= L; v *= 2) {
+            if (pp < 2) continue;
+            for (int64_t v = 2; (S->sched_mask & 8) && v <= S->v_max && pp * v <= ORC_MAX_PP && pp * v <= L; v *= 2) {
                 const int P = (int)(pp * v);
                 for (int mi = 0; mi < S->n_m; ++mi) {
                     int64_t m = S->m_list[mi];
@@ -305,6 +324,25 @@ static int64_t walk_space(const orc_table *T, const orc_space *S, orc_visit_fn v
                         ++index;
                     } while (S->partition_mode == 1 && next_partition(x.bounds, P, L));
                 }
+            }
+            /* bidirectional pipelines: half of the (even number of) micro-batches each way */
+            if (!(S->sched_mask & 16)) continue;
+            for (int mi = 0; mi < S->n_m; ++mi) {
+                int64_t m = S->m_list[mi];
+                if (!valid_m(S, Bp, m) || m % 2 != 0) continue;
+                orc_candidate x;
+                memset(&x, 0, sizeof x);
+                x.mp = (int32_t)mp; x.pp = (int32_t)pp; x.dp = (int32_t)dp; x.m = (int32_t)m;
+                x.sched = 4;
+                x.bounds[0] = 0; x.bounds[pp] = L;
+                if (S->partition_mode == 0)
+                    for (int j = 1; j < pp; ++j) x.bounds[j] = (int32_t)((int64_t)j * L / pp);
+                else
+                    for (int j = 1; j < pp; ++j) x.bounds[j] = j;
+                do {
+                    if (visit && visit(ctx, index, &x)) return index + 1;
+                    ++index;
+                } while (S->partition_mode == 1 && next_partition(x.bounds, (int)pp, L));
             }
         }
     return index;
@@ -377,6 +415,81 @@ static int64_t union_measure(const orc_list *l)
 }
 
 /*
+ * Bidirectional pipelines (sched 4; Chimera, which the paper names among the pipeline scheduling
+ * algorithms in Sec. 2; the schedule is, as for the others, the input of the pipeline modeling
+ * of Sec. 4.3).  Two pipelines run over the same pp devices (pp even) in opposite directions:
+ * pipeline "down" has stage s on device s and takes micro-batches 0 .. m/2 - 1, pipeline "up" has
+ * stage s on device pp - 1 - s and takes micro-batches m/2 .. m - 1 (m even).  Each pipeline, on
+ * its own, runs the 1F1B order.  A device holds one stage of each and merges the two orders; the
+ * merged order is the one in which the items run when every item takes one time slot and every
+ * device, slot by slot, runs the first of its two pipelines' next items whose input was produced
+ * in an earlier slot - preferring the item whose micro-batch comes earlier within its pipeline
+ * (the two never hold the same position when both could run - checked for pp <= 32, m <= 64 -
+ * a backward item, then pipeline "down", would go first).  With m = pp that takes 3 pp - 2 slots (pp - 2 idle
+ * slots per device, the published property of the schedule), with any even m, 2 m + pp - 2.
+ * ops[d * 2m + k]: the k-th item of device d (chunk = pipeline).  Returns 0, or -1 (no memory).
+ */
+static int bidirectional_order(int pp, int m, orc_op *ops)
+{
+    const int half = m / 2, n_ops = 2 * m;
+    /* the two 1F1B orders of every device, and when each item finished (slot number; -1: not yet) */
+    orc_op *q = (orc_op *)malloc((size_t)2 * pp * m * sizeof(orc_op));     /* [device][pipeline][m] */
+    int *endF = (int *)malloc((size_t)2 * pp * m * sizeof(int));           /* [pipeline][stage][micro-batch] */
+    int *endB = (int *)malloc((size_t)2 * pp * m * sizeof(int));
+    if (!q || !endF || !endB) { free(q); free(endF); free(endB); return -1; }
+    for (int i = 0; i < 2 * pp * m; ++i) endF[i] = endB[i] = -1;
+    for (int d = 0; d < pp; ++d)
+        for (int u = 0; u < 2; ++u) {
+            const int s = u ? pp - 1 - d : d, first = u ? half : 0;
+            orc_op *o = q + ((int64_t)d * 2 + u) * m;
+            const int w = pp - s < half ? pp - s : half;
+            int k = 0, nf = 0, nb = 0;
+            for (; nf < w; ++nf) { o[k].is_bwd = 0; o[k].chunk = u; o[k++].mb = first + nf; }
+            while (nb < half) {
+                o[k].is_bwd = 1; o[k].chunk = u; o[k++].mb = first + nb++;
+                if (nf < half) { o[k].is_bwd = 0; o[k].chunk = u; o[k++].mb = first + nf++; }
+            }
+        }
+    int head[ORC_MAX_PP][2], n_done[ORC_MAX_PP], pick[ORC_MAX_PP];
+    for (int d = 0; d < pp; ++d) { head[d][0] = head[d][1] = 0; n_done[d] = 0; }
+    int left = pp * n_ops;
+    for (int t = 0; left > 0; ++t) {
+        if (t > 4 * (m + pp)) { free(q); free(endF); free(endB); return -1; }
+        /* every device chooses on what earlier slots produced ... */
+        for (int d = 0; d < pp; ++d) {
+            pick[d] = -1;
+            int best_mb = 0, best_bwd = 0;
+            for (int u = 0; u < 2; ++u) {
+                if (head[d][u] == m) continue;
+                const orc_op o = q[((int64_t)d * 2 + u) * m + head[d][u]];
+                const int s = u ? pp - 1 - d : d;
+                const int64_t at = ((int64_t)u * pp + s) * m + o.mb;
+                int dep;
+                if (!o.is_bwd) dep = s == 0 ? 0 : endF[at - m];
+                else dep = s == pp - 1 ? endF[at] : endB[at + m];
+                if (dep < 0 || dep > t) continue;
+                const int local = o.mb - (u ? half : 0);
+                if (pick[d] < 0 || local < best_mb || (local == best_mb && o.is_bwd > best_bwd)) {
+                    pick[d] = u; best_mb = local; best_bwd = o.is_bwd;
+                }
+            }
+        }
+        /* ... then the chosen items run, one slot each */
+        for (int d = 0; d < pp; ++d) {
+            const int u = pick[d];
+            if (u < 0) continue;
+            const orc_op o = q[((int64_t)d * 2 + u) * m + head[d][u]];
+            const int s = u ? pp - 1 - d : d;
+            (o.is_bwd ? endB : endF)[((int64_t)u * pp + s) * m + o.mb] = t + 1;
+            ops[(int64_t)d * n_ops + n_done[d]++] = o;
+            ++head[d][u]; --left;
+        }
+    }
+    free(q); free(endF); free(endB);
+    return 0;
+}
+
+/*
  * Interleaved 1F1B (sched 3; the paper names further scheduling algorithms as input to the same
  * pipeline modeling, Sec. 4.3 "the pipeline schedule generated from the pipeline algorithm",
  * and cites Megatron-LM, whose interleaved schedule this is).  Every device holds v model
@@ -414,8 +527,9 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
 
     if (pp < 1 || pp > ORC_MAX_PP || mp < 1 || dp < 1 || m < 1 || v < 1 || P > ORC_MAX_PP ||
         (int64_t)mp * pp * dp != T->n_devices || T->global_batch % dp != 0 ||
-        x->bounds[0] != 0 || x->bounds[P] != L || x->sched < 0 || x->sched > 3 ||
+        x->bounds[0] != 0 || x->bounds[P] != L || x->sched < 0 || x->sched > 4 ||
         (x->sched == 3 && (m % pp != 0 || T->n_jitter > 0)) ||
+        (x->sched == 4 && (pp % 2 != 0 || m % 2 != 0 || T->n_jitter > 0)) ||
         (T->n_jitter > 0 && (T->jitter_stages < pp || !T->jitter_fwd_ns || !T->jitter_bwd_ns))) {
         e = ORC_E_ARG; goto fail;
     }
@@ -432,6 +546,9 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
 
     int64_t AR = 0, A2A = 0, P2P[ORC_MAX_PP];
     int loc_dp = 0;
+    const int two_way = x->sched == 4;           /* bidirectional pipelines                */
+    const int64_t n_sync = two_way ? 2 * (int64_t)dp : dp;      /* devices that hold a stage's weights */
+    int loc_sync[ORC_MAX_PP];                    /* per device: locality of its gradient groups */
     if (mp > 1) {
         int loc = loc_mp_groups(T, x);
         if (loc < 0) { e = ORC_E_LOCALITY; goto fail; }
@@ -441,6 +558,10 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
         loc_dp = loc_dp_groups(T, x);
         if (loc_dp < 0) { e = ORC_E_LOCALITY; goto fail; }
         A2A = orc_all_to_all_ns(dp, act, alpha_of(T, loc_dp), beta_of(T, loc_dp));
+    }
+    for (int d = 0; d < pp; ++d) {
+        loc_sync[d] = two_way ? loc_mirror_group(T, x, d) : loc_dp;
+        if (loc_sync[d] < 0) { e = ORC_E_LOCALITY; goto fail; }
     }
     /* P2P[s]: transfer between virtual stages s and s + 1, i.e. between devices s mod pp and
      * (s + 1) mod pp */
@@ -453,14 +574,17 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
     /* ---- Step 2: the pipeline schedule S(D, L, M) -------------------------- */
     const int n_ops = 2 * m * v;                 /* items of one device                    */
     ops = (orc_op *)malloc((size_t)pp * n_ops * sizeof(orc_op));
-    endF = (int64_t *)malloc((size_t)P * m * sizeof(int64_t));      /* [virtual stage][micro-batch] */
-    endB = (int64_t *)malloc((size_t)P * m * sizeof(int64_t));
+    const int n_vs = two_way ? 2 * pp : P;       /* rows of endF / endB: virtual stages, or
+                                                    [pipeline][stage] of the bidirectional schedule */
+    endF = (int64_t *)malloc((size_t)n_vs * m * sizeof(int64_t));   /* [virtual stage][micro-batch] */
+    endB = (int64_t *)malloc((size_t)n_vs * m * sizeof(int64_t));
     tmp = (orc_event *)malloc((size_t)(3 * L + 2) * sizeof(orc_event));
     const int mp_lists = replicate ? mp : 1;
     F = (orc_list *)calloc((size_t)pp * mp_lists, sizeof(orc_list));
     if (!ops || !endF || !endB || !tmp || !F) { e = ORC_E_NOMEM; goto fail; }
-    for (int64_t i = 0; i < (int64_t)P * m; ++i) endF[i] = endB[i] = -1;
-    for (int d = 0; d < pp; ++d) {
+    for (int64_t i = 0; i < (int64_t)n_vs * m; ++i) endF[i] = endB[i] = -1;
+    if (two_way && bidirectional_order(pp, m, ops) != 0) { e = ORC_E_NOMEM; goto fail; }
+    for (int d = 0; d < pp && !two_way; ++d) {
         orc_op *o = ops + (int64_t)d * n_ops;
         int k = 0;
         for (int i = 0; i < n_ops; ++i) o[i].chunk = 0;
@@ -512,18 +636,27 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                 int d = reverse_scan ? pp - 1 - s : s;
                 if (head[d] == n_ops) continue;
                 orc_op o = ops[(int64_t)d * n_ops + head[d]];
-                const int vs = o.chunk * pp + d;
+                /* the item's stage in its chain of stages, and its row in endF / endB */
+                const int st = two_way ? (o.chunk ? pp - 1 - d : d) : o.chunk * pp + d;
+                const int vs = two_way ? o.chunk * pp + st : st;
+                const int n_st = two_way ? pp : P;
                 int64_t dep;
-                if (!o.is_bwd) dep = vs == 0 ? 0 : endF[(int64_t)(vs - 1) * m + o.mb];
-                else dep = vs == P - 1 ? endF[(int64_t)vs * m + o.mb] : endB[(int64_t)(vs + 1) * m + o.mb];
+                if (!o.is_bwd) dep = st == 0 ? 0 : endF[(int64_t)(vs - 1) * m + o.mb];
+                else dep = st == n_st - 1 ? endF[(int64_t)vs * m + o.mb] : endB[(int64_t)(vs + 1) * m + o.mb];
                 if (dep < 0) continue;
                 pick = d; t = max64(device_free[d], dep);
             }
             if (pick < 0) { e = ORC_E_DEADLOCK; goto fail; }
             const int d = pick;
             const orc_op o = ops[(int64_t)d * n_ops + head[d]];
-            const int vs = o.chunk * pp + d;
-            const int la = x->bounds[vs], le = x->bounds[vs + 1];   /* the item's layers [la, le) */
+            const int st = two_way ? (o.chunk ? pp - 1 - d : d) : o.chunk * pp + d;
+            const int vs = two_way ? o.chunk * pp + st : st;
+            const int n_st = two_way ? pp : P;
+            const int la = x->bounds[st], le = x->bounds[st + 1];   /* the item's layers [la, le) */
+            /* transfers to the next / previous stage of the item's pipeline: pipeline "up" of the
+             * bidirectional schedule crosses the device boundaries the other way round */
+            const int64_t send_f = st < n_st - 1 ? (two_way && o.chunk ? P2P[pp - 2 - st] : P2P[st]) : 0;
+            const int64_t send_b = st > 0 ? (two_way && o.chunk ? P2P[pp - 1 - st] : P2P[st - 1]) : 0;
             /* Look-up step of Algorithm 1: the events MP modeling mapped the item's layers to -
              * per layer a computation event, then its all-reduce event (mp > 1) and its
              * all-to-all event (expert layer, dp > 1) - followed by the communication event of
@@ -546,7 +679,7 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                     if (mp > 1) { tmp[n++] = (orc_event){ ORC_MP_AR_F, l, o.mb, t, t + AR }; t += AR; }
                     if (T->layer_is_expert[l] && dp > 1) { tmp[n++] = (orc_event){ ORC_A2A_F, l, o.mb, t, t + A2A }; t += A2A; }
                 }
-                if (vs < P - 1) { tmp[n++] = (orc_event){ ORC_SEND_F, le - 1, o.mb, t, t + P2P[vs] }; t += P2P[vs]; }
+                if (st < n_st - 1) { tmp[n++] = (orc_event){ ORC_SEND_F, le - 1, o.mb, t, t + send_f }; t += send_f; }
                 endF[(int64_t)vs * m + o.mb] = t;
             } else {
                 for (int l = le - 1; l >= la; --l) {
@@ -554,7 +687,7 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                     if (mp > 1) { tmp[n++] = (orc_event){ ORC_MP_AR_B, l, o.mb, t, t + AR }; t += AR; }
                     if (T->layer_is_expert[l] && dp > 1) { tmp[n++] = (orc_event){ ORC_A2A_B, l, o.mb, t, t + A2A }; t += A2A; }
                 }
-                if (vs > 0) { tmp[n++] = (orc_event){ ORC_SEND_B, la, o.mb, t, t + P2P[vs - 1] }; t += P2P[vs - 1]; }
+                if (st > 0) { tmp[n++] = (orc_event){ ORC_SEND_B, la, o.mb, t, t + send_b }; t += send_b; }
                 endB[(int64_t)vs * m + o.mb] = t;
             }
             device_free[d] = t;
@@ -583,7 +716,7 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                     orc_list *dst = &R->lists[(r * pp + d) * mp_lists + q];
                     for (int64_t i = 0; i < src->n; ++i)
                         if ((e = list_push(dst, src->ev[i])) != ORC_OK) goto fail;
-                    if (dp == 1) continue;
+                    if (n_sync == 1) continue;
                     /* Asynchronous pipeline parallelism (the paper's discussion of new
                      * algorithms in "Related Work And Discussion": the pipeline schedule
                      * is built in the same way, only without the global synchronisation
@@ -597,9 +730,19 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                     const int64_t main_end = src->n ? src->ev[src->n - 1].end : 0;
                     int64_t prev_end = 0, kb = 0;      /* the device's one lane; bucket numbers run on */
                     /* one gradient stream per model chunk (one stream without chunks), the
-                     * chunks in the order their last backward runs: chunk v - 1 first */
-                    for (int c = v - 1; c >= 0; --c) {
-                        const int vs = c * pp + d;
+                     * chunks in the order their last backward runs: chunk v - 1 first.
+                     * Bidirectional pipelines: one stream per pipeline - the device's stage in
+                     * it, reduced over the 2 dp devices that hold that stage - and the stream of
+                     * the later stage first (its backward items end first). */
+                    const int n_streams = two_way ? 2 : v;
+                    for (int c = n_streams - 1; c >= 0; --c) {
+                        int vs = c * pp + d, last_mb = m - 1;
+                        if (two_way) {
+                            const int up_first = pp - 1 - d > d;            /* the stage held in pipeline "up" is the later one */
+                            const int u = (c == 1) == up_first;             /* c = 1 comes first */
+                            vs = u ? pp - 1 - d : d;
+                            last_mb = u ? m - 1 : m / 2 - 1;
+                        }
                         const int la = x->bounds[vs], le = x->bounds[vs + 1];
                         int64_t W = 0;
                         for (int l = la; l < le; ++l) W += cdiv(T->grad_bytes[l], mp);
@@ -623,14 +766,14 @@ orc_result *orc_simulate(const orc_table *T, const orc_candidate *x, int replica
                                 ready = -1;
                                 for (int64_t i = 0; i < src->n; ++i) {
                                     const orc_event *ev = &src->ev[i];
-                                    if (ev->layer == last && ev->mb == m - 1 &&
+                                    if (ev->layer == last && ev->mb == last_mb &&
                                         (ev->kind == ORC_COMPUTE_B || ev->kind == ORC_MP_AR_B || ev->kind == ORC_A2A_B))
                                         ready = max64(ready, ev->end);
                                 }
                                 if (ready < 0) { e = ORC_E_ARG; goto fail; }
                             }
                             const int64_t start = max64(ready, prev_end);
-                            const int64_t end = start + orc_allreduce_ns(T->allreduce_profile_max, dp, hi - lo, alpha_of(T, loc_dp), beta_of(T, loc_dp));
+                            const int64_t end = start + orc_allreduce_ns(T->allreduce_profile_max, n_sync, hi - lo, alpha_of(T, loc_sync[d]), beta_of(T, loc_sync[d]));
                             if ((e = list_push(dst, (orc_event){ ORC_DP_AR, kb++, -1, start, end })) != ORC_OK) goto fail;
                             prev_end = end;
                         }

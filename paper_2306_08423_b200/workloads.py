@@ -156,7 +156,8 @@ def space_shape(table, space):
     """Rows of the search space for reporting: a list of (mp, pp, dp, [valid m], partitions,
     schedules, v) in canonical order; v = 1 for the plain schedules, the number of model chunks
     per device for a row of interleaved candidates (which has one schedule and partitions the
-    layers into pp * v virtual stages).  Pure counting; candidates = sum(len(ms) * partitions *
+    layers into pp * v virtual stages); a row of bidirectional-pipeline candidates (sched_mask
+    bit 4: one schedule, even m, v = 1) follows the interleaved rows of its (mp, pp).  Pure counting; candidates = sum(len(ms) * partitions *
     schedules)."""
     rows = []
     n_sched = bin(space.sched_mask & 7).count("1")
@@ -184,6 +185,12 @@ def space_shape(table, space):
                     continue
                 parts = 1 if space.partition_mode == PARTITION_BALANCED else math.comb(table.n_layers - 1, pp * v - 1)
                 rows.append((mp, pp, dp, mv, parts, 1, v))
+            if space.sched_mask & 16:
+                # bidirectional pipelines: half of the micro-batches each way, pp stages
+                me = [m for m in ms if m % 2 == 0]
+                if me:
+                    parts = 1 if space.partition_mode == PARTITION_BALANCED else math.comb(table.n_layers - 1, pp - 1)
+                    rows.append((mp, pp, dp, me, parts, 1, 1))
     return rows
 
 

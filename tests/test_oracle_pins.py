@@ -14,7 +14,7 @@ import pytest
 import oracle
 from oracle import Candidate, KINDS
 from paper_2306_08423_b200 import workloads as W
-from tests.dag_bruteforce import longest_path_timeline
+from tests.dag_bruteforce import bidirectional_order, longest_path_bidirectional, longest_path_timeline
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -314,6 +314,140 @@ def test_interleaved_rejects_what_the_schedule_does_not_define():
         oracle.simulate(T, Candidate(1, 2, 1, 3, 3, (0, 2, 4, 6, 8), 2))      # m is not a multiple of pp
     with pytest.raises(Exception):
         oracle.simulate(T, Candidate(1, 2, 1, 6, 3, (0, 4, 8), 2))            # bounds for pp stages, not pp * v
+
+
+# --------------------------------------------------------------------------- #
+# bidirectional pipelines (schedule 4)
+
+@pytest.mark.parametrize("pp,groups", [(2, 1), (2, 3), (4, 1), (4, 2), (6, 1), (8, 1), (8, 3), (16, 1)])
+def test_bidirectional_uniform_closed_form(pp, groups):
+    # Equal forward and backward item times on uniform stages, no communication: the timeline is
+    # the schedule's grid of unit slots, 2 m + pp - 2 of them - for m = pp the published property
+    # of the schedule (pp - 2 idle slots per device, against 2 (pp - 1) of the plain pipeline) -
+    # and every device is busy in 2 m of them.
+    t, per, m = 11, 3, pp * groups
+    L = pp * per
+    T = make_table([t] * L, [t] * L, n_devices=pp, gpus_per_node=1, global_batch=m, classes=[(1, 1)],
+                   alpha_intra_ns=0, alpha_inter_ns=0)
+    r = oracle.simulate(T, Candidate(1, pp, 1, m, 4, balanced(L, pp)))
+    assert r.batch_ns == (2 * m + pp - 2) * per * t
+    assert (r.busy_ns == 2 * m * per * t).all()
+    if groups == 1:
+        assert r.batch_ns == (3 * pp - 2) * per * t
+    plain = oracle.simulate(T, Candidate(1, pp, 1, m, 1, balanced(L, pp)))
+    assert plain.batch_ns == 2 * (m + pp - 1) * per * t >= r.batch_ns
+    # the device order used is the unit-slot order, restated independently as a token game
+    order, slots = bidirectional_order(pp, m)
+    assert slots == 2 * m + pp - 2
+    for d in range(pp):
+        a = r.records[r.offsets[d]:r.offsets[d + 1]]
+        firsts = a[(a[:, 0] <= 1) & (a[:, 1] == np.where(a[:, 0] == 0, d * per, (d + 1) * per - 1))]
+        # (the first layer event of each item of the device's stage in pipeline "down" ...)
+        down = [(k, j) for (k, j, u) in order[d] if u == 0]
+        assert [("F" if k == 0 else "B", j) for k, _, j in firsts[:, :3].tolist()] == down
+
+
+def test_hand_worked_bidirectional_example():
+    # tests/golden/worked_bidirectional_example.txt: four devices, four micro-batches, every item
+    # one time unit, worked by hand on squared paper; rows "device slot kind micro-batch pipeline"
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "worked_bidirectional_example.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    T = make_table([1] * 4, [1] * 4, n_devices=4, gpus_per_node=1, global_batch=4, classes=[(1, 1)],
+                   alpha_intra_ns=0, alpha_inter_ns=0)
+    r = oracle.simulate(T, Candidate(1, 4, 1, 4, 4, (0, 1, 2, 3, 4)))
+    assert r.batch_ns == 10
+    want = {d: [] for d in range(4)}
+    for dev, slot, kind, mb, pipe in rows:
+        d, u = int(dev), int(pipe)
+        layer = d if u == 0 else 3 - d
+        want[d].append((0 if kind == "F" else 1, layer, int(mb), int(slot), int(slot) + 1))
+    for d in range(4):
+        got = [tuple(x) for x in r.records[r.offsets[d]:r.offsets[d + 1]].tolist()]
+        assert all(e[3] == e[4] for e in got if e[0] in (6, 7))              # transfers cost nothing here
+        assert [e for e in got if e[0] <= 1] == sorted(want[d], key=lambda e: e[3]), d
+
+
+def _bidirectional_cases():
+    for seed in range(12):
+        rng = np.random.default_rng(900 + seed)
+        pp = [2, 4, 4, 6][seed % 4] if seed % 4 != 3 else 2
+        mp = 1 + seed % 2
+        dp = [1, 2][(seed // 2) % 2]
+        m = 2 * int(rng.integers(1, 4))
+        L = pp + int(rng.integers(0, 4))
+        cuts = sorted(rng.choice(np.arange(1, L), size=pp - 1, replace=False).tolist())
+        w = W.random_small(950 + seed, n_devices=pp * mp * dp, gpus_per_node=2, n_layers=L,
+                           global_batch=dp * m * int(rng.integers(1, 3)), mp_max=2, pp_max=4, m_list=(m,),
+                           dp_overlap=seed % 2, dp_bucket_bytes=0 if seed % 5 == 4 else 700)
+        yield w, Candidate(mp, pp, dp, m, 4, (0, *cuts, L))
+
+
+@pytest.mark.parametrize("w,cand", list(_bidirectional_cases()), ids=lambda x: getattr(x, "name", None))
+def test_bidirectional_brute_force_and_invariants(w, cand):
+    T = w.table
+    r = oracle.simulate(T, cand, replicate=False)
+    batch, lanes = longest_path_bidirectional(T, cand)     # independent DAG, order from the token game
+    assert r.batch_ns == batch
+    for d in range(cand.pp):
+        got = [tuple(x) for x in r.records[r.offsets[d]:r.offsets[d + 1]].tolist()]
+        assert got == lanes[d], (cand, d)
+    assert oracle.simulate(T, cand, replicate=False, reverse_scan=True).batch_ns == r.batch_ns
+    full = oracle.simulate(T, cand, replicate=True)
+    assert full.batch_ns == r.batch_ns
+    for rr in range(cand.dp):
+        for d in range(cand.pp):
+            for q in range(cand.mp):
+                dev = (rr * cand.pp + d) * cand.mp + q
+                a = full.records[full.offsets[dev]:full.offsets[dev + 1]]
+                assert (a == r.records[r.offsets[d]:r.offsets[d + 1]]).all()
+    for d in range(cand.pp):
+        a = r.records[r.offsets[d]:r.offsets[d + 1]]
+        main, buckets = a[a[:, 0] != 8], a[a[:, 0] == 8]
+        assert (main[1:, 3] >= main[:-1, 4]).all() and (buckets[1:, 3] >= buckets[:-1, 4]).all()
+        # the device runs every micro-batch of pipeline "down" through stage d and every one of
+        # pipeline "up" through stage pp - 1 - d, forward and backward
+        comp_f = main[main[:, 0] == 0]
+        for u, s in ((0, d), (1, cand.pp - 1 - d)):
+            mine = comp_f[comp_f[:, 1] == cand.bounds[s]]
+            assert sorted(mine[:, 2].tolist()) == list(range(u * cand.m // 2, (u + 1) * cand.m // 2))
+        # the weights of a stage are on two devices even without data parallelism: gradient
+        # events whenever the stage has gradient bytes
+        has_grad = any(T.grad_bytes[l] > 0 for s in (d, cand.pp - 1 - d) for l in range(cand.bounds[s], cand.bounds[s + 1]))
+        assert (len(buckets) > 0) == has_grad
+    assert r.batch_ns >= int(r.busy_ns.max())
+
+
+def test_bidirectional_on_unequal_links():
+    # six devices on nodes of four: the link between devices 3 and 4 is the slow one, so the two
+    # pipelines cross it at different stages (pipeline "down" after its stage 3, pipeline "up"
+    # after its stage 1), and the gradient groups {0, 5}, {1, 4} span nodes while {2, 3} does not
+    T = make_table([5, 7, 4, 6, 8, 9, 3], [9, 11, 8, 7, 13, 12, 6], n_devices=6, gpus_per_node=4, global_batch=4,
+                   classes=[(1, 1), (1, 2)], seq=16, hidden=8, alpha_intra_ns=3, alpha_inter_ns=50, beta_intra=64,
+                   beta_inter=4, grad=np.array([100, 0, 300, 50, 0, 700, 20]), dp_bucket_bytes=256, dp_overlap=1)
+    for m in (2, 4):
+        c = Candidate(1, 6, 1, m, 4, (0, 1, 2, 3, 4, 5, 7))
+        r = oracle.simulate(T, c, replicate=False)
+        batch, lanes = longest_path_bidirectional(T, c)
+        assert r.batch_ns == batch
+        for d in range(6):
+            assert [tuple(x) for x in r.records[r.offsets[d]:r.offsets[d + 1]].tolist()] == lanes[d], d
+        sends = {d: sorted({(int(e[0]), int(e[4] - e[3])) for e in r.records[r.offsets[d]:r.offsets[d + 1]] if e[0] in (6, 7)})
+                 for d in range(6)}
+        slow, fast = 50 + -(-(4 // m) * 16 * 8 * 2 // 4), 3 + -(-(4 // m) * 16 * 8 * 2 // 64)
+        assert sends[3] == [(6, fast), (6, slow), (7, fast), (7, slow)]      # forward down and backward up cross 3|4
+        assert sends[0] == [(6, fast), (7, fast)] and sends[5] == [(6, fast), (7, fast)]
+
+
+def test_bidirectional_rejects_what_the_schedule_does_not_define():
+    T = make_table([5] * 8, [9] * 8, n_devices=4, gpus_per_node=2, global_batch=6, classes=[(1, 1), (1, 2), (1, 3), (1, 6)],
+                   alpha_intra_ns=1, alpha_inter_ns=1, beta_intra=1, beta_inter=1)
+    assert oracle.simulate(T, Candidate(1, 4, 1, 6, 4, (0, 2, 4, 6, 8))).batch_ns > 0
+    with pytest.raises(Exception):
+        oracle.simulate(T, Candidate(1, 4, 1, 3, 4, (0, 2, 4, 6, 8)))         # an odd number of micro-batches
+    T1 = make_table([5] * 8, [9] * 8, n_devices=1, gpus_per_node=1, global_batch=6, classes=[(1, 1)],
+                    alpha_intra_ns=1, alpha_inter_ns=1, beta_intra=1, beta_inter=1)
+    with pytest.raises(Exception):
+        oracle.simulate(T1, Candidate(1, 1, 1, 6, 4, (0, 8)))                  # one device: nothing to run against
 
 
 # per-micro-batch jitter
@@ -649,7 +783,8 @@ def test_canonical_order_with_interleaved_rows():
     # every (mp, pp) is followed by its interleaved candidates: v ascending over powers of two, m
     # among the multiples of pp, partitions of the layers into pp * v virtual stages in
     # lexicographic order
-    for mask, mode in ((15, W.PARTITION_ALL), (8, W.PARTITION_ALL), (11, W.PARTITION_BALANCED)):
+    for mask, mode in ((15, W.PARTITION_ALL), (8, W.PARTITION_ALL), (11, W.PARTITION_BALANCED),
+                       (31, W.PARTITION_ALL), (16, W.PARTITION_ALL), (19, W.PARTITION_BALANCED)):
         w = W.random_small(5, n_devices=8, gpus_per_node=4, n_layers=9, global_batch=16, mp_max=2, pp_max=4,
                            m_list=(1, 2, 4, 6, 8), partition_mode=mode, sched_mask=mask, v_max=4)
         T, sp = w.table, w.space
@@ -669,19 +804,24 @@ def test_canonical_order_with_interleaved_rows():
                         for sc in (0, 1, 2):
                             if mask & (1 << sc):
                                 expect.append((mp, pp, dp, m, sc, b, 1))
-                if pp >= 2:
+                if pp >= 2 and mask & 8:
                     for v in (2, 4):
                         if pp * v > L:
                             continue
                         for m in ms:
                             if m % pp == 0:
                                 expect += [(mp, pp, dp, m, 3, b, v) for b in parts(pp * v)]
+                # ... and then by its bidirectional candidates: even m, partitions into pp stages
+                if pp >= 2 and mask & 16:
+                    for m in ms:
+                        if m % 2 == 0:
+                            expect += [(mp, pp, dp, m, 4, b, 1) for b in parts(pp)]
         n = oracle.count(T, sp)
-        assert n == len(expect) == W.count_candidates_and_cells(T, sp)[0] and any(e[4] == 3 for e in expect)
+        assert n == len(expect) == W.count_candidates_and_cells(T, sp)[0] and any(e[4] >= 3 for e in expect)
         got = oracle.enumerate_at(T, sp, np.arange(n))
         assert [(c.mp, c.pp, c.dp, c.m, c.sched, c.bounds, c.v) for c in got] == expect
         # and the enumerated interleaved candidates simulate like the same candidates given explicitly
-        for c in [c for c in got if c.sched == 3][::7]:
+        for c in [c for c in got if c.sched >= 3][::7]:
             b, _ = oracle.eval_indices(T, sp, np.array([got.index(c)]))
             assert b[0] == oracle.simulate(T, c, replicate=False, want_records=False).batch_ns
 
