@@ -155,6 +155,16 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *h_tabl
  * into pp*v virtual stages (virtual stage c*pp + d is chunk c of device d).  Such candidates have
  * schedule id 3; tables with per-micro-batch jitter do not combine with them
  * (DISTSIM_E_UNSUPPORTED).
+ * Bit 4 adds bidirectional pipelines (Chimera, which Sec. 2 names among the pipeline scheduling
+ * algorithms; schedule id 4): every (mp, pp) with pp >= 2 is then followed by the candidates
+ * that run two pipelines in opposite directions over the same devices - pipeline "down" with
+ * stage s on device s and the first m/2 micro-batches, pipeline "up" with stage s on device
+ * pp-1-s and the others, each in 1F1B order, merged on a device in the order they would
+ * interleave with unit item times - m ascending over the valid even entries, then the partition
+ * into pp stages.  A stage's gradients are reduced over the 2 dp devices that hold it (also when
+ * dp = 1).  Needs pp_max <= 32 and a table without jitter (DISTSIM_E_UNSUPPORTED otherwise);
+ * such candidates are evaluated, decoded and selected like the others, their timelines are not
+ * emitted (distsim_emit_timelines: DISTSIM_E_UNSUPPORTED).
  * Candidates are never materialised: the device decodes them from the index.
  * Fails with DISTSIM_E_ARG if a needed class (mp, b) is not in the table, with
  * DISTSIM_E_OVERFLOW if the count does not fit 62 bits.  *n_candidates receives
@@ -172,7 +182,8 @@ typedef struct {
 int distsim_set_space(distsim_ctx *ctx, const distsim_space *h_space, int64_t *n_candidates);
 
 typedef struct {
-    int32_t mp, pp, dp, m, sched;   /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B, 3: interleaved 1F1B */
+    int32_t mp, pp, dp, m, sched;   /* sched 0: GPipe, 1: 1F1B, 2: asynchronous 1F1B, 3: interleaved 1F1B,
+                                       4: bidirectional pipelines */
     int32_t micro_batch_size;       /* b = ceil(Bp / m)                            */
     int32_t class_index;            /* row of the event table                      */
     int32_t bounds[DISTSIM_MAX_PP + 1];   /* c_0 .. c_pp (c_0 .. c_{pp*v} for sched 3) */

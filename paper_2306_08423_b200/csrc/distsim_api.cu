@@ -1,6 +1,7 @@
 // Host side of the C ABI: context, validation, search-space bookkeeping, kernel launches.
 // No timeline arithmetic happens here; the host only counts the space, looks up event classes
 // and decides launch shapes.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <map>
@@ -78,6 +79,9 @@ struct distsim_ctx {
 
     // scratch
     DevBuf d_status, d_sel, d_result, d_plans, d_plan_sums, d_op_start, d_totals, d_batch, d_topk;
+    DevBuf d_order, d_order_off;          // item orders of the bidirectional schedule (see DeviceView)
+    bool have_order = false;
+    int two_way_words = 0;                // shared-memory words a warp needs for the bidirectional rows
     SideStream side;                      // extra streams of an evaluation (lock-step launches)
     cudaEvent_t planned = nullptr;        // recorded behind the emission-planning kernel
     int64_t *h_pinned = nullptr;          // 16 words of pinned host memory for small results:
@@ -98,6 +102,8 @@ struct distsim_ctx {
         v.dt32 = have_narrow && have_dt ? d_dt32.as<uint32_t>() : nullptr;
         v.next_grad = d_next_grad.as<int32_t>(); v.pe = d_pe.as<int32_t>();
         v.jsum = tc.n_jitter > 0 ? d_jsum.as<int64_t>() : nullptr;
+        v.order = have_order ? d_order.as<uint16_t>() : nullptr;
+        v.order_off = have_order ? d_order_off.as<int64_t>() : nullptr;
         v.status = d_status.as<int32_t>();
         v.stage_polls = stage_polls;
         return v;
@@ -173,6 +179,7 @@ int take_status(distsim_ctx *ctx, cudaStream_t s, int32_t code, bool *stalled)
         if (code == kStatusCopyPending)
             return fail(ctx, DISTSIM_E_TIMEOUT, "a bulk copy into shared memory never completed: results computed on this device since may be wrong");
         if (code == DISTSIM_E_RANGE) return fail(ctx, code, "candidate index out of range");
+        if (code == DISTSIM_E_UNSUPPORTED) return fail(ctx, code, "timelines of bidirectional-pipeline candidates are not emitted");
         return fail(ctx, code, "device reported an error");
     }
     return DISTSIM_OK;
@@ -189,6 +196,74 @@ void destroy_side(SideStream &ss)
 }
 
 int floor_log2(int64_t v) { int b = -1; while (v > 0) { ++b; v >>= 1; } return b; }
+
+// Item orders of the bidirectional schedule for (pp, m), both even: pipeline 0 puts stage s on
+// device s and takes the first m / 2 micro-batches, pipeline 1 puts it on device pp - 1 - s and
+// takes the others; each keeps its 1F1B order, and a device merges its two orders the way they
+// would interleave if every item took one time slot: slot by slot it runs the next item of either
+// pipeline whose input is there from an earlier slot, the one earlier in its pipeline's sequence
+// of micro-batches first.  out[d * 2 m + k] = pipeline << 15 | is-backward << 14 | micro-batch
+// within its pipeline; *kept = the most items any device runs from the last backward item of its
+// later stage on (its gradients are complete first).  Returns false if the merge does not end.
+bool bidirectional_orders(int pp, int m, std::vector<uint16_t> &out, int *kept)
+{
+    const int half = m / 2;
+    struct Item { bool bwd; int j; };
+    auto stage_of = [&](int d, int u) { return u ? pp - 1 - d : d; };
+    std::vector<std::vector<Item>> queue((size_t)2 * pp);          // [device * 2 + pipeline]
+    for (int d = 0; d < pp; ++d)
+        for (int u = 0; u < 2; ++u) {
+            const int warm = std::min(pp - stage_of(d, u), half);
+            std::vector<Item> &q = queue[(size_t)d * 2 + u];
+            int nf = 0, nb = 0;
+            for (; nf < warm; ++nf) q.push_back({false, nf});
+            while (nb < half) {
+                q.push_back({true, nb++});
+                if (nf < half) q.push_back({false, nf++});
+            }
+        }
+    // slot after which an item's result exists, [pipeline][stage][micro-batch]; 0: not yet
+    std::vector<int> done_f((size_t)2 * pp * half, 0), done_b((size_t)2 * pp * half, 0);
+    auto at = [&](int u, int s, int j) { return ((size_t)u * pp + s) * half + j; };
+    std::vector<size_t> head((size_t)2 * pp, 0);
+    std::vector<int> n_out(pp, 0), last_b_pos((size_t)2 * pp, 0);
+    out.assign((size_t)pp * 2 * m, 0);
+    int left = pp * 2 * m;
+    for (int slot = 1; left > 0; ++slot) {
+        if (slot > 4 * (m + pp)) return false;
+        std::vector<int> pick(pp, -1);
+        for (int d = 0; d < pp; ++d) {
+            int best = 0;
+            for (int u = 0; u < 2; ++u) {
+                const std::vector<Item> &q = queue[(size_t)d * 2 + u];
+                if (head[(size_t)d * 2 + u] == q.size()) continue;
+                const Item it = q[head[(size_t)d * 2 + u]];
+                const int s = stage_of(d, u);
+                int ready;                           // slot after which the input exists
+                if (!it.bwd) ready = s == 0 ? -1 : done_f[at(u, s - 1, it.j)];
+                else ready = s == pp - 1 ? done_f[at(u, s, it.j)] : done_b[at(u, s + 1, it.j)];
+                if (ready == 0 || ready >= slot) continue;
+                if (pick[d] < 0 || it.j < best) { pick[d] = u; best = it.j; }
+            }
+        }
+        for (int d = 0; d < pp; ++d) {
+            const int u = pick[d];
+            if (u < 0) continue;
+            const Item it = queue[(size_t)d * 2 + u][head[(size_t)d * 2 + u]++];
+            const int s = stage_of(d, u);
+            (it.bwd ? done_b : done_f)[at(u, s, it.j)] = slot;
+            if (it.bwd && it.j == half - 1) last_b_pos[(size_t)d * 2 + u] = n_out[d];
+            out[(size_t)d * 2 * m + n_out[d]++] = (uint16_t)((u << 15) | ((it.bwd ? 1 : 0) << 14) | it.j);
+            --left;
+        }
+    }
+    *kept = 2;
+    for (int d = 0; d < pp; ++d) {
+        const int u_first = stage_of(d, 0) > stage_of(d, 1) ? 0 : 1;      // the pipeline in which the device holds the later stage
+        *kept = std::max(*kept, 2 * m - last_b_pos[(size_t)d * 2 + u_first]);
+    }
+    return true;
+}
 
 }  // namespace
 
@@ -330,7 +405,11 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     if (!ctx->table_loaded) return fail(ctx, DISTSIM_E_STATE, "no event table loaded");
     if (sp->mp_max < 1 || sp->pp_max < 1 || sp->n_m < 1 || !sp->m_list) return fail(ctx, DISTSIM_E_ARG, "empty space");
     if (sp->pp_max > DISTSIM_MAX_PP) return fail(ctx, DISTSIM_E_ARG, "pp_max too large");
-    if ((sp->sched_mask & 15) == 0 || (sp->sched_mask & ~15)) return fail(ctx, DISTSIM_E_ARG, "bad sched_mask");
+    if ((sp->sched_mask & 31) == 0 || (sp->sched_mask & ~31)) return fail(ctx, DISTSIM_E_ARG, "bad sched_mask");
+    if ((sp->sched_mask & 16) && sp->pp_max > 32)
+        return fail(ctx, DISTSIM_E_UNSUPPORTED, "the bidirectional schedule is evaluated for at most 32 stages");
+    if ((sp->sched_mask & 16) && ctx->tc.n_jitter > 0)
+        return fail(ctx, DISTSIM_E_UNSUPPORTED, "the bidirectional schedule does not combine with per-micro-batch jitter");
     if ((sp->sched_mask & 8) && (sp->v_max < 2 || sp->v_max > DISTSIM_MAX_PP / 2))
         return fail(ctx, DISTSIM_E_ARG, "interleaved schedule needs 2 <= v_max <= 32");
     if ((sp->sched_mask & 8) && ctx->tc.n_jitter > 0)
@@ -393,16 +472,23 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
             const int64_t dp = N / (mp * pp);
             if (B % dp) continue;
             const int64_t Bp = B / dp;
-            // the row of the plain schedules, then one row of interleaved candidates per chunk count
-            for (int64_t vc = 1; vc <= (((sp->sched_mask & 8) && pp >= 2) ? sp->v_max : 1); vc *= 2) {
-                if (vc == 1 && n_sched == 0) continue;
+            // the row of the plain schedules, then one row of interleaved candidates per chunk
+            // count, then the row of bidirectional-pipeline candidates
+            std::vector<std::pair<int64_t, bool>> kinds;          // (chunks per device, two_way)
+            if (n_sched > 0) kinds.emplace_back(1, false);
+            if ((sp->sched_mask & 8) && pp >= 2)
+                for (int64_t vc = 2; vc <= sp->v_max && pp * vc <= DISTSIM_MAX_PP && pp * vc <= L; vc *= 2) kinds.emplace_back(vc, false);
+            if ((sp->sched_mask & 16) && pp >= 2) kinds.emplace_back(1, true);
+            for (const auto &kind : kinds) {
+                const int64_t vc = kind.first;
+                const bool two_way = kind.second;
+                const bool plain = vc == 1 && !two_way;
                 const int64_t P = pp * vc;              // (virtual) stages
-                if (vc > 1 && (P > DISTSIM_MAX_PP || P > L)) break;
                 Row r{};
                 r.mp = (int32_t)mp; r.pp = (int32_t)pp; r.dp = (int32_t)dp; r.log2_mp = floor_log2(mp);
-                r.v = (int32_t)vc;
+                r.v = (int32_t)vc; r.two_way = two_way ? 1 : 0;
                 r.entry0 = (int32_t)entries.size(); r.n_entries = 0;
-                r.n_sched = vc == 1 ? n_sched : 1; r.sched_list = vc == 1 ? sched_list : 3;
+                r.n_sched = plain ? n_sched : 1; r.sched_list = plain ? sched_list : 3;
                 r.p2p_period = mp >= tc.gpus_per_node ? 1 : (int32_t)(tc.gpus_per_node / mp);
                 r.n_part = sp->partition_mode == 0 ? 1 : binom[(size_t)(L - 1) * bk + (P - 1)];
                 for (int i = 0; i < sp->n_m; ++i) {
@@ -410,6 +496,7 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
                     if (m > Bp) continue;
                     if (sp->m_rule == 0 && Bp % m) continue;
                     if (vc > 1 && m % pp) continue;     // the interleaved order needs whole groups of pp micro-batches
+                    if (two_way && m % 2) continue;     // half of the micro-batches go each way
                     const int64_t b = (Bp + m - 1) / m;
                     auto it = class_of.find(std::make_pair((int)mp, (int)b));
                     if (it == class_of.end()) {
@@ -426,10 +513,11 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
                     const long double act = (long double)b * tc.seq * tc.hidden * tc.elem_bytes;
                     const long double comm = 2.0L * mp * a_max + 4.0L * act / b_min + 2 + dp * a_max + act / b_min + 2;
                     const long double p2p = a_max + act / b_min + 2;
-                    const long double nbk = (tc.bucket > 0 ? gsum / tc.bucket + L + 1 : L + 1) + vc;
+                    // (a device of a two_way row sends two streams of buckets, each over 2 dp devices)
+                    const long double nbk = ((tc.bucket > 0 ? gsum / tc.bucket + L + 1 : L + 1) + vc) * (two_way ? 2 : 1);
                     const long double bsz = tc.bucket > 0 ? (long double)tc.bucket : gsum;
                     const long double e_bound = (long double)m * (fg_max + 2.0L * L * comm + 2.0L * P * p2p) +
-                                                nbk * (2.0L * dp * a_max + 2.0L * bsz / b_min + 2);
+                                                nbk * (2.0L * (two_way ? 2 : 1) * dp * a_max + 2.0L * bsz / b_min + 2);
                     if (e_bound > tb) tb = e_bound;
                 }
                 if (r.n_entries == 0) continue;
@@ -453,6 +541,37 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     ctx->ilv_words = 0;
     for (const Row &r : rows)
         if (r.v > 1 && interleaved_words_of(r.pp, r.v) > ctx->ilv_words) ctx->ilv_words = interleaved_words_of(r.pp, r.v);
+    // item orders of the bidirectional rows: one per (pp, m), shared by the rows that differ in mp
+    ctx->have_order = false;
+    ctx->two_way_words = 0;
+    {
+        std::vector<uint16_t> all_orders;
+        std::vector<int64_t> order_off(entries.size(), 0);
+        std::map<std::pair<int, int>, std::pair<int64_t, int>> made;       // (pp, m) -> (offset, kept items)
+        for (const Row &r : rows) {
+            if (!r.two_way) continue;
+            for (int e = 0; e < r.n_entries; ++e) {
+                const int m = entries[r.entry0 + e].m;
+                auto it = made.find(std::make_pair((int)r.pp, m));
+                if (it == made.end()) {
+                    std::vector<uint16_t> one;
+                    int kept = 0;
+                    if (!bidirectional_orders(r.pp, m, one, &kept))
+                        return fail(ctx, DISTSIM_E_STATE, "the bidirectional item order could not be built");
+                    it = made.emplace(std::make_pair((int)r.pp, m), std::make_pair((int64_t)all_orders.size(), kept)).first;
+                    all_orders.insert(all_orders.end(), one.begin(), one.end());
+                }
+                order_off[r.entry0 + e] = it->second.first | ((int64_t)it->second.second << 48);
+                const int words = bidirectional_words_of(r.pp, it->second.second);
+                if (words > ctx->two_way_words) ctx->two_way_words = words;
+            }
+        }
+        if (!all_orders.empty()) {
+            if (int rc = upload(ctx, ctx->d_order, all_orders.data(), all_orders.size(), "upload item orders")) return rc;
+            if (int rc = upload(ctx, ctx->d_order_off, order_off.data(), order_off.size(), "upload item orders")) return rc;
+            ctx->have_order = true;
+        }
+    }
     SpaceConst &sc = ctx->sc;
     sc.n_rows = (int32_t)rows.size(); sc.n_entries = (int32_t)entries.size();
     sc.pp_max = sp->pp_max; sc.partition_mode = sp->partition_mode; sc.binom_k = bk; sc.pad = 0;
@@ -553,7 +672,7 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const DeviceView v = ctx->view();
     launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
-                d_batch_ns, d_stage_busy_ns, &ctx->launches);
+                d_batch_ns, d_stage_busy_ns, &ctx->launches, ctx->two_way_words);
     CU(cudaGetLastError(), "evaluation launch");
     return DISTSIM_OK;
 }
@@ -575,7 +694,7 @@ int distsim_eval_select(distsim_ctx *ctx, void *stream, int64_t first, int64_t c
     const SelectScratch sc = ctx->select_scratch();
     if (ctx->phase_timing) cudaEventRecord(ctx->phase_ev[0], s);
     launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
-                d_batch_ns, nullptr, &ctx->launches);
+                d_batch_ns, nullptr, &ctx->launches, ctx->two_way_words);
     CU(cudaGetLastError(), "evaluation launch");
     if (ctx->phase_timing) cudaEventRecord(ctx->phase_ev[1], s);
     const bool want_best = d_best || h_best_index;
@@ -736,7 +855,7 @@ int distsim_testing_space_cells(distsim_ctx *ctx, int64_t *h_cells, int64_t *h_c
             total += c;
             // 32-bit arithmetic is used where the entry's time bound allows it and the row is
             // evaluated by the one-partition-per-thread kernel
-            if (en.bound < ((int64_t)1 << 32) && row.pp <= 16 && row.v == 1) narrow += c;
+            if (en.bound < ((int64_t)1 << 32) && row.pp <= 16 && row.v == 1 && !row.two_way) narrow += c;
         }
     *h_cells = total >= (__int128)kSat ? kSat : (int64_t)total;
     *h_cells_32bit = narrow >= (__int128)kSat ? kSat : (int64_t)narrow;

@@ -16,7 +16,7 @@
 //   emit_buckets_kernel  gradient-bucket records of every stage.
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
-#include "interleaved.cuh"
+#include "bidirectional.cuh"
 
 namespace distsim {
 
@@ -312,6 +312,15 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
         } else {
             const int r = find_row(v, index);
             const Row row = v.rows[r];
+            if (row.two_way) {
+                // timelines of bidirectional-pipeline candidates are not emitted
+                if ((threadIdx.x & 31) == 0) {
+                    plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0; plan->v = 1;
+                    plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
+                    for (int w = 0; w < kSumWords; ++w) sums[(int64_t)i * kSumWords + w] = 0;
+                    atomicCAS(v.status, 0, DISTSIM_E_UNSUPPORTED);
+                }
+            } else {
             int64_t *rec_i = op_start + (int64_t)i * op_words_per_cand;
             if (row.v > 1) {
                 plan_interleaved(v, row, r, index, plan, rec_i, binom, sums + (int64_t)i * kSumWords,
@@ -320,6 +329,7 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
             int64_t *rec = op_start + (int64_t)i * op_words_per_cand;
             if (row.pp > 32) plan_candidate<2>(v, row, r, index, plan, rec, binom, sums + (int64_t)i * kSumWords);
             else plan_candidate<1>(v, row, r, index, plan, rec, binom, sums + (int64_t)i * kSumWords);
+            }
             }
         }
     }
@@ -777,6 +787,7 @@ void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const 
 }
 
 int interleaved_words_of(int pp, int v) { return interleaved_words(pp, v); }
+int bidirectional_words_of(int pp, int kept) { return bidirectional_words(pp, kept); }
 
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,

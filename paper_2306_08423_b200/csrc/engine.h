@@ -61,10 +61,15 @@ struct Row {
     int32_t p2p_period;   // boundary d|d+1 is inter-node iff ((d+1) & (p2p_period-1)) == 0
     int32_t v;            // model chunks per device: 1, or > 1 for a row of interleaved 1F1B candidates
                           // (one schedule, id 3; partitions into pp * v virtual stages)
+    int32_t two_way;      // 1 for a row of bidirectional-pipeline candidates (one schedule, id 4; v = 1;
+                          // even micro-batch counts), else 0
+    int64_t t_full_near;  // two_way rows: t_full is the cost of a full gradient bucket over the 2 dp holders
+                          // of a stage when they span nodes, this one when a node holds them all   [device-filled]
 };
 
-// Schedule id (0 GPipe, 1 1F1B, 2 asynchronous 1F1B, 3 interleaved 1F1B) of position sc among a row's schedules.
-__host__ __device__ inline int row_sched(const Row &row, int sc) { return (row.sched_list >> (2 * sc)) & 3; }
+// Schedule id (0 GPipe, 1 1F1B, 2 asynchronous 1F1B, 3 interleaved 1F1B, 4 bidirectional pipelines)
+// of position sc among a row's schedules.
+__host__ __device__ inline int row_sched(const Row &row, int sc) { return row.two_way ? 4 : (row.sched_list >> (2 * sc)) & 3; }
 
 struct Entry {
     int32_t m, b, cls, row;
@@ -111,6 +116,12 @@ struct DeviceView {
     const int32_t *pe;               // [L+1] number of expert layers before layer l
     const int64_t *jsum;             // [n_entries][DISTSIM_MAX_PP] total jitter of the m forward and
                                      // m backward items of a stage (nullptr without jitter)
+    const uint16_t *order;           // bidirectional schedule: every device's items in its order,
+                                     // [entry's offset + device * 2 m + position]: pipeline << 15 |
+                                     // is-backward << 14 | micro-batch within its pipeline
+    const int64_t *order_off;        // [n_entries] offset of the entry's orders in `order` (low 48 bits) and,
+                                     // above them, the items a device may run from the last backward item
+                                     // of its earlier-finishing pipeline on (nullptr: no such rows)
     int32_t *status;                 // device status word: 0 ok, else first error code
     int32_t stage_polls;             // polls of the first wait for staged tables (the drain wait keeps its own limit)
 };
@@ -186,7 +197,8 @@ struct SideStream {
 // is ordered after what `s` held before the call and before what is enqueued on `s` after it.
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
-                 int64_t *launches);
+                 int64_t *launches,
+                 int two_way_words = 0 /* shared-memory words a warp needs for the space's bidirectional rows */);
 // Cuts candidates [lo, hi) of a row of pp stages into pieces of at most max_blocks lock-step
 // blocks each; returns the number of pieces and writes the first max_pieces of them.
 int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
@@ -266,6 +278,7 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
                       cudaEvent_t planned /* nullable: recorded behind the planning kernel */,
                       int64_t *launches);
 int interleaved_words_of(int pp, int v);           // those words for one row
+int bidirectional_words_of(int pp, int kept);      // shared-memory words a warp needs for a bidirectional candidate
 // out[k] = order-sensitive checksum of the records [offsets[k], offsets[k + 1]).
 void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const int64_t *offsets, int64_t n_lists,
                            uint64_t *out, int64_t *launches);

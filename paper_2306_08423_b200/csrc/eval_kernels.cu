@@ -17,7 +17,7 @@
 #include "recurrence.cuh"
 #include "smem_stage.cuh"
 #include "eval_thread.cuh"
-#include "interleaved.cuh"
+#include "bidirectional.cuh"
 
 namespace distsim {
 
@@ -105,7 +105,8 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     else lockstep_block<1, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar, binom);
 }
 
-// Interleaved 1F1B candidates: a candidate per warp (interleaved.cuh).
+// Interleaved 1F1B and bidirectional-pipeline candidates: a candidate per warp (interleaved.cuh,
+// bidirectional.cuh).
 __global__ void __launch_bounds__(kIlvThreads)
 eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
                         int64_t *__restrict__ busy_out, int words_per_warp)
@@ -123,8 +124,10 @@ eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *_
     if (!valid) local = wk.hi - 1;                 // an idle warp shadows a real candidate
     const CandidateCoords cc = split_local(row, local);
     const Entry en = v.entries[cc.entry];
-    const IlvArrays A = interleaved_arrays(ilv_s + (int64_t)warp * words_per_warp, row.pp, row.v);
-    const IlvResult R = interleaved_candidate(v, row, en, cc, binom, A, nullptr);
+    int64_t *mine = ilv_s + (int64_t)warp * words_per_warp;
+    const IlvResult R = row.two_way
+        ? bidirectional_candidate(v, row, en, cc, binom, bidirectional_arrays(mine, row.pp, order_kept(v, cc.entry)), nullptr)
+        : interleaved_candidate(v, row, en, cc, binom, interleaved_arrays(mine, row.pp, row.v), nullptr);
     if (!valid) return;
     const int64_t out = row.offset + local - first;
     if (lane == 0) batch_out[out] = R.batch;
@@ -259,7 +262,7 @@ int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int6
 
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
-                 int64_t *launches)
+                 int64_t *launches, int two_way_words)
 {
     const int64_t last = first + count;
     struct ThreadItem { EvalWork w; int lg; bool narrow; int blocks, words; };
@@ -287,7 +290,7 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
         const int64_t lo = first > row.offset ? first - row.offset : 0;
         const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
         if (hi <= lo) continue;
-        if (row.v > 1) {
+        if (row.v > 1 || row.two_way) {
             constexpr int64_t cpb = kIlvThreads / 32;
             for (int64_t a = lo; a < hi; a += kPieceBlocks * cpb) {
                 EvalWork w{};
@@ -295,7 +298,7 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
                 w.nx = (int)((w.hi - w.lo + cpb - 1) / cpb);
                 ilv_items.push_back(w);
             }
-            const int words = interleaved_words(row.pp, row.v);
+            const int words = row.two_way ? two_way_words : interleaved_words(row.pp, row.v);
             if (words > ilv_words) ilv_words = words;
             continue;
         }

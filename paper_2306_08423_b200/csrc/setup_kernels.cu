@@ -2,28 +2,11 @@
 // They run once per (table, search space), so they favour clarity over speed; every
 // division of the communication cost model happens here and none in the hot kernels.
 #include "engine.h"
+#include "costs.cuh"
 
 namespace distsim {
 
 namespace {
-
-__device__ __forceinline__ int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
-
-// Ring all-reduce over n devices of `bytes`: 2(n-1) steps, each paying the latency and moving
-// 1/n of the tensor, i.e. a per-device volume of 2(n-1)*bytes/n (paper Sec. 4.2).
-__device__ __forceinline__ int64_t ring_cost(int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
-{
-    return 2 * (n - 1) * alpha + ceil_div(2 * (n - 1) * bytes, n * beta);
-}
-
-// All-reduce event time: directly modelled up to k = ar_profile_max devices; above, the k-device
-// time scaled by the per-device volume 2(n-1)S/n of the actual device count (paper Sec. 4.2).
-__device__ __forceinline__ int64_t allreduce_cost(const TableConst &tc, int64_t n, int64_t bytes, int64_t alpha, int64_t beta)
-{
-    const int64_t k = tc.ar_profile_max;
-    if (k <= 1 || n <= k) return ring_cost(n, bytes, alpha, beta);
-    return ceil_div(ring_cost(k, bytes, alpha, beta) * k * (n - 1), (k - 1) * n);
-}
 
 // One thread per entry: the communication-event costs that depend on (mp, dp, b).
 // The first thread of each row also fills the row's full-bucket cost.
@@ -53,11 +36,19 @@ __global__ void fill_entries_kernel(TableConst tc, Row *rows, int n_rows, Entry 
     en.p2p_inter = tc.alpha_inter + ceil_div(act, tc.beta_inter);
     entries[i] = en;
     if (i == row.entry0) {
-        int64_t t_full = 0;
-        if (row.dp > 1 && tc.bucket > 0)
+        int64_t t_full = 0, t_full_near = 0;
+        if (row.two_way) {
+            // a stage's gradients are reduced over its 2 dp holders: across nodes, or inside one
+            if (tc.bucket > 0) {
+                t_full = allreduce_cost(tc, 2 * (int64_t)row.dp, tc.bucket, tc.alpha_inter, tc.beta_inter);
+                t_full_near = allreduce_cost(tc, 2 * (int64_t)row.dp, tc.bucket, tc.alpha_intra, tc.beta_intra);
+            }
+        } else if (row.dp > 1 && tc.bucket > 0) {
             t_full = allreduce_cost(tc, row.dp, tc.bucket, dp_inter ? tc.alpha_inter : tc.alpha_intra,
                                dp_inter ? tc.beta_inter : tc.beta_intra);
+        }
         rows[en.row].t_full = t_full;
+        rows[en.row].t_full_near = t_full_near;
     }
 }
 
@@ -106,7 +97,8 @@ __global__ void build_bucket_tables_kernel(TableConst tc, RawTable raw, const Ro
         int64_t full = 0, rem = w;
         if (tc.bucket > 0) { full = w / tc.bucket; rem = w - full * tc.bucket; }
         nbr[l] = full;
-        tpr[l] = (rem > 0 && row.dp > 1) ? allreduce_cost(tc, row.dp, rem, a, be) : 0;
+        // (a two_way row keeps the bytes of the trailing bucket: its cost depends on the device)
+        tpr[l] = row.two_way ? rem : (rem > 0 && row.dp > 1) ? allreduce_cost(tc, row.dp, rem, a, be) : 0;
     }
     for (int l = e + 1; l < L1; ++l) { nbr[l] = 0; tpr[l] = 0; }
 }
@@ -192,7 +184,16 @@ __global__ void entry_bound_kernel(DeviceView v, Entry *entries, int64_t *jsum)
     // interleaved candidates: the last device sends to the first between chunks
     if (row.v > 1) per_mb += 2 * (row.v - 1) * (en.p2p_inter > en.p2p_intra ? en.p2p_inter : en.p2p_intra);
     int64_t excess = 0;
-    if (row.dp > 1) {
+    if (row.two_way) {
+        // two streams of buckets per device, each at most the whole model's, priced across nodes
+        const int64_t *nbL = v.nb + row.row_tab_off + (int64_t)L * L1;
+        const int64_t *tpL = v.tp + row.row_tab_off + (int64_t)L * L1;
+        const int64_t t_max = row.t_full > row.t_full_near ? row.t_full : row.t_full_near;
+        const int64_t one = v.tc.bucket > 0 ? t_max
+                                            : allreduce_cost(v.tc, 2 * (int64_t)row.dp, tpL[0], v.tc.alpha_inter, v.tc.beta_inter) +
+                                              allreduce_cost(v.tc, 2 * (int64_t)row.dp, tpL[0], v.tc.alpha_intra, v.tc.beta_intra);
+        excess = 2 * (nbL[0] * t_max + one);
+    } else if (row.dp > 1) {
         const int64_t *nbL = v.nb + row.row_tab_off + (int64_t)L * L1;
         const int64_t *tpL = v.tp + row.row_tab_off + (int64_t)L * L1;
         // a device's buckets cost at most all full buckets of the model plus one more bucket per

@@ -251,6 +251,72 @@ def test_interleaved_1f1b_on_the_64_device_shape(E, ctx):
     check_emission(E, ctx, w, [ilv[0], ilv[len(ilv) // 2], ilv[-1], 0])
 
 
+@pytest.mark.parametrize("case", range(6))
+def test_bidirectional_pipelines_every_candidate(E, ctx, case):
+    """Spaces with bidirectional-pipeline candidates (sched_mask bit 4) beside the other schedules
+    and alone: every candidate's batch time and per-device activity time, the decoded candidates,
+    the best one and the k fastest, sub-ranges; emission of such a candidate is refused."""
+    mask = (31, 16, 19, 23, 17, 24)[case]
+    kw = dict(n_devices=(8, 8, 8, 16, 4, 8)[case], gpus_per_node=(4, 2, 4, 8, 4, 2)[case],
+              n_layers=(9, 8, 10, 9, 12, 16)[case], global_batch=16, mp_max=2, pp_max=(4, 4, 4, 8, 4, 8)[case],
+              m_list=(1, 2, 4, 6, 8, 16), partition_mode=(W.PARTITION_ALL, W.PARTITION_ALL, W.PARTITION_BALANCED,
+                                                          W.PARTITION_ALL, W.PARTITION_ALL, W.PARTITION_BALANCED)[case],
+              dp_overlap=case % 2, dp_bucket_bytes=0 if case == 2 else 3000, sched_mask=mask, v_max=2)
+    w = W.random_small(720 + case, **kw)
+    n = load(E, ctx, w)
+    cands = oracle.enumerate_at(w.table, w.space, np.arange(n))
+    assert any(c.sched == 4 and c.pp == kw["pp_max"] for c in cands) and (mask == 16 or any(c.sched != 4 for c in cands))
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices_parallel(w.table, w.space, np.arange(n), THREADS, replicate=False,
+                                             pp_stride=w.space.pp_max)
+    gb = batch.cpu().numpy()
+    assert (gb == ob).all(), [(i, cands[i]) for i in np.argwhere(gb != ob)[:3, 0]]
+    assert (sb.cpu().numpy() == obusy).all()
+    for i in range(0, n, max(1, n // 97)):
+        d = E.distsim_decode(ctx, i)
+        c = cands[i]
+        assert (d["mp"], d["pp"], d["dp"], d["m"], d["sched"], d["bounds"], d["v"]) == (c.mp, c.pp, c.dp, c.m, c.sched, c.bounds, c.v)
+    order = np.lexsort((np.arange(n), ob))
+    k = min(n, 64)
+    ki, kt, got = dev(k), dev(k), dev(n)
+    assert E.distsim_eval_select(ctx, 0, n, got, k, ki, kt) == (order[0], ob[order[0]])
+    assert (ki.cpu().numpy() == order[:k]).all() and (kt.cpu().numpy() == ob[order[:k]]).all()
+    rng = np.random.default_rng(case)
+    for _ in range(6):
+        first = int(rng.integers(0, n)); count = int(rng.integers(1, n - first + 1))
+        out = dev(count)
+        E.distsim_eval_strategies(ctx, first, count, out)
+        assert (out.cpu().numpy() == ob[first:first + count]).all()
+    cells, _ = E.distsim_testing_space_cells(ctx)
+    assert cells == W.count_candidates_and_cells(w.table, w.space)[1]
+    two_way = [i for i, c in enumerate(cands) if c.sched == 4]
+    with pytest.raises(E.DistsimError) as err:
+        E.distsim_emit_timelines(ctx, torch.tensor(two_way[:1], dtype=torch.int64, device="cuda"), 1, None, 0)
+    assert err.value.code == E.E_UNSUPPORTED
+    others = [i for i, c in enumerate(cands) if c.sched != 4]
+    if others:
+        check_emission(E, ctx, w, others[:: max(1, len(others) // 5)][:5])      # the context is as usable as before
+
+
+def test_bidirectional_pipelines_on_the_64_device_shape(E, ctx):
+    """The 64-device workload with bidirectional pipelines added to its schedules: sampled
+    candidates of every row against the oracle, the best candidate over the whole space."""
+    w = W.config1()
+    w.space.sched_mask = 19
+    n = load(E, ctx, w)
+    assert n > 38_838_764
+    idx, total = stratified_indices(w.table, w.space, 60, 5)
+    assert total == n
+    cands = oracle.enumerate_at(w.table, w.space, idx)
+    assert sum(c.sched == 4 for c in cands) > 500 and any(c.sched == 4 and c.pp == 16 and c.m == 128 for c in cands)
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    ob, _ = oracle.eval_indices_parallel(w.table, w.space, idx, THREADS, replicate=False)
+    gb = batch[torch.from_numpy(idx).cuda()].cpu().numpy()
+    assert (gb == ob).all(), idx[np.argwhere(gb != ob)[:5, 0]]
+    bi, bt = E.distsim_argmin(ctx, batch, 0, n)
+    assert oracle.eval_indices(w.table, w.space, np.array([bi]))[0][0] == bt == int(batch.min().item())
+
+
 @pytest.mark.parametrize("case", range(12))
 def test_randomised_spaces_sampled_parity(E, ctx, case):
     """Randomly drawn clusters, layer counts, micro-batch lists (around m = pp, where the
