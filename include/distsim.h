@@ -162,9 +162,7 @@ int distsim_load_event_table(distsim_ctx *ctx, const distsim_event_table *h_tabl
  * pp-1-s and the others, each in 1F1B order, merged on a device in the order they would
  * interleave with unit item times - m ascending over the valid even entries, then the partition
  * into pp stages.  A stage's gradients are reduced over the 2 dp devices that hold it (also when
- * dp = 1).  Needs pp_max <= 32 and a table without jitter (DISTSIM_E_UNSUPPORTED otherwise);
- * such candidates are evaluated, decoded and selected like the others, their timelines are not
- * emitted (distsim_emit_timelines: DISTSIM_E_UNSUPPORTED).
+ * dp = 1).  Needs pp_max <= 32 and a table without jitter (DISTSIM_E_UNSUPPORTED otherwise).
  * Candidates are never materialised: the device decodes them from the index.
  * Fails with DISTSIM_E_ARG if a needed class (mp, b) is not in the table, with
  * DISTSIM_E_OVERFLOW if the count does not fit 62 bits.  *n_candidates receives

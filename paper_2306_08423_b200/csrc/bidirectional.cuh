@@ -4,7 +4,7 @@
 // Pipeline 0 ("down") has stage s on device s and takes micro-batches 0 .. m/2 - 1, pipeline 1
 // ("up") has stage s on device pp - 1 - s and takes m/2 .. m - 1 (pp and m even); both cut the
 // model at the same pp - 1 bounds.  A device holds one stage of each and runs their items in the
-// merged order the host worked out for (pp, m) (DeviceView::order): each pipeline keeps its 1F1B
+// merged order the host worked out for (pp, m) (DeviceView::order, 2 m + 1 slots per device): each pipeline keeps its 1F1B
 // order, the merge is the one of unit time slots.  Algorithm 1 of the paper runs unchanged over
 // the 2 pp (pipeline, stage) pairs with one free time per device.  The weights of a stage are on
 // two devices of every replica, so its gradients are reduced over 2 dp devices - also when
@@ -45,6 +45,17 @@ __device__ __forceinline__ IlvArrays bidirectional_arrays(int64_t *base, int pp,
     A.cnt_b = A.cnt_f + P;
     A.bounds = A.cnt_b + P;
     return A;
+}
+
+// How many items of each kind precede position `pos` (0 .. 2 m) of device d's order.
+struct ItemsBefore { int f0, b0, f1, b1; };
+__device__ __forceinline__ ItemsBefore items_before(const DeviceView &v, int64_t entry_off, int m, int d, int pos)
+{
+    const uint32_t w = __ldg(&v.order_before[entry_off + (int64_t)d * (2 * m + 1) + pos]);
+    ItemsBefore n;
+    n.f0 = (int)(w & 511u); n.b0 = (int)((w >> 9) & 511u); n.f1 = (int)((w >> 18) & 511u);
+    n.b1 = pos - n.f0 - n.b0 - n.f1;
+    return n;
 }
 
 // Where an entry's orders start in DeviceView::order, and its kept items per device.
@@ -156,7 +167,7 @@ __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v
 
     // ---- the rounds: every device whose next item has its input runs it ---------------------
     const int d = lane;
-    const uint16_t *mine = v.order + order_offset(v, cc.entry) + (int64_t)d * 2 * m;
+    const uint16_t *mine = v.order + order_offset(v, cc.entry) + (int64_t)d * (2 * m + 1);
     int n_done = 0;
     int64_t free_at = 0;
     const int limit = 2 * (m + pp) + 8;             // the merged order takes 2 m + pp - 2 rounds when m >= pp, never more than 2 (m + pp)

@@ -79,7 +79,7 @@ struct distsim_ctx {
 
     // scratch
     DevBuf d_status, d_sel, d_result, d_plans, d_plan_sums, d_op_start, d_totals, d_batch, d_topk;
-    DevBuf d_order, d_order_off;          // item orders of the bidirectional schedule (see DeviceView)
+    DevBuf d_order, d_order_before, d_order_off;          // item orders of the bidirectional schedule (see DeviceView)
     bool have_order = false;
     int two_way_words = 0;                // shared-memory words a warp needs for the bidirectional rows
     SideStream side;                      // extra streams of an evaluation (lock-step launches)
@@ -104,6 +104,7 @@ struct distsim_ctx {
         v.jsum = tc.n_jitter > 0 ? d_jsum.as<int64_t>() : nullptr;
         v.order = have_order ? d_order.as<uint16_t>() : nullptr;
         v.order_off = have_order ? d_order_off.as<int64_t>() : nullptr;
+        v.order_before = have_order ? d_order_before.as<uint32_t>() : nullptr;
         v.status = d_status.as<int32_t>();
         v.stage_polls = stage_polls;
         return v;
@@ -179,7 +180,6 @@ int take_status(distsim_ctx *ctx, cudaStream_t s, int32_t code, bool *stalled)
         if (code == kStatusCopyPending)
             return fail(ctx, DISTSIM_E_TIMEOUT, "a bulk copy into shared memory never completed: results computed on this device since may be wrong");
         if (code == DISTSIM_E_RANGE) return fail(ctx, code, "candidate index out of range");
-        if (code == DISTSIM_E_UNSUPPORTED) return fail(ctx, code, "timelines of bidirectional-pipeline candidates are not emitted");
         return fail(ctx, code, "device reported an error");
     }
     return DISTSIM_OK;
@@ -202,10 +202,10 @@ int floor_log2(int64_t v) { int b = -1; while (v > 0) { ++b; v >>= 1; } return b
 // takes the others; each keeps its 1F1B order, and a device merges its two orders the way they
 // would interleave if every item took one time slot: slot by slot it runs the next item of either
 // pipeline whose input is there from an earlier slot, the one earlier in its pipeline's sequence
-// of micro-batches first.  out[d * 2 m + k] = pipeline << 15 | is-backward << 14 | micro-batch
+// of micro-batches first.  out[d * (2 m + 1) + k] = pipeline << 15 | is-backward << 14 | micro-batch
 // within its pipeline; *kept = the most items any device runs from the last backward item of its
 // later stage on (its gradients are complete first).  Returns false if the merge does not end.
-bool bidirectional_orders(int pp, int m, std::vector<uint16_t> &out, int *kept)
+bool bidirectional_orders(int pp, int m, std::vector<uint16_t> &out, std::vector<uint32_t> &before, int *kept)
 {
     const int half = m / 2;
     struct Item { bool bwd; int j; };
@@ -227,7 +227,10 @@ bool bidirectional_orders(int pp, int m, std::vector<uint16_t> &out, int *kept)
     auto at = [&](int u, int s, int j) { return ((size_t)u * pp + s) * half + j; };
     std::vector<size_t> head((size_t)2 * pp, 0);
     std::vector<int> n_out(pp, 0), last_b_pos((size_t)2 * pp, 0);
-    out.assign((size_t)pp * 2 * m, 0);
+    const size_t stride = (size_t)2 * m + 1;
+    out.assign((size_t)pp * stride, 0);
+    before.assign((size_t)pp * stride, 0);
+    std::vector<uint32_t> so_far(pp, 0);            // counts packed as in DeviceView::order_before
     int left = pp * 2 * m;
     for (int slot = 1; left > 0; ++slot) {
         if (slot > 4 * (m + pp)) return false;
@@ -253,10 +256,14 @@ bool bidirectional_orders(int pp, int m, std::vector<uint16_t> &out, int *kept)
             const int s = stage_of(d, u);
             (it.bwd ? done_b : done_f)[at(u, s, it.j)] = slot;
             if (it.bwd && it.j == half - 1) last_b_pos[(size_t)d * 2 + u] = n_out[d];
-            out[(size_t)d * 2 * m + n_out[d]++] = (uint16_t)((u << 15) | ((it.bwd ? 1 : 0) << 14) | it.j);
+            before[(size_t)d * stride + n_out[d]] = so_far[d];
+            out[(size_t)d * stride + n_out[d]++] = (uint16_t)((u << 15) | ((it.bwd ? 1 : 0) << 14) | it.j);
+            if (u == 0) so_far[d] += it.bwd ? (1u << 9) : 1u;
+            else if (!it.bwd) so_far[d] += 1u << 18;
             --left;
         }
     }
+    for (int d = 0; d < pp; ++d) before[(size_t)d * stride + 2 * m] = so_far[d];
     *kept = 2;
     for (int d = 0; d < pp; ++d) {
         const int u_first = stage_of(d, 0) > stage_of(d, 1) ? 0 : 1;      // the pipeline in which the device holds the later stage
@@ -546,6 +553,7 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
     ctx->two_way_words = 0;
     {
         std::vector<uint16_t> all_orders;
+        std::vector<uint32_t> all_before;
         std::vector<int64_t> order_off(entries.size(), 0);
         std::map<std::pair<int, int>, std::pair<int64_t, int>> made;       // (pp, m) -> (offset, kept items)
         for (const Row &r : rows) {
@@ -555,11 +563,13 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
                 auto it = made.find(std::make_pair((int)r.pp, m));
                 if (it == made.end()) {
                     std::vector<uint16_t> one;
+                    std::vector<uint32_t> one_before;
                     int kept = 0;
-                    if (!bidirectional_orders(r.pp, m, one, &kept))
+                    if (!bidirectional_orders(r.pp, m, one, one_before, &kept))
                         return fail(ctx, DISTSIM_E_STATE, "the bidirectional item order could not be built");
                     it = made.emplace(std::make_pair((int)r.pp, m), std::make_pair((int64_t)all_orders.size(), kept)).first;
                     all_orders.insert(all_orders.end(), one.begin(), one.end());
+                    all_before.insert(all_before.end(), one_before.begin(), one_before.end());
                 }
                 order_off[r.entry0 + e] = it->second.first | ((int64_t)it->second.second << 48);
                 const int words = bidirectional_words_of(r.pp, it->second.second);
@@ -568,6 +578,7 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
         }
         if (!all_orders.empty()) {
             if (int rc = upload(ctx, ctx->d_order, all_orders.data(), all_orders.size(), "upload item orders")) return rc;
+            if (int rc = upload(ctx, ctx->d_order_before, all_before.data(), all_before.size(), "upload item orders")) return rc;
             if (int rc = upload(ctx, ctx->d_order_off, order_off.data(), order_off.size(), "upload item orders")) return rc;
             ctx->have_order = true;
         }
@@ -779,7 +790,8 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     CU(ctx->d_plan_sums.reserve((size_t)n * kEmitSumWords * sizeof(int64_t)), "alloc plan summaries");
     const DeviceView v = ctx->view();
     launch_emit_plan(s, v, d_indices, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
-                     ctx->op_words_per_cand, ctx->d_plan_sums.as<int64_t>(), d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(), ctx->ilv_words,
+                     ctx->op_words_per_cand, ctx->d_plan_sums.as<int64_t>(), d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>(),
+                     std::max(ctx->ilv_words, ctx->two_way_words),
                      ctx->h_pinned + 8, ctx->planned, &ctx->launches);
     CU(cudaGetLastError(), "emission planning launch");
     // The planning kernel's last block writes the totals and the status word straight into the

@@ -140,7 +140,7 @@ __device__ __forceinline__ void plan_candidate(const DeviceView &v, const Row &r
     if (lane == 0) {
         plan->index = index; plan->batch_ns = R.batch;
         plan->row = row_index; plan->entry = cc.entry; plan->m = en.m; plan->sched = cc.sched;
-        plan->pp = row.pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1; plan->v = 1;
+        plan->pp = row.pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1; plan->v = 1; plan->two_way = 0;
         plan->stage_rec_prefix[row.pp] = total;
         plan->rec_total = total * row.mp * row.dp;
         // a run of tile_items items of any mix must fit the image of kTileWords words
@@ -220,7 +220,7 @@ __device__ __forceinline__ void plan_interleaved(const DeviceView &v, const Row 
     if (lane == 0) {
         plan->index = index; plan->batch_ns = R.batch;
         plan->row = row_index; plan->entry = cc.entry; plan->m = en.m; plan->sched = 3;
-        plan->pp = pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1; plan->v = vch;
+        plan->pp = pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1; plan->v = vch; plan->two_way = 0;
         plan->stage_rec_prefix[pp] = total;
         plan->rec_total = total * row.mp * row.dp;
         const int n_items = 2 * en.m * vch;                       // items of a device
@@ -229,6 +229,83 @@ __device__ __forceinline__ void plan_interleaved(const DeviceView &v, const Row 
         plan->tile_items = (n_items + n_chunks - 1) / n_chunks;
         plan->run_words = plan->tile_items * widest * 5;
         plan->tmpl_words = both * 5;                              // the templates of all chunks of the widest device
+        const int64_t reps = (int64_t)row.mp * row.dp;
+        sum[kSumRecords] = plan->rec_total;
+        sum[kSumItemTiles] = (int64_t)pp * ((n_items + plan->tile_items - 1) / plan->tile_items) *
+                             ((reps + kTileReplicas - 1) / kTileReplicas);
+        sum[kSumBucketTiles] = (int64_t)pp * ((reps + kBucketReplicas - 1) / kBucketReplicas);
+        sum[kSumTmplWords] = plan->tmpl_words;
+        sum[kSumBucketRecs] = most_buckets;
+        sum[kSumRunWords] = plan->run_words;
+    }
+}
+
+// The same for a bidirectional-pipeline candidate: the plan's "chunks" are its two pipelines, the
+// per-stage arrays are indexed pipeline * pp + device, bounds holds the pp + 1 shared bounds.
+__device__ __forceinline__ void plan_bidirectional(const DeviceView &v, const Row &row, int row_index, int64_t index,
+                                                   EmitPlan *plan, int64_t *rec, const int64_t *binom, int64_t *sum,
+                                                   const IlvArrays &A)
+{
+    const int lane = threadIdx.x & 31;
+    const int pp = row.pp;
+    const CandidateCoords cc = split_local(row, index - row.offset);
+    const Entry en = v.entries[cc.entry];
+    const IlvResult R = bidirectional_candidate(v, row, en, cc, binom, A, rec);
+    const int L1 = v.tc.n_layers + 1, half = en.m / 2;
+    int widest = 1, both = 0;
+    int64_t dev_recs = 0, dev_buckets = 0;
+    if (lane < pp) {
+        const int d = lane;
+        for (int c = 0; c < 2; ++c) {
+            const int st = c ? pp - 1 - d : d;                     // the device's stage in pipeline c
+            const int a = A.bounds[st], e = A.bounds[st + 1];
+            const int64_t per_dir = (int64_t)(e - a) * (row.mp > 1 ? 2 : 1) + (row.dp > 1 ? v.pe[e] - v.pe[a] : 0);
+            const int64_t rf = per_dir + (st < pp - 1 ? 1 : 0);
+            const int64_t rb = per_dir + (st > 0 ? 1 : 0);
+            // the stage's gradients go to its other holder at least: buckets whenever it has gradient bytes
+            const int64_t *nbt = v.nb + row.row_tab_off, *tpt = v.tp + row.row_tab_off;
+            const int64_t kb = nbt[(int64_t)e * L1 + a] + (tpt[(int64_t)e * L1 + a] > 0 ? 1 : 0);
+            const int x = c * pp + d;
+            plan->rf[x] = (int32_t)rf; plan->rb[x] = (int32_t)rb;
+            plan->last_b_start[x] = A.last_b[c * pp + st];
+            dev_recs += (int64_t)half * (rf + rb) + kb;
+            dev_buckets += kb;
+            widest = max(widest, (int)max(rf, rb));
+            both += (int)(rf + rb);
+        }
+        plan->bounds[d] = A.bounds[d];
+        if (d == pp - 1) plan->bounds[pp] = A.bounds[pp];
+        plan->n_buckets[d] = dev_buckets;
+        plan->stage_recs[d] = dev_recs;
+        plan->busy[d] = R.busy;
+        plan->main_end[d] = R.main_end;
+    }
+    int64_t incl = dev_recs, most_buckets = dev_buckets;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int64_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    const int64_t total = __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        widest = max(widest, __shfl_xor_sync(0xffffffffu, widest, o));
+        both = max(both, __shfl_xor_sync(0xffffffffu, both, o));
+        most_buckets = max64(most_buckets, __shfl_xor_sync(0xffffffffu, most_buckets, o));
+    }
+    if (lane < pp) plan->stage_rec_prefix[lane] = incl - dev_recs;
+    if (lane == 0) {
+        plan->index = index; plan->batch_ns = R.batch;
+        plan->row = row_index; plan->entry = cc.entry; plan->m = en.m; plan->sched = 4;
+        plan->pp = pp; plan->mp = row.mp; plan->dp = row.dp; plan->ok = 1; plan->v = 2; plan->two_way = 1;
+        plan->stage_rec_prefix[pp] = total;
+        plan->rec_total = total * row.mp * row.dp;
+        const int n_items = 2 * en.m;                             // items of a device
+        const int cap = max(1, min(kMaxTileItems, kRunWords / (widest * 5)));
+        const int n_chunks = (n_items + cap - 1) / cap;
+        plan->tile_items = (n_items + n_chunks - 1) / n_chunks;
+        plan->run_words = plan->tile_items * widest * 5;
+        plan->tmpl_words = both * 5;                              // the templates of both pipelines of the widest device
         const int64_t reps = (int64_t)row.mp * row.dp;
         sum[kSumRecords] = plan->rec_total;
         sum[kSumItemTiles] = (int64_t)pp * ((n_items + plan->tile_items - 1) / plan->tile_items) *
@@ -304,7 +381,7 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
         const int64_t index = indices[i];
         if (index < 0 || index >= v.sc.n_candidates) {
             if ((threadIdx.x & 31) == 0) {
-                plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0; plan->v = 1;
+                plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0; plan->v = 1; plan->two_way = 0;
                 plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
                 for (int w = 0; w < kSumWords; ++w) sums[(int64_t)i * kSumWords + w] = 0;
                 atomicCAS(v.status, 0, DISTSIM_E_RANGE);
@@ -313,13 +390,11 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
             const int r = find_row(v, index);
             const Row row = v.rows[r];
             if (row.two_way) {
-                // timelines of bidirectional-pipeline candidates are not emitted
-                if ((threadIdx.x & 31) == 0) {
-                    plan->ok = 0; plan->rec_total = 0; plan->index = index; plan->pp = 0; plan->m = 0; plan->v = 1;
-                    plan->mp = 1; plan->dp = 1; plan->tile_items = 8; plan->tmpl_words = 0; plan->run_words = 0;
-                    for (int w = 0; w < kSumWords; ++w) sums[(int64_t)i * kSumWords + w] = 0;
-                    atomicCAS(v.status, 0, DISTSIM_E_UNSUPPORTED);
-                }
+                int64_t *rec_i = op_start + (int64_t)i * op_words_per_cand;
+                const CandidateCoords cc = split_local(row, index - row.offset);
+                plan_bidirectional(v, row, r, index, plan, rec_i, binom, sums + (int64_t)i * kSumWords,
+                                   bidirectional_arrays(plan_dyn + (int64_t)(threadIdx.x >> 5) * ilv_words, row.pp,
+                                                        order_kept(v, cc.entry)));
             } else {
             int64_t *rec_i = op_start + (int64_t)i * op_words_per_cand;
             if (row.v > 1) {
@@ -408,7 +483,8 @@ __device__ __forceinline__ void emit_buckets_block(const DeviceView &v, const Em
     int64_t *g_start = img_b + run * 5 + 1;             // [L + 1] start of the first bucket ending in layer a+i
     int64_t *g_first = g_start + DISTSIM_MAX_LAYERS + 1;  // [L + 1] number of that bucket
     __shared__ int64_t part_start_s, lane_end_s;
-    if (!p.ok || p.dp == 1) return;
+    const bool two_way = p.two_way != 0;                // two streams (pipelines), each reduced over 2 dp devices
+    if (!p.ok || (p.dp == 1 && !two_way)) return;
     const int mp = p.mp, reps = mp * p.dp;
     const int rep_chunks = (reps + kBucketReplicas - 1) / kBucketReplicas;
     const int d = tile / rep_chunks, rc = tile - d * rep_chunks;
@@ -417,7 +493,8 @@ __device__ __forceinline__ void emit_buckets_block(const DeviceView &v, const Em
     const Row &row = v.rows[p.row];
     const int L1 = v.tc.n_layers + 1;
     const int64_t *pb = v.etb + (int64_t)p.entry * v.tc.lp;
-    const int64_t t_full = row.t_full, main_end = p.main_end[d];
+    const bool near = two_way && mirror_group_near(v, row, d);
+    const int64_t t_full = near ? row.t_full_near : row.t_full, main_end = p.main_end[d];
     const int64_t stage_words = p.stage_recs[d] * 5;
     const int64_t replica_words = (int64_t)mp * p.stage_rec_prefix[p.pp] * 5;
     // the device's bucket records follow its main-lane records
@@ -426,11 +503,18 @@ __device__ __forceinline__ void emit_buckets_block(const DeviceView &v, const Em
     int64_t kb0 = 0;                                    // buckets of the chunks already written
     // one gradient stream per model chunk the device holds (one without chunks), the last chunk
     // first, all on the device's one lane
-    for (int c = p.v - 1; c >= 0; --c) {
-        const int s = c * p.pp + d;                     // (virtual) stage
-        const int a = p.bounds[s], e = p.bounds[s + 1];
+    for (int k = p.v - 1; k >= 0; --k) {
+        // bidirectional candidates: the stream of the device's later stage first
+        const int c = two_way ? ((k == 1) == (p.pp - 1 - d > d) ? 1 : 0) : k;
+        const int s = c * p.pp + d;                     // (virtual) stage; index of the per-stage arrays
+        const int st = two_way ? (c ? p.pp - 1 - d : d) : s;
+        const int a = p.bounds[st], e = p.bounds[st + 1];
         const int64_t *nbe = v.nb + row.row_tab_off + (int64_t)e * L1;
-        const int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
+        int64_t part = v.tp[row.row_tab_off + (int64_t)e * L1 + a];
+        // (the table of a two_way row holds the trailing bucket's bytes: its cost depends on the device)
+        if (two_way && part > 0)
+            part = allreduce_cost(v.tc, 2 * (int64_t)p.dp, part, near ? v.tc.alpha_intra : v.tc.alpha_inter,
+                                  near ? v.tc.beta_intra : v.tc.beta_inter);
         const int64_t n_full = nbe[a];
         const int64_t kb = n_full + (part > 0 ? 1 : 0);
         if (kb == 0) continue;
@@ -575,9 +659,10 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     const EmitPlan &p = plans[i];
     if (!p.ok) return;
     const int m = p.m, pp = p.pp, sched = p.sched, mp = p.mp, vch = p.v, P = pp * vch;
+    const bool two_way = p.two_way != 0;                // vch = 2 stands for the two pipelines
     const int reps = mp * p.dp;
     const int tile_items = p.tile_items;
-    const int dev_items = 2 * m * vch;                  // items of a device
+    const int dev_items = two_way ? 2 * m : 2 * m * vch;   // items of a device
     const int item_chunks = (dev_items + tile_items - 1) / tile_items;
     const int rep_chunks = (reps + kTileReplicas - 1) / kTileReplicas;
     int tile = blockIdx.x;
@@ -601,8 +686,10 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     //      templates per model chunk of the device (one without chunks) ----------------------
     int tmpl_acc = 0;
     for (int c = 0; c < vch; ++c) {
-        const int s = c * pp + d;                       // (virtual) stage
-        const int a = p.bounds[s], e = p.bounds[s + 1];
+        const int s = c * pp + d;                       // (virtual) stage; index of the per-stage arrays
+        // the stage's place in its chain of stages: a bidirectional candidate has two chains of pp
+        const int st = two_way ? (c ? pp - 1 - d : d) : s, n_st = two_way ? pp : P;
+        const int a = p.bounds[st], e = p.bounds[st + 1];
         const int rf = p.rf[s], rb = p.rb[s];
         int64_t *tf = tmpl + tmpl_acc, *tb = tf + (int64_t)rf * 5;
         if (threadIdx.x == 0) { toff_s[c][0] = tmpl_acc; toff_s[c][1] = tmpl_acc + rf * 5; }
@@ -631,17 +718,19 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
             }
         }
         if (threadIdx.x == 0) {
-            if (s < P - 1) {
+            if (st < n_st - 1) {
                 int64_t *w = tf + (int64_t)(rf - 1) * 5;
                 const int64_t t = pf[e] - pf[a];
                 w[0] = DISTSIM_SEND_F; w[1] = e - 1; w[2] = 0; w[3] = t;
-                w[4] = t + (vch > 1 ? virtual_p2p_cost(v, row, en, s) : p2p_cost(row, en, d));
+                w[4] = t + (two_way ? p2p_cost(row, en, c ? pp - 2 - st : st)
+                                    : vch > 1 ? virtual_p2p_cost(v, row, en, s) : p2p_cost(row, en, d));
             }
-            if (s > 0) {
+            if (st > 0) {
                 int64_t *w = tb + (int64_t)(rb - 1) * 5;
                 const int64_t t = pb[e] - pb[a];
                 w[0] = DISTSIM_SEND_B; w[1] = a; w[2] = 0; w[3] = t;
-                w[4] = t + (vch > 1 ? virtual_p2p_cost(v, row, en, s - 1) : p2p_cost(row, en, d - 1));
+                w[4] = t + (two_way ? p2p_cost(row, en, c ? pp - 1 - st : st - 1)
+                                    : vch > 1 ? virtual_p2p_cost(v, row, en, s - 1) : p2p_cost(row, en, d - 1));
             }
         }
     }
@@ -650,7 +739,14 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     const int s0 = ic * tile_items;
     const int n_items = min(dev_items, s0 + tile_items) - s0;
     int64_t base0;                                       // words of the device's records before the run
-    {
+    const int64_t order_at = two_way ? order_offset(v, p.entry) : 0;
+    // words of the device's records before position `pos` of its order (bidirectional candidates)
+    auto two_way_words_before = [&](int pos) {
+        const ItemsBefore n = items_before(v, order_at, m, d, pos);
+        return ((int64_t)n.f0 * p.rf[d] + (int64_t)n.b0 * p.rb[d] + (int64_t)n.f1 * p.rf[pp + d] + (int64_t)n.b1 * p.rb[pp + d]) * 5;
+    };
+    if (two_way) base0 = two_way_words_before(s0);
+    else {
         bool bwd0; int c0, j0, nf0, nb0;
         if (vch > 1) {
             interleaved_item_at(pp, vch, m, d, s0, bwd0, c0, j0, nf0, nb0);
@@ -663,7 +759,13 @@ emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_
     for (int k = threadIdx.x; k <= n_items; k += blockDim.x) {
         bool bwd; int c = 0, j, nf, nb;
         int64_t before;
-        if (vch > 1) {
+        if (two_way) {
+            before = two_way_words_before(s0 + k);                             // k == n_items: one past the run
+            const int item = k < n_items ? v.order[order_at + (int64_t)d * (2 * m + 1) + s0 + k] : 0;
+            c = (item & kOrderUp) ? 1 : 0;
+            bwd = (item & kOrderBackward) != 0;
+            j = (item & kOrderMicroBatch) + c * (m / 2);
+        } else if (vch > 1) {
             interleaved_item_at(pp, vch, m, d, s0 + k, bwd, c, j, nf, nb);     // k == n_items: one past the run
             before = interleaved_words_before(p, d, nf, nb);
         } else {

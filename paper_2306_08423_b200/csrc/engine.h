@@ -117,8 +117,11 @@ struct DeviceView {
     const int64_t *jsum;             // [n_entries][DISTSIM_MAX_PP] total jitter of the m forward and
                                      // m backward items of a stage (nullptr without jitter)
     const uint16_t *order;           // bidirectional schedule: every device's items in its order,
-                                     // [entry's offset + device * 2 m + position]: pipeline << 15 |
+                                     // [entry's offset + device * (2 m + 1) + position]: pipeline << 15 |
                                      // is-backward << 14 | micro-batch within its pipeline
+    const uint32_t *order_before;    // same index, position 0 .. 2 m: how many forward items of pipeline 0,
+                                     // backward items of pipeline 0 and forward items of pipeline 1 come before
+                                     // that position in the device's order, 9 bits each
     const int64_t *order_off;        // [n_entries] offset of the entry's orders in `order` (low 48 bits) and,
                                      // above them, the items a device may run from the last backward item
                                      // of its earlier-finishing pipeline on (nullptr: no such rows)
@@ -241,8 +244,11 @@ struct EmitPlan {                    // per selected candidate, written by the p
     int64_t rec_base;                // first record of the selection (after the scan)
     int64_t rec_total;               // records of all its devices
     int32_t row, entry, m, sched, pp, mp, dp, ok;
-    int32_t v, pad;                  // model chunks per device (1 unless interleaved 1F1B); then the arrays
-                                     // indexed "per stage" below are per virtual stage c * pp + d where noted
+    int32_t v, two_way;              // model chunks per device (1 unless interleaved 1F1B); then the arrays
+                                     // indexed "per stage" below are per virtual stage c * pp + d where noted.
+                                     // two_way: a bidirectional-pipeline candidate - v = 2 stands for its two
+                                     // pipelines, rf / rb / last_b_start are indexed pipeline * pp + device, and
+                                     // bounds holds the pp + 1 bounds both pipelines share
     int32_t bounds[DISTSIM_MAX_PP + 1];              // per (virtual) stage
     int32_t tile_items;              // schedule items per block of the record kernel
     int32_t tmpl_words;              // words of the widest stage's forward + backward item templates

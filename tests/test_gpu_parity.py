@@ -289,13 +289,10 @@ def test_bidirectional_pipelines_every_candidate(E, ctx, case):
         assert (out.cpu().numpy() == ob[first:first + count]).all()
     cells, _ = E.distsim_testing_space_cells(ctx)
     assert cells == W.count_candidates_and_cells(w.table, w.space)[1]
+    # every record of the timelines of bidirectional candidates (and some of the others beside them)
     two_way = [i for i, c in enumerate(cands) if c.sched == 4]
-    with pytest.raises(E.DistsimError) as err:
-        E.distsim_emit_timelines(ctx, torch.tensor(two_way[:1], dtype=torch.int64, device="cuda"), 1, None, 0)
-    assert err.value.code == E.E_UNSUPPORTED
-    others = [i for i, c in enumerate(cands) if c.sched != 4]
-    if others:
-        check_emission(E, ctx, w, others[:: max(1, len(others) // 5)][:5])      # the context is as usable as before
+    pick = two_way[:: max(1, len(two_way) // 14)][:14] + [two_way[-1], 0, n - 1]
+    check_emission(E, ctx, w, pick)
 
 
 def test_bidirectional_pipelines_on_the_64_device_shape(E, ctx):
@@ -315,6 +312,10 @@ def test_bidirectional_pipelines_on_the_64_device_shape(E, ctx):
     assert (gb == ob).all(), idx[np.argwhere(gb != ob)[:5, 0]]
     bi, bt = E.distsim_argmin(ctx, batch, 0, n)
     assert oracle.eval_indices(w.table, w.space, np.array([bi]))[0][0] == bt == int(batch.min().item())
+    # timelines: bidirectional candidates with few and many micro-batches, one of the others beside them
+    two_way = [int(i) for i, c in zip(idx, cands) if c.sched == 4]
+    deep = [int(i) for i, c in zip(idx, cands) if c.sched == 4 and c.pp == 16 and c.m == 128]
+    check_emission(E, ctx, w, [two_way[0], two_way[len(two_way) // 2], deep[0], deep[-1], 0])
 
 
 @pytest.mark.parametrize("case", range(12))
