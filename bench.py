@@ -45,8 +45,10 @@ RECORD_BYTES = 40
 # kernel sources it was taken on: a figure whose sources have changed since reads as null.
 TRAFFIC_FILE = os.path.join(ROOT, "profiles", "bench_config1_dram_bytes.md")
 KERNEL_SOURCES = {
-    "eval": ("eval_thread.cuh", "eval_kernels.cu", "recurrence.cuh", "smem_stage.cuh", "interleaved.cuh", "engine.h"),
-    "emit": ("emit_kernels.cu", "recurrence.cuh", "interleaved.cuh", "smem_stage.cuh", "engine.h"),
+    "eval": ("eval_thread.cuh", "eval_kernels.cu", "recurrence.cuh", "smem_stage.cuh", "interleaved.cuh",
+             "bidirectional.cuh", "costs.cuh", "engine.h"),
+    "emit": ("emit_kernels.cu", "recurrence.cuh", "interleaved.cuh", "bidirectional.cuh", "costs.cuh",
+             "smem_stage.cuh", "engine.h"),
 }
 
 
@@ -546,8 +548,12 @@ def other_workloads(E, ctx, torch, dev, peaks, cell32_peak, cell64_peak):
     candidates of the 1024-device workload (device-resident, CUDA events)."""
     out = {}
     stream = torch.cuda.current_stream()
-    for cfg in (0, 2, 3):
-        w = W.CONFIGS[cfg]()
+    # the 64-device workload once more with the two further schedules in its space: interleaved
+    # 1F1B with two chunks per device and bidirectional pipelines (a warp per candidate)
+    more = W.config1()
+    more.space.sched_mask, more.space.v_max = 27, 2
+    more.name = "config1_with_interleaved_and_bidirectional"
+    for w in (W.CONFIGS[0](), W.CONFIGS[2](), W.CONFIGS[3](), more):
         n, cells = W.count_candidates_and_cells(w.table, w.space)
         E.distsim_load_event_table(ctx, w.table)
         E.distsim_set_space(ctx, w.space)
@@ -558,20 +564,27 @@ def other_workloads(E, ctx, torch, dev, peaks, cell32_peak, cell64_peak):
         for _ in range(3):
             E.distsim_eval_strategies(ctx, 0, n, batch)
         best = E.distsim_argmin(ctx, batch, 0, n)
-        times, reps, how = [], 10, "cuda graph of one evaluation, replayed 10x per sample"
+        # replays per sample: ten of a short evaluation, fewer of one that takes milliseconds
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
+        E.distsim_eval_strategies(ctx, 0, n, batch)
+        p1.record(stream)
+        torch.cuda.synchronize()
+        reps = max(1, min(10, int(20.0 / max(p0.elapsed_time(p1), 1e-3))))
+        times, how = [], f"cuda graph of one evaluation, replayed {reps}x per sample"
         try:
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
                 E.distsim_eval_strategies(ctx, 0, n, batch)
             stream = torch.cuda.current_stream()
-            for it in range(8):
+            for it in range(8 if reps > 1 else 5):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
                 for _ in range(reps):
                     graph.replay()
                 e1.record(stream)
                 torch.cuda.synchronize()
-                if it >= 3:
+                if it >= (3 if reps > 1 else 2):
                     times.append(e0.elapsed_time(e1) * 1e-3 / reps)
             del graph
         except RuntimeError:
@@ -646,7 +659,10 @@ def profile_case(name):
     emit4  - emission of 16 of the fastest candidates of the 1024-device workload (~1.9 GB)
     emit1  - emission of the 1024 fastest candidates of the 64-device workload (~1.8 GB)
     emit4x128 - as emit4 for 128 candidates, one call of the benchmark's size (~10 GB; for
-             one-pass launch lists only)"""
+             one-pass launch lists only)
+    select1 - the 1024 fastest of the whole 64-device workload (evaluation, then three selections)
+    evalx  - 400 000 candidates of the 64-device workload's interleaved (two chunks per device) and
+             bidirectional-pipeline rows (a warp per candidate)"""
     import torch
     from paper_2306_08423_b200 import engine as E
     torch.cuda.set_device(0)
@@ -676,6 +692,31 @@ def profile_case(name):
         for _ in range(3):
             E.distsim_eval_strategies(ctx, first, count, batch)
         print(name, "best", E.distsim_argmin(ctx, batch, first, count))
+    elif name == "select1":
+        w = W.config1()
+        E.distsim_load_event_table(ctx, w.table)
+        n = E.distsim_set_space(ctx, w.space)
+        batch = torch.empty(n, dtype=torch.int64, device="cuda")
+        top_i = torch.empty(TOP_K, dtype=torch.int64, device="cuda")
+        top_t = torch.empty(TOP_K, dtype=torch.int64, device="cuda")
+        E.distsim_eval_strategies(ctx, 0, n, batch)
+        for _ in range(3):
+            E.distsim_topk(ctx, batch, 0, n, TOP_K, top_i, top_t)
+        print(name, "k-th time", int(top_t[-1]))
+    elif name == "evalx":
+        w = W.config1()
+        w.space.sched_mask, w.space.v_max = 24, 2
+        E.distsim_load_event_table(ctx, w.table)
+        n = E.distsim_set_space(ctx, w.space)
+        # a slice that ends in the bidirectional row of the first (mp, pp): both kinds of candidates
+        rows = W.space_shape(w.table, w.space)
+        first_two_rows = sum(len(ms) * parts * n_sched for (_mp, _pp, _dp, ms, parts, n_sched, _v) in rows[:2])
+        count = min(n, 400_000)
+        first = max(0, first_two_rows - count // 2)
+        batch = torch.empty(count, dtype=torch.int64, device="cuda")
+        for _ in range(3):
+            E.distsim_eval_strategies(ctx, first, count, batch)
+        print(name, "candidates", count, "of", n, "best", E.distsim_argmin(ctx, batch, first, count))
     elif name in ("emit4", "emit4x128", "emit1"):
         k = {"emit4": 16, "emit4x128": 128, "emit1": TOP_K}[name]
         w = W.config4() if name != "emit1" else W.config1()
