@@ -58,6 +58,10 @@ __device__ __forceinline__ ItemsBefore items_before(const DeviceView &v, int64_t
     return n;
 }
 
+// No (pp, m) keeps more items than this per device (the host checks it when it builds the orders):
+// the shared memory of a candidate is sized with it.
+__host__ __device__ inline int bidirectional_kept_cap(int pp) { return pp / 2 + 2; }
+
 // Where an entry's orders start in DeviceView::order, and its kept items per device.
 __device__ __forceinline__ int64_t order_offset(const DeviceView &v, int entry) { return __ldg(&v.order_off[entry]) & (((int64_t)1 << 48) - 1); }
 __device__ __forceinline__ int order_kept(const DeviceView &v, int entry) { return (int)(__ldg(&v.order_off[entry]) >> 48); }
@@ -117,14 +121,16 @@ __device__ __forceinline__ int64_t mirror_bucket_chain(const DeviceView &v, cons
     return end;
 }
 
-// Evaluates one candidate of a two_way row by the calling warp (all 32 lanes; lane d < pp owns
-// device d; pp <= 32).  A: the warp's arrays; afterwards A.bounds, A.cost and A.last_b describe the
-// candidate.  rec (nullable): item start times go to rec[d * 2 m + position in the device's order].
+// Evaluates one candidate of a two_way row by `seg` consecutive lanes of the calling warp (seg a
+// power of two >= pp, pp <= 32; lane d < pp of the segment owns device d), every lane of the warp
+// calling this together.  A: the candidate's arrays; afterwards A.bounds, A.cost and A.last_b
+// describe the candidate.  rec (nullable): item start times go to rec[d * 2 m + position in the
+// device's order].
 __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v, const Row &row, const Entry &en,
                                                              const CandidateCoords &cc, const int64_t *binom,
-                                                             const IlvArrays &A, int64_t *rec)
+                                                             const IlvArrays &A, int64_t *rec, int seg)
 {
-    const int lane = threadIdx.x & 31;
+    const int lane = (threadIdx.x & 31) & (seg - 1);         // lane within the candidate's segment
     const int pp = row.pp, P = 2 * pp, m = en.m, half = m >> 1, L = v.tc.n_layers;
     int64_t *ring_f = A.ring_f, *ring_b = A.ring_b, *cost = A.cost, *last_b = A.last_b, *tail = A.tail;
     int *cnt_f = A.cnt_f, *cnt_b = A.cnt_b, *bounds = A.bounds;
@@ -132,7 +138,7 @@ __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v
 
     // ---- the partition into pp stages -------------------------------------------------------
     if (v.sc.partition_mode == 0) {
-        for (int s = lane; s <= pp; s += 32) bounds[s] = (int)((int64_t)s * L / pp);
+        for (int s = lane; s <= pp; s += seg) bounds[s] = (int)((int64_t)s * L / pp);
     } else if (lane == 0) {
         // the (pp-1)-subsets of {1..L-1} in lexicographic order (combinatorial number system)
         int64_t r = cc.part_rank;
@@ -152,7 +158,7 @@ __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v
     __syncwarp();
     const int64_t *pf = v.etf + (int64_t)cc.entry * v.tc.lp;
     const int64_t *pb = v.etb + (int64_t)cc.entry * v.tc.lp;
-    for (int x = lane; x < P; x += 32) {
+    for (int x = lane; x < P; x += seg) {
         const int u = x >= pp, s = x - u * pp;
         const int a = bounds[s], e = bounds[s + 1];
         // pipeline "down" sends across the boundary s | s + 1 (forward) and s - 1 | s (backward);
@@ -170,9 +176,10 @@ __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v
     const uint16_t *mine = v.order + order_offset(v, cc.entry) + (int64_t)d * (2 * m + 1);
     int n_done = 0;
     int64_t free_at = 0;
-    const int limit = 2 * (m + pp) + 8;             // the merged order takes 2 m + pp - 2 rounds when m >= pp, never more than 2 (m + pp)
-    int round = 0;
-    for (; round < limit; ++round) {
+    // the merged order takes 2 m + pp - 2 rounds when m >= pp, never more than 2 (m + pp); the
+    // segments of a warp may differ in m: all of them make the rounds of the longest
+    const int limit = __reduce_max_sync(0xffffffffu, 2 * (m + pp) + 8);
+    for (int round = 0; round < limit; ++round) {
         const bool pending = d < pp && n_done < 2 * m;
         if (!__any_sync(0xffffffffu, pending)) break;
         bool run = false, is_b = false;
@@ -215,7 +222,7 @@ __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v
         }
         __syncwarp();
     }
-    if (round == limit && lane == 0) atomicCAS(v.status, 0, kStatusScheduleStuck);
+    if (d < pp && n_done < 2 * m) atomicCAS(v.status, 0, kStatusScheduleStuck);
 
     // ---- gradient buckets: the stream of the later stage first, both on the device's one lane --
     IlvResult R{0, 0, 0, 0};
@@ -255,8 +262,7 @@ __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v
         R.main_end = main_end; R.dp_end = dp_end;
     }
     int64_t mx = max64(R.main_end, R.dp_end);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int o = seg >> 1; o > 0; o >>= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     R.batch = mx;
     return R;
 }

@@ -572,7 +572,9 @@ int distsim_set_space(distsim_ctx *ctx, const distsim_space *sp, int64_t *n_cand
                     all_before.insert(all_before.end(), one_before.begin(), one_before.end());
                 }
                 order_off[r.entry0 + e] = it->second.first | ((int64_t)it->second.second << 48);
-                const int words = bidirectional_words_of(r.pp, it->second.second);
+                if (it->second.second > bidirectional_kept_cap_of(r.pp))
+                    return fail(ctx, DISTSIM_E_STATE, "the bidirectional item order keeps more items than the kernels allow for");
+                const int words = bidirectional_words_of(r.pp, bidirectional_kept_cap_of(r.pp));
                 if (words > ctx->two_way_words) ctx->two_way_words = words;
             }
         }
@@ -683,7 +685,7 @@ int distsim_eval_strategies(distsim_ctx *ctx, void *stream, int64_t first, int64
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const DeviceView v = ctx->view();
     launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
-                d_batch_ns, d_stage_busy_ns, &ctx->launches, ctx->two_way_words);
+                d_batch_ns, d_stage_busy_ns, &ctx->launches);
     CU(cudaGetLastError(), "evaluation launch");
     return DISTSIM_OK;
 }
@@ -705,7 +707,7 @@ int distsim_eval_select(distsim_ctx *ctx, void *stream, int64_t first, int64_t c
     const SelectScratch sc = ctx->select_scratch();
     if (ctx->phase_timing) cudaEventRecord(ctx->phase_ev[0], s);
     launch_eval(s, ctx->side, v, ctx->rows.data(), (int)ctx->rows.size(), ctx->entries.data(), first, count,
-                d_batch_ns, nullptr, &ctx->launches, ctx->two_way_words);
+                d_batch_ns, nullptr, &ctx->launches);
     CU(cudaGetLastError(), "evaluation launch");
     if (ctx->phase_timing) cudaEventRecord(ctx->phase_ev[1], s);
     const bool want_best = d_best || h_best_index;

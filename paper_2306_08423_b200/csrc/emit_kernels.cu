@@ -172,7 +172,7 @@ __device__ __forceinline__ void plan_interleaved(const DeviceView &v, const Row 
     const int pp = row.pp, vch = row.v, P = pp * vch;
     const CandidateCoords cc = split_local(row, index - row.offset);
     const Entry en = v.entries[cc.entry];
-    const IlvResult R = interleaved_candidate(v, row, en, cc, binom, A, rec);
+    const IlvResult R = interleaved_candidate(v, row, en, cc, binom, A, rec, 32);
     const int L1 = v.tc.n_layers + 1;
     int widest = 1, both = 0;
     int64_t dev_recs = 0, dev_buckets = 0;
@@ -250,7 +250,7 @@ __device__ __forceinline__ void plan_bidirectional(const DeviceView &v, const Ro
     const int pp = row.pp;
     const CandidateCoords cc = split_local(row, index - row.offset);
     const Entry en = v.entries[cc.entry];
-    const IlvResult R = bidirectional_candidate(v, row, en, cc, binom, A, rec);
+    const IlvResult R = bidirectional_candidate(v, row, en, cc, binom, A, rec, 32);
     const int L1 = v.tc.n_layers + 1, half = en.m / 2;
     int widest = 1, both = 0;
     int64_t dev_recs = 0, dev_buckets = 0;
@@ -890,6 +890,7 @@ void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const 
 
 int interleaved_words_of(int pp, int v) { return interleaved_words(pp, v); }
 int bidirectional_words_of(int pp, int kept) { return bidirectional_words(pp, kept); }
+int bidirectional_kept_cap_of(int pp) { return bidirectional_kept_cap(pp); }
 
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,

@@ -200,8 +200,7 @@ struct SideStream {
 // is ordered after what `s` held before the call and before what is enqueued on `s` after it.
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
-                 int64_t *launches,
-                 int two_way_words = 0 /* shared-memory words a warp needs for the space's bidirectional rows */);
+                 int64_t *launches);
 // Cuts candidates [lo, hi) of a row of pp stages into pieces of at most max_blocks lock-step
 // blocks each; returns the number of pieces and writes the first max_pieces of them.
 int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int64_t max_pieces,
@@ -284,7 +283,8 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
                       cudaEvent_t planned /* nullable: recorded behind the planning kernel */,
                       int64_t *launches);
 int interleaved_words_of(int pp, int v);           // those words for one row
-int bidirectional_words_of(int pp, int kept);      // shared-memory words a warp needs for a bidirectional candidate
+int bidirectional_words_of(int pp, int kept);      // shared-memory words a bidirectional candidate needs
+int bidirectional_kept_cap_of(int pp);             // most items the kernels keep per device of such a candidate
 // out[k] = order-sensitive checksum of the records [offsets[k], offsets[k + 1]).
 void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const int64_t *offsets, int64_t n_lists,
                            uint64_t *out, int64_t *launches);

@@ -105,11 +105,17 @@ eval_lockstep_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__re
     else lockstep_block<1, kJit>(v, wk, row, local_block, first, batch_out, busy_out, smem_words, smem_raw, &bar, binom);
 }
 
-// Interleaved 1F1B and bidirectional-pipeline candidates: a candidate per warp (interleaved.cuh,
-// bidirectional.cuh).
+// Interleaved 1F1B and bidirectional-pipeline candidates (interleaved.cuh, bidirectional.cuh):
+// pp lanes per candidate, 32 / pp candidates per warp, each with arrays of its own in shared memory.
+__host__ __device__ inline int warp_candidate_words(const Row &row)
+{
+    return row.two_way ? bidirectional_words(row.pp, bidirectional_kept_cap(row.pp)) : interleaved_words(row.pp, row.v);
+}
+__host__ __device__ inline int warp_candidate_lanes(const Row &row) { return row.pp < 32 ? row.pp : 32; }
+
 __global__ void __launch_bounds__(kIlvThreads)
 eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *__restrict__ batch_out,
-                        int64_t *__restrict__ busy_out, int words_per_warp)
+                        int64_t *__restrict__ busy_out)
 {
     extern __shared__ __align__(16) int64_t ilv_s[];
     __shared__ int64_t binom_s[512];
@@ -118,23 +124,26 @@ eval_interleaved_kernel(DeviceView v, EvalBatch batch, int64_t first, int64_t *_
     while (wi + 1 < batch.n && (int)blockIdx.x >= batch.w[wi + 1].block_begin) ++wi;
     const EvalWork &wk = batch.w[wi];
     const Row row = v.rows[wk.row];
+    const int seg = warp_candidate_lanes(row), per_warp = 32 / seg;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int64_t local = wk.lo + (int64_t)((int)blockIdx.x - wk.block_begin) * (kIlvThreads / 32) + warp;
+    const int slot = warp * per_warp + lane / seg;          // the candidate's number inside the block
+    int64_t local = wk.lo + (int64_t)((int)blockIdx.x - wk.block_begin) * (kIlvThreads / 32) * per_warp + slot;
     const bool valid = local < wk.hi;
-    if (!valid) local = wk.hi - 1;                 // an idle warp shadows a real candidate
+    if (!valid) local = wk.hi - 1;                 // an idle segment shadows a real candidate
     const CandidateCoords cc = split_local(row, local);
     const Entry en = v.entries[cc.entry];
-    int64_t *mine = ilv_s + (int64_t)warp * words_per_warp;
+    int64_t *mine = ilv_s + (int64_t)slot * warp_candidate_words(row);
     const IlvResult R = row.two_way
-        ? bidirectional_candidate(v, row, en, cc, binom, bidirectional_arrays(mine, row.pp, order_kept(v, cc.entry)), nullptr)
-        : interleaved_candidate(v, row, en, cc, binom, interleaved_arrays(mine, row.pp, row.v), nullptr);
+        ? bidirectional_candidate(v, row, en, cc, binom, bidirectional_arrays(mine, row.pp, order_kept(v, cc.entry)), nullptr, seg)
+        : interleaved_candidate(v, row, en, cc, binom, interleaved_arrays(mine, row.pp, row.v), nullptr, seg);
     if (!valid) return;
+    const int d = lane & (seg - 1);
     const int64_t out = row.offset + local - first;
-    if (lane == 0) batch_out[out] = R.batch;
+    if (d == 0) batch_out[out] = R.batch;
     if (busy_out) {
         int64_t *bo = busy_out + out * v.sc.pp_max;
-        if (lane < row.pp) bo[lane] = R.busy;
-        for (int z = row.pp + lane; z < v.sc.pp_max; z += 32) bo[z] = 0;
+        if (d < row.pp) bo[d] = R.busy;
+        for (int z = row.pp + d; z < v.sc.pp_max; z += seg) bo[z] = 0;
     }
 }
 
@@ -262,7 +271,7 @@ int64_t lockstep_pieces(int pp, int64_t lo, int64_t hi, int64_t max_blocks, int6
 
 void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, const Row *rows, int n_rows,
                  const Entry *entries, int64_t first, int64_t count, int64_t *batch_out, int64_t *busy_out,
-                 int64_t *launches, int two_way_words)
+                 int64_t *launches)
 {
     const int64_t last = first + count;
     struct ThreadItem { EvalWork w; int lg; bool narrow; int blocks, words; };
@@ -291,14 +300,14 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
         const int64_t hi = last < row.offset + row.size ? last - row.offset : row.size;
         if (hi <= lo) continue;
         if (row.v > 1 || row.two_way) {
-            constexpr int64_t cpb = kIlvThreads / 32;
+            const int64_t cpb = (kIlvThreads / 32) * (32 / warp_candidate_lanes(row));      // candidates per block
             for (int64_t a = lo; a < hi; a += kPieceBlocks * cpb) {
                 EvalWork w{};
                 w.row = r; w.lo = a; w.hi = hi - a < kPieceBlocks * cpb ? hi : a + kPieceBlocks * cpb;
                 w.nx = (int)((w.hi - w.lo + cpb - 1) / cpb);
                 ilv_items.push_back(w);
             }
-            const int words = row.two_way ? two_way_words : interleaved_words(row.pp, row.v);
+            const int words = (int)cpb * warp_candidate_words(row);                        // of a block
             if (words > ilv_words) ilv_words = words;
             continue;
         }
@@ -372,9 +381,9 @@ void launch_eval(cudaStream_t s, const SideStream &ss, const DeviceView &v, cons
     // interleaved candidates: a kernel of their own, on the caller's stream
     auto flush_interleaved = [&]() {
         if (p.batch.n == 0) return;
-        const size_t smem = (size_t)(kIlvThreads / 32) * ilv_words * sizeof(int64_t);
+        const size_t smem = (size_t)ilv_words * sizeof(int64_t);
         ensure_dynamic_smem(reinterpret_cast<const void *>(&eval_interleaved_kernel), smem);
-        eval_interleaved_kernel<<<p.blocks, kIlvThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out, ilv_words);
+        eval_interleaved_kernel<<<p.blocks, kIlvThreads, smem, s>>>(v, p.batch, first, batch_out, busy_out);
         ++*launches;
         p = Pending{};
     };

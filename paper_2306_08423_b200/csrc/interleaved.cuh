@@ -23,7 +23,7 @@
 
 namespace distsim {
 
-constexpr int kIlvThreads = 64;                 // two warps, a candidate each
+constexpr int kIlvThreads = 64;                 // two warps of 32 / pp candidates each
 constexpr int32_t kStatusScheduleStuck = -71;   // device status: the rounds ran out (never seen)
 
 // The last items of a device that are kept with their start and end: from the last backward item
@@ -76,14 +76,16 @@ __device__ __forceinline__ IlvArrays interleaved_arrays(int64_t *base, int pp, i
 // What a lane knows of its device after the evaluation.
 struct IlvResult { int64_t main_end, dp_end, busy, batch; };
 
-// Evaluates one interleaved candidate by the calling warp (all 32 lanes; lane d < pp owns device
-// d).  A: the warp's arrays; afterwards A.bounds, A.cost and A.last_b describe the candidate.
+// Evaluates one interleaved candidate by `seg` consecutive lanes of the calling warp (seg a power
+// of two >= pp; lane d < pp of the segment owns device d), every lane of the warp calling this
+// together: the other segments work on candidates of their own.  A: the candidate's arrays;
+// afterwards A.bounds, A.cost and A.last_b describe the candidate.
 // rec (nullable): item start times go to rec[d * 2 m v + position in the device's order].
 __device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, const Row &row, const Entry &en,
                                                            const CandidateCoords &cc, const int64_t *binom,
-                                                           const IlvArrays &A, int64_t *rec)
+                                                           const IlvArrays &A, int64_t *rec, int seg)
 {
-    const int lane = threadIdx.x & 31;
+    const int lane = (threadIdx.x & 31) & (seg - 1);         // lane within the candidate's segment
     const int pp = row.pp, vch = row.v, P = pp * vch, m = en.m, L = v.tc.n_layers;
     const int log_pp = 31 - __clz(pp), log_v = 31 - __clz(vch);
     int64_t *ring_f = A.ring_f, *ring_b = A.ring_b, *cost = A.cost, *last_b = A.last_b, *tail = A.tail;
@@ -92,7 +94,7 @@ __device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, 
 
     // ---- the partition into P virtual stages --------------------------------------------------
     if (v.sc.partition_mode == 0) {
-        for (int s = lane; s <= P; s += 32) bounds[s] = (int)((int64_t)s * L / P);
+        for (int s = lane; s <= P; s += seg) bounds[s] = (int)((int64_t)s * L / P);
     } else if (lane == 0) {
         // the (P-1)-subsets of {1..L-1} in lexicographic order (combinatorial number system)
         int64_t r = cc.part_rank;
@@ -112,7 +114,7 @@ __device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, 
     __syncwarp();
     const int64_t *pf = v.etf + (int64_t)cc.entry * v.tc.lp;
     const int64_t *pb = v.etb + (int64_t)cc.entry * v.tc.lp;
-    for (int s = lane; s < P; s += 32) {
+    for (int s = lane; s < P; s += seg) {
         const int a = bounds[s], e = bounds[s + 1];
         cost[2 * s] = __ldg(&pf[e]) - __ldg(&pf[a]) + (s < P - 1 ? virtual_p2p_cost(v, row, en, s) : 0);
         cost[2 * s + 1] = __ldg(&pb[e]) - __ldg(&pb[a]) + (s > 0 ? virtual_p2p_cost(v, row, en, s - 1) : 0);
@@ -127,9 +129,9 @@ __device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, 
     if (m == pp || warm > total) warm = total;
     int n_f = 0, n_b = 0;
     int64_t free_at = 0;
-    const int limit = 2 * (total + pp) + 8;
-    int round = 0;
-    for (; round < limit; ++round) {
+    // (the segments of a warp may differ in m: all of them make the rounds of the longest)
+    const int limit = __reduce_max_sync(0xffffffffu, 2 * (total + pp) + 8);
+    for (int round = 0; round < limit; ++round) {
         const bool pending = d < pp && n_f + n_b < 2 * total;
         if (!__any_sync(0xffffffffu, pending)) break;
         // the device's next item and, if it is there, its input
@@ -175,7 +177,7 @@ __device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, 
         }
         __syncwarp();
     }
-    if (round == limit && lane == 0) atomicCAS(v.status, 0, kStatusScheduleStuck);
+    if (d < pp && n_f + n_b < 2 * total) atomicCAS(v.status, 0, kStatusScheduleStuck);
 
     // ---- gradient buckets: one stream per chunk, the chunk whose backward finishes first (the
     //      last one) first, chained on the device's one lane; then the reduction --------------
@@ -210,8 +212,7 @@ __device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, 
         R.main_end = main_end; R.dp_end = dp_end;
     }
     int64_t mx = max64(R.main_end, R.dp_end);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int o = seg >> 1; o > 0; o >>= 1) mx = max64(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     R.batch = mx;
     return R;
 }
