@@ -175,6 +175,7 @@ __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v
     const int d = lane;
     const uint16_t *mine = v.order + order_offset(v, cc.entry) + (int64_t)d * (2 * m + 1);
     int n_done = 0;
+    int kept_at = 0;                                // n_done mod kt: where the next kept interval goes
     int64_t free_at = 0;
     // the merged order takes 2 m + pp - 2 rounds when m >= pp, never more than 2 (m + pp); the
     // segments of a warp may differ in m: all of them make the rounds of the longest
@@ -207,8 +208,9 @@ __device__ __forceinline__ IlvResult bidirectional_candidate(const DeviceView &v
         if (run) {
             const int64_t start = max64(dep, free_at);
             free_at = start + cost[2 * x + (is_b ? 1 : 0)];
-            int64_t *slot = tail + 2 * (d * kt + n_done % kt);
+            int64_t *slot = tail + 2 * (d * kt + kept_at);
             slot[0] = start; slot[1] = free_at;
+            kept_at = kept_at + 1 == kt ? 0 : kept_at + 1;
             if (rec) rec[(int64_t)d * 2 * m + n_done] = start;
             if (is_b) {
                 ring_b[x * pp + (j & (pp - 1))] = free_at;

@@ -128,6 +128,7 @@ __device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, 
     int warm = (pp - d - 1) * 2 + (vch - 1) * pp;
     if (m == pp || warm > total) warm = total;
     int n_f = 0, n_b = 0;
+    int kept_at = 0;                                // (items run) mod kt: where the next kept interval goes
     int64_t free_at = 0;
     // (the segments of a warp may differ in m: all of them make the rounds of the longest)
     const int limit = __reduce_max_sync(0xffffffffu, 2 * (total + pp) + 8);
@@ -161,8 +162,9 @@ __device__ __forceinline__ IlvResult interleaved_candidate(const DeviceView &v, 
         if (run) {
             const int64_t start = max64(dep, free_at);
             free_at = start + cost[2 * s + (is_b ? 1 : 0)];
-            int64_t *slot = tail + 2 * (d * kt + (n_f + n_b) % kt);
+            int64_t *slot = tail + 2 * (d * kt + kept_at);
             slot[0] = start; slot[1] = free_at;
+            kept_at = kept_at + 1 == kt ? 0 : kept_at + 1;
             if (rec) rec[(int64_t)d * 2 * total + n_f + n_b] = start;
             if (is_b) {
                 ring_b[s * pp + (j & (pp - 1))] = free_at;
