@@ -286,6 +286,34 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
                            int64_t *h_total_records);
 
 /*
+ * The same without any wait on the host, for a loop that emits timelines step after step (the
+ * paper's search loop, Sec. 6, keeps the host out of the way of the device).  What the
+ * synchronising call learns from its planning pass - how much output and how much of the
+ * kernels' resources the selection needs - the caller passes in instead: distsim_emit_shape()
+ * returns those figures for the context's most recent planning pass (a sizing call, say, on a
+ * selection of the kind the loop will see), and the caller may enlarge any of them for headroom.
+ *   shape      host: upper bounds this call provisions for (see distsim_emit_shape)
+ * The call plans the n selections, then writes their records, all in stream order.  If the
+ * selection needs more than `shape` or capacity_records allow, no record is written, the device
+ * status becomes DISTSIM_E_CAPACITY and the next synchronising call on the context returns it;
+ * d_offsets, d_busy_ns and d_util are written either way, and d_offsets[n*N] is the number of
+ * records needed.  Errors found on the host (arguments, state) are returned at once.
+ */
+typedef struct {
+    int64_t records;        /* records of all selections                                    */
+    int64_t item_tiles;     /* most blocks of the item kernel any selection needs            */
+    int64_t bucket_tiles;   /* most blocks of the gradient-bucket kernel any selection needs */
+    int64_t tmpl_words;     /* most 64-bit words of a device's item templates                */
+    int64_t bucket_recs;    /* most gradient-bucket records of a device                      */
+    int64_t run_words;      /* most 64-bit words of one block's run of items                 */
+} distsim_emit_shape;
+int distsim_emit_shape_of_last_plan(distsim_ctx *ctx, distsim_emit_shape *h_shape);
+int distsim_emit_timelines_async(distsim_ctx *ctx, void *stream, const int64_t *d_indices, int32_t n,
+                                 distsim_record *d_records, int64_t capacity_records,
+                                 const distsim_emit_shape *h_shape,
+                                 int64_t *d_offsets, int64_t *d_busy_ns, double *d_util);
+
+/*
  * Order-sensitive 64-bit checksum of every device's record stream (the paper has no counterpart:
  * a way to check emitted timelines, e.g. after they have been moved, without comparing gigabytes).
  * List k holds the records [d_offsets[k], d_offsets[k+1]) of d_records, as written by

@@ -84,6 +84,8 @@ struct distsim_ctx {
     int two_way_words = 0;                // shared-memory words a warp needs for the bidirectional rows
     SideStream side;                      // extra streams of an evaluation (lock-step launches)
     cudaEvent_t planned = nullptr;        // recorded behind the emission-planning kernel
+    EmitTotals last_plan{};               // totals of the most recent synchronising planning pass
+    bool have_last_plan = false;
     int64_t *h_pinned = nullptr;          // 16 words of pinned host memory for small results:
                                           // [0..3] results, [4] status, [8..15] emission totals
 
@@ -180,6 +182,8 @@ int take_status(distsim_ctx *ctx, cudaStream_t s, int32_t code, bool *stalled)
         if (code == kStatusCopyPending)
             return fail(ctx, DISTSIM_E_TIMEOUT, "a bulk copy into shared memory never completed: results computed on this device since may be wrong");
         if (code == DISTSIM_E_RANGE) return fail(ctx, code, "candidate index out of range");
+        if (code == DISTSIM_E_CAPACITY)
+            return fail(ctx, code, "an asynchronous emission needed more than its shape or capacity allowed: it wrote no records");
         return fail(ctx, code, "device reported an error");
     }
     return DISTSIM_OK;
@@ -804,6 +808,7 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     bool stalled = false;
     if (int rc = take_status(ctx, s, (int32_t)ctx->h_pinned[8 + 7], &stalled)) return rc;
     *h_total_records = totals->records;
+    ctx->last_plan = *totals; ctx->have_last_plan = true;
     if (d_records) {
         if (totals->records > capacity_records) return fail(ctx, DISTSIM_E_CAPACITY, "record buffer too small");
         launch_emit_records(s, ctx->side, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
@@ -812,6 +817,57 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
     }
     // the records are written in stream order
     return stalled ? fail(ctx, DISTSIM_E_TIMEOUT, kTimeoutText) : DISTSIM_OK;
+}
+
+int distsim_emit_shape_of_last_plan(distsim_ctx *ctx, distsim_emit_shape *h_shape)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!h_shape) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (!ctx->have_last_plan) return fail(ctx, DISTSIM_E_STATE, "no timelines have been planned yet");
+    const EmitTotals &t = ctx->last_plan;
+    h_shape->records = t.records; h_shape->item_tiles = t.item_tiles; h_shape->bucket_tiles = t.bucket_tiles;
+    h_shape->tmpl_words = t.tmpl_words; h_shape->bucket_recs = t.bucket_recs; h_shape->run_words = t.run_words;
+    return DISTSIM_OK;
+}
+
+int distsim_emit_timelines_async(distsim_ctx *ctx, void *stream, const int64_t *d_indices, int32_t n,
+                                 distsim_record *d_records, int64_t capacity_records,
+                                 const distsim_emit_shape *h_shape,
+                                 int64_t *d_offsets, int64_t *d_busy_ns, double *d_util)
+{
+    if (!ctx) return DISTSIM_E_ARG;
+    if (!ctx->space_set) return fail(ctx, DISTSIM_E_STATE, "no search space set");
+    if (!d_indices || !d_records || !h_shape) return fail(ctx, DISTSIM_E_ARG, "null argument");
+    if (n < 1 || n > 65535) return fail(ctx, DISTSIM_E_ARG, "n must be in [1, 65535]");
+    if (capacity_records < 0) return fail(ctx, DISTSIM_E_ARG, "negative capacity");
+    // what one launch can be given: the grids' first dimension, the item kernel's shared memory
+    // (two images of a run and the templates) and the bucket kernel's
+    const int64_t item_smem = (2 * ((h_shape->run_words + 1) & ~(int64_t)1) + 2 + h_shape->tmpl_words) * 8;
+    if (h_shape->records < 0 || h_shape->item_tiles < 0 || h_shape->item_tiles > 0x7fffffff ||
+        h_shape->bucket_tiles < 0 || h_shape->bucket_tiles > 0x7fffffff || h_shape->tmpl_words < 0 ||
+        h_shape->bucket_recs < 0 || h_shape->run_words < 0 || item_smem > 227 * 1024)
+        return fail(ctx, DISTSIM_E_ARG, "the shape asks for more than a launch can be given");
+    if (int rc = set_device(ctx)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CU(ctx->d_plans.reserve((size_t)n * sizeof(EmitPlan)), "alloc emission plans");
+    CU(ctx->d_op_start.reserve((size_t)n * ctx->op_words_per_cand * sizeof(int64_t)), "alloc item start times");
+    CU(ctx->d_plan_sums.reserve((size_t)n * kEmitSumWords * sizeof(int64_t)), "alloc plan summaries");
+    const DeviceView v = ctx->view();
+    EmitTotals lim{};
+    lim.records = capacity_records;           // (shape.records is the sizing pass's count, for the caller's buffer)
+    lim.item_tiles = h_shape->item_tiles; lim.bucket_tiles = h_shape->bucket_tiles; lim.tmpl_words = h_shape->tmpl_words;
+    lim.bucket_recs = h_shape->bucket_recs; lim.run_words = h_shape->run_words;
+    launch_emit_plan(s, v, d_indices, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
+                     ctx->op_words_per_cand, ctx->d_plan_sums.as<int64_t>(), nullptr, nullptr, nullptr, ctx->d_totals.as<int64_t>(),
+                     std::max(ctx->ilv_words, ctx->two_way_words), nullptr, nullptr, &ctx->launches, &lim);
+    CU(cudaGetLastError(), "emission planning launch");
+    // the record kernels are sized by the shape; they write only if the plans stay within it
+    // (the per-device words are written beside them: nothing waits for those)
+    const EmitDeviceWords words{d_offsets, d_busy_ns, d_util, ctx->d_totals.as<int64_t>()};
+    launch_emit_records(s, ctx->side, v, n, ctx->d_plans.as<EmitPlan>(), ctx->d_op_start.as<int64_t>(),
+                        ctx->op_words_per_cand, lim, d_records, &ctx->launches, ctx->d_totals.as<int64_t>(), &words);
+    CU(cudaGetLastError(), "emission launch");
+    return DISTSIM_OK;
 }
 
 int distsim_checksum_timelines(distsim_ctx *ctx, void *stream, const distsim_record *d_records,

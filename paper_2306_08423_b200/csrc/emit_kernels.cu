@@ -369,7 +369,9 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
                  int64_t *op_start, int64_t op_words_per_cand, int64_t *sums, int64_t *totals,
                  int ilv_words /* shared-memory words per warp for interleaved candidates */,
                  int64_t *h_totals /* nullable; host memory the device can write: the totals' words, then
-                                      (word 7) the device status word as this kernel leaves it */)
+                                      (word 7) the device status word as this kernel leaves it */,
+                 EmitTotals limits /* limits.pad[0] != 0: what the caller has provisioned; word 7 of the
+                                      totals then says whether the plans stay within it */)
 {
     extern __shared__ __align__(16) int64_t plan_dyn[];
     __shared__ int64_t binom_s[kPlanBinomWords];
@@ -416,6 +418,16 @@ emit_plan_kernel(DeviceView v, const int64_t *__restrict__ indices, int n, EmitP
     __threadfence();
     if (threadIdx.x == 0) totals[6] = 0;               // the next launch counts its blocks from zero
     scan_plans(plans, sums, n, totals);
+    if (limits.pad[0]) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int64_t *lim = reinterpret_cast<const int64_t *>(&limits);
+            bool fits = true;
+            for (int w = 0; w <= kSumRunWords; ++w) fits = fits && __ldcg(&totals[w]) <= lim[w];
+            totals[7] = fits ? 1 : 0;
+            if (!fits) atomicCAS(v.status, 0, DISTSIM_E_CAPACITY);
+        }
+    }
     if (!h_totals) return;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -600,8 +612,10 @@ __device__ __forceinline__ void emit_buckets_block(const DeviceView &v, const Em
 // the item launch they take the places of item blocks and cost more than they save).
 constexpr int kBucketThreads = 128;
 __global__ void __launch_bounds__(kBucketThreads)
-emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *__restrict__ out, int run /* buckets per image */)
+emit_buckets_kernel(DeviceView v, const EmitPlan *__restrict__ plans, int64_t *__restrict__ out, int run /* buckets per image */,
+                    const int64_t *__restrict__ gate /* nullable: totals whose word 7 says whether to write at all */)
 {
+    if (gate && __ldcg(&gate[7]) == 0) return;
     extern __shared__ __align__(16) int64_t dyn_b[];
     emit_buckets_block(v, plans[blockIdx.y], (int)blockIdx.x, out, run, dyn_b);
 }
@@ -642,8 +656,10 @@ __device__ __forceinline__ int64_t interleaved_words_before(const EmitPlan &p, i
 __global__ void __launch_bounds__(kItemThreads)
 emit_items_kernel(DeviceView v, const EmitPlan *__restrict__ plans, const int64_t *__restrict__ op_start,
                   int64_t op_words_per_cand, int64_t *__restrict__ out /* records as flat words */,
-                  int cap /* words of one image: even, at least the longest run of any selection */)
+                  int cap /* words of one image: even, at least the longest run of any selection */,
+                  const int64_t *__restrict__ gate /* nullable: totals whose word 7 says whether to write at all */)
 {
+    if (gate && __ldcg(&gate[7]) == 0) return;
     extern __shared__ __align__(16) int64_t dyn_s[];
     int64_t *img_a = dyn_s;                             // word x of the run at img_a[x]
     int64_t *img_b = dyn_s + cap;                       // the same word at img_b[x + 1]
@@ -895,26 +911,36 @@ int bidirectional_kept_cap_of(int pp) { return bidirectional_kept_cap(pp); }
 void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indices, int n,
                       EmitPlan *plans, int64_t *op_start, int64_t op_words_per_cand, int64_t *sums,
                       int64_t *offsets, int64_t *busy, double *util, int64_t *d_totals, int ilv_words,
-                      int64_t *h_totals, cudaEvent_t planned, int64_t *launches)
+                      int64_t *h_totals, cudaEvent_t planned, int64_t *launches, const EmitTotals *limits)
 {
+    EmitTotals lim{};
+    if (limits) { lim = *limits; lim.pad[0] = 1; }
     const size_t plan_smem = (size_t)4 * ilv_words * sizeof(int64_t);
     ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_plan_kernel), plan_smem);
     emit_plan_kernel<<<(n + 3) / 4, 128, plan_smem, s>>>(v, d_indices, n, plans, op_start, op_words_per_cand, sums, d_totals,
-                                                     ilv_words, h_totals);
+                                                     ilv_words, h_totals, lim);
     ++*launches;
     if (planned) cudaEventRecord(planned, s);       // the host can go on while the per-device words are written
-    if (offsets || busy || util) {
-        const int64_t total = (int64_t)n * v.tc.n_devices + 1;
-        emit_devices_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(v, plans, n, offsets, busy, util, d_totals);
-        ++*launches;
-    }
+    launch_emit_devices(s, v, plans, n, offsets, busy, util, d_totals, launches);
+}
+
+void launch_emit_devices(cudaStream_t s, const DeviceView &v, const EmitPlan *plans, int n, int64_t *offsets,
+                         int64_t *busy, double *util, const int64_t *d_totals, int64_t *launches)
+{
+    if (!offsets && !busy && !util) return;
+    const int64_t total = (int64_t)n * v.tc.n_devices + 1;
+    emit_devices_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(v, plans, n, offsets, busy, util, d_totals);
+    ++*launches;
 }
 
 void launch_emit_records(cudaStream_t s, const SideStream &ss, const DeviceView &v, int n, const EmitPlan *plans,
                          const int64_t *op_start, int64_t op_words_per_cand, const EmitTotals &t,
-                         distsim_record *records, int64_t *launches)
+                         distsim_record *records, int64_t *launches, const int64_t *gate, const EmitDeviceWords *words)
 {
-    if (n == 0 || t.item_tiles == 0) return;
+    if (n == 0 || t.item_tiles == 0) {
+        if (words) launch_emit_devices(s, v, plans, n, words->offsets, words->busy, words->util, words->d_totals, launches);
+        return;
+    }
     // two images of the run, then the forward and backward item templates of the widest stage
     const int cap = (int)((t.run_words + 1) & ~(int64_t)1);
     const size_t smem = (size_t)(2 * cap + 2 + t.tmpl_words) * sizeof(int64_t);
@@ -924,27 +950,25 @@ void launch_emit_records(cudaStream_t s, const SideStream &ss, const DeviceView 
     // The bucket records are few and their blocks wait more than they write: on the side stream
     // they run beside the item kernel (both only read the plans and write disjoint records).  The
     // fork event is recorded before the item kernel is enqueued, the item kernel goes first.
-    const bool beside = buckets && ss.side[0];
+    const bool beside = (buckets || words) && ss.side[0];
     if (beside) cudaEventRecord(ss.fork, s);
     emit_items_kernel<<<dim3((unsigned)t.item_tiles, (unsigned)n), kItemThreads, smem, s>>>(
-        v, plans, op_start, op_words_per_cand, out, cap);
+        v, plans, op_start, op_words_per_cand, out, cap, gate);
     ++*launches;
+    if (beside) cudaStreamWaitEvent(ss.side[0], ss.fork, 0);
+    if (words) launch_emit_devices(beside ? ss.side[0] : s, v, plans, n, words->offsets, words->busy, words->util, words->d_totals, launches);
     if (buckets) {
         // an odd number of buckets per image keeps both images 16-byte aligned
         const int run = (int)(t.bucket_recs < kBucketRun ? t.bucket_recs : kBucketRun) | 1;
         const size_t bsmem = (size_t)(2 * (run * 5 + 1) + 2 * (DISTSIM_MAX_LAYERS + 1)) * sizeof(int64_t);
         ensure_dynamic_smem(reinterpret_cast<const void *>(&emit_buckets_kernel), bsmem);
-        cudaStream_t bs = s;
-        if (beside) {
-            cudaStreamWaitEvent(ss.side[0], ss.fork, 0);
-            bs = ss.side[0];
-        }
-        emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, bs>>>(v, plans, out, run);
+        const cudaStream_t bs = beside ? ss.side[0] : s;
+        emit_buckets_kernel<<<dim3((unsigned)t.bucket_tiles, (unsigned)n), kBucketThreads, bsmem, bs>>>(v, plans, out, run, gate);
         ++*launches;
-        if (beside) {
-            cudaEventRecord(ss.join[0], ss.side[0]);
-            cudaStreamWaitEvent(s, ss.join[0], 0);
-        }
+    }
+    if (beside) {
+        cudaEventRecord(ss.join[0], ss.side[0]);
+        cudaStreamWaitEvent(s, ss.join[0], 0);
     }
 }
 

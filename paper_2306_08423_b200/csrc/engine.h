@@ -281,15 +281,26 @@ void launch_emit_plan(cudaStream_t s, const DeviceView &v, const int64_t *d_indi
                       int64_t *h_totals /* nullable: host memory the device can write; receives the totals' words
                                            and, in word 7, the device status word after planning */,
                       cudaEvent_t planned /* nullable: recorded behind the planning kernel */,
-                      int64_t *launches);
+                      int64_t *launches,
+                      const EmitTotals *limits = nullptr /* nullable: what the caller has provisioned (records:
+                                           its capacity); the last block sets word 7 of d_totals to 1 if the
+                                           plans stay within it, else to 0 and the status to DISTSIM_E_CAPACITY */);
+// Offsets, activity times and utilisations of every device of the planned selections (each nullable).
+void launch_emit_devices(cudaStream_t s, const DeviceView &v, const EmitPlan *plans, int n, int64_t *offsets,
+                         int64_t *busy, double *util, const int64_t *d_totals, int64_t *launches);
 int interleaved_words_of(int pp, int v);           // those words for one row
 int bidirectional_words_of(int pp, int kept);      // shared-memory words a bidirectional candidate needs
 int bidirectional_kept_cap_of(int pp);             // most items the kernels keep per device of such a candidate
 // out[k] = order-sensitive checksum of the records [offsets[k], offsets[k + 1]).
 void launch_checksum_lists(cudaStream_t s, const distsim_record *records, const int64_t *offsets, int64_t n_lists,
                            uint64_t *out, int64_t *launches);
+// gate (nullable): device words of an EmitTotals; the kernels write nothing unless word 7 is non-zero.
+// words (nullable): the per-device outputs, written beside the item kernel (on the side stream) rather
+// than by launch_emit_plan before it.
+struct EmitDeviceWords { int64_t *offsets, *busy; double *util; const int64_t *d_totals; };
 void launch_emit_records(cudaStream_t s, const SideStream &ss, const DeviceView &v, int n, const EmitPlan *plans,
                          const int64_t *op_start, int64_t op_words_per_cand, const EmitTotals &totals,
-                         distsim_record *records, int64_t *launches);
+                         distsim_record *records, int64_t *launches, const int64_t *gate = nullptr,
+                         const EmitDeviceWords *words = nullptr);
 
 }  // namespace distsim

@@ -24,7 +24,8 @@ EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error",
            "distsim_load_event_table", "distsim_set_space", "distsim_decode",
            "distsim_eval_strategies", "distsim_eval_select", "distsim_argmin", "distsim_topk",
            "distsim_merge_topk",
-           "distsim_emit_timelines", "distsim_checksum_timelines", "distsim_search_host",
+           "distsim_emit_timelines", "distsim_emit_shape_of_last_plan", "distsim_emit_timelines_async",
+           "distsim_checksum_timelines", "distsim_search_host",
            "distsim_topk_static")
 # hooks of include/distsim_testing.h (test-suite and benchmark accounting; not the stable ABI)
 TESTING_EXPORTS = ("distsim_testing_set_stage_wait_polls", "distsim_testing_launch_count",
@@ -98,6 +99,9 @@ _lib.distsim_merge_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void
 _lib.distsim_emit_timelines.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                         C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.POINTER(C.c_int64)]
+_lib.distsim_emit_shape_of_last_plan.argtypes = [C.c_void_p, C.c_void_p]
+_lib.distsim_emit_timelines_async.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                              C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.distsim_checksum_timelines.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
 _lib.distsim_search_host.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_Space), C.c_int32,
                                      C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
@@ -296,6 +300,35 @@ def distsim_emit_timelines(ctx: Context, d_indices, n: int, d_records, capacity_
         raise e
     ctx._check(rc)
     return int(total.value)
+
+
+class EmitShape(C.Structure):
+    """distsim_emit_shape: what an emission needs, as upper bounds an asynchronous call provisions for."""
+    _fields_ = [("records", C.c_int64), ("item_tiles", C.c_int64), ("bucket_tiles", C.c_int64),
+                ("tmpl_words", C.c_int64), ("bucket_recs", C.c_int64), ("run_words", C.c_int64)]
+
+
+def distsim_emit_shape_of_last_plan(ctx: Context) -> EmitShape:
+    """The shape of the context's most recent synchronising emission call (a sizing call, say)."""
+    shape = EmitShape()
+    ctx._check(_lib.distsim_emit_shape_of_last_plan(ctx._h, C.byref(shape)))
+    return shape
+
+
+def distsim_emit_timelines_async(ctx: Context, d_indices, n: int, d_records, capacity_records: int, shape: EmitShape,
+                                 d_offsets=None, d_busy_ns=None, d_util=None, stream=None) -> None:
+    """Emission without any wait on the host: plans and writes in stream order, provisioned by
+    ``shape``.  If the selection needs more than the shape or the capacity allow, nothing is written
+    to ``d_records`` and the next synchronising call on the context raises E_CAPACITY;
+    ``d_offsets[n * N]`` is the number of records needed either way."""
+    pi = _dev_ptr(d_indices, "int64", n, "d_indices")
+    pr = _dev_ptr(d_records, "int64", 5 * capacity_records, "d_records")
+    nn = n * ctx.n_devices
+    po = _dev_ptr(d_offsets, "int64", nn + 1, "d_offsets")
+    pbz = _dev_ptr(d_busy_ns, "int64", nn, "d_busy_ns")
+    pu = _dev_ptr(d_util, "float64", nn, "d_util")
+    ctx._check(_lib.distsim_emit_timelines_async(ctx._h, _stream(stream), pi, n, pr, capacity_records, C.byref(shape),
+                                                 po, pbz, pu))
 
 
 def distsim_checksum_timelines(ctx: Context, d_records, d_offsets, n_lists: int, d_checksums, stream=None) -> None:

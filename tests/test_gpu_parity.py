@@ -84,6 +84,14 @@ def check_emission(E, ctx, w, indices):
     rec = records.cpu().numpy()[: total * 5].reshape(total, 5)
     off = offsets.cpu().numpy(); bz = busy.cpu().numpy(); ut = util.cpu().numpy()
     assert off[0] == 0 and off[-1] == total
+    # the call that never waits on the host, provisioned by the shape of the pass above: the same output
+    shape = E.distsim_emit_shape_of_last_plan(ctx)
+    assert shape.records == total
+    records2, offsets2, busy2, util2 = dev(max(1, total) * 5), dev(n * N + 1), dev(n * N), dev(n * N, torch.float64)
+    records2.fill_(-7)
+    E.distsim_emit_timelines_async(ctx, idx, n, records2, total, shape, offsets2, busy2, util2)
+    torch.cuda.synchronize()
+    assert torch.equal(records2, records) and torch.equal(offsets2, offsets) and torch.equal(busy2, busy) and torch.equal(util2, util)
     sums = device_checksums(E, ctx, records, offsets, n * N)
     order = np.argsort(np.asarray(indices), kind="stable")
     cands = oracle.enumerate_at(w.table, w.space, np.asarray(indices)[order])
@@ -860,6 +868,63 @@ def test_eval_select_matches_separate_calls(E, ctx):
     n = load(E, ctx, w)
     assert n > 4096
     _check_eval_select(E, ctx, 0, n, 500)
+
+
+def test_asynchronous_emission_provisioning(E, ctx):
+    """distsim_emit_timelines_async with shapes larger than needed (same records), with a shape or a
+    capacity that is too small (nothing written, DISTSIM_E_CAPACITY from the next synchronising call,
+    the count of records needed in the last offset), and the context usable afterwards."""
+    w = W.config3()
+    n = load(E, ctx, w)
+    N = w.table.n_devices
+    batch, _ = eval_all(E, ctx, n, busy=False)
+    k = 48
+    top = dev(k)
+    E.distsim_topk(ctx, batch, 0, n, k, top)
+    offsets, busy, util = dev(k * N + 1), dev(k * N), dev(k * N, torch.float64)
+    total = E.distsim_emit_timelines(ctx, top, k, None, 0, offsets, busy, util)
+    want = dev(total * 5)
+    E.distsim_emit_timelines(ctx, top, k, want, total, offsets, busy, util)
+    shape = E.distsim_emit_shape_of_last_plan(ctx)
+    # a selection of another kind through a shape sized on this one, with headroom
+    roomy = E.EmitShape(2 * shape.records, 2 * shape.item_tiles + 3, 2 * shape.bucket_tiles + 1, shape.tmpl_words + 40,
+                        shape.bucket_recs + 7, shape.run_words)
+    got, off2 = dev(total * 5 + 50), dev(k * N + 1)
+    got.fill_(-7)
+    E.distsim_emit_timelines_async(ctx, top, k, got, total + 10, roomy, off2, None, None)
+    torch.cuda.synchronize()
+    assert torch.equal(got[: total * 5], want) and bool((got[total * 5:] == -7).all()) and torch.equal(off2, offsets)
+    other = torch.arange(0, n, n // 8, dtype=torch.int64, device="cuda")[:8].contiguous()
+    t8 = E.distsim_emit_timelines(ctx, other, 8, None, 0)
+    want8 = dev(t8 * 5)
+    E.distsim_emit_timelines(ctx, other, 8, want8, t8)
+    s8 = E.distsim_emit_shape_of_last_plan(ctx)
+    big = E.EmitShape(*[max(getattr(roomy, f), getattr(s8, f)) for f, _ in E.EmitShape._fields_])
+    got8 = dev(t8 * 5)
+    E.distsim_emit_timelines_async(ctx, other, 8, got8, t8, big)
+    torch.cuda.synchronize()
+    assert torch.equal(got8, want8)
+    # too little: each in turn
+    for what in ("capacity", "item_tiles", "run_words", "tmpl_words", "bucket_recs", "bucket_tiles"):
+        small = E.EmitShape(*[getattr(shape, f) for f, _ in E.EmitShape._fields_])
+        cap = total
+        if what == "capacity":
+            cap = total - 1
+        elif getattr(shape, what) == 0:
+            continue
+        else:
+            setattr(small, what, getattr(shape, what) - 1)
+        got.fill_(-7); off2.fill_(-1)
+        E.distsim_emit_timelines_async(ctx, top, k, got, cap, small, off2, None, None)
+        torch.cuda.synchronize()
+        assert bool((got == -7).all()), what
+        assert int(off2[-1]) == total and torch.equal(off2, offsets), what
+        with pytest.raises(E.DistsimError) as err:
+            E.distsim_argmin(ctx, batch, 0, n)
+        assert err.value.code == E.E_CAPACITY, what
+        assert E.distsim_argmin(ctx, batch, 0, n)[1] == int(batch.min().item())       # the status is cleared
+    with pytest.raises(E.DistsimError):
+        E.distsim_emit_timelines_async(ctx, top, k, got, total, E.EmitShape(total, 1 << 40, 1, 1, 1, 1))
 
 
 def test_merged_rank_lists_equal_the_global_topk(E, ctx):
