@@ -643,6 +643,27 @@ def test_long_pipelines_every_composition(E, ctx, pp, n_layers):
     check_emission(E, ctx, w, [int(idx[1]), int(idx[-2])])
 
 
+def test_long_pipelines_with_chunks_and_two_ways(E, ctx):
+    # the longest pipelines the warp-per-candidate kernel takes: up to 32 devices running
+    # interleaved 1F1B with two chunks each (64 virtual stages) and bidirectional pipelines (one
+    # candidate per warp, the largest shared-memory arrays), few and many micro-batches, balanced
+    # partitions of an odd number of layers: every candidate
+    space = W.SearchSpace(mp_max=1, pp_max=32, m_list=[2, 32, 64, 70, 96], m_rule=W.M_RULE_CEIL,
+                          partition_mode=W.PARTITION_BALANCED, sched_mask=24, v_max=2)
+    table = _flat_table(67, 32, 8, 141, space, 50_000, 32)        # odd global batch: dp = 1 only
+    w = W.Workload("long_32_chunks_two_ways", table, space, 32)
+    n = load(E, ctx, w)
+    cands = oracle.enumerate_at(table, space, np.arange(n))
+    kinds = {(c.pp, c.sched, c.m) for c in cands}
+    assert (32, 3, 96) in kinds and (32, 4, 70) in kinds and (32, 4, 2) in kinds, kinds
+    batch, sb = eval_all(E, ctx, n)
+    ob, obusy = oracle.eval_indices_parallel(table, space, np.arange(n), THREADS, pp_stride=space.pp_max)
+    assert (batch.cpu().numpy() == ob).all()
+    assert (sb.cpu().numpy() == obusy).all()
+    pick = [i for i, c in enumerate(cands) if (c.pp, c.sched, c.m) in ((32, 3, 96), (32, 4, 70), (32, 4, 2))]
+    check_emission(E, ctx, w, pick)
+
+
 @pytest.mark.parametrize("cfg,stride", [(1, 39_119), (2, 1), (3, 653)])
 def test_index_decoding_matches_loop_enumeration(E, ctx, cfg, stride):
     # the library's index -> candidate mapping against the oracle's nested loops
