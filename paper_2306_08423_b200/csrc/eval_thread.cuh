@@ -696,7 +696,8 @@ eval_thread_kernel(DeviceView v, EvalBatch batch, int64_t first,
                 res_sc = main_only;
             } else {
                 T free_at[PP];
-                if (id == 0) {
+                // (with one micro-batch every stage runs its forward, then its backward item: the GPipe order)
+                if (id == 0 || (m == 1 && !kJit)) {
                     if (kJit || !rel) run_gpipe<PP, T, kJit>(st, m, free_at, jt);
                     else run_gpipe_rel<PP, T>(st, m, free_at);
                 } else {
