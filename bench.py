@@ -402,6 +402,16 @@ def run_ours(args):
     e2e_times = [(time.perf_counter() - t0) / n_ovl]
     overlap_ok = bool(torch.equal(h_rec2[(n_ovl - 1) & 1][: tot * 5], records2[(n_ovl - 1) & 1][: tot * 5].cpu())
                       and torch.equal(h_small[(n_ovl - 1) & 1][0], top_i.cpu()))
+    # what the link gives: the same records copied device -> pinned host, nothing else running
+    pe0, pe1 = ev(), ev()
+    h_rec[: tot * 5].copy_(records[: tot * 5], non_blocking=True)
+    torch.cuda.synchronize()
+    pe0.record(stream)
+    for _ in range(3):
+        h_rec[: tot * 5].copy_(records[: tot * 5], non_blocking=True)
+    pe1.record(stream)
+    torch.cuda.synchronize()
+    d2h_gbs = 3 * tot * RECORD_BYTES / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
     barrier()
     clocks = sampler.stop() if sampler else None
 
@@ -514,6 +524,8 @@ def run_ours(args):
                         "step; a step's download runs on a copy stream beside the next step's work (two record "
                         "buffers), the time is that of the whole loop / its steps",
                 "steps": n_ovl, "downloads_match_device": overlap_ok,
+                "d2h_copy_GB_per_sec_measured": d2h_gbs,
+                "frac_of_d2h_copy_rate": (d2h / e2e_s_max / 1e9) / d2h_gbs,
                 "one_step_at_a_time": {"value": job_candidates / serial_s_max,
                                        "unit": "candidates/s", "ms_per_step": serial_s_max * 1e3},
                 "records_left_on_device": {"value": job_candidates / results_only_s, "unit": "candidates/s",
@@ -653,6 +665,51 @@ def other_workloads(E, ctx, torch, dev, peaks, cell32_peak, cell64_peak):
                    "frac_of_measured_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
                    "frac_of_nominal_8TBs": nbytes / t / 1e9 / 8000.0,
                    "chunk_candidates": chunk, "buffer_GB": cap * RECORD_BYTES / 1e9}
+    # The same emission brought to the host: 32 candidates per call into one of two device buffers,
+    # each downloaded to pinned memory on a copy stream while the next call writes the other.
+    del records
+    torch.cuda.empty_cache()
+    small = 32
+    sizes = [E.distsim_emit_timelines(ctx, top[i:i + small], min(small, w.top_k - i), None, 0)
+             for i in range(0, w.top_k, small)]
+    cap2 = max(sizes) + 1024
+    d_rec = [torch.empty(cap2 * 5, dtype=torch.int64, device=dev) for _ in range(2)]
+    h_rec = [torch.empty(cap2 * 5, dtype=torch.int64).pin_memory() for _ in range(2)]
+    copy_stream = torch.cuda.Stream(device=dev)
+    emitted = [torch.cuda.Event(), torch.cuda.Event()]
+    downloaded = [torch.cuda.Event(), torch.cuda.Event()]
+    # the link alone: one buffer copied device -> pinned host
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h_rec[0].copy_(d_rec[0], non_blocking=True)
+    torch.cuda.synchronize()
+    c0.record(stream)
+    h_rec[0].copy_(d_rec[0], non_blocking=True)
+    c1.record(stream)
+    torch.cuda.synchronize()
+    link_gbs = cap2 * RECORD_BYTES / (c0.elapsed_time(c1) * 1e-3) / 1e9
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    moved = 0
+    for k, i in enumerate(range(0, w.top_k, small)):
+        b, c = k & 1, min(small, w.top_k - i)
+        if k >= 2:
+            stream.wait_event(downloaded[b])
+        got = E.distsim_emit_timelines(ctx, top[i:i + c], c, d_rec[b], cap2, offsets[: c * N + 1], busy[: c * N], util[: c * N])
+        emitted[b].record(stream)
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(emitted[b])
+            h_rec[b][: got * 5].copy_(d_rec[b][: got * 5], non_blocking=True)
+            downloaded[b].record(copy_stream)
+        moved += got * RECORD_BYTES
+    torch.cuda.synchronize()
+    t2 = time.perf_counter() - t0
+    last = (w.top_k - 1) // small
+    ok = bool(torch.equal(h_rec[last & 1][: got * 5], d_rec[last & 1][: got * 5].cpu()))
+    out[w.name]["to_host"] = {"seconds": t2, "GB_per_sec": moved / t2 / 1e9, "d2h_copy_GB_per_sec_measured": link_gbs,
+                              "frac_of_d2h_copy_rate": moved / t2 / 1e9 / link_gbs, "chunk_candidates": small,
+                              "last_download_matches_device": ok,
+                              "how": "two device buffers and two pinned host buffers; a chunk's download runs on a copy "
+                                     "stream beside the emission of the next chunk"}
     return out
 
 
