@@ -289,10 +289,11 @@ int distsim_emit_timelines(distsim_ctx *ctx, void *stream, const int64_t *d_indi
  * The same without any wait on the host, for a loop that emits timelines step after step (the
  * paper's search loop, Sec. 6, keeps the host out of the way of the device).  What the
  * synchronising call learns from its planning pass - how much output and how much of the
- * kernels' resources the selection needs - the caller passes in instead: distsim_emit_shape()
- * returns those figures for the context's most recent planning pass (a sizing call, say, on a
- * selection of the kind the loop will see), and the caller may enlarge any of them for headroom.
- *   shape      host: upper bounds this call provisions for (see distsim_emit_shape)
+ * kernels' resources the selection needs - the caller passes in instead:
+ * distsim_emit_shape_of_last_plan() returns those figures for the context's most recent
+ * synchronising planning pass (a sizing call, say, on a selection of the kind the loop will see),
+ * and the caller may enlarge any of them for headroom.
+ *   h_shape    host: upper bounds this call provisions for (the fields of distsim_emit_shape)
  * The call plans the n selections, then writes their records, all in stream order.  If the
  * selection needs more than `shape` or capacity_records allow, no record is written, the device
  * status becomes DISTSIM_E_CAPACITY and the next synchronising call on the context returns it;
