@@ -35,6 +35,15 @@ int64_t distsim_testing_lockstep_pieces(int32_t pp, int64_t lo, int64_t hi, int6
                                         int64_t *h_lo, int64_t *h_hi, int32_t *h_blocks);
 
 /*
+ * Host logic of the bidirectional schedule (no device involved): the merged item order the library
+ * builds for pp devices and m micro-batches (both even, 2 <= pp <= 32, 2 <= m <= DISTSIM_MAX_M).
+ * h_order[d * 2 m + k] = pipeline << 15 | is-backward << 14 | micro-batch within its pipeline for
+ * the k-th item of device d; *h_kept = the items a device may run from the last backward item of
+ * its later stage on.  Returns DISTSIM_OK or DISTSIM_E_ARG.
+ */
+int distsim_testing_bidirectional_order(int32_t pp, int32_t m, uint16_t *h_order, int32_t *h_kept);
+
+/*
  * Phase timing of distsim_eval_select for the benchmark: with enable != 0 the call records CUDA
  * events on its stream before the evaluation launches, after them and after the selection
  * launches; distsim_testing_last_phase_ms returns the two durations of the most recent such

@@ -941,6 +941,19 @@ int64_t distsim_testing_lockstep_pieces(int32_t pp, int64_t lo, int64_t hi, int6
     return lockstep_pieces(pp, lo, hi, max_blocks, max_pieces, h_lo, h_hi, h_blocks);
 }
 
+int distsim_testing_bidirectional_order(int32_t pp, int32_t m, uint16_t *h_order, int32_t *h_kept)
+{
+    if (pp < 2 || pp > 32 || (pp & 1) || m < 2 || m > DISTSIM_MAX_M || (m & 1) || !h_order || !h_kept) return DISTSIM_E_ARG;
+    std::vector<uint16_t> order;
+    std::vector<uint32_t> before;
+    int kept = 0;
+    if (!bidirectional_orders(pp, m, order, before, &kept)) return DISTSIM_E_ARG;
+    for (int d = 0; d < pp; ++d)
+        for (int k = 0; k < 2 * m; ++k) h_order[(size_t)d * 2 * m + k] = order[(size_t)d * (2 * m + 1) + k];
+    *h_kept = kept;
+    return DISTSIM_OK;
+}
+
 int distsim_testing_time_phases(distsim_ctx *ctx, int32_t enable)
 {
     if (!ctx) return DISTSIM_E_ARG;

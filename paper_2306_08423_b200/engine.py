@@ -30,6 +30,7 @@ EXPORTS = ("distsim_create", "distsim_destroy", "distsim_last_error",
 # hooks of include/distsim_testing.h (test-suite and benchmark accounting; not the stable ABI)
 TESTING_EXPORTS = ("distsim_testing_set_stage_wait_polls", "distsim_testing_launch_count",
                    "distsim_testing_space_cells", "distsim_testing_lockstep_pieces",
+                   "distsim_testing_bidirectional_order",
                    "distsim_testing_time_phases", "distsim_testing_last_phase_ms")
 TOPK_STATIC_MAX_K = 1024
 
@@ -82,6 +83,7 @@ _lib.distsim_testing_set_stage_wait_polls.argtypes = [C.c_void_p, C.c_int32]
 _lib.distsim_testing_lockstep_pieces.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
                                                  C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.distsim_testing_lockstep_pieces.restype = C.c_int64
+_lib.distsim_testing_bidirectional_order.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.POINTER(C.c_int32)]
 _lib.distsim_testing_time_phases.argtypes = [C.c_void_p, C.c_int32]
 _lib.distsim_testing_last_phase_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_float)]
 _lib.distsim_load_event_table.argtypes = [C.c_void_p, C.POINTER(_Table)]
@@ -378,6 +380,26 @@ def distsim_topk_static(d_batch_ns, first: int, count: int, k: int, d_indices, d
         raise DistsimError(rc, f"k = {k} exceeds the fixed scratch (at most {TOPK_STATIC_MAX_K})")
     if rc != OK:
         raise DistsimError(rc, "distsim_topk_static failed")
+
+
+def distsim_testing_bidirectional_order(pp: int, m: int):
+    """(order, kept): the library's merged item order of the bidirectional schedule for (pp, m) as a
+    list per device of ('F'|'B', micro-batch, pipeline), and its kept-item count.  Host logic only."""
+    buf = (C.c_uint16 * (pp * 2 * m))()
+    kept = C.c_int32(0)
+    rc = _lib.distsim_testing_bidirectional_order(pp, m, buf, C.byref(kept))
+    if rc != OK:
+        raise DistsimError(rc, "distsim_testing_bidirectional_order failed")
+    half = m // 2
+    order = []
+    for d in range(pp):
+        items = []
+        for k in range(2 * m):
+            w = buf[d * 2 * m + k]
+            u = w >> 15
+            items.append(("B" if w & (1 << 14) else "F", (w & 0x3FFF) + u * half, u))
+        order.append(items)
+    return order, int(kept.value)
 
 
 def distsim_testing_space_cells(ctx: Context):

@@ -71,3 +71,28 @@ def test_long_pipeline_ranges_are_cut_into_launchable_pieces():
                 assert pos == (hi if hi > lo else lo)
     with __import__("pytest").raises(engine.DistsimError):
         engine.distsim_testing_lockstep_pieces(3, 0, 10, 16)
+
+
+def test_bidirectional_item_order_built_on_the_host():
+    # the merged order the library builds for the bidirectional schedule (host code, no device)
+    # against the token game restated in Python for the oracle's pins, and the schedule's slot count
+    from paper_2306_08423_b200 import engine as E
+    from tests.dag_bruteforce import bidirectional_order
+    for pp in (2, 4, 6, 8, 16, 32):
+        for m in (2, 4, 6, 8, 16, 34, 64, 128):
+            got, kept = E.distsim_testing_bidirectional_order(pp, m)
+            want, slots = bidirectional_order(pp, m)
+            assert got == [want[d] for d in range(pp)], (pp, m)
+            if m % pp == 0:
+                assert slots == 2 * m + pp - 2
+            # the kept tail: from the last backward item of the device's later stage on
+            longest = 2
+            for d in range(pp):
+                u_first = 0 if d > pp - 1 - d else 1
+                last = m // 2 - 1 + u_first * (m // 2)
+                longest = max(longest, 2 * m - want[d].index(("B", last, u_first)))
+            assert kept == longest <= pp // 2 + 2, (pp, m, kept, longest)
+    import pytest
+    for bad in ((3, 4), (4, 3), (34, 4), (0, 2)):
+        with pytest.raises(E.DistsimError):
+            E.distsim_testing_bidirectional_order(*bad)
